@@ -1,0 +1,184 @@
+"""ctypes front-end of the CPU oracle (oracle/kb_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The product package never imports this module.
+Arguments and results are numpy arrays; the arithmetic lives in the C++ file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kb_oracle.cpp")
+_LIB = os.path.join(_HERE, "libkb_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (plain -O2, one translation unit)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _check(rc: int, name: str):
+    if rc != 0:
+        raise ValueError(f"oracle {name} rejected its arguments (code {rc})")
+
+
+def normalize(x):
+    x = _f32(x)
+    B, N, D = x.shape
+    z = np.empty_like(x)
+    mean = np.empty((B, D), np.float32)
+    scale = np.empty((B, D), np.float32)
+    _check(_load().kbo_normalize(B, N, D, _p(x), _p(z), _p(mean), _p(scale)), "normalize")
+    return z, mean, scale
+
+
+def prune(flops, bytes_, peak_flops, peak_bw, t_inc, t_cur=None, labels=None, hsig=None, target=None,
+          theta_sat=75.0, K=0, want_bound=False, want_margin=False):
+    flops, bytes_ = _f32(flops), _f32(bytes_)
+    B, N = flops.shape
+    peak_flops, peak_bw, t_inc = _f32(peak_flops), _f32(peak_bw), _f32(t_inc)
+    S = peak_flops.shape[0]
+    R = 0
+    if labels is not None:
+        labels, hsig, target = _i32(labels), _f32(hsig), _i32(target)
+        K, R = hsig.shape[1], hsig.shape[2]
+    if t_cur is not None:
+        t_cur = _f32(t_cur)
+    keep = np.empty((B, N), np.uint32)
+    kept = np.empty((B,), np.uint32)
+    bound = np.empty((B, N, S), np.float32) if want_bound else None
+    margin = np.empty((B, N, S), np.float64) if want_margin else None
+    _check(_load().kbo_prune(B, N, S, K, R, _p(flops), _p(bytes_), _p(peak_flops), _p(peak_bw), _p(t_inc),
+                             _p(t_cur), _p(labels), _p(hsig), _p(target), ctypes.c_float(theta_sat),
+                             _p(keep), _p(kept), _p(bound), _p(margin)), "prune")
+    return {"keep": keep, "kept_count": kept, "bound": bound, "margin": margin}
+
+
+def cluster_assign(z, centroids, want_rep=True, want_margins=False):
+    z, centroids = _f32(z), _f32(centroids)
+    B, N, D = z.shape
+    K = centroids.shape[1]
+    labels = np.empty((B, N), np.int32)
+    dist2 = np.empty((B, N), np.float32)
+    inertia = np.empty((B,), np.float32)
+    rep = np.empty((B, K), np.int32) if want_rep else None
+    best = np.empty((B, N), np.float64) if want_margins else None
+    second = np.empty((B, N), np.float64) if want_margins else None
+    _check(_load().kbo_cluster_assign(B, N, D, K, _p(z), _p(centroids), _p(labels), _p(dist2), _p(inertia),
+                                      _p(rep), _p(best), _p(second)), "cluster_assign")
+    return {"labels": labels, "dist2": dist2, "inertia": inertia, "rep": rep, "best": best, "second": second}
+
+
+def dist2_at(z, centroids, labels):
+    z, centroids, labels = _f32(z), _f32(centroids), _i32(labels)
+    B, N, D = z.shape
+    K = centroids.shape[1]
+    out = np.empty((B, N), np.float64)
+    _check(_load().kbo_dist2_at(B, N, D, K, _p(z), _p(centroids), _p(labels), _p(out)), "dist2_at")
+    return out
+
+
+def cluster_update(z, labels, centroids):
+    """Returns (new centroids, counts); `centroids` (previous) is not modified."""
+    z, labels = _f32(z), _i32(labels)
+    c = np.array(centroids, dtype=np.float32, order="C", copy=True)
+    B, N, D = z.shape
+    K = c.shape[1]
+    counts = np.empty((B, K), np.int32)
+    _check(_load().kbo_cluster_update(B, N, D, K, _p(z), _p(labels), _p(c), _p(counts)), "cluster_update")
+    return c, counts
+
+
+def score_select(labels, dist2, pulls, reward_sum, t, K, keep=None, bound=None, c=2.0, lipschitz_L=0.0,
+                 prior_pulls=1.0, prior_mean=0.5, cap_with_bound=False, want_arm_index=True):
+    labels, pulls, reward_sum, t = _i32(labels), _i32(pulls), _f32(reward_sum), _i32(t)
+    B, N, S = pulls.shape
+    if dist2 is not None:
+        dist2 = _f32(dist2)
+    if keep is not None:
+        keep = np.ascontiguousarray(keep, dtype=np.uint32)
+    if bound is not None:
+        bound = _f32(bound)
+    cl_pulls = np.empty((B, K, S), np.float32)
+    cl_mean = np.empty((B, K, S), np.float32)
+    cl_index = np.empty((B, K, S), np.float32)
+    arm_index = np.empty((B, N, S), np.float32) if want_arm_index else None
+    best_arm = np.empty((B,), np.int32)
+    best_val = np.empty((B,), np.float32)
+    best_cl = np.empty((B,), np.int32)
+    margin = np.empty((B, 2), np.float64)
+    _check(_load().kbo_score_select(B, N, K, S, ctypes.c_float(c), ctypes.c_float(lipschitz_L),
+                                    ctypes.c_float(prior_pulls), ctypes.c_float(prior_mean),
+                                    int(bool(cap_with_bound)), _p(labels), _p(dist2), _p(pulls), _p(reward_sum),
+                                    _p(keep), _p(bound), _p(t), _p(cl_pulls), _p(cl_mean), _p(cl_index),
+                                    _p(arm_index), _p(best_arm), _p(best_val), _p(best_cl), _p(margin)),
+           "score_select")
+    return {"cl_pulls": cl_pulls, "cl_mean": cl_mean, "cl_index": cl_index, "arm_index": arm_index,
+            "best_arm": best_arm, "best_val": best_val, "best_cluster_arm": best_cl, "margin": margin}
+
+
+def init_centroids(z, rows):
+    z, rows = _f32(z), _i32(rows)
+    B, N, D = z.shape
+    K = rows.shape[1]
+    c = np.empty((B, K, D), np.float32)
+    _check(_load().kbo_init_centroids(B, N, D, K, _p(z), _p(rows), _p(c)), "init_centroids")
+    return c
+
+
+def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
+    """One whole bandit step in the order the library runs it: normalise, seed
+    the centroids from data rows, `iters` x (assign, update), a final assign,
+    prune (both masks), cluster statistics + index + selection."""
+    z, mean, scale = normalize(inp["x"])
+    c = init_centroids(z, inp["init_rows"])
+    K = c.shape[1]
+    inertia_trace = []
+    counts = None
+    for _ in range(iters):
+        a = cluster_assign(z, c, want_rep=False)
+        inertia_trace.append(a["inertia"].copy())
+        c, counts = cluster_update(z, a["labels"], c)
+    a = cluster_assign(z, c, want_rep=True)
+    inertia_trace.append(a["inertia"].copy())
+    p = prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+              a["labels"], inp["hsig"], inp["target"], float(inp["theta_sat"]), want_bound=True)
+    s = score_select(a["labels"], a["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], K, keep=p["keep"],
+                     bound=p["bound"], c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
+                     prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]),
+                     cap_with_bound=False, want_arm_index=want_arm_index)
+    out = {"z": z, "mean": mean, "scale": scale, "centroids": c, "counts": counts, "labels": a["labels"],
+           "dist2": a["dist2"], "inertia": a["inertia"], "rep": a["rep"], "inertia_trace": np.array(inertia_trace),
+           "keep": p["keep"], "kept_count": p["kept_count"], "bound": p["bound"]}
+    out.update({k: v for k, v in s.items() if k != "margin"})
+    return out

@@ -1,0 +1,313 @@
+// CPU oracle for the batched bandit step (KernelBand decision layer).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, single-threaded
+// definition of what the CUDA library must compute.  It is called from the
+// tests, from the smoke check and from the benchmark's CPU-baseline leg, and
+// from nowhere else; the product path never routes through it.  It shares no
+// code, header, table or helper with the CUDA sources.
+//
+// Arithmetic: inputs and stored outputs are fp32 (the library's types); every
+// sum, distance, mean, ratio and index is evaluated in double and rounded to
+// fp32 only when it is stored in an fp32 output.  Every decision (argmin,
+// argmax, threshold test) is taken on the double values.  Ties go to the
+// lowest index.  One thread, no blocking, no fusion, no reordering.
+//
+// Parity pins: every function below is pinned by the CPU test-suite against
+// closed forms, worked values, invariants, brute force and a library K-Means
+// with a fixed initialisation.
+//
+// Arrays are dense, row-major, batch-major: X[B][N][D], C[B][K][D],
+// labels[B][N], pulls[B][N][S], hsig[B][K][R].
+
+#include <cmath>
+#include <cstddef>
+#include <cstdint>
+#include <limits>
+#include <vector>
+
+namespace {
+inline size_t ix2(size_t a, size_t b, size_t nb) { return a * nb + b; }
+inline size_t ix3(size_t a, size_t b, size_t c, size_t nb, size_t nc) { return (a * nb + b) * nc + c; }
+const double kInf = std::numeric_limits<double>::infinity();
+}  // namespace
+
+extern "C" {
+
+// ---------------------------------------------------------------------------
+// Feature normalisation: per instance and column, population z-score.
+// The paper only says the features are "normalized"/"log-transformed"
+// (Sec. 3.2, App. A.1); the workloads fix the reading: z = (x - mean) / std
+// with the population std (divide by N); a column whose std is below 1e-12
+// gets scale 1 (so it becomes all zeros).
+// ---------------------------------------------------------------------------
+int kbo_normalize(int B, int N, int D, const float* x, float* z, float* mean, float* scale) {
+    for (int b = 0; b < B; ++b) {
+        for (int d = 0; d < D; ++d) {
+            double sum = 0.0;
+            for (int k = 0; k < N; ++k) sum += (double)x[ix3(b, k, d, N, D)];
+            double m = N > 0 ? sum / (double)N : 0.0;
+            double ss = 0.0;
+            for (int k = 0; k < N; ++k) {
+                double e = (double)x[ix3(b, k, d, N, D)] - m;
+                ss += e * e;
+            }
+            double sd = N > 0 ? std::sqrt(ss / (double)N) : 0.0;
+            double sc = sd < 1e-12 ? 1.0 : sd;
+            for (int k = 0; k < N; ++k)
+                z[ix3(b, k, d, N, D)] = (float)(((double)x[ix3(b, k, d, N, D)] - m) / sc);
+            if (mean) mean[ix2(b, d, D)] = (float)m;
+            if (scale) scale[ix2(b, d, D)] = (float)sc;
+        }
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Hardware-aware pruning.
+//  roofline floor   T_lb(k,s) = max(F_k / P_s, Q_k / W_s)      (the roofline
+//      model Assumption 1 cites for its bounding function)
+//  roofline keep    T_lb(k,s) < T_inc     (an arm whose floor cannot beat the
+//      incumbent, the best runtime found so far in Algorithm 1's return line)
+//  saturation keep  h_c[label(k)][Target(s)] < theta_sat   (mask equation of
+//      Sec. 3.4, strict <; applied only when labels/hsig/target are given)
+//  bound            B(k,s) = clip((T_k - T_lb) / T_k, 0, 1)   (Assumption 1:
+//      the gap between current performance and the limit, in reward units of
+//      the reward definition in Sec. 2.2)
+// keep[b][k] bit s = roofline keep AND saturation keep.
+// margin (optional, [B][N][S]): smallest relative distance of a deciding
+// comparison from its threshold, for near-tie accounting in the tests.
+// ---------------------------------------------------------------------------
+int kbo_prune(int B, int N, int S, int K, int R, const float* flops, const float* bytes,
+              const float* peak_flops, const float* peak_bw, const float* t_incumbent,
+              const float* t_cur, const int32_t* labels, const float* hsig, const int32_t* target,
+              float theta_sat, uint32_t* keep, uint32_t* kept_count, float* bound, double* margin) {
+    if (S > 32) return 1;
+    const bool sat = labels && hsig && target;
+    for (int b = 0; b < B; ++b) {
+        uint64_t kept = 0;
+        const double tinc = (double)t_incumbent[b];
+        for (int k = 0; k < N; ++k) {
+            uint32_t bits = 0;
+            for (int s = 0; s < S; ++s) {
+                double tf = (double)flops[ix2(b, k, N)] / (double)peak_flops[s];
+                double tq = (double)bytes[ix2(b, k, N)] / (double)peak_bw[s];
+                double tlb = tf > tq ? tf : tq;
+                bool ok = tlb < tinc;
+                double mg = std::fabs(tlb - tinc) / std::fabs(tinc);
+                if (sat) {
+                    int lab = labels[ix2(b, k, N)];
+                    if (lab < 0 || lab >= K) return 2;
+                    int r = target[s];
+                    if (r < 0 || r >= R) return 3;
+                    double h = (double)hsig[ix3(b, lab, r, K, R)];
+                    ok = ok && (h < (double)theta_sat);
+                    double mh = std::fabs(h - (double)theta_sat) / std::fabs((double)theta_sat);
+                    if (mh < mg) mg = mh;
+                }
+                if (ok) { bits |= (1u << s); ++kept; }
+                if (margin) margin[ix3(b, k, s, N, S)] = mg;
+                if (bound) {
+                    double tk = (double)t_cur[ix2(b, k, N)];
+                    double g = (tk - tlb) / tk;
+                    if (!(g > 0.0)) g = 0.0;
+                    if (g > 1.0) g = 1.0;
+                    bound[ix3(b, k, s, N, S)] = (float)g;
+                }
+            }
+            keep[ix2(b, k, N)] = bits;
+        }
+        if (kept_count) kept_count[b] = (uint32_t)kept;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// K-Means assignment (Sec. 3.3; Algorithm 1 "KMeans" line): nearest centroid
+// in squared Euclidean distance (the L2 norm of Assumption 2), direct form
+// sum_d (z_d - c_d)^2.  label = lowest j attaining the minimum.
+// inertia[b] = sum_k dist2.  rep[b][i] = the member of cluster i nearest its
+// centroid (the "centroid kernel" that Sec. 3.3 profiles), lowest k on ties,
+// -1 for an empty cluster.
+// best/second (optional, double [B][N]): smallest and second smallest d^2.
+// ---------------------------------------------------------------------------
+int kbo_cluster_assign(int B, int N, int D, int K, const float* z, const float* centroids,
+                       int32_t* labels, float* dist2, float* inertia, int32_t* rep,
+                       double* best_out, double* second_out) {
+    std::vector<double> repd((size_t)(K > 0 ? K : 1));
+    for (int b = 0; b < B; ++b) {
+        double total = 0.0;
+        if (rep) for (int i = 0; i < K; ++i) { rep[ix2(b, i, K)] = -1; repd[i] = kInf; }
+        for (int k = 0; k < N; ++k) {
+            double best = kInf, second = kInf;
+            int arg = -1;
+            for (int j = 0; j < K; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    double e = (double)z[ix3(b, k, d, N, D)] - (double)centroids[ix3(b, j, d, K, D)];
+                    acc += e * e;
+                }
+                if (acc < best) { second = best; best = acc; arg = j; }
+                else if (acc < second) { second = acc; }
+            }
+            labels[ix2(b, k, N)] = arg;
+            if (dist2) dist2[ix2(b, k, N)] = (float)best;
+            if (best_out) best_out[ix2(b, k, N)] = best;
+            if (second_out) second_out[ix2(b, k, N)] = second;
+            total += best;
+            if (rep && arg >= 0 && best < repd[arg]) { repd[arg] = best; rep[ix2(b, arg, K)] = k; }
+        }
+        if (inertia) inertia[b] = (float)total;
+    }
+    return 0;
+}
+
+// d^2 of every row to the centroid named by `labels` (double), so a test can
+// judge a disagreeing label by how far from optimal it is.
+int kbo_dist2_at(int B, int N, int D, int K, const float* z, const float* centroids,
+                 const int32_t* labels, double* out) {
+    for (int b = 0; b < B; ++b)
+        for (int k = 0; k < N; ++k) {
+            int j = labels[ix2(b, k, N)];
+            if (j < 0 || j >= K) { out[ix2(b, k, N)] = kInf; continue; }
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) {
+                double e = (double)z[ix3(b, k, d, N, D)] - (double)centroids[ix3(b, j, d, K, D)];
+                acc += e * e;
+            }
+            out[ix2(b, k, N)] = acc;
+        }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// K-Means centroid update (Sec. 3.3; Algorithm 1 "Update centroids"): each
+// centroid becomes the arithmetic mean of its members; an empty cluster keeps
+// its previous centroid and reports count 0.
+// ---------------------------------------------------------------------------
+int kbo_cluster_update(int B, int N, int D, int K, const float* z, const int32_t* labels,
+                       float* centroids, int32_t* counts) {
+    std::vector<double> sum((size_t)K * (size_t)D);
+    std::vector<int64_t> cnt((size_t)(K > 0 ? K : 1));
+    for (int b = 0; b < B; ++b) {
+        for (size_t i = 0; i < sum.size(); ++i) sum[i] = 0.0;
+        for (int i = 0; i < K; ++i) cnt[i] = 0;
+        for (int k = 0; k < N; ++k) {
+            int j = labels[ix2(b, k, N)];
+            if (j < 0 || j >= K) return 2;
+            ++cnt[j];
+            for (int d = 0; d < D; ++d) sum[ix2(j, d, D)] += (double)z[ix3(b, k, d, N, D)];
+        }
+        for (int i = 0; i < K; ++i) {
+            if (counts) counts[ix2(b, i, K)] = (int32_t)cnt[i];
+            if (cnt[i] > 0)
+                for (int d = 0; d < D; ++d)
+                    centroids[ix3(b, i, d, K, D)] = (float)(sum[ix2(i, d, D)] / (double)cnt[i]);
+        }
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Cluster-level statistics, optimistic index, arm selection.
+//  statistics (Algorithm 1 initialisation N=1, mu=0.5 and its running-mean
+//  lines, applied pull by pull, give exactly):
+//      N_{i,s}  = n0 + sum_{k in C_i} pulls[k][s]
+//      mu_{i,s} = (n0*mu0 + sum_{k in C_i} reward_sum[k][s]) / N_{i,s}
+//  cluster index (masked-UCB equation, Sec. 3.4):
+//      U_cl(i,s) = mu_{i,s} + c * sqrt(ln t / N_{i,s})
+//  arm index (Assumption 2: mu(k,s) <= mu(centre,s) + L*||phi(k) - centre||):
+//      U(k,s) = U_cl(label(k), s) + L * sqrt(dist2(k)),
+//      optionally capped by B(k,s) (Assumption 1).
+//  selection: best_arm = lowest flat index k*S+s maximising U over kept arms
+//  (-1 and -inf if none); best_cluster_arm = lowest i*S+s maximising U_cl over
+//  pairs with at least one kept member arm (the paper's M_{i,s} when the mask
+//  is constant within a cluster), -1 if none.
+//  arm_index holds -inf for a pruned arm.
+//  sel_margin (optional, double [B][2]): (best - runner-up with a different
+//  value) / |best| at arm level and at cluster level; +inf if no runner-up.
+// ---------------------------------------------------------------------------
+int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, float prior_pulls,
+                     float prior_mean, int cap_with_bound, const int32_t* labels, const float* dist2,
+                     const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
+                     const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean,
+                     float* cl_index, float* arm_index, int32_t* best_arm, float* best_val,
+                     int32_t* best_cluster_arm, double* sel_margin) {
+    if (S > 32) return 1;
+    const size_t KS = (size_t)K * (size_t)S;
+    std::vector<int64_t> np_(KS ? KS : 1);
+    std::vector<double> rs(KS ? KS : 1), ucl(KS ? KS : 1);
+    std::vector<char> anyk(KS ? KS : 1);
+    for (int b = 0; b < B; ++b) {
+        for (size_t i = 0; i < KS; ++i) { np_[i] = 0; rs[i] = 0.0; anyk[i] = 0; }
+        for (int k = 0; k < N; ++k) {
+            int lab = labels[ix2(b, k, N)];
+            if (lab < 0 || lab >= K) return 2;
+            uint32_t bits = keep ? keep[ix2(b, k, N)] : 0xffffffffu;
+            for (int s = 0; s < S; ++s) {
+                np_[ix2(lab, s, S)] += (int64_t)pulls[ix3(b, k, s, N, S)];
+                rs[ix2(lab, s, S)] += (double)reward_sum[ix3(b, k, s, N, S)];
+                if ((bits >> s) & 1u) anyk[ix2(lab, s, S)] = 1;
+            }
+        }
+        const double lnt = std::log((double)t[b]);
+        double cbest = -kInf, csecond = -kInf;
+        int carg = -1;
+        for (int i = 0; i < K; ++i)
+            for (int s = 0; s < S; ++s) {
+                double n = (double)prior_pulls + (double)np_[ix2(i, s, S)];
+                double mu = ((double)prior_pulls * (double)prior_mean + rs[ix2(i, s, S)]) / n;
+                double u = mu + (double)c * std::sqrt(lnt / n);
+                ucl[ix2(i, s, S)] = u;
+                cl_pulls[ix3(b, i, s, K, S)] = (float)n;
+                cl_mean[ix3(b, i, s, K, S)] = (float)mu;
+                cl_index[ix3(b, i, s, K, S)] = (float)u;
+                if (anyk[ix2(i, s, S)]) {
+                    if (u > cbest) { csecond = cbest; cbest = u; carg = i * S + s; }
+                    else if (u < cbest && u > csecond) { csecond = u; }
+                }
+            }
+        best_cluster_arm[b] = carg;
+
+        double abest = -kInf, asecond = -kInf;
+        int64_t aarg = -1;
+        for (int k = 0; k < N; ++k) {
+            int lab = labels[ix2(b, k, N)];
+            uint32_t bits = keep ? keep[ix2(b, k, N)] : 0xffffffffu;
+            double smooth = 0.0;
+            if (lipschitz_L != 0.0f) smooth = (double)lipschitz_L * std::sqrt((double)dist2[ix2(b, k, N)]);
+            for (int s = 0; s < S; ++s) {
+                double u = ucl[ix2(lab, s, S)] + smooth;
+                if (cap_with_bound && bound) {
+                    double cap = (double)bound[ix3(b, k, s, N, S)];
+                    if (cap < u) u = cap;
+                }
+                bool ok = (bits >> s) & 1u;
+                if (arm_index) arm_index[ix3(b, k, s, N, S)] = ok ? (float)u : -std::numeric_limits<float>::infinity();
+                if (!ok) continue;
+                if (u > abest) { asecond = abest; abest = u; aarg = (int64_t)k * S + s; }
+                else if (u < abest && u > asecond) { asecond = u; }
+            }
+        }
+        best_arm[b] = (int32_t)aarg;
+        best_val[b] = aarg >= 0 ? (float)abest : -std::numeric_limits<float>::infinity();
+        if (sel_margin) {
+            sel_margin[2 * b + 0] = (aarg >= 0 && asecond > -kInf) ? (abest - asecond) / std::fabs(abest) : kInf;
+            sel_margin[2 * b + 1] = (carg >= 0 && csecond > -kInf) ? (cbest - csecond) / std::fabs(cbest) : kInf;
+        }
+    }
+    return 0;
+}
+
+// Gather of initial centroids: C[b][i][:] = Z[b][rows[b][i]][:] (plain Lloyd
+// started from K data rows supplied by the caller).
+int kbo_init_centroids(int B, int N, int D, int K, const float* z, const int32_t* rows, float* centroids) {
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < K; ++i) {
+            int r = rows[ix2(b, i, K)];
+            if (r < 0 || r >= N) return 2;
+            for (int d = 0; d < D; ++d) centroids[ix3(b, i, d, K, D)] = z[ix3(b, r, d, N, D)];
+        }
+    return 0;
+}
+
+}  // extern "C"

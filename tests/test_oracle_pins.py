@@ -1,0 +1,386 @@
+"""CPU pins of the oracle: worked values, closed forms, invariants, brute force
+and library special cases.  None of these tests touches the CUDA library."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import scipy.spatial.distance
+import scipy.stats
+
+import oracle
+from conftest import read_golden
+from paper_2511_18868_b200 import workloads as wl
+
+
+# ----------------------------------------------------------------- normalise
+def test_normalize_worked_column():
+    rows = read_golden("zscore.txt")
+    x = np.array([[r[0]] for r in rows], np.float32)[None]          # [1,4,1]
+    z, mean, scale = oracle.normalize(x)
+    assert mean[0, 0] == pytest.approx(2.5, abs=1e-7)
+    assert scale[0, 0] == pytest.approx(1.1180340, abs=1e-6)
+    np.testing.assert_allclose(z[0, :, 0], [r[1] for r in rows], atol=1e-6)
+
+
+def test_normalize_matches_scipy_zscore_and_postconditions():
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal((3, 500, 7)) * rng.uniform(0.1, 50, 7) + rng.uniform(-100, 100, 7)).astype(np.float32)
+    x[:, :, 3] = 4.25                                               # a constant column
+    z, mean, scale = oracle.normalize(x)
+    for b in range(3):
+        ref = scipy.stats.zscore(x[b].astype(np.float64), axis=0, ddof=0)
+        ok = np.arange(7) != 3
+        np.testing.assert_allclose(z[b][:, ok], ref[:, ok], rtol=1e-5, atol=1e-6)
+        assert np.all(z[b][:, 3] == 0.0) and scale[b, 3] == 1.0
+        zz = z[b].astype(np.float64)
+        assert np.all(np.abs(zz[:, ok].mean(0)) < 1e-6)
+        np.testing.assert_allclose(zz[:, ok].var(0), 1.0, atol=1e-5)
+    z2, _, _ = oracle.normalize(z)                                   # idempotent
+    np.testing.assert_allclose(z2, z, atol=2e-6)
+
+
+def test_normalize_then_k1_inertia_is_N_times_D():
+    # closed form: after z-scoring, one cluster at the mean has inertia N * D
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((1, 300, 5)).astype(np.float32) * 3 + 1
+    z, _, _ = oracle.normalize(x)
+    c, counts = oracle.cluster_update(z, np.zeros((1, 300), np.int32), np.zeros((1, 1, 5), np.float32))
+    a = oracle.cluster_assign(z, c)
+    assert counts[0, 0] == 300 and np.all(a["labels"] == 0)
+    assert a["inertia"][0] == pytest.approx(300 * 5, rel=1e-5)
+
+
+# --------------------------------------------------------------------- prune
+def test_prune_worked_floor_values():
+    for F, Q, P, W, tlb in read_golden("roofline_floor.txt"):
+        args = dict(flops=[[F]], bytes_=[[Q]], peak_flops=[P], peak_bw=[W])
+        # the floor itself is observable through the threshold: kept iff T_lb < T_inc
+        assert oracle.prune(t_inc=[tlb * (1 + 1e-4)], **args)["keep"][0, 0] == 1
+        assert oracle.prune(t_inc=[tlb * (1 - 1e-4)], **args)["keep"][0, 0] == 0
+        # and through the bound: T_k = 2 * T_lb  ->  B = 0.5 ; T_k < T_lb -> 0
+        b = oracle.prune(t_inc=[1.0], t_cur=[[2 * tlb]], want_bound=True, **args)["bound"]
+        assert b[0, 0, 0] == pytest.approx(0.5, abs=1e-6)
+        b = oracle.prune(t_inc=[1.0], t_cur=[[0.5 * tlb]], want_bound=True, **args)["bound"]
+        assert b[0, 0, 0] == 0.0
+
+
+def test_prune_invariants_and_saturation_mask():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], N=400, S=13, K=5)
+    inp = wl.make_inputs(cfg, seed=3)
+    labels = np.random.default_rng(3).integers(0, cfg.K, (1, cfg.N)).astype(np.int32)
+    r = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+                     labels, inp["hsig"], inp["target"], 75.0, want_bound=True)
+    F, Q = inp["flops"].astype(np.float64), inp["bytes"].astype(np.float64)
+    P, W = inp["peak_flops"].astype(np.float64), inp["peak_bw"].astype(np.float64)
+    tlb = np.maximum(F[..., None] / P, Q[..., None] / W)
+    h = inp["hsig"].astype(np.float64)[0][labels[0]][:, inp["target"]][None]
+    bits = (r["keep"][..., None] >> np.arange(cfg.S)) & 1
+    # every kept arm: both strict inequalities; every pruned arm: at least one fails
+    assert np.all((tlb < inp["t_inc"][0])[bits == 1]) and np.all((h < 75.0)[bits == 1])
+    assert np.all(((tlb >= inp["t_inc"][0]) | (h >= 75.0))[bits == 0])
+    assert r["kept_count"][0] == bits.sum()
+    assert np.all(r["keep"] < (1 << cfg.S))
+    assert np.all((r["bound"] >= 0) & (r["bound"] <= 1))
+    # the incumbent is the 20th-percentile floor: about a fifth passes the roofline test
+    roof = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"])
+    frac = roof["kept_count"][0] / (cfg.N * cfg.S)
+    assert 0.17 < frac < 0.23
+    # monotone: raising the incumbent never clears a set bit
+    roof2 = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"] * 3)
+    assert np.all((roof["keep"] & ~roof2["keep"]) == 0) and roof2["kept_count"][0] > roof["kept_count"][0]
+    # saturation threshold is strict: h == theta is pruned
+    hs = np.array([[[75.0, 74.999, 80.0]]], np.float32)
+    r = oracle.prune([[1.0]], [[1.0]], [1e12] * 3, [1e12] * 3, [1.0], None, [[0]], hs, [0, 1, 2], 75.0)
+    assert r["keep"][0, 0] == 0b010
+
+
+# -------------------------------------------------------------------- assign
+def test_assign_against_cdist_and_optimality():
+    rng = np.random.default_rng(4)
+    B, N, D, K = 2, 700, 9, 11
+    z = rng.standard_normal((B, N, D)).astype(np.float32)
+    c = rng.standard_normal((B, K, D)).astype(np.float32)
+    a = oracle.cluster_assign(z, c, want_margins=True)
+    for b in range(B):
+        d2 = scipy.spatial.distance.cdist(z[b].astype(np.float64), c[b].astype(np.float64), "sqeuclidean")
+        assert np.array_equal(a["labels"][b], d2.argmin(1))
+        np.testing.assert_allclose(a["dist2"][b], d2.min(1), rtol=1e-6)
+        np.testing.assert_allclose(a["best"][b], d2.min(1), rtol=1e-12)
+        np.testing.assert_allclose(a["second"][b], np.sort(d2, 1)[:, 1], rtol=1e-12)
+        assert a["inertia"][b] == pytest.approx(d2.min(1).sum(), rel=1e-6)
+        # representative: the member nearest its centroid
+        for i in range(K):
+            members = np.flatnonzero(a["labels"][b] == i)
+            if len(members) == 0:
+                assert a["rep"][b, i] == -1
+            else:
+                assert a["rep"][b, i] == members[np.argmin(d2[members, i])]
+        np.testing.assert_allclose(oracle.dist2_at(z, c, a["labels"])[b], d2.min(1), rtol=1e-12)
+
+
+def test_assign_special_cases():
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((1, 50, 4)).astype(np.float32)
+    # K = 1: everything in cluster 0
+    assert np.all(oracle.cluster_assign(z, z[:, :1])["labels"] == 0)
+    # centroids that are data rows: those rows are at distance 0 with their own label
+    rows = np.array([7, 3, 41, 19])
+    a = oracle.cluster_assign(z, z[:, rows])
+    assert np.array_equal(a["labels"][0, rows], np.arange(4)) and np.all(a["dist2"][0, rows] == 0)
+    assert np.array_equal(a["rep"][0], rows)
+    # permuting centroids permutes labels
+    perm = np.array([2, 0, 3, 1])
+    a2 = oracle.cluster_assign(z, z[:, rows[perm]])
+    assert np.array_equal(perm[a2["labels"][0]], a["labels"][0])
+    # duplicate centroids: the lowest index wins; an unused one is empty
+    a3 = oracle.cluster_assign(z, z[:, [7, 7]])
+    assert np.all(a3["labels"] == 0) and a3["rep"][0, 1] == -1
+
+
+def test_lloyd_textbook_1d():
+    rows = read_golden("lloyd_1d.txt")
+    z = np.array([0, 1, 9, 10], np.float32).reshape(1, 4, 1)
+    c = np.array([rows[0][1], rows[0][2]], np.float32).reshape(1, 2, 1)
+    for it, c0, c1, l0, l1, l2, l3, inertia in rows:
+        np.testing.assert_allclose(c[0, :, 0], [c0, c1], rtol=1e-6)
+        a = oracle.cluster_assign(z, c)
+        assert list(a["labels"][0]) == [l0, l1, l2, l3]
+        assert a["inertia"][0] == pytest.approx(inertia, rel=1e-6)
+        c, counts = oracle.cluster_update(z, a["labels"], c)
+        assert counts.sum() == 4
+
+
+def test_lloyd_matches_sklearn_with_fixed_init():
+    from sklearn.cluster import KMeans
+    cfg = wl.scaled(wl.CONFIGS["medium"], N=1500, D=6, K=7, components=7)
+    inp = wl.make_inputs(cfg, seed=6)
+    z, _, _ = oracle.normalize(inp["x"])
+    c = oracle.init_centroids(z, inp["init_rows"])
+    c0 = c.copy()
+    iters = 12
+    for _ in range(iters):
+        a = oracle.cluster_assign(z, c)
+        c, counts = oracle.cluster_update(z, a["labels"], c)
+    a = oracle.cluster_assign(z, c)
+    km = KMeans(n_clusters=cfg.K, init=c0[0].astype(np.float64), n_init=1, max_iter=iters, tol=0.0,
+                algorithm="lloyd").fit(z[0].astype(np.float64))
+    np.testing.assert_allclose(c[0], km.cluster_centers_, rtol=1e-4, atol=1e-5)
+    assert a["inertia"][0] == pytest.approx(km.inertia_, rel=1e-4)
+    assert np.mean(a["labels"][0] == km.labels_) > 0.999
+
+
+# -------------------------------------------------------------------- update
+def test_update_is_group_mean():
+    rng = np.random.default_rng(7)
+    B, N, D, K = 2, 900, 5, 6
+    z = rng.standard_normal((B, N, D)).astype(np.float32)
+    labels = rng.integers(0, K - 1, (B, N)).astype(np.int32)      # cluster K-1 stays empty
+    prev = rng.standard_normal((B, K, D)).astype(np.float32)
+    c, counts = oracle.cluster_update(z, labels, prev)
+    for b in range(B):
+        sums = np.zeros((K, D))
+        np.add.at(sums, labels[b], z[b].astype(np.float64))
+        cnt = np.bincount(labels[b], minlength=K)
+        assert np.array_equal(counts[b], cnt) and cnt.sum() == N
+        np.testing.assert_allclose(c[b, :K - 1], sums[:K - 1] / cnt[:K - 1, None], rtol=1e-6, atol=1e-7)
+        assert np.array_equal(c[b, K - 1], prev[b, K - 1])         # empty cluster keeps its centroid
+        # count-weighted centroids reproduce the column sums of the members
+        np.testing.assert_allclose((counts[b, :K - 1, None] * c[b, :K - 1].astype(np.float64)).sum(0),
+                                   z[b].astype(np.float64).sum(0), atol=1e-3)
+
+
+def test_lloyd_objective_never_increases_and_is_a_local_optimum():
+    cfg = wl.scaled(wl.CONFIGS["medium"], N=2000, D=8, K=12, components=10)
+    inp = wl.make_inputs(cfg, seed=8)
+    out = oracle.bandit_step(inp, iters=15)
+    tr = out["inertia_trace"][:, 0].astype(np.float64)
+    assert np.all(np.diff(tr) <= 1e-6 * tr[:-1])
+    assert tr[-1] < 0.5 * tr[0]
+
+
+def test_lloyd_vs_exhaustive_labelings():
+    rng = np.random.default_rng(9)
+    N, D, K = 9, 2, 3
+    z = rng.standard_normal((1, N, D)).astype(np.float32)
+    c = z[:, :K].copy()
+    for _ in range(20):
+        a = oracle.cluster_assign(z, c)
+        c, _ = oracle.cluster_update(z, a["labels"], c)
+    a = oracle.cluster_assign(z, c)
+    zz = z[0].astype(np.float64)
+
+    def cost(lab):
+        tot = 0.0
+        for i in range(K):
+            m = zz[np.array(lab) == i]
+            if len(m):
+                tot += ((m - m.mean(0)) ** 2).sum()
+        return tot
+    best = min(cost(lab) for lab in itertools.product(range(K), repeat=N))
+    mine = cost(tuple(a["labels"][0]))
+    assert a["inertia"][0] == pytest.approx(mine, rel=1e-5)        # converged: centroids are the member means
+    assert mine >= best - 1e-9
+    # no single reassignment against the fixed centroids improves the objective
+    d2 = scipy.spatial.distance.cdist(zz, c[0].astype(np.float64), "sqeuclidean")
+    assert np.all(d2[np.arange(N), a["labels"][0]] <= d2.min(1) + 1e-12)
+
+
+# ----------------------------------------------------- statistics and index
+def _single_cluster_scores(pulls, rewards, t, **kw):
+    pulls = np.asarray(pulls, np.int32)
+    N, S = pulls.shape
+    return oracle.score_select(np.zeros((1, N), np.int32), np.zeros((1, N), np.float32), pulls[None],
+                               np.asarray(rewards, np.float32)[None], [t], K=1, **kw)
+
+
+def test_index_worked_values():
+    for t, n, mu, c, u in read_golden("masked_ucb_index.txt"):
+        # one cluster, one strategy: N = 1 + pulls, mu = (0.5 + sum r) / N
+        pulls = int(n) - 1
+        rsum = mu * n - 0.5
+        r = _single_cluster_scores([[pulls]], [[rsum]], int(t), c=c)
+        assert r["cl_pulls"][0, 0, 0] == n
+        assert r["cl_mean"][0, 0, 0] == pytest.approx(mu, abs=1e-6)
+        assert r["cl_index"][0, 0, 0] == pytest.approx(u, abs=2e-6)
+        # the same number read backwards: ((U - mu) / c)^2 * N = ln t
+        assert math.exp(((r["cl_index"][0, 0, 0] - mu) / c) ** 2 * n) == pytest.approx(t, rel=1e-4)
+
+
+def test_statistics_equal_algorithm1_running_mean():
+    for r1, r2, r3, r4, n_fin, mu_fin in read_golden("running_mean.txt"):
+        rewards = [r1, r2, r3, r4]
+        # pull-by-pull recursion of Algorithm 1, from its initialisation
+        n, mu = 1, 0.5
+        for r in rewards:
+            n += 1
+            mu += (r - mu) / n
+        assert (n, mu) == (n_fin, pytest.approx(mu_fin, abs=1e-12))
+        # the four pulls spread over two member kernels of the same cluster
+        out = _single_cluster_scores([[3], [1]], [[r1 + r2 + r3], [r4]], t=1)
+        assert out["cl_pulls"][0, 0, 0] == n_fin
+        assert out["cl_mean"][0, 0, 0] == pytest.approx(mu_fin, abs=1e-6)
+    # random histories: the batch aggregate equals the online recursion
+    rng = np.random.default_rng(10)
+    N, S, K = 40, 3, 4
+    labels = rng.integers(0, K, (1, N)).astype(np.int32)
+    pulls = rng.poisson(2.0, (1, N, S)).astype(np.int32)
+    per_pull = [[rng.uniform(0, 1, pulls[0, k, s]) for s in range(S)] for k in range(N)]
+    rsum = np.array([[per_pull[k][s].sum() for s in range(S)] for k in range(N)], np.float32)[None]
+    out = oracle.score_select(labels, np.zeros((1, N), np.float32), pulls, rsum, [5], K=K)
+    for i in range(K):
+        for s in range(S):
+            n, mu = 1, 0.5
+            for k in np.flatnonzero(labels[0] == i):
+                for r in per_pull[k][s]:
+                    n += 1
+                    mu += (r - mu) / n
+            assert out["cl_pulls"][0, i, s] == n
+            assert out["cl_mean"][0, i, s] == pytest.approx(mu, abs=1e-5)
+    assert (out["cl_pulls"].sum() - K * S) == pulls.sum()
+
+
+def test_unplayed_cluster_arms_outrank_played_ones():
+    # 3 clusters x 2 strategies; cluster 2 has never been played on strategy 1
+    labels = np.array([[0, 0, 1, 1, 2, 2]], np.int32)
+    pulls = np.array([[[4, 3], [2, 5], [6, 1], [3, 3], [2, 0], [5, 0]]], np.int32)
+    rsum = (pulls * 0.95).astype(np.float32)                      # played arms have a high mean
+    out = oracle.score_select(labels, np.zeros((1, 6), np.float32), pulls, rsum, [int(1 + pulls.sum())], K=3)
+    assert out["best_cluster_arm"][0] == 2 * 2 + 1
+    assert out["cl_pulls"][0, 2, 1] == 1 and out["cl_mean"][0, 2, 1] == 0.5
+    # with L = 0 all members of the winning cluster tie: the lowest k wins
+    assert out["best_arm"][0] == 4 * 2 + 1
+    # index is decreasing in N at fixed mean and increasing in t
+    a = _single_cluster_scores([[3]], [[0.5 * 4 - 0.5]], 50)["cl_index"][0, 0, 0]
+    b = _single_cluster_scores([[9]], [[0.5 * 10 - 0.5]], 50)["cl_index"][0, 0, 0]
+    c = _single_cluster_scores([[3]], [[0.5 * 4 - 0.5]], 500)["cl_index"][0, 0, 0]
+    assert b < a < c
+
+
+def test_select_k1_is_ucb1_and_masks():
+    rng = np.random.default_rng(11)
+    N, S = 30, 6
+    pulls = rng.poisson(3.0, (N, S)).astype(np.int32)
+    rsum = (pulls * rng.uniform(0, 1, (N, S))).astype(np.float32)
+    t = int(1 + pulls.sum())
+    out = _single_cluster_scores(pulls, rsum, t)
+    # K = 1, L = 0: plain UCB1 over the S strategies with pooled statistics
+    n = 1 + pulls.sum(0)
+    mu = (0.5 + rsum.astype(np.float64).sum(0)) / n
+    ucb = mu + 2.0 * np.sqrt(np.log(t) / n)
+    assert out["best_cluster_arm"][0] == int(np.argmax(ucb))
+    assert out["best_arm"][0] == int(np.argmax(ucb))               # k = 0 wins the tie inside the cluster
+    np.testing.assert_allclose(out["cl_index"][0, 0], ucb, rtol=1e-6)
+    # mask the winner everywhere: the runner-up strategy is chosen
+    s_best = int(np.argmax(ucb))
+    keep = np.full((1, N), (1 << S) - 1, np.uint32) & ~np.uint32(1 << s_best)
+    out2 = _single_cluster_scores(pulls, rsum, t, keep=keep)
+    order = np.argsort(-ucb)
+    assert out2["best_cluster_arm"][0] == order[1] and out2["best_arm"][0] == order[1]
+    assert np.all(np.isneginf(out2["arm_index"][0, :, s_best]))
+    # the winner kept only on candidate 17: that arm is chosen
+    keep[0, 17] |= np.uint32(1 << s_best)
+    out3 = _single_cluster_scores(pulls, rsum, t, keep=keep)
+    assert out3["best_arm"][0] == 17 * S + s_best and out3["best_cluster_arm"][0] == s_best
+    # everything masked
+    out4 = _single_cluster_scores(pulls, rsum, t, keep=np.zeros((1, N), np.uint32))
+    assert out4["best_arm"][0] == -1 and np.isneginf(out4["best_val"][0]) and out4["best_cluster_arm"][0] == -1
+
+
+def test_lipschitz_term_and_bound_cap():
+    labels = np.array([[0, 0, 0]], np.int32)
+    dist2 = np.array([[0.0, 4.0, 9.0]], np.float32)
+    pulls = np.ones((1, 3, 2), np.int32)
+    rsum = np.full((1, 3, 2), 0.25, np.float32)
+    out = oracle.score_select(labels, dist2, pulls, rsum, [1], K=1, lipschitz_L=0.5)
+    base = out["cl_index"][0, 0]
+    # t = 1: no exploration bonus, so U(k,s) = mu + L * sqrt(d2)
+    np.testing.assert_allclose(out["arm_index"][0], base[None] + 0.5 * np.array([[0.0], [2.0], [3.0]]), rtol=1e-6)
+    assert out["best_arm"][0] == 2 * 2 + 0
+    bound = np.full((1, 3, 2), 10.0, np.float32)
+    bound[0, 2, :] = 0.1
+    out = oracle.score_select(labels, dist2, pulls, rsum, [1], K=1, lipschitz_L=0.5, bound=bound, cap_with_bound=True)
+    np.testing.assert_allclose(out["arm_index"][0, 2], 0.1, rtol=1e-6)
+    assert out["best_arm"][0] == 1 * 2 + 0
+
+
+def test_select_brute_force_on_tiny_inputs():
+    rng = np.random.default_rng(12)
+    for trial in range(20):
+        N, S, K = 12, 3, 4
+        labels = rng.integers(0, K, (1, N)).astype(np.int32)
+        dist2 = rng.uniform(0, 4, (1, N)).astype(np.float32)
+        pulls = rng.poisson(1.5, (1, N, S)).astype(np.int32)
+        rsum = (pulls * rng.uniform(0, 2, (1, N, S))).astype(np.float32)
+        keep = rng.integers(0, 1 << S, (1, N)).astype(np.uint32)
+        t = int(1 + pulls.sum())
+        out = oracle.score_select(labels, dist2, pulls, rsum, [t], K=K, keep=keep, lipschitz_L=0.1)
+        # exhaustive evaluation, arm by arm, from the per-cluster sums
+        best, arg = -np.inf, -1
+        for k in range(N):
+            for s in range(S):
+                if not (keep[0, k] >> s) & 1:
+                    continue
+                m = labels[0] == labels[0, k]
+                n = 1 + pulls[0, m, s].sum()
+                mu = (0.5 + rsum[0, m, s].astype(np.float64).sum()) / n
+                u = mu + 2.0 * math.sqrt(math.log(t) / n) + 0.1 * math.sqrt(dist2[0, k])
+                if u > best:
+                    best, arg = u, k * S + s
+        assert out["best_arm"][0] == arg
+        assert out["best_val"][0] == pytest.approx(best, rel=1e-6)
+
+
+# ------------------------------------------------------------ input recipes
+def test_workload_shapes_and_determinism():
+    cfg = wl.CONFIGS["tiny"]
+    a, b = wl.make_inputs(cfg), wl.make_inputs(cfg)
+    for k in a:
+        assert np.array_equal(a[k], b[k])
+    assert a["x"].shape == (1, 256, 16) and a["pulls"].shape == (1, 256, 8)
+    assert len(set(a["init_rows"][0])) == cfg.K
+    assert a["t"][0] == 1 + a["pulls"].sum()
+    assert np.all(a["t_cur"] > 0)
+    assert wl.CONFIGS["contraction"].arms == 33554432 and wl.CONFIGS["batched"].arms == 8388608
+    m = wl.make_inputs(wl.scaled(wl.CONFIGS["medium"], N=4096))
+    assert 0.08 < np.mean(m["pulls"] == 0) < 0.16       # 10 % forced zeros + Poisson(4) zeros (1.8 %)
