@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the batched bandit step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (normalise, seed centroids, iters x
+(assign, update), final assign, prune, score/select) over one synthetic batch.
+`value` is arms scored per second with all inputs resident in HBM; `e2e` is the
+same step through the host-buffer entry point (host->device copies of every
+input and device->host copies of the results inside the timed region).
+With N > 1 (one process per GPU under torchrun) every rank runs an independent
+replica of the workload; there is no data-path collective.
+
+`--impl reference` times the CPU oracle instead (rank 0 only), each step being a
+bounded row sample of the same workload, extrapolated to the full size.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_18868_b200 import workloads as wl  # noqa: E402
+
+METRIC = "arms scored/sec per bandit step"
+UNIT = "arms/s"
+DEFAULT_WORKLOAD = "large"
+
+# rows of the workload the CPU oracle is timed on (per instance), and instances
+ORACLE_SAMPLE = {
+    # name: (instances, rows) for the in-run cpu_baseline; the reference arm uses a quarter of the rows
+    "tiny": (1, 256),
+    "medium": (1, 16384),
+    "large": (1, 262144),
+    "batched": (256, 512),
+    "contraction": (1, 65536),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+def algorithmic(cfg: wl.Workload):
+    """Algorithmic bytes and flops of ONE call of each class (what the method must move/compute)."""
+    R = cfg.B * cfg.N
+    B, D, K, S = cfg.B, cfg.D, cfg.K, cfg.S
+    return {
+        "normalize": {"bytes": 12 * R * D, "flops": 4 * R * D},
+        "assign": {"bytes": 4 * R * D + 4 * B * K * D + 8 * R, "flops": 2 * R * K * D},
+        "update": {"bytes": 4 * R * D + 4 * R + 4 * B * K * (D + 1), "flops": R * D},
+        "prune": {"bytes": 16 * R + 4 * R + 4 * R * S, "flops": 4 * R * S},
+        "score": {"bytes": 8 * R * S + 16 * R + 4 * R * S, "flops": 3 * R * S},
+    }
+
+
+# ------------------------------------------------------------------ CPU oracle
+def oracle_sample_step(cfg: wl.Workload, inst: int, rows: int, seed: int = 0):
+    """Times one pass of every oracle call on a row sample and extrapolates to the full step.
+    Returns (seconds per full step, seconds actually spent, description)."""
+    import oracle
+    inst, rows = min(inst, cfg.B), min(rows, cfg.N)
+    sub = wl.scaled(cfg, B=inst, N=rows)
+    inp = wl.make_inputs(sub, seed=seed)
+    t0 = time.perf_counter()
+    z, _, _ = oracle.normalize(inp["x"])
+    t1 = time.perf_counter()
+    c = oracle.init_centroids(z, inp["init_rows"])
+    ta = time.perf_counter()
+    a = oracle.cluster_assign(z, c, want_rep=True)
+    t2 = time.perf_counter()
+    c, _ = oracle.cluster_update(z, a["labels"], c)
+    t3 = time.perf_counter()
+    p = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+                     a["labels"], inp["hsig"], inp["target"], float(inp["theta_sat"]), want_bound=True)
+    t4 = time.perf_counter()
+    oracle.score_select(a["labels"], a["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], sub.K, keep=p["keep"],
+                        c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]))
+    t5 = time.perf_counter()
+    per_pass = (t1 - t0) + (cfg.iters + 1) * (t2 - ta) + cfg.iters * (t3 - t2) + (t4 - t3) + (t5 - t4)
+    scale = (cfg.B * cfg.N) / float(inst * rows)
+    desc = (f"oracle, 1 thread: one pass of each call on {inst} instance(s) x {rows} rows of the workload "
+            f"(K, D, S unchanged); assign x{cfg.iters + 1}, update x{cfg.iters}, scaled x{scale:g} to full size")
+    return per_pass * scale, t5 - t0, desc
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inst, rows = ORACLE_SAMPLE[cfg.name]
+    rows = max(1, rows // 4) if cfg.N > 4096 else rows
+    inst = max(1, inst // 4)
+    import oracle
+    oracle.build()
+    for _ in range(args.warmup):
+        oracle_sample_step(cfg, inst, rows)
+    secs, desc = [], ""
+    for k in range(args.steps):
+        s, _, desc = oracle_sample_step(cfg, inst, rows, seed=k)
+        secs.append(s)
+    per_step = float(np.mean(secs))
+    value = cfg.arms / per_step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "D": cfg.D, "K": cfg.K, "S": cfg.S, "iters": cfg.iters,
+            "arms": cfg.arms, "parallelism": "replicas (one independent step per GPU)",
+            "l2": "flushed between timed steps (256 MiB write)"}
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0])); mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args, cfg):
+    import torch
+    from paper_2511_18868_b200 import kb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    peaks = load_peaks()
+
+    inp = wl.make_inputs(cfg, seed=cfg.seed + rank)   # every replica draws its own batch
+    ctx = kb.KB(local)
+    R = wl.R_RESOURCES
+    dims = dict(B=cfg.B, N=cfg.N, D=cfg.D, K=cfg.K, S=cfg.S, R=R, iters=cfg.iters)
+    params = dict(theta_sat=float(inp["theta_sat"]), c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
+                  prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]))
+    ctx.ensure_workspace(max(ctx.workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S),
+                             ctx.step_workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S, R)))
+    dev_t = kb.step_tensors(inp, device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------
+    ctx.timing_enable(True)
+    for _ in range(args.warmup):
+        flush.zero_()
+        ctx.bandit_step(dims, params, dev_t)
+    ctx.timing_read()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    k0, m0 = ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in ev:
+        flush.zero_()
+        a.record()
+        ctx.bandit_step(dims, params, dev_t)
+        b.record()
+    barrier()
+    k1, m1 = ctx.launch_count()
+    clocks = sampler.stop()
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    per_class = ctx.timing_read()
+    ctx.timing_enable(False)
+    status = ctx.device_status()
+
+    # ---- end to end through the host-buffer entry point ----------------------------
+    host_t = kb.step_tensors(inp, None, pinned_host=True)
+    h2d = sum(host_t[n].numel() * 4 for n in kb._STEP_IN)
+    # results a caller of Algorithm 1 consumes: the selection, the cluster tables, the per-arm index
+    wanted = ["inertia", "rep", "kept_count", "bound", "cl_pulls", "cl_mean", "cl_index", "arm_index", "best_arm",
+              "best_val", "best_cluster_arm", "counts"]
+    e2e_t = {k: v for k, v in host_t.items() if k in kb._STEP_IN or k in wanted}
+    d2h = sum(e2e_t[n].numel() * 4 for n in wanted)
+    e2e_steps = max(1, min(args.steps, 5))
+    for _ in range(min(args.warmup, 2)):
+        ctx.bandit_step_host(dims, params, e2e_t)
+    barrier()
+    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e2e_steps)]
+    for a, b in e2e_ev:
+        flush.zero_()
+        a.record()
+        ctx.bandit_step_host(dims, params, e2e_t)
+        b.record()
+    barrier()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
+
+    # ---- max over ranks -----------------------------------------------------------
+    if dist is not None:
+        tt = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(tt[0]), float(tt[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.arms / (ms_per_step * 1e-3)
+    e2e_value = world * cfg.arms / (e2e_ms / e2e_steps * 1e-3)
+
+    # ---- per-call rooflines ---------------------------------------------------------
+    alg = algorithmic(cfg)
+    hbm = peaks["hbm_gbs"]
+    ffma_tflops = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # 148 SMs x 128 fp32 lanes x 2 flop x clock
+    kernels = {}
+    for name in ["normalize", "assign", "update", "prune", "score"]:
+        ms, calls = per_class[name]
+        if calls == 0:
+            continue
+        avg_s = ms / calls * 1e-3
+        gbs = alg[name]["bytes"] / avg_s / 1e9
+        kernels[name] = {"calls": int(calls), "avg_us": avg_s * 1e6, "share": ms / max(total_ms, 1e-9),
+                         "GBps": gbs, "hbm_frac": gbs / hbm, "TFLOPs": alg[name]["flops"] / avg_s / 1e12}
+    dominant = max(kernels, key=lambda n: kernels[n]["share"])
+    dk = kernels[dominant]
+    hbm_time = alg[dominant]["bytes"] / (hbm * 1e9)
+    alu_time = alg[dominant]["flops"] / (ffma_tflops * 1e12)
+    if dominant == "assign" and alu_time > hbm_time:
+        roof = {"bound": "alu", "achieved": dk["TFLOPs"], "peak": ffma_tflops, "unit": "TFLOP/s",
+                "frac": dk["TFLOPs"] / ffma_tflops, "traffic": None, "kernel": "kb_cluster_assign (fp32 FFMA path)",
+                "peak_source": "148 SM x 128 lanes x 2 flop x max SM clock",
+                "algorithmic_flops_per_launch": alg["assign"]["flops"]}
+    else:
+        roof = {"bound": "hbm", "achieved": dk["GBps"], "peak": hbm, "unit": "GB/s", "frac": dk["hbm_frac"],
+                "traffic": None, "kernel": f"kb_{dominant}", "peak_source": f"{peaks['source']} copy bandwidth",
+                "algorithmic_bytes_per_launch": alg[dominant]["bytes"]}
+
+    # ---- CPU oracle beside it (bounded sample) ----------------------------------------
+    cpu = None
+    if not args.no_cpu_baseline:
+        inst, rows = ORACLE_SAMPLE[cfg.name]
+        sec, spent, desc = oracle_sample_step(cfg, inst, rows)
+        cpu = {"value": cfg.arms / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+               "seconds_spent": spent, "host_cores": os.cpu_count()}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(cfg),
+        "roofline": roof, "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+        "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
+        "device_status": int(status), "peaks": peaks,
+    }
+    print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,261 @@
+/*
+ * kb.h -- C ABI of the batched bandit step (KernelBand decision layer) for
+ * NVIDIA B200 (sm_100a).
+ *
+ * One bandit step scores every arm (candidate kernel k, optimisation strategy
+ * s) of the action space A_t = P_t x S (Sec. 2.2) for B independent search
+ * instances:
+ *
+ *   kb_normalize        z-score of the trace features phi(k)       (Sec. 3.2)
+ *   kb_cluster_assign   K-Means nearest-centroid assignment        (Sec. 3.3)
+ *   kb_cluster_update   K-Means centroid update                    (Sec. 3.3)
+ *   kb_prune            roofline bound + saturation mask M_{i,s}   (Assumption 1, Sec. 3.4)
+ *   kb_score_select     cluster statistics, masked-UCB index with a
+ *                       Lipschitz term, arm selection    (Sec. 3.4, Assumption 2)
+ *
+ * Conventions (all entry points unless stated otherwise)
+ *  - Arrays are dense, row-major, batch-major: X[B][N][D], C[B][K][D],
+ *    labels[B][N], pulls[B][N][S], hsig[B][K][R].  B instances, N candidates,
+ *    D features, K clusters, S <= 32 strategies, R hardware resources.
+ *  - Every array pointer is a DEVICE pointer, borrowed: the caller allocates
+ *    and frees it; the library neither keeps nor frees it once the work queued
+ *    by the call has run.  fp32 arrays must be 16-byte aligned.
+ *  - Calls are asynchronous on the context's CUDA stream, allocate nothing and
+ *    do not synchronise with the host.  Scratch memory comes from the workspace
+ *    the caller registers with kb_set_workspace; calls that share a workspace
+ *    must be ordered on one stream.
+ *  - Outputs marked "nullable" are skipped when NULL.  Inputs and outputs must
+ *    not overlap unless stated.
+ *  - Return value: KB_OK or an error code; on error nothing has been queued.
+ *    B == 0 or N == 0 is valid: outputs that do not depend on candidates are
+ *    still written (counts 0, best_arm -1, ...).
+ *  - Non-finite inputs give unspecified results.  Ties go to the lowest index.
+ */
+#ifndef KB_H_
+#define KB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kb_ctx kb_ctx;
+
+typedef int kb_status;
+#define KB_OK 0
+#define KB_ERR_INVALID_ARG 1 /* null pointer, negative size, label/target out of contract */
+#define KB_ERR_UNSUPPORTED 2 /* valid request outside the implemented range (e.g. S > 32) */
+#define KB_ERR_WORKSPACE 3   /* no workspace registered or it is too small */
+#define KB_ERR_CUDA 4        /* a CUDA runtime call failed; see kb_last_error */
+#define KB_ERR_TIMEOUT 5     /* a bounded device-side wait expired (device status word) */
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context bound to `device` and to `cuda_stream` (a borrowed
+ * cudaStream_t; NULL = the legacy default stream).  Allocates a few bytes of
+ * device memory for the status word; that is the only allocation the library
+ * ever makes.  `out` is a host pointer. */
+kb_status kb_create(kb_ctx** out, int device, void* cuda_stream);
+kb_status kb_destroy(kb_ctx* ctx);
+/* Rebinds the context to another stream (borrowed). */
+kb_status kb_set_stream(kb_ctx* ctx, void* cuda_stream);
+
+/* Bytes of scratch the five calls and kb_cluster_fit need for these sizes
+ * (host pointer `out`).  kb_bandit_step* need kb_step_workspace_bytes. */
+kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out);
+/* Registers a device buffer (borrowed, 256-byte aligned) as scratch.  Its
+ * contents need not be initialised and are not preserved between calls. */
+kb_status kb_set_workspace(kb_ctx* ctx, void* dev_ptr, size_t bytes);
+
+const char* kb_status_string(kb_status s);
+/* Text of the last failure on this context (host string owned by the context). */
+const char* kb_last_error(kb_ctx* ctx);
+/* Reads the device status word (0 = fine).  Synchronises the stream; not for
+ * the hot path.  `out` is a host pointer. */
+kb_status kb_get_device_status(kb_ctx* ctx, int* out);
+/* Number of kernels of this library the context has queued since creation
+ * (`kernels`) and of memset nodes (`memsets`, nullable).  Host pointers. */
+kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets);
+
+/* Per-call device timing, a diagnostic that is off by default.  While on,
+ * each of the calls below brackets the work it queues with a pair of CUDA
+ * events on the context's stream (events come from a pool created by
+ * kb_timing_enable, so the calls still allocate nothing; calls beyond the
+ * pool's 4096 pairs between two reads go unrecorded).  kb_timing_read
+ * synchronises the stream, adds up the recorded pairs per class into
+ * ms[KB_T_COUNT] / calls[KB_T_COUNT] (host arrays) and empties the pool. */
+#define KB_T_NORMALIZE 0
+#define KB_T_ASSIGN 1
+#define KB_T_UPDATE 2
+#define KB_T_PRUNE 3
+#define KB_T_SCORE 4
+#define KB_T_INIT 5
+#define KB_T_COUNT 6
+kb_status kb_timing_enable(kb_ctx* ctx, int on);
+kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
+
+/* ---- the five calls ----------------------------------------------------- */
+
+/* Feature normalisation (Sec. 3.2 / App. A.1 say the features are normalised;
+ * the workloads fix the reading): per instance and column, the population
+ * z-score z = (x - mean) / std, std over N rows with divisor N; a column whose
+ * std is below 1e-12 gets scale 1 (it becomes all zeros).
+ *   x     [B][N][D] in
+ *   z     [B][N][D] out; may be the same pointer as x (in place)
+ *   mean  [B][D]    out, nullable
+ *   scale [B][D]    out, nullable (the divisor actually used) */
+kb_status kb_normalize(kb_ctx* ctx, int B, int N, int D, const float* x, float* z, float* mean,
+                       float* scale);
+
+/* Hardware-aware pruning.
+ *   roofline floor   T_lb(k,s) = max(flops[k] / peak_flops[s], bytes[k] / peak_bw[s])
+ *                    (the roofline model Assumption 1 cites for B(k,s))
+ *   keep bit s of keep[b][k] =  T_lb(k,s) < t_incumbent[b]
+ *                          AND  hsig[b][labels[b][k]][target[s]] < theta_sat
+ *                    (second factor: the mask equation of Sec. 3.4, strict <;
+ *                     applied only when labels, hsig and target are all given)
+ *   bound[b][k][s]   = clip((t_cur[k] - T_lb(k,s)) / t_cur[k], 0, 1)
+ *                    (Assumption 1: gap between current performance and the limit)
+ *   flops, bytes  [B][N] in;  peak_flops, peak_bw [S] in;  t_incumbent [B] in
+ *   t_cur         [B][N] in, nullable unless `bound` is requested
+ *   labels [B][N], hsig [B][K][R] (percent), target [S] (values in [0,R)): in,
+ *                 nullable together
+ *   keep          [B][N] out;  kept_count [B] out, nullable (number of set bits)
+ *   bound         [B][N][S] out, nullable */
+kb_status kb_prune(kb_ctx* ctx, int B, int N, int S, int K, int R, const float* flops,
+                   const float* bytes, const float* peak_flops, const float* peak_bw,
+                   const float* t_incumbent, const float* t_cur, const int32_t* labels,
+                   const float* hsig, const int32_t* target, float theta_sat, uint32_t* keep,
+                   uint32_t* kept_count, float* bound);
+
+/* K-Means assignment (Sec. 3.3; the KMeans line of Algorithm 1): for every
+ * row, the nearest centroid in squared Euclidean distance (the norm of
+ * Assumption 2); the lowest centroid id wins a tie.
+ *   z [B][N][D], centroids [B][K][D] in
+ *   labels  [B][N] out
+ *   dist2   [B][N] out, nullable: squared distance to the chosen centroid
+ *   inertia [B]    out, nullable: sum of dist2 over the instance
+ *   rep     [B][K] out, nullable: the member nearest its centroid (the
+ *           "centroid kernel" that Sec. 3.3 profiles), lowest k on ties,
+ *           -1 for an empty cluster */
+kb_status kb_cluster_assign(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
+                            const float* centroids, int32_t* labels, float* dist2, float* inertia,
+                            int32_t* rep);
+
+/* K-Means centroid update (Sec. 3.3; "Update centroids" in Algorithm 1): each
+ * centroid becomes the mean of its members; an empty cluster keeps its
+ * previous centroid.  labels must lie in [0,K).
+ *   centroids [B][K][D] in: previous, out: new;  counts [B][K] out, nullable */
+kb_status kb_cluster_update(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
+                            const int32_t* labels, float* centroids, int32_t* counts);
+
+typedef struct {
+    float c;            /* exploration weight of the masked-UCB index (paper: 2.0) */
+    float lipschitz_L;  /* L of Assumption 2; 0 reproduces the paper's index exactly */
+    float prior_pulls;  /* N_{i,s} before any pull (Algorithm 1: 1) */
+    float prior_mean;   /* mu_{i,s} before any pull (Algorithm 1: 0.5) */
+    int cap_with_bound; /* non-zero: U(k,s) = min(U(k,s), bound[k][s]) (Assumption 1) */
+} kb_score_params;
+
+/* Cluster statistics, optimistic index and selection.
+ *   N_{i,s}  = prior_pulls + sum over members k of cluster i of pulls[k][s]
+ *   mu_{i,s} = (prior_pulls*prior_mean + sum of reward_sum[k][s]) / N_{i,s}
+ *              (closed form of Algorithm 1's running-mean lines)
+ *   U_cl(i,s) = mu_{i,s} + c*sqrt(ln t / N_{i,s})      (masked-UCB equation, Sec. 3.4)
+ *   U(k,s)   = U_cl(labels[k], s) + L*sqrt(dist2[k])    (Assumption 2), optionally
+ *              capped by bound[k][s]
+ *   best_arm         = lowest k*S+s maximising U over arms whose keep bit is set
+ *                      (-1, best_val = -inf if none)
+ *   best_cluster_arm = lowest i*S+s maximising U_cl over pairs with at least
+ *                      one kept member arm (-1 if none)
+ *   labels [B][N] in; dist2 [B][N] in, nullable iff L == 0
+ *   pulls [B][N][S] (>= 0), reward_sum [B][N][S] in
+ *   keep [B][N] in, nullable = every arm valid; bound [B][N][S] in, nullable
+ *   t [B] in, >= 1
+ *   cl_pulls, cl_mean, cl_index [B][K][S] out
+ *   arm_index [B][N][S] out, nullable (-inf for a pruned arm)
+ *   best_arm, best_val, best_cluster_arm [B] out */
+kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p,
+                          const int32_t* labels, const float* dist2, const int32_t* pulls,
+                          const float* reward_sum, const uint32_t* keep, const float* bound,
+                          const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
+                          float* arm_index, int32_t* best_arm, float* best_val,
+                          int32_t* best_cluster_arm);
+
+/* ---- conveniences built from the five calls ----------------------------- */
+
+/* centroids[b][i][:] = z[b][rows[b][i]][:]  (plain Lloyd started from K data
+ * rows chosen by the caller; the paper leaves the initialisation open).
+ * rows [B][K] in, values in [0,N). */
+kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
+                            const int32_t* rows, float* centroids);
+
+/* iters x (assign, update) followed by a final assign, so that labels/dist2
+ * are consistent with the returned centroids (Sec. 3.3).  Same arguments as
+ * the two calls it is made of; counts are those of the last update. */
+kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z,
+                         float* centroids, int32_t* labels, float* dist2, float* inertia,
+                         int32_t* rep, int32_t* counts);
+
+/* Sizes and inputs/outputs of one whole bandit step.  Every pointer is a
+ * device pointer for kb_bandit_step and a HOST pointer for kb_bandit_step_host. */
+typedef struct {
+    int B, N, D, K, S, R, iters;
+    float theta_sat;
+    kb_score_params score;
+    /* inputs */
+    const float* x;             /* [B][N][D] raw features */
+    const int32_t* init_rows;   /* [B][K] */
+    const float* flops;         /* [B][N] */
+    const float* bytes;         /* [B][N] */
+    const float* peak_flops;    /* [S] */
+    const float* peak_bw;       /* [S] */
+    const float* t_incumbent;   /* [B] */
+    const float* t_cur;         /* [B][N] */
+    const float* hsig;          /* [B][K][R] */
+    const int32_t* target;      /* [S] */
+    const int32_t* pulls;       /* [B][N][S] */
+    const float* reward_sum;    /* [B][N][S] */
+    const int32_t* t;           /* [B] */
+    /* outputs (kb_bandit_step: all required except arm_index and bound;
+     * kb_bandit_step_host: any may be NULL and is then not copied back) */
+    float* z;                   /* [B][N][D] */
+    float* centroids;           /* [B][K][D] */
+    int32_t* counts;            /* [B][K] */
+    int32_t* labels;            /* [B][N] */
+    float* dist2;               /* [B][N] */
+    float* inertia;             /* [B] */
+    int32_t* rep;               /* [B][K] */
+    uint32_t* keep;             /* [B][N] */
+    uint32_t* kept_count;       /* [B] */
+    float* bound;               /* [B][N][S], nullable */
+    float* cl_pulls;            /* [B][K][S] */
+    float* cl_mean;             /* [B][K][S] */
+    float* cl_index;            /* [B][K][S] */
+    float* arm_index;           /* [B][N][S], nullable */
+    int32_t* best_arm;          /* [B] */
+    float* best_val;            /* [B] */
+    int32_t* best_cluster_arm;  /* [B] */
+} kb_step_args;
+
+/* The whole step on device-resident data: normalise, seed centroids, fit,
+ * prune (both masks, after the final assign because the saturation mask is
+ * indexed by the candidate's cluster), score and select.  Needs the workspace
+ * of kb_workspace_bytes. */
+kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
+
+/* The same step for a caller whose data lives in HOST memory: copies the
+ * inputs to the device, runs kb_bandit_step, copies the requested outputs
+ * back and synchronises the stream before returning.  The device staging
+ * area is carved from the registered workspace, which must hold
+ * kb_step_workspace_bytes(...) bytes.  Pinned host memory makes the copies
+ * asynchronous; pageable memory works too. */
+kb_status kb_step_workspace_bytes(int B, int N, int D, int K, int S, int R, size_t* out);
+kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* host_args);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KB_H_ */

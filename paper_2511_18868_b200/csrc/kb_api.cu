@@ -1,0 +1,447 @@
+// C ABI of libkb: context, argument validation, the call sequence of a whole
+// bandit step (device-resident and host-buffer variants).
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+
+#include "kb_internal.cuh"
+
+kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+namespace {
+
+__global__ void gather_rows_kernel(int N, int D, int K, const float* __restrict__ z, const int32_t* __restrict__ rows,
+                                   float* __restrict__ c, int* __restrict__ dev_status) {
+    const int b = blockIdx.y, i = blockIdx.x;
+    int r = rows[(size_t)b * K + i];
+    if (r < 0 || r >= N) { if (threadIdx.x == 0) atomicOr(dev_status, 4); return; }
+    const float* src = z + ((size_t)b * N + r) * D;
+    float* dst = c + ((size_t)b * K + i) * D;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = src[d];
+}
+
+size_t max_sz(size_t a, size_t b) { return a > b ? a : b; }
+
+// brackets the work one public call queues with a pair of events (when timing is on)
+struct TimeScope {
+    kb_ctx* ctx;
+    int slot;
+    TimeScope(kb_ctx* c, int cls) : ctx(c), slot(-1) {
+        if (c && c->timing && c->ev_used < KB_EV_PAIRS) {
+            slot = c->ev_used++;
+            c->ev_class[slot] = (unsigned char)cls;
+            cudaEventRecord(c->ev[2 * slot], c->stream);
+        }
+    }
+    ~TimeScope() {
+        if (slot >= 0) cudaEventRecord(ctx->ev[2 * slot + 1], ctx->stream);
+    }
+};
+
+}  // namespace
+
+kb_status kb_launch_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
+                                   float* c) {
+    if (B == 0 || K == 0) return KB_OK;
+    gather_rows_kernel<<<dim3(K, B), 64, 0, ctx->stream>>>(N, D, K, z, rows, c, ctx->dev_status);
+    KB_LAUNCH_CHECK(ctx, "gather_rows_kernel");
+    return KB_OK;
+}
+
+extern "C" {
+
+const char* kb_status_string(kb_status s) {
+    switch (s) {
+        case KB_OK: return "KB_OK";
+        case KB_ERR_INVALID_ARG: return "KB_ERR_INVALID_ARG";
+        case KB_ERR_UNSUPPORTED: return "KB_ERR_UNSUPPORTED";
+        case KB_ERR_WORKSPACE: return "KB_ERR_WORKSPACE";
+        case KB_ERR_CUDA: return "KB_ERR_CUDA";
+        case KB_ERR_TIMEOUT: return "KB_ERR_TIMEOUT";
+        default: return "KB_ERR_UNKNOWN";
+    }
+}
+
+kb_status kb_create(kb_ctx** out, int device, void* cuda_stream) {
+    if (!out) return KB_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return KB_ERR_CUDA;
+    kb_ctx* ctx = new (std::nothrow) kb_ctx();
+    if (!ctx) return KB_ERR_CUDA;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
+    if (e != cudaSuccess) {
+        if (ctx->dev_status) cudaFree(ctx->dev_status);
+        delete ctx;
+        return KB_ERR_CUDA;
+    }
+    *out = ctx;
+    return KB_OK;
+}
+
+kb_status kb_timing_enable(kb_ctx* ctx, int on) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    if (on && !ctx->ev) {
+        ctx->ev = new (std::nothrow) cudaEvent_t[2 * KB_EV_PAIRS];
+        ctx->ev_class = new (std::nothrow) unsigned char[KB_EV_PAIRS];
+        if (!ctx->ev || !ctx->ev_class) return kb_fail(ctx, KB_ERR_CUDA, "kb_timing_enable: out of host memory");
+        for (int i = 0; i < 2 * KB_EV_PAIRS; ++i) KB_CUDA(ctx, cudaEventCreate(&ctx->ev[i]));
+    }
+    ctx->timing = on != 0;
+    ctx->ev_used = 0;
+    return KB_OK;
+}
+
+kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls) {
+    if (!ctx || !ms || !calls) return KB_ERR_INVALID_ARG;
+    for (int i = 0; i < KB_T_COUNT; ++i) { ms[i] = 0.0; calls[i] = 0; }
+    KB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    for (int s = 0; s < ctx->ev_used; ++s) {
+        float t = 0.f;
+        KB_CUDA(ctx, cudaEventElapsedTime(&t, ctx->ev[2 * s], ctx->ev[2 * s + 1]));
+        ms[ctx->ev_class[s]] += (double)t;
+        calls[ctx->ev_class[s]]++;
+    }
+    ctx->ev_used = 0;
+    return KB_OK;
+}
+
+kb_status kb_destroy(kb_ctx* ctx) {
+    if (!ctx) return KB_OK;
+    cudaSetDevice(ctx->device);
+    if (ctx->ev) {
+        for (int i = 0; i < 2 * KB_EV_PAIRS; ++i) cudaEventDestroy(ctx->ev[i]);
+        delete[] ctx->ev;
+        delete[] ctx->ev_class;
+    }
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    delete ctx;
+    return KB_OK;
+}
+
+kb_status kb_set_stream(kb_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    return KB_OK;
+}
+
+kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
+    if (!out || B < 0 || N < 0 || D < 0 || K < 0 || S < 0) return KB_ERR_INVALID_ARG;
+    size_t need = 256;
+    need = max_sz(need, kb_ws_need_normalize(B, N, D));
+    need = max_sz(need, kb_ws_need_assign(B, N, D, K));
+    need = max_sz(need, kb_ws_need_update(B, N, D, K));
+    need = max_sz(need, kb_ws_need_score(B, N, K, S));
+    *out = need;
+    return KB_OK;
+}
+
+kb_status kb_set_workspace(kb_ctx* ctx, void* dev_ptr, size_t bytes) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    KB_REQUIRE(ctx, (dev_ptr != nullptr) == (bytes != 0), "kb_set_workspace: pointer and size disagree");
+    KB_REQUIRE(ctx, ((uintptr_t)dev_ptr & 255) == 0, "kb_set_workspace: workspace must be 256-byte aligned");
+    ctx->ws = static_cast<char*>(dev_ptr);
+    ctx->ws_bytes = bytes;
+    return KB_OK;
+}
+
+const char* kb_last_error(kb_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+
+kb_status kb_get_device_status(kb_ctx* ctx, int* out) {
+    if (!ctx || !out) return KB_ERR_INVALID_ARG;
+    KB_CUDA(ctx, cudaMemcpyAsync(out, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    KB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return KB_OK;
+}
+
+kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets) {
+    if (!ctx || !kernels) return KB_ERR_INVALID_ARG;
+    *kernels = ctx->launches;
+    if (memsets) *memsets = ctx->memsets;
+    return KB_OK;
+}
+
+#define KB_COMMON(ctx, B, N)                                                                   \
+    do {                                                                                       \
+        if (!(ctx)) return KB_ERR_INVALID_ARG;                                                 \
+        KB_REQUIRE(ctx, (B) >= 0 && (N) >= 0, "negative size");                                \
+        if ((B) > 65535) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "B = %d exceeds 65535", (B)); \
+    } while (0)
+
+kb_status kb_normalize(kb_ctx* ctx, int B, int N, int D, const float* x, float* z, float* mean, float* scale) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1, "kb_normalize: D must be >= 1");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, x && z, "kb_normalize: x and z are required");
+    if (D % 4 == 0)
+        KB_REQUIRE(ctx, (((uintptr_t)x | (uintptr_t)z) & 15) == 0, "kb_normalize: x and z must be 16-byte aligned");
+    TimeScope ts__(ctx, KB_T_NORMALIZE);
+    return kb_launch_normalize(ctx, B, N, D, x, z, mean, scale);
+}
+
+kb_status kb_prune(kb_ctx* ctx, int B, int N, int S, int K, int R, const float* flops, const float* bytes,
+                   const float* peak_flops, const float* peak_bw, const float* t_incumbent, const float* t_cur,
+                   const int32_t* labels, const float* hsig, const int32_t* target, float theta_sat, uint32_t* keep,
+                   uint32_t* kept_count, float* bound) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, S >= 1, "kb_prune: S must be >= 1");
+    if (S > 32) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_prune: S = %d exceeds 32 (keep bits are 32 wide)", S);
+    KB_REQUIRE(ctx, peak_flops && peak_bw, "kb_prune: the ceilings table is required");
+    if (B > 0) KB_REQUIRE(ctx, t_incumbent, "kb_prune: t_incumbent is required");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, flops && bytes && keep, "kb_prune: flops, bytes and keep are required");
+    const int nsat = (labels != nullptr) + (hsig != nullptr) + (target != nullptr);
+    KB_REQUIRE(ctx, nsat == 0 || nsat == 3, "kb_prune: labels, hsig and target must be given together");
+    if (nsat == 3) KB_REQUIRE(ctx, K >= 1 && R >= 1, "kb_prune: K and R must be >= 1 with the saturation mask");
+    if (bound) KB_REQUIRE(ctx, t_cur, "kb_prune: bound needs t_cur");
+    TimeScope ts__(ctx, KB_T_PRUNE);
+    return kb_launch_prune(ctx, B, N, S, K, R, flops, bytes, peak_flops, peak_bw, t_incumbent, t_cur, labels, hsig,
+                           target, theta_sat, keep, kept_count, bound);
+}
+
+kb_status kb_cluster_assign(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* centroids,
+                            int32_t* labels, float* dist2, float* inertia, int32_t* rep) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_assign: D and K must be >= 1");
+    if (B > 0) KB_REQUIRE(ctx, centroids, "kb_cluster_assign: centroids are required");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, z && labels, "kb_cluster_assign: z and labels are required");
+    if (D % 4 == 0)
+        KB_REQUIRE(ctx, (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0,
+                   "kb_cluster_assign: z and centroids must be 16-byte aligned");
+    TimeScope ts__(ctx, KB_T_ASSIGN);
+    return kb_launch_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+}
+
+kb_status kb_cluster_update(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* labels,
+                            float* centroids, int32_t* counts) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_update: D and K must be >= 1");
+    if (B > 0) KB_REQUIRE(ctx, centroids, "kb_cluster_update: centroids are required");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, z && labels, "kb_cluster_update: z and labels are required");
+    if (D % 4 == 0) KB_REQUIRE(ctx, ((uintptr_t)z & 15) == 0, "kb_cluster_update: z must be 16-byte aligned");
+    TimeScope ts__(ctx, KB_T_UPDATE);
+    return kb_launch_update(ctx, B, N, D, K, z, labels, centroids, counts);
+}
+
+kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p, const int32_t* labels,
+                          const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
+                          const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
+                          float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, K >= 1 && S >= 1, "kb_score_select: K and S must be >= 1");
+    if (S > 32) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_score_select: S = %d exceeds 32", S);
+    if ((long long)N * S > 0x7fffffffLL)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_score_select: N*S exceeds the 31-bit arm index");
+    KB_REQUIRE(ctx, p.prior_pulls > 0.f, "kb_score_select: prior_pulls must be positive");
+    if (B > 0)
+        KB_REQUIRE(ctx, t && cl_pulls && cl_mean && cl_index && best_arm && best_val && best_cluster_arm,
+                   "kb_score_select: t and the per-cluster / per-instance outputs are required");
+    if ((size_t)B * N > 0) {
+        KB_REQUIRE(ctx, labels && pulls && reward_sum, "kb_score_select: labels, pulls and reward_sum are required");
+        KB_REQUIRE(ctx, p.lipschitz_L == 0.f || dist2, "kb_score_select: dist2 is required when L != 0");
+        KB_REQUIRE(ctx, !p.cap_with_bound || bound, "kb_score_select: cap_with_bound needs bound");
+    }
+    TimeScope ts__(ctx, KB_T_SCORE);
+    return kb_launch_score(ctx, B, N, K, S, p, labels, dist2, pulls, reward_sum, keep, bound, t, cl_pulls, cl_mean,
+                           cl_index, arm_index, best_arm, best_val, best_cluster_arm);
+}
+
+kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
+                            float* centroids) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_init_centroids: D and K must be >= 1");
+    if (B > 0) {
+        KB_REQUIRE(ctx, N >= 1, "kb_init_centroids: needs at least one row to copy from");
+        KB_REQUIRE(ctx, z && rows && centroids, "kb_init_centroids: z, rows and centroids are required");
+    }
+    TimeScope ts__(ctx, KB_T_INIT);
+    return kb_launch_init_centroids(ctx, B, N, D, K, z, rows, centroids);
+}
+
+kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* centroids,
+                         int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, iters >= 0, "kb_cluster_fit: iters must be >= 0");
+    for (int it = 0; it < iters; ++it) {
+        kb_status s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
+        if (s != KB_OK) return s;
+        s = kb_cluster_update(ctx, B, N, D, K, z, labels, centroids, counts);
+        if (s != KB_OK) return s;
+    }
+    return kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+}
+
+kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
+    if (!ctx || !a) return KB_ERR_INVALID_ARG;
+    KB_COMMON(ctx, a->B, a->N);
+    kb_status s = kb_normalize(ctx, a->B, a->N, a->D, a->x, a->z, nullptr, nullptr);
+    if (s != KB_OK) return s;
+    s = kb_init_centroids(ctx, a->B, a->N, a->D, a->K, a->z, a->init_rows, a->centroids);
+    if (s != KB_OK) return s;
+    s = kb_cluster_fit(ctx, a->B, a->N, a->D, a->K, a->iters, a->z, a->centroids, a->labels, a->dist2, a->inertia,
+                       a->rep, a->counts);
+    if (s != KB_OK) return s;
+    s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
+                 a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count, a->bound);
+    if (s != KB_OK) return s;
+    return kb_score_select(ctx, a->B, a->N, a->K, a->S, a->score, a->labels, a->dist2, a->pulls, a->reward_sum,
+                           a->keep, a->bound, a->t, a->cl_pulls, a->cl_mean, a->cl_index, a->arm_index, a->best_arm,
+                           a->best_val, a->best_cluster_arm);
+}
+
+}  // extern "C"
+
+// ---- host-buffer step ----------------------------------------------------------
+namespace {
+struct Carver {
+    char* base;
+    size_t off;
+    template <typename T> T* take(size_t n) {
+        T* p = reinterpret_cast<T*>(base + off);
+        off += kb_align256(n * sizeof(T));
+        return p;
+    }
+};
+
+// device staging area of the host step; `base` may be null to only measure
+size_t carve_step(char* base, const kb_step_args& h, kb_step_args* d) {
+    Carver c{base, 0};
+    const size_t B = h.B, N = h.N, D = h.D, K = h.K, S = h.S, R = h.R;
+    kb_step_args t = h;
+    float* x = c.take<float>(B * N * D);
+    t.x = x; t.z = x;  // normalised in place
+    t.init_rows = c.take<int32_t>(B * K);
+    t.flops = c.take<float>(B * N);
+    t.bytes = c.take<float>(B * N);
+    t.peak_flops = c.take<float>(S);
+    t.peak_bw = c.take<float>(S);
+    t.t_incumbent = c.take<float>(B);
+    t.t_cur = c.take<float>(B * N);
+    t.hsig = c.take<float>(B * K * R);
+    t.target = c.take<int32_t>(S);
+    t.pulls = c.take<int32_t>(B * N * S);
+    t.reward_sum = c.take<float>(B * N * S);
+    t.t = c.take<int32_t>(B);
+    t.centroids = c.take<float>(B * K * D);
+    t.counts = c.take<int32_t>(B * K);
+    t.labels = c.take<int32_t>(B * N);
+    t.dist2 = c.take<float>(B * N);
+    t.inertia = c.take<float>(B);
+    t.rep = c.take<int32_t>(B * K);
+    t.keep = c.take<uint32_t>(B * N);
+    t.kept_count = c.take<uint32_t>(B);
+    t.bound = h.bound ? c.take<float>(B * N * S) : nullptr;
+    t.cl_pulls = c.take<float>(B * K * S);
+    t.cl_mean = c.take<float>(B * K * S);
+    t.cl_index = c.take<float>(B * K * S);
+    t.arm_index = h.arm_index ? c.take<float>(B * N * S) : nullptr;
+    t.best_arm = c.take<int32_t>(B);
+    t.best_val = c.take<float>(B);
+    t.best_cluster_arm = c.take<int32_t>(B);
+    if (d) *d = t;
+    return c.off;
+}
+}  // namespace
+
+extern "C" {
+
+kb_status kb_step_workspace_bytes(int B, int N, int D, int K, int S, int R, size_t* out) {
+    if (!out || B < 0 || N < 0 || D < 0 || K < 0 || S < 0 || R < 0) return KB_ERR_INVALID_ARG;
+    kb_step_args h;
+    memset(&h, 0, sizeof(h));
+    h.B = B; h.N = N; h.D = D; h.K = K; h.S = S; h.R = R;
+    // measured with both optional outputs present
+    h.bound = reinterpret_cast<float*>(1);
+    h.arm_index = reinterpret_cast<float*>(1);
+    size_t scratch = 0;
+    kb_workspace_bytes(B, N, D, K, S, &scratch);
+    *out = kb_align256(scratch) + carve_step(nullptr, h, nullptr);
+    return KB_OK;
+}
+
+kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
+    if (!ctx || !h) return KB_ERR_INVALID_ARG;
+    KB_COMMON(ctx, h->B, h->N);
+    KB_REQUIRE(ctx, h->D >= 1 && h->K >= 1 && h->S >= 1 && h->R >= 1, "kb_bandit_step_host: sizes must be >= 1");
+    size_t scratch = 0;
+    kb_workspace_bytes(h->B, h->N, h->D, h->K, h->S, &scratch);
+    scratch = kb_align256(scratch);
+    kb_step_args d;
+    const size_t stage = carve_step(nullptr, *h, nullptr);
+    if (ctx->ws_bytes < scratch + stage)
+        return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_bandit_step_host needs %zu bytes of workspace", scratch + stage);
+    carve_step(ctx->ws + scratch, *h, &d);
+    const size_t B = h->B, N = h->N, D = h->D, K = h->K, S = h->S, R = h->R;
+    cudaStream_t st = ctx->stream;
+#define KB_H2D(field, count, type)                                                                     \
+    do {                                                                                               \
+        if ((count) > 0) {                                                                             \
+            KB_REQUIRE(ctx, h->field, "kb_bandit_step_host: input " #field " is required");            \
+            KB_CUDA(ctx, cudaMemcpyAsync(const_cast<type*>(d.field), h->field, (count) * sizeof(type), \
+                                         cudaMemcpyHostToDevice, st));                                 \
+        }                                                                                              \
+    } while (0)
+    KB_H2D(x, B * N * D, float);
+    KB_H2D(init_rows, B * K, int32_t);
+    KB_H2D(flops, B * N, float);
+    KB_H2D(bytes, B * N, float);
+    KB_H2D(peak_flops, S, float);
+    KB_H2D(peak_bw, S, float);
+    KB_H2D(t_incumbent, B, float);
+    KB_H2D(t_cur, B * N, float);
+    KB_H2D(hsig, B * K * R, float);
+    KB_H2D(target, S, int32_t);
+    KB_H2D(pulls, B * N * S, int32_t);
+    KB_H2D(reward_sum, B * N * S, float);
+    KB_H2D(t, B, int32_t);
+#undef KB_H2D
+    // run on the workspace's scratch part only
+    char* ws_saved = ctx->ws;
+    size_t bytes_saved = ctx->ws_bytes;
+    ctx->ws_bytes = scratch;
+    kb_status s = kb_bandit_step(ctx, &d);
+    ctx->ws = ws_saved;
+    ctx->ws_bytes = bytes_saved;
+    if (s != KB_OK) return s;
+#define KB_D2H(field, count, type)                                                                          \
+    do {                                                                                                    \
+        if (h->field && (count) > 0)                                                                        \
+            KB_CUDA(ctx, cudaMemcpyAsync(h->field, d.field, (count) * sizeof(type), cudaMemcpyDeviceToHost, st)); \
+    } while (0)
+    KB_D2H(z, B * N * D, float);
+    KB_D2H(centroids, B * K * D, float);
+    KB_D2H(counts, B * K, int32_t);
+    KB_D2H(labels, B * N, int32_t);
+    KB_D2H(dist2, B * N, float);
+    KB_D2H(inertia, B, float);
+    KB_D2H(rep, B * K, int32_t);
+    KB_D2H(keep, B * N, uint32_t);
+    KB_D2H(kept_count, B, uint32_t);
+    KB_D2H(bound, B * N * S, float);
+    KB_D2H(cl_pulls, B * K * S, float);
+    KB_D2H(cl_mean, B * K * S, float);
+    KB_D2H(cl_index, B * K * S, float);
+    KB_D2H(arm_index, B * N * S, float);
+    KB_D2H(best_arm, B, int32_t);
+    KB_D2H(best_val, B, float);
+    KB_D2H(best_cluster_arm, B, int32_t);
+#undef KB_D2H
+    KB_CUDA(ctx, cudaStreamSynchronize(st));
+    return KB_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,114 @@
+// Internal declarations shared by the CUDA translation units of libkb.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "kb.h"
+
+struct kb_ctx {
+    int device;
+    cudaStream_t stream;
+    int sm_count;
+    int max_smem_optin;   // bytes of dynamic shared memory a block may opt into
+    char* ws;             // caller's workspace (device)
+    size_t ws_bytes;
+    int* dev_status;      // device status word (owned)
+    uint64_t launches;    // kernels queued so far
+    uint64_t memsets;     // memset nodes queued so far
+    // optional per-call event timing
+    bool timing;
+    cudaEvent_t* ev;      // 2 * KB_EV_PAIRS events
+    int ev_used;          // pairs in use
+    unsigned char* ev_class;
+    char err[256];
+};
+#define KB_EV_PAIRS 4096
+
+// ---- error plumbing ---------------------------------------------------------
+kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...);
+
+#define KB_CUDA(ctx, expr)                                                                     \
+    do {                                                                                       \
+        cudaError_t e__ = (expr);                                                              \
+        if (e__ != cudaSuccess)                                                                \
+            return kb_fail(ctx, KB_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__));        \
+    } while (0)
+
+#define KB_LAUNCH_CHECK(ctx, name)                                                             \
+    do {                                                                                       \
+        cudaError_t e__ = cudaGetLastError();                                                  \
+        if (e__ != cudaSuccess)                                                                \
+            return kb_fail(ctx, KB_ERR_CUDA, "launch of %s: %s", name, cudaGetErrorString(e__)); \
+        (ctx)->launches++;                                                                     \
+    } while (0)
+
+#define KB_MEMSET(ctx, ptr, val, bytes)                                                        \
+    do {                                                                                       \
+        KB_CUDA(ctx, cudaMemsetAsync(ptr, val, bytes, (ctx)->stream));                         \
+        (ctx)->memsets++;                                                                      \
+    } while (0)
+
+#define KB_REQUIRE(ctx, cond, msg)                                                             \
+    do {                                                                                       \
+        if (!(cond)) return kb_fail(ctx, KB_ERR_INVALID_ARG, "%s", msg);                       \
+    } while (0)
+
+// ---- workspace ------------------------------------------------------------------
+// Every call carves its scratch from the start of the workspace and clears the
+// control words it relies on, so nothing in the workspace has to survive from
+// one call to the next.  kb_workspace_bytes is the largest of these needs.
+size_t kb_ws_need_normalize(int B, int N, int D);
+size_t kb_ws_need_assign(int B, int N, int D, int K);
+size_t kb_ws_need_update(int B, int N, int D, int K);
+size_t kb_ws_need_score(int B, int N, int K, int S);
+#define KB_NORM_MAXG 1024
+int kb_norm_blocks_per_instance(int B, int N);
+static inline size_t kb_align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// ---- per-call launchers (each validates nothing: the API layer does) ----------
+kb_status kb_launch_normalize(kb_ctx*, int B, int N, int D, const float* x, float* z, float* mean, float* scale);
+kb_status kb_launch_prune(kb_ctx*, int B, int N, int S, int K, int R, const float* flops, const float* bytes,
+                          const float* peak_flops, const float* peak_bw, const float* t_inc, const float* t_cur,
+                          const int32_t* labels, const float* hsig, const int32_t* target, float theta,
+                          uint32_t* keep, uint32_t* kept, float* bound);
+kb_status kb_launch_assign(kb_ctx*, int B, int N, int D, int K, const float* z, const float* c, int32_t* labels,
+                           float* dist2, float* inertia, int32_t* rep);
+kb_status kb_launch_update(kb_ctx*, int B, int N, int D, int K, const float* z, const int32_t* labels,
+                           float* c, int32_t* counts);
+kb_status kb_launch_score(kb_ctx*, int B, int N, int K, int S, kb_score_params p, const int32_t* labels,
+                          const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
+                          const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
+                          float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm);
+kb_status kb_launch_init_centroids(kb_ctx*, int B, int N, int D, int K, const float* z, const int32_t* rows,
+                                   float* c);
+
+// Opts a kernel into more than 48 KB of dynamic shared memory when it needs it.
+#define KB_SMEM_OPTIN(ctx, kernel, bytes)                                                        \
+    do {                                                                                         \
+        if ((bytes) > 48 * 1024)                                                                 \
+            KB_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes))); \
+    } while (0)
+
+// ---- small device helpers -----------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ float kb_warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double kb_warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// monotone map float -> uint32 (larger float <=> larger uint)
+__device__ __forceinline__ uint32_t kb_orderable(float f) {
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float kb_from_orderable(uint32_t u) {
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+#endif

@@ -1,0 +1,313 @@
+"""Thin ctypes binding of libkb.so (include/kb.h).
+
+Argument marshalling only: every method passes `tensor.data_ptr()` and sizes to
+the C entry point of the same name.  PyTorch supplies device memory and the
+CUDA stream; no torch operator runs on the path.  There is no CPU fallback:
+if the library has not been built or no CUDA device is present, loading fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkb.so")
+
+KB_OK = 0
+STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3: "KB_ERR_WORKSPACE",
+                4: "KB_ERR_CUDA", 5: "KB_ERR_TIMEOUT"}
+
+# every symbol include/kb.h declares
+EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
+           "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
+           "kb_timing_enable", "kb_timing_read",
+           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select",
+           "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
+           "kb_bandit_step_host"]
+
+
+TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init"]
+
+
+class KbError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} {detail}".rstrip())
+
+
+class ScoreParams(ctypes.Structure):
+    _fields_ = [("c", ctypes.c_float), ("lipschitz_L", ctypes.c_float), ("prior_pulls", ctypes.c_float),
+                ("prior_mean", ctypes.c_float), ("cap_with_bound", ctypes.c_int)]
+
+
+_VP = ctypes.c_void_p
+_STEP_IN = ["x", "init_rows", "flops", "bytes", "peak_flops", "peak_bw", "t_incumbent", "t_cur", "hsig", "target",
+            "pulls", "reward_sum", "t"]
+_STEP_OUT = ["z", "centroids", "counts", "labels", "dist2", "inertia", "rep", "keep", "kept_count", "bound",
+             "cl_pulls", "cl_mean", "cl_index", "arm_index", "best_arm", "best_val", "best_cluster_arm"]
+
+
+class StepArgs(ctypes.Structure):
+    _fields_ = ([(n, ctypes.c_int) for n in ["B", "N", "D", "K", "S", "R", "iters"]] +
+                [("theta_sat", ctypes.c_float), ("score", ScoreParams)] +
+                [(n, _VP) for n in _STEP_IN + _STEP_OUT])
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libkb.so and declare the prototypes; raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2511_18868_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i, f, sz = ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.kb_create.argtypes = [ctypes.POINTER(_VP), i, _VP]
+    lib.kb_destroy.argtypes = [_VP]
+    lib.kb_set_stream.argtypes = [_VP, _VP]
+    lib.kb_workspace_bytes.argtypes = [i, i, i, i, i, ctypes.POINTER(sz)]
+    lib.kb_set_workspace.argtypes = [_VP, _VP, sz]
+    lib.kb_status_string.argtypes = [i]
+    lib.kb_status_string.restype = ctypes.c_char_p
+    lib.kb_last_error.argtypes = [_VP]
+    lib.kb_last_error.restype = ctypes.c_char_p
+    lib.kb_get_device_status.argtypes = [_VP, ctypes.POINTER(i)]
+    lib.kb_get_launch_count.argtypes = [_VP, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
+    lib.kb_timing_enable.argtypes = [_VP, i]
+    lib.kb_timing_read.argtypes = [_VP, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    lib.kb_normalize.argtypes = [_VP, i, i, i, _VP, _VP, _VP, _VP]
+    lib.kb_prune.argtypes = [_VP, i, i, i, i, i] + [_VP] * 9 + [f] + [_VP] * 3
+    lib.kb_cluster_assign.argtypes = [_VP, i, i, i, i] + [_VP] * 6
+    lib.kb_cluster_update.argtypes = [_VP, i, i, i, i] + [_VP] * 4
+    lib.kb_score_select.argtypes = [_VP, i, i, i, i, ScoreParams] + [_VP] * 14
+    lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
+    lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
+    lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
+    lib.kb_step_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(sz)]
+    lib.kb_bandit_step_host.argtypes = [_VP, ctypes.POINTER(StepArgs)]
+    for name in EXPORTS:
+        if name not in ("kb_status_string", "kb_last_error"):
+            getattr(lib, name).restype = i
+    _lib = lib
+    return lib
+
+
+# uint32 arrays (keep, kept_count) travel in int32 tensors: same storage, reinterpreted by the library
+
+
+def _ptr(t: Optional[torch.Tensor], device: Optional[torch.device] = None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("libkb takes dense row-major tensors")
+    if device is not None and t.device != device:
+        raise ValueError(f"tensor on {t.device}, context on {device}")
+    if t.element_size() != 4:
+        raise ValueError("libkb arrays are 32-bit")
+    return t.data_ptr()
+
+
+class KB:
+    """One library context bound to a device and to the current torch stream."""
+
+    def __init__(self, device: int = 0, stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libkb needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.device("cuda", device)
+        self._stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        h = _VP()
+        self._check(self.lib.kb_create(ctypes.byref(h), device, _VP(self._stream.cuda_stream)), "kb_create", ctx=None)
+        self.h = h
+        self._ws: Optional[torch.Tensor] = None
+
+    # -- plumbing -----------------------------------------------------------
+    def _check(self, status: int, where: str, ctx="self"):
+        if status != KB_OK:
+            detail = ""
+            if ctx is not None and getattr(self, "h", None):
+                detail = self.lib.kb_last_error(self.h).decode()
+            raise KbError(status, where, detail)
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.kb_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_stream(self, stream: torch.cuda.Stream):
+        self._stream = stream
+        self._check(self.lib.kb_set_stream(self.h, _VP(stream.cuda_stream)), "kb_set_stream")
+
+    def workspace_bytes(self, B, N, D, K, S) -> int:
+        out = ctypes.c_size_t()
+        self._check(self.lib.kb_workspace_bytes(B, N, D, K, S, ctypes.byref(out)), "kb_workspace_bytes")
+        return out.value
+
+    def step_workspace_bytes(self, B, N, D, K, S, R) -> int:
+        out = ctypes.c_size_t()
+        self._check(self.lib.kb_step_workspace_bytes(B, N, D, K, S, R, ctypes.byref(out)), "kb_step_workspace_bytes")
+        return out.value
+
+    def set_workspace(self, ws: Optional[torch.Tensor]):
+        self._ws = ws
+        n = 0 if ws is None else ws.numel() * ws.element_size()
+        self._check(self.lib.kb_set_workspace(self.h, None if ws is None else ws.data_ptr(), n), "kb_set_workspace")
+
+    def ensure_workspace(self, nbytes: int):
+        """Registers a torch-allocated workspace of at least `nbytes` (grows only)."""
+        have = 0 if self._ws is None else self._ws.numel()
+        if have < nbytes:
+            self.set_workspace(torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device))
+
+    def device_status(self) -> int:
+        out = ctypes.c_int()
+        self._check(self.lib.kb_get_device_status(self.h, ctypes.byref(out)), "kb_get_device_status")
+        return out.value
+
+    def launch_count(self):
+        """(kernels, memset nodes) queued by this context so far."""
+        k, m = ctypes.c_uint64(), ctypes.c_uint64()
+        self._check(self.lib.kb_get_launch_count(self.h, ctypes.byref(k), ctypes.byref(m)), "kb_get_launch_count")
+        return k.value, m.value
+
+    def timing_enable(self, on: bool = True):
+        self._check(self.lib.kb_timing_enable(self.h, int(on)), "kb_timing_enable")
+
+    def timing_read(self):
+        """{class name: (milliseconds, calls)} since the last read; synchronises."""
+        ms = (ctypes.c_double * len(TIMING_CLASSES))()
+        n = (ctypes.c_int64 * len(TIMING_CLASSES))()
+        self._check(self.lib.kb_timing_read(self.h, ms, n), "kb_timing_read")
+        return {name: (ms[i], n[i]) for i, name in enumerate(TIMING_CLASSES)}
+
+    def _p(self, t):
+        return _ptr(t, self.device)
+
+    # -- the five calls -----------------------------------------------------
+    def normalize(self, x, z=None, mean=None, scale=None):
+        B, N, D = x.shape
+        z = x if z is None else z
+        self._check(self.lib.kb_normalize(self.h, B, N, D, self._p(x), self._p(z), self._p(mean), self._p(scale)),
+                    "kb_normalize")
+        return z
+
+    def prune(self, flops, bytes_, peak_flops, peak_bw, t_incumbent, keep, t_cur=None, labels=None, hsig=None,
+              target=None, theta_sat=75.0, kept_count=None, bound=None):
+        B, N = flops.shape
+        S = peak_flops.shape[0]
+        K, R = (hsig.shape[1], hsig.shape[2]) if hsig is not None else (0, 0)
+        self._check(self.lib.kb_prune(self.h, B, N, S, K, R, self._p(flops), self._p(bytes_), self._p(peak_flops),
+                                      self._p(peak_bw), self._p(t_incumbent), self._p(t_cur), self._p(labels),
+                                      self._p(hsig), self._p(target), float(theta_sat), self._p(keep),
+                                      self._p(kept_count), self._p(bound)), "kb_prune")
+
+    def cluster_assign(self, z, centroids, labels, dist2=None, inertia=None, rep=None):
+        B, N, D = z.shape
+        K = centroids.shape[1]
+        self._check(self.lib.kb_cluster_assign(self.h, B, N, D, K, self._p(z), self._p(centroids), self._p(labels),
+                                               self._p(dist2), self._p(inertia), self._p(rep)), "kb_cluster_assign")
+
+    def cluster_update(self, z, labels, centroids, counts=None):
+        B, N, D = z.shape
+        K = centroids.shape[1]
+        self._check(self.lib.kb_cluster_update(self.h, B, N, D, K, self._p(z), self._p(labels), self._p(centroids),
+                                               self._p(counts)), "kb_cluster_update")
+
+    def score_select(self, labels, dist2, pulls, reward_sum, t, cl_pulls, cl_mean, cl_index, best_arm, best_val,
+                     best_cluster_arm, keep=None, bound=None, arm_index=None, c=2.0, lipschitz_L=0.0,
+                     prior_pulls=1.0, prior_mean=0.5, cap_with_bound=False):
+        B, N, S = pulls.shape
+        K = cl_index.shape[1]
+        p = ScoreParams(c, lipschitz_L, prior_pulls, prior_mean, int(bool(cap_with_bound)))
+        self._check(self.lib.kb_score_select(self.h, B, N, K, S, p, self._p(labels), self._p(dist2), self._p(pulls),
+                                             self._p(reward_sum), self._p(keep), self._p(bound), self._p(t),
+                                             self._p(cl_pulls), self._p(cl_mean), self._p(cl_index),
+                                             self._p(arm_index), self._p(best_arm), self._p(best_val),
+                                             self._p(best_cluster_arm)), "kb_score_select")
+
+    # -- conveniences -------------------------------------------------------
+    def init_centroids(self, z, rows, centroids):
+        B, N, D = z.shape
+        K = rows.shape[1]
+        self._check(self.lib.kb_init_centroids(self.h, B, N, D, K, self._p(z), self._p(rows), self._p(centroids)),
+                    "kb_init_centroids")
+
+    def cluster_fit(self, z, centroids, labels, iters, dist2=None, inertia=None, rep=None, counts=None):
+        B, N, D = z.shape
+        K = centroids.shape[1]
+        self._check(self.lib.kb_cluster_fit(self.h, B, N, D, K, int(iters), self._p(z), self._p(centroids),
+                                            self._p(labels), self._p(dist2), self._p(inertia), self._p(rep),
+                                            self._p(counts)), "kb_cluster_fit")
+
+    def _step_args(self, dims: Dict[str, int], params: Dict[str, float], tensors: Dict[str, torch.Tensor], host: bool):
+        a = StepArgs()
+        for k in ["B", "N", "D", "K", "S", "R", "iters"]:
+            setattr(a, k, int(dims[k]))
+        a.theta_sat = float(params.get("theta_sat", 75.0))
+        a.score = ScoreParams(float(params.get("c", 2.0)), float(params.get("lipschitz_L", 0.0)),
+                              float(params.get("prior_pulls", 1.0)), float(params.get("prior_mean", 0.5)),
+                              int(bool(params.get("cap_with_bound", False))))
+        for name in _STEP_IN + _STEP_OUT:
+            t = tensors.get(name)
+            setattr(a, name, None if t is None else _ptr(t, None if host else self.device))
+        return a
+
+    def bandit_step(self, dims, params, tensors):
+        """Whole step on device tensors (dict keyed by the field names of kb_step_args)."""
+        a = self._step_args(dims, params, tensors, host=False)
+        self._check(self.lib.kb_bandit_step(self.h, ctypes.byref(a)), "kb_bandit_step")
+
+    def bandit_step_host(self, dims, params, tensors):
+        """Whole step on HOST tensors (ideally pinned); returns after the results are in host memory."""
+        a = self._step_args(dims, params, tensors, host=True)
+        self._check(self.lib.kb_bandit_step_host(self.h, ctypes.byref(a)), "kb_bandit_step_host")
+
+
+def step_tensors(inp: Dict, device, want_arm_index=True, want_bound=True, pinned_host=False) -> Dict[str, torch.Tensor]:
+    """Moves a workload dict (numpy arrays of `workloads.make_inputs`) into the
+    tensors one bandit step takes, plus freshly allocated outputs."""
+    import numpy as np
+    names = {"x": "x", "init_rows": "init_rows", "flops": "flops", "bytes": "bytes", "peak_flops": "peak_flops",
+             "peak_bw": "peak_bw", "t_inc": "t_incumbent", "t_cur": "t_cur", "hsig": "hsig", "target": "target",
+             "pulls": "pulls", "reward_sum": "reward_sum", "t": "t"}
+    out: Dict[str, torch.Tensor] = {}
+    for src, dst in names.items():
+        t = torch.from_numpy(np.ascontiguousarray(inp[src]))
+        if pinned_host:
+            t = t.pin_memory() if torch.cuda.is_available() else t
+        else:
+            t = t.to(device)
+        out[dst] = t
+    B, N, D = inp["x"].shape
+    K, S = inp["init_rows"].shape[1], inp["pulls"].shape[2]
+    kw = dict(device="cpu", pin_memory=torch.cuda.is_available()) if pinned_host else dict(device=device)
+
+    def new(shape, dt):
+        return torch.empty(shape, dtype=dt, **kw)
+    out.update(
+        z=new((B, N, D), torch.float32),
+        centroids=new((B, K, D), torch.float32), counts=new((B, K), torch.int32),
+        labels=new((B, N), torch.int32), dist2=new((B, N), torch.float32), inertia=new((B,), torch.float32),
+        rep=new((B, K), torch.int32), keep=new((B, N), torch.int32), kept_count=new((B,), torch.int32),
+        cl_pulls=new((B, K, S), torch.float32), cl_mean=new((B, K, S), torch.float32),
+        cl_index=new((B, K, S), torch.float32), best_arm=new((B,), torch.int32),
+        best_val=new((B,), torch.float32), best_cluster_arm=new((B,), torch.int32))
+    if want_bound:
+        out["bound"] = new((B, N, S), torch.float32)
+    if want_arm_index:
+        out["arm_index"] = new((B, N, S), torch.float32)
+    return out
