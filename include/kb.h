@@ -184,6 +184,29 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
                           float* arm_index, int32_t* best_arm, float* best_val,
                           int32_t* best_cluster_arm);
 
+/* Which kernel kb_cluster_assign uses.
+ *   path: 0 = automatic (tensor cores when K >= 128, D a multiple of 32 and
+ *             <= 128 and there are at least 4096 rows; else the fp32 row-wise
+ *             kernel), 1 = always the fp32 row-wise kernel, 2 = always the
+ *             tensor-core kernel (KB_ERR_UNSUPPORTED where it cannot run).
+ *   tc_eps:   the tensor-core kernel ranks centroids by ||c||^2 - 2 z.c
+ *             evaluated as a 3xTF32 split product; a row whose best and
+ *             second-best scores differ by no more than
+ *             tc_eps * (||z||^2 + ||c||^2) is re-evaluated exactly (direct
+ *             form, fp32).  <= 0 keeps the default 2^-16.
+ * kb_get_assign_path reports what the last kb_cluster_assign ran (1 or 2). */
+kb_status kb_set_assign_options(kb_ctx* ctx, int path, float tc_eps);
+kb_status kb_get_assign_path(kb_ctx* ctx, int* out);
+
+/* Diagnostic for the tensor-core assign kernel: runs it on (z, centroids) and
+ * returns, besides the labels, the expanded-form squared distance it ranked
+ * by (approx_dist2 [B][N], nullable) and the number of rows that went through
+ * the exact re-evaluation (flagged, one int32 in DEVICE memory, nullable).
+ * Same workspace as kb_cluster_assign. */
+kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
+                             const float* centroids, int32_t* labels, float* approx_dist2,
+                             int32_t* flagged);
+
 /* ---- conveniences built from the five calls ----------------------------- */
 
 /* centroids[b][i][:] = z[b][rows[b][i]][:]  (plain Lloyd started from K data

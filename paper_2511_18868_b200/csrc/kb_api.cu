@@ -81,6 +81,7 @@ kb_status kb_create(kb_ctx** out, int device, void* cuda_stream) {
     memset(ctx, 0, sizeof(*ctx));
     ctx->device = device;
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->tc_eps = 1.0f / 65536.0f;
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -224,6 +225,36 @@ kb_status kb_cluster_assign(kb_ctx* ctx, int B, int N, int D, int K, const float
                    "kb_cluster_assign: z and centroids must be 16-byte aligned");
     TimeScope ts__(ctx, KB_T_ASSIGN);
     return kb_launch_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+}
+
+kb_status kb_set_assign_options(kb_ctx* ctx, int path, float tc_eps) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    KB_REQUIRE(ctx, path >= 0 && path <= 2, "kb_set_assign_options: path must be 0, 1 or 2");
+    ctx->assign_path = path;
+    ctx->tc_eps = tc_eps > 0.f ? tc_eps : 1.0f / 65536.0f;
+    return KB_OK;
+}
+
+kb_status kb_get_assign_path(kb_ctx* ctx, int* out) {
+    if (!ctx || !out) return KB_ERR_INVALID_ARG;
+    *out = ctx->last_assign_path;
+    return KB_OK;
+}
+
+kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* centroids,
+                             int32_t* labels, float* approx_dist2, int32_t* flagged) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_assign_tc_probe: D and K must be >= 1");
+    KB_REQUIRE(ctx, z && centroids && labels, "kb_assign_tc_probe: z, centroids and labels are required");
+    if (!kb_assign_tc_supported(ctx, D, K))
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_assign_tc_probe: needs D %% 32 == 0, D <= 128, K <= 8192");
+    if (B == 0 || N == 0) return KB_OK;
+    const size_t off = kb_ws_need_assign(B, N, D, K) - kb_ws_need_assign_tc(B, N, D, K);
+    if (ctx->ws_bytes < kb_ws_need_assign(B, N, D, K))
+        return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_assign_tc_probe needs %zu bytes of workspace",
+                       kb_ws_need_assign(B, N, D, K));
+    TimeScope ts__(ctx, KB_T_ASSIGN);
+    return kb_launch_assign_tc(ctx, ctx->ws + off, B, N, D, K, z, centroids, labels, approx_dist2, flagged, ctx->tc_eps);
 }
 
 kb_status kb_cluster_update(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* labels,

@@ -130,53 +130,76 @@ assign_rowwise_kernel(int N, int D, int K, int TM, int CT, const float* __restri
 }  // namespace
 
 size_t kb_ws_need_assign(int B, int N, int D, int K) {
-    (void)N; (void)D;
-    return kb_align256((size_t)B * sizeof(double)) + kb_align256((size_t)B * K * sizeof(unsigned long long));
+    // generic scratch (inertia double[B] | rep uint64[B][K]) followed by the tensor path's scratch
+    return kb_align256((size_t)B * sizeof(double)) + kb_align256((size_t)B * K * sizeof(unsigned long long)) +
+           kb_ws_need_assign_tc(B, N, D, K);
+}
+
+static kb_status launch_rowwise(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* c,
+                                int32_t* labels, float* dist2, double* ws_inertia, unsigned long long* ws_rep) {
+    // rows per block: as many as fit beside the centroid tile in 96 KB, at most 128
+    const size_t budget = 96 * 1024;
+    int CT = (int)((16 * 1024) / ((size_t)D * 4));
+    CT = CT / AS_GROUP * AS_GROUP;
+    if (CT < AS_GROUP) CT = AS_GROUP;
+    if (CT > ((K + AS_GROUP - 1) / AS_GROUP) * AS_GROUP) CT = ((K + AS_GROUP - 1) / AS_GROUP) * AS_GROUP;
+    size_t cbytes = (size_t)CT * D * 4;
+    if (cbytes + (size_t)32 * (D + 1) * 4 > budget)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_assign: D = %d is beyond the row-wise path", D);
+    int TM = (int)((budget - cbytes) / ((size_t)(D + 1) * 4));
+    TM = TM >= 128 ? 128 : (TM / 32 * 32);
+    size_t smem = cbytes + (size_t)TM * (D + 1) * 4;
+    dim3 grid((N + TM - 1) / TM, B);
+    if (D % 4 == 0) {
+        KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<true>, smem);
+        assign_rowwise_kernel<true><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
+                                                                     ws_inertia, ws_rep);
+    } else {
+        KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<false>, smem);
+        assign_rowwise_kernel<false><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
+                                                                      ws_inertia, ws_rep);
+    }
+    KB_LAUNCH_CHECK(ctx, "assign_rowwise_kernel");
+    return KB_OK;
 }
 
 kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* c, int32_t* labels,
                            float* dist2, float* inertia, int32_t* rep) {
     if (B == 0) return KB_OK;
+    const bool use_tc = N > 0 && ctx->assign_path != 1 &&
+                        (ctx->assign_path == 2 ? kb_assign_tc_supported(ctx, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
+    if (ctx->assign_path == 2 && N > 0 && !use_tc)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_assign: the tensor path needs D %% 32 == 0, D <= 128");
     double* ws_inertia = nullptr;
     unsigned long long* ws_rep = nullptr;
-    if (inertia || rep) {
-        if (ctx->ws_bytes < kb_ws_need_assign(B, N, D, K))
-            return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_cluster_assign needs %zu bytes of workspace",
-                           kb_ws_need_assign(B, N, D, K));
-        size_t off_rep = kb_align256((size_t)B * sizeof(double));
-        if (inertia) {
-            ws_inertia = reinterpret_cast<double*>(ctx->ws);
-            KB_MEMSET(ctx, ws_inertia, 0, (size_t)B * sizeof(double));
-        }
-        if (rep) {
-            ws_rep = reinterpret_cast<unsigned long long*>(ctx->ws + off_rep);
-            KB_MEMSET(ctx, ws_rep, 0xff, (size_t)B * K * sizeof(unsigned long long));
-        }
+    const size_t off_rep = kb_align256((size_t)B * sizeof(double));
+    const size_t off_tc = off_rep + kb_align256((size_t)B * K * sizeof(unsigned long long));
+    if (inertia || rep || use_tc) {
+        const size_t need = use_tc ? kb_ws_need_assign(B, N, D, K) : off_tc;
+        if (ctx->ws_bytes < need)
+            return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_cluster_assign needs %zu bytes of workspace", need);
     }
+    if (inertia) {
+        ws_inertia = reinterpret_cast<double*>(ctx->ws);
+        KB_MEMSET(ctx, ws_inertia, 0, (size_t)B * sizeof(double));
+    }
+    if (rep) {
+        ws_rep = reinterpret_cast<unsigned long long*>(ctx->ws + off_rep);
+        KB_MEMSET(ctx, ws_rep, 0xff, (size_t)B * K * sizeof(unsigned long long));
+    }
+    ctx->last_assign_path = 0;
     if (N > 0) {
-        // rows per block: as many as fit beside an 8-centroid tile in 96 KB, at most 128
-        const size_t budget = 96 * 1024;
-        int CT = (int)((16 * 1024) / ((size_t)D * 4));
-        CT = CT / AS_GROUP * AS_GROUP;
-        if (CT < AS_GROUP) CT = AS_GROUP;
-        if (CT > ((K + AS_GROUP - 1) / AS_GROUP) * AS_GROUP) CT = ((K + AS_GROUP - 1) / AS_GROUP) * AS_GROUP;
-        size_t cbytes = (size_t)CT * D * 4;
-        if (cbytes + (size_t)32 * (D + 1) * 4 > budget)
-            return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_assign: D = %d is beyond the row-wise path", D);
-        int TM = (int)((budget - cbytes) / ((size_t)(D + 1) * 4));
-        TM = TM >= 128 ? 128 : (TM / 32 * 32);
-        size_t smem = cbytes + (size_t)TM * (D + 1) * 4;
-        dim3 grid((N + TM - 1) / TM, B);
-        if (D % 4 == 0) {
-            KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<true>, smem);
-            assign_rowwise_kernel<true><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
-                                                                         ws_inertia, ws_rep);
+        kb_status s;
+        if (use_tc) {
+            s = kb_launch_assign_tc(ctx, ctx->ws + off_tc, B, N, D, K, z, c, labels, nullptr, nullptr, ctx->tc_eps);
+            if (s == KB_OK && (dist2 || inertia || rep))
+                s = kb_launch_assign_finish(ctx, B, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
+            ctx->last_assign_path = 2;
         } else {
-            KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<false>, smem);
-            assign_rowwise_kernel<false><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
-                                                                          ws_inertia, ws_rep);
+            s = launch_rowwise(ctx, B, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
+            ctx->last_assign_path = 1;
         }
-        KB_LAUNCH_CHECK(ctx, "assign_rowwise_kernel");
+        if (s != KB_OK) return s;
     }
     if (inertia || rep) {
         int total = B * (rep ? K : 1);

@@ -1,0 +1,639 @@
+// kb_cluster_assign, tensor-core path (sm_100a: tcgen05.mma kind::tf32, TMEM).
+//
+// The assignment argmin_j ||z - c_j||^2 = argmin_j (||c_j||^2 - 2 z.c_j) is a
+// dense contraction Z[N x D] . C^T[D x K] when N*K*D is large.  It runs on the
+// 5th-generation tensor cores as a 3xTF32 split product (hi.hi + hi.lo + lo.hi,
+// each operand split into two TF32 pieces by round-to-nearest), fp32 accumulate:
+//
+//   * A = a 128-row tile of Z, split hi/lo in registers and stored in TENSOR
+//     MEMORY (tcgen05.st); the MMA reads it from there (no shared-memory traffic
+//     for A, and the three products of a k-step reuse it).
+//   * B = 128 centroids x 32 features per stage, pre-split hi/lo by a small
+//     kernel into 128-byte-swizzled K-major panels, so a stage is one linear
+//     32 KB bulk copy (cp.async.bulk + mbarrier), 4-stage ring, re-read from L2
+//     by every CTA (no multicast of any kind).
+//   * accumulators: two 128 x 128 fp32 buffers in TMEM; the epilogue warps read
+//     one with tcgen05.ld while the MMA fills the other.
+//   * epilogue: score = ||c||^2 - 2 acc, running (best, second best, argbest) per
+//     row across all centroid tiles.  A row whose gap second-best is inside the
+//     error bound of the split product is queued and re-evaluated in the exact
+//     direct form by a fix-up kernel, so labels follow the fp32 direct-form
+//     distances wherever it matters.
+//
+// Roles in a 320-thread persistent CTA (one per SM):
+//   warps 0-3  A producers   (cp.async prefetch of the next Z tile -> split -> TMEM)
+//   warps 4-7  epilogue      (TMEM -> registers -> argmin)
+//   warp  8    MMA issuer    (one elected lane), owns the TMEM allocation
+//   warp  9    B loader      (one elected lane)
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all
+// roles drain, TMEM is released and the device status word reports a timeout.
+#include "kb_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128;            // rows per tile = TMEM lanes
+constexpr int BN = 128;            // centroids per accumulator buffer
+constexpr int KBF = 32;            // floats per k-block (one 128-byte swizzle row)
+constexpr int PANEL = BN * KBF * 4;      // 16 KB: one hi or lo panel
+constexpr int STAGE = 2 * PANEL;         // hi + lo
+constexpr int NSTAGE = 4;
+constexpr int TC_THREADS = 320;
+constexpr int TMEM_COLS = 512;
+constexpr int COL_ACC = 0;         // two accumulators: columns [0,128) and [128,256)
+constexpr int COL_A = 256;         // A hi at [256, 256+D), A lo at [256+D, 256+2D)
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int STATUS_TIMEOUT = 0x100;
+
+// ---- PTX helpers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit
+// or another role has already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 127u) == 127u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bar_sync_producers() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc], kind::tf32
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t to_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+
+#define TC_LD32(taddr, r)                                                                                  \
+    asm volatile(                                                                                          \
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                          \
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                          \
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"          \
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),  \
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),         \
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),       \
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),       \
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])                                                            \
+        : "r"(taddr)                                                                                       \
+        : "memory")
+
+// The loaded registers are only valid after tcgen05.wait::ld; naming them as read-write
+// operands of the wait keeps the compiler from consuming them earlier.
+#define TC_WAIT_LD(r)                                                                                      \
+    asm volatile("tcgen05.wait::ld.sync.aligned;"                                                          \
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),  \
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),         \
+          "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),       \
+          "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),       \
+          "+r"(r[29]), "+r"(r[30]), "+r"(r[31])                                                            \
+        :: "memory")
+
+#define TC_ST32(taddr, r)                                                                                  \
+    asm volatile(                                                                                          \
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                    \
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "                         \
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"                 \
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),         \
+          "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]),     \
+          "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]),  \
+          "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),  \
+          "r"(r[31])                                                                                       \
+        : "memory")
+
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                 // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return d;
+}
+// kind::tf32, fp32 accumulate, A and B K-major, M = 128, N = BN
+constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct TcParams {
+    int B, N, D, K, Kpad;
+    int tiles_per_inst, total_tiles;
+    int nxb;                       // Z staging buffers (1 or 2)
+    float eps;                     // near-tie bound, relative to ||z||^2 + ||c||^2
+    const float* z;
+    const unsigned char* bimg;     // [B][NT][NKB][STAGE]
+    const float* cnorm;            // [B][Kpad]
+    int32_t* labels;
+    float* approx;                 // optional: ||z||^2 + best score (expanded-form d^2), diagnostics
+    int* flag_count;               // rows queued for the exact re-evaluation
+    int32_t* flag_rows;            // flat row ids (b * N + k)
+    int* dev_status;
+};
+
+// ---- preparation: split centroids into swizzled hi/lo panels, squared norms ----------
+__global__ void __launch_bounds__(256)
+tc_prep_kernel(int K, int D, int Kpad, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
+               float* __restrict__ cnorm) {
+    const int b = blockIdx.y;
+    const int nkb = D / KBF, nt = Kpad / BN;
+    const int chunks = Kpad * (D / 4);           // 16-byte chunks of this instance
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < chunks; e += gridDim.x * blockDim.x) {
+        const int j = e / (D / 4), q = e - j * (D / 4);       // centroid, float4 index within the row
+        const int kb = q >> 3, c = q & 7;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < K) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + q);
+        const float f[4] = {v.x, v.y, v.z, v.w};
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            hi[i] = to_tf32(f[i]);
+            lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
+        }
+        const int tile = j / BN, r = j - tile * BN;
+        size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
+                     ((c ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < Kpad; j += gridDim.x * blockDim.x) {
+        float n = INFINITY;                      // padding centroids can never win
+        if (j < K) {
+            double s = 0.0;
+            const float* c = cent + ((size_t)b * K + j) * D;
+            for (int d = 0; d < D; ++d) s += (double)c[d] * (double)c[d];
+            n = (float)s;
+        }
+        cnorm[(size_t)b * Kpad + j] = n;
+    }
+}
+
+// ---- the contraction -------------------------------------------------------------------
+__global__ void __launch_bounds__(TC_THREADS, 1)
+assign_tc_kernel(const TcParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the swizzled panels
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int D = p.D, nkb = D / KBF, nt_count = p.Kpad / BN;
+    const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
+    unsigned char* st_base = smem;                                        // NSTAGE x STAGE
+    float* xs = reinterpret_cast<float*>(smem + NSTAGE * STAGE);          // nxb x [BM][D+4]
+    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // [Kpad]
+    float* xnorm = cn + p.Kpad;                                           // [2][BM]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(xnorm + 2 * BM);
+    // barrier indices
+    enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 4, ACC_FULL = A_EMPTY + 4,
+           ACC_EMPTY = ACC_FULL + 2, XN_FULL = ACC_EMPTY + 2, XN_EMPTY = XN_FULL + 2, NBAR = XN_EMPTY + 2 };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar0 = smem_u32(bars);
+    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(BAR(B_FULL + s), 1); mbar_init(BAR(B_EMPTY + s), 1); }
+        for (int k = 0; k < 4; ++k) { mbar_init(BAR(A_FULL + k), 128); mbar_init(BAR(A_EMPTY + k), 1); }
+        for (int k = 0; k < 2; ++k) {
+            mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 128);
+            mbar_init(BAR(XN_FULL + k), 128); mbar_init(BAR(XN_EMPTY + k), 128);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {   // TMEM allocation (whole warp), address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int first = blockIdx.x, stride = gridDim.x;
+    bool ok = true;
+
+    if (warp < 4) {
+        // ============================ A producers ====================================
+        const int row_in_tile = tid;                       // = TMEM lane
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int vpr = D >> 2;                            // float4 per row
+        auto prefetch = [&](int tile, int buf) {
+            const int b = tile / p.tiles_per_inst, r0 = (tile - b * p.tiles_per_inst) * BM;
+            const float* src = p.z + ((size_t)b * p.N + r0) * D;
+            const int rows = min(BM, p.N - r0);
+            float* dst = xs + (size_t)buf * BM * xs_stride;
+            for (int e = tid; e < BM * vpr; e += 128) {
+                const int r = e / vpr, q = e - r * vpr;
+                const bool valid = r < rows;
+                cp_async16(smem_u32(dst + (size_t)r * xs_stride + 4 * q), src + (size_t)(valid ? r : 0) * D + 4 * q,
+                           valid ? 16u : 0u);
+            }
+            cp_async_commit();
+        };
+        int it = 0;
+        if (first < p.total_tiles) prefetch(first, 0);
+        for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+            const int buf = p.nxb == 2 ? (it & 1) : 0;
+            const int next = tile + stride;
+            if (p.nxb == 2) {
+                if (next < p.total_tiles) { prefetch(next, buf ^ 1); cp_async_wait<1>(); }
+                else cp_async_wait<0>();
+            } else {
+                cp_async_wait<0>();
+            }
+            bar_sync_producers();                          // the staged tile is visible to all four warps
+            const float* xr = xs + (size_t)buf * BM * xs_stride + (size_t)row_in_tile * xs_stride;
+            float xn = 0.f;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                uint32_t hi[32], lo[32];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 v = *reinterpret_cast<const float4*>(xr + kb * KBF + 4 * q);
+                    const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        xn = fmaf(f[i], f[i], xn);
+                        hi[4 * q + i] = to_tf32(f[i]);
+                        lo[4 * q + i] = to_tf32(f[i] - __uint_as_float(hi[4 * q + i]));
+                    }
+                }
+                ok = mbar_wait(BAR(A_EMPTY + kb), (uint32_t)((it & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                TC_ST32(lane_addr + COL_A + kb * KBF, hi);
+                TC_ST32(lane_addr + COL_A + D + kb * KBF, lo);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(BAR(A_FULL + kb));
+            }
+            if (!ok) break;
+            if (p.nxb == 1) {
+                bar_sync_producers();                      // everyone has read the staging buffer
+                if (next < p.total_tiles) prefetch(next, 0);
+            }
+            ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
+            if (!ok) break;
+            xnorm[(it & 1) * BM + row_in_tile] = xn;
+            mbar_arrive(BAR(XN_FULL + (it & 1)));
+        }
+        cp_async_wait<0>();
+    } else if (warp < 8) {
+        // ============================ epilogue ========================================
+        const int row_in_tile = tid - 128;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp - 4) * 32) << 16);
+        // squared norms of this instance's centroids (reloaded when the instance changes)
+        int cn_inst = -1;
+        uint32_t q = 0;
+        int it = 0;
+        for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+            const int b = tile / p.tiles_per_inst, r0 = (tile - b * p.tiles_per_inst) * BM;
+            if (b != cn_inst) {
+                asm volatile("bar.sync 2, 128;" ::: "memory");     // nobody still reads the old norms
+                for (int j = row_in_tile; j < p.Kpad; j += 128) cn[j] = p.cnorm[(size_t)b * p.Kpad + j];
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                cn_inst = b;
+            }
+            float best = INFINITY, second = INFINITY;
+            int arg = 0;
+            for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
+                const uint32_t buf = q & 1u;
+                ok = mbar_wait(BAR(ACC_FULL + buf), (q >> 1) & 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t acc = lane_addr + COL_ACC + buf * BN;
+                uint32_t r[2][32];
+                TC_LD32(acc, r[0]);
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c) {
+                    TC_WAIT_LD(r[c & 1]);
+                    if (c + 1 < BN / 32) TC_LD32(acc + (c + 1) * 32, r[(c + 1) & 1]);
+                    const float* cnp = cn + nt * BN + c * 32;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 n4 = *reinterpret_cast<const float4*>(cnp + j);
+                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float s = fmaf(-2.f, __uint_as_float(r[c & 1][j + i]), nn[i]);
+                            second = fminf(second, fmaxf(best, s));
+                            if (s < best) { best = s; arg = nt * BN + c * 32 + j + i; }
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(BAR(ACC_EMPTY + buf));
+            }
+            if (!ok) break;
+            ok = mbar_wait(BAR(XN_FULL + (it & 1)), (uint32_t)((it >> 1) & 1), abort_flag);
+            if (!ok) break;
+            const float xn = xnorm[(it & 1) * BM + row_in_tile];
+            mbar_arrive(BAR(XN_EMPTY + (it & 1)));
+            const int row = r0 + row_in_tile;
+            if (row < p.N) {
+                const size_t flat = (size_t)b * p.N + row;
+                p.labels[flat] = arg;
+                if (p.approx) p.approx[flat] = xn + best;
+                if (second - best <= p.eps * (xn + cn[arg])) {
+                    const int slot = atomicAdd(p.flag_count, 1);
+                    p.flag_rows[slot] = (int32_t)flat;
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ============================ MMA issuer ======================================
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0, q = 0;
+            int it = 0;
+            for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+                for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
+                    const uint32_t buf = q & 1u;
+                    ok = mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
+                    for (int kb = 0; kb < nkb; ++kb) {
+                        if (nt == 0) {
+                            ok = mbar_wait(BAR(A_FULL + kb), (uint32_t)(it & 1), abort_flag);
+                            if (!ok) break;
+                        }
+                        ok = mbar_wait(BAR(B_FULL + s), ph, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t sb = smem_u32(st_base + (size_t)s * STAGE);
+#pragma unroll
+                        for (int k8 = 0; k8 < KBF / 8; ++k8) {
+                            const uint32_t a_hi = tmem + COL_A + kb * KBF + k8 * 8;
+                            const uint32_t a_lo = a_hi + D;
+                            const uint64_t b_hi = smem_desc_sw128(sb + k8 * 32);
+                            const uint64_t b_lo = smem_desc_sw128(sb + PANEL + k8 * 32);
+                            tc_mma_ts(d_tmem, a_lo, b_hi, IDESC, (kb | k8) != 0 ? 1u : 0u);
+                            tc_mma_ts(d_tmem, a_hi, b_lo, IDESC, 1u);
+                            tc_mma_ts(d_tmem, a_hi, b_hi, IDESC, 1u);
+                        }
+                        tc_commit(BAR(B_EMPTY + s));                       // stage reusable once these MMAs retire
+                        if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + kb));  // A panel reusable for the next tile
+                        if (++s == NSTAGE) { s = 0; ph ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit(BAR(ACC_FULL + buf));
+                }
+            }
+        }
+    } else {
+        // ============================ B loader ========================================
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            uint32_t issued = 0;
+            for (int tile = first; tile < p.total_tiles && ok; tile += stride) {
+                const int b = tile / p.tiles_per_inst;
+                const unsigned char* src = p.bimg + (size_t)b * nt_count * nkb * STAGE;
+                for (int i = 0; i < nt_count * nkb; ++i) {
+                    ok = mbar_wait(BAR(B_EMPTY + s), ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(BAR(B_FULL + s), STAGE);
+                    bulk_g2s(smem_u32(st_base + (size_t)s * STAGE), src + (size_t)i * STAGE, STAGE, BAR(B_FULL + s));
+                    ++issued;
+                    if (++s == NSTAGE) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // let copies that are still in flight land before the CTA's shared memory goes away
+                const uint32_t pending = issued < NSTAGE ? issued : NSTAGE;
+                for (uint32_t k = 0; k < pending; ++k) {
+                    const uint32_t idx = issued - 1 - k;
+                    const uint32_t st = idx % NSTAGE, par = (idx / NSTAGE) & 1u;
+                    for (uint32_t i = 0; i < WAIT_LIMIT && !mbar_try(BAR(B_FULL + st), par); ++i) {}
+                }
+            }
+        }
+    }
+
+    // ---- teardown: every role arrives here, on success or abort ----------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *abort_flag) atomicOr(p.dev_status, STATUS_TIMEOUT);
+}
+
+// ---- exact re-evaluation of queued rows (direct form, all K centroids) -----------------
+constexpr int FX_ROWS = 8;
+__global__ void __launch_bounds__(128)
+assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                    const int* __restrict__ flag_count, const int32_t* __restrict__ flag_rows,
+                    int32_t* __restrict__ labels) {
+    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows, then reduction scratch
+    float* xrow = fx;
+    float* red_v = fx + FX_ROWS * D;                       // [FX_ROWS][128]
+    int* red_i = reinterpret_cast<int*>(red_v + FX_ROWS * 128);
+    const int total = *flag_count;
+    const int tid = threadIdx.x;
+    for (int g0 = blockIdx.x * FX_ROWS; g0 < total; g0 += gridDim.x * FX_ROWS) {
+        const int nrow = min(FX_ROWS, total - g0);
+        __syncthreads();
+        for (int e = tid; e < nrow * D; e += 128) {
+            const int r = e / D, d = e - r * D;
+            xrow[r * D + d] = z[(size_t)flag_rows[g0 + r] * D + d];
+        }
+        __syncthreads();
+        float best[FX_ROWS];
+        int arg[FX_ROWS];
+#pragma unroll
+        for (int r = 0; r < FX_ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
+        // rows of one group may belong to different instances: evaluate per row's instance
+        for (int j = tid; j < K; j += 128) {
+#pragma unroll
+            for (int r = 0; r < FX_ROWS; ++r) {
+                if (r >= nrow) break;
+                const int b = flag_rows[g0 + r] / N;
+                const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D);
+                const float4* x4 = reinterpret_cast<const float4*>(xrow + r * D);
+                float acc = 0.f;
+                for (int d = 0; d < D / 4; ++d) {
+                    const float4 c = __ldg(c4 + d), x = x4[d];
+                    float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                    acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+                }
+                if (acc < best[r]) { best[r] = acc; arg[r] = j; }     // ascending j: lowest index on ties
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < FX_ROWS; ++r) { red_v[r * 128 + tid] = best[r]; red_i[r * 128 + tid] = arg[r]; }
+        __syncthreads();
+        if (tid < nrow) {
+            float bv = INFINITY;
+            int bi = 0x7fffffff;
+            for (int t = 0; t < 128; ++t) {
+                const float v = red_v[tid * 128 + t];
+                const int i = red_i[tid * 128 + t];
+                if (v < bv || (v == bv && i < bi)) { bv = v; bi = i; }
+            }
+            labels[flag_rows[g0 + tid]] = bi;
+        }
+    }
+}
+
+// ---- dist2 / inertia / representative from final labels (direct form) -------------------
+__global__ void __launch_bounds__(256)
+assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                     const int32_t* __restrict__ labels, float* __restrict__ dist2, double* __restrict__ ws_inertia,
+                     unsigned long long* __restrict__ ws_rep) {
+    const int b = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rows_per_block = (N + gridDim.x - 1) / gridDim.x;
+    const int r0 = blockIdx.x * rows_per_block, r1 = min(N, r0 + rows_per_block);
+    double local = 0.0;
+    for (int r = r0 + warp; r < r1; r += 8) {
+        const size_t flat = (size_t)b * N + r;
+        const int lab = labels[flat];
+        const float4* x4 = reinterpret_cast<const float4*>(z + flat * D);
+        const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + lab) * D);
+        float acc = 0.f;
+        for (int q = lane; q < D / 4; q += 32) {
+            const float4 x = __ldg(x4 + q), c = __ldg(c4 + q);
+            float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+            acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+        }
+        acc = kb_warp_sum(acc);
+        if (lane == 0) {
+            if (dist2) dist2[flat] = acc;
+            local += (double)acc;
+            if (ws_rep) {
+                unsigned long long key = ((unsigned long long)__float_as_uint(acc) << 32) | (unsigned)r;
+                atomicMin(&ws_rep[(size_t)b * K + lab], key);
+            }
+        }
+    }
+    if (ws_inertia && lane == 0 && local != 0.0) atomicAdd(&ws_inertia[b], local);
+}
+
+size_t tc_smem_bytes(int D, int Kpad, int nxb) {
+    size_t s = 1024;                                       // alignment slack
+    s += (size_t)NSTAGE * STAGE;
+    s += (size_t)nxb * BM * (D + 4) * 4;
+    s += (size_t)Kpad * 4 + 2 * BM * 4;
+    s += 32 * 8 + 16;                                      // barriers, TMEM slot, abort flag
+    return s;
+}
+
+}  // namespace
+
+// Scratch of the tensor path beyond the generic assign scratch:
+// B image | centroid norms | queue counter | queue
+size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
+    const size_t Kpad = (size_t)(K + BN - 1) / BN * BN;
+    return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 4);
+}
+
+// what the kernel can run at all
+bool kb_assign_tc_supported(const kb_ctx* ctx, int D, int K) {
+    if (D % KBF != 0 || D > 128 || K < 1 || K > 8192) return false;
+    const int Kpad = (K + BN - 1) / BN * BN;
+    return tc_smem_bytes(D, Kpad, 1) <= (size_t)ctx->max_smem_optin;
+}
+// what the automatic choice sends there: enough centroids to fill an accumulator tile
+// and enough rows for the contraction to outweigh the preparation and fix-up launches
+bool kb_assign_tc_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
+    return kb_assign_tc_supported(ctx, D, K) && K >= 128 && (long long)B * N >= 4096;
+}
+
+// Labels through the tensor path.  `ws` points at kb_ws_need_assign_tc bytes.  `approx`
+// (nullable) receives the expanded-form squared distance; `flagged` (nullable, device)
+// receives the number of rows that went through the exact re-evaluation.
+kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K, const float* z, const float* c,
+                              int32_t* labels, float* approx, int* flagged, float eps) {
+    const int Kpad = (K + BN - 1) / BN * BN;
+    unsigned char* bimg = reinterpret_cast<unsigned char*>(ws);
+    float* cnorm = reinterpret_cast<float*>(ws + kb_align256((size_t)B * Kpad * D * 8));
+    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
+    int32_t* flag_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(flag_count) + 256);
+    KB_MEMSET(ctx, flag_count, 0, 256);
+
+    const int chunks = Kpad * (D / 4);
+    int pgrid = (chunks + 255) / 256;
+    if (pgrid > 592) pgrid = 592;
+    tc_prep_kernel<<<dim3(pgrid, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm);
+    KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
+
+    TcParams p;
+    p.B = B; p.N = N; p.D = D; p.K = K; p.Kpad = Kpad;
+    p.tiles_per_inst = (N + BM - 1) / BM;
+    p.total_tiles = p.tiles_per_inst * B;
+    p.nxb = tc_smem_bytes(D, Kpad, 2) <= (size_t)ctx->max_smem_optin ? 2 : 1;
+    p.eps = eps;
+    p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.labels = labels; p.approx = approx;
+    p.flag_count = flag_count; p.flag_rows = flag_rows; p.dev_status = ctx->dev_status;
+    const size_t smem = tc_smem_bytes(D, Kpad, p.nxb);
+    KB_SMEM_OPTIN(ctx, assign_tc_kernel, smem);
+    const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
+    assign_tc_kernel<<<grid, TC_THREADS, smem, ctx->stream>>>(p);
+    KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
+
+    const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_ROWS * 128 * 8;
+    assign_fixup_kernel<<<2 * ctx->sm_count, 128, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, flag_rows, labels);
+    KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
+    if (flagged) {
+        KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    return KB_OK;
+}
+
+kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* c,
+                                  const int32_t* labels, float* dist2, double* ws_inertia,
+                                  unsigned long long* ws_rep) {
+    long want = (4L * ctx->sm_count + B - 1) / B;
+    long cap = ((long)N + 63) / 64;
+    int G = (int)(want > cap ? cap : want);
+    if (G < 1) G = 1;
+    assign_finish_kernel<<<dim3(G, B), 256, 0, ctx->stream>>>(N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
+    KB_LAUNCH_CHECK(ctx, "assign_finish_kernel");
+    return KB_OK;
+}

@@ -22,6 +22,10 @@ struct kb_ctx {
     cudaEvent_t* ev;      // 2 * KB_EV_PAIRS events
     int ev_used;          // pairs in use
     unsigned char* ev_class;
+    // assign path control: 0 = automatic, 1 = row-wise FFMA, 2 = tensor cores
+    int assign_path;
+    int last_assign_path;  // path the most recent kb_cluster_assign took (1 or 2; 0 = nothing ran)
+    float tc_eps;          // near-tie bound of the tensor path, relative to ||z||^2 + ||c||^2
     char err[256];
 };
 #define KB_EV_PAIRS 4096
@@ -61,6 +65,14 @@ kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...);
 // one call to the next.  kb_workspace_bytes is the largest of these needs.
 size_t kb_ws_need_normalize(int B, int N, int D);
 size_t kb_ws_need_assign(int B, int N, int D, int K);
+size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
+bool kb_assign_tc_supported(const kb_ctx* ctx, int D, int K);
+bool kb_assign_tc_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
+kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K, const float* z, const float* c,
+                              int32_t* labels, float* approx, int* flagged, float eps);
+kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* c,
+                                  const int32_t* labels, float* dist2, double* ws_inertia,
+                                  unsigned long long* ws_rep);
 size_t kb_ws_need_update(int B, int N, int D, int K);
 size_t kb_ws_need_score(int B, int N, int K, int S);
 #define KB_NORM_MAXG 1024

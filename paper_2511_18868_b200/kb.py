@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 # every symbol include/kb.h declares
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
-           "kb_timing_enable", "kb_timing_read",
+           "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
            "kb_bandit_step_host"]
@@ -88,6 +88,9 @@ def load_library() -> ctypes.CDLL:
     lib.kb_cluster_assign.argtypes = [_VP, i, i, i, i] + [_VP] * 6
     lib.kb_cluster_update.argtypes = [_VP, i, i, i, i] + [_VP] * 4
     lib.kb_score_select.argtypes = [_VP, i, i, i, i, ScoreParams] + [_VP] * 14
+    lib.kb_set_assign_options.argtypes = [_VP, i, f]
+    lib.kb_get_assign_path.argtypes = [_VP, ctypes.POINTER(i)]
+    lib.kb_assign_tc_probe.argtypes = [_VP, i, i, i, i] + [_VP] * 5
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
     lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
@@ -238,6 +241,21 @@ class KB:
                                              self._p(cl_pulls), self._p(cl_mean), self._p(cl_index),
                                              self._p(arm_index), self._p(best_arm), self._p(best_val),
                                              self._p(best_cluster_arm)), "kb_score_select")
+
+    def set_assign_options(self, path: int = 0, tc_eps: float = 0.0):
+        """path: 0 automatic, 1 fp32 row-wise kernel, 2 tensor-core kernel."""
+        self._check(self.lib.kb_set_assign_options(self.h, int(path), float(tc_eps)), "kb_set_assign_options")
+
+    def assign_path(self) -> int:
+        out = ctypes.c_int()
+        self._check(self.lib.kb_get_assign_path(self.h, ctypes.byref(out)), "kb_get_assign_path")
+        return out.value
+
+    def assign_tc_probe(self, z, centroids, labels, approx_dist2=None, flagged=None):
+        B, N, D = z.shape
+        K = centroids.shape[1]
+        self._check(self.lib.kb_assign_tc_probe(self.h, B, N, D, K, self._p(z), self._p(centroids), self._p(labels),
+                                                self._p(approx_dist2), self._p(flagged)), "kb_assign_tc_probe")
 
     # -- conveniences -------------------------------------------------------
     def init_centroids(self, z, rows, centroids):

@@ -362,3 +362,57 @@ def test_argument_errors(kbx):
     assert e.value.status == 3
     kbx.set_workspace(saved)
     assert kbx.device_status() == 0
+
+
+# ------------------------------------------------- tensor-core assign path
+TC_CASES = [(1, 4096, 32, 128), (1, 5000, 64, 256), (2, 3000, 128, 200), (1, 4097, 96, 1024), (3, 1111, 64, 130),
+            (1, 20000, 128, 1024)]
+
+
+@pytest.mark.parametrize("B,N,D,K", TC_CASES)
+def test_assign_tensor_path(kbx, B, N, D, K):
+    """kb_cluster_assign forced onto the tcgen05 kernel: same rules as the fp32 path."""
+    cfg = wl.scaled(wl.CONFIGS["large"], B=B, N=N, D=D, K=K, components=max(8, K // 2), S=2)
+    inp = wl.make_inputs(cfg, seed=N + K)
+    z, _, _ = oracle.normalize(inp["x"])
+    rng = np.random.default_rng(K)
+    c = z[:, rng.choice(N, K, replace=False)] + (0.02 * rng.standard_normal((B, K, D))).astype(np.float32)
+    c[:, K - 1] = c[:, 0]                       # exact duplicate: gap 0, resolved by the exact re-evaluation
+    ws(kbx, B, N, D, K, 1)
+    kbx.set_assign_options(path=2)
+    try:
+        labels, d2, inertia, rep = empty((B, N), torch.int32), empty((B, N)), empty((B,)), empty((B, K), torch.int32)
+        kbx.cluster_assign(dev(z), dev(c), labels, d2, inertia, rep)
+        assert kbx.assign_path() == 2
+        approx, flagged, lab2 = empty((B, N)), empty((1,), torch.int32), empty((B, N), torch.int32)
+        kbx.assign_tc_probe(dev(z), dev(c), lab2, approx, flagged)
+    finally:
+        kbx.set_assign_options(path=0)
+    assert kbx.device_status() == 0
+    ref = oracle.cluster_assign(z, c, want_margins=True)
+    got = host(labels)
+    ties = parity.labels_match(z, c, got, ref)
+    assert not np.any(got == K - 1)
+    assert np.array_equal(host(lab2), got)
+    same = got == ref["labels"]
+    parity.close(host(d2)[same], ref["dist2"][same], atol=1e-7, what="dist2")
+    parity.close(host(inertia), ref["inertia"], atol=1e-6, what="inertia")
+    parity.rep_match(host(rep), ref, ref["dist2"], ref["labels"])
+    # how far the ranked (expanded-form, 3xTF32) distance is from the exact one
+    xn = (z.astype(np.float64) ** 2).sum(-1)
+    cnn = (c.astype(np.float64) ** 2).sum(-1)
+    scale = xn + np.take_along_axis(cnn, ref["labels"].astype(np.int64), axis=1)
+    err = np.abs(host(approx).astype(np.float64) - ref["best"])[same] / scale[same]
+    frac = int(host(flagged)[0]) / (B * N)
+    print(f"[tc B={B} N={N} D={D} K={K}] near-ties={ties} flagged={frac:.5f} "
+          f"max |d2_ranked - d2_exact| / (|z|^2+|c|^2) = {err.max():.3e} (eps = {1 / 65536:.3e})")
+    assert err.max() < 0.25 / 65536               # the re-evaluation bound covers the ranking error with margin
+
+
+def test_step_uses_tensor_path_when_eligible(kbx):
+    cfg = wl.scaled(wl.CONFIGS["large"], N=8192 + 37, iters=2)
+    inp = wl.make_inputs(cfg)
+    got = run_step(kbx, cfg, inp)
+    assert kbx.assign_path() == 2
+    a_chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
+    parity.labels_match(got["z"], got["centroids"], got["labels"], a_chk)
