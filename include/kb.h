@@ -201,7 +201,8 @@ kb_status kb_get_assign_path(kb_ctx* ctx, int* out);
 /* Diagnostic for the tensor-core assign kernel: runs it on (z, centroids) and
  * returns, besides the labels, the expanded-form squared distance it ranked
  * by (approx_dist2 [B][N], nullable) and the number of rows that went through
- * the exact re-evaluation (flagged, one int32 in DEVICE memory, nullable).
+ * the exact re-evaluation (flagged, two int32 in DEVICE memory, nullable:
+ * rows compared against their runner-up, rows re-evaluated against all K).
  * Same workspace as kb_cluster_assign. */
 kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
                              const float* centroids, int32_t* labels, float* approx_dist2,

@@ -15,10 +15,12 @@
 //   * accumulators: two 128 x 128 fp32 buffers in TMEM; the epilogue warps read
 //     one with tcgen05.ld while the MMA fills the other.
 //   * epilogue: score = ||c||^2 - 2 acc, running (best, second best, argbest) per
-//     row across all centroid tiles.  A row whose gap second-best is inside the
-//     error bound of the split product is queued and re-evaluated in the exact
-//     direct form by a fix-up kernel, so labels follow the fp32 direct-form
-//     distances wherever it matters.
+//     row across all centroid tiles (plus the runner-up's index and the third
+//     smallest score).  A row whose runner-up lies inside the error bound of the
+//     split product is queued and decided in the exact direct form by a fix-up
+//     kernel (two candidates: a warp compares them; three or more: all K are
+//     re-evaluated), so labels follow the fp32 direct-form distances wherever it
+//     matters.
 //
 // Roles in a 320-thread persistent CTA (one per SM):
 //   warps 0-3  A producers   (cp.async prefetch of the next Z tile -> split -> TMEM)
@@ -170,8 +172,9 @@ struct TcParams {
     const float* cnorm;            // [B][Kpad]
     int32_t* labels;
     float* approx;                 // optional: ||z||^2 + best score (expanded-form d^2), diagnostics
-    int* flag_count;               // rows queued for the exact re-evaluation
-    int32_t* flag_rows;            // flat row ids (b * N + k)
+    int* flag_count;               // [0]: rows queued for a two-candidate check, [1]: for a full re-evaluation
+    int2* pair_rows;               // (flat row id b * N + k, runner-up centroid)
+    int32_t* full_rows;            // flat row ids
     int* dev_status;
 };
 
@@ -179,37 +182,33 @@ struct TcParams {
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(int K, int D, int Kpad, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
                float* __restrict__ cnorm) {
+    // one warp per centroid: lane q owns the 16-byte chunk q of the row (D <= 128)
     const int b = blockIdx.y;
     const int nkb = D / KBF, nt = Kpad / BN;
-    const int chunks = Kpad * (D / 4);           // 16-byte chunks of this instance
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < chunks; e += gridDim.x * blockDim.x) {
-        const int j = e / (D / 4), q = e - j * (D / 4);       // centroid, float4 index within the row
-        const int kb = q >> 3, c = q & 7;
+    const int lane = threadIdx.x & 31;
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (j >= Kpad) return;
+    double sq = 0.0;
+    if (lane < D / 4) {
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < K) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + q);
+        if (j < K) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + lane);
         const float f[4] = {v.x, v.y, v.z, v.w};
         uint32_t hi[4], lo[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             hi[i] = to_tf32(f[i]);
             lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
+            sq += (double)f[i] * (double)f[i];
         }
+        const int kb = lane >> 3, c = lane & 7;
         const int tile = j / BN, r = j - tile * BN;
-        size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
-                     ((c ^ (r & 7)) << 4);
+        const size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
+                           ((c ^ (r & 7)) << 4);
         *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
         *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
-    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < Kpad; j += gridDim.x * blockDim.x) {
-        float n = INFINITY;                      // padding centroids can never win
-        if (j < K) {
-            double s = 0.0;
-            const float* c = cent + ((size_t)b * K + j) * D;
-            for (int d = 0; d < D; ++d) s += (double)c[d] * (double)c[d];
-            n = (float)s;
-        }
-        cnorm[(size_t)b * Kpad + j] = n;
-    }
+    sq = kb_warp_sum(sq);
+    if (lane == 0) cnorm[(size_t)b * Kpad + j] = j < K ? (float)sq : INFINITY;   // padding can never win
 }
 
 // ---- the contraction -------------------------------------------------------------------
@@ -339,8 +338,8 @@ assign_tc_kernel(const TcParams p) {
                 asm volatile("bar.sync 2, 128;" ::: "memory");
                 cn_inst = b;
             }
-            float best = INFINITY, second = INFINITY;
-            int arg = 0;
+            float best = INFINITY, second = INFINITY, third = INFINITY;
+            int arg = 0, arg2 = 0;
             for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                 const uint32_t buf = q & 1u;
                 ok = mbar_wait(BAR(ACC_FULL + buf), (q >> 1) & 1u, abort_flag);
@@ -361,8 +360,14 @@ assign_tc_kernel(const TcParams p) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const float s = fmaf(-2.f, __uint_as_float(r[c & 1][j + i]), nn[i]);
+                            const int col = nt * BN + c * 32 + j + i;
+                            // running three smallest scores, indices of the two smallest
+                            third = fminf(third, fmaxf(second, s));
+                            const bool c1 = s < best, c2 = s < second;
+                            arg2 = c1 ? arg : (c2 ? col : arg2);
                             second = fminf(second, fmaxf(best, s));
-                            if (s < best) { best = s; arg = nt * BN + c * 32 + j + i; }
+                            arg = c1 ? col : arg;
+                            best = fminf(best, s);
                         }
                     }
                 }
@@ -379,9 +384,13 @@ assign_tc_kernel(const TcParams p) {
                 const size_t flat = (size_t)b * p.N + row;
                 p.labels[flat] = arg;
                 if (p.approx) p.approx[flat] = xn + best;
-                if (second - best <= p.eps * (xn + cn[arg])) {
+                const float delta = p.eps * (xn + cn[arg]);
+                if (third - best <= delta) {            // three or more candidates: exact scan over all centroids
+                    const int slot = atomicAdd(p.flag_count + 1, 1);
+                    p.full_rows[slot] = (int32_t)flat;
+                } else if (second - best <= delta) {    // two candidates: compare them exactly
                     const int slot = atomicAdd(p.flag_count, 1);
-                    p.flag_rows[slot] = (int32_t)flat;
+                    p.pair_rows[slot] = make_int2((int)flat, arg2);
                 }
             }
         }
@@ -464,46 +473,98 @@ assign_tc_kernel(const TcParams p) {
     if (tid == 0 && *abort_flag) atomicOr(p.dev_status, STATUS_TIMEOUT);
 }
 
-// ---- exact re-evaluation of queued rows (direct form, all K centroids) -----------------
+// ---- exact re-evaluation of queued rows (direct form) ------------------------------------
+// Two candidates: one warp per row compares the best and the runner-up of the ranking.
+__global__ void __launch_bounds__(256)
+assign_fixup_pair_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                         const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                         int32_t* __restrict__ labels) {
+    const int total = flag_count[0];
+    const int lane = threadIdx.x & 31;
+    const int wpb = blockDim.x >> 5;
+    for (int e = blockIdx.x * wpb + (threadIdx.x >> 5); e < total; e += gridDim.x * wpb) {
+        const int2 ent = pair_rows[e];
+        const size_t flat = (size_t)ent.x;
+        const int b = (int)(flat / N);
+        const int a1 = labels[flat], a2 = ent.y;
+        const float4* x4 = reinterpret_cast<const float4*>(z + flat * D);
+        const float4* c1 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + a1) * D);
+        const float4* c2 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + a2) * D);
+        float d1 = 0.f, d2 = 0.f;
+        for (int q = lane; q < D / 4; q += 32) {
+            const float4 x = __ldg(x4 + q), u = __ldg(c1 + q), v = __ldg(c2 + q);
+            float e0 = x.x - u.x, e1 = x.y - u.y, e2 = x.z - u.z, e3 = x.w - u.w;
+            d1 = fmaf(e0, e0, d1); d1 = fmaf(e1, e1, d1); d1 = fmaf(e2, e2, d1); d1 = fmaf(e3, e3, d1);
+            e0 = x.x - v.x; e1 = x.y - v.y; e2 = x.z - v.z; e3 = x.w - v.w;
+            d2 = fmaf(e0, e0, d2); d2 = fmaf(e1, e1, d2); d2 = fmaf(e2, e2, d2); d2 = fmaf(e3, e3, d2);
+        }
+        d1 = kb_warp_sum(d1);
+        d2 = kb_warp_sum(d2);
+        if (lane == 0 && (d2 < d1 || (d2 == d1 && a2 < a1))) labels[flat] = a2;
+    }
+}
+
+// Three or more candidates: all K centroids, eight queued rows share every centroid read.
 constexpr int FX_ROWS = 8;
 __global__ void __launch_bounds__(128)
-assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                    const int* __restrict__ flag_count, const int32_t* __restrict__ flag_rows,
-                    int32_t* __restrict__ labels) {
+assign_fixup_full_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                         const int* __restrict__ flag_count, const int32_t* __restrict__ full_rows,
+                         int32_t* __restrict__ labels) {
     extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows, then reduction scratch
     float* xrow = fx;
     float* red_v = fx + FX_ROWS * D;                       // [FX_ROWS][128]
     int* red_i = reinterpret_cast<int*>(red_v + FX_ROWS * 128);
-    const int total = *flag_count;
+    __shared__ int s_inst[FX_ROWS];
+    const int total = flag_count[1];
     const int tid = threadIdx.x;
     for (int g0 = blockIdx.x * FX_ROWS; g0 < total; g0 += gridDim.x * FX_ROWS) {
         const int nrow = min(FX_ROWS, total - g0);
         __syncthreads();
-        for (int e = tid; e < nrow * D; e += 128) {
+        for (int e = tid; e < FX_ROWS * D; e += 128) {
             const int r = e / D, d = e - r * D;
-            xrow[r * D + d] = z[(size_t)flag_rows[g0 + r] * D + d];
+            // rows past the end of the queue repeat the last one (their result is discarded)
+            xrow[e] = z[(size_t)full_rows[g0 + min(r, nrow - 1)] * D + d];
         }
+        if (tid < FX_ROWS) s_inst[tid] = full_rows[g0 + min(tid, nrow - 1)] / N;
         __syncthreads();
+        bool same_inst = true;
+        for (int r = 1; r < FX_ROWS; ++r) same_inst = same_inst && (s_inst[r] == s_inst[0]);
         float best[FX_ROWS];
         int arg[FX_ROWS];
 #pragma unroll
         for (int r = 0; r < FX_ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
-        // rows of one group may belong to different instances: evaluate per row's instance
         for (int j = tid; j < K; j += 128) {
+            float acc[FX_ROWS];
 #pragma unroll
-            for (int r = 0; r < FX_ROWS; ++r) {
-                if (r >= nrow) break;
-                const int b = flag_rows[g0 + r] / N;
-                const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D);
-                const float4* x4 = reinterpret_cast<const float4*>(xrow + r * D);
-                float acc = 0.f;
+            for (int r = 0; r < FX_ROWS; ++r) acc[r] = 0.f;
+            if (same_inst) {                               // the common case: one centroid read serves all rows
+                const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[0] * K + j) * D);
                 for (int d = 0; d < D / 4; ++d) {
-                    const float4 c = __ldg(c4 + d), x = x4[d];
-                    float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
-                    acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+                    const float4 c = __ldg(c4 + d);
+#pragma unroll
+                    for (int r = 0; r < FX_ROWS; ++r) {
+                        const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
+                        float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                        acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
+                        acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
+                    }
                 }
-                if (acc < best[r]) { best[r] = acc; arg[r] = j; }     // ascending j: lowest index on ties
+            } else {
+#pragma unroll
+                for (int r = 0; r < FX_ROWS; ++r) {
+                    const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[r] * K + j) * D);
+                    for (int d = 0; d < D / 4; ++d) {
+                        const float4 c = __ldg(c4 + d);
+                        const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
+                        float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                        acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
+                        acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
+                    }
+                }
             }
+#pragma unroll
+            for (int r = 0; r < FX_ROWS; ++r)
+                if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j; }   // ascending j: lowest index on ties
         }
 #pragma unroll
         for (int r = 0; r < FX_ROWS; ++r) { red_v[r * 128 + tid] = best[r]; red_i[r * 128 + tid] = arg[r]; }
@@ -516,7 +577,7 @@ assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const floa
                 const int i = red_i[tid * 128 + t];
                 if (v < bv || (v == bv && i < bi)) { bv = v; bi = i; }
             }
-            labels[flag_rows[g0 + tid]] = bi;
+            labels[full_rows[g0 + tid]] = bi;
         }
     }
 }
@@ -570,7 +631,8 @@ size_t tc_smem_bytes(int D, int Kpad, int nxb) {
 // B image | centroid norms | queue counter | queue
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
     const size_t Kpad = (size_t)(K + BN - 1) / BN * BN;
-    return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 4);
+    return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 8) +
+           kb_align256((size_t)B * N * 4);
 }
 
 // what the kernel can run at all
@@ -594,13 +656,11 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     unsigned char* bimg = reinterpret_cast<unsigned char*>(ws);
     float* cnorm = reinterpret_cast<float*>(ws + kb_align256((size_t)B * Kpad * D * 8));
     int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
-    int32_t* flag_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(flag_count) + 256);
+    int2* pair_rows = reinterpret_cast<int2*>(reinterpret_cast<char*>(flag_count) + 256);
+    int32_t* full_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(pair_rows) + kb_align256((size_t)B * N * 8));
     KB_MEMSET(ctx, flag_count, 0, 256);
 
-    const int chunks = Kpad * (D / 4);
-    int pgrid = (chunks + 255) / 256;
-    if (pgrid > 592) pgrid = 592;
-    tc_prep_kernel<<<dim3(pgrid, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm);
+    tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm);
     KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
 
     TcParams p;
@@ -610,7 +670,7 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     p.nxb = tc_smem_bytes(D, Kpad, 2) <= (size_t)ctx->max_smem_optin ? 2 : 1;
     p.eps = eps;
     p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.labels = labels; p.approx = approx;
-    p.flag_count = flag_count; p.flag_rows = flag_rows; p.dev_status = ctx->dev_status;
+    p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
     const size_t smem = tc_smem_bytes(D, Kpad, p.nxb);
     KB_SMEM_OPTIN(ctx, assign_tc_kernel, smem);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
@@ -618,10 +678,13 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
     const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_ROWS * 128 * 8;
-    assign_fixup_kernel<<<2 * ctx->sm_count, 128, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, flag_rows, labels);
-    KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
-    if (flagged) {
-        KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
+    assign_fixup_pair_kernel<<<2 * ctx->sm_count, 256, 0, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows, labels);
+    KB_LAUNCH_CHECK(ctx, "assign_fixup_pair_kernel");
+    assign_fixup_full_kernel<<<2 * ctx->sm_count, 128, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, full_rows,
+                                                                            labels);
+    KB_LAUNCH_CHECK(ctx, "assign_fixup_full_kernel");
+    if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
+        KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
     }
     return KB_OK;
 }
