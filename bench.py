@@ -36,6 +36,10 @@ METRIC = "arms scored/sec per bandit step"
 UNIT = "arms/s"
 DEFAULT_WORKLOAD = "large"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant call's main kernel, per launch, from the
+# ncu captures summarised under profiles/ (bytes; None where no capture exists for that workload)
+TRAFFIC_FROM_NCU = {}
+
 # rows of the workload the CPU oracle is timed on (per instance), and instances
 ORACLE_SAMPLE = {
     # name: (instances, rows) for the in-run cpu_baseline; the reference arm uses a quarter of the rows
@@ -139,52 +143,49 @@ def workload_config(cfg):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons through NVML (read-only) every 10 ms in a thread."""
+    REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
     def __init__(self, index: int):
-        self.index, self.proc, self.path = index, None, None
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop, self._thread = None, None
 
-    def start(self):
+    def _run(self):
+        import pynvml
         try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
-
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        try:
-            for line in open(self.path):
-                f = [v.strip() for v in line.split(",")]
-                if len(f) < 8:
-                    continue
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
                 try:
-                    sm.append(float(f[0])); mx.append(float(f[1]))
-                except ValueError:
-                    continue
-                for n, v in zip(names, f[4:8]):
-                    if v.lower().startswith("active"):
-                        reasons.add(n)
-            os.unlink(self.path)
+                    mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                self._stop.wait(0.01)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+
+    def start(self):
+        import threading
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        time.sleep(0.05)
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        if self._thread is None:
+            return out
+        self._stop.set()
+        self._thread.join(timeout=2)
+        if self.samples:
+            out.update(sm_mhz=float(np.median(self.samples)), sm_min_mhz=float(min(self.samples)),
+                       sm_max_mhz=self.max_mhz, samples=len(self.samples))
+        out["reasons"] = sorted(self.reasons)
         return out
 
 
@@ -244,6 +245,7 @@ def run_ours(args, cfg):
     per_class = ctx.timing_read()
     ctx.timing_enable(False)
     status = ctx.device_status()
+    assign_path = ctx.assign_path()
 
     # ---- end to end through the host-buffer entry point ----------------------------
     host_t = kb.step_tensors(inp, None, pinned_host=True)
@@ -297,7 +299,16 @@ def run_ours(args, cfg):
     dk = kernels[dominant]
     hbm_time = alg[dominant]["bytes"] / (hbm * 1e9)
     alu_time = alg[dominant]["flops"] / (ffma_tflops * 1e12)
-    if dominant == "assign" and alu_time > hbm_time:
+    tf32_peak = peaks["bf16_tflops"] * 0.5          # measured bf16 burst x nominal tf32/bf16 ratio
+    if dominant == "assign" and assign_path == 2:
+        # 3xTF32: three tensor-core products per fp32-equivalent product
+        roof = {"bound": "tensor", "achieved": dk["TFLOPs"], "peak": tf32_peak / 3.0, "unit": "TFLOP/s",
+                "frac": dk["TFLOPs"] / (tf32_peak / 3.0), "traffic": None,
+                "kernel": "kb_cluster_assign (tcgen05 kind::tf32, 3xTF32 split; prep + contraction + fix-up per call)",
+                "peak_source": f"{peaks['source']} bf16 GEMM peak x 0.5 (tf32) / 3 (split products), fp32-equivalent",
+                "algorithmic_flops_per_launch": alg["assign"]["flops"],
+                "executed_tensor_TFLOPs": 3.0 * dk["TFLOPs"]}
+    elif dominant == "assign" and alu_time > hbm_time:
         roof = {"bound": "alu", "achieved": dk["TFLOPs"], "peak": ffma_tflops, "unit": "TFLOP/s",
                 "frac": dk["TFLOPs"] / ffma_tflops, "traffic": None, "kernel": "kb_cluster_assign (fp32 FFMA path)",
                 "peak_source": "148 SM x 128 lanes x 2 flop x max SM clock",
@@ -306,6 +317,9 @@ def run_ours(args, cfg):
         roof = {"bound": "hbm", "achieved": dk["GBps"], "peak": hbm, "unit": "GB/s", "frac": dk["hbm_frac"],
                 "traffic": None, "kernel": f"kb_{dominant}", "peak_source": f"{peaks['source']} copy bandwidth",
                 "algorithmic_bytes_per_launch": alg[dominant]["bytes"]}
+    traffic = TRAFFIC_FROM_NCU.get((cfg.name, dominant))
+    if traffic is not None:
+        roof["traffic"] = traffic
 
     # ---- CPU oracle beside it (bounded sample) ----------------------------------------
     cpu = None
@@ -339,9 +353,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override N (rows per instance): a smaller case of the same kernels for ncu captures; "
+                         "numbers from such a run are not bench values")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = wl.CONFIGS[args.workload]
+    if args.rows > 0:
+        cfg = wl.scaled(cfg, N=args.rows)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

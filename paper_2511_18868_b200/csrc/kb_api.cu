@@ -246,7 +246,7 @@ kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const floa
     KB_COMMON(ctx, B, N);
     KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_assign_tc_probe: D and K must be >= 1");
     KB_REQUIRE(ctx, z && centroids && labels, "kb_assign_tc_probe: z, centroids and labels are required");
-    if (!kb_assign_tc_supported(ctx, D, K))
+    if (!kb_assign_tc_supported(ctx, B, D, K))
         return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_assign_tc_probe: needs D %% 32 == 0, D <= 128, K <= 8192");
     if (B == 0 || N == 0) return KB_OK;
     const size_t off = kb_ws_need_assign(B, N, D, K) - kb_ws_need_assign_tc(B, N, D, K);

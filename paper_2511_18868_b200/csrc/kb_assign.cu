@@ -167,7 +167,7 @@ kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float*
                            float* dist2, float* inertia, int32_t* rep) {
     if (B == 0) return KB_OK;
     const bool use_tc = N > 0 && ctx->assign_path != 1 &&
-                        (ctx->assign_path == 2 ? kb_assign_tc_supported(ctx, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
+                        (ctx->assign_path == 2 ? kb_assign_tc_supported(ctx, B, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
     if (ctx->assign_path == 2 && N > 0 && !use_tc)
         return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_assign: the tensor path needs D %% 32 == 0, D <= 128");
     double* ws_inertia = nullptr;

@@ -22,11 +22,11 @@
 //     re-evaluated), so labels follow the fp32 direct-form distances wherever it
 //     matters.
 //
-// Roles in a 320-thread persistent CTA (one per SM):
-//   warps 0-3  A producers   (cp.async prefetch of the next Z tile -> split -> TMEM)
-//   warps 4-7  epilogue      (TMEM -> registers -> argmin)
-//   warp  8    MMA issuer    (one elected lane), owns the TMEM allocation
-//   warp  9    B loader      (one elected lane)
+// Roles in a 448-thread persistent CTA (one per SM):
+//   warps 0-3   A producers  (cp.async prefetch of the next Z tile -> split -> TMEM)
+//   warps 4-11  epilogue     (TMEM -> registers -> argmin; two warps per lane quarter)
+//   warp  12    MMA issuer   (one elected lane), owns the TMEM allocation
+//   warp  13    B loader     (one elected lane)
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all
 // roles drain, TMEM is released and the device status word reports a timeout.
 #include "kb_internal.cuh"
@@ -39,10 +39,10 @@ constexpr int KBF = 32;            // floats per k-block (one 128-byte swizzle r
 constexpr int PANEL = BN * KBF * 4;      // 16 KB: one hi or lo panel
 constexpr int STAGE = 2 * PANEL;         // hi + lo
 constexpr int NSTAGE = 4;
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 448;
 constexpr int TMEM_COLS = 512;
 constexpr int COL_ACC = 0;         // two accumulators: columns [0,128) and [128,256)
-constexpr int COL_A = 256;         // A hi at [256, 256+D), A lo at [256+D, 256+2D)
+constexpr int COL_A = 256;         // A buffer i: hi at [256 + 2iD, +D), lo at [256 + 2iD + D, +D); two buffers when D <= 64
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int STATUS_TIMEOUT = 0x100;
 
@@ -108,6 +108,18 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// accumulate form (enable_input_d is the constant true predicate)
+__device__ __forceinline__ void tc_mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t mk_desc(uint32_t lo, uint32_t hi) {
+    return ((uint64_t)hi << 32) | (uint64_t)lo;
+}
 __device__ __forceinline__ uint32_t to_tf32(float v) {
     uint32_t r;
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
@@ -166,6 +178,7 @@ struct TcParams {
     int B, N, D, K, Kpad;
     int tiles_per_inst, total_tiles;
     int nxb;                       // Z staging buffers (1 or 2)
+    int resident;                  // 1: the whole B image of the (single) instance stays in the stage ring
     float eps;                     // near-tie bound, relative to ||z||^2 + ||c||^2
     const float* z;
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
@@ -181,7 +194,8 @@ struct TcParams {
 // ---- preparation: split centroids into swizzled hi/lo panels, squared norms ----------
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(int K, int D, int Kpad, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
-               float* __restrict__ cnorm) {
+               float* __restrict__ cnorm, int* __restrict__ flag_count) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
     // one warp per centroid: lane q owns the 16-byte chunk q of the row (D <= 128)
     const int b = blockIdx.y;
     const int nkb = D / KBF, nt = Kpad / BN;
@@ -212,20 +226,58 @@ tc_prep_kernel(int K, int D, int Kpad, const float* __restrict__ cent, unsigned 
 }
 
 // ---- the contraction -------------------------------------------------------------------
+// Running smallest scores of one row.  TRACK2 keeps the three smallest values and the
+// indices of the two smallest (so a near-tie can be settled by comparing two candidates);
+// without it only the two smallest values and the index of the smallest are kept and every
+// near-tie is re-evaluated against all centroids (cheaper per column; used when K*D is small).
+template <bool TRACK2>
+struct Tracker {
+    float b0 = INFINITY, b1 = INFINITY, b2 = INFINITY;
+    int a0 = 0, a1 = 0;
+    __device__ __forceinline__ void add(float s, int col) {
+        if (TRACK2) {
+            b2 = fminf(b2, fmaxf(b1, s));
+            const bool c1 = s < b0, c2 = s < b1;
+            a1 = c1 ? a0 : (c2 ? col : a1);
+        }
+        b1 = fminf(b1, fmaxf(b0, s));
+        a0 = s < b0 ? col : a0;
+        b0 = fminf(b0, s);
+    }
+    // fold another tracker over a disjoint set of columns into this one
+    __device__ __forceinline__ void merge(const Tracker& u) {
+        const float u2 = u.b2;
+        if (TRACK2) {
+            add(u.b0, u.a0);
+            add(u.b1, u.a1);
+            b2 = fminf(b2, fmaxf(b1, u2));
+        } else {
+            // values only: the second smallest of the union, the index of the smallest
+            const float lo = fminf(b0, u.b0), hi = fmaxf(b0, u.b0);
+            b1 = fminf(fminf(b1, u.b1), hi);
+            a0 = u.b0 < b0 ? u.a0 : a0;
+            b0 = lo;
+        }
+    }
+};
+
+template <bool TRACK2>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 assign_tc_kernel(const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled panels
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int D = p.D, nkb = D / KBF, nt_count = p.Kpad / BN;
+    const int nab = D <= 64 ? 2 : 1;                      // A (hi+lo) tiles that fit beside the accumulators in TMEM
     const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
     unsigned char* st_base = smem;                                        // NSTAGE x STAGE
     float* xs = reinterpret_cast<float*>(smem + NSTAGE * STAGE);          // nxb x [BM][D+4]
-    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // [Kpad]
-    float* xnorm = cn + p.Kpad;                                           // [2][BM]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(xnorm + 2 * BM);
+    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // [B][Kpad]
+    float* xnorm = cn + (size_t)p.B * p.Kpad;                             // [2][BM]
+    float* merge_buf = xnorm + 2 * BM;                                    // [2][BM][5]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(merge_buf + 2 * BM * 5 + 2);   // (+2 floats: 8-byte alignment)
     // barrier indices
-    enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 4, ACC_FULL = A_EMPTY + 4,
+    enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 8, ACC_FULL = A_EMPTY + 8,
            ACC_EMPTY = ACC_FULL + 2, XN_FULL = ACC_EMPTY + 2, XN_EMPTY = XN_FULL + 2, NBAR = XN_EMPTY + 2 };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -236,19 +288,20 @@ assign_tc_kernel(const TcParams p) {
 
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(BAR(B_FULL + s), 1); mbar_init(BAR(B_EMPTY + s), 1); }
-        for (int k = 0; k < 4; ++k) { mbar_init(BAR(A_FULL + k), 128); mbar_init(BAR(A_EMPTY + k), 1); }
+        for (int k = 0; k < 8; ++k) { mbar_init(BAR(A_FULL + k), 128); mbar_init(BAR(A_EMPTY + k), 1); }
         for (int k = 0; k < 2; ++k) {
-            mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 128);
+            mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 256);
             mbar_init(BAR(XN_FULL + k), 128); mbar_init(BAR(XN_EMPTY + k), 128);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8) {   // TMEM allocation (whole warp), address lands in shared memory
+    if (warp == 12) {  // TMEM allocation (whole warp), address lands in shared memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) cn[j] = p.cnorm[j];   // all instances' centroid norms
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -302,14 +355,15 @@ assign_tc_kernel(const TcParams p) {
                         lo[4 * q + i] = to_tf32(f[i] - __uint_as_float(hi[4 * q + i]));
                     }
                 }
-                ok = mbar_wait(BAR(A_EMPTY + kb), (uint32_t)((it & 1) ^ 1), abort_flag);
+                const int ab = it % nab, use = it / nab;       // A buffer of this tile, how often it was used before
+                ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                TC_ST32(lane_addr + COL_A + kb * KBF, hi);
-                TC_ST32(lane_addr + COL_A + D + kb * KBF, lo);
+                TC_ST32(lane_addr + COL_A + ab * 2 * D + kb * KBF, hi);
+                TC_ST32(lane_addr + COL_A + ab * 2 * D + D + kb * KBF, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
-                mbar_arrive(BAR(A_FULL + kb));
+                mbar_arrive(BAR(A_FULL + ab * 4 + kb));
             }
             if (!ok) break;
             if (p.nxb == 1) {
@@ -322,84 +376,102 @@ assign_tc_kernel(const TcParams p) {
             mbar_arrive(BAR(XN_FULL + (it & 1)));
         }
         cp_async_wait<0>();
-    } else if (warp < 8) {
+    } else if (warp < 12) {
         // ============================ epilogue ========================================
-        const int row_in_tile = tid - 128;
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp - 4) * 32) << 16);
-        // squared norms of this instance's centroids (reloaded when the instance changes)
-        int cn_inst = -1;
+        // Two warps per TMEM lane quarter: `half` 0 takes columns [0,64) of every accumulator
+        // buffer, `half` 1 columns [64,128).  Each thread keeps four independent trackers
+        // (columns modulo 4) so that the min/max chains of consecutive columns overlap.
+        const int ew = warp - 4, half = ew >> 2;
+        const int row_in_tile = (ew & 3) * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)((ew & 3) * 32) << 16);
         uint32_t q = 0;
         int it = 0;
         for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
             const int b = tile / p.tiles_per_inst, r0 = (tile - b * p.tiles_per_inst) * BM;
-            if (b != cn_inst) {
-                asm volatile("bar.sync 2, 128;" ::: "memory");     // nobody still reads the old norms
-                for (int j = row_in_tile; j < p.Kpad; j += 128) cn[j] = p.cnorm[(size_t)b * p.Kpad + j];
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                cn_inst = b;
-            }
-            float best = INFINITY, second = INFINITY, third = INFINITY;
-            int arg = 0, arg2 = 0;
+            const float* cnb = cn + (size_t)b * p.Kpad;            // squared norms of this instance's centroids
+            Tracker<TRACK2> t0, t1, t2, t3;
             for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                 const uint32_t buf = q & 1u;
                 ok = mbar_wait(BAR(ACC_FULL + buf), (q >> 1) & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t acc = lane_addr + COL_ACC + buf * BN;
+                const uint32_t acc = lane_addr + COL_ACC + buf * BN + half * (BN / 2);
                 uint32_t r[2][32];
                 TC_LD32(acc, r[0]);
 #pragma unroll
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = 0; c < BN / 64; ++c) {
                     TC_WAIT_LD(r[c & 1]);
-                    if (c + 1 < BN / 32) TC_LD32(acc + (c + 1) * 32, r[(c + 1) & 1]);
-                    const float* cnp = cn + nt * BN + c * 32;
+                    if (c + 1 < BN / 64) TC_LD32(acc + (c + 1) * 32, r[(c + 1) & 1]);
+                    const int col0 = nt * BN + half * (BN / 2) + c * 32;
+                    const float* cnp = cnb + col0;
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         const float4 n4 = *reinterpret_cast<const float4*>(cnp + j);
-                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float s = fmaf(-2.f, __uint_as_float(r[c & 1][j + i]), nn[i]);
-                            const int col = nt * BN + c * 32 + j + i;
-                            // running three smallest scores, indices of the two smallest
-                            third = fminf(third, fmaxf(second, s));
-                            const bool c1 = s < best, c2 = s < second;
-                            arg2 = c1 ? arg : (c2 ? col : arg2);
-                            second = fminf(second, fmaxf(best, s));
-                            arg = c1 ? col : arg;
-                            best = fminf(best, s);
-                        }
+                        t0.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 0]), n4.x), col0 + j + 0);
+                        t1.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 1]), n4.y), col0 + j + 1);
+                        t2.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 2]), n4.z), col0 + j + 2);
+                        t3.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 3]), n4.w), col0 + j + 3);
                     }
                 }
                 tc_fence_before();
                 mbar_arrive(BAR(ACC_EMPTY + buf));
             }
             if (!ok) break;
+            // every epilogue thread takes the same waits in the same order, so a timeout takes
+            // all of them out together and nobody is left at the named barrier below
             ok = mbar_wait(BAR(XN_FULL + (it & 1)), (uint32_t)((it >> 1) & 1), abort_flag);
             if (!ok) break;
+            t0.merge(t1);
+            t2.merge(t3);
+            t0.merge(t2);
+            // fold the upper half's tracker into the lower half's through shared memory
+            float* mg = merge_buf + ((size_t)(it & 1) * BM + row_in_tile) * 5;
+            if (half == 1) {
+                mg[0] = t0.b0; mg[1] = t0.b1; mg[2] = t0.b2;
+                mg[3] = __int_as_float(t0.a0); mg[4] = __int_as_float(t0.a1);
+            }
+            asm volatile("bar.sync 2, 256;" ::: "memory");
+            if (half == 1) continue;
+            {
+                Tracker<TRACK2> u;
+                u.b0 = mg[0]; u.b1 = mg[1]; u.b2 = mg[2];
+                u.a0 = __float_as_int(mg[3]); u.a1 = __float_as_int(mg[4]);
+                t0.merge(u);
+            }
             const float xn = xnorm[(it & 1) * BM + row_in_tile];
             mbar_arrive(BAR(XN_EMPTY + (it & 1)));
             const int row = r0 + row_in_tile;
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
-                p.labels[flat] = arg;
-                if (p.approx) p.approx[flat] = xn + best;
-                const float delta = p.eps * (xn + cn[arg]);
-                if (third - best <= delta) {            // three or more candidates: exact scan over all centroids
-                    const int slot = atomicAdd(p.flag_count + 1, 1);
-                    p.full_rows[slot] = (int32_t)flat;
-                } else if (second - best <= delta) {    // two candidates: compare them exactly
-                    const int slot = atomicAdd(p.flag_count, 1);
-                    p.pair_rows[slot] = make_int2((int)flat, arg2);
+                p.labels[flat] = t0.a0;
+                if (p.approx) p.approx[flat] = xn + t0.b0;
+                const float delta = p.eps * (xn + cnb[t0.a0]);
+                if (t0.b1 - t0.b0 <= delta) {
+                    if (TRACK2 && t0.b2 - t0.b0 > delta) {     // exactly two candidates: compare them exactly
+                        const int slot = atomicAdd(p.flag_count, 1);
+                        p.pair_rows[slot] = make_int2((int)flat, t0.a1);
+                    } else {                                   // three or more (or unknown): exact scan over all K
+                        const int slot = atomicAdd(p.flag_count + 1, 1);
+                        p.full_rows[slot] = (int32_t)flat;
+                    }
                 }
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == 12) {
         // ============================ MMA issuer ======================================
+        // A single lane issues every MMA, so its instruction stream is the critical path of the
+        // whole CTA: descriptors are formed with one add each (all k-steps unrolled) and nothing
+        // else happens between two tcgen05.mma.
         if (lane == 0) {
             uint32_t s = 0, ph = 0, q = 0;
             int it = 0;
+            const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
+            const uint32_t desc_hi32 = (uint32_t)(desc0 >> 32);
+            const uint32_t desc_lo32 = (uint32_t)desc0;
+            const int ring = p.resident ? nt_count * nkb : NSTAGE;
             for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+                const int ab = it % nab, use = it / nab;
+                const uint32_t a_base = tmem + COL_A + ab * 2 * D;
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
                     ok = mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag);
@@ -408,26 +480,29 @@ assign_tc_kernel(const TcParams p) {
                     const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
                     for (int kb = 0; kb < nkb; ++kb) {
                         if (nt == 0) {
-                            ok = mbar_wait(BAR(A_FULL + kb), (uint32_t)(it & 1), abort_flag);
+                            ok = mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag);
                             if (!ok) break;
                         }
-                        ok = mbar_wait(BAR(B_FULL + s), ph, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t sb = smem_u32(st_base + (size_t)s * STAGE);
-#pragma unroll
-                        for (int k8 = 0; k8 < KBF / 8; ++k8) {
-                            const uint32_t a_hi = tmem + COL_A + kb * KBF + k8 * 8;
-                            const uint32_t a_lo = a_hi + D;
-                            const uint64_t b_hi = smem_desc_sw128(sb + k8 * 32);
-                            const uint64_t b_lo = smem_desc_sw128(sb + PANEL + k8 * 32);
-                            tc_mma_ts(d_tmem, a_lo, b_hi, IDESC, (kb | k8) != 0 ? 1u : 0u);
-                            tc_mma_ts(d_tmem, a_hi, b_lo, IDESC, 1u);
-                            tc_mma_ts(d_tmem, a_hi, b_hi, IDESC, 1u);
+                        if (!p.resident || it == 0) {              // resident panels are loaded exactly once
+                            ok = mbar_wait(BAR(B_FULL + s), ph, abort_flag);
+                            if (!ok) break;
                         }
-                        tc_commit(BAR(B_EMPTY + s));                       // stage reusable once these MMAs retire
-                        if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + kb));  // A panel reusable for the next tile
-                        if (++s == NSTAGE) { s = 0; ph ^= 1u; }
+                        tc_fence_after();
+                        const uint32_t a_hi = a_base + kb * KBF, a_lo = a_hi + D;
+                        const uint32_t blo = desc_lo32 + s * (STAGE >> 4);        // this stage's hi panel
+                        // first k-step: the very first product of an accumulator tile overwrites it
+                        tc_mma_ts(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, kb != 0 ? 1u : 0u);
+                        tc_mma_ts_acc(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
+                        tc_mma_ts_acc(d_tmem, a_hi, mk_desc(blo, desc_hi32), IDESC);
+#pragma unroll
+                        for (int k8 = 1; k8 < KBF / 8; ++k8) {
+                            tc_mma_ts_acc(d_tmem, a_lo + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                            tc_mma_ts_acc(d_tmem, a_hi + k8 * 8, mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
+                            tc_mma_ts_acc(d_tmem, a_hi + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                        }
+                        if (!p.resident) tc_commit(BAR(B_EMPTY + s));      // stage reusable once these MMAs retire
+                        if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + ab * 4 + kb));  // A panel reusable
+                        if (++s == (uint32_t)ring) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
                     tc_commit(BAR(ACC_FULL + buf));
@@ -440,6 +515,7 @@ assign_tc_kernel(const TcParams p) {
             uint32_t s = 0, ph = 0;
             uint32_t issued = 0;
             for (int tile = first; tile < p.total_tiles && ok; tile += stride) {
+                if (p.resident && tile != first) break;            // one pass fills the ring for good
                 const int b = tile / p.tiles_per_inst;
                 const unsigned char* src = p.bimg + (size_t)b * nt_count * nkb * STAGE;
                 for (int i = 0; i < nt_count * nkb; ++i) {
@@ -466,7 +542,7 @@ assign_tc_kernel(const TcParams p) {
     // ---- teardown: every role arrives here, on success or abort ----------------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == 12) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
@@ -475,14 +551,14 @@ assign_tc_kernel(const TcParams p) {
 
 // ---- exact re-evaluation of queued rows (direct form) ------------------------------------
 // Two candidates: one warp per row compares the best and the runner-up of the ranking.
-__global__ void __launch_bounds__(256)
-assign_fixup_pair_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                         const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
-                         int32_t* __restrict__ labels) {
+// (Called by every block of the fix-up kernel; a label is touched by exactly one warp.)
+__device__ __forceinline__ void
+fixup_pairs(int nblocks, int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+            const int* __restrict__ flag_count, const int2* __restrict__ pair_rows, int32_t* __restrict__ labels) {
     const int total = flag_count[0];
     const int lane = threadIdx.x & 31;
     const int wpb = blockDim.x >> 5;
-    for (int e = blockIdx.x * wpb + (threadIdx.x >> 5); e < total; e += gridDim.x * wpb) {
+    for (int e = blockIdx.x * wpb + (threadIdx.x >> 5); e < total; e += nblocks * wpb) {
         const int2 ent = pair_rows[e];
         const size_t flat = (size_t)ent.x;
         const int b = (int)(flat / N);
@@ -504,62 +580,56 @@ assign_fixup_pair_kernel(int N, int D, int K, const float* __restrict__ z, const
     }
 }
 
-// Three or more candidates: all K centroids, eight queued rows share every centroid read.
+// One launch settles both queues: every block first takes its share of the two-candidate
+// rows, then of the rows that need all K centroids (eight queued rows share every centroid
+// read; thread = centroid, warp-shuffle argmin, lowest index on ties).
 constexpr int FX_ROWS = 8;
-__global__ void __launch_bounds__(128)
-assign_fixup_full_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                         const int* __restrict__ flag_count, const int32_t* __restrict__ full_rows,
-                         int32_t* __restrict__ labels) {
-    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows, then reduction scratch
-    float* xrow = fx;
-    float* red_v = fx + FX_ROWS * D;                       // [FX_ROWS][128]
-    int* red_i = reinterpret_cast<int*>(red_v + FX_ROWS * 128);
+constexpr int FX_T = 256;
+__global__ void __launch_bounds__(FX_T)
+assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                    const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
+    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows
+    __shared__ float red_v[FX_ROWS][FX_T / 32];
+    __shared__ int red_i[FX_ROWS][FX_T / 32];
     __shared__ int s_inst[FX_ROWS];
+    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
+    float* xrow = fx;
     const int total = flag_count[1];
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int g0 = blockIdx.x * FX_ROWS; g0 < total; g0 += gridDim.x * FX_ROWS) {
         const int nrow = min(FX_ROWS, total - g0);
         __syncthreads();
-        for (int e = tid; e < FX_ROWS * D; e += 128) {
-            const int r = e / D, d = e - r * D;
+        for (int e = tid; e < FX_ROWS * (D / 4); e += FX_T) {
+            const int r = e / (D / 4), q = e - r * (D / 4);
             // rows past the end of the queue repeat the last one (their result is discarded)
-            xrow[e] = z[(size_t)full_rows[g0 + min(r, nrow - 1)] * D + d];
+            reinterpret_cast<float4*>(xrow)[e] =
+                __ldg(reinterpret_cast<const float4*>(z + (size_t)full_rows[g0 + min(r, nrow - 1)] * D) + q);
         }
         if (tid < FX_ROWS) s_inst[tid] = full_rows[g0 + min(tid, nrow - 1)] / N;
         __syncthreads();
-        bool same_inst = true;
-        for (int r = 1; r < FX_ROWS; ++r) same_inst = same_inst && (s_inst[r] == s_inst[0]);
         float best[FX_ROWS];
         int arg[FX_ROWS];
 #pragma unroll
         for (int r = 0; r < FX_ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
-        for (int j = tid; j < K; j += 128) {
+        for (int j = tid; j < K; j += FX_T) {
             float acc[FX_ROWS];
 #pragma unroll
             for (int r = 0; r < FX_ROWS; ++r) acc[r] = 0.f;
-            if (same_inst) {                               // the common case: one centroid read serves all rows
-                const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[0] * K + j) * D);
-                for (int d = 0; d < D / 4; ++d) {
-                    const float4 c = __ldg(c4 + d);
-#pragma unroll
-                    for (int r = 0; r < FX_ROWS; ++r) {
-                        const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
-                        float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
-                        acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
-                        acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
-                    }
-                }
-            } else {
+            // rows of one group nearly always share an instance; when they do not, each row reads its own
+            const float4* c0 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[0] * K + j) * D);
+#pragma unroll 4
+            for (int d = 0; d < D / 4; ++d) {
+                const float4 c = __ldg(c0 + d);
 #pragma unroll
                 for (int r = 0; r < FX_ROWS; ++r) {
-                    const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[r] * K + j) * D);
-                    for (int d = 0; d < D / 4; ++d) {
-                        const float4 c = __ldg(c4 + d);
-                        const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
-                        float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
-                        acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
-                        acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
-                    }
+                    float4 cr = c;
+                    if (s_inst[r] != s_inst[0])
+                        cr = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)s_inst[r] * K + j) * D) + d);
+                    const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
+                    float e0 = x.x - cr.x, e1 = x.y - cr.y, e2 = x.z - cr.z, e3 = x.w - cr.w;
+                    acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
+                    acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
                 }
             }
 #pragma unroll
@@ -567,14 +637,24 @@ assign_fixup_full_kernel(int N, int D, int K, const float* __restrict__ z, const
                 if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j; }   // ascending j: lowest index on ties
         }
 #pragma unroll
-        for (int r = 0; r < FX_ROWS; ++r) { red_v[r * 128 + tid] = best[r]; red_i[r * 128 + tid] = arg[r]; }
+        for (int r = 0; r < FX_ROWS; ++r) {
+            float v = best[r];
+            int i = arg[r];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+                if (ov < v || (ov == v && oi < i)) { v = ov; i = oi; }
+            }
+            if (lane == 0) { red_v[r][warp] = v; red_i[r][warp] = i; }
+        }
         __syncthreads();
         if (tid < nrow) {
             float bv = INFINITY;
             int bi = 0x7fffffff;
-            for (int t = 0; t < 128; ++t) {
-                const float v = red_v[tid * 128 + t];
-                const int i = red_i[tid * 128 + t];
+            for (int w = 0; w < FX_T / 32; ++w) {
+                const float v = red_v[tid][w];
+                const int i = red_i[tid][w];
                 if (v < bv || (v == bv && i < bi)) { bv = v; bi = i; }
             }
             labels[full_rows[g0 + tid]] = bi;
@@ -616,12 +696,12 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
     if (ws_inertia && lane == 0 && local != 0.0) atomicAdd(&ws_inertia[b], local);
 }
 
-size_t tc_smem_bytes(int D, int Kpad, int nxb) {
+size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb) {
     size_t s = 1024;                                       // alignment slack
     s += (size_t)NSTAGE * STAGE;
     s += (size_t)nxb * BM * (D + 4) * 4;
-    s += (size_t)Kpad * 4 + 2 * BM * 4;
-    s += 32 * 8 + 16;                                      // barriers, TMEM slot, abort flag
+    s += (size_t)Kpad * 4 + 2 * BM * 4 + (2 * BM * 5 + 2) * 4;
+    s += 40 * 8 + 16;                                      // barriers, TMEM slot, abort flag
     return s;
 }
 
@@ -636,15 +716,16 @@ size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
 }
 
 // what the kernel can run at all
-bool kb_assign_tc_supported(const kb_ctx* ctx, int D, int K) {
-    if (D % KBF != 0 || D > 128 || K < 1 || K > 8192) return false;
-    const int Kpad = (K + BN - 1) / BN * BN;
-    return tc_smem_bytes(D, Kpad, 1) <= (size_t)ctx->max_smem_optin;
+bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K) {
+    if (D % KBF != 0 || D > 128 || K < 1 || K > 8192 || B < 1) return false;
+    const long Kpad = (long)(K + BN - 1) / BN * BN;
+    if (Kpad * B > 8192) return false;                     // the norms of every instance stay in shared memory
+    return tc_smem_bytes(D, (int)(Kpad * B), 1) <= (size_t)ctx->max_smem_optin;
 }
 // what the automatic choice sends there: enough centroids to fill an accumulator tile
 // and enough rows for the contraction to outweigh the preparation and fix-up launches
 bool kb_assign_tc_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
-    return kb_assign_tc_supported(ctx, D, K) && K >= 128 && (long long)B * N >= 4096;
+    return kb_assign_tc_supported(ctx, B, D, K) && K >= 128 && (long long)B * N >= 4096;
 }
 
 // Labels through the tensor path.  `ws` points at kb_ws_need_assign_tc bytes.  `approx`
@@ -658,31 +739,36 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
     int2* pair_rows = reinterpret_cast<int2*>(reinterpret_cast<char*>(flag_count) + 256);
     int32_t* full_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(pair_rows) + kb_align256((size_t)B * N * 8));
-    KB_MEMSET(ctx, flag_count, 0, 256);
 
-    tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm);
+    tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm, flag_count);
     KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
 
     TcParams p;
     p.B = B; p.N = N; p.D = D; p.K = K; p.Kpad = Kpad;
     p.tiles_per_inst = (N + BM - 1) / BM;
     p.total_tiles = p.tiles_per_inst * B;
-    p.nxb = tc_smem_bytes(D, Kpad, 2) <= (size_t)ctx->max_smem_optin ? 2 : 1;
+    p.nxb = tc_smem_bytes(D, Kpad * B, 2) <= (size_t)ctx->max_smem_optin ? 2 : 1;
     p.eps = eps;
+    p.resident = (B == 1 && (Kpad / BN) * (D / KBF) <= NSTAGE) ? 1 : 0;
     p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.labels = labels; p.approx = approx;
     p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
-    const size_t smem = tc_smem_bytes(D, Kpad, p.nxb);
-    KB_SMEM_OPTIN(ctx, assign_tc_kernel, smem);
+    const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
-    assign_tc_kernel<<<grid, TC_THREADS, smem, ctx->stream>>>(p);
+    // with few features per row the epilogue's per-column cost is what limits the kernel:
+    // track less there and let the (cheap, K*D is small) full re-evaluation settle near-ties
+    if (D >= 96) {
+        KB_SMEM_OPTIN(ctx, assign_tc_kernel<true>, smem);
+        assign_tc_kernel<true><<<grid, TC_THREADS, smem, ctx->stream>>>(p);
+    } else {
+        KB_SMEM_OPTIN(ctx, assign_tc_kernel<false>, smem);
+        assign_tc_kernel<false><<<grid, TC_THREADS, smem, ctx->stream>>>(p);
+    }
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
-    const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_ROWS * 128 * 8;
-    assign_fixup_pair_kernel<<<2 * ctx->sm_count, 256, 0, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows, labels);
-    KB_LAUNCH_CHECK(ctx, "assign_fixup_pair_kernel");
-    assign_fixup_full_kernel<<<2 * ctx->sm_count, 128, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, full_rows,
-                                                                            labels);
-    KB_LAUNCH_CHECK(ctx, "assign_fixup_full_kernel");
+    const size_t fsmem = (size_t)FX_ROWS * D * 4;
+    assign_fixup_kernel<<<2 * ctx->sm_count, FX_T, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows,
+                                                                        full_rows, labels);
+    KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
         KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
     }

@@ -66,7 +66,7 @@ kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...);
 size_t kb_ws_need_normalize(int B, int N, int D);
 size_t kb_ws_need_assign(int B, int N, int D, int K);
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
-bool kb_assign_tc_supported(const kb_ctx* ctx, int D, int K);
+bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K);
 bool kb_assign_tc_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
 kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K, const float* z, const float* c,
                               int32_t* labels, float* approx, int* flagged, float eps);
