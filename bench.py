@@ -141,6 +141,27 @@ def workload_config(cfg):
             "l2": "flushed between timed steps (256 MiB write)"}
 
 
+# ------------------------------------------------------------------ replicas (N > 1)
+def replica_seed(cfg, rank: int) -> int:
+    """Every rank runs an independent replica of the workload on its own batch."""
+    return cfg.seed + rank
+
+
+def reduce_max(values, dist, device):
+    """Max over ranks of a list of floats (the slowest replica defines the job's time)."""
+    import torch
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_value(world: int, arms: int, ms_per_step: float) -> float:
+    """Whole-job throughput: arms scored by all replicas per second."""
+    return world * arms / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) every 10 ms in a thread."""
@@ -205,7 +226,7 @@ def run_ours(args, cfg):
     device = torch.device("cuda", local)
     peaks = load_peaks()
 
-    inp = wl.make_inputs(cfg, seed=cfg.seed + rank)   # every replica draws its own batch
+    inp = wl.make_inputs(cfg, seed=replica_seed(cfg, rank))
     ctx = kb.KB(local)
     R = wl.R_RESOURCES
     dims = dict(B=cfg.B, N=cfg.N, D=cfg.D, K=cfg.K, S=cfg.S, R=R, iters=cfg.iters)
@@ -269,18 +290,15 @@ def run_ours(args, cfg):
     e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
 
     # ---- max over ranks -----------------------------------------------------------
-    if dist is not None:
-        tt = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(tt[0]), float(tt[1])
+    total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], dist, device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     ms_per_step = total_ms / args.steps
-    value = world * cfg.arms / (ms_per_step * 1e-3)
-    e2e_value = world * cfg.arms / (e2e_ms / e2e_steps * 1e-3)
+    value = job_value(world, cfg.arms, ms_per_step)
+    e2e_value = job_value(world, cfg.arms, e2e_ms / e2e_steps)
 
     # ---- per-call rooflines ---------------------------------------------------------
     alg = algorithmic(cfg)
