@@ -667,33 +667,59 @@ __global__ void __launch_bounds__(256)
 assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                      const int32_t* __restrict__ labels, float* __restrict__ dist2, double* __restrict__ ws_inertia,
                      unsigned long long* __restrict__ ws_rep) {
+    // lanes of a warp cover the float4 columns of a row; when a row needs fewer than 32 lanes several
+    // rows share a warp step, and four steps are in flight per lane
     const int b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int vpr = D >> 2;                                      // float4 per row
+    const int lpr = vpr >= 32 ? 32 : (32 % vpr == 0 ? vpr : 32); // lanes per row
+    const int rpw = 32 / lpr;                                    // rows per warp step
+    const int lane_c = lane % lpr, lane_r = lane / lpr;
     const int rows_per_block = (N + gridDim.x - 1) / gridDim.x;
     const int r0 = blockIdx.x * rows_per_block, r1 = min(N, r0 + rows_per_block);
+    constexpr int U = 4;
     double local = 0.0;
-    for (int r = r0 + warp; r < r1; r += 8) {
-        const size_t flat = (size_t)b * N + r;
-        const int lab = labels[flat];
-        const float4* x4 = reinterpret_cast<const float4*>(z + flat * D);
-        const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + lab) * D);
-        float acc = 0.f;
-        for (int q = lane; q < D / 4; q += 32) {
-            const float4 x = __ldg(x4 + q), c = __ldg(c4 + q);
-            float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
-            acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+    const int step = 8 * rpw;                                    // rows per block step
+    const int trips = (max(r1 - r0, 0) + U * step - 1) / (U * step);
+    for (int it = 0; it < trips; ++it) {
+        const int rb = r0 + it * U * step + warp * rpw + lane_r;
+        int lab[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) lab[u] = __ldg(labels + (size_t)b * N + min(rb + u * step, r1 - 1));
+        float acc[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t flat = (size_t)b * N + min(rb + u * step, r1 - 1);
+            const float4* x4 = reinterpret_cast<const float4*>(z + flat * D);
+            const float4* c4 = reinterpret_cast<const float4*>(cent + ((size_t)b * K + lab[u]) * D);
+            float a = 0.f;
+            for (int q = lane_c; q < vpr; q += lpr) {
+                const float4 x = __ldg(x4 + q), c = __ldg(c4 + q);
+                float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                a = fmaf(e0, e0, a); a = fmaf(e1, e1, a); a = fmaf(e2, e2, a); a = fmaf(e3, e3, a);
+            }
+            acc[u] = a;
         }
-        acc = kb_warp_sum(acc);
-        if (lane == 0) {
-            if (dist2) dist2[flat] = acc;
-            local += (double)acc;
-            if (ws_rep) {
-                unsigned long long key = ((unsigned long long)__float_as_uint(acc) << 32) | (unsigned)r;
-                atomicMin(&ws_rep[(size_t)b * K + lab], key);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float a = acc[u];
+            for (int o = 1; o < lpr; o <<= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            const int r = rb + u * step;
+            if (lane_c == 0 && r < r1) {
+                const size_t flat = (size_t)b * N + r;
+                if (dist2) dist2[flat] = a;
+                local += (double)a;
+                if (ws_rep) {
+                    unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned)r;
+                    atomicMin(&ws_rep[(size_t)b * K + lab[u]], key);
+                }
             }
         }
     }
-    if (ws_inertia && lane == 0 && local != 0.0) atomicAdd(&ws_inertia[b], local);
+    if (ws_inertia) {
+        local = kb_warp_sum(local);
+        if (lane == 0 && local != 0.0) atomicAdd(&ws_inertia[b], local);
+    }
 }
 
 size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb) {

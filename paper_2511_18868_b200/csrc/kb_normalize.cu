@@ -61,18 +61,27 @@ norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, doubl
     if (active) {
         float shift[V];
         ld<V>(xb + (size_t)cq * V, shift);  // first row of the instance: same pivot in every block
-        int r = r0 + rl;
-        while (r < r1) {
+        for (int rb = r0 + rl; rb < r1; rb += 8 * g.rl) {
+            // eight independent loads in flight, a short fp32 run over them, then widen
+            float v[8][V];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int r = rb + u * g.rl;
+                if (r < r1) {
+                    ld<V>(xb + (size_t)r * D + (size_t)cq * V, v[u]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < V; ++i) v[u][i] = shift[i];   // contributes exactly zero
+                }
+            }
             float f1[V], f2[V];
 #pragma unroll
             for (int i = 0; i < V; ++i) { f1[i] = 0.f; f2[i] = 0.f; }
-#pragma unroll 4
-            for (int u = 0; u < 8 && r < r1; ++u, r += g.rl) {  // short fp32 run, then widen
-                float v[V];
-                ld<V>(xb + (size_t)r * D + (size_t)cq * V, v);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
 #pragma unroll
                 for (int i = 0; i < V; ++i) {
-                    float e = v[i] - shift[i];
+                    float e = v[u][i] - shift[i];
                     f1[i] += e;
                     f2[i] = fmaf(e, e, f2[i]);
                 }

@@ -11,6 +11,12 @@
 // A second small kernel divides by the counts; empty clusters keep their centroid.
 // The fp32 sums depend on the order in which runs are flushed (last-bit
 // run-to-run differences); counts never do.
+//
+// When the whole K x D table of sums fits in shared memory (K*D <= 24K floats) a simpler path
+// runs instead: each CTA accumulates its rows straight into a shared-memory table (shared
+// atomics, rows of a warp hit different banks), writes the table out as a plain per-CTA
+// partial, and the finalize kernel adds the partials in CTA order.  No global atomics, no
+// memset, and the only run-to-run variation is the order of shared-memory adds inside a CTA.
 #include "kb_internal.cuh"
 
 namespace {
@@ -88,79 +94,175 @@ update_sorted_kernel(int N, int D, int K, int G, int CH, const float* __restrict
     __syncthreads();
     const int sorted = offs[K];                                 // rows with a valid label
 
-    // 2. chunks of the sorted order, one label run at a time
+    // 2. Each lane group (LPR lanes = the float4 columns of one row; RPW groups per warp) takes a
+    //    contiguous piece of the sorted order.  It keeps U row loads in flight regardless of where
+    //    label runs end, adds the rows up in registers and flushes with one vector reduction per
+    //    lane whenever the label changes.  No warp-collective operation inside a piece.
     const int LPR = (D / V) < 32 ? (D / V) : 32;                // lanes per row
-    const int RPW = (32 % LPR == 0) ? 32 / LPR : 1;             // rows in flight per warp step
+    const int RPW = (32 % LPR == 0) ? 32 / LPR : 1;             // lane groups per warp
     const int lane_c = lane % LPR, lane_r = lane / LPR;
     const bool lane_on = lane_r < RPW;
     const float* zb = z + ((size_t)b * N + r0) * D;
     float* gs = g_sums + (size_t)b * K * D;
-    const int nchunks = (sorted + CH - 1) / CH;
+    const int npieces = (sorted + CH - 1) / CH;
+    const int ngrabs = (npieces + RPW - 1) / RPW;
+    constexpr int U = 8;
     for (;;) {
-        int chunk = 0;
-        if (lane == 0) chunk = atomicAdd(&s_next, 1);
-        chunk = __shfl_sync(0xffffffffu, chunk, 0);
-        if (chunk >= nchunks) break;
-        const int p0 = chunk * CH, p1 = min(sorted, p0 + CH);
-        // first label of the chunk: the last j with offs[j] <= p0
+        int grab = 0;
+        if (lane == 0) grab = atomicAdd(&s_next, 1);
+        grab = __shfl_sync(0xffffffffu, grab, 0);
+        if (grab >= ngrabs) break;
+        const int piece = grab * RPW + lane_r;
+        if (!lane_on || piece >= npieces) continue;
+        const int p0 = piece * CH, p1 = min(sorted, p0 + CH);
+        // label of the first position: the last j with offs[j] <= p0
         int lo = 0, hi = K - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
             if (offs[mid] <= p0) lo = mid; else hi = mid - 1;
         }
-        int j = lo, p = p0;
-        while (p < p1) {
-            while (offs[j + 1] <= p) ++j;                        // skip empty labels
-            const int pe = min(p1, offs[j + 1]);
-            for (int cc = lane_c * V; cc < D; cc += 32 * V) {    // column chunks (one pass unless D > 32 V)
-                float a[V];
+        for (int cc = lane_c * V; cc < D; cc += 32 * V) {       // column chunks (one pass unless D > 32 V)
+            int j = lo, jend = offs[lo + 1];
+            float a[V];
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] = 0.f;
-                if (lane_on) {
-                    int q = p + lane_r;
-#pragma unroll 1
-                    for (; q + 3 * RPW < pe; q += 4 * RPW) {     // four independent rows in flight per lane
-                        const float* s0 = zb + (size_t)perm[q] * D + cc;
-                        const float* s1 = zb + (size_t)perm[q + RPW] * D + cc;
-                        const float* s2 = zb + (size_t)perm[q + 2 * RPW] * D + cc;
-                        const float* s3 = zb + (size_t)perm[q + 3 * RPW] * D + cc;
-                        if (V == 4) {
-                            const float4 v0 = __ldg(reinterpret_cast<const float4*>(s0));
-                            const float4 v1 = __ldg(reinterpret_cast<const float4*>(s1));
-                            const float4 v2 = __ldg(reinterpret_cast<const float4*>(s2));
-                            const float4 v3 = __ldg(reinterpret_cast<const float4*>(s3));
-                            a[0] += (v0.x + v1.x) + (v2.x + v3.x);
-                            a[1 % V] += (v0.y + v1.y) + (v2.y + v3.y);
-                            a[2 % V] += (v0.z + v1.z) + (v2.z + v3.z);
-                            a[3 % V] += (v0.w + v1.w) + (v2.w + v3.w);
-                        } else {
-                            a[0] += (__ldg(s0) + __ldg(s1)) + (__ldg(s2) + __ldg(s3));
-                        }
-                    }
-                    for (; q < pe; q += RPW) {
-                        const float* s0 = zb + (size_t)perm[q] * D + cc;
-                        if (V == 4) {
-                            const float4 v0 = __ldg(reinterpret_cast<const float4*>(s0));
-                            a[0] += v0.x; a[1 % V] += v0.y; a[2 % V] += v0.z; a[3 % V] += v0.w;
-                        } else {
-                            a[0] += __ldg(s0);
-                        }
+            for (int i = 0; i < V; ++i) a[i] = 0.f;
+            bool dirty = false;
+            for (int p = p0; p < p1; p += U) {
+                float v[U][V];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const float* src = zb + (size_t)perm[min(p + u, p1 - 1)] * D + cc;   // clamped index
+                    if (V == 4) {
+                        const float4 t = __ldg(reinterpret_cast<const float4*>(src));
+                        v[u][0] = t.x; v[u][1 % V] = t.y; v[u][2 % V] = t.z; v[u][3 % V] = t.w;
+                    } else {
+                        v[u][0] = __ldg(src);
                     }
                 }
-                // fold the rows that ran in parallel lanes
-                for (int o = LPR; o < LPR * RPW; o <<= 1) {
 #pragma unroll
-                    for (int i = 0; i < V; ++i) a[i] += __shfl_xor_sync(0xffffffffu, a[i], o);
-                }
-                if (lane < LPR && cc < D) {
-                    float* dst = gs + (size_t)j * D + cc;
-                    if (V == 4) red_add_v4(dst, a[0], a[1 % V], a[2 % V], a[3 % V]);
-                    else atomicAdd(dst, a[0]);
+                for (int u = 0; u < U; ++u) {
+                    const int pos = p + u;
+                    if (pos >= p1) break;
+                    if (pos >= jend) {                           // the label run ended: flush and move on
+                        if (dirty) {
+                            float* dst = gs + (size_t)j * D + cc;
+                            if (V == 4) red_add_v4(dst, a[0], a[1 % V], a[2 % V], a[3 % V]);
+                            else atomicAdd(dst, a[0]);
+#pragma unroll
+                            for (int i = 0; i < V; ++i) a[i] = 0.f;
+                        }
+                        do { ++j; jend = offs[j + 1]; } while (pos >= jend);   // skip empty labels
+                    }
+#pragma unroll
+                    for (int i = 0; i < V; ++i) a[i] += v[u][i];
+                    dirty = true;
                 }
             }
-            p = pe;
+            if (dirty) {
+                float* dst = gs + (size_t)j * D + cc;
+                if (V == 4) red_add_v4(dst, a[0], a[1 % V], a[2 % V], a[3 % V]);
+                else atomicAdd(dst, a[0]);
+            }
         }
     }
+}
+
+// ---- shared-memory table path ------------------------------------------------------------
+constexpr int UT_T = 512;
+
+template <int V>
+__global__ void __launch_bounds__(UT_T)
+update_table_kernel(int N, int D, int K, int G, const float* __restrict__ z, const int32_t* __restrict__ labels,
+                    float* __restrict__ part_sums, int* __restrict__ part_cnt, int* __restrict__ dev_status) {
+    extern __shared__ __align__(16) float tb[];
+    float* acc = tb;                                       // [K][D]
+    int* cnt = reinterpret_cast<int*>(tb + (size_t)K * D); // [K]
+    const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x;
+    const int KD = K * D;
+    for (int e = tid; e < KD + K; e += UT_T) tb[e] = 0.f;  // int 0 == float +0 bit pattern
+    __syncthreads();
+    const int vpr = D / V;                                 // vectors per row
+    const int rstep = UT_T / vpr;                          // rows per block step (vpr <= UT_T)
+    const int rows_per = (N + G - 1) / G;
+    const int r0 = g * rows_per, r1 = min(N, r0 + rows_per);
+    const float* zb = z + (size_t)b * N * D;
+    const int32_t* lb = labels + (size_t)b * N;
+    if (tid < rstep * vpr) {
+        const int q = tid % vpr;
+        constexpr int U = 4;                               // rows in flight per thread
+        for (int rb = r0 + tid / vpr; rb < r1; rb += U * rstep) {
+            int lab[U];
+            float v[U][V];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int r = min(rb + u * rstep, r1 - 1); // clamped: loads stay in range
+                lab[u] = __ldg(lb + r);
+                if (V == 4) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(zb + (size_t)r * D) + q);
+                    v[u][0] = t.x; v[u][1 % V] = t.y; v[u][2 % V] = t.z; v[u][3 % V] = t.w;
+                } else {
+                    v[u][0] = __ldg(zb + (size_t)r * D + q);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (rb + u * rstep >= r1) break;
+                if (lab[u] < 0 || lab[u] >= K) { atomicOr(dev_status, 1); continue; }
+                float* a = acc + (size_t)lab[u] * D + q * V;
+#pragma unroll
+                for (int i = 0; i < V; ++i) atomicAdd(a + i, v[u][i]);
+                if (q == 0) atomicAdd(&cnt[lab[u]], 1);
+            }
+        }
+    }
+    __syncthreads();
+    float* ps = part_sums + ((size_t)b * G + g) * KD;
+    for (int e = tid; e < KD; e += UT_T) ps[e] = acc[e];
+    int* pc = part_cnt + ((size_t)b * G + g) * K;
+    for (int j = tid; j < K; j += UT_T) pc[j] = cnt[j];
+}
+
+constexpr int UF_E = 32, UF_Y = 8;   // entries x slices of the partial index per block
+__global__ void __launch_bounds__(UF_E * UF_Y)
+update_table_finalize_kernel(int D, int K, int G, const float* __restrict__ part_sums,
+                             const int* __restrict__ part_cnt, float* __restrict__ cent,
+                             int32_t* __restrict__ counts) {
+    __shared__ float s_sum[UF_Y][UF_E];
+    __shared__ int s_cnt[UF_Y][UF_E];
+    const int b = blockIdx.y, x = threadIdx.x, y = threadIdx.y, KD = K * D;
+    const int e = blockIdx.x * UF_E + x;
+    // slice y adds the partials of CTAs [y*per, (y+1)*per) in order; slices are then added in order
+    const int per = (G + UF_Y - 1) / UF_Y;
+    float sum = 0.f;
+    int n = 0;
+    if (e < KD) {
+        const int j = e / D;
+        const int g1 = min(G, (y + 1) * per);
+#pragma unroll 4
+        for (int g = y * per; g < g1; ++g) {
+            sum += part_sums[((size_t)b * G + g) * KD + e];
+            n += part_cnt[((size_t)b * G + g) * K + j];
+        }
+    }
+    s_sum[y][x] = sum; s_cnt[y][x] = n;
+    __syncthreads();
+    if (y == 0 && e < KD) {
+        for (int k = 1; k < UF_Y; ++k) { sum += s_sum[k][x]; n += s_cnt[k][x]; }
+        const int j = e / D;
+        if (n > 0) cent[(size_t)b * KD + e] = sum / (float)n;
+        if (counts && e - j * D == 0) counts[(size_t)b * K + j] = n;
+    }
+}
+
+int table_ctas(int B, int N) {
+    long want = (148 + (long)B - 1) / B;
+    long cap = ((long)N + 255) / 256;
+    long g = want < cap ? want : cap;
+    return (int)(g < 1 ? 1 : g);
+}
+bool table_mode(int B, int N, int D, int K) {
+    // shared-memory float atomics are slow; worth it only where launch count dominates
+    return (long)B * N <= 32768 && (long)K * D <= 24 * 1024 && (D % 4 == 0 ? D / 4 : D) <= UT_T;
 }
 
 __global__ void update_finalize_kernel(size_t total, int D, const float* __restrict__ g_sums,
@@ -182,8 +284,13 @@ __global__ void update_empty_kernel(int total, int32_t* counts) {
 }  // namespace
 
 size_t kb_ws_need_update(int B, int N, int D, int K) {
-    (void)N;
-    return kb_align256((size_t)B * K * D * sizeof(float)) + kb_align256((size_t)B * K * sizeof(int));
+    size_t need = kb_align256((size_t)B * K * D * sizeof(float)) + kb_align256((size_t)B * K * sizeof(int));
+    if (table_mode(B, N, D, K)) {
+        const size_t G = table_ctas(B, N);
+        const size_t t = kb_align256((size_t)B * G * K * D * sizeof(float)) + kb_align256((size_t)B * G * K * sizeof(int));
+        if (t > need) need = t;
+    }
+    return need;
 }
 
 kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* labels,
@@ -199,6 +306,26 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     const size_t need = kb_ws_need_update(B, N, D, K);
     if (ctx->ws_bytes < need)
         return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_cluster_update needs %zu bytes of workspace", need);
+    if (table_mode(B, N, D, K)) {
+        const int G = table_ctas(B, N);
+        float* part_sums = reinterpret_cast<float*>(ctx->ws);
+        int* part_cnt = reinterpret_cast<int*>(ctx->ws + kb_align256((size_t)B * G * K * D * sizeof(float)));
+        const size_t smem = ((size_t)K * D + K) * sizeof(float);
+        if (D % 4 == 0) {
+            KB_SMEM_OPTIN(ctx, update_table_kernel<4>, smem);
+            update_table_kernel<4><<<dim3(G, B), UT_T, smem, ctx->stream>>>(N, D, K, G, z, labels, part_sums, part_cnt,
+                                                                         ctx->dev_status);
+        } else {
+            KB_SMEM_OPTIN(ctx, update_table_kernel<1>, smem);
+            update_table_kernel<1><<<dim3(G, B), UT_T, smem, ctx->stream>>>(N, D, K, G, z, labels, part_sums, part_cnt,
+                                                                         ctx->dev_status);
+        }
+        KB_LAUNCH_CHECK(ctx, "update_table_kernel");
+        update_table_finalize_kernel<<<dim3((K * D + UF_E - 1) / UF_E, B), dim3(UF_E, UF_Y), 0, ctx->stream>>>(
+            D, K, G, part_sums, part_cnt, c, counts);
+        KB_LAUNCH_CHECK(ctx, "update_table_finalize_kernel");
+        return KB_OK;
+    }
     float* g_sums = reinterpret_cast<float*>(ctx->ws);
     int* g_counts = reinterpret_cast<int*>(ctx->ws + kb_align256((size_t)B * K * D * sizeof(float)));
     KB_MEMSET(ctx, ctx->ws, 0, need);
@@ -219,10 +346,10 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     const int V = (D % 4 == 0) ? 4 : 1;
     const int lpr = (D / V) < 32 ? (D / V) : 32;
     const int rpw = (32 % lpr == 0) ? 32 / lpr : 1;
-    // chunk of the sorted order a warp takes at a time: about four chunks per warp, 32..256 positions
-    int CH = (rows_per + 4 * (UP_T / 32) - 1) / (4 * (UP_T / 32));
-    CH = CH < 32 ? 32 : (CH > 256 ? 256 : CH);
-    CH = (CH + rpw - 1) / rpw * rpw;
+    // piece of the sorted order a lane group takes at a time: about four pieces per group, 8..128 positions
+    const int groups = (UP_T / 32) * rpw;
+    int CH = (rows_per + 4 * groups - 1) / (4 * groups);
+    CH = CH < 8 ? 8 : (CH > 128 ? 128 : CH);
     dim3 grid((unsigned)G, B);
     if (V == 4) {
         KB_SMEM_OPTIN(ctx, update_sorted_kernel<4>, smem);
