@@ -117,6 +117,12 @@ __device__ __forceinline__ void tc_mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, 
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
         : "memory");
 }
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ uint64_t mk_desc(uint32_t lo, uint32_t hi) {
     return ((uint64_t)hi << 32) | (uint64_t)lo;
 }
@@ -459,10 +465,12 @@ assign_tc_kernel(const TcParams p) {
         }
     } else if (warp == 12) {
         // ============================ MMA issuer ======================================
-        // A single lane issues every MMA, so its instruction stream is the critical path of the
-        // whole CTA: descriptors are formed with one add each (all k-steps unrolled) and nothing
-        // else happens between two tcgen05.mma.
-        if (lane == 0) {
+        // One elected lane issues every MMA, so this instruction stream is the critical path of
+        // the whole CTA.  The WHOLE warp runs the loops and the waits, and only the tcgen05
+        // instructions sit under the elected-lane predicate: in warp-uniform control flow the
+        // descriptor arithmetic stays on the uniform datapath (measured: 64 cycles per 128x128x8
+        // MMA, the tensor pipe's own rate, against 83-100 when a single lane runs the loop alone).
+        {
             uint32_t s = 0, ph = 0, q = 0;
             int it = 0;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
@@ -474,22 +482,23 @@ assign_tc_kernel(const TcParams p) {
                 const uint32_t a_base = tmem + COL_A + ab * 2 * D;
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
-                    ok = mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
                     for (int kb = 0; kb < nkb; ++kb) {
                         if (nt == 0) {
-                            ok = mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag);
+                            ok = __all_sync(0xffffffffu, mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag));
                             if (!ok) break;
                         }
                         if (!p.resident || it == 0) {              // resident panels are loaded exactly once
-                            ok = mbar_wait(BAR(B_FULL + s), ph, abort_flag);
+                            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + s), ph, abort_flag));
                             if (!ok) break;
                         }
                         tc_fence_after();
                         const uint32_t a_hi = a_base + kb * KBF, a_lo = a_hi + D;
                         const uint32_t blo = desc_lo32 + s * (STAGE >> 4);        // this stage's hi panel
+                        if (elect_one()) {
                         // first k-step: the very first product of an accumulator tile overwrites it
                         tc_mma_ts(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, kb != 0 ? 1u : 0u);
                         tc_mma_ts_acc(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
@@ -502,10 +511,12 @@ assign_tc_kernel(const TcParams p) {
                         }
                         if (!p.resident) tc_commit(BAR(B_EMPTY + s));      // stage reusable once these MMAs retire
                         if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + ab * 4 + kb));  // A panel reusable
+                        if (kb == nkb - 1) tc_commit(BAR(ACC_FULL + buf));             // accumulator tile complete
+                        }
+                        __syncwarp();
                         if (++s == (uint32_t)ring) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
-                    tc_commit(BAR(ACC_FULL + buf));
                 }
             }
         }
