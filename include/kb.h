@@ -208,6 +208,33 @@ kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const floa
                              const float* centroids, int32_t* labels, float* approx_dist2,
                              int32_t* flagged);
 
+/* kb_cluster_update for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the centroid update above.)
+ *
+ * Some hosts of this library own every byte of device memory themselves: a serving process
+ * whose memory plan is fixed when it starts, a plug-in running inside another framework's
+ * arena, a latency-critical loop that must never hit the implicit device-wide
+ * synchronisation of an allocation call.  Such a caller can neither cudaMalloc a workspace
+ * nor hand one over.  This entry point therefore takes no context and no workspace: its
+ * scratch (sums and counts) is a fixed array compiled into the library, which every GPU
+ * that loads the library carries until the process exits (about 0.27 MB).  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   single instance (B = 1); same meaning of z [N][D], labels [N], centroids [K][D]
+ *   (in: previous, out: new) and counts [K] (nullable) as kb_cluster_update; all DEVICE
+ *   pointers on the CURRENT device; cuda_stream is a borrowed cudaStream_t.
+ *   Limits: K * D <= KB_NOALLOC_MAX_KD and K <= KB_NOALLOC_MAX_K; anything larger
+ *   returns KB_ERR_UNSUPPORTED and queues nothing.
+ *   The first call on a device looks up the scratch array's device address and reads two
+ *   device attributes; make that first call before any stream capture begins.
+ *   Every call on a device shares the one array (the call clears what it needs first), so
+ *   two calls that overlap on the GPU -- different streams, no ordering -- race: order them.
+ *   Label errors are recorded in the array's own status word, not in a context. */
+#define KB_NOALLOC_MAX_KD 65536
+#define KB_NOALLOC_MAX_K 4096
+kb_status kb_cluster_update_noalloc(void* cuda_stream, int N, int D, int K, const float* z,
+                                    const int32_t* labels, float* centroids, int32_t* counts);
+
 /* ---- conveniences built from the five calls ----------------------------- */
 
 /* centroids[b][i][:] = z[b][rows[b][i]][:]  (plain Lloyd started from K data

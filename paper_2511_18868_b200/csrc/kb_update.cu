@@ -367,3 +367,88 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     KB_LAUNCH_CHECK(ctx, "update_finalize_kernel");
     return KB_OK;
 }
+
+// ---- centroid update for callers that must not allocate ------------------------------------
+// Scratch for kb_cluster_update_noalloc lives in the library image itself: one file-scope
+// device array, present on every GPU that loads the library until the process exits.
+// Layout: [0, 256) status word | sums float[KB_NOALLOC_MAX_KD] | counts int[KB_NOALLOC_MAX_K].
+#define KB_NOALLOC_SCRATCH_BYTES (256 + (size_t)KB_NOALLOC_MAX_KD * sizeof(float) + (size_t)KB_NOALLOC_MAX_K * sizeof(int))
+static __device__ __align__(256) unsigned char kb_noalloc_scratch[KB_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+// Device address of the array above, per device.  In host code the array's NAME is only a
+// stand-in for the symbol, not a device pointer, so the address is asked for once per
+// device with cudaGetSymbolAddress and remembered here.
+void* g_noalloc_ptr[NOALLOC_MAX_DEVICES];
+int g_noalloc_sms[NOALLOC_MAX_DEVICES];
+int g_noalloc_smem[NOALLOC_MAX_DEVICES];
+}  // namespace
+
+extern "C" kb_status kb_cluster_update_noalloc(void* cuda_stream, int N, int D, int K, const float* z,
+                                               const int32_t* labels, float* centroids, int32_t* counts) {
+    if (N < 0 || D < 1 || K < 1) return KB_ERR_INVALID_ARG;
+    if (!centroids || (N > 0 && (!z || !labels))) return KB_ERR_INVALID_ARG;
+    if (D % 4 == 0 && (((uintptr_t)z) & 15) != 0) return KB_ERR_INVALID_ARG;
+    // sizes beyond the built-in scratch are refused, never truncated
+    if ((long long)K * D > KB_NOALLOC_MAX_KD || K > KB_NOALLOC_MAX_K) return KB_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return KB_ERR_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        // first call on this device (it is the current one): look the symbol up, read two attributes
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, kb_noalloc_scratch) != cudaSuccess || !p) return KB_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&g_noalloc_smem[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return KB_ERR_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
+    int* status = reinterpret_cast<int*>(base);
+    float* g_sums = reinterpret_cast<float*>(base + 256);
+    int* g_counts = reinterpret_cast<int*>(base + 256 + (size_t)KB_NOALLOC_MAX_KD * sizeof(float));
+    if (N == 0) {
+        if (counts) {
+            update_empty_kernel<<<(K + 255) / 256, 256, 0, st>>>(K, counts);
+            if (cudaGetLastError() != cudaSuccess) return KB_ERR_CUDA;
+        }
+        return KB_OK;
+    }
+    // the array keeps whatever the previous call left: clear the part this call accumulates into
+    if (cudaMemsetAsync(g_sums, 0, (size_t)K * D * sizeof(float), st) != cudaSuccess) return KB_ERR_CUDA;
+    if (cudaMemsetAsync(g_counts, 0, (size_t)K * sizeof(int), st) != cudaSuccess) return KB_ERR_CUDA;
+    long want = 2L * g_noalloc_sms[dev];
+    long lo = ((long)N + UP_MAXROWS - 1) / UP_MAXROWS;
+    long hi = ((long)N + 511) / 512;
+    long G = want < lo ? lo : want;
+    if (G > hi) G = hi;
+    if (G < lo) G = lo;
+    if (G < 1) G = 1;
+    const int rows_per = (int)((N + G - 1) / G);
+    const size_t smem = ((size_t)2 * K + 1) * sizeof(int) + (size_t)rows_per * sizeof(unsigned short) + 16;
+    if (smem > (size_t)g_noalloc_smem[dev] - 256) return KB_ERR_UNSUPPORTED;
+    const int V = (D % 4 == 0) ? 4 : 1;
+    const int lpr = (D / V) < 32 ? (D / V) : 32;
+    const int rpw = (32 % lpr == 0) ? 32 / lpr : 1;
+    const int groups = (UP_T / 32) * rpw;
+    int CH = (rows_per + 4 * groups - 1) / (4 * groups);
+    CH = CH < 8 ? 8 : (CH > 128 ? 128 : CH);
+    dim3 grid((unsigned)G, 1);
+    if (V == 4) {
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(update_sorted_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return KB_ERR_CUDA;
+        update_sorted_kernel<4><<<grid, UP_T, smem, st>>>(N, D, K, (int)G, CH, z, labels, g_sums, g_counts, status);
+    } else {
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(update_sorted_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return KB_ERR_CUDA;
+        update_sorted_kernel<1><<<grid, UP_T, smem, st>>>(N, D, K, (int)G, CH, z, labels, g_sums, g_counts, status);
+    }
+    if (cudaGetLastError() != cudaSuccess) return KB_ERR_CUDA;
+    const size_t total = (size_t)K * D;
+    update_finalize_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(total, D, g_sums, g_counts, centroids, counts);
+    if (cudaGetLastError() != cudaSuccess) return KB_ERR_CUDA;
+    return KB_OK;
+}

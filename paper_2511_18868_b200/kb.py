@@ -26,7 +26,7 @@ EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb
            "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
-           "kb_bandit_step_host"]
+           "kb_bandit_step_host", "kb_cluster_update_noalloc"]
 
 
 TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init"]
@@ -91,6 +91,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_set_assign_options.argtypes = [_VP, i, f]
     lib.kb_get_assign_path.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_assign_tc_probe.argtypes = [_VP, i, i, i, i] + [_VP] * 5
+    lib.kb_cluster_update_noalloc.argtypes = [_VP, i, i, i, _VP, _VP, _VP, _VP]
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
     lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
@@ -293,6 +294,20 @@ class KB:
         """Whole step on HOST tensors (ideally pinned); returns after the results are in host memory."""
         a = self._step_args(dims, params, tensors, host=True)
         self._check(self.lib.kb_bandit_step_host(self.h, ctypes.byref(a)), "kb_bandit_step_host")
+
+
+def cluster_update_noalloc(z, labels, centroids, counts=None, stream=None):
+    """kb_cluster_update_noalloc: one instance, scratch built into the library, nothing allocated.
+    z [N][D], labels [N], centroids [K][D] (updated in place), counts [K] or None; device tensors."""
+    lib = load_library()
+    N, D = z.shape
+    K = centroids.shape[0]
+    st = stream if stream is not None else torch.cuda.current_stream(z.device)
+    with torch.cuda.device(z.device):
+        rc = lib.kb_cluster_update_noalloc(_VP(st.cuda_stream), N, D, K, _ptr(z), _ptr(labels), _ptr(centroids),
+                                           _ptr(counts))
+    if rc != KB_OK:
+        raise KbError(rc, "kb_cluster_update_noalloc")
 
 
 def step_tensors(inp: Dict, device, want_arm_index=True, want_bound=True, pinned_host=False) -> Dict[str, torch.Tensor]:
