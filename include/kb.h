@@ -92,7 +92,8 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_PRUNE 3
 #define KB_T_SCORE 4
 #define KB_T_INIT 5
-#define KB_T_COUNT 6
+#define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
+#define KB_T_COUNT 7
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
 
@@ -245,7 +246,10 @@ kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float
 
 /* iters x (assign, update) followed by a final assign, so that labels/dist2
  * are consistent with the returned centroids (Sec. 3.3).  Same arguments as
- * the two calls it is made of; counts are those of the last update. */
+ * the two calls it is made of; counts are those of the last update.
+ * Instances of at most 512 rows with D in {16, 32, 64} run the whole loop in one launch
+ * (one CTA per instance, the instance resident on chip), unless kb_set_assign_options
+ * forces an assign path. */
 kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z,
                          float* centroids, int32_t* labels, float* dist2, float* inertia,
                          int32_t* rep, int32_t* counts);

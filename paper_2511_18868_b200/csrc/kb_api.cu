@@ -307,6 +307,13 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
                          int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
     KB_COMMON(ctx, B, N);
     KB_REQUIRE(ctx, iters >= 0, "kb_cluster_fit: iters must be >= 0");
+    if (ctx->assign_path == 0 && kb_fit_fused_eligible(ctx, B, N, D, K) && z && centroids && labels &&
+        (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
+        // small instances: the whole loop in one launch, one CTA per instance
+        KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_fit: D and K must be >= 1");
+        TimeScope ts__(ctx, KB_T_FIT);
+        return kb_launch_fit_fused(ctx, B, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
+    }
     for (int it = 0; it < iters; ++it) {
         kb_status s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
         if (s != KB_OK) return s;

@@ -1,0 +1,184 @@
+// kb_cluster_fit for small instances: one CTA per instance, the whole Lloyd loop in one launch.
+//
+// When an instance has at most 512 rows and D is 16, 32 or 64, per-call launches dominate
+// (a call moves a few KB): iters x (assign, update) + the final assign would be 2*iters+1
+// calls of several kernels each.  Here a CTA keeps its instance on chip for all iterations:
+//   * thread = row, the row lives in registers (D floats);
+//   * centroids live in shared memory and are read as warp-wide float4 broadcasts;
+//     the distance is the direct form sum (z - c)^2, ascending centroid id, strict <
+//     (lowest id on ties) -- the same arithmetic as the row-wise assign kernel;
+//   * update: counting sort of the row ids by label in shared memory (integer atomics),
+//     then thread (cluster, column) adds up its cluster's rows from a padded shared copy
+//     of the instance: no floating-point atomics, bank-conflict free;
+//   * the final assign also produces dist2, inertia (double, fixed-order block reduction)
+//     and the representative member per cluster (64-bit shared atomicMin on (dist2, row)).
+// X is read from HBM exactly once per fit.
+#include "kb_internal.cuh"
+
+namespace {
+
+constexpr int FF_T = 512;
+
+template <int D>
+__global__ void __launch_bounds__(FF_T)
+fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
+                 int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
+                 int32_t* __restrict__ rep, int32_t* __restrict__ counts) {
+    extern __shared__ __align__(16) unsigned char ff_raw[];
+    constexpr int ZS = D + 1;                                       // padded row stride: conflict-free column walks
+    float* cs = reinterpret_cast<float*>(ff_raw);                   // [K][D] centroids (16-byte aligned rows)
+    float* zs = cs + (size_t)K * D;                                 // [N][D+1] the instance
+    // [K] counts, then scatter cursors; 8-byte aligned because the space is reused for 64-bit keys
+    int* hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(zs + (size_t)N * ZS) + 7) & ~(uintptr_t)7);
+    int* offs = hist + K;                                           // [K+1]
+    unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [N] row ids in label order
+    __shared__ double s_red[FF_T / 32];
+    __shared__ int s_scan[FF_T / 32];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* zb = z + (size_t)b * N * D;
+    float* cb = cent + (size_t)b * K * D;
+
+    // stage the instance (coalesced float4 reads) and the initial centroids
+    for (int e = tid; e < N * (D / 4); e += FF_T) {
+        const int r = e / (D / 4), q = e - r * (D / 4);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(zb) + e);
+        float* d = zs + (size_t)r * ZS + 4 * q;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+    for (int e = tid; e < K * D / 4; e += FF_T)
+        reinterpret_cast<float4*>(cs)[e] = __ldg(reinterpret_cast<const float4*>(cb) + e);
+    __syncthreads();
+    const bool active = tid < N;
+    float x[D];
+#pragma unroll
+    for (int d = 0; d < D; ++d) x[d] = active ? zs[(size_t)tid * ZS + d] : 0.f;
+
+    float best = 0.f;
+    int arg = 0;
+    for (int it = 0; it <= iters; ++it) {
+        // ---- assign: nearest centroid of my row -------------------------------------------
+        best = INFINITY;
+        arg = 0;
+        for (int j = 0; j < K; ++j) {
+            const float4* c4 = reinterpret_cast<const float4*>(cs + (size_t)j * D);
+            float acc = 0.f;
+#pragma unroll
+            for (int q = 0; q < D / 4; ++q) {
+                const float4 c = c4[q];
+                const float e0 = x[4 * q] - c.x, e1 = x[4 * q + 1] - c.y, e2 = x[4 * q + 2] - c.z, e3 = x[4 * q + 3] - c.w;
+                acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+            }
+            if (acc < best) { best = acc; arg = j; }
+        }
+        if (it == iters) break;                                     // the final assign has no update after it
+        // ---- update: counting sort by label, then (cluster, column) sums ----------------------
+        for (int j = tid; j < K; j += FF_T) hist[j] = 0;
+        __syncthreads();
+        if (active) atomicAdd(&hist[arg], 1);
+        __syncthreads();
+        {   // exclusive scan of hist (K may exceed the block: contiguous slices per thread)
+            const int per = (K + FF_T - 1) / FF_T;
+            const int j0 = min(K, tid * per), j1 = min(K, j0 + per);
+            int local = 0;
+            for (int j = j0; j < j1; ++j) local += hist[j];
+            int incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) s_scan[warp] = incl;
+            __syncthreads();
+            int base = 0;
+            for (int w = 0; w < warp; ++w) base += s_scan[w];
+            int run = base + incl - local;
+            for (int j = j0; j < j1; ++j) { offs[j] = run; run += hist[j]; }
+            if (tid == FF_T - 1) offs[K] = run;
+        }
+        __syncthreads();
+        for (int j = tid; j < K; j += FF_T) hist[j] = offs[j];      // scatter cursors
+        __syncthreads();
+        if (active) perm[atomicAdd(&hist[arg], 1)] = (unsigned short)tid;
+        __syncthreads();
+        if (it == iters - 1 && counts)
+            for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = offs[j + 1] - offs[j];
+        for (int e = tid; e < K * D; e += FF_T) {
+            const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
+            const int p0 = offs[j], p1 = offs[j + 1];
+            if (p1 > p0) {                                          // an empty cluster keeps its centroid
+                float s0 = 0.f, s1 = 0.f;
+                int p = p0;
+                for (; p + 1 < p1; p += 2) {
+                    s0 += zs[(size_t)perm[p] * ZS + d];
+                    s1 += zs[(size_t)perm[p + 1] * ZS + d];
+                }
+                if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
+                cs[e] = (s0 + s1) / (float)(p1 - p0);
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- outputs of the final assign --------------------------------------------------------
+    unsigned long long* rep_key = reinterpret_cast<unsigned long long*>(hist);   // hist/offs are free now: [K] keys
+    if (rep) {
+        __syncthreads();
+        for (int j = tid; j < K; j += FF_T) rep_key[j] = ~0ull;
+        __syncthreads();
+    }
+    if (active) {
+        const size_t flat = (size_t)b * N + tid;
+        labels[flat] = arg;
+        if (dist2) dist2[flat] = best;
+        if (rep) atomicMin(&rep_key[arg], ((unsigned long long)__float_as_uint(best) << 32) | (unsigned)tid);
+    }
+    for (int e = tid; e < K * D / 4; e += FF_T)
+        reinterpret_cast<float4*>(cb)[e] = reinterpret_cast<const float4*>(cs)[e];
+    if (iters == 0 && counts)
+        for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = 0;
+    if (inertia) {
+        double s = kb_warp_sum(active ? (double)best : 0.0);
+        if (lane == 0) s_red[warp] = s;
+    }
+    __syncthreads();
+    if (inertia && tid == 0) {
+        double s = 0.0;
+        for (int w = 0; w < FF_T / 32; ++w) s += s_red[w];
+        inertia[b] = (float)s;
+    }
+    if (rep)
+        for (int j = tid; j < K; j += FF_T) {
+            const unsigned long long key = rep_key[j];
+            rep[(size_t)b * K + j] = key == ~0ull ? -1 : (int32_t)(key & 0xffffffffull);
+        }
+}
+
+size_t ff_smem(int N, int D, int K) {
+    // centroids | instance (padded) | hist [K] + offs [K+1] (reused as K 64-bit keys: needs 2K ints) | perm
+    return (size_t)K * D * 4 + (size_t)N * (D + 1) * 4 + 8 + (size_t)(2 * K + 2) * 4 + (size_t)N * 2 + 16;
+}
+
+}  // namespace
+
+bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
+    if (B < 1 || N < 1 || N > FF_T || K < 1 || K > 4096) return false;
+    if (D != 16 && D != 32 && D != 64) return false;
+    return ff_smem(N, D, K) + 256 <= (size_t)ctx->max_smem_optin;
+}
+
+kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* cent,
+                              int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+    const size_t smem = ff_smem(N, D, K);
+    if (D == 16) {
+        KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
+        fit_fused_kernel<16><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+    } else if (D == 32) {
+        KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
+        fit_fused_kernel<32><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+    } else {
+        KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
+        fit_fused_kernel<64><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+    }
+    KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
+    return KB_OK;
+}

@@ -73,6 +73,9 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
 kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* c,
                                   const int32_t* labels, float* dist2, double* ws_inertia,
                                   unsigned long long* ws_rep);
+bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
+kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* cent,
+                              int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts);
 size_t kb_ws_need_update(int B, int N, int D, int K);
 size_t kb_ws_need_score(int B, int N, int K, int S);
 #define KB_NORM_MAXG 1024
