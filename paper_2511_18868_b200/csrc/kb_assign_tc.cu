@@ -600,12 +600,13 @@ __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                     const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
                     const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
-    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows
+    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_ROWS][FX_T / 32];
     __shared__ int red_i[FX_ROWS][FX_T / 32];
     __shared__ int s_inst[FX_ROWS];
     fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
     float* xrow = fx;
+    float* ctile = fx + FX_ROWS * D;                       // [FX_T][D+4] centroid tile
     const int total = flag_count[1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int g0 = blockIdx.x * FX_ROWS; g0 < total; g0 += gridDim.x * FX_ROWS) {
@@ -623,6 +624,44 @@ assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const floa
         int arg[FX_ROWS];
 #pragma unroll
         for (int r = 0; r < FX_ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
+        bool same_inst = true;
+#pragma unroll
+        for (int r = 1; r < FX_ROWS; ++r) same_inst = same_inst && (s_inst[r] == s_inst[0]);
+        if (same_inst) {
+            // the usual case: tiles of FX_T centroids are staged through shared memory with coalesced,
+            // independent loads (one memory round trip per tile), thread t then owns centroid t of the tile
+            const int CS = D + 4;                                  // 16-byte aligned, conflict-free float4 rows
+            const float* cbase = cent + (size_t)s_inst[0] * K * D;
+            for (int j0 = 0; j0 < K; j0 += FX_T) {
+                const int nc = min(FX_T, K - j0);
+                __syncthreads();
+                for (int e = tid; e < nc * (D / 4); e += FX_T) {
+                    const int jr = e / (D / 4), q = e - jr * (D / 4);
+                    *reinterpret_cast<float4*>(ctile + (size_t)jr * CS + 4 * q) =
+                        __ldg(reinterpret_cast<const float4*>(cbase + (size_t)(j0 + jr) * D) + q);
+                }
+                __syncthreads();
+                if (tid < nc) {
+                    float acc[FX_ROWS];
+#pragma unroll
+                    for (int r = 0; r < FX_ROWS; ++r) acc[r] = 0.f;
+                    const float4* c4 = reinterpret_cast<const float4*>(ctile + (size_t)tid * CS);
+                    for (int d = 0; d < D / 4; ++d) {
+                        const float4 c = c4[d];
+#pragma unroll
+                        for (int r = 0; r < FX_ROWS; ++r) {
+                            const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
+                            float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                            acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
+                            acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < FX_ROWS; ++r)
+                        if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j0 + tid; }   // ascending tiles: lowest index on ties
+                }
+            }
+        } else
         for (int j = tid; j < K; j += FX_T) {
             float acc[FX_ROWS];
 #pragma unroll
@@ -802,8 +841,9 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     }
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
-    const size_t fsmem = (size_t)FX_ROWS * D * 4;
-    assign_fixup_kernel<<<2 * ctx->sm_count, FX_T, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows,
+    const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
+    KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
+    assign_fixup_kernel<<<4 * ctx->sm_count, FX_T, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows,
                                                                         full_rows, labels);
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
