@@ -117,13 +117,38 @@ norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, doubl
     __syncthreads();
     if (!last) return;
     __threadfence();
-    for (int col = tid; col < D; col += blockDim.x) {
+    // all threads take part: columns in chunks of CP, each chunk split into SL slices of the partial
+    // index; a slice adds its partials in order (four loads in flight), slices are added in order
+    const int CP = D < (int)blockDim.x ? D : (int)blockDim.x;
+    const int SL = (int)blockDim.x / CP;
+    const int cc = tid % CP, sl = tid / CP;
+    const int per = (G + SL - 1) / SL;
+    for (int c0 = 0; c0 < D; c0 += CP) {
+        const int col = c0 + cc;
         double a = 0.0, q = 0.0;
-        for (int k = 0; k < G; ++k) {
-            const double* p = part + (((size_t)b * G + k) * D + col) * 2;
-            a += __ldcg(p);  // written by other blocks of this launch: read through L2
-            q += __ldcg(p + 1);
+        if (sl < SL && col < D) {
+            const int k1 = min(G, (sl + 1) * per);
+            int k = sl * per;
+            for (; k + 3 < k1; k += 4) {
+                const double* p0 = part + (((size_t)b * G + k) * D + col) * 2;
+                const size_t st = (size_t)D * 2;
+                const double a0 = __ldcg(p0), q0 = __ldcg(p0 + 1), a1 = __ldcg(p0 + st), q1 = __ldcg(p0 + st + 1);
+                const double a2 = __ldcg(p0 + 2 * st), q2 = __ldcg(p0 + 2 * st + 1);
+                const double a3 = __ldcg(p0 + 3 * st), q3 = __ldcg(p0 + 3 * st + 1);
+                a += a0; a += a1; a += a2; a += a3;
+                q += q0; q += q1; q += q2; q += q3;
+            }
+            for (; k < k1; ++k) {
+                const double* p = part + (((size_t)b * G + k) * D + col) * 2;
+                a += __ldcg(p);  // written by other blocks of this launch: read through L2
+                q += __ldcg(p + 1);
+            }
         }
+        __syncthreads();
+        red[2 * tid] = a; red[2 * tid + 1] = q;
+        __syncthreads();
+        if (sl != 0 || col >= D) continue;
+        for (int k = 1; k < SL; ++k) { a += red[2 * (k * CP + cc)]; q += red[2 * (k * CP + cc) + 1]; }
         double ms = a / (double)N;
         double var = q / (double)N - ms * ms;
         if (var < 0.0) var = 0.0;
