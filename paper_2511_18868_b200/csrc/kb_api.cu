@@ -229,7 +229,7 @@ kb_status kb_cluster_assign(kb_ctx* ctx, int B, int N, int D, int K, const float
 
 kb_status kb_set_assign_options(kb_ctx* ctx, int path, float tc_eps) {
     if (!ctx) return KB_ERR_INVALID_ARG;
-    KB_REQUIRE(ctx, path >= 0 && path <= 2, "kb_set_assign_options: path must be 0, 1 or 2");
+    KB_REQUIRE(ctx, path >= 0 && path <= 3, "kb_set_assign_options: path must be 0, 1, 2 or 3");
     ctx->assign_path = path;
     ctx->tc_eps = tc_eps > 0.f ? tc_eps : 1.0f / 65536.0f;
     return KB_OK;

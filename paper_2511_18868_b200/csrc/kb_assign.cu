@@ -167,8 +167,8 @@ kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float*
                            float* dist2, float* inertia, int32_t* rep) {
     if (B == 0) return KB_OK;
     const bool use_tc = N > 0 && ctx->assign_path != 1 &&
-                        (ctx->assign_path == 2 ? kb_assign_tc_supported(ctx, B, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
-    if (ctx->assign_path == 2 && N > 0 && !use_tc)
+                        (ctx->assign_path >= 2 ? kb_assign_tc_supported(ctx, B, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
+    if (ctx->assign_path >= 2 && N > 0 && !use_tc)
         return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_assign: the tensor path needs D %% 32 == 0, D <= 128");
     double* ws_inertia = nullptr;
     unsigned long long* ws_rep = nullptr;
@@ -194,7 +194,7 @@ kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float*
             s = kb_launch_assign_tc(ctx, ctx->ws + off_tc, B, N, D, K, z, c, labels, nullptr, nullptr, ctx->tc_eps);
             if (s == KB_OK && (dist2 || inertia || rep))
                 s = kb_launch_assign_finish(ctx, B, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
-            ctx->last_assign_path = 2;
+            ctx->last_assign_path = ctx->assign_path == 3 ? 3 : 2;
         } else {
             s = launch_rowwise(ctx, B, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
             ctx->last_assign_path = 1;

@@ -30,6 +30,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all
 // roles drain, TMEM is released and the device status word reports a timeout.
 #include "kb_internal.cuh"
+#include <cuda_fp16.h>
 
 namespace {
 
@@ -43,7 +44,8 @@ constexpr int TC_THREADS = 448;
 constexpr int TMEM_COLS = 512;
 constexpr int COL_ACC = 0;         // two accumulators: columns [0,128) and [128,256)
 constexpr int COL_A = 256;         // A buffer i: hi at [256 + 2iD, +D), lo at [256 + 2iD + D, +D); two buffers when D <= 64
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 19;          // polls of a bounded wait, each suspended for up to WAIT_SUSPEND_NS
+constexpr uint32_t WAIT_SUSPEND_NS = 2000;
 constexpr int STATUS_TIMEOUT = 0x100;
 
 // ---- PTX helpers ------------------------------------------------------------------
@@ -54,6 +56,14 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// One arrival for the whole warp: every lane's earlier work (shared-memory stores, completed
+// tensor-memory loads/stores followed by the tcgen05 fence) is ordered before it by the warp
+// barrier.  Barriers signalled this way count warps, not threads: 32 times fewer shared-memory
+// atomics on the path between the roles.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -69,12 +79,28 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit
-// or another role has already aborted.
+// The same test, but the hardware may keep the thread suspended for up to `ns` nanoseconds while
+// the phase is incomplete (it resumes at once when the phase completes).  A waiting role then
+// executes one instruction per `ns` instead of spinning, which matters here: the waiting roles
+// share their schedulers with the epilogue warps.
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait (about a second at most).  Returns false (and raises the CTA's abort flag) when
+// the limit is hit or another role has already aborted.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
     for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-        if (mbar_try(bar, parity)) return true;
-        if ((i & 127u) == 127u && *abort_flag) return false;
+        if (mbar_try_suspend(bar, parity, WAIT_SUSPEND_NS)) return true;
+        if ((i & 7u) == 7u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -99,23 +125,41 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc], kind::tf32
+template <bool F16>
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (F16)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
 }
 // accumulate form (enable_input_d is the constant true predicate)
+template <bool F16>
 __device__ __forceinline__ void tc_mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.eq.b32 p, 0, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
-        : "memory");
+    if (F16)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.eq.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.eq.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
+            : "memory");
 }
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one() {
@@ -178,10 +222,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 // kind::tf32, fp32 accumulate, A and B K-major, M = 128, N = BN
-constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC_TF32 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// kind::f16 with fp16 operands (format 0), fp32 accumulate, same shape; one instruction covers K = 16
+constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
 
 struct TcParams {
     int B, N, D, K, Kpad;
+    int nkb;                       // k-blocks (128-byte swizzle rows) per centroid: D/32 tf32, ceil(D/64) fp16
+    int DC;                        // TMEM columns of one A part (hi or lo): D for tf32, 32 * nkb for fp16
     int tiles_per_inst, total_tiles;
     int nxb;                       // Z staging buffers (1 or 2)
     int resident;                  // 1: the whole B image of the (single) instance stays in the stage ring
@@ -189,6 +238,7 @@ struct TcParams {
     const float* z;
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
     const float* cnorm;            // [B][Kpad]
+    const float* cweight;          // [B][Kpad]  -2 / (the centroid's power-of-two scale)
     int32_t* labels;
     float* approx;                 // optional: ||z||^2 + best score (expanded-form d^2), diagnostics
     int* flag_count;               // [0]: rows queued for a two-candidate check, [1]: for a full re-evaluation
@@ -198,89 +248,153 @@ struct TcParams {
 };
 
 // ---- preparation: split centroids into swizzled hi/lo panels, squared norms ----------
+// Power-of-two factor that brings a vector with largest magnitude m into [0.5, 1): the fp16 split
+// keeps 22 significant bits only while hi and lo stay inside fp16's normal range, so every row
+// and every centroid is scaled by its own exact factor and the product is unscaled afterwards.
+__device__ __forceinline__ float pow2_scale(float m) {
+    if (!(m > 0.f) || !(m < INFINITY)) return 1.f;
+    int e;
+    frexpf(m, &e);
+    e = e < -100 ? -100 : (e > 100 ? 100 : e);
+    return ldexpf(1.f, -e);
+}
+// (hi, lo) fp16 split of two scaled values, packed the way the tensor core reads 16-bit
+// operands: the lower k index in the low half of the 32-bit word
+__device__ __forceinline__ void split_f16x2(float a, float b, uint32_t& hi, uint32_t& lo) {
+    const __half2 h = __floats2half2_rn(a, b);
+    const float2 hf = __half22float2(h);
+    const __half2 l = __floats2half2_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+// One warp per centroid: lane q owns the 16-byte chunk q of the fp32 row (D <= 128).
+//   F16 = false: tf32 hi/lo panels, 32 features per 128-byte swizzle row, weight -2
+//   F16 = true : fp16 hi/lo panels of the centroid scaled by its own power of two, 64 features
+//                per 128-byte swizzle row (features past D are zero), weight -2 / scale
+template <bool F16>
 __global__ void __launch_bounds__(256)
-tc_prep_kernel(int K, int D, int Kpad, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
-               float* __restrict__ cnorm, int* __restrict__ flag_count) {
+tc_prep_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
+               float* __restrict__ cnorm, float* __restrict__ cweight, int* __restrict__ flag_count) {
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
-    // one warp per centroid: lane q owns the 16-byte chunk q of the row (D <= 128)
     const int b = blockIdx.y;
-    const int nkb = D / KBF, nt = Kpad / BN;
+    const int nt = Kpad / BN;
     const int lane = threadIdx.x & 31;
     const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (j >= Kpad) return;
+    const int fpr = F16 ? 64 : 32;                         // features per swizzle row
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j < K && lane < D / 4) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + lane);
+    const float f[4] = {v.x, v.y, v.z, v.w};
     double sq = 0.0;
-    if (lane < D / 4) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < K) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + lane);
-        const float f[4] = {v.x, v.y, v.z, v.w};
-        uint32_t hi[4], lo[4];
+    float m = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            hi[i] = to_tf32(f[i]);
-            lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
-            sq += (double)f[i] * (double)f[i];
-        }
-        const int kb = lane >> 3, c = lane & 7;
-        const int tile = j / BN, r = j - tile * BN;
-        const size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
-                           ((c ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-    }
+    for (int i = 0; i < 4; ++i) { sq += (double)f[i] * (double)f[i]; m = fmaxf(m, fabsf(f[i])); }
     sq = kb_warp_sum(sq);
-    if (lane == 0) cnorm[(size_t)b * Kpad + j] = j < K ? (float)sq : INFINITY;   // padding can never win
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    const float sc = F16 ? pow2_scale(m) : 1.f;
+    if (lane < nkb * fpr / 4) {
+        const int kb = (4 * lane) / fpr, within = 4 * lane - kb * fpr;     // feature offset inside the swizzle row
+        const int tile = j / BN, r = j - tile * BN;
+        const int bytes_in_row = within * (F16 ? 2 : 4);
+        const int chunk = bytes_in_row >> 4;
+        const size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
+                           ((chunk ^ (r & 7)) << 4) + (bytes_in_row & 15);
+        if (F16) {
+            uint32_t h0, l0, h1, l1;
+            split_f16x2(f[0] * sc, f[1] * sc, h0, l0);
+            split_f16x2(f[2] * sc, f[3] * sc, h1, l1);
+            *reinterpret_cast<uint2*>(bimg + off) = make_uint2(h0, h1);
+            *reinterpret_cast<uint2*>(bimg + off + PANEL) = make_uint2(l0, l1);
+        } else {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                hi[i] = to_tf32(f[i]);
+                lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
+            }
+            *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    if (lane == 0) {
+        cnorm[(size_t)b * Kpad + j] = j < K ? (float)sq : INFINITY;   // padding can never win
+        cweight[(size_t)b * Kpad + j] = j < K ? -2.f / sc : 0.f;
+    }
 }
 
 // ---- the contraction -------------------------------------------------------------------
-// Running smallest scores of one row.  TRACK2 keeps the three smallest values and the
-// indices of the two smallest (so a near-tie can be settled by comparing two candidates);
-// without it only the two smallest values and the index of the smallest are kept and every
-// near-tie is re-evaluated against all centroids (cheaper per column; used when K*D is small).
+// Running smallest squared distances of one row, kept as integer KEYS: the fp32 bits of
+// d2 = ||z||^2 + ||c||^2 - 2 z.c with the low KEY_BITS replaced by the column's index inside
+// the 128-column accumulator tile.  Positive floats order like their bit patterns, so one
+// integer min/max both ranks the value and carries the index along (no compare+select per
+// column); dropping KEY_BITS mantissa bits moves a value by less than 2^-16 of itself, which the
+// near-tie bound absorbs.  A d2 that rounding made slightly negative is a negative integer: it
+// beats every positive key, and any two such values are closer than the near-tie bound, so the
+// exact fix-up decides between them.
+// TRACK2 keeps the three smallest keys (a near-tie between exactly two candidates is settled by
+// comparing those two); without it only the two smallest are kept and every near-tie is
+// re-evaluated against all centroids (cheaper per column; used when K*D is small).
+constexpr int KEY_BITS = 7;
+constexpr int KEY_MASK = ~((1 << KEY_BITS) - 1);
+constexpr int KEY_INF = 0x7fffffff;
+static_assert(BN == (1 << KEY_BITS), "a key's index field addresses one accumulator tile");
+
 template <bool TRACK2>
-struct Tracker {
-    float b0 = INFINITY, b1 = INFINITY, b2 = INFINITY;
-    int a0 = 0, a1 = 0;
-    __device__ __forceinline__ void add(float s, int col) {
-        if (TRACK2) {
-            b2 = fminf(b2, fmaxf(b1, s));
-            const bool c1 = s < b0, c2 = s < b1;
-            a1 = c1 ? a0 : (c2 ? col : a1);
-        }
-        b1 = fminf(b1, fmaxf(b0, s));
-        a0 = s < b0 ? col : a0;
-        b0 = fminf(b0, s);
+struct KeyTracker {
+    int b0 = KEY_INF, b1 = KEY_INF, b2 = KEY_INF;
+    // two more columns: five (eight with TRACK2) integer min/max operations per pair
+    __device__ __forceinline__ void add2(int k, int k2) {
+        const int lo = min(k, k2), hi = max(k, k2);
+        if (TRACK2) b2 = __vimin3_s32(b2, max(b1, lo), max(b0, hi));
+        b1 = __vimin3_s32(b1, max(b0, lo), hi);
+        b0 = min(b0, lo);
     }
     // fold another tracker over a disjoint set of columns into this one
-    __device__ __forceinline__ void merge(const Tracker& u) {
-        const float u2 = u.b2;
-        if (TRACK2) {
-            add(u.b0, u.a0);
-            add(u.b1, u.a1);
-            b2 = fminf(b2, fmaxf(b1, u2));
-        } else {
-            // values only: the second smallest of the union, the index of the smallest
-            const float lo = fminf(b0, u.b0), hi = fmaxf(b0, u.b0);
-            b1 = fminf(fminf(b1, u.b1), hi);
-            a0 = u.b0 < b0 ? u.a0 : a0;
-            b0 = lo;
-        }
+    __device__ __forceinline__ void merge(const KeyTracker& u) {
+        if (TRACK2) b2 = min(__vimin3_s32(b2, u.b2, max(b1, u.b0)), max(b0, u.b1));
+        b1 = __vimin3_s32(b1, u.b1, max(b0, u.b0));
+        b0 = min(b0, u.b0);
     }
 };
 
+// The smallest keys of a row across accumulator tiles, each with the tile it came from.
 template <bool TRACK2>
+struct RowBest {
+    int r0 = KEY_INF, r1 = KEY_INF, r2 = KEY_INF;
+    int t0 = 0, t1 = 0;
+    __device__ __forceinline__ void insert(int k, int tile) {
+        const bool c0 = k < r0, c1 = k < r1;
+        if (TRACK2) {
+            r2 = c1 ? r1 : min(r2, k);
+            t1 = c0 ? t0 : (c1 ? tile : t1);
+        }
+        r1 = c0 ? r0 : (c1 ? k : r1);
+        t0 = c0 ? tile : t0;
+        r0 = c0 ? k : r0;
+    }
+    __device__ __forceinline__ float value(int key) const { return __int_as_float(key & KEY_MASK); }
+    __device__ __forceinline__ int column(int key, int tile) const { return tile * BN + (key & ~KEY_MASK); }
+};
+
+template <bool TRACK2, bool F16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 assign_tc_kernel(const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled panels
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int D = p.D, nkb = D / KBF, nt_count = p.Kpad / BN;
-    const int nab = D <= 64 ? 2 : 1;                      // A (hi+lo) tiles that fit beside the accumulators in TMEM
+    const int D = p.D, nkb = p.nkb, nt_count = p.Kpad / BN;
+    const int DC = p.DC;                                  // TMEM columns of one A part (hi or lo)
+    const int nab = DC <= 64 ? 2 : 1;                     // A (hi+lo) tiles that fit beside the accumulators in TMEM
     const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
     unsigned char* st_base = smem;                                        // NSTAGE x STAGE
     float* xs = reinterpret_cast<float*>(smem + NSTAGE * STAGE);          // nxb x [BM][D+4]
     float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // [B][Kpad]
-    float* xnorm = cn + (size_t)p.B * p.Kpad;                             // [2][BM]
-    float* merge_buf = xnorm + 2 * BM;                                    // [2][BM][5]
+    float* cw = cn + (size_t)p.B * p.Kpad;                                // [B][Kpad]  (fp16 split only)
+    float* xnorm = cw + (F16 ? (size_t)p.B * p.Kpad : 0);                 // [2][BM]
+    float* xscale = xnorm + 2 * BM;                                       // [2][BM]  1 / (the row's power-of-two scale)
+    float* merge_buf = xscale + 2 * BM;                                   // [2][BM][5]
     uint64_t* bars = reinterpret_cast<uint64_t*>(merge_buf + 2 * BM * 5 + 2);   // (+2 floats: 8-byte alignment)
     // barrier indices
     enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 8, ACC_FULL = A_EMPTY + 8,
@@ -294,10 +408,10 @@ assign_tc_kernel(const TcParams p) {
 
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(BAR(B_FULL + s), 1); mbar_init(BAR(B_EMPTY + s), 1); }
-        for (int k = 0; k < 8; ++k) { mbar_init(BAR(A_FULL + k), 128); mbar_init(BAR(A_EMPTY + k), 1); }
+        for (int k = 0; k < 8; ++k) { mbar_init(BAR(A_FULL + k), 4); mbar_init(BAR(A_EMPTY + k), 1); }
         for (int k = 0; k < 2; ++k) {
-            mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 256);
-            mbar_init(BAR(XN_FULL + k), 128); mbar_init(BAR(XN_EMPTY + k), 128);
+            mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 8);
+            mbar_init(BAR(XN_FULL + k), 4); mbar_init(BAR(XN_EMPTY + k), 8);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -307,7 +421,10 @@ assign_tc_kernel(const TcParams p) {
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) cn[j] = p.cnorm[j];   // all instances' centroid norms
+    for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) {   // all instances' centroid norms (and weights)
+        cn[j] = p.cnorm[j];
+        if (F16) cw[j] = p.cweight[j];
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -347,7 +464,38 @@ assign_tc_kernel(const TcParams p) {
             }
             bar_sync_producers();                          // the staged tile is visible to all four warps
             const float* xr = xs + (size_t)buf * BM * xs_stride + (size_t)row_in_tile * xs_stride;
-            float xn = 0.f;
+            float xn = 0.f, rscale = 1.f;
+            const int ab = it % nab, use = it / nab;           // A buffer of this tile, how often it was used before
+            if (F16) {
+                // the row's own power-of-two scale (largest magnitude into [0.5, 1)) and its squared norm
+                float m = 0.f;
+                for (int q = 0; q < D / 4; ++q) {
+                    const float4 v = *reinterpret_cast<const float4*>(xr + 4 * q);
+                    xn = fmaf(v.x, v.x, xn); xn = fmaf(v.y, v.y, xn); xn = fmaf(v.z, v.z, xn); xn = fmaf(v.w, v.w, xn);
+                    m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+                }
+                const float sc = pow2_scale(m);
+                rscale = 1.f / sc;
+                for (int kb = 0; kb < nkb && ok; ++kb) {
+                    uint32_t hi[32], lo[32];
+                    const int nq = min(16, (D - kb * 64) / 4);     // float4 groups of this k-block that hold features
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (q < nq) v = *reinterpret_cast<const float4*>(xr + kb * 64 + 4 * q);
+                        split_f16x2(v.x * sc, v.y * sc, hi[2 * q], lo[2 * q]);
+                        split_f16x2(v.z * sc, v.w * sc, hi[2 * q + 1], lo[2 * q + 1]);
+                    }
+                    ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    TC_ST32(lane_addr + COL_A + ab * 2 * DC + kb * 32, hi);
+                    TC_ST32(lane_addr + COL_A + ab * 2 * DC + DC + kb * 32, lo);
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    tc_fence_before();
+                    mbar_arrive_warp(BAR(A_FULL + ab * 4 + kb));
+                }
+            } else {
             for (int kb = 0; kb < nkb && ok; ++kb) {
                 uint32_t hi[32], lo[32];
 #pragma unroll
@@ -361,15 +509,15 @@ assign_tc_kernel(const TcParams p) {
                         lo[4 * q + i] = to_tf32(f[i] - __uint_as_float(hi[4 * q + i]));
                     }
                 }
-                const int ab = it % nab, use = it / nab;       // A buffer of this tile, how often it was used before
                 ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                TC_ST32(lane_addr + COL_A + ab * 2 * D + kb * KBF, hi);
-                TC_ST32(lane_addr + COL_A + ab * 2 * D + D + kb * KBF, lo);
+                TC_ST32(lane_addr + COL_A + ab * 2 * DC + kb * KBF, hi);
+                TC_ST32(lane_addr + COL_A + ab * 2 * DC + DC + kb * KBF, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
-                mbar_arrive(BAR(A_FULL + ab * 4 + kb));
+                mbar_arrive_warp(BAR(A_FULL + ab * 4 + kb));
+            }
             }
             if (!ok) break;
             if (p.nxb == 1) {
@@ -379,83 +527,130 @@ assign_tc_kernel(const TcParams p) {
             ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
             if (!ok) break;
             xnorm[(it & 1) * BM + row_in_tile] = xn;
-            mbar_arrive(BAR(XN_FULL + (it & 1)));
+            xscale[(it & 1) * BM + row_in_tile] = rscale;
+            mbar_arrive_warp(BAR(XN_FULL + (it & 1)));
         }
         cp_async_wait<0>();
     } else if (warp < 12) {
         // ============================ epilogue ========================================
         // Two warps per TMEM lane quarter: `half` 0 takes columns [0,64) of every accumulator
-        // buffer, `half` 1 columns [64,128).  Each thread keeps four independent trackers
-        // (columns modulo 4) so that the min/max chains of consecutive columns overlap.
+        // buffer, `half` 1 columns [64,128).  Each thread keeps two independent key trackers per
+        // accumulator tile (alternate column pairs) and folds them into the row's running best
+        // after the accumulator buffer has been handed back to the MMA warp.
         const int ew = warp - 4, half = ew >> 2;
         const int row_in_tile = (ew & 3) * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)((ew & 3) * 32) << 16);
         uint32_t q = 0;
         int it = 0;
+        uint32_t r[2][32];                                   // two 32-column register buffers, reused in turn
+        bool pref = false;                                   // the next tile's first load is already in flight
         for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
             const int b = tile / p.tiles_per_inst, r0 = (tile - b * p.tiles_per_inst) * BM;
             const float* cnb = cn + (size_t)b * p.Kpad;            // squared norms of this instance's centroids
-            Tracker<TRACK2> t0, t1, t2, t3;
-            for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
-                const uint32_t buf = q & 1u;
-                ok = mbar_wait(BAR(ACC_FULL + buf), (q >> 1) & 1u, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t acc = lane_addr + COL_ACC + buf * BN + half * (BN / 2);
-                uint32_t r[2][32];
-                TC_LD32(acc, r[0]);
-#pragma unroll
-                for (int c = 0; c < BN / 64; ++c) {
-                    TC_WAIT_LD(r[c & 1]);
-                    if (c + 1 < BN / 64) TC_LD32(acc + (c + 1) * 32, r[(c + 1) & 1]);
-                    const int col0 = nt * BN + half * (BN / 2) + c * 32;
-                    const float* cnp = cnb + col0;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const float4 n4 = *reinterpret_cast<const float4*>(cnp + j);
-                        t0.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 0]), n4.x), col0 + j + 0);
-                        t1.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 1]), n4.y), col0 + j + 1);
-                        t2.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 2]), n4.z), col0 + j + 2);
-                        t3.add(fmaf(-2.f, __uint_as_float(r[c & 1][j + 3]), n4.w), col0 + j + 3);
-                    }
-                }
-                tc_fence_before();
-                mbar_arrive(BAR(ACC_EMPTY + buf));
-            }
-            if (!ok) break;
             // every epilogue thread takes the same waits in the same order, so a timeout takes
             // all of them out together and nobody is left at the named barrier below
             ok = mbar_wait(BAR(XN_FULL + (it & 1)), (uint32_t)((it >> 1) & 1), abort_flag);
             if (!ok) break;
-            t0.merge(t1);
-            t2.merge(t3);
-            t0.merge(t2);
-            // fold the upper half's tracker into the lower half's through shared memory
+            const float xn = xnorm[(it & 1) * BM + row_in_tile];
+            const float rscale = xscale[(it & 1) * BM + row_in_tile];
+            mbar_arrive_warp(BAR(XN_EMPTY + (it & 1)));
+            const float* cwb = cw + (size_t)b * p.Kpad;
+            RowBest<TRACK2> rb;
+            for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
+                const uint32_t buf = q & 1u;
+                const uint32_t acc = lane_addr + COL_ACC + buf * BN + half * (BN / 2);
+                if (!pref) {                                   // first 32 columns not requested yet
+                    ok = mbar_wait(BAR(ACC_FULL + buf), (q >> 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    TC_LD32(acc, r[0]);
+                }
+                pref = false;
+                KeyTracker<TRACK2> ta, tb;
+                const float* cnp = cnb + nt * BN + half * (BN / 2);
+                const float* cwp = cwb + nt * BN + half * (BN / 2);
+                // Two passes over a 32-column register buffer.  The first turns every accumulator value
+                // into its key in place: 32 independent short chains (load the column's constants,
+                // three fp32 operations, one logic operation), which the scheduler can overlap freely.
+                // The second feeds the keys to four independent trackers.
+                auto process = [&](uint32_t (&v)[32], int c) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 n4 = *reinterpret_cast<const float4*>(cnp + c * 32 + j);
+                        const int l = c * 32 + j;                  // column inside this thread's 64
+                        float d0, d1, d2, d3;
+                        if (F16) {      // undo the row's and the centroid's scales: d2 = ||z||^2 + ||c||^2 - 2 acc / (s_z s_c)
+                            const float4 w4 = *reinterpret_cast<const float4*>(cwp + c * 32 + j);
+                            d0 = fmaf(__uint_as_float(v[j + 0]) * rscale, w4.x, n4.x + xn);
+                            d1 = fmaf(__uint_as_float(v[j + 1]) * rscale, w4.y, n4.y + xn);
+                            d2 = fmaf(__uint_as_float(v[j + 2]) * rscale, w4.z, n4.z + xn);
+                            d3 = fmaf(__uint_as_float(v[j + 3]) * rscale, w4.w, n4.w + xn);
+                        } else {
+                            d0 = fmaf(-2.f, __uint_as_float(v[j + 0]), n4.x + xn);
+                            d1 = fmaf(-2.f, __uint_as_float(v[j + 1]), n4.y + xn);
+                            d2 = fmaf(-2.f, __uint_as_float(v[j + 2]), n4.z + xn);
+                            d3 = fmaf(-2.f, __uint_as_float(v[j + 3]), n4.w + xn);
+                        }
+                        const int k0 = (__float_as_int(d0) & KEY_MASK) | (l + 0);
+                        const int k1 = (__float_as_int(d1) & KEY_MASK) | (l + 1);
+                        const int k2 = (__float_as_int(d2) & KEY_MASK) | (l + 2);
+                        const int k3 = (__float_as_int(d3) & KEY_MASK) | (l + 3);
+                        ta.add2(k0, k1);
+                        tb.add2(k2, k3);
+                    }
+                };
+                TC_WAIT_LD(r[0]);
+                TC_LD32(acc + 32, r[1]);
+                process(r[0], 0);
+                TC_WAIT_LD(r[1]);
+                // both loads have landed: the accumulator goes back to the MMA warp before its second
+                // half is even looked at
+                tc_fence_before();
+                mbar_arrive_warp(BAR(ACC_EMPTY + buf));
+                // If the next accumulator tile is already complete (the usual case once the epilogue is
+                // what the MMA warp waits for), request its first 32 columns now: the load then runs
+                // under the arithmetic below instead of in front of the next tile's.
+                const bool more = nt + 1 < nt_count || tile + stride < p.total_tiles;
+                if (more) {
+                    const uint32_t qn = q + 1u, bufn = qn & 1u;
+                    if (__all_sync(0xffffffffu, mbar_try(BAR(ACC_FULL + bufn), (qn >> 1) & 1u))) {
+                        tc_fence_after();
+                        TC_LD32(lane_addr + COL_ACC + bufn * BN + half * (BN / 2), r[0]);
+                        pref = true;
+                    }
+                }
+                process(r[1], 1);
+                ta.merge(tb);
+                const int hbit = half * (BN / 2);                  // the upper half's columns start at 64
+                rb.insert(ta.b0 | hbit, nt);
+                rb.insert(ta.b1 | hbit, nt);
+                if (TRACK2) rb.insert(ta.b2 | hbit, nt);
+            }
+            if (!ok) break;
+            // fold the upper half's running best into the lower half's through shared memory
             float* mg = merge_buf + ((size_t)(it & 1) * BM + row_in_tile) * 5;
             if (half == 1) {
-                mg[0] = t0.b0; mg[1] = t0.b1; mg[2] = t0.b2;
-                mg[3] = __int_as_float(t0.a0); mg[4] = __int_as_float(t0.a1);
+                mg[0] = __int_as_float(rb.r0); mg[1] = __int_as_float(rb.r1); mg[2] = __int_as_float(rb.r2);
+                mg[3] = __int_as_float(rb.t0); mg[4] = __int_as_float(rb.t1);
             }
             asm volatile("bar.sync 2, 256;" ::: "memory");
             if (half == 1) continue;
-            {
-                Tracker<TRACK2> u;
-                u.b0 = mg[0]; u.b1 = mg[1]; u.b2 = mg[2];
-                u.a0 = __float_as_int(mg[3]); u.a1 = __float_as_int(mg[4]);
-                t0.merge(u);
-            }
-            const float xn = xnorm[(it & 1) * BM + row_in_tile];
-            mbar_arrive(BAR(XN_EMPTY + (it & 1)));
+            rb.insert(__float_as_int(mg[0]), __float_as_int(mg[3]));
+            rb.insert(__float_as_int(mg[1]), __float_as_int(mg[4]));
+            if (TRACK2) rb.r2 = min(rb.r2, __float_as_int(mg[2]));
             const int row = r0 + row_in_tile;
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
-                p.labels[flat] = t0.a0;
-                if (p.approx) p.approx[flat] = xn + t0.b0;
-                const float delta = p.eps * (xn + cnb[t0.a0]);
-                if (t0.b1 - t0.b0 <= delta) {
-                    if (TRACK2 && t0.b2 - t0.b0 > delta) {     // exactly two candidates: compare them exactly
+                const int a0 = rb.column(rb.r0, rb.t0);
+                const float b0 = rb.value(rb.r0), b1 = rb.value(rb.r1);
+                p.labels[flat] = a0;
+                if (p.approx) p.approx[flat] = b0;
+                // near-tie bound: the split product's error plus what the dropped key bits can hide
+                const float delta = p.eps * (xn + cnb[a0]) + 1.52587890625e-5f * fabsf(b1);
+                if (fabsf(b1 - b0) <= delta) {
+                    if (TRACK2 && fabsf(rb.value(rb.r2) - b0) > delta) {   // exactly two candidates: compare them exactly
                         const int slot = atomicAdd(p.flag_count, 1);
-                        p.pair_rows[slot] = make_int2((int)flat, t0.a1);
+                        p.pair_rows[slot] = make_int2((int)flat, rb.column(rb.r1, rb.t1));
                     } else {                                   // three or more (or unknown): exact scan over all K
                         const int slot = atomicAdd(p.flag_count + 1, 1);
                         p.full_rows[slot] = (int32_t)flat;
@@ -463,6 +658,7 @@ assign_tc_kernel(const TcParams p) {
                 }
             }
         }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");   // no load may outlive the role (abort path)
     } else if (warp == 12) {
         // ============================ MMA issuer ======================================
         // One elected lane issues every MMA, so this instruction stream is the critical path of
@@ -473,13 +669,14 @@ assign_tc_kernel(const TcParams p) {
         {
             uint32_t s = 0, ph = 0, q = 0;
             int it = 0;
+            constexpr uint32_t IDESC = F16 ? IDESC_F16 : IDESC_TF32;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
             const uint32_t desc_hi32 = (uint32_t)(desc0 >> 32);
             const uint32_t desc_lo32 = (uint32_t)desc0;
             const int ring = p.resident ? nt_count * nkb : NSTAGE;
             for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
                 const int ab = it % nab, use = it / nab;
-                const uint32_t a_base = tmem + COL_A + ab * 2 * D;
+                const uint32_t a_base = tmem + COL_A + ab * 2 * DC;
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
@@ -496,18 +693,18 @@ assign_tc_kernel(const TcParams p) {
                             if (!ok) break;
                         }
                         tc_fence_after();
-                        const uint32_t a_hi = a_base + kb * KBF, a_lo = a_hi + D;
+                        const uint32_t a_hi = a_base + kb * 32, a_lo = a_hi + DC;
                         const uint32_t blo = desc_lo32 + s * (STAGE >> 4);        // this stage's hi panel
                         if (elect_one()) {
                         // first k-step: the very first product of an accumulator tile overwrites it
-                        tc_mma_ts(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, kb != 0 ? 1u : 0u);
-                        tc_mma_ts_acc(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
-                        tc_mma_ts_acc(d_tmem, a_hi, mk_desc(blo, desc_hi32), IDESC);
+                        tc_mma_ts<F16>(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, kb != 0 ? 1u : 0u);
+                        tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
+                        tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo, desc_hi32), IDESC);
 #pragma unroll
                         for (int k8 = 1; k8 < KBF / 8; ++k8) {
-                            tc_mma_ts_acc(d_tmem, a_lo + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
-                            tc_mma_ts_acc(d_tmem, a_hi + k8 * 8, mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
-                            tc_mma_ts_acc(d_tmem, a_hi + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                            tc_mma_ts_acc<F16>(d_tmem, a_lo + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                            tc_mma_ts_acc<F16>(d_tmem, a_hi + k8 * 8, mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
+                            tc_mma_ts_acc<F16>(d_tmem, a_hi + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
                         }
                         if (!p.resident) tc_commit(BAR(B_EMPTY + s));      // stage reusable once these MMAs retire
                         if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + ab * 4 + kb));  // A panel reusable
@@ -772,11 +969,11 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
     }
 }
 
-size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb) {
+size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool f16) {
     size_t s = 1024;                                       // alignment slack
     s += (size_t)NSTAGE * STAGE;
     s += (size_t)nxb * BM * (D + 4) * 4;
-    s += (size_t)Kpad * 4 + 2 * BM * 4 + (2 * BM * 5 + 2) * 4;
+    s += (size_t)Kpad * 4 * (f16 ? 2 : 1) + 4 * BM * 4 + (2 * BM * 5 + 2) * 4;
     s += 40 * 8 + 16;                                      // barriers, TMEM slot, abort flag
     return s;
 }
@@ -787,7 +984,7 @@ size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb) {
 // B image | centroid norms | queue counter | queue
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
     const size_t Kpad = (size_t)(K + BN - 1) / BN * BN;
-    return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 8) +
+    return kb_align256(B * Kpad * D * 8) + 2 * kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 8) +
            kb_align256((size_t)B * N * 4);
 }
 
@@ -796,7 +993,7 @@ bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K) {
     if (D % KBF != 0 || D > 128 || K < 1 || K > 8192 || B < 1) return false;
     const long Kpad = (long)(K + BN - 1) / BN * BN;
     if (Kpad * B > 8192) return false;                     // the norms of every instance stay in shared memory
-    return tc_smem_bytes(D, (int)(Kpad * B), 1) <= (size_t)ctx->max_smem_optin;
+    return tc_smem_bytes(D, (int)(Kpad * B), 1, true) <= (size_t)ctx->max_smem_optin;
 }
 // what the automatic choice sends there: enough centroids to fill an accumulator tile
 // and enough rows for the contraction to outweigh the preparation and fix-up launches
@@ -812,33 +1009,46 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     const int Kpad = (K + BN - 1) / BN * BN;
     unsigned char* bimg = reinterpret_cast<unsigned char*>(ws);
     float* cnorm = reinterpret_cast<float*>(ws + kb_align256((size_t)B * Kpad * D * 8));
-    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
+    float* cweight = reinterpret_cast<float*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
+    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cweight) + kb_align256((size_t)B * Kpad * 4));
     int2* pair_rows = reinterpret_cast<int2*>(reinterpret_cast<char*>(flag_count) + 256);
     int32_t* full_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(pair_rows) + kb_align256((size_t)B * N * 8));
 
-    tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, c, bimg, cnorm, flag_count);
+    // the split: fp16 hi/lo (kind::f16, 16 features per instruction) unless the tf32 split is forced
+    const bool f16 = ctx->assign_path != 3;
+    const int nkb = f16 ? (D + 63) / 64 : D / KBF;
+    if (f16)
+        tc_prep_kernel<true><<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, cweight, flag_count);
+    else
+        tc_prep_kernel<false><<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, cweight, flag_count);
     KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
 
     TcParams p;
     p.B = B; p.N = N; p.D = D; p.K = K; p.Kpad = Kpad;
+    p.nkb = nkb;
+    p.DC = f16 ? 32 * nkb : D;
     p.tiles_per_inst = (N + BM - 1) / BM;
     p.total_tiles = p.tiles_per_inst * B;
-    p.nxb = tc_smem_bytes(D, Kpad * B, 2) <= (size_t)ctx->max_smem_optin ? 2 : 1;
+    p.nxb = tc_smem_bytes(D, Kpad * B, 2, f16) <= (size_t)ctx->max_smem_optin ? 2 : 1;
     p.eps = eps;
-    p.resident = (B == 1 && (Kpad / BN) * (D / KBF) <= NSTAGE) ? 1 : 0;
-    p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.labels = labels; p.approx = approx;
+    p.resident = (B == 1 && (Kpad / BN) * nkb <= NSTAGE) ? 1 : 0;
+    p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.cweight = cweight; p.labels = labels; p.approx = approx;
     p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
-    const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb);
+    const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb, f16);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
     // with few features per row the epilogue's per-column cost is what limits the kernel:
     // track less there and let the (cheap, K*D is small) full re-evaluation settle near-ties
-    if (D >= 96) {
-        KB_SMEM_OPTIN(ctx, assign_tc_kernel<true>, smem);
-        assign_tc_kernel<true><<<grid, TC_THREADS, smem, ctx->stream>>>(p);
-    } else {
-        KB_SMEM_OPTIN(ctx, assign_tc_kernel<false>, smem);
-        assign_tc_kernel<false><<<grid, TC_THREADS, smem, ctx->stream>>>(p);
-    }
+    const bool track2 = D >= 96;
+#define KB_TC_LAUNCH(T2, F)                                                                    \
+    do {                                                                                       \
+        KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F>), smem);                                   \
+        assign_tc_kernel<T2, F><<<grid, TC_THREADS, smem, ctx->stream>>>(p);                   \
+    } while (0)
+    if (track2 && f16) KB_TC_LAUNCH(true, true);
+    else if (track2) KB_TC_LAUNCH(true, false);
+    else if (f16) KB_TC_LAUNCH(false, true);
+    else KB_TC_LAUNCH(false, false);
+#undef KB_TC_LAUNCH
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
     const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
@@ -863,3 +1073,4 @@ kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const
     KB_LAUNCH_CHECK(ctx, "assign_finish_kernel");
     return KB_OK;
 }
+

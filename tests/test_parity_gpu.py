@@ -369,9 +369,10 @@ TC_CASES = [(1, 4096, 32, 128), (1, 5000, 64, 256), (2, 3000, 128, 200), (1, 409
             (1, 20000, 128, 1024)]
 
 
+@pytest.mark.parametrize("path", [2, 3], ids=["f16x3", "tf32x3"])
 @pytest.mark.parametrize("B,N,D,K", TC_CASES)
-def test_assign_tensor_path(kbx, B, N, D, K):
-    """kb_cluster_assign forced onto the tcgen05 kernel: same rules as the fp32 path."""
+def test_assign_tensor_path(kbx, B, N, D, K, path):
+    """kb_cluster_assign forced onto the tcgen05 kernel (fp16 or tf32 split): same rules as the fp32 path."""
     cfg = wl.scaled(wl.CONFIGS["large"], B=B, N=N, D=D, K=K, components=max(8, K // 2), S=2)
     inp = wl.make_inputs(cfg, seed=N + K)
     z, _, _ = oracle.normalize(inp["x"])
@@ -379,11 +380,11 @@ def test_assign_tensor_path(kbx, B, N, D, K):
     c = z[:, rng.choice(N, K, replace=False)] + (0.02 * rng.standard_normal((B, K, D))).astype(np.float32)
     c[:, K - 1] = c[:, 0]                       # exact duplicate: gap 0, resolved by the exact re-evaluation
     ws(kbx, B, N, D, K, 1)
-    kbx.set_assign_options(path=2)
+    kbx.set_assign_options(path=path)
     try:
         labels, d2, inertia, rep = empty((B, N), torch.int32), empty((B, N)), empty((B,)), empty((B, K), torch.int32)
         kbx.cluster_assign(dev(z), dev(c), labels, d2, inertia, rep)
-        assert kbx.assign_path() == 2
+        assert kbx.assign_path() == path
         approx, flagged, lab2 = empty((B, N)), empty((2,), torch.int32), empty((B, N), torch.int32)
         kbx.assign_tc_probe(dev(z), dev(c), lab2, approx, flagged)
     finally:
@@ -402,10 +403,13 @@ def test_assign_tensor_path(kbx, B, N, D, K):
     xn = (z.astype(np.float64) ** 2).sum(-1)
     cnn = (c.astype(np.float64) ** 2).sum(-1)
     scale = xn + np.take_along_axis(cnn, ref["labels"].astype(np.int64), axis=1)
-    err = np.abs(host(approx).astype(np.float64) - ref["best"])[same] / scale[same]
+    # (the ranked value also drops its low 7 mantissa bits, which hold the column index: up to 2^-16 of itself,
+    # a term the kernel's near-tie bound adds on top of eps)
+    err = (np.abs(host(approx).astype(np.float64) - ref["best"]) - ref["best"] / 65536)[same] / scale[same]
     frac, frac_full = host(flagged) / (B * N)
-    print(f"[tc B={B} N={N} D={D} K={K}] near-ties={ties} pair-checked={frac:.5f} fully re-evaluated={frac_full:.5f} "
-          f"max |d2_ranked - d2_exact| / (|z|^2+|c|^2) = {err.max():.3e} (eps = {1 / 65536:.3e})")
+    print(f"[tc path={path} B={B} N={N} D={D} K={K}] near-ties={ties} pair-checked={frac:.5f} "
+          f"fully re-evaluated={frac_full:.5f} max (|d2_ranked - d2_exact| - 2^-16 d2) / (|z|^2+|c|^2) = {err.max():.3e} "
+          f"(eps = {1 / 65536:.3e})")
     assert err.max() < 0.25 / 65536               # the re-evaluation bound covers the ranking error with margin
 
 
