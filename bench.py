@@ -334,13 +334,16 @@ def run_ours(args, cfg):
     dk = kernels[dominant]
     hbm_time = alg[dominant]["bytes"] / (hbm * 1e9)
     alu_time = alg[dominant]["flops"] / (ffma_tflops * 1e12)
-    tf32_peak = peaks["bf16_tflops"] * 0.5          # measured bf16 burst x nominal tf32/bf16 ratio
-    if dominant == "assign" and assign_path == 2:
-        # 3xTF32: three tensor-core products per fp32-equivalent product
-        roof = {"bound": "tensor", "achieved": dk["TFLOPs"], "peak": tf32_peak / 3.0, "unit": "TFLOP/s",
-                "frac": dk["TFLOPs"] / (tf32_peak / 3.0), "traffic": None,
-                "kernel": "kb_cluster_assign (tcgen05 kind::tf32, 3xTF32 split; prep + contraction + fix-up per call)",
-                "peak_source": f"{peaks['source']} bf16 GEMM peak x 0.5 (tf32) / 3 (split products), fp32-equivalent",
+    if dominant == "assign" and assign_path in (2, 3):
+        # three tensor-core products per fp32-equivalent product.  fp16 split (path 2): the measured bf16
+        # GEMM peak is the 16-bit tensor rate itself; tf32 split (path 3): half of it (nominal ratio).
+        kind_peak = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5)
+        split = "fp16 hi/lo split, kind::f16" if assign_path == 2 else "3xTF32, kind::tf32"
+        roof = {"bound": "tensor", "achieved": dk["TFLOPs"], "peak": kind_peak / 3.0, "unit": "TFLOP/s",
+                "frac": dk["TFLOPs"] / (kind_peak / 3.0), "traffic": None,
+                "kernel": f"kb_cluster_assign (tcgen05 {split}; prep + contraction + fix-up per call)",
+                "peak_source": f"{peaks['source']} bf16 GEMM peak" + (" x 0.5 (tf32)" if assign_path == 3 else "") +
+                               " / 3 (split products), fp32-equivalent",
                 "algorithmic_flops_per_launch": alg["assign"]["flops"],
                 "executed_tensor_TFLOPs": 3.0 * dk["TFLOPs"]}
     elif dominant in ("assign", "fit") and alu_time > hbm_time:

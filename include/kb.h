@@ -189,13 +189,20 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
  *   path: 0 = automatic (tensor cores when K >= 128, D a multiple of 32 and
  *             <= 128 and there are at least 4096 rows; else the fp32 row-wise
  *             kernel), 1 = always the fp32 row-wise kernel, 2 = always the
- *             tensor-core kernel (KB_ERR_UNSUPPORTED where it cannot run).
- *   tc_eps:   the tensor-core kernel ranks centroids by ||c||^2 - 2 z.c
- *             evaluated as a 3xTF32 split product; a row whose best and
- *             second-best scores differ by no more than
- *             tc_eps * (||z||^2 + ||c||^2) is re-evaluated exactly (direct
- *             form, fp32).  <= 0 keeps the default 2^-16.
- * kb_get_assign_path reports what the last kb_cluster_assign ran (1 or 2). */
+ *             tensor-core kernel with the fp16 split (what "automatic" picks;
+ *             KB_ERR_UNSUPPORTED where it cannot run), 3 = the tensor-core
+ *             kernel with the tf32 split (3xTF32).
+ *             Both splits carry 22 significant bits per operand (two pieces of
+ *             11 bits) and three products per k-step; the fp16 one runs at
+ *             twice the tensor rate and scales rows and centroids by exact
+ *             powers of two to stay inside fp16's range.
+ *   tc_eps:   the tensor-core kernel ranks centroids by the split product's
+ *             squared distance; a row whose best and second-best values differ
+ *             by no more than tc_eps * (||z||^2 + ||c||^2) (||c||^2: of the
+ *             chosen centroid for the tf32 split, the largest of the instance
+ *             for the fp16 split) is re-evaluated exactly (direct form, fp32).
+ *             <= 0 keeps the default 2^-16.
+ * kb_get_assign_path reports what the last kb_cluster_assign ran (1, 2 or 3). */
 kb_status kb_set_assign_options(kb_ctx* ctx, int path, float tc_eps);
 kb_status kb_get_assign_path(kb_ctx* ctx, int* out);
 

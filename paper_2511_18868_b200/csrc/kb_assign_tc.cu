@@ -1,34 +1,46 @@
-// kb_cluster_assign, tensor-core path (sm_100a: tcgen05.mma kind::tf32, TMEM).
+// kb_cluster_assign, tensor-core path (sm_100a: tcgen05.mma, TMEM).
 //
-// The assignment argmin_j ||z - c_j||^2 = argmin_j (||c_j||^2 - 2 z.c_j) is a
-// dense contraction Z[N x D] . C^T[D x K] when N*K*D is large.  It runs on the
-// 5th-generation tensor cores as a 3xTF32 split product (hi.hi + hi.lo + lo.hi,
-// each operand split into two TF32 pieces by round-to-nearest), fp32 accumulate:
+// The assignment argmin_j ||z - c_j||^2 is a dense contraction Z[N x D] . C^T[D x K] when
+// N*K*D is large.  It runs on the 5th-generation tensor cores as a three-product split
+// (hi.hi + hi.lo + lo.hi, each operand split into two pieces of 11 significant bits by
+// round-to-nearest, 22 bits in all), fp32 accumulate.  Two splits are built:
 //
-//   * A = a 128-row tile of Z, split hi/lo in registers and stored in TENSOR
-//     MEMORY (tcgen05.st); the MMA reads it from there (no shared-memory traffic
-//     for A, and the three products of a k-step reuse it).
-//   * B = 128 centroids x 32 features per stage, pre-split hi/lo by a small
-//     kernel into 128-byte-swizzled K-major panels, so a stage is one linear
-//     32 KB bulk copy (cp.async.bulk + mbarrier), 4-stage ring, re-read from L2
-//     by every CTA (no multicast of any kind).
-//   * accumulators: two 128 x 128 fp32 buffers in TMEM; the epilogue warps read
-//     one with tcgen05.ld while the MMA fills the other.
-//   * epilogue: score = ||c||^2 - 2 acc, running (best, second best, argbest) per
-//     row across all centroid tiles (plus the runner-up's index and the third
-//     smallest score).  A row whose runner-up lies inside the error bound of the
-//     split product is queued and decided in the exact direct form by a fix-up
-//     kernel (two candidates: a warp compares them; three or more: all K are
-//     re-evaluated), so labels follow the fp32 direct-form distances wherever it
-//     matters.
+//   fp16 (default, kind::f16, 16 features per instruction).  fp16 and tf32 carry the same 11
+//     significant bits, so the split is as exact as the tf32 one at half the tensor time.  fp16's
+//     narrow exponent is handled by exact power-of-two scales: one per row (s_z), one per
+//     instance for its centroids (s_c).  The constant terms ride along as 16 extra features
+//     (pieces of s_z s_c ||z||^2 against 1, s_z / s_c against pieces of s_c^2 ||c||^2), so an
+//     accumulator entry is g_i d2(i, j) with g_i = s_z s_c > 0 and the epilogue ranks the
+//     accumulator as it is: no per-column constants, no floating-point work per column.
+//   tf32 (kind::tf32, 8 features per instruction; kb_set_assign_options path 3).  No scales; the
+//     epilogue forms ||z||^2 + ||c||^2 - 2 acc per column from the norms kept in shared memory.
+//
+//   * A = a 128-row tile of Z.  Every producer thread owns one row: it requests the row with one
+//     bulk copy into its slot of the staging buffer, splits it hi/lo in registers and stores it
+//     in TENSOR MEMORY (tcgen05.st); the MMA reads A from there (no shared-memory traffic for A,
+//     and the three products of a k-step reuse it).
+//   * B = 128 centroids x one 128-byte swizzle row of features per stage, pre-split hi/lo by a
+//     small kernel into 128-byte-swizzled K-major panels, so a stage is one linear 32 KB bulk
+//     copy (cp.async.bulk + mbarrier; the fp16 stage of a tile's first k-block also brings the
+//     tile's 4 KB constant-term operand, K-major without swizzle), 4-stage ring, re-read from L2
+//     by every CTA (no multicast of any kind).  The whole image stays resident when it fits.
+//   * accumulators: two 128 x 128 fp32 buffers in TMEM; the epilogue warps read one with
+//     tcgen05.ld while the MMA fills the other.
+//   * epilogue: every value becomes an integer key (fp32 bits, low 7 bits replaced by the column
+//     index), so integer min/max rank value and index together; per row the three smallest keys
+//     are kept across all centroid tiles.  A row whose runner-up lies inside the error bound of
+//     the split product is queued and decided in the exact direct form by a fix-up kernel (two
+//     candidates: a warp compares them; three or more: all K are re-evaluated), so labels follow
+//     the fp32 direct-form distances wherever it matters.
 //
 // Roles in a 448-thread persistent CTA (one per SM):
-//   warps 0-3   A producers  (cp.async prefetch of the next Z tile -> split -> TMEM)
-//   warps 4-11  epilogue     (TMEM -> registers -> argmin; two warps per lane quarter)
+//   warps 0-3   A producers  (bulk copy of the next Z tile -> split -> TMEM)
+//   warps 4-11  epilogue     (TMEM -> registers -> keys -> argmin; two warps per lane quarter)
 //   warp  12    MMA issuer   (one elected lane), owns the TMEM allocation
 //   warp  13    B loader     (one elected lane)
-// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all
-// roles drain, TMEM is released and the device status word reports a timeout.
+// The roles meet only at mbarriers (one arrival per warp).  Every wait is bounded and suspends
+// the waiting thread between polls; on expiry the CTA raises an abort flag, all roles drain,
+// copies in flight are awaited, TMEM is released and the device status word reports a timeout.
 #include "kb_internal.cuh"
 #include <cuda_fp16.h>
 
@@ -39,11 +51,14 @@ constexpr int BN = 128;            // centroids per accumulator buffer
 constexpr int KBF = 32;            // floats per k-block (one 128-byte swizzle row)
 constexpr int PANEL = BN * KBF * 4;      // 16 KB: one hi or lo panel
 constexpr int STAGE = 2 * PANEL;         // hi + lo
+constexpr int EXT = 4096;                // fp16 split: the constant-term operand of one centroid tile (128 x 16 halfs)
+constexpr int SLOT_F16 = STAGE + EXT;    // a stage slot of the fp16 kernel (a multiple of 1024 bytes)
+constexpr int XCOLS = 8;                 // TMEM columns of a row's constant-term operand (16 halfs)
 constexpr int NSTAGE = 4;
 constexpr int TC_THREADS = 448;
 constexpr int TMEM_COLS = 512;
 constexpr int COL_ACC = 0;         // two accumulators: columns [0,128) and [128,256)
-constexpr int COL_A = 256;         // A buffer i: hi at [256 + 2iD, +D), lo at [256 + 2iD + D, +D); two buffers when D <= 64
+constexpr int COL_A = 256;         // A buffers from here: hi part | lo part (| constant terms), two buffers when they fit
 constexpr uint32_t WAIT_LIMIT = 1u << 19;          // polls of a bounded wait, each suspended for up to WAIT_SUSPEND_NS
 constexpr uint32_t WAIT_SUSPEND_NS = 2000;
 constexpr int STATUS_TIMEOUT = 0x100;
@@ -110,14 +125,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bar_sync_producers() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -238,7 +245,8 @@ struct TcParams {
     const float* z;
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
     const float* cnorm;            // [B][Kpad]
-    const float* cweight;          // [B][Kpad]  -2 / (the centroid's power-of-two scale)
+    const unsigned char* bext;     // fp16 split: [B][NT][EXT] constant-term operand of every centroid tile
+    const float* inst;             // fp16 split: [B][2] the instance's centroid scale s_c and its largest ||c||^2
     int32_t* labels;
     float* approx;                 // optional: ||z||^2 + best score (expanded-form d^2), diagnostics
     int* flag_count;               // [0]: rows queued for a two-candidate check, [1]: for a full re-evaluation
@@ -268,60 +276,125 @@ __device__ __forceinline__ void split_f16x2(float a, float b, uint32_t& hi, uint
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// One warp per centroid: lane q owns the 16-byte chunk q of the fp32 row (D <= 128).
-//   F16 = false: tf32 hi/lo panels, 32 features per 128-byte swizzle row, weight -2
-//   F16 = true : fp16 hi/lo panels of the centroid scaled by its own power of two, 64 features
-//                per 128-byte swizzle row (features past D are zero), weight -2 / scale
-template <bool F16>
+// tf32 split: one warp per centroid, lane q owns the 16-byte chunk q of the fp32 row (D <= 128);
+// hi/lo panels with 32 features per 128-byte swizzle row, squared norms in double.
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
-               float* __restrict__ cnorm, float* __restrict__ cweight, int* __restrict__ flag_count) {
+               float* __restrict__ cnorm, int* __restrict__ flag_count) {
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
     const int b = blockIdx.y;
     const int nt = Kpad / BN;
     const int lane = threadIdx.x & 31;
     const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (j >= Kpad) return;
-    const int fpr = F16 ? 64 : 32;                         // features per swizzle row
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (j < K && lane < D / 4) v = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)b * K + j) * D) + lane);
     const float f[4] = {v.x, v.y, v.z, v.w};
     double sq = 0.0;
-    float m = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) { sq += (double)f[i] * (double)f[i]; m = fmaxf(m, fabsf(f[i])); }
+    for (int i = 0; i < 4; ++i) sq += (double)f[i] * (double)f[i];
     sq = kb_warp_sum(sq);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    const float sc = F16 ? pow2_scale(m) : 1.f;
-    if (lane < nkb * fpr / 4) {
-        const int kb = (4 * lane) / fpr, within = 4 * lane - kb * fpr;     // feature offset inside the swizzle row
+    if (lane < nkb * 8) {
+        const int kb = lane >> 3, c = lane & 7;
         const int tile = j / BN, r = j - tile * BN;
-        const int bytes_in_row = within * (F16 ? 2 : 4);
-        const int chunk = bytes_in_row >> 4;
         const size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
-                           ((chunk ^ (r & 7)) << 4) + (bytes_in_row & 15);
-        if (F16) {
-            uint32_t h0, l0, h1, l1;
-            split_f16x2(f[0] * sc, f[1] * sc, h0, l0);
-            split_f16x2(f[2] * sc, f[3] * sc, h1, l1);
-            *reinterpret_cast<uint2*>(bimg + off) = make_uint2(h0, h1);
-            *reinterpret_cast<uint2*>(bimg + off + PANEL) = make_uint2(l0, l1);
-        } else {
-            uint32_t hi[4], lo[4];
+                           ((c ^ (r & 7)) << 4);
+        uint32_t hi[4], lo[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                hi[i] = to_tf32(f[i]);
-                lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
-            }
-            *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        for (int i = 0; i < 4; ++i) {
+            hi[i] = to_tf32(f[i]);
+            lo[i] = to_tf32(f[i] - __uint_as_float(hi[i]));
+        }
+        *reinterpret_cast<uint4*>(bimg + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(bimg + off + PANEL) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    if (lane == 0) cnorm[(size_t)b * Kpad + j] = j < K ? (float)sq : INFINITY;   // padding can never win
+}
+
+// Three fp16 pieces of a non-negative fp32 value (33 significant bits; a piece that falls below
+// fp16's range simply contributes less, an absolute error far below the ranking bound).
+__device__ __forceinline__ void split3_f16(float v, __half& a, __half& b, __half& c) {
+    a = __float2half_rn(v);
+    const float r1 = v - __half2float(a);
+    b = __float2half_rn(r1);
+    c = __float2half_rn(r1 - __half2float(b));
+}
+__device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
+    return (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
+}
+
+// Preparation for the fp16 split with the constant terms folded into the product.
+// With one power-of-two scale s_c per instance (largest |coordinate| of its centroids into
+// [0.5, 1)) and one scale s_z per row, the tensor core is given
+//     A row  i : s_z z_i (hi, lo)           | pieces of s_z s_c ||z_i||^2 | s_z / s_c (three times)
+//     B row  j : -2 s_c c_j (hi, lo)        | 1, 1, 1                     | pieces of s_c^2 ||c_j||^2
+// so that one accumulator entry is  s_z s_c (||z_i||^2 + ||c_j||^2 - 2 z_i.c_j)  =  g_i d2(i, j)  with
+// g_i > 0: the epilogue ranks the accumulator as it is.  This kernel writes the B side:
+//   bimg  [B][NT][nkb][hi panel | lo panel]   128-byte-swizzled K-major panels, 64 features per row
+//   bext  [B][NT][EXT]   the 16 extra features of each centroid, K-major without swizzle
+//                        (8-row x 16-byte core matrices: k-halves 128 bytes apart, row groups 256)
+//   inst  [B][2]         s_c and the largest ||c_j||^2 of the instance
+// Every block first scans its instance's centroids for the two maxima (the table is small and
+// sits in L2), then converts its share of the centroids: one warp per centroid, lane q owns the
+// 16-byte chunk q of the fp32 row (D <= 128).
+__global__ void __launch_bounds__(256)
+tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
+                   unsigned char* __restrict__ bext, float* __restrict__ inst, int* __restrict__ flag_count) {
+    __shared__ float s_m[8];
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
+    const int b = blockIdx.y, nt = Kpad / BN;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float* cb = cent + (size_t)b * K * D;
+    // largest |coordinate| of the instance's centroids: every block scans the whole table (coalesced,
+    // all loads independent), so that all of them derive the same scale without a grid-wide step
+    float m = 0.f;
+    {
+        const float4* c4 = reinterpret_cast<const float4*>(cb);
+        const int n4 = K * D / 4;
+        for (int e = threadIdx.x; e < n4; e += 256) {
+            const float4 v = __ldg(c4 + e);
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
         }
     }
-    if (lane == 0) {
-        cnorm[(size_t)b * Kpad + j] = j < K ? (float)sq : INFINITY;   // padding can never win
-        cweight[(size_t)b * Kpad + j] = j < K ? -2.f / sc : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) s_m[warp] = m;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = fmaxf(m, s_m[w]);
+    const float sc = pow2_scale(m);
+    if (blockIdx.x == 0 && threadIdx.x == 0) inst[2 * b] = sc;
+    float nmax = 0.f;                                      // largest ||c_j||^2 among this warp's centroids
+
+    for (int j = blockIdx.x * 8 + warp; j < Kpad; j += gridDim.x * 8) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < K && lane < D / 4) v = __ldg(reinterpret_cast<const float4*>(cb + (size_t)j * D) + lane);
+        const double sq = kb_warp_sum((double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w);
+        nmax = fmaxf(nmax, (float)sq * 1.0000005f);
+        const int tile = j / BN, r = j - tile * BN;
+        if (lane < nkb * 16) {
+            const int kb = lane >> 4, within = (lane & 15) * 8;            // byte offset inside the 128-byte row
+            const size_t off = (((size_t)b * nt + tile) * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
+                               (((within >> 4) ^ (r & 7)) << 4) + (within & 15);
+            const float w = -2.f * sc;
+            uint32_t h0, l0, h1, l1;
+            split_f16x2(v.x * w, v.y * w, h0, l0);
+            split_f16x2(v.z * w, v.w * w, h1, l1);
+            *reinterpret_cast<uint2*>(bimg + off) = make_uint2(h0, h1);
+            *reinterpret_cast<uint2*>(bimg + off + PANEL) = make_uint2(l0, l1);
+        }
+        if (lane == 0) {
+            const __half one = __float2half_rn(1.f), zero = __float2half_rn(0.f);
+            __half q0 = __float2half_rn(INFINITY), q1 = zero, q2 = zero;   // a padding centroid can never win
+            if (j < K) split3_f16((float)((double)sc * (double)sc * sq), q0, q1, q2);
+            unsigned char* e = bext + ((size_t)b * nt + tile) * EXT + (size_t)(r >> 3) * 256 + (r & 7) * 16;
+            *reinterpret_cast<uint4*>(e) = make_uint4(pack_h2(one, one), pack_h2(one, q0), pack_h2(q1, q2), 0u);
+            *reinterpret_cast<uint4*>(e + 128) = make_uint4(0u, 0u, 0u, 0u);
+        }
     }
+    // the instance's largest squared norm (the caller cleared the word; non-negative floats order
+    // like their bit patterns)
+    if (lane == 0 && nmax > 0.f) atomicMax(reinterpret_cast<int*>(inst) + 2 * b + 1, __float_as_int(nmax));
 }
 
 // ---- the contraction -------------------------------------------------------------------
@@ -386,19 +459,21 @@ assign_tc_kernel(const TcParams p) {
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int D = p.D, nkb = p.nkb, nt_count = p.Kpad / BN;
     const int DC = p.DC;                                  // TMEM columns of one A part (hi or lo)
-    const int nab = DC <= 64 ? 2 : 1;                     // A (hi+lo) tiles that fit beside the accumulators in TMEM
+    const int AST = 2 * DC + (F16 ? XCOLS : 0);           // TMEM columns of one A buffer: hi | lo | constant terms
+    const int nab = 2 * AST <= 256 ? 2 : 1;               // A buffers that fit beside the accumulators in TMEM
+    constexpr int SLOT = F16 ? SLOT_F16 : STAGE;          // bytes of one stage slot
     const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
-    unsigned char* st_base = smem;                                        // NSTAGE x STAGE
-    float* xs = reinterpret_cast<float*>(smem + NSTAGE * STAGE);          // nxb x [BM][D+4]
-    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // [B][Kpad]
-    float* cw = cn + (size_t)p.B * p.Kpad;                                // [B][Kpad]  (fp16 split only)
-    float* xnorm = cw + (F16 ? (size_t)p.B * p.Kpad : 0);                 // [2][BM]
-    float* xscale = xnorm + 2 * BM;                                       // [2][BM]  1 / (the row's power-of-two scale)
+    unsigned char* st_base = smem;                                        // NSTAGE x SLOT
+    float* xs = reinterpret_cast<float*>(smem + NSTAGE * SLOT);           // nxb x [BM][D+4]
+    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // tf32: [B][Kpad] norms; fp16: [B][2] (s_c, max norm)
+    float* xnorm = cn + (F16 ? (size_t)2 * p.B : (size_t)p.B * p.Kpad);   // [2][BM]
+    float* xscale = xnorm + 2 * BM;                                       // [2][BM]  fp16: 1 / g_i (negative: row out of range)
     float* merge_buf = xscale + 2 * BM;                                   // [2][BM][5]
     uint64_t* bars = reinterpret_cast<uint64_t*>(merge_buf + 2 * BM * 5 + 2);   // (+2 floats: 8-byte alignment)
     // barrier indices
     enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 8, ACC_FULL = A_EMPTY + 8,
-           ACC_EMPTY = ACC_FULL + 2, XN_FULL = ACC_EMPTY + 2, XN_EMPTY = XN_FULL + 2, NBAR = XN_EMPTY + 2 };
+           ACC_EMPTY = ACC_FULL + 2, XN_FULL = ACC_EMPTY + 2, XN_EMPTY = XN_FULL + 2, X_FULL = XN_EMPTY + 2,
+           NBAR = X_FULL + 2 };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -412,6 +487,7 @@ assign_tc_kernel(const TcParams p) {
         for (int k = 0; k < 2; ++k) {
             mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 8);
             mbar_init(BAR(XN_FULL + k), 4); mbar_init(BAR(XN_EMPTY + k), 8);
+            mbar_init(BAR(X_FULL + k), 128);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -421,9 +497,10 @@ assign_tc_kernel(const TcParams p) {
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) {   // all instances' centroid norms (and weights)
-        cn[j] = p.cnorm[j];
-        if (F16) cw[j] = p.cweight[j];
+    if (F16) {
+        for (int j = tid; j < 2 * p.B; j += TC_THREADS) cn[j] = p.inst[j];     // per instance: s_c, largest ||c||^2
+    } else {
+        for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) cn[j] = p.cnorm[j];   // all instances' centroid norms
     }
     tc_fence_before();
     __syncthreads();
@@ -437,45 +514,58 @@ assign_tc_kernel(const TcParams p) {
         // ============================ A producers ====================================
         const int row_in_tile = tid;                       // = TMEM lane
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        const int vpr = D >> 2;                            // float4 per row
+        // Staging: every producer thread owns one row slot of the staging buffer.  It requests its
+        // row with ONE bulk copy (the row is contiguous in global memory) that completes on the
+        // buffer's mbarrier, and later reads only that slot, so a slot is never shared between
+        // threads and needs no block-level barrier.  A row past the end of the instance is zeros.
         auto prefetch = [&](int tile, int buf) {
             const int b = tile / p.tiles_per_inst, r0 = (tile - b * p.tiles_per_inst) * BM;
-            const float* src = p.z + ((size_t)b * p.N + r0) * D;
-            const int rows = min(BM, p.N - r0);
-            float* dst = xs + (size_t)buf * BM * xs_stride;
-            for (int e = tid; e < BM * vpr; e += 128) {
-                const int r = e / vpr, q = e - r * vpr;
-                const bool valid = r < rows;
-                cp_async16(smem_u32(dst + (size_t)r * xs_stride + 4 * q), src + (size_t)(valid ? r : 0) * D + 4 * q,
-                           valid ? 16u : 0u);
+            float* dst = xs + (size_t)buf * BM * xs_stride + (size_t)row_in_tile * xs_stride;
+            if (r0 + row_in_tile < p.N) {
+                mbar_expect_tx(BAR(X_FULL + buf), (uint32_t)D * 4u);
+                bulk_g2s(smem_u32(dst), p.z + ((size_t)b * p.N + r0 + row_in_tile) * D, (uint32_t)D * 4u, BAR(X_FULL + buf));
+            } else {
+                for (int q = 0; q < D / 4; ++q) reinterpret_cast<float4*>(dst)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                mbar_arrive(BAR(X_FULL + buf));
             }
-            cp_async_commit();
         };
         int it = 0;
-        if (first < p.total_tiles) prefetch(first, 0);
+        int uses0 = 0, uses1 = 0;                          // requests issued so far into staging buffer 0 / 1
+        if (first < p.total_tiles) { prefetch(first, 0); ++uses0; }
         for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
             const int buf = p.nxb == 2 ? (it & 1) : 0;
             const int next = tile + stride;
-            if (p.nxb == 2) {
-                if (next < p.total_tiles) { prefetch(next, buf ^ 1); cp_async_wait<1>(); }
-                else cp_async_wait<0>();
-            } else {
-                cp_async_wait<0>();
+            if (p.nxb == 2 && next < p.total_tiles) {
+                prefetch(next, buf ^ 1);
+                if (buf) ++uses0; else ++uses1;
             }
-            bar_sync_producers();                          // the staged tile is visible to all four warps
+            // this tile's rows have landed (request k into a buffer completes the barrier's phase k)
+            ok = mbar_wait(BAR(X_FULL + buf), (uint32_t)((p.nxb == 2 ? (it >> 1) : it) & 1), abort_flag);
+            if (!ok) break;
             const float* xr = xs + (size_t)buf * BM * xs_stride + (size_t)row_in_tile * xs_stride;
             float xn = 0.f, rscale = 1.f;
             const int ab = it % nab, use = it / nab;           // A buffer of this tile, how often it was used before
             if (F16) {
-                // the row's own power-of-two scale (largest magnitude into [0.5, 1)) and its squared norm
+                // squared norm and largest magnitude of the row, then its power-of-two scale s_z: the
+                // largest magnitude goes into [0.5, 1) unless that would put s_z / s_c outside fp16's
+                // normal range
                 float m = 0.f;
                 for (int q = 0; q < D / 4; ++q) {
                     const float4 v = *reinterpret_cast<const float4*>(xr + 4 * q);
                     xn = fmaf(v.x, v.x, xn); xn = fmaf(v.y, v.y, xn); xn = fmaf(v.z, v.z, xn); xn = fmaf(v.w, v.w, xn);
                     m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
                 }
-                const float sc = pow2_scale(m);
-                rscale = 1.f / sc;
+                const int binst = tile / p.tiles_per_inst;
+                const float s_c = cn[2 * binst];
+                float rho = fminf(fmaxf(pow2_scale(m) / s_c, 6.103515625e-05f), 16384.f);   // s_z / s_c in [2^-14, 2^14]
+                float sz = rho * s_c;
+                const float g = sz * s_c;
+                float pterm = g * xn;                              // s_z s_c ||z||^2
+                // a row far outside the centroids' range (its scaled entries or its norm term would
+                // overflow fp16) contributes zeros and is handed to the exact re-evaluation
+                const bool out_of_range = !(m * sz < 32768.f) || !(pterm < 60000.f);
+                rscale = out_of_range ? -1.f : 1.f / g;
+                if (out_of_range) { sz = 0.f; rho = 0.f; pterm = 0.f; }
                 for (int kb = 0; kb < nkb && ok; ++kb) {
                     uint32_t hi[32], lo[32];
                     const int nq = min(16, (D - kb * 64) / 4);     // float4 groups of this k-block that hold features
@@ -483,14 +573,24 @@ assign_tc_kernel(const TcParams p) {
                     for (int q = 0; q < 16; ++q) {
                         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (q < nq) v = *reinterpret_cast<const float4*>(xr + kb * 64 + 4 * q);
-                        split_f16x2(v.x * sc, v.y * sc, hi[2 * q], lo[2 * q]);
-                        split_f16x2(v.z * sc, v.w * sc, hi[2 * q + 1], lo[2 * q + 1]);
+                        split_f16x2(v.x * sz, v.y * sz, hi[2 * q], lo[2 * q]);
+                        split_f16x2(v.z * sz, v.w * sz, hi[2 * q + 1], lo[2 * q + 1]);
                     }
                     ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    TC_ST32(lane_addr + COL_A + ab * 2 * DC + kb * 32, hi);
-                    TC_ST32(lane_addr + COL_A + ab * 2 * DC + DC + kb * 32, lo);
+                    TC_ST32(lane_addr + COL_A + ab * AST + kb * 32, hi);
+                    TC_ST32(lane_addr + COL_A + ab * AST + DC + kb * 32, lo);
+                    if (kb == 0) {     // the row's constant-term operand travels with the first k-block
+                        __half p0, p1, p2;
+                        split3_f16(pterm, p0, p1, p2);
+                        const __half hr = __float2half_rn(rho);
+                        const uint32_t e0 = pack_h2(p0, p1), e1 = pack_h2(p2, hr), e2 = pack_h2(hr, hr), ez = 0u;
+                        asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                     ::"r"(lane_addr + COL_A + ab * AST + 2 * DC), "r"(e0), "r"(e1), "r"(e2), "r"(ez), "r"(ez),
+                                       "r"(ez), "r"(ez), "r"(ez)
+                                     : "memory");
+                    }
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     tc_fence_before();
                     mbar_arrive_warp(BAR(A_FULL + ab * 4 + kb));
@@ -512,25 +612,27 @@ assign_tc_kernel(const TcParams p) {
                 ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                TC_ST32(lane_addr + COL_A + ab * 2 * DC + kb * KBF, hi);
-                TC_ST32(lane_addr + COL_A + ab * 2 * DC + DC + kb * KBF, lo);
+                TC_ST32(lane_addr + COL_A + ab * AST + kb * KBF, hi);
+                TC_ST32(lane_addr + COL_A + ab * AST + DC + kb * KBF, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 mbar_arrive_warp(BAR(A_FULL + ab * 4 + kb));
             }
             }
             if (!ok) break;
-            if (p.nxb == 1) {
-                bar_sync_producers();                      // everyone has read the staging buffer
-                if (next < p.total_tiles) prefetch(next, 0);
-            }
+            if (p.nxb == 1 && next < p.total_tiles) { prefetch(next, 0); ++uses0; }   // own slot: already read
             ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
             if (!ok) break;
             xnorm[(it & 1) * BM + row_in_tile] = xn;
             xscale[(it & 1) * BM + row_in_tile] = rscale;
             mbar_arrive_warp(BAR(XN_FULL + (it & 1)));
         }
-        cp_async_wait<0>();
+        if (!ok) {
+            // abort path: let row copies that may still be in flight land before shared memory goes
+            // away (a phase that was already waited for answers at once)
+            for (uint32_t i = 0; uses0 > 0 && i < WAIT_LIMIT && !mbar_try(BAR(X_FULL + 0), (uint32_t)((uses0 - 1) & 1)); ++i) {}
+            for (uint32_t i = 0; uses1 > 0 && i < WAIT_LIMIT && !mbar_try(BAR(X_FULL + 1), (uint32_t)((uses1 - 1) & 1)); ++i) {}
+        }
     } else if (warp < 12) {
         // ============================ epilogue ========================================
         // Two warps per TMEM lane quarter: `half` 0 takes columns [0,64) of every accumulator
@@ -554,7 +656,6 @@ assign_tc_kernel(const TcParams p) {
             const float xn = xnorm[(it & 1) * BM + row_in_tile];
             const float rscale = xscale[(it & 1) * BM + row_in_tile];
             mbar_arrive_warp(BAR(XN_EMPTY + (it & 1)));
-            const float* cwb = cw + (size_t)b * p.Kpad;
             RowBest<TRACK2> rb;
             for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                 const uint32_t buf = q & 1u;
@@ -568,7 +669,6 @@ assign_tc_kernel(const TcParams p) {
                 pref = false;
                 KeyTracker<TRACK2> ta, tb;
                 const float* cnp = cnb + nt * BN + half * (BN / 2);
-                const float* cwp = cwb + nt * BN + half * (BN / 2);
                 // Two passes over a 32-column register buffer.  The first turns every accumulator value
                 // into its key in place: 32 independent short chains (load the column's constants,
                 // three fp32 operations, one logic operation), which the scheduler can overlap freely.
@@ -576,25 +676,20 @@ assign_tc_kernel(const TcParams p) {
                 auto process = [&](uint32_t (&v)[32], int c) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
-                        const float4 n4 = *reinterpret_cast<const float4*>(cnp + c * 32 + j);
                         const int l = c * 32 + j;                  // column inside this thread's 64
-                        float d0, d1, d2, d3;
-                        if (F16) {      // undo the row's and the centroid's scales: d2 = ||z||^2 + ||c||^2 - 2 acc / (s_z s_c)
-                            const float4 w4 = *reinterpret_cast<const float4*>(cwp + c * 32 + j);
-                            d0 = fmaf(__uint_as_float(v[j + 0]) * rscale, w4.x, n4.x + xn);
-                            d1 = fmaf(__uint_as_float(v[j + 1]) * rscale, w4.y, n4.y + xn);
-                            d2 = fmaf(__uint_as_float(v[j + 2]) * rscale, w4.z, n4.z + xn);
-                            d3 = fmaf(__uint_as_float(v[j + 3]) * rscale, w4.w, n4.w + xn);
+                        int k0, k1, k2, k3;
+                        if (F16) {      // the accumulator already is g_i d2(i, j): rank it as it is
+                            k0 = ((int)v[j + 0] & KEY_MASK) | (l + 0);
+                            k1 = ((int)v[j + 1] & KEY_MASK) | (l + 1);
+                            k2 = ((int)v[j + 2] & KEY_MASK) | (l + 2);
+                            k3 = ((int)v[j + 3] & KEY_MASK) | (l + 3);
                         } else {
-                            d0 = fmaf(-2.f, __uint_as_float(v[j + 0]), n4.x + xn);
-                            d1 = fmaf(-2.f, __uint_as_float(v[j + 1]), n4.y + xn);
-                            d2 = fmaf(-2.f, __uint_as_float(v[j + 2]), n4.z + xn);
-                            d3 = fmaf(-2.f, __uint_as_float(v[j + 3]), n4.w + xn);
+                            const float4 n4 = *reinterpret_cast<const float4*>(cnp + c * 32 + j);
+                            k0 = (__float_as_int(fmaf(-2.f, __uint_as_float(v[j + 0]), n4.x + xn)) & KEY_MASK) | (l + 0);
+                            k1 = (__float_as_int(fmaf(-2.f, __uint_as_float(v[j + 1]), n4.y + xn)) & KEY_MASK) | (l + 1);
+                            k2 = (__float_as_int(fmaf(-2.f, __uint_as_float(v[j + 2]), n4.z + xn)) & KEY_MASK) | (l + 2);
+                            k3 = (__float_as_int(fmaf(-2.f, __uint_as_float(v[j + 3]), n4.w + xn)) & KEY_MASK) | (l + 3);
                         }
-                        const int k0 = (__float_as_int(d0) & KEY_MASK) | (l + 0);
-                        const int k1 = (__float_as_int(d1) & KEY_MASK) | (l + 1);
-                        const int k2 = (__float_as_int(d2) & KEY_MASK) | (l + 2);
-                        const int k3 = (__float_as_int(d3) & KEY_MASK) | (l + 3);
                         ta.add2(k0, k1);
                         tb.add2(k2, k3);
                     }
@@ -642,13 +737,22 @@ assign_tc_kernel(const TcParams p) {
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
                 const int a0 = rb.column(rb.r0, rb.t0);
-                const float b0 = rb.value(rb.r0), b1 = rb.value(rb.r1);
+                // fp16 split: the ranked values carry the row's factor g_i; take it out again
+                const float unscale = F16 ? fabsf(rscale) : 1.f;
+                const float b0 = rb.value(rb.r0) * unscale, b1 = rb.value(rb.r1) * unscale;
+                const float b2 = rb.value(rb.r2) * unscale;
                 p.labels[flat] = a0;
                 if (p.approx) p.approx[flat] = b0;
-                // near-tie bound: the split product's error plus what the dropped key bits can hide
-                const float delta = p.eps * (xn + cnb[a0]) + 1.52587890625e-5f * fabsf(b1);
-                if (fabsf(b1 - b0) <= delta) {
-                    if (TRACK2 && fabsf(rb.value(rb.r2) - b0) > delta) {   // exactly two candidates: compare them exactly
+                // near-tie bound: the split product's error (relative to ||z||^2 plus the centroid's
+                // norm; the fp16 split shares one scale among an instance's centroids, so there the
+                // largest norm of the instance) plus what the dropped key bits can hide
+                const float cref = F16 ? cn[2 * b + 1] : cnb[a0];
+                const float delta = p.eps * (xn + cref) + 1.52587890625e-5f * fabsf(b1);
+                if (F16 && rscale < 0.f) {                     // row outside the fp16 range: exact scan over all K
+                    const int slot = atomicAdd(p.flag_count + 1, 1);
+                    p.full_rows[slot] = (int32_t)flat;
+                } else if (fabsf(b1 - b0) <= delta) {
+                    if (TRACK2 && fabsf(b2 - b0) > delta) {   // exactly two candidates: compare them exactly
                         const int slot = atomicAdd(p.flag_count, 1);
                         p.pair_rows[slot] = make_int2((int)flat, rb.column(rb.r1, rb.t1));
                     } else {                                   // three or more (or unknown): exact scan over all K
@@ -673,10 +777,14 @@ assign_tc_kernel(const TcParams p) {
             const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
             const uint32_t desc_hi32 = (uint32_t)(desc0 >> 32);
             const uint32_t desc_lo32 = (uint32_t)desc0;
+            // K-major, no swizzle: 8-row x 16-byte core matrices, the two k-halves 128 bytes apart
+            // (leading byte offset), 8-row groups 256 bytes apart (stride byte offset)
+            const uint32_t ext_lo32 = ((smem_u32(st_base + STAGE) & 0x3FFFFu) >> 4) | ((128u >> 4) << 16);
+            const uint32_t ext_hi32 = (256u >> 4) | (1u << 14);
             const int ring = p.resident ? nt_count * nkb : NSTAGE;
             for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
                 const int ab = it % nab, use = it / nab;
-                const uint32_t a_base = tmem + COL_A + ab * 2 * DC;
+                const uint32_t a_base = tmem + COL_A + ab * AST;
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
@@ -694,10 +802,14 @@ assign_tc_kernel(const TcParams p) {
                         }
                         tc_fence_after();
                         const uint32_t a_hi = a_base + kb * 32, a_lo = a_hi + DC;
-                        const uint32_t blo = desc_lo32 + s * (STAGE >> 4);        // this stage's hi panel
+                        const uint32_t blo = desc_lo32 + s * (SLOT >> 4);         // this stage's hi panel
                         if (elect_one()) {
-                        // first k-step: the very first product of an accumulator tile overwrites it
-                        tc_mma_ts<F16>(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, kb != 0 ? 1u : 0u);
+                        // The very first product of an accumulator tile overwrites it.  fp16 split: that is
+                        // the constant-term product (the row's 16 extra features against the centroid
+                        // tile's, which sit behind the first k-block's panels without swizzle).
+                        if (F16 && kb == 0)
+                            tc_mma_ts<F16>(d_tmem, a_base + 2 * DC, mk_desc(ext_lo32 + s * (SLOT >> 4), ext_hi32), IDESC, 0u);
+                        tc_mma_ts<F16>(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, (F16 || kb != 0) ? 1u : 0u);
                         tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
                         tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo, desc_hi32), IDESC);
 #pragma unroll
@@ -729,8 +841,12 @@ assign_tc_kernel(const TcParams p) {
                 for (int i = 0; i < nt_count * nkb; ++i) {
                     ok = mbar_wait(BAR(B_EMPTY + s), ph ^ 1u, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(BAR(B_FULL + s), STAGE);
-                    bulk_g2s(smem_u32(st_base + (size_t)s * STAGE), src + (size_t)i * STAGE, STAGE, BAR(B_FULL + s));
+                    const bool with_ext = F16 && (i % nkb == 0);   // a tile's first k-block brings its constant terms
+                    mbar_expect_tx(BAR(B_FULL + s), with_ext ? STAGE + EXT : STAGE);
+                    bulk_g2s(smem_u32(st_base + (size_t)s * SLOT), src + (size_t)i * STAGE, STAGE, BAR(B_FULL + s));
+                    if (with_ext)
+                        bulk_g2s(smem_u32(st_base + (size_t)s * SLOT + STAGE),
+                                 p.bext + ((size_t)b * nt_count + i / nkb) * EXT, EXT, BAR(B_FULL + s));
                     ++issued;
                     if (++s == NSTAGE) { s = 0; ph ^= 1u; }
                 }
@@ -788,45 +904,38 @@ fixup_pairs(int nblocks, int N, int D, int K, const float* __restrict__ z, const
     }
 }
 
-// One launch settles both queues: every block first takes its share of the two-candidate
-// rows, then of the rows that need all K centroids (eight queued rows share every centroid
-// read; thread = centroid, warp-shuffle argmin, lowest index on ties).
-constexpr int FX_ROWS = 8;
+// Exact re-evaluation of queued rows against all K centroids.  ROWS queued rows form a group and
+// share every centroid read: tiles of FX_T centroids are staged through shared memory with
+// coalesced, independent loads, thread t then owns centroid t of the tile (warp-shuffle argmin,
+// lowest index on ties).  Few queued rows: ROWS = 1, so that a row costs one short pass instead of
+// the eight-row loop (the kernel's time is then the latency of its slowest block).
 constexpr int FX_T = 256;
-__global__ void __launch_bounds__(FX_T)
-assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                    const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
-                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
-    extern __shared__ __align__(16) float fx[];            // [FX_ROWS][D] rows | [FX_T][D+4] centroid tile
-    __shared__ float red_v[FX_ROWS][FX_T / 32];
-    __shared__ int red_i[FX_ROWS][FX_T / 32];
-    __shared__ int s_inst[FX_ROWS];
-    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
-    float* xrow = fx;
-    float* ctile = fx + FX_ROWS * D;                       // [FX_T][D+4] centroid tile
-    const int total = flag_count[1];
+constexpr int FX_MAXROWS = 8;
+template <int ROWS>
+__device__ __forceinline__ void
+fixup_full(int N, int D, int K, int total, const float* __restrict__ z, const float* __restrict__ cent,
+           const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels, float* xrow, float* ctile,
+           float (*red_v)[FX_T / 32], int (*red_i)[FX_T / 32], int* s_inst) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int g0 = blockIdx.x * FX_ROWS; g0 < total; g0 += gridDim.x * FX_ROWS) {
-        const int nrow = min(FX_ROWS, total - g0);
+    for (int g0 = blockIdx.x * ROWS; g0 < total; g0 += gridDim.x * ROWS) {
+        const int nrow = min(ROWS, total - g0);
         __syncthreads();
-        for (int e = tid; e < FX_ROWS * (D / 4); e += FX_T) {
+        for (int e = tid; e < ROWS * (D / 4); e += FX_T) {
             const int r = e / (D / 4), q = e - r * (D / 4);
             // rows past the end of the queue repeat the last one (their result is discarded)
             reinterpret_cast<float4*>(xrow)[e] =
                 __ldg(reinterpret_cast<const float4*>(z + (size_t)full_rows[g0 + min(r, nrow - 1)] * D) + q);
         }
-        if (tid < FX_ROWS) s_inst[tid] = full_rows[g0 + min(tid, nrow - 1)] / N;
+        if (tid < ROWS) s_inst[tid] = full_rows[g0 + min(tid, nrow - 1)] / N;
         __syncthreads();
-        float best[FX_ROWS];
-        int arg[FX_ROWS];
+        float best[ROWS];
+        int arg[ROWS];
 #pragma unroll
-        for (int r = 0; r < FX_ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
+        for (int r = 0; r < ROWS; ++r) { best[r] = INFINITY; arg[r] = 0x7fffffff; }
         bool same_inst = true;
 #pragma unroll
-        for (int r = 1; r < FX_ROWS; ++r) same_inst = same_inst && (s_inst[r] == s_inst[0]);
+        for (int r = 1; r < ROWS; ++r) same_inst = same_inst && (s_inst[r] == s_inst[0]);
         if (same_inst) {
-            // the usual case: tiles of FX_T centroids are staged through shared memory with coalesced,
-            // independent loads (one memory round trip per tile), thread t then owns centroid t of the tile
             const int CS = D + 4;                                  // 16-byte aligned, conflict-free float4 rows
             const float* cbase = cent + (size_t)s_inst[0] * K * D;
             for (int j0 = 0; j0 < K; j0 += FX_T) {
@@ -839,14 +948,14 @@ assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const floa
                 }
                 __syncthreads();
                 if (tid < nc) {
-                    float acc[FX_ROWS];
+                    float acc[ROWS];
 #pragma unroll
-                    for (int r = 0; r < FX_ROWS; ++r) acc[r] = 0.f;
+                    for (int r = 0; r < ROWS; ++r) acc[r] = 0.f;
                     const float4* c4 = reinterpret_cast<const float4*>(ctile + (size_t)tid * CS);
                     for (int d = 0; d < D / 4; ++d) {
                         const float4 c = c4[d];
 #pragma unroll
-                        for (int r = 0; r < FX_ROWS; ++r) {
+                        for (int r = 0; r < ROWS; ++r) {
                             const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
                             float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
                             acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
@@ -854,37 +963,33 @@ assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const floa
                         }
                     }
 #pragma unroll
-                    for (int r = 0; r < FX_ROWS; ++r)
+                    for (int r = 0; r < ROWS; ++r)
                         if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j0 + tid; }   // ascending tiles: lowest index on ties
                 }
             }
-        } else
-        for (int j = tid; j < K; j += FX_T) {
-            float acc[FX_ROWS];
-#pragma unroll
-            for (int r = 0; r < FX_ROWS; ++r) acc[r] = 0.f;
+        } else {
             // rows of one group nearly always share an instance; when they do not, each row reads its own
-            const float4* c0 = reinterpret_cast<const float4*>(cent + ((size_t)s_inst[0] * K + j) * D);
-#pragma unroll 4
-            for (int d = 0; d < D / 4; ++d) {
-                const float4 c = __ldg(c0 + d);
+            for (int j = tid; j < K; j += FX_T) {
+                float acc[ROWS];
 #pragma unroll
-                for (int r = 0; r < FX_ROWS; ++r) {
-                    float4 cr = c;
-                    if (s_inst[r] != s_inst[0])
-                        cr = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)s_inst[r] * K + j) * D) + d);
-                    const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
-                    float e0 = x.x - cr.x, e1 = x.y - cr.y, e2 = x.z - cr.z, e3 = x.w - cr.w;
-                    acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
-                    acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
+                for (int r = 0; r < ROWS; ++r) acc[r] = 0.f;
+                for (int d = 0; d < D / 4; ++d) {
+#pragma unroll
+                    for (int r = 0; r < ROWS; ++r) {
+                        const float4 c = __ldg(reinterpret_cast<const float4*>(cent + ((size_t)s_inst[r] * K + j) * D) + d);
+                        const float4 x = reinterpret_cast<const float4*>(xrow + r * D)[d];
+                        float e0 = x.x - c.x, e1 = x.y - c.y, e2 = x.z - c.z, e3 = x.w - c.w;
+                        acc[r] = fmaf(e0, e0, acc[r]); acc[r] = fmaf(e1, e1, acc[r]);
+                        acc[r] = fmaf(e2, e2, acc[r]); acc[r] = fmaf(e3, e3, acc[r]);
+                    }
                 }
-            }
 #pragma unroll
-            for (int r = 0; r < FX_ROWS; ++r)
-                if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j; }   // ascending j: lowest index on ties
+                for (int r = 0; r < ROWS; ++r)
+                    if (acc[r] < best[r]) { best[r] = acc[r]; arg[r] = j; }   // ascending j: lowest index on ties
+            }
         }
 #pragma unroll
-        for (int r = 0; r < FX_ROWS; ++r) {
+        for (int r = 0; r < ROWS; ++r) {
             float v = best[r];
             int i = arg[r];
 #pragma unroll
@@ -907,6 +1012,28 @@ assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const floa
             labels[full_rows[g0 + tid]] = bi;
         }
     }
+}
+
+// One launch settles both queues: every block first takes its share of the two-candidate rows,
+// then of the rows that need all K centroids, in groups sized to the queue's length.
+__global__ void __launch_bounds__(FX_T)
+assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                    const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
+    extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
+    __shared__ float red_v[FX_MAXROWS][FX_T / 32];
+    __shared__ int red_i[FX_MAXROWS][FX_T / 32];
+    __shared__ int s_inst[FX_MAXROWS];
+    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
+    float* xrow = fx;
+    float* ctile = fx + FX_MAXROWS * D;
+    const int total = flag_count[1];
+    if (total <= 0) return;
+    const int per_block = (total + gridDim.x - 1) / gridDim.x;     // uniform over the grid
+    if (per_block <= 1) fixup_full<1>(N, D, K, total, z, cent, full_rows, labels, xrow, ctile, red_v, red_i, s_inst);
+    else if (per_block <= 2) fixup_full<2>(N, D, K, total, z, cent, full_rows, labels, xrow, ctile, red_v, red_i, s_inst);
+    else if (per_block <= 4) fixup_full<4>(N, D, K, total, z, cent, full_rows, labels, xrow, ctile, red_v, red_i, s_inst);
+    else fixup_full<8>(N, D, K, total, z, cent, full_rows, labels, xrow, ctile, red_v, red_i, s_inst);
 }
 
 // ---- dist2 / inertia / representative from final labels (direct form) -------------------
@@ -971,9 +1098,9 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
 
 size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool f16) {
     size_t s = 1024;                                       // alignment slack
-    s += (size_t)NSTAGE * STAGE;
+    s += (size_t)NSTAGE * (f16 ? SLOT_F16 : STAGE);
     s += (size_t)nxb * BM * (D + 4) * 4;
-    s += (size_t)Kpad * 4 * (f16 ? 2 : 1) + 4 * BM * 4 + (2 * BM * 5 + 2) * 4;
+    s += (f16 ? (size_t)2 * (Kpad / BN) * 4 : (size_t)Kpad * 4) + 4 * BM * 4 + (2 * BM * 5 + 2) * 4;
     s += 40 * 8 + 16;                                      // barriers, TMEM slot, abort flag
     return s;
 }
@@ -984,8 +1111,8 @@ size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool 
 // B image | centroid norms | queue counter | queue
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
     const size_t Kpad = (size_t)(K + BN - 1) / BN * BN;
-    return kb_align256(B * Kpad * D * 8) + 2 * kb_align256(B * Kpad * 4) + 256 + kb_align256((size_t)B * N * 8) +
-           kb_align256((size_t)B * N * 4);
+    return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + kb_align256(B * Kpad * 32) +
+           kb_align256((size_t)B * 8) + 256 + kb_align256((size_t)B * N * 8) + kb_align256((size_t)B * N * 4);
 }
 
 // what the kernel can run at all
@@ -993,7 +1120,8 @@ bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K) {
     if (D % KBF != 0 || D > 128 || K < 1 || K > 8192 || B < 1) return false;
     const long Kpad = (long)(K + BN - 1) / BN * BN;
     if (Kpad * B > 8192) return false;                     // the norms of every instance stay in shared memory
-    return tc_smem_bytes(D, (int)(Kpad * B), 1, true) <= (size_t)ctx->max_smem_optin;
+    return tc_smem_bytes(D, (int)(Kpad * B), 1, true) <= (size_t)ctx->max_smem_optin &&
+           tc_smem_bytes(D, (int)(Kpad * B), 1, false) <= (size_t)ctx->max_smem_optin;
 }
 // what the automatic choice sends there: enough centroids to fill an accumulator tile
 // and enough rows for the contraction to outweigh the preparation and fix-up launches
@@ -1009,18 +1137,21 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     const int Kpad = (K + BN - 1) / BN * BN;
     unsigned char* bimg = reinterpret_cast<unsigned char*>(ws);
     float* cnorm = reinterpret_cast<float*>(ws + kb_align256((size_t)B * Kpad * D * 8));
-    float* cweight = reinterpret_cast<float*>(reinterpret_cast<char*>(cnorm) + kb_align256((size_t)B * Kpad * 4));
-    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(cweight) + kb_align256((size_t)B * Kpad * 4));
+    unsigned char* bext = reinterpret_cast<unsigned char*>(cnorm) + kb_align256((size_t)B * Kpad * 4);
+    float* inst = reinterpret_cast<float*>(bext + kb_align256((size_t)B * Kpad * 32));
+    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(inst) + kb_align256((size_t)B * 8));
     int2* pair_rows = reinterpret_cast<int2*>(reinterpret_cast<char*>(flag_count) + 256);
     int32_t* full_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(pair_rows) + kb_align256((size_t)B * N * 8));
 
     // the split: fp16 hi/lo (kind::f16, 16 features per instruction) unless the tf32 split is forced
     const bool f16 = ctx->assign_path != 3;
     const int nkb = f16 ? (D + 63) / 64 : D / KBF;
-    if (f16)
-        tc_prep_kernel<true><<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, cweight, flag_count);
-    else
-        tc_prep_kernel<false><<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, cweight, flag_count);
+    if (f16) {
+        KB_MEMSET(ctx, inst, 0, (size_t)B * 8);
+        const int gprep = (Kpad + 7) / 8 < 64 ? (Kpad + 7) / 8 : 64;
+        tc_prep_f16_kernel<<<dim3(gprep, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, bext, inst, flag_count);
+    } else
+        tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, flag_count);
     KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
 
     TcParams p;
@@ -1032,13 +1163,13 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     p.nxb = tc_smem_bytes(D, Kpad * B, 2, f16) <= (size_t)ctx->max_smem_optin ? 2 : 1;
     p.eps = eps;
     p.resident = (B == 1 && (Kpad / BN) * nkb <= NSTAGE) ? 1 : 0;
-    p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.cweight = cweight; p.labels = labels; p.approx = approx;
+    p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.bext = bext; p.inst = inst; p.labels = labels; p.approx = approx;
     p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
     const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb, f16);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
     // with few features per row the epilogue's per-column cost is what limits the kernel:
     // track less there and let the (cheap, K*D is small) full re-evaluation settle near-ties
-    const bool track2 = D >= 96;
+    const bool track2 = f16 || D >= 96;
 #define KB_TC_LAUNCH(T2, F)                                                                    \
     do {                                                                                       \
         KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F>), smem);                                   \
@@ -1051,7 +1182,7 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
 #undef KB_TC_LAUNCH
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
-    const size_t fsmem = (size_t)FX_ROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
+    const size_t fsmem = (size_t)FX_MAXROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
     assign_fixup_kernel<<<4 * ctx->sm_count, FX_T, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows,
                                                                         full_rows, labels);

@@ -402,7 +402,10 @@ def test_assign_tensor_path(kbx, B, N, D, K, path):
     # how far the ranked (expanded-form, 3xTF32) distance is from the exact one
     xn = (z.astype(np.float64) ** 2).sum(-1)
     cnn = (c.astype(np.float64) ** 2).sum(-1)
-    scale = xn + np.take_along_axis(cnn, ref["labels"].astype(np.int64), axis=1)
+    # the fp16 split shares one power-of-two scale among an instance's centroids: its error is relative to
+    # the largest centroid norm of the instance; the tf32 split's to the chosen centroid's
+    scale = xn + (cnn.max(axis=1, keepdims=True) if path == 2 else
+                  np.take_along_axis(cnn, ref["labels"].astype(np.int64), axis=1))
     # (the ranked value also drops its low 7 mantissa bits, which hold the column index: up to 2^-16 of itself,
     # a term the kernel's near-tie bound adds on top of eps)
     err = (np.abs(host(approx).astype(np.float64) - ref["best"]) - ref["best"] / 65536)[same] / scale[same]
