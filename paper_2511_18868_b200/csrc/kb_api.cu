@@ -21,6 +21,7 @@ namespace {
 
 __global__ void gather_rows_kernel(int N, int D, int K, const float* __restrict__ z, const int32_t* __restrict__ rows,
                                    float* __restrict__ c, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     const int b = blockIdx.y, i = blockIdx.x;
     int r = rows[(size_t)b * K + i];
     if (r < 0 || r >= N) { if (threadIdx.x == 0) atomicOr(dev_status, 4); return; }
@@ -52,7 +53,7 @@ struct TimeScope {
 kb_status kb_launch_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
                                    float* c) {
     if (B == 0 || K == 0) return KB_OK;
-    gather_rows_kernel<<<dim3(K, B), 64, 0, ctx->stream>>>(N, D, K, z, rows, c, ctx->dev_status);
+    kb_launch(gather_rows_kernel, dim3(K, B), 64, 0, ctx->stream, N, D, K, z, rows, c, ctx->dev_status);
     KB_LAUNCH_CHECK(ctx, "gather_rows_kernel");
     return KB_OK;
 }

@@ -18,6 +18,7 @@ constexpr int AS_GROUP = 8;  // centroids evaluated per pass over a row
 __global__ void assign_finalize_kernel(int B, int K, const double* __restrict__ ws_inertia,
                                        const unsigned long long* __restrict__ ws_rep, float* __restrict__ inertia,
                                        int32_t* __restrict__ rep) {
+    kb_grid_dependency_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (inertia && i < B) inertia[i] = (float)ws_inertia[i];
     if (rep && i < B * K) {
@@ -31,6 +32,7 @@ __global__ void __launch_bounds__(128)
 assign_rowwise_kernel(int N, int D, int K, int TM, int CT, const float* __restrict__ z,
                       const float* __restrict__ cent, int32_t* __restrict__ labels, float* __restrict__ dist2,
                       double* __restrict__ ws_inertia, unsigned long long* __restrict__ ws_rep) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) float smem[];
     const int XS = D + 1;                    // odd stride when D is even; any stride is correct
     float* cs = smem;                        // [CT][D]     (16-byte aligned rows when D % 4 == 0)
@@ -152,11 +154,11 @@ static kb_status launch_rowwise(kb_ctx* ctx, int B, int N, int D, int K, const f
     dim3 grid((N + TM - 1) / TM, B);
     if (D % 4 == 0) {
         KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<true>, smem);
-        assign_rowwise_kernel<true><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
+        kb_launch(assign_rowwise_kernel<true>, grid, 128, smem, ctx->stream, N, D, K, TM, CT, z, c, labels, dist2,
                                                                      ws_inertia, ws_rep);
     } else {
         KB_SMEM_OPTIN(ctx, assign_rowwise_kernel<false>, smem);
-        assign_rowwise_kernel<false><<<grid, 128, smem, ctx->stream>>>(N, D, K, TM, CT, z, c, labels, dist2,
+        kb_launch(assign_rowwise_kernel<false>, grid, 128, smem, ctx->stream, N, D, K, TM, CT, z, c, labels, dist2,
                                                                       ws_inertia, ws_rep);
     }
     KB_LAUNCH_CHECK(ctx, "assign_rowwise_kernel");
@@ -203,7 +205,7 @@ kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float*
     }
     if (inertia || rep) {
         int total = B * (rep ? K : 1);
-        assign_finalize_kernel<<<(total + 255) / 256, 256, 0, ctx->stream>>>(B, K, ws_inertia, ws_rep, inertia, rep);
+        kb_launch(assign_finalize_kernel, (total + 255) / 256, 256, 0, ctx->stream, B, K, ws_inertia, ws_rep, inertia, rep);
         KB_LAUNCH_CHECK(ctx, "assign_finalize_kernel");
     }
     return KB_OK;

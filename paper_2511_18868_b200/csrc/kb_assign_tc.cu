@@ -281,6 +281,7 @@ __device__ __forceinline__ void split_f16x2(float a, float b, uint32_t& hi, uint
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
                float* __restrict__ cnorm, int* __restrict__ flag_count) {
+    kb_grid_dependency_wait();
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
     const int b = blockIdx.y;
     const int nt = Kpad / BN;
@@ -340,6 +341,7 @@ __device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
 __global__ void __launch_bounds__(256)
 tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ cent, unsigned char* __restrict__ bimg,
                    unsigned char* __restrict__ bext, float* __restrict__ inst, int* __restrict__ flag_count) {
+    kb_grid_dependency_wait();
     __shared__ float s_m[8];
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 2) flag_count[threadIdx.x] = 0;   // empty both queues
     const int b = blockIdx.y, nt = Kpad / BN;
@@ -497,6 +499,9 @@ assign_tc_kernel(const TcParams p) {
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // everything above touches only this CTA's shared and tensor memory: it may overlap the tail of
+    // the preceding kernel; from here on its results are read
+    kb_grid_dependency_wait();
     if (F16) {
         for (int j = tid; j < 2 * p.B; j += TC_THREADS) cn[j] = p.inst[j];     // per instance: s_c, largest ||c||^2
     } else {
@@ -1020,6 +1025,7 @@ __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                     const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
                     const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_MAXROWS][FX_T / 32];
     __shared__ int red_i[FX_MAXROWS][FX_T / 32];
@@ -1041,6 +1047,7 @@ __global__ void __launch_bounds__(256)
 assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                      const int32_t* __restrict__ labels, float* __restrict__ dist2, double* __restrict__ ws_inertia,
                      unsigned long long* __restrict__ ws_rep) {
+    kb_grid_dependency_wait();
     // lanes of a warp cover the float4 columns of a row; when a row needs fewer than 32 lanes several
     // rows share a warp step, and four steps are in flight per lane
     const int b = blockIdx.y;
@@ -1149,9 +1156,9 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     if (f16) {
         KB_MEMSET(ctx, inst, 0, (size_t)B * 8);
         const int gprep = (Kpad + 7) / 8 < 64 ? (Kpad + 7) / 8 : 64;
-        tc_prep_f16_kernel<<<dim3(gprep, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, bext, inst, flag_count);
+        kb_launch(tc_prep_f16_kernel, dim3(gprep, B), 256, 0, ctx->stream, K, D, Kpad, nkb, c, bimg, bext, inst, flag_count);
     } else
-        tc_prep_kernel<<<dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream>>>(K, D, Kpad, nkb, c, bimg, cnorm, flag_count);
+        kb_launch(tc_prep_kernel, dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream, K, D, Kpad, nkb, c, bimg, cnorm, flag_count);
     KB_LAUNCH_CHECK(ctx, "tc_prep_kernel");
 
     TcParams p;
@@ -1173,7 +1180,7 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
 #define KB_TC_LAUNCH(T2, F)                                                                    \
     do {                                                                                       \
         KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F>), smem);                                   \
-        assign_tc_kernel<T2, F><<<grid, TC_THREADS, smem, ctx->stream>>>(p);                   \
+        kb_launch(assign_tc_kernel<T2, F>, grid, TC_THREADS, smem, ctx->stream, p);                   \
     } while (0)
     if (track2 && f16) KB_TC_LAUNCH(true, true);
     else if (track2) KB_TC_LAUNCH(true, false);
@@ -1184,7 +1191,7 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
 
     const size_t fsmem = (size_t)FX_MAXROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
-    assign_fixup_kernel<<<4 * ctx->sm_count, FX_T, fsmem, ctx->stream>>>(N, D, K, z, c, flag_count, pair_rows,
+    kb_launch(assign_fixup_kernel, 4 * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count, pair_rows,
                                                                         full_rows, labels);
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
@@ -1200,7 +1207,7 @@ kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const
     long cap = ((long)N + 63) / 64;
     int G = (int)(want > cap ? cap : want);
     if (G < 1) G = 1;
-    assign_finish_kernel<<<dim3(G, B), 256, 0, ctx->stream>>>(N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
+    kb_launch(assign_finish_kernel, dim3(G, B), 256, 0, ctx->stream, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
     KB_LAUNCH_CHECK(ctx, "assign_finish_kernel");
     return KB_OK;
 }

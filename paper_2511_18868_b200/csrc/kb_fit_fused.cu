@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(FF_T)
 fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
                  int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                  int32_t* __restrict__ rep, int32_t* __restrict__ counts) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char ff_raw[];
     constexpr int ZS = D + 1;                                       // padded row stride: conflict-free column walks
     float* cs = reinterpret_cast<float*>(ff_raw);                   // [K][D] centroids (16-byte aligned rows)
@@ -171,13 +172,13 @@ kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters
     const size_t smem = ff_smem(N, D, K);
     if (D == 16) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        fit_fused_kernel<16><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<16>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     } else if (D == 32) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        fit_fused_kernel<32><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<32>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     } else {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        fit_fused_kernel<64><<<B, FF_T, smem, ctx->stream>>>(N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<64>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     }
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;

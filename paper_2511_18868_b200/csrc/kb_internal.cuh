@@ -106,6 +106,33 @@ kb_status kb_launch_init_centroids(kb_ctx*, int B, int N, int D, int K, const fl
             KB_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes))); \
     } while (0)
 
+// ---- launches with programmatic dependent launch ------------------------------
+// Every kernel of the library is launched with the programmatic-stream-serialization attribute and
+// begins with kb_grid_dependency_wait(): the next kernel's blocks may be scheduled, and run their
+// prologue up to that wait, while the previous kernel drains, which hides most of the launch gap
+// between the many short dependent kernels of a Lloyd iteration.  The wait returns when the
+// preceding kernel has completed and its writes are visible; as every kernel takes it before
+// touching global memory, completion is transitive along the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void kb_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t kb_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                             Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // ---- small device helpers -----------------------------------------------------
 #ifdef __CUDACC__
 __device__ __forceinline__ float kb_warp_sum(float v) {

@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(256)
 norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, double* __restrict__ part,
                   float* __restrict__ stat, unsigned* __restrict__ ticket, float* __restrict__ mean_out,
                   float* __restrict__ scale_out) {
+    kb_grid_dependency_wait();
     extern __shared__ double red[];  // [threads][2V]
     const int b = blockIdx.z, chunk = blockIdx.y, blk = blockIdx.x;
     const int tid = threadIdx.x, T = g.cw * g.rl;
@@ -169,6 +170,7 @@ norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, doubl
 template <int V>
 __global__ void __launch_bounds__(256)
 norm_apply_kernel(int N, int D, Geo g, int G, const float* x, float* z, const float* __restrict__ stat) {
+    kb_grid_dependency_wait();
     const int b = blockIdx.z, chunk = blockIdx.y, blk = blockIdx.x;
     const int tid = threadIdx.x, T = g.cw * g.rl;
     const int cl = tid % g.cw, rl = tid / g.cw;
@@ -195,6 +197,7 @@ norm_apply_kernel(int N, int D, Geo g, int G, const float* x, float* z, const fl
 }
 
 __global__ void norm_empty_kernel(int total, float* mean, float* scale) {
+    kb_grid_dependency_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < total) {
         if (mean) mean[i] = 0.f;
@@ -221,9 +224,9 @@ kb_status run(kb_ctx* ctx, int B, int N, int D, const float* x, float* z, float*
     KB_MEMSET(ctx, ticket, 0, (size_t)B * 4);
     dim3 grid(G, chunks, B);
     size_t smem = (size_t)256 * 2 * V * sizeof(double);
-    norm_stats_kernel<V><<<grid, 256, smem, ctx->stream>>>(N, D, g, G, x, part, stat, ticket, mean, scale);
+    kb_launch(norm_stats_kernel<V>, grid, 256, smem, ctx->stream, N, D, g, G, x, part, stat, ticket, mean, scale);
     KB_LAUNCH_CHECK(ctx, "norm_stats_kernel");
-    norm_apply_kernel<V><<<grid, 256, 0, ctx->stream>>>(N, D, g, G, x, z, stat);
+    kb_launch(norm_apply_kernel<V>, grid, 256, 0, ctx->stream, N, D, g, G, x, z, stat);
     KB_LAUNCH_CHECK(ctx, "norm_apply_kernel");
     return KB_OK;
 }
@@ -252,7 +255,7 @@ kb_status kb_launch_normalize(kb_ctx* ctx, int B, int N, int D, const float* x, 
     if (N == 0) {
         if (mean || scale) {
             int total = B * D;
-            norm_empty_kernel<<<(total + 255) / 256, 256, 0, ctx->stream>>>(total, mean, scale);
+            kb_launch(norm_empty_kernel, (total + 255) / 256, 256, 0, ctx->stream, total, mean, scale);
             KB_LAUNCH_CHECK(ctx, "norm_empty_kernel");
         }
         return KB_OK;

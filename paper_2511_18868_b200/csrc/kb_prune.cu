@@ -23,6 +23,7 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
                  const int32_t* __restrict__ labels, const float* __restrict__ hsig,
                  const int32_t* __restrict__ target, float theta, uint32_t* __restrict__ keep,
                  uint32_t* __restrict__ kept, float* __restrict__ bound, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     __shared__ unsigned s_kept[PV_T / 32];
     const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
     const int vps = S >> 2;                  // lanes per row: 1, 2, 4 or 8
@@ -104,6 +105,7 @@ prune_kernel(int N, int S, int K, int R, const float* __restrict__ flops, const 
              const float* __restrict__ hsig, const int32_t* __restrict__ target, float theta,
              uint32_t* __restrict__ keep, uint32_t* __restrict__ kept, float* __restrict__ bound,
              int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     extern __shared__ float tile[];  // [PR_T][S+1] when the bound is written
     __shared__ float sP[32], sW[32];
     __shared__ int sT[32];
@@ -182,7 +184,7 @@ kb_status kb_launch_prune(kb_ctx* ctx, int B, int N, int S, int K, int R, const 
         long cap = ((long)N * (S / 4) + PV_T - 1) / PV_T;
         int G = (int)(want > cap ? cap : want);
         if (G < 1) G = 1;
-        prune_vec_kernel<<<dim3(G, B), PV_T, 0, ctx->stream>>>(N, S, K, R, G, flops, bytes, peak_flops, peak_bw, t_inc,
+        kb_launch(prune_vec_kernel, dim3(G, B), PV_T, 0, ctx->stream, N, S, K, R, G, flops, bytes, peak_flops, peak_bw, t_inc,
                                                              t_cur, labels, hsig, target, theta, keep, kept, bound,
                                                              ctx->dev_status);
         KB_LAUNCH_CHECK(ctx, "prune_vec_kernel");
@@ -190,7 +192,7 @@ kb_status kb_launch_prune(kb_ctx* ctx, int B, int N, int S, int K, int R, const 
     }
     dim3 grid((N + PR_T - 1) / PR_T, B);
     size_t smem = bound ? (size_t)PR_T * (S + 1) * sizeof(float) : 0;
-    prune_kernel<<<grid, PR_T, smem, ctx->stream>>>(N, S, K, R, flops, bytes, peak_flops, peak_bw, t_inc, t_cur,
+    kb_launch(prune_kernel, grid, PR_T, smem, ctx->stream, N, S, K, R, flops, bytes, peak_flops, peak_bw, t_inc, t_cur,
                                                     labels, hsig, target, theta, keep, kept, bound,
                                                     ctx->dev_status);
     KB_LAUNCH_CHECK(ctx, "prune_kernel");

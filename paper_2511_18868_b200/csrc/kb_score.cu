@@ -75,6 +75,7 @@ score_stats_kernel(int N, int K, int S, int G, RowWalk wk, const int32_t* __rest
                    const int32_t* __restrict__ pulls, const float* __restrict__ reward_sum,
                    const uint32_t* __restrict__ keep, int* __restrict__ part_p, float* __restrict__ part_r,
                    unsigned* __restrict__ part_a, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char sraw[];
     const int KS = K * S;
     int* sp = reinterpret_cast<int*>(sraw);                      // [K][S]
@@ -148,6 +149,7 @@ score_table_kernel(int K, int S, int G, kb_score_params prm, const int32_t* __re
                    const unsigned* __restrict__ part_a, float* __restrict__ table, unsigned* __restrict__ anyk,
                    float* __restrict__ cl_pulls, float* __restrict__ cl_mean, float* __restrict__ cl_index,
                    unsigned long long* __restrict__ g_key) {
+    kb_grid_dependency_wait();
     __shared__ long long s_np[TB_Y][TB_E];
     __shared__ float s_rs[TB_Y][TB_E];
     __shared__ unsigned s_any[TB_Y][TB_E];
@@ -204,6 +206,7 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
                   const float* __restrict__ dist2, const uint32_t* __restrict__ keep,
                   const float* __restrict__ bound, const float* __restrict__ table, float* __restrict__ arm_index,
                   unsigned long long* __restrict__ g_key) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) float stab[];  // [K][S]
     __shared__ unsigned long long s_best[8];
     const int b = blockIdx.y, tid = threadIdx.x, KS = K * S;
@@ -291,6 +294,7 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
 
 __global__ void score_decode_kernel(int B, const unsigned long long* __restrict__ g_key, int32_t* __restrict__ best_arm,
                                     float* __restrict__ best_val, int32_t* __restrict__ best_cluster_arm) {
+    kb_grid_dependency_wait();
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const unsigned long long key = g_key[2 * b], ckey = g_key[2 * b + 1];
@@ -331,15 +335,15 @@ kb_status kb_launch_score(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
     const RowWalk ws_walk = make_walk(SC_T, S, vec ? 4 : 1);
     if (vec) {
         KB_SMEM_OPTIN(ctx, score_stats_kernel<4>, smem_stats);
-        score_stats_kernel<4><<<dim3(G, B), SC_T, smem_stats, ctx->stream>>>(
+        kb_launch(score_stats_kernel<4>, dim3(G, B), SC_T, smem_stats, ctx->stream, 
             N, K, S, G, ws_walk, labels, pulls, reward_sum, keep, w.part_p, w.part_r, w.part_a, ctx->dev_status);
     } else {
         KB_SMEM_OPTIN(ctx, score_stats_kernel<1>, smem_stats);
-        score_stats_kernel<1><<<dim3(G, B), SC_T, smem_stats, ctx->stream>>>(
+        kb_launch(score_stats_kernel<1>, dim3(G, B), SC_T, smem_stats, ctx->stream, 
             N, K, S, G, ws_walk, labels, pulls, reward_sum, keep, w.part_p, w.part_r, w.part_a, ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "score_stats_kernel");
-    score_table_kernel<<<dim3((K * S + TB_E - 1) / TB_E, B), dim3(TB_E, TB_Y), 0, ctx->stream>>>(
+    kb_launch(score_table_kernel, dim3((K * S + TB_E - 1) / TB_E, B), dim3(TB_E, TB_Y), 0, ctx->stream, 
         K, S, G, p, t, w.part_p, w.part_r, w.part_a, w.table, w.anyk, cl_pulls, cl_mean, cl_index, w.key);
     KB_LAUNCH_CHECK(ctx, "score_table_kernel");
     if (N > 0) {
@@ -350,16 +354,16 @@ kb_status kb_launch_score(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
         const RowWalk wa = make_walk(256, S, vec ? 4 : 1);
         if (vec) {
             KB_SMEM_OPTIN(ctx, score_arms_kernel<4>, smem_arms);
-            score_arms_kernel<4><<<dim3(GA, B), 256, smem_arms, ctx->stream>>>(
+            kb_launch(score_arms_kernel<4>, dim3(GA, B), 256, smem_arms, ctx->stream, 
                 N, K, S, GA, wa, p, labels, dist2, keep, bound, w.table, arm_index, w.key);
         } else {
             KB_SMEM_OPTIN(ctx, score_arms_kernel<1>, smem_arms);
-            score_arms_kernel<1><<<dim3(GA, B), 256, smem_arms, ctx->stream>>>(
+            kb_launch(score_arms_kernel<1>, dim3(GA, B), 256, smem_arms, ctx->stream, 
                 N, K, S, GA, wa, p, labels, dist2, keep, bound, w.table, arm_index, w.key);
         }
         KB_LAUNCH_CHECK(ctx, "score_arms_kernel");
     }
-    score_decode_kernel<<<(B + 255) / 256, 256, 0, ctx->stream>>>(B, w.key, best_arm, best_val, best_cluster_arm);
+    kb_launch(score_decode_kernel, (B + 255) / 256, 256, 0, ctx->stream, B, w.key, best_arm, best_val, best_cluster_arm);
     KB_LAUNCH_CHECK(ctx, "score_decode_kernel");
     return KB_OK;
 }

@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(UP_T)
 update_sorted_kernel(int N, int D, int K, int G, int CH, const float* __restrict__ z,
                      const int32_t* __restrict__ labels, float* __restrict__ g_sums, int* __restrict__ g_counts,
                      int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char sm_raw[];
     int* hist = reinterpret_cast<int*>(sm_raw);                // [K]  counts, then scatter cursors
     int* offs = hist + K;                                      // [K+1] exclusive prefix
@@ -174,6 +175,7 @@ template <int V>
 __global__ void __launch_bounds__(UT_T)
 update_table_kernel(int N, int D, int K, int G, const float* __restrict__ z, const int32_t* __restrict__ labels,
                     float* __restrict__ part_sums, int* __restrict__ part_cnt, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
     extern __shared__ __align__(16) float tb[];
     float* acc = tb;                                       // [K][D]
     int* cnt = reinterpret_cast<int*>(tb + (size_t)K * D); // [K]
@@ -227,6 +229,7 @@ __global__ void __launch_bounds__(UF_E * UF_Y)
 update_table_finalize_kernel(int D, int K, int G, const float* __restrict__ part_sums,
                              const int* __restrict__ part_cnt, float* __restrict__ cent,
                              int32_t* __restrict__ counts) {
+    kb_grid_dependency_wait();
     __shared__ float s_sum[UF_Y][UF_E];
     __shared__ int s_cnt[UF_Y][UF_E];
     const int b = blockIdx.y, x = threadIdx.x, y = threadIdx.y, KD = K * D;
@@ -268,6 +271,7 @@ bool table_mode(int B, int N, int D, int K) {
 __global__ void update_finalize_kernel(size_t total, int D, const float* __restrict__ g_sums,
                                        const int* __restrict__ g_counts, float* __restrict__ cent,
                                        int32_t* __restrict__ counts) {
+    kb_grid_dependency_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
     size_t j = i / D;  // flat (b, cluster)
@@ -277,6 +281,7 @@ __global__ void update_finalize_kernel(size_t total, int D, const float* __restr
 }
 
 __global__ void update_empty_kernel(int total, int32_t* counts) {
+    kb_grid_dependency_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < total) counts[i] = 0;
 }
@@ -298,7 +303,7 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     if (B == 0) return KB_OK;
     if (N == 0) {
         if (counts) {
-            update_empty_kernel<<<(B * K + 255) / 256, 256, 0, ctx->stream>>>(B * K, counts);
+            kb_launch(update_empty_kernel, (B * K + 255) / 256, 256, 0, ctx->stream, B * K, counts);
             KB_LAUNCH_CHECK(ctx, "update_empty_kernel");
         }
         return KB_OK;
@@ -313,15 +318,15 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
         const size_t smem = ((size_t)K * D + K) * sizeof(float);
         if (D % 4 == 0) {
             KB_SMEM_OPTIN(ctx, update_table_kernel<4>, smem);
-            update_table_kernel<4><<<dim3(G, B), UT_T, smem, ctx->stream>>>(N, D, K, G, z, labels, part_sums, part_cnt,
+            kb_launch(update_table_kernel<4>, dim3(G, B), UT_T, smem, ctx->stream, N, D, K, G, z, labels, part_sums, part_cnt,
                                                                          ctx->dev_status);
         } else {
             KB_SMEM_OPTIN(ctx, update_table_kernel<1>, smem);
-            update_table_kernel<1><<<dim3(G, B), UT_T, smem, ctx->stream>>>(N, D, K, G, z, labels, part_sums, part_cnt,
+            kb_launch(update_table_kernel<1>, dim3(G, B), UT_T, smem, ctx->stream, N, D, K, G, z, labels, part_sums, part_cnt,
                                                                          ctx->dev_status);
         }
         KB_LAUNCH_CHECK(ctx, "update_table_kernel");
-        update_table_finalize_kernel<<<dim3((K * D + UF_E - 1) / UF_E, B), dim3(UF_E, UF_Y), 0, ctx->stream>>>(
+        kb_launch(update_table_finalize_kernel, dim3((K * D + UF_E - 1) / UF_E, B), dim3(UF_E, UF_Y), 0, ctx->stream, 
             D, K, G, part_sums, part_cnt, c, counts);
         KB_LAUNCH_CHECK(ctx, "update_table_finalize_kernel");
         return KB_OK;
@@ -353,16 +358,16 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     dim3 grid((unsigned)G, B);
     if (V == 4) {
         KB_SMEM_OPTIN(ctx, update_sorted_kernel<4>, smem);
-        update_sorted_kernel<4><<<grid, UP_T, smem, ctx->stream>>>(N, D, K, (int)G, CH, z, labels, g_sums, g_counts,
+        kb_launch(update_sorted_kernel<4>, grid, UP_T, smem, ctx->stream, N, D, K, (int)G, CH, z, labels, g_sums, g_counts,
                                                                   ctx->dev_status);
     } else {
         KB_SMEM_OPTIN(ctx, update_sorted_kernel<1>, smem);
-        update_sorted_kernel<1><<<grid, UP_T, smem, ctx->stream>>>(N, D, K, (int)G, CH, z, labels, g_sums, g_counts,
+        kb_launch(update_sorted_kernel<1>, grid, UP_T, smem, ctx->stream, N, D, K, (int)G, CH, z, labels, g_sums, g_counts,
                                                                   ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "update_sorted_kernel");
     size_t total = (size_t)B * K * D;
-    update_finalize_kernel<<<(unsigned)((total + 255) / 256), 256, 0, ctx->stream>>>(total, D, g_sums, g_counts, c,
+    kb_launch(update_finalize_kernel, (unsigned)((total + 255) / 256), 256, 0, ctx->stream, total, D, g_sums, g_counts, c,
                                                                                     counts);
     KB_LAUNCH_CHECK(ctx, "update_finalize_kernel");
     return KB_OK;
