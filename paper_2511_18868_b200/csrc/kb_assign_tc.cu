@@ -53,7 +53,9 @@ constexpr int PANEL = BN * KBF * 4;      // 16 KB: one hi or lo panel
 constexpr int STAGE = 2 * PANEL;         // hi + lo
 constexpr int EXT = 4096;                // fp16 split: the constant-term operand of one centroid tile (128 x 16 halfs)
 constexpr int SLOT_F16 = STAGE + EXT;    // a stage slot of the fp16 kernel (a multiple of 1024 bytes)
-constexpr int XCOLS = 8;                 // TMEM columns of a row's constant-term operand (16 halfs)
+constexpr int XCOLS = 8;
+constexpr int PREP_MAXG = 64;             // blocks per instance of the fp16 preparation kernel (at most)
+constexpr int INST_STRIDE = 1 + PREP_MAXG; // floats per instance: s_c, then every preparation block's largest ||c||^2                 // TMEM columns of a row's constant-term operand (16 halfs)
 constexpr int NSTAGE = 4;
 constexpr int TC_THREADS = 448;
 constexpr int TMEM_COLS = 512;
@@ -246,7 +248,8 @@ struct TcParams {
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
     const float* cnorm;            // [B][Kpad]
     const unsigned char* bext;     // fp16 split: [B][NT][EXT] constant-term operand of every centroid tile
-    const float* inst;             // fp16 split: [B][2] the instance's centroid scale s_c and its largest ||c||^2
+    const float* inst;             // fp16 split: [B][INST_STRIDE] centroid scale s_c, then per-block largest ||c||^2
+    int gprep;                     // blocks per instance the preparation kernel ran with
     int32_t* labels;
     float* approx;                 // optional: ||z||^2 + best score (expanded-form d^2), diagnostics
     int* flag_count;               // [0]: rows queued for a two-candidate check, [1]: for a full re-evaluation
@@ -334,7 +337,7 @@ __device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
 //   bimg  [B][NT][nkb][hi panel | lo panel]   128-byte-swizzled K-major panels, 64 features per row
 //   bext  [B][NT][EXT]   the 16 extra features of each centroid, K-major without swizzle
 //                        (8-row x 16-byte core matrices: k-halves 128 bytes apart, row groups 256)
-//   inst  [B][2]         s_c and the largest ||c_j||^2 of the instance
+//   inst  [B][1 + blocks] s_c, then each block's largest ||c_j||^2 (plain stores: nothing to clear)
 // Every block first scans its instance's centroids for the two maxima (the table is small and
 // sits in L2), then converts its share of the centroids: one warp per centroid, lane q owns the
 // 16-byte chunk q of the fp32 row (D <= 128).
@@ -365,7 +368,8 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
 #pragma unroll
     for (int w = 0; w < 8; ++w) m = fmaxf(m, s_m[w]);
     const float sc = pow2_scale(m);
-    if (blockIdx.x == 0 && threadIdx.x == 0) inst[2 * b] = sc;
+    __shared__ float s_n[8];
+    if (blockIdx.x == 0 && threadIdx.x == 0) inst[(size_t)b * INST_STRIDE] = sc;
     float nmax = 0.f;                                      // largest ||c_j||^2 among this warp's centroids
 
     for (int j = blockIdx.x * 8 + warp; j < Kpad; j += gridDim.x * 8) {
@@ -394,9 +398,14 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
             *reinterpret_cast<uint4*>(e + 128) = make_uint4(0u, 0u, 0u, 0u);
         }
     }
-    // the instance's largest squared norm (the caller cleared the word; non-negative floats order
-    // like their bit patterns)
-    if (lane == 0 && nmax > 0.f) atomicMax(reinterpret_cast<int*>(inst) + 2 * b + 1, __float_as_int(nmax));
+    // this block's largest squared norm; the contraction kernel takes the maximum over the blocks
+    if (lane == 0) s_n[warp] = nmax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) nmax = fmaxf(nmax, s_n[w]);
+        inst[(size_t)b * INST_STRIDE + 1 + blockIdx.x] = nmax;
+    }
 }
 
 // ---- the contraction -------------------------------------------------------------------
@@ -503,7 +512,13 @@ assign_tc_kernel(const TcParams p) {
     // the preceding kernel; from here on its results are read
     kb_grid_dependency_wait();
     if (F16) {
-        for (int j = tid; j < 2 * p.B; j += TC_THREADS) cn[j] = p.inst[j];     // per instance: s_c, largest ||c||^2
+        for (int j = tid; j < p.B; j += TC_THREADS) {                          // per instance: s_c, largest ||c||^2
+            const float* ib = p.inst + (size_t)j * INST_STRIDE;
+            float nm = 0.f;
+            for (int g = 0; g < p.gprep; ++g) nm = fmaxf(nm, ib[1 + g]);
+            cn[2 * j] = ib[0];
+            cn[2 * j + 1] = nm;
+        }
     } else {
         for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) cn[j] = p.cnorm[j];   // all instances' centroid norms
     }
@@ -1119,7 +1134,7 @@ size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool 
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
     const size_t Kpad = (size_t)(K + BN - 1) / BN * BN;
     return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + kb_align256(B * Kpad * 32) +
-           kb_align256((size_t)B * 8) + 256 + kb_align256((size_t)B * N * 8) + kb_align256((size_t)B * N * 4);
+           kb_align256((size_t)B * INST_STRIDE * 4) + 256 + kb_align256((size_t)B * N * 8) + kb_align256((size_t)B * N * 4);
 }
 
 // what the kernel can run at all
@@ -1146,16 +1161,16 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     float* cnorm = reinterpret_cast<float*>(ws + kb_align256((size_t)B * Kpad * D * 8));
     unsigned char* bext = reinterpret_cast<unsigned char*>(cnorm) + kb_align256((size_t)B * Kpad * 4);
     float* inst = reinterpret_cast<float*>(bext + kb_align256((size_t)B * Kpad * 32));
-    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(inst) + kb_align256((size_t)B * 8));
+    int* flag_count = reinterpret_cast<int*>(reinterpret_cast<char*>(inst) + kb_align256((size_t)B * INST_STRIDE * 4));
     int2* pair_rows = reinterpret_cast<int2*>(reinterpret_cast<char*>(flag_count) + 256);
     int32_t* full_rows = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(pair_rows) + kb_align256((size_t)B * N * 8));
 
     // the split: fp16 hi/lo (kind::f16, 16 features per instruction) unless the tf32 split is forced
     const bool f16 = ctx->assign_path != 3;
     const int nkb = f16 ? (D + 63) / 64 : D / KBF;
+    int gprep = 1;
     if (f16) {
-        KB_MEMSET(ctx, inst, 0, (size_t)B * 8);
-        const int gprep = (Kpad + 7) / 8 < 64 ? (Kpad + 7) / 8 : 64;
+        gprep = (Kpad + 7) / 8 < PREP_MAXG ? (Kpad + 7) / 8 : PREP_MAXG;
         kb_launch(tc_prep_f16_kernel, dim3(gprep, B), 256, 0, ctx->stream, K, D, Kpad, nkb, c, bimg, bext, inst, flag_count);
     } else
         kb_launch(tc_prep_kernel, dim3((Kpad + 7) / 8, B), 256, 0, ctx->stream, K, D, Kpad, nkb, c, bimg, cnorm, flag_count);
@@ -1165,6 +1180,7 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     p.B = B; p.N = N; p.D = D; p.K = K; p.Kpad = Kpad;
     p.nkb = nkb;
     p.DC = f16 ? 32 * nkb : D;
+    p.gprep = gprep;
     p.tiles_per_inst = (N + BM - 1) / BM;
     p.total_tiles = p.tiles_per_inst * B;
     p.nxb = tc_smem_bytes(D, Kpad * B, 2, f16) <= (size_t)ctx->max_smem_optin ? 2 : 1;

@@ -280,6 +280,14 @@ __global__ void update_finalize_kernel(size_t total, int D, const float* __restr
     if (counts && i - j * D == 0) counts[j] = n;
 }
 
+// clears the accumulators (a kernel rather than a memset node, so that it chains with its
+// neighbours by programmatic dependent launch)
+__global__ void update_zero_kernel(size_t n16, uint4* __restrict__ p) {
+    kb_grid_dependency_wait();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n16) p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
 __global__ void update_empty_kernel(int total, int32_t* counts) {
     kb_grid_dependency_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -333,7 +341,9 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
     }
     float* g_sums = reinterpret_cast<float*>(ctx->ws);
     int* g_counts = reinterpret_cast<int*>(ctx->ws + kb_align256((size_t)B * K * D * sizeof(float)));
-    KB_MEMSET(ctx, ctx->ws, 0, need);
+    kb_launch(update_zero_kernel, (unsigned)((need / 16 + 255) / 256), 256, 0, ctx->stream, need / 16,
+              reinterpret_cast<uint4*>(ctx->ws));
+    KB_LAUNCH_CHECK(ctx, "update_zero_kernel");
 
     // CTAs per instance: about two per SM in total, each with at most UP_MAXROWS rows and
     // enough rows to be worth a sort
