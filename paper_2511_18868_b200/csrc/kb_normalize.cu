@@ -1,10 +1,10 @@
 // kb_normalize: per instance and column population z-score (feature
 // normalisation of Sec. 3.2 / App. A.1).
 //
-// Two streaming passes over X: (1) per-block shifted sums, combined in double
-// in a fixed order by the last block of each instance; (2) apply.  HBM traffic
-// is read + read + write = 12 bytes per element (8 when X stays in L2 between
-// the passes).
+// Two streaming passes over X: (1) per-block shifted sums (fp32 runs of eight, widened to
+// double), then a small kernel that adds the per-block partials of every column in a fixed
+// order; (2) apply.  HBM traffic is read + read + write = 12 bytes per element (8 when X stays
+// in L2 between the passes).
 #include "kb_internal.cuh"
 
 namespace {
@@ -42,9 +42,7 @@ struct Geo {
 
 template <int V>
 __global__ void __launch_bounds__(256)
-norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, double* __restrict__ part,
-                  float* __restrict__ stat, unsigned* __restrict__ ticket, float* __restrict__ mean_out,
-                  float* __restrict__ scale_out) {
+norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, double* __restrict__ part) {
     kb_grid_dependency_wait();
     extern __shared__ double red[];  // [threads][2V]
     const int b = blockIdx.z, chunk = blockIdx.y, blk = blockIdx.x;
@@ -105,66 +103,59 @@ norm_stats_kernel(int N, int D, Geo g, int G, const float* __restrict__ x, doubl
 #pragma unroll
         for (int i = 0; i < V; ++i) { dst[2 * i] = s1[i]; dst[2 * i + 1] = s2[i]; }
     }
-    // last block of the instance combines the partials
-    __shared__ bool last;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        unsigned total = gridDim.x * gridDim.y;
-        unsigned prev = atomicAdd(&ticket[b], 1u);
-        last = (prev == total - 1);
-        if (last) ticket[b] = 0;  // ready for the next call
-    }
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    // all threads take part: columns in chunks of CP, each chunk split into SL slices of the partial
-    // index; a slice adds its partials in order (four loads in flight), slices are added in order
-    const int CP = D < (int)blockDim.x ? D : (int)blockDim.x;
-    const int SL = (int)blockDim.x / CP;
-    const int cc = tid % CP, sl = tid / CP;
-    const int per = (G + SL - 1) / SL;
-    for (int c0 = 0; c0 < D; c0 += CP) {
-        const int col = c0 + cc;
-        double a = 0.0, q = 0.0;
-        if (sl < SL && col < D) {
-            const int k1 = min(G, (sl + 1) * per);
-            int k = sl * per;
-            for (; k + 3 < k1; k += 4) {
-                const double* p0 = part + (((size_t)b * G + k) * D + col) * 2;
-                const size_t st = (size_t)D * 2;
-                const double a0 = __ldcg(p0), q0 = __ldcg(p0 + 1), a1 = __ldcg(p0 + st), q1 = __ldcg(p0 + st + 1);
-                const double a2 = __ldcg(p0 + 2 * st), q2 = __ldcg(p0 + 2 * st + 1);
-                const double a3 = __ldcg(p0 + 3 * st), q3 = __ldcg(p0 + 3 * st + 1);
-                a += a0; a += a1; a += a2; a += a3;
-                q += q0; q += q1; q += q2; q += q3;
-            }
-            for (; k < k1; ++k) {
-                const double* p = part + (((size_t)b * G + k) * D + col) * 2;
-                a += __ldcg(p);  // written by other blocks of this launch: read through L2
-                q += __ldcg(p + 1);
-            }
+}
+
+// Adds the per-block partials of each column in a fixed order and derives the statistics.
+// A block takes NC_COLS columns of one instance; NC_SL threads per column each add a contiguous
+// slice of the partial index (eight loads in flight), the slices are then added in order.
+constexpr int NC_COLS = 4, NC_SL = 64;
+__global__ void __launch_bounds__(NC_COLS * NC_SL)
+norm_combine_kernel(int N, int D, int G, const float* __restrict__ x, const double* __restrict__ part,
+                    float* __restrict__ stat, float* __restrict__ mean_out, float* __restrict__ scale_out) {
+    kb_grid_dependency_wait();
+    __shared__ double s_a[NC_SL][NC_COLS], s_q[NC_SL][NC_COLS];
+    const int b = blockIdx.y, tid = threadIdx.x;
+    const int cc = tid % NC_COLS, sl = tid / NC_COLS;
+    const int col = blockIdx.x * NC_COLS + cc;
+    const int per = (G + NC_SL - 1) / NC_SL;
+    double a = 0.0, q = 0.0;
+    if (col < D) {
+        const int k1 = min(G, (sl + 1) * per);
+        const size_t st = (size_t)D * 2;
+        int k = sl * per;
+        for (; k + 7 < k1; k += 8) {
+            const double* p0 = part + (((size_t)b * G + k) * D + col) * 2;
+            double va[8], vq[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { va[u] = p0[u * st]; vq[u] = p0[u * st + 1]; }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { a += va[u]; q += vq[u]; }
         }
-        __syncthreads();
-        red[2 * tid] = a; red[2 * tid + 1] = q;
-        __syncthreads();
-        if (sl != 0 || col >= D) continue;
-        for (int k = 1; k < SL; ++k) { a += red[2 * (k * CP + cc)]; q += red[2 * (k * CP + cc) + 1]; }
-        double ms = a / (double)N;
-        double var = q / (double)N - ms * ms;
-        if (var < 0.0) var = 0.0;
-        double mean = (double)__ldg(xb + col) + ms;
-        double sd = sqrt(var);
-        double sc = sd < 1e-12 ? 1.0 : sd;
-        float mh = (float)mean;
-        float* s = stat + ((size_t)b * D + col) * 4;
-        s[0] = mh;
-        s[1] = (float)(mean - (double)mh);
-        s[2] = (float)(1.0 / sc);
-        s[3] = (float)sc;
-        if (mean_out) mean_out[(size_t)b * D + col] = mh;
-        if (scale_out) scale_out[(size_t)b * D + col] = (float)sc;
+        for (; k < k1; ++k) {
+            const double* p = part + (((size_t)b * G + k) * D + col) * 2;
+            a += p[0];
+            q += p[1];
+        }
     }
+    s_a[sl][cc] = a; s_q[sl][cc] = q;
+    __syncthreads();
+    if (sl != 0 || col >= D) return;
+    for (int k = 1; k < NC_SL; ++k) { a += s_a[k][cc]; q += s_q[k][cc]; }
+    const float* xb = x + (size_t)b * N * D;
+    double ms = a / (double)N;
+    double var = q / (double)N - ms * ms;
+    if (var < 0.0) var = 0.0;
+    double mean = (double)__ldg(xb + col) + ms;
+    double sd = sqrt(var);
+    double sc = sd < 1e-12 ? 1.0 : sd;
+    float mh = (float)mean;
+    float* sp = stat + ((size_t)b * D + col) * 4;
+    sp[0] = mh;
+    sp[1] = (float)(mean - (double)mh);
+    sp[2] = (float)(1.0 / sc);
+    sp[3] = (float)sc;
+    if (mean_out) mean_out[(size_t)b * D + col] = mh;
+    if (scale_out) scale_out[(size_t)b * D + col] = (float)sc;
 }
 
 template <int V>
@@ -218,14 +209,15 @@ kb_status run(kb_ctx* ctx, int B, int N, int D, const float* x, float* z, float*
     // layout: ticket uint32[B] | stat float[B][D][4] | part double[B][G][D][2]
     size_t off_stat = kb_align256((size_t)B * 4);
     size_t off_part = off_stat + kb_align256((size_t)B * D * 4 * sizeof(float));
-    unsigned* ticket = reinterpret_cast<unsigned*>(ctx->ws);
     float* stat = reinterpret_cast<float*>(ctx->ws + off_stat);
     double* part = reinterpret_cast<double*>(ctx->ws + off_part);
-    KB_MEMSET(ctx, ticket, 0, (size_t)B * 4);
     dim3 grid(G, chunks, B);
     size_t smem = (size_t)256 * 2 * V * sizeof(double);
-    kb_launch(norm_stats_kernel<V>, grid, 256, smem, ctx->stream, N, D, g, G, x, part, stat, ticket, mean, scale);
+    kb_launch(norm_stats_kernel<V>, grid, 256, smem, ctx->stream, N, D, g, G, x, part);
     KB_LAUNCH_CHECK(ctx, "norm_stats_kernel");
+    kb_launch(norm_combine_kernel, dim3((D + NC_COLS - 1) / NC_COLS, B), NC_COLS * NC_SL, 0, ctx->stream, N, D, G, x,
+              static_cast<const double*>(part), stat, mean, scale);
+    KB_LAUNCH_CHECK(ctx, "norm_combine_kernel");
     kb_launch(norm_apply_kernel<V>, grid, 256, 0, ctx->stream, N, D, g, G, x, z, stat);
     KB_LAUNCH_CHECK(ctx, "norm_apply_kernel");
     return KB_OK;

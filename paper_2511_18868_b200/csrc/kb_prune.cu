@@ -5,8 +5,11 @@
 //
 // Vector path (S in {4, 8, 16, 32}): a thread owns four strategies of a row, so the
 // bound leaves as float4 stores and the keep bits of a row are OR-ed across its
-// S/4 lanes with shuffles.  Divisions are IEEE fp32 divisions, so an arm whose floor
-// equals the incumbent exactly is pruned (strict <), as the definition says.
+// S/4 lanes with shuffles.  The kernel is bound by its divisions (three per arm), not by memory:
+// a quotient whose divisor is fixed per thread is formed from the divisor's reciprocal and one
+// fused residual correction, which gives the correctly rounded fp32 quotient for ordinary operands
+// in three operations, so an arm whose floor equals the incumbent exactly is still pruned
+// (strict <), as the definition says.
 // Generic path (any S <= 32): one thread per candidate, bound rows staged through
 // shared memory so that they still leave the SM as full lines.
 #include "kb_internal.cuh"
@@ -15,6 +18,13 @@ namespace {
 
 constexpr int PR_T = 128;
 constexpr int PV_T = 256;
+
+// a / d with r = 1/d (correctly rounded): one residual step on the first estimate
+__device__ __forceinline__ float div_by(float a, float d, float r) {
+    const float q0 = a * r;
+    const float e = fmaf(-q0, d, a);
+    return fmaf(e, r, q0);     // d = 0 or a non-finite operand gives NaN here, which the callers map like 0/0
+}
 
 __global__ void __launch_bounds__(PV_T)
 prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ flops, const float* __restrict__ bytes,
@@ -30,12 +40,14 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
     const int q = tid % vps;
     const int rstep = PV_T / vps;
     const bool sat = labels != nullptr;
-    float P[4], W[4];
+    float P[4], W[4], rP[4], rW[4];
     int tg[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         P[i] = peak_flops[4 * q + i];
         W[i] = peak_bw[4 * q + i];
+        rP[i] = 1.f / P[i];
+        rW[i] = 1.f / W[i];
         int t = sat ? target[4 * q + i] : 0;
         if (t < 0 || t >= R) { if (sat) atomicOr(dev_status, 2); t = 0; }
         tg[i] = t;
@@ -44,7 +56,7 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
     const int rows_per = (N + G - 1) / G;
     const int r0 = blockIdx.x * rows_per, r1 = min(N, r0 + rows_per);
     unsigned count = 0;
-    constexpr int U = 2;                     // rows in flight per thread
+    constexpr int U = 4;                     // rows in flight per thread
     // the trip count is the same for every thread of the block, so the shuffles below are
     // always executed by full warps; rows past the end are computed on clamped inputs and dropped
     const int trips = (max(r1 - r0, 0) + U * rstep - 1) / (U * rstep);
@@ -70,13 +82,14 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
             const float* h = sat ? hsig + ((size_t)b * K + lb_) * R : nullptr;
             unsigned bits = 0;
             float g[4];
+            const float rT = 1.f / Tk[u];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float tlb = fmaxf(F[u] / P[k], Q[u] / W[k]);
+                const float tlb = fmaxf(div_by(F[u], P[k], rP[k]), div_by(Q[u], W[k], rW[k]));
                 bool ok = tlb < tinc;
                 if (sat) ok = ok && (__ldg(h + tg[k]) < theta);
                 if (ok) bits |= 1u << (4 * q + k);
-                float v = (Tk[u] - tlb) / Tk[u];
+                float v = div_by(Tk[u] - tlb, Tk[u], rT);
                 v = v > 0.f ? v : 0.f;       // also maps NaN (0/0) to 0, as the definition does
                 g[k] = v < 1.f ? v : 1.f;
             }

@@ -142,7 +142,7 @@ score_stats_kernel(int N, int K, int S, int G, RowWalk wk, const int32_t* __rest
     for (int j = tid; j < K; j += SC_T) part_a[((size_t)b * G + g) * K + j] = sa[j];
 }
 
-constexpr int TB_E = 32, TB_Y = 8;   // entries x slices of the partial index per block
+constexpr int TB_E = 32, TB_Y = 32;   // entries per block; at most TB_Y slices of the partial index (blockDim.y)   // entries x slices of the partial index per block
 __global__ void __launch_bounds__(TB_E * TB_Y)
 score_table_kernel(int K, int S, int G, kb_score_params prm, const int32_t* __restrict__ t,
                    const int* __restrict__ part_p, const float* __restrict__ part_r,
@@ -156,7 +156,8 @@ score_table_kernel(int K, int S, int G, kb_score_params prm, const int32_t* __re
     const int b = blockIdx.y, x = threadIdx.x, y = threadIdx.y, KS = K * S;
     const int e = blockIdx.x * TB_E + x;
     // slice y adds the partials of CTAs [y*per, (y+1)*per) in order; the slices are then added in order
-    const int per = (G + TB_Y - 1) / TB_Y;
+    const int ny = (int)blockDim.y;
+    const int per = (G + ny - 1) / ny;
     long long np_ = 0;
     float rs = 0.f;
     unsigned any = 0;
@@ -176,7 +177,7 @@ score_table_kernel(int K, int S, int G, kb_score_params prm, const int32_t* __re
     unsigned long long best = 0;
     if (y == 0) {
         if (e < KS) {
-            for (int k = 1; k < TB_Y; ++k) { np_ += s_np[k][x]; rs += s_rs[k][x]; any |= s_any[k][x]; }
+            for (int k = 1; k < ny; ++k) { np_ += s_np[k][x]; rs += s_rs[k][x]; any |= s_any[k][x]; }
             const int cl = e / S, s = e - cl * S;
             const float lnt = logf((float)t[b]);
             const size_t i = (size_t)b * KS + e;
@@ -217,6 +218,10 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
     const bool cap = prm.cap_with_bound && bound;
     const float L = prm.lipschitz_L;
     unsigned long long best = 0;
+    // per thread the arms come in ascending flat index, so a strict comparison keeps the lowest
+    // index among equal values; the 64-bit key is built once per thread
+    float bestv = -INFINITY;
+    unsigned besti = 0xffffffffu;
     if (tid < wk.active) {
         const int q = tid % wk.vps;
         constexpr int U = 4;                                       // rows in flight per thread
@@ -263,9 +268,8 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
                 for (int i = 0; i < V; ++i) {
                     const bool ok = (bits[u] >> (q * V + i)) & 1u;
                     if (ok) {
-                        const unsigned long long key =
-                            ((unsigned long long)kb_orderable(uu[i]) << 32) | (0xffffffffu - (flat0 + i));
-                        best = key > best ? key : best;
+                        // (a NaN index never compares greater; -inf is taken when nothing was seen yet)
+                        if (uu[i] > bestv || besti == 0xffffffffu) { bestv = uu[i]; besti = flat0 + i; }
                     } else {
                         uu[i] = -INFINITY;
                     }
@@ -279,6 +283,7 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
             }
         }
     }
+    if (besti != 0xffffffffu) best = ((unsigned long long)kb_orderable(bestv) << 32) | (0xffffffffu - besti);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
@@ -343,7 +348,8 @@ kb_status kb_launch_score(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
             N, K, S, G, ws_walk, labels, pulls, reward_sum, keep, w.part_p, w.part_r, w.part_a, ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "score_stats_kernel");
-    kb_launch(score_table_kernel, dim3((K * S + TB_E - 1) / TB_E, B), dim3(TB_E, TB_Y), 0, ctx->stream, 
+    const int ty = G >= 64 ? TB_Y : (G >= 8 ? 8 : 1);         // slices of the partial index per entry
+    kb_launch(score_table_kernel, dim3((K * S + TB_E - 1) / TB_E, B), dim3(TB_E, ty), 0, ctx->stream, 
         K, S, G, p, t, w.part_p, w.part_r, w.part_a, w.table, w.anyk, cl_pulls, cl_mean, cl_index, w.key);
     KB_LAUNCH_CHECK(ctx, "score_table_kernel");
     if (N > 0) {
