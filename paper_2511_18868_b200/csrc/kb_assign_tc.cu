@@ -423,6 +423,15 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
 constexpr int KEY_BITS = 7;
 constexpr int KEY_MASK = ~((1 << KEY_BITS) - 1);
 constexpr int KEY_INF = 0x7fffffff;
+// fp16 split: the accumulator g_i d2 is turned into a FIXED-POINT key instead.  One FFMA maps it onto
+// [2^23, 2^23 + 2^22) (the row's largest possible value, 2 g_i (||z||^2 + max ||c||^2), lands on the
+// top), whose fp32 bits are 0x4B000000 + n with n the 22-bit quantised distance; one integer
+// multiply-add turns the bits into n * KQ_MUL + column.  Both run on the FMA pipe, which the
+// epilogue leaves idle, while the integer/logic pipe is what bounds the kernel.  KQ_MUL is odd and
+// above 64 so that the product is not rewritten as shifts.
+constexpr uint32_t KQ_MUL = 157u;
+constexpr float KQ_TOP = 4194303.f;                                  // 2^22 - 1
+constexpr uint32_t KQ_BASE = 0u - 0x4B000000u * KQ_MUL;              // removes the bits of 2^23
 static_assert(BN == (1 << KEY_BITS), "a key's index field addresses one accumulator tile");
 
 template <bool TRACK2>
@@ -465,6 +474,12 @@ struct RowBest {
 template <bool TRACK2, bool F16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 assign_tc_kernel(const TcParams p) {
+    // fp16 split: the hot loop keeps the two smallest keys of each sub-chunk (the 32 columns one
+    // tracker sees in an accumulator tile); the row's running best keeps three keys.  The third
+    // smallest distance of the row is then known unless the two smallest come from the same
+    // sub-chunk, in which case a near-tie goes to the full re-evaluation.
+    constexpr bool HOT3 = F16 ? false : TRACK2;           // hot-loop trackers keep a third key
+    constexpr bool ROW3 = F16 ? true : TRACK2;            // the running best keeps three keys, two tiles
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled panels
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -676,7 +691,13 @@ assign_tc_kernel(const TcParams p) {
             const float xn = xnorm[(it & 1) * BM + row_in_tile];
             const float rscale = xscale[(it & 1) * BM + row_in_tile];
             mbar_arrive_warp(BAR(XN_EMPTY + (it & 1)));
-            RowBest<TRACK2> rb;
+            RowBest<ROW3> rb;
+            // fp16 split: quantisation step of the keys in units of d2, and the factor that maps an
+            // accumulator value onto the key range
+            const float cmaxn = F16 ? cn[2 * b + 1] : 0.f;
+            const float range_d2 = fmaxf(2.f * (xn + cmaxn), 1e-30f);
+            const float kstep = range_d2 * (1.f / KQ_TOP);
+            const float kmul = KQ_TOP * fabsf(rscale) / range_d2;
             for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                 const uint32_t buf = q & 1u;
                 const uint32_t acc = lane_addr + COL_ACC + buf * BN + half * (BN / 2);
@@ -687,7 +708,7 @@ assign_tc_kernel(const TcParams p) {
                     TC_LD32(acc, r[0]);
                 }
                 pref = false;
-                KeyTracker<TRACK2> ta, tb;
+                KeyTracker<HOT3> ta, tb;
                 const float* cnp = cnb + nt * BN + half * (BN / 2);
                 // Two passes over a 32-column register buffer.  The first turns every accumulator value
                 // into its key in place: 32 independent short chains (load the column's constants,
@@ -698,11 +719,11 @@ assign_tc_kernel(const TcParams p) {
                     for (int j = 0; j < 32; j += 4) {
                         const int l = c * 32 + j;                  // column inside this thread's 64
                         int k0, k1, k2, k3;
-                        if (F16) {      // the accumulator already is g_i d2(i, j): rank it as it is
-                            k0 = ((int)v[j + 0] & KEY_MASK) | (l + 0);
-                            k1 = ((int)v[j + 1] & KEY_MASK) | (l + 1);
-                            k2 = ((int)v[j + 2] & KEY_MASK) | (l + 2);
-                            k3 = ((int)v[j + 3] & KEY_MASK) | (l + 3);
+                        if (F16) {      // the accumulator already is g_i d2(i, j): quantise it and append the column
+                            k0 = (int)(__float_as_uint(fmaf(__uint_as_float(v[j + 0]), kmul, 8388608.f)) * KQ_MUL + (KQ_BASE + (uint32_t)(l + 0)));
+                            k1 = (int)(__float_as_uint(fmaf(__uint_as_float(v[j + 1]), kmul, 8388608.f)) * KQ_MUL + (KQ_BASE + (uint32_t)(l + 1)));
+                            k2 = (int)(__float_as_uint(fmaf(__uint_as_float(v[j + 2]), kmul, 8388608.f)) * KQ_MUL + (KQ_BASE + (uint32_t)(l + 2)));
+                            k3 = (int)(__float_as_uint(fmaf(__uint_as_float(v[j + 3]), kmul, 8388608.f)) * KQ_MUL + (KQ_BASE + (uint32_t)(l + 3)));
                         } else {
                             const float4 n4 = *reinterpret_cast<const float4*>(cnp + c * 32 + j);
                             k0 = (__float_as_int(fmaf(-2.f, __uint_as_float(v[j + 0]), n4.x + xn)) & KEY_MASK) | (l + 0);
@@ -735,11 +756,20 @@ assign_tc_kernel(const TcParams p) {
                     }
                 }
                 process(r[1], 1);
-                ta.merge(tb);
-                const int hbit = half * (BN / 2);                  // the upper half's columns start at 64
-                rb.insert(ta.b0 | hbit, nt);
-                rb.insert(ta.b1 | hbit, nt);
-                if (TRACK2) rb.insert(ta.b2 | hbit, nt);
+                if (F16) {
+                    // both sub-chunks hand over their two smallest keys; the tile id carries the half
+                    const int tid2 = nt * 2 + half;
+                    rb.insert(ta.b0, tid2);
+                    rb.insert(ta.b1, tid2);
+                    rb.insert(tb.b0, tid2);
+                    rb.insert(tb.b1, tid2);
+                } else {
+                    ta.merge(tb);
+                    const int hbit = half * (BN / 2);              // the upper half's columns start at 64
+                    rb.insert(ta.b0 | hbit, nt);
+                    rb.insert(ta.b1 | hbit, nt);
+                    if (TRACK2) rb.insert(ta.b2 | hbit, nt);
+                }
             }
             if (!ok) break;
             // fold the upper half's running best into the lower half's through shared memory
@@ -752,29 +782,49 @@ assign_tc_kernel(const TcParams p) {
             if (half == 1) continue;
             rb.insert(__float_as_int(mg[0]), __float_as_int(mg[3]));
             rb.insert(__float_as_int(mg[1]), __float_as_int(mg[4]));
-            if (TRACK2) rb.r2 = min(rb.r2, __float_as_int(mg[2]));
+            if (ROW3) rb.r2 = min(rb.r2, __float_as_int(mg[2]));
             const int row = r0 + row_in_tile;
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
-                const int a0 = rb.column(rb.r0, rb.t0);
-                // fp16 split: the ranked values carry the row's factor g_i; take it out again
-                const float unscale = F16 ? fabsf(rscale) : 1.f;
-                const float b0 = rb.value(rb.r0) * unscale, b1 = rb.value(rb.r1) * unscale;
-                const float b2 = rb.value(rb.r2) * unscale;
+                int a0, a1;
+                float b0, b1, b2, delta;
+                bool third_known = ROW3;
+                if (F16) {
+                    // key = n * KQ_MUL + column (column inside the thread's 64; the tile id carries the
+                    // half); n * kstep is the squared distance.  A slightly negative distance gives a
+                    // negative key: it ranks first and reads as zero.
+                    auto quant = [](int key) {             // floor division: a negative key keeps its column
+                        return key >= 0 ? key / (int)KQ_MUL : -((-key + (int)KQ_MUL - 1) / (int)KQ_MUL);
+                    };
+                    const int n0 = quant(rb.r0), n1 = quant(rb.r1), n2 = quant(rb.r2);
+                    const int l0 = rb.r0 - n0 * (int)KQ_MUL, l1 = rb.r1 - n1 * (int)KQ_MUL;
+                    a0 = (rb.t0 >> 1) * BN + (rb.t0 & 1) * (BN / 2) + l0;
+                    a1 = (rb.t1 >> 1) * BN + (rb.t1 & 1) * (BN / 2) + l1;
+                    b0 = (float)max(n0, 0) * kstep; b1 = (float)max(n1, 0) * kstep; b2 = (float)max(n2, 0) * kstep;
+                    // near-tie bound: the split product's error, relative to ||z||^2 plus the largest
+                    // centroid norm of the instance (its centroids share one scale), plus two
+                    // quantisation steps
+                    delta = p.eps * (xn + cmaxn) + 2.f * kstep;
+                    // the third smallest is only known when the two smallest come from different
+                    // sub-chunks (same accumulator tile, same half, same tracker = same sub-chunk)
+                    third_known = !(rb.t0 == rb.t1 && ((l0 ^ l1) & 2) == 0);
+                } else {
+                    a0 = rb.column(rb.r0, rb.t0);
+                    a1 = rb.column(rb.r1, rb.t1);
+                    b0 = rb.value(rb.r0); b1 = rb.value(rb.r1); b2 = rb.value(rb.r2);
+                    // near-tie bound: the split product's error, relative to ||z||^2 plus the chosen
+                    // centroid's norm, plus what the dropped key bits can hide
+                    delta = p.eps * (xn + cnb[a0]) + 1.52587890625e-5f * fabsf(b1);
+                }
                 p.labels[flat] = a0;
                 if (p.approx) p.approx[flat] = b0;
-                // near-tie bound: the split product's error (relative to ||z||^2 plus the centroid's
-                // norm; the fp16 split shares one scale among an instance's centroids, so there the
-                // largest norm of the instance) plus what the dropped key bits can hide
-                const float cref = F16 ? cn[2 * b + 1] : cnb[a0];
-                const float delta = p.eps * (xn + cref) + 1.52587890625e-5f * fabsf(b1);
                 if (F16 && rscale < 0.f) {                     // row outside the fp16 range: exact scan over all K
                     const int slot = atomicAdd(p.flag_count + 1, 1);
                     p.full_rows[slot] = (int32_t)flat;
                 } else if (fabsf(b1 - b0) <= delta) {
-                    if (TRACK2 && fabsf(b2 - b0) > delta) {   // exactly two candidates: compare them exactly
+                    if (third_known && fabsf(b2 - b0) > delta) {   // exactly two candidates: compare them exactly
                         const int slot = atomicAdd(p.flag_count, 1);
-                        p.pair_rows[slot] = make_int2((int)flat, rb.column(rb.r1, rb.t1));
+                        p.pair_rows[slot] = make_int2((int)flat, a1);
                     } else {                                   // three or more (or unknown): exact scan over all K
                         const int slot = atomicAdd(p.flag_count + 1, 1);
                         p.full_rows[slot] = (int32_t)flat;
@@ -1034,18 +1084,26 @@ fixup_full(int N, int D, int K, int total, const float* __restrict__ z, const fl
     }
 }
 
-// One launch settles both queues: every block first takes its share of the two-candidate rows,
-// then of the rows that need all K centroids, in groups sized to the queue's length.
+// The two queues are settled by two kernels: the two-candidate rows by warps that need no shared
+// memory (full occupancy), the rows that need all K centroids by blocks that stage centroid tiles
+// in shared memory, in groups sized to the queue's length.
+__global__ void __launch_bounds__(FX_T)
+assign_fixup_pairs_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                          const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                          int32_t* __restrict__ labels) {
+    kb_grid_dependency_wait();
+    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
+}
+
 __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                    const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
-                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
+                    const int* __restrict__ flag_count, const int32_t* __restrict__ full_rows,
+                    int32_t* __restrict__ labels) {
     kb_grid_dependency_wait();
     extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_MAXROWS][FX_T / 32];
     __shared__ int red_i[FX_MAXROWS][FX_T / 32];
     __shared__ int s_inst[FX_MAXROWS];
-    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
     float* xrow = fx;
     float* ctile = fx + FX_MAXROWS * D;
     const int total = flag_count[1];
@@ -1205,10 +1263,13 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
 #undef KB_TC_LAUNCH
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
+    kb_launch(assign_fixup_pairs_kernel, 8 * ctx->sm_count, FX_T, 0, ctx->stream, N, D, K, z, c, flag_count, pair_rows, labels);
+    KB_LAUNCH_CHECK(ctx, "assign_fixup_pairs_kernel");
     const size_t fsmem = (size_t)FX_MAXROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
+    const int fblocks = (int)(((size_t)ctx->max_smem_optin / (fsmem + 2048)) < 1 ? 1 : ((size_t)ctx->max_smem_optin / (fsmem + 2048)));
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
-    kb_launch(assign_fixup_kernel, 4 * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count, pair_rows,
-                                                                        full_rows, labels);
+    kb_launch(assign_fixup_kernel, (fblocks > 4 ? 4 : fblocks) * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count,
+              full_rows, labels);
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
         KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));

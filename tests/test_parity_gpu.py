@@ -416,6 +416,40 @@ def test_assign_tensor_path(kbx, B, N, D, K, path):
     assert err.max() < 0.25 / 65536               # the re-evaluation bound covers the ranking error with margin
 
 
+@pytest.mark.parametrize("path", [2, 3], ids=["f16x3", "tf32x3"])
+@pytest.mark.parametrize("scale", [1e-6, 1.0, 3e4], ids=["tiny", "unit", "huge"])
+def test_assign_tensor_path_value_ranges(kbx, path, scale):
+    """The fp16 split scales rows and centroids by exact powers of two: data of any magnitude, rows far
+    outside the centroids' range, zero rows and a zero centroid must all come out like the fp32 definition."""
+    B, N, D, K = 1, 6000, 64, 256
+    cfg = wl.scaled(wl.CONFIGS["large"], B=B, N=N, D=D, K=K, components=96, S=2)
+    z, _, _ = oracle.normalize(wl.make_inputs(cfg, seed=17)["x"])
+    rng = np.random.default_rng(5)
+    c = z[:, rng.choice(N, K, replace=False)].copy()
+    z = z.copy()
+    z[0, 10:20] *= 1e5            # rows five orders of magnitude beyond every centroid
+    z[0, 20:24] *= 1e9            # ... and far outside what fp16 can scale to
+    z[0, 30:34] = 0.0             # zero rows
+    z[0, 40:44] *= 1e-7           # rows far smaller than the centroids
+    c[0, 7] = 0.0                 # a centroid at the origin
+    z, c = (z * np.float32(scale)).astype(np.float32), (c * np.float32(scale)).astype(np.float32)
+    ws(kbx, B, N, D, K, 1)
+    kbx.set_assign_options(path=path)
+    try:
+        labels, d2 = empty((B, N), torch.int32), empty((B, N))
+        kbx.cluster_assign(dev(z), dev(c), labels, d2)
+        assert kbx.assign_path() == path
+    finally:
+        kbx.set_assign_options(path=0)
+    assert kbx.device_status() == 0
+    ref = oracle.cluster_assign(z, c, want_margins=True)
+    got = host(labels)
+    ties = parity.labels_match(z, c, got, ref)
+    same = got == ref["labels"]
+    parity.close(host(d2)[same], ref["dist2"][same], atol=1e-7 * scale * scale, what="dist2")
+    print(f"[tc ranges path={path} scale={scale:g}] near-ties={ties}")
+
+
 def test_step_uses_tensor_path_when_eligible(kbx):
     cfg = wl.scaled(wl.CONFIGS["large"], N=8192 + 37, iters=2)
     inp = wl.make_inputs(cfg)
