@@ -39,10 +39,10 @@ DEFAULT_WORKLOAD = "large"
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant call's main kernel, per launch, from the
 # ncu captures summarised under profiles/ (bytes; None where no capture exists for that workload)
 TRAFFIC_FROM_NCU = {
-    # assign_tc_kernel, one launch: 67.30 MB read + 0.58 MB written (profiles/assign_tc_and_update_kernels.txt)
-    ("large", "assign"): 67.88e6,
-    # assign_tc_kernel at N = 262144: 135.35 + 3.96 MB; traffic grows with N, scaled x16 to N = 4194304
-    ("contraction", "assign"): 16 * 139.31e6,
+    # assign_tc_kernel, one launch: 67.25 MB read + 0.77 MB written (profiles/assign_tc_and_update_kernels.txt)
+    ("large", "assign"): 68.02e6,
+    # assign_tc_kernel at N = 262144: 134.84 + 5.47 MB; traffic grows with N, scaled x16 to N = 4194304
+    ("contraction", "assign"): 16 * 140.31e6,
 }
 
 # rows of the workload the CPU oracle is timed on (per instance), and instances
