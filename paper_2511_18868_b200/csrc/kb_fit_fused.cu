@@ -3,8 +3,11 @@
 // When an instance has at most 512 rows and D is 16, 32 or 64, per-call launches dominate
 // (a call moves a few KB): iters x (assign, update) + the final assign would be 2*iters+1
 // calls of several kernels each.  Here a CTA keeps its instance on chip for all iterations:
-//   * thread = row, the row lives in registers (D floats);
-//   * centroids live in shared memory and are read as warp-wide float4 broadcasts;
+//   * a thread owns FF_R rows, kept in registers (FF_R x D floats): every centroid value read
+//     from shared memory (a warp-wide float4 broadcast, which costs the shared-memory pipe as
+//     much as a full 512-byte access) then feeds FF_R rows, so the loop is bound by its FMAs
+//     and not by the broadcasts;
+//   * centroids live in shared memory;
 //     the distance is the direct form sum (z - c)^2, ascending centroid id, strict <
 //     (lowest id on ties) -- the same arithmetic as the row-wise assign kernel;
 //   * update: counting sort of the row ids by label in shared memory (integer atomics),
@@ -17,14 +20,17 @@
 
 namespace {
 
-constexpr int FF_T = 512;
+constexpr int FF_MAXROWS = 512;   // rows per instance at most
+// rows per thread (row = tid + u * threads): as many as the register file holds
+__host__ __device__ constexpr int ff_rows(int D) { return D <= 32 ? 4 : 2; }
 
 template <int D>
-__global__ void __launch_bounds__(FF_T)
+__global__ void __launch_bounds__(FF_MAXROWS / ff_rows(D))
 fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
                  int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                  int32_t* __restrict__ rep, int32_t* __restrict__ counts) {
     kb_grid_dependency_wait();
+    constexpr int FF_R = ff_rows(D), FF_T = FF_MAXROWS / FF_R;
     extern __shared__ __align__(16) unsigned char ff_raw[];
     constexpr int ZS = D + 1;                                       // padded row stride: conflict-free column walks
     float* cs = reinterpret_cast<float*>(ff_raw);                   // [K][D] centroids (16-byte aligned rows)
@@ -33,8 +39,8 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
     int* hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(zs + (size_t)N * ZS) + 7) & ~(uintptr_t)7);
     int* offs = hist + K;                                           // [K+1]
     unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [N] row ids in label order
-    __shared__ double s_red[FF_T / 32];
-    __shared__ int s_scan[FF_T / 32];
+    __shared__ double s_red[FF_MAXROWS / 64];
+    __shared__ int s_scan[FF_MAXROWS / 64];
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* zb = z + (size_t)b * N * D;
     float* cb = cent + (size_t)b * K * D;
@@ -49,33 +55,48 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
     for (int e = tid; e < K * D / 4; e += FF_T)
         reinterpret_cast<float4*>(cs)[e] = __ldg(reinterpret_cast<const float4*>(cb) + e);
     __syncthreads();
-    const bool active = tid < N;
-    float x[D];
+    bool active[FF_R];
+    float x[FF_R][D];
 #pragma unroll
-    for (int d = 0; d < D; ++d) x[d] = active ? zs[(size_t)tid * ZS + d] : 0.f;
+    for (int u = 0; u < FF_R; ++u) {
+        active[u] = tid + u * FF_T < N;
+#pragma unroll
+        for (int d = 0; d < D; ++d) x[u][d] = active[u] ? zs[(size_t)(tid + u * FF_T) * ZS + d] : 0.f;
+    }
 
-    float best = 0.f;
-    int arg = 0;
+    float best[FF_R];
+    int arg[FF_R];
     for (int it = 0; it <= iters; ++it) {
-        // ---- assign: nearest centroid of my row -------------------------------------------
-        best = INFINITY;
-        arg = 0;
+        // ---- assign: nearest centroid of my rows ------------------------------------------
+#pragma unroll
+        for (int u = 0; u < FF_R; ++u) { best[u] = INFINITY; arg[u] = 0; }
         for (int j = 0; j < K; ++j) {
             const float4* c4 = reinterpret_cast<const float4*>(cs + (size_t)j * D);
-            float acc = 0.f;
+            float acc[FF_R];
+#pragma unroll
+            for (int u = 0; u < FF_R; ++u) acc[u] = 0.f;
 #pragma unroll
             for (int q = 0; q < D / 4; ++q) {
                 const float4 c = c4[q];
-                const float e0 = x[4 * q] - c.x, e1 = x[4 * q + 1] - c.y, e2 = x[4 * q + 2] - c.z, e3 = x[4 * q + 3] - c.w;
-                acc = fmaf(e0, e0, acc); acc = fmaf(e1, e1, acc); acc = fmaf(e2, e2, acc); acc = fmaf(e3, e3, acc);
+#pragma unroll
+                for (int u = 0; u < FF_R; ++u) {
+                    const float e0 = x[u][4 * q] - c.x, e1 = x[u][4 * q + 1] - c.y, e2 = x[u][4 * q + 2] - c.z,
+                                e3 = x[u][4 * q + 3] - c.w;
+                    acc[u] = fmaf(e0, e0, acc[u]); acc[u] = fmaf(e1, e1, acc[u]);
+                    acc[u] = fmaf(e2, e2, acc[u]); acc[u] = fmaf(e3, e3, acc[u]);
+                }
             }
-            if (acc < best) { best = acc; arg = j; }
+#pragma unroll
+            for (int u = 0; u < FF_R; ++u)
+                if (acc[u] < best[u]) { best[u] = acc[u]; arg[u] = j; }
         }
         if (it == iters) break;                                     // the final assign has no update after it
         // ---- update: counting sort by label, then (cluster, column) sums ----------------------
         for (int j = tid; j < K; j += FF_T) hist[j] = 0;
         __syncthreads();
-        if (active) atomicAdd(&hist[arg], 1);
+#pragma unroll
+        for (int u = 0; u < FF_R; ++u)
+            if (active[u]) atomicAdd(&hist[arg[u]], 1);
         __syncthreads();
         {   // exclusive scan of hist (K may exceed the block: contiguous slices per thread)
             const int per = (K + FF_T - 1) / FF_T;
@@ -99,7 +120,9 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
         __syncthreads();
         for (int j = tid; j < K; j += FF_T) hist[j] = offs[j];      // scatter cursors
         __syncthreads();
-        if (active) perm[atomicAdd(&hist[arg], 1)] = (unsigned short)tid;
+#pragma unroll
+        for (int u = 0; u < FF_R; ++u)
+            if (active[u]) perm[atomicAdd(&hist[arg[u]], 1)] = (unsigned short)(tid + u * FF_T);
         __syncthreads();
         if (it == iters - 1 && counts)
             for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = offs[j + 1] - offs[j];
@@ -127,18 +150,24 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
         for (int j = tid; j < K; j += FF_T) rep_key[j] = ~0ull;
         __syncthreads();
     }
-    if (active) {
-        const size_t flat = (size_t)b * N + tid;
-        labels[flat] = arg;
-        if (dist2) dist2[flat] = best;
-        if (rep) atomicMin(&rep_key[arg], ((unsigned long long)__float_as_uint(best) << 32) | (unsigned)tid);
-    }
+#pragma unroll
+    for (int u = 0; u < FF_R; ++u)
+        if (active[u]) {
+            const int r = tid + u * FF_T;
+            const size_t flat = (size_t)b * N + r;
+            labels[flat] = arg[u];
+            if (dist2) dist2[flat] = best[u];
+            if (rep) atomicMin(&rep_key[arg[u]], ((unsigned long long)__float_as_uint(best[u]) << 32) | (unsigned)r);
+        }
     for (int e = tid; e < K * D / 4; e += FF_T)
         reinterpret_cast<float4*>(cb)[e] = reinterpret_cast<const float4*>(cs)[e];
     if (iters == 0 && counts)
         for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = 0;
     if (inertia) {
-        double s = kb_warp_sum(active ? (double)best : 0.0);
+        double mine = 0.0;
+#pragma unroll
+        for (int u = 0; u < FF_R; ++u) mine += active[u] ? (double)best[u] : 0.0;
+        double s = kb_warp_sum(mine);
         if (lane == 0) s_red[warp] = s;
     }
     __syncthreads();
@@ -162,7 +191,7 @@ size_t ff_smem(int N, int D, int K) {
 }  // namespace
 
 bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
-    if (B < 1 || N < 1 || N > FF_T || K < 1 || K > 4096) return false;
+    if (B < 1 || N < 1 || N > FF_MAXROWS || K < 1 || K > 4096) return false;
     if (D != 16 && D != 32 && D != 64) return false;
     return ff_smem(N, D, K) + 256 <= (size_t)ctx->max_smem_optin;
 }
@@ -172,13 +201,13 @@ kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters
     const size_t smem = ff_smem(N, D, K);
     if (D == 16) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        kb_launch(fit_fused_kernel<16>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     } else if (D == 32) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        kb_launch(fit_fused_kernel<32>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     } else {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        kb_launch(fit_fused_kernel<64>, B, FF_T, smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
     }
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;
