@@ -335,17 +335,25 @@ def run_ours(args, cfg):
     hbm_time = alg[dominant]["bytes"] / (hbm * 1e9)
     alu_time = alg[dominant]["flops"] / (ffma_tflops * 1e12)
     if dominant == "assign" and assign_path in (2, 3):
+        # the dominant KERNEL is the contraction kernel: its own event pairs give its launch duration; the
+        # whole call (preparation + contraction + fix-up kernels) is reported beside it
+        kms, kcalls = per_class.get("assign_kernel", (0.0, 0))
+        k_s = (kms / kcalls * 1e-3) if kcalls else dk["avg_us"] * 1e-6
+        k_tflops = alg["assign"]["flops"] / k_s / 1e12
         # three tensor-core products per fp32-equivalent product.  fp16 split (path 2): the measured bf16
         # GEMM peak is the 16-bit tensor rate itself; tf32 split (path 3): half of it (nominal ratio).
         kind_peak = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5)
         split = "fp16 hi/lo split, kind::f16" if assign_path == 2 else "3xTF32, kind::tf32"
-        roof = {"bound": "tensor", "achieved": dk["TFLOPs"], "peak": kind_peak / 3.0, "unit": "TFLOP/s",
-                "frac": dk["TFLOPs"] / (kind_peak / 3.0), "traffic": None,
-                "kernel": f"kb_cluster_assign (tcgen05 {split}; prep + contraction + fix-up per call)",
+        roof = {"bound": "tensor", "achieved": k_tflops, "peak": kind_peak / 3.0, "unit": "TFLOP/s",
+                "frac": k_tflops / (kind_peak / 3.0), "traffic": None,
+                "kernel": f"assign_tc_kernel (tcgen05 {split}), the contraction kernel of kb_cluster_assign",
+                "kernel_avg_us": k_s * 1e6, "kernel_launches": int(kcalls),
+                "whole_call": {"avg_us": dk["avg_us"], "TFLOPs": dk["TFLOPs"], "frac": dk["TFLOPs"] / (kind_peak / 3.0),
+                               "what": "preparation + contraction + fix-up kernels of one kb_cluster_assign"},
                 "peak_source": f"{peaks['source']} bf16 GEMM peak" + (" x 0.5 (tf32)" if assign_path == 3 else "") +
                                " / 3 (split products), fp32-equivalent",
                 "algorithmic_flops_per_launch": alg["assign"]["flops"],
-                "executed_tensor_TFLOPs": 3.0 * dk["TFLOPs"]}
+                "executed_tensor_TFLOPs": 3.0 * k_tflops}
     elif dominant in ("assign", "fit") and alu_time > hbm_time:
         roof = {"bound": "alu", "achieved": dk["TFLOPs"], "peak": ffma_tflops, "unit": "TFLOP/s",
                 "frac": dk["TFLOPs"] / ffma_tflops, "traffic": None,

@@ -93,7 +93,8 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_SCORE 4
 #define KB_T_INIT 5
 #define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
-#define KB_T_COUNT 7
+#define KB_T_ASSIGN_KERNEL 7 /* the tensor-core contraction kernel alone (nested inside KB_T_ASSIGN or KB_T_FIT) */
+#define KB_T_COUNT 8
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
 
@@ -255,8 +256,10 @@ kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float
  * are consistent with the returned centroids (Sec. 3.3).  Same arguments as
  * the two calls it is made of; counts are those of the last update.
  * Instances of at most 512 rows with D in {16, 32, 64} run the whole loop in one launch
- * (one CTA per instance, the instance resident on chip), unless kb_set_assign_options
- * forces an assign path. */
+ * (one CTA per instance, the instance resident on chip); a single instance of up to about
+ * 75 000 rows with D in {16, 32, 64} that is too small for the tensor-core kernel (K < 128)
+ * runs it in one cooperative launch (its rows spread over the SMs and kept on chip, one
+ * grid-wide barrier per iteration); both unless kb_set_assign_options forces an assign path. */
 kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z,
                          float* centroids, int32_t* labels, float* dist2, float* inertia,
                          int32_t* rep, int32_t* counts);

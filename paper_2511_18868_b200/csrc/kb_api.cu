@@ -86,6 +86,7 @@ kb_status kb_create(kb_ctx** out, int device, void* cuda_stream) {
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->coop_launch, cudaDevAttrCooperativeLaunch, device);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
     if (e != cudaSuccess) {
@@ -150,6 +151,7 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     need = max_sz(need, kb_ws_need_assign(B, N, D, K));
     need = max_sz(need, kb_ws_need_update(B, N, D, K));
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
+    need = max_sz(need, kb_ws_need_fit_coop(B, N, D, K));
     *out = need;
     return KB_OK;
 }
@@ -314,6 +316,12 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
         KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_fit: D and K must be >= 1");
         TimeScope ts__(ctx, KB_T_FIT);
         return kb_launch_fit_fused(ctx, B, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
+    }
+    if (ctx->assign_path == 0 && !kb_assign_tc_eligible(ctx, B, N, D, K) && kb_fit_coop_eligible(ctx, B, N, D, K) && z &&
+        centroids && labels && (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
+        // one mid-sized instance: the whole loop in one cooperative launch, the rows resident on chip
+        TimeScope ts__(ctx, KB_T_FIT);
+        return kb_launch_fit_coop(ctx, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
     }
     for (int it = 0; it < iters; ++it) {
         kb_status s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);

@@ -53,9 +53,9 @@ constexpr int PANEL = BN * KBF * 4;      // 16 KB: one hi or lo panel
 constexpr int STAGE = 2 * PANEL;         // hi + lo
 constexpr int EXT = 4096;                // fp16 split: the constant-term operand of one centroid tile (128 x 16 halfs)
 constexpr int SLOT_F16 = STAGE + EXT;    // a stage slot of the fp16 kernel (a multiple of 1024 bytes)
-constexpr int XCOLS = 8;
+constexpr int XCOLS = 8;                 // TMEM columns of a row's constant-term operand (16 halfs)
 constexpr int PREP_MAXG = 64;             // blocks per instance of the fp16 preparation kernel (at most)
-constexpr int INST_STRIDE = 1 + PREP_MAXG; // floats per instance: s_c, then every preparation block's largest ||c||^2                 // TMEM columns of a row's constant-term operand (16 halfs)
+constexpr int INST_STRIDE = 1 + PREP_MAXG; // floats per instance: s_c, then every preparation block's largest ||c||^2
 constexpr int NSTAGE = 4;
 constexpr int TC_THREADS = 448;
 constexpr int TMEM_COLS = 512;
@@ -1256,11 +1256,13 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
         KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F>), smem);                                   \
         kb_launch(assign_tc_kernel<T2, F>, grid, TC_THREADS, smem, ctx->stream, p);                   \
     } while (0)
+    const int tslot = kb_time_begin(ctx, KB_T_ASSIGN_KERNEL);
     if (track2 && f16) KB_TC_LAUNCH(true, true);
     else if (track2) KB_TC_LAUNCH(true, false);
     else if (f16) KB_TC_LAUNCH(false, true);
     else KB_TC_LAUNCH(false, false);
 #undef KB_TC_LAUNCH
+    kb_time_end(ctx, tslot);
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
     kb_launch(assign_fixup_pairs_kernel, 8 * ctx->sm_count, FX_T, 0, ctx->stream, N, D, K, z, c, flag_count, pair_rows, labels);

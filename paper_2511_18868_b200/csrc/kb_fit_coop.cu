@@ -1,0 +1,369 @@
+// kb_cluster_fit for one mid-sized instance: the whole Lloyd loop in ONE cooperative launch.
+//
+// Between the instances that fit a single CTA (kb_fit_fused.cu) and those large enough for the
+// tensor-core kernel lies the launch-latency regime: with N of a few ten thousand rows an
+// assign or an update moves about a megabyte, so an iteration of several dependent launches is
+// all launch gaps.  Here every CTA keeps its share of the rows on chip (registers and shared
+// memory) for all iterations and the CTAs meet once per iteration at a grid-wide barrier:
+//   * assign: a thread owns two rows in registers and scans a part of the centroids in shared memory
+//     (the threads that share a row each take a contiguous part, the best over the parts is taken
+//     in ascending order);
+//     the distance is the direct form sum (z - c)^2, ascending centroid id, strict < (lowest id
+//     on ties) -- the same arithmetic as the row-wise assign kernel;
+//   * update: CTA-local counting sort by label, (cluster, column) sums of the CTA's rows without
+//     atomics, then one reduction per non-empty (cluster, column) into a global table;
+//   * grid barrier (a monotone arrival counter; the launch is cooperative, so all CTAs are
+//     resident; the wait is bounded and raises the device status word when it expires);
+//   * every CTA reads the table back and forms the new centroids itself.
+// The global table is triple-buffered: iteration i accumulates into table i % 3, table
+// (i + 1) % 3 is cleared by CTA 0 before barrier i, and nobody reads table (i - 2) % 3 any more.
+// Z is read from HBM exactly once per fit.
+#include "kb_internal.cuh"
+
+namespace {
+
+constexpr int CF_MAXROWS = 512;    // rows per CTA at most
+constexpr int CF_R = 2;            // rows per thread
+// threads per CTA: the register file holds CF_R rows of D floats per thread for this many
+__host__ __device__ constexpr int cf_threads(int D) { return D <= 32 ? 512 : 256; }
+constexpr unsigned CF_SPIN_LIMIT = 1u << 22;
+constexpr int CF_STATUS_TIMEOUT = 0x200;
+
+struct CoopScratch {               // device scratch, cleared before the launch
+    unsigned arrive;               // grid barrier: arrivals so far
+    unsigned abort;                // a wait expired
+    double inertia;
+    unsigned long long pad;
+};
+
+// Grid-wide barrier number `epoch` (1, 2, ...) for G CTAs.  Returns false when the wait expired or
+// another CTA gave up.
+__device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, unsigned G) {
+    __syncthreads();
+    __shared__ int s_ok;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&sc->arrive, 1u);
+        int ok = 0;
+        for (unsigned i = 0; i < CF_SPIN_LIMIT; ++i) {
+            if (*reinterpret_cast<volatile unsigned*>(&sc->arrive) >= epoch * G) { ok = 1; break; }
+            if ((i & 255u) == 255u && *reinterpret_cast<volatile unsigned*>(&sc->abort)) break;
+            __nanosleep(32);
+        }
+        if (!ok) atomicExch(&sc->abort, 1u);
+        __threadfence();
+        s_ok = ok;
+    }
+    __syncthreads();
+    return s_ok != 0;
+}
+
+// SLOTS threads share the rows of the CTA (a thread owns rows slot and slot + SLOTS); the P = threads / SLOTS
+// threads of a slot each scan a contiguous P-th of the centroids, so a CTA with few rows still fills its SM.
+template <int D, int SLOTS>
+__global__ void __launch_bounds__(cf_threads(D))
+fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
+                int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
+                int32_t* __restrict__ rep, int32_t* __restrict__ counts, CoopScratch* __restrict__ sc,
+                float* __restrict__ table /* [3][K*D + K] sums then counts (as int) */,
+                unsigned long long* __restrict__ rep_key /* [K], cleared */, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
+    constexpr int CF_T = cf_threads(D), P = CF_T / SLOTS, CAP = SLOTS * CF_R;
+    static_assert(SLOTS % 32 == 0 && P >= 1, "a warp scans one part of the centroids");
+    extern __shared__ __align__(16) unsigned char cf_raw[];
+    constexpr int ZS = D + 1;                                       // padded row stride: conflict-free column walks
+    float* cs = reinterpret_cast<float*>(cf_raw);                   // [K][D] centroids
+    float* zs = cs + (size_t)K * D;                                 // [CAP][D+1] this CTA's rows
+    float* pbest = zs + (size_t)CAP * ZS;                           // [P][CAP] best distance of each part
+    int* parg = reinterpret_cast<int*>(pbest + P * CAP);            // [P][CAP] and its centroid
+    float* rbest = reinterpret_cast<float*>(parg + P * CAP);        // [CAP] best over the parts
+    int* rarg = reinterpret_cast<int*>(rbest + CAP);                // [CAP]
+    int* hist = rarg + CAP;                                         // [K] counts, then scatter cursors
+    int* offs = hist + K;                                           // [K+1]
+    unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [CAP] local row ids in label order
+    __shared__ int s_scan[CF_T / 32];
+    __shared__ double s_red[CF_T / 32];
+    const int G = gridDim.x, g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rows_per = (N + G - 1) / G;
+    const int r0 = g * rows_per, rows = max(0, min(N, r0 + rows_per) - r0);      // rows <= CAP (host)
+    const int KD = K * D, TS = KD + K;                              // floats per table
+    const int slot = tid % SLOTS, part = tid / SLOTS;
+    const int kper = (K + P - 1) / P;
+    const int jlo = min(K, part * kper), jhi = min(K, jlo + kper);
+
+    // stage this CTA's rows (coalesced float4 reads) and the initial centroids
+    const float* zb = z + (size_t)r0 * D;
+    for (int e = tid; e < rows * (D / 4); e += CF_T) {
+        const int r = e / (D / 4), q = e - r * (D / 4);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(zb) + e);
+        float* d = zs + (size_t)r * ZS + 4 * q;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+    for (int e = tid; e < KD / 4; e += CF_T)
+        reinterpret_cast<float4*>(cs)[e] = __ldg(reinterpret_cast<const float4*>(cent) + e);
+    __syncthreads();
+    float x[CF_R][D];
+#pragma unroll
+    for (int u = 0; u < CF_R; ++u) {
+        const bool active = slot + u * SLOTS < rows;
+#pragma unroll
+        for (int d = 0; d < D; ++d) x[u][d] = active ? zs[(size_t)(slot + u * SLOTS) * ZS + d] : 0.f;
+    }
+
+    bool ok = true;
+    for (int it = 0; it <= iters; ++it) {
+        // ---- assign: nearest centroid of my rows among my part, then the best over the parts -------------
+        {
+            float best[CF_R];
+            int arg[CF_R];
+#pragma unroll
+            for (int u = 0; u < CF_R; ++u) { best[u] = INFINITY; arg[u] = 0; }
+            for (int j = jlo; j < jhi; ++j) {
+                const float4* c4 = reinterpret_cast<const float4*>(cs + (size_t)j * D);
+                float acc[CF_R];
+#pragma unroll
+                for (int u = 0; u < CF_R; ++u) acc[u] = 0.f;
+#pragma unroll
+                for (int q = 0; q < D / 4; ++q) {
+                    const float4 c = c4[q];
+#pragma unroll
+                    for (int u = 0; u < CF_R; ++u) {
+                        const float e0 = x[u][4 * q] - c.x, e1 = x[u][4 * q + 1] - c.y, e2 = x[u][4 * q + 2] - c.z,
+                                    e3 = x[u][4 * q + 3] - c.w;
+                        acc[u] = fmaf(e0, e0, acc[u]); acc[u] = fmaf(e1, e1, acc[u]);
+                        acc[u] = fmaf(e2, e2, acc[u]); acc[u] = fmaf(e3, e3, acc[u]);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < CF_R; ++u) {
+                    if (acc[u] < best[u]) { best[u] = acc[u]; arg[u] = j; }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < CF_R; ++u) {
+                pbest[part * CAP + slot + u * SLOTS] = best[u];
+                parg[part * CAP + slot + u * SLOTS] = arg[u];
+            }
+        }
+        __syncthreads();
+        for (int r = tid; r < rows; r += CF_T) {
+            float bb = pbest[r];
+            int aa = parg[r];
+#pragma unroll
+            for (int p = 1; p < P; ++p) {                           // parts hold ascending ids: strict < keeps the lowest
+                const float v = pbest[p * CAP + r];
+                if (v < bb) { bb = v; aa = parg[p * CAP + r]; }
+            }
+            rbest[r] = bb;
+            rarg[r] = aa;
+        }
+        if (it == iters) break;                                     // the final assign has no update after it
+
+        float* tab = table + (size_t)(it % 3) * TS;
+        // CTA 0 clears the table of the next iteration (nobody reads or writes it during this one)
+        if (g == 0) {
+            float* nxt = table + (size_t)((it + 1) % 3) * TS;
+            for (int e = tid; e < TS; e += CF_T) nxt[e] = 0.f;
+        }
+        // ---- update: counting sort by label, then (cluster, column) sums of this CTA's rows ----
+        for (int j = tid; j < K; j += CF_T) hist[j] = 0;
+        __syncthreads();
+        for (int r = tid; r < rows; r += CF_T) atomicAdd(&hist[rarg[r]], 1);
+        __syncthreads();
+        {   // exclusive scan of hist (contiguous slices per thread)
+            const int per = (K + CF_T - 1) / CF_T;
+            const int j0 = min(K, tid * per), j1 = min(K, j0 + per);
+            int local = 0;
+            for (int j = j0; j < j1; ++j) local += hist[j];
+            int incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) s_scan[warp] = incl;
+            __syncthreads();
+            int base = 0;
+            for (int w = 0; w < warp; ++w) base += s_scan[w];
+            int run = base + incl - local;
+            for (int j = j0; j < j1; ++j) { offs[j] = run; run += hist[j]; }
+            if (tid == CF_T - 1) offs[K] = run;
+        }
+        __syncthreads();
+        for (int j = tid; j < K; j += CF_T) hist[j] = offs[j];      // scatter cursors
+        __syncthreads();
+        for (int r = tid; r < rows; r += CF_T) perm[atomicAdd(&hist[rarg[r]], 1)] = (unsigned short)r;
+        __syncthreads();
+        for (int e = tid; e < KD; e += CF_T) {
+            const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
+            const int p0 = offs[j], p1 = offs[j + 1];
+            if (p1 > p0) {
+                float s0 = 0.f, s1 = 0.f;
+                int p = p0;
+                for (; p + 1 < p1; p += 2) {
+                    s0 += zs[(size_t)perm[p] * ZS + d];
+                    s1 += zs[(size_t)perm[p + 1] * ZS + d];
+                }
+                if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
+                atomicAdd(tab + e, s0 + s1);
+                if (d == 0) atomicAdd(reinterpret_cast<int*>(tab + KD) + j, p1 - p0);
+            }
+        }
+        // ---- everybody's sums are in the table after the barrier ---------------------------------
+        ok = grid_barrier(sc, (unsigned)(it + 1), (unsigned)G);
+        if (!ok) break;
+        for (int e0 = 0; e0 < KD; e0 += 4 * CF_T) {                 // written by other CTAs: read through L2
+            int n[4];
+            float v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = min(e0 + u * CF_T + tid, KD - 1);
+                n[u] = __ldcg(reinterpret_cast<const int*>(tab + KD) + e / D);
+                v[u] = __ldcg(tab + e);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = e0 + u * CF_T + tid;
+                if (e < KD && n[u] > 0) cs[e] = v[u] / (float)n[u]; // an empty cluster keeps its centroid
+            }
+        }
+        if (g == 0 && it == iters - 1 && counts)
+            for (int j = tid; j < K; j += CF_T) counts[j] = __ldcg(reinterpret_cast<const int*>(tab + KD) + j);
+        __syncthreads();
+    }
+    if (!ok) {
+        if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
+        return;
+    }
+    __syncthreads();
+
+    // ---- outputs of the final assign --------------------------------------------------------
+    double mine = 0.0;
+    for (int lr = tid; lr < rows; lr += CF_T) {
+        const int r = r0 + lr, a = rarg[lr];
+        const float bb = rbest[lr];
+        labels[r] = a;
+        if (dist2) dist2[r] = bb;
+        mine += (double)bb;
+        // the representative is the member with the smallest (dist2, row): keys are stored inverted so
+        // that the cleared word means "no member" and atomicMax keeps the smallest key
+        if (rep) atomicMax(&rep_key[a], ~(((unsigned long long)__float_as_uint(bb) << 32) | (unsigned)r));
+    }
+    if (g == 0) {
+        for (int e = tid; e < KD / 4; e += CF_T)
+            reinterpret_cast<float4*>(cent)[e] = reinterpret_cast<const float4*>(cs)[e];
+        if (iters == 0 && counts)
+            for (int j = tid; j < K; j += CF_T) counts[j] = 0;
+    }
+    if (inertia) {
+        const double s = kb_warp_sum(mine);
+        if (lane == 0) s_red[warp] = s;
+        __syncthreads();
+        if (tid == 0) {
+            double t = 0.0;
+            for (int w = 0; w < CF_T / 32; ++w) t += s_red[w];
+            if (t != 0.0) atomicAdd(&sc->inertia, t);
+        }
+    }
+    if (inertia || rep) {
+        // one more barrier, then CTA 0 publishes what needed every CTA's contribution
+        if (!grid_barrier(sc, (unsigned)(iters + 1), (unsigned)G)) {
+            if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
+            return;
+        }
+        if (g == 0) {
+            if (inertia && tid == 0) inertia[0] = (float)*reinterpret_cast<volatile double*>(&sc->inertia);
+            if (rep)
+                for (int j = tid; j < K; j += CF_T) {
+                    const unsigned long long inv = __ldcg(rep_key + j);
+                    rep[j] = inv == 0ull ? -1 : (int32_t)((~inv) & 0xffffffffull);
+                }
+        }
+    }
+}
+
+__global__ void coop_zero_kernel(size_t n16, uint4* __restrict__ p) {
+    kb_grid_dependency_wait();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n16) p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+int cf_slots(int rows_per) { return rows_per <= 128 ? 64 : (rows_per <= 256 ? 128 : 256); }
+size_t cf_smem(int rows_per, int D, int K) {
+    const size_t cap = (size_t)cf_slots(rows_per) * CF_R, P = cf_threads(D) / cf_slots(rows_per);
+    // centroids | rows (padded) | per-part best and argument | per-row best and argument | hist, offs | perm
+    return (size_t)K * D * 4 + cap * (D + 1) * 4 + P * cap * 8 + cap * 8 + (size_t)(2 * K + 2) * 4 + cap * 2 + 32;
+}
+int cf_ctas(const kb_ctx* ctx, int N) {
+    long cap = ((long)N + 63) / 64;                     // at least 64 rows per CTA
+    long G = ctx->sm_count < cap ? ctx->sm_count : cap;
+    return (int)(G < 1 ? 1 : G);
+}
+size_t cf_scratch(int D, int K) {
+    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)3 * (K * D + K) * 4) + kb_align256((size_t)K * 8);
+}
+
+}  // namespace
+
+size_t kb_ws_need_fit_coop(int B, int N, int D, int K) {
+    return (B == 1 && (D == 16 || D == 32 || D == 64) && K >= 1 && K <= 1024) ? cf_scratch(D, K) : 0;
+}
+
+bool kb_fit_coop_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
+    if (B != 1 || N < 1024 || K < 1 || K > 1024) return false;
+    if (D != 16 && D != 32 && D != 64) return false;
+    if (!ctx->coop_launch) return false;
+    const int G = cf_ctas(ctx, N);
+    const int rows_per = (N + G - 1) / G;
+    if (rows_per > CF_MAXROWS) return false;
+    return cf_smem(rows_per, D, K) + 1024 <= (size_t)ctx->max_smem_optin && ctx->ws_bytes >= cf_scratch(D, K);
+}
+
+kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, float* cent, int32_t* labels,
+                             float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+    const int G = cf_ctas(ctx, N);
+    const int rows_per = (N + G - 1) / G;
+    const size_t smem = cf_smem(rows_per, D, K);
+    char* ws = ctx->ws;
+    CoopScratch* sc = reinterpret_cast<CoopScratch*>(ws);
+    float* table = reinterpret_cast<float*>(ws + kb_align256(sizeof(CoopScratch)));
+    unsigned long long* rep_key =
+        reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(table) + kb_align256((size_t)3 * (K * D + K) * 4));
+    const size_t zbytes = cf_scratch(D, K);
+    kb_launch(coop_zero_kernel, (unsigned)((zbytes / 16 + 255) / 256), 256, 0, ctx->stream, zbytes / 16,
+              reinterpret_cast<uint4*>(ws));
+    KB_LAUNCH_CHECK(ctx, "coop_zero_kernel");
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(G);
+    cfg.blockDim = dim3(cf_threads(D));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = ctx->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;     // all CTAs resident: they wait on one another
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+#define KB_CF_LAUNCH(DD, SS)                                                                                      \
+    do {                                                                                                          \
+        KB_SMEM_OPTIN(ctx, (fit_coop_kernel<DD, SS>), smem);                                                      \
+        e = cudaLaunchKernelEx(&cfg, fit_coop_kernel<DD, SS>, N, K, iters, z, cent, labels, dist2, inertia, rep,  \
+                               counts, sc, table, rep_key, ctx->dev_status);                                      \
+    } while (0)
+#define KB_CF_LAUNCH_D(DD)                            \
+    do {                                              \
+        if (slots == 64) KB_CF_LAUNCH(DD, 64);        \
+        else if (slots == 128) KB_CF_LAUNCH(DD, 128); \
+        else KB_CF_LAUNCH(DD, 256);                   \
+    } while (0)
+    const int slots = cf_slots(rows_per);
+    if (D == 16) KB_CF_LAUNCH_D(16);
+    else if (D == 32) KB_CF_LAUNCH_D(32);
+    else KB_CF_LAUNCH_D(64);
+#undef KB_CF_LAUNCH_D
+#undef KB_CF_LAUNCH
+    if (e != cudaSuccess) return kb_fail(ctx, KB_ERR_CUDA, "launch of fit_coop_kernel: %s", cudaGetErrorString(e));
+    KB_LAUNCH_CHECK(ctx, "fit_coop_kernel");
+    return KB_OK;
+}

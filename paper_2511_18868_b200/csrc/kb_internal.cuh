@@ -12,6 +12,7 @@ struct kb_ctx {
     cudaStream_t stream;
     int sm_count;
     int max_smem_optin;   // bytes of dynamic shared memory a block may opt into
+    int coop_launch;      // the device supports cooperative launches
     char* ws;             // caller's workspace (device)
     size_t ws_bytes;
     int* dev_status;      // device status word (owned)
@@ -59,6 +60,18 @@ kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...);
         if (!(cond)) return kb_fail(ctx, KB_ERR_INVALID_ARG, "%s", msg);                       \
     } while (0)
 
+// optional event pair around a single kernel (while per-call timing is on); returns the slot or -1
+static inline int kb_time_begin(kb_ctx* ctx, int cls) {
+    if (!ctx->timing || ctx->ev_used >= KB_EV_PAIRS) return -1;
+    const int slot = ctx->ev_used++;
+    ctx->ev_class[slot] = (unsigned char)cls;
+    cudaEventRecord(ctx->ev[2 * slot], ctx->stream);
+    return slot;
+}
+static inline void kb_time_end(kb_ctx* ctx, int slot) {
+    if (slot >= 0) cudaEventRecord(ctx->ev[2 * slot + 1], ctx->stream);
+}
+
 // ---- workspace ------------------------------------------------------------------
 // Every call carves its scratch from the start of the workspace and clears the
 // control words it relies on, so nothing in the workspace has to survive from
@@ -74,6 +87,10 @@ kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const
                                   const int32_t* labels, float* dist2, double* ws_inertia,
                                   unsigned long long* ws_rep);
 bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
+bool kb_fit_coop_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
+size_t kb_ws_need_fit_coop(int B, int N, int D, int K);
+kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, float* cent, int32_t* labels,
+                             float* dist2, float* inertia, int32_t* rep, int32_t* counts);
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* cent,
                               int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts);
 size_t kb_ws_need_update(int B, int N, int D, int K);

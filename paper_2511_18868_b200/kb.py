@@ -29,7 +29,7 @@ EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb
            "kb_bandit_step_host", "kb_cluster_update_noalloc"]
 
 
-TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fit"]
+TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fit", "assign_kernel"]
 
 
 class KbError(RuntimeError):

@@ -346,6 +346,48 @@ def test_step_free_running(kbx, name, host_buffers):
     print(f"[{name}] label agreement with the free-running oracle: {agree:.6f}")
 
 
+@pytest.mark.parametrize("N,D,K,iters", [(16384, 32, 64, 20), (5000, 16, 8, 7), (1025, 64, 100, 3), (40000, 32, 17, 4),
+                                         (2048, 32, 64, 0)])
+def test_cluster_fit_cooperative(kbx, N, D, K, iters):
+    """One mid-sized instance: kb_cluster_fit runs the whole Lloyd loop in one cooperative launch.  Its result
+    must be a Lloyd fixed-point sequence like the call-by-call path's: same objective, labels optimal for the
+    returned centroids (checked in double), counts, representative members and inertia consistent with them."""
+    cfg = wl.scaled(wl.CONFIGS["medium"], N=N, D=D, K=K, components=max(4, K // 2), S=2, iters=iters)
+    inp = wl.make_inputs(cfg, seed=N + K)
+    z, _, _ = oracle.normalize(inp["x"])
+    c0 = oracle.init_centroids(z, inp["init_rows"])
+    ws(kbx, 1, N, D, K, 2)
+    out = {}
+    for path in (0, 1):                      # 0: automatic (cooperative launch), 1: assign/update calls, fp32 kernels
+        kbx.set_assign_options(path=path)
+        try:
+            c = dev(c0.copy())
+            labels, d2 = empty((1, N), torch.int32), empty((1, N))
+            inertia, rep, counts = empty((1,)), empty((1, K), torch.int32), empty((1, K), torch.int32)
+            kbx.cluster_fit(dev(z), c, labels, iters, dist2=d2, inertia=inertia, rep=rep, counts=counts)
+        finally:
+            kbx.set_assign_options(path=0)
+        out[path] = dict(c=host(c), labels=host(labels), d2=host(d2), inertia=host(inertia), rep=host(rep),
+                         counts=host(counts))
+    assert kbx.device_status() == 0
+    got, ref = out[0], out[1]
+    parity.close(got["inertia"], ref["inertia"], atol=0, rtol=1e-3, what="inertia")
+    assert np.mean(got["labels"] == ref["labels"]) > 0.99
+    # self-consistency in double against the returned centroids
+    chk = oracle.cluster_assign(z, got["c"], want_margins=True, want_rep=True)
+    parity.labels_match(z, got["c"], got["labels"], chk)
+    same = got["labels"] == chk["labels"]
+    parity.close(got["d2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
+    parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia vs own labels")
+    if iters > 0:
+        assert got["counts"].sum() == N
+        assert np.abs(got["counts"] - ref["counts"]).sum() <= 0.02 * N      # sizes at the last update
+    else:
+        assert np.all(got["counts"] == 0)
+        np.testing.assert_array_equal(got["c"], c0)
+    parity.rep_match(got["rep"], chk, chk["dist2"], chk["labels"])
+
+
 def test_argument_errors(kbx):
     from paper_2511_18868_b200.kb import KbError
     z = empty((1, 8, 4))
