@@ -10,13 +10,16 @@
 //     in ascending order);
 //     the distance is the direct form sum (z - c)^2, ascending centroid id, strict < (lowest id
 //     on ties) -- the same arithmetic as the row-wise assign kernel;
-//   * update: CTA-local counting sort by label, (cluster, column) sums of the CTA's rows without
-//     atomics, then one reduction per non-empty (cluster, column) into a global table;
+//   * update: the CTA's rows are added into a (cluster, column) table in shared memory (a warp adds
+//     consecutive columns of one row: conflict-free), then one reduction per (cluster, column) of a
+//     non-empty cluster into a global table;
 //   * grid barrier (a monotone arrival counter; the launch is cooperative, so all CTAs are
 //     resident; the wait is bounded and raises the device status word when it expires);
 //   * every CTA reads the table back and forms the new centroids itself.
 // The global table is triple-buffered: iteration i accumulates into table i % 3, table
-// (i + 1) % 3 is cleared by CTA 0 before barrier i, and nobody reads table (i - 2) % 3 any more.
+// (i + 1) % 3 is cleared before barrier i, and nobody reads table (i - 2) % 3 any more.  Each table
+// is kept in CF_NC copies (CTA g adds into copy g % CF_NC and the readers add the copies up): all
+// CTAs reduce into the same few lines, and the reductions on one line are serviced one at a time.
 // Z is read from HBM exactly once per fit.
 #include "kb_internal.cuh"
 
@@ -26,14 +29,18 @@ constexpr int CF_MAXROWS = 512;    // rows per CTA at most
 constexpr int CF_R = 2;            // rows per thread
 // threads per CTA: the register file holds CF_R rows of D floats per thread for this many
 __host__ __device__ constexpr int cf_threads(int D) { return D <= 32 ? 512 : 256; }
+constexpr int CF_NC = 4;           // copies of the global table: CTA g adds into copy g % CF_NC
 constexpr unsigned CF_SPIN_LIMIT = 1u << 22;
 constexpr int CF_STATUS_TIMEOUT = 0x200;
 
 struct CoopScratch {               // device scratch, cleared before the launch
     unsigned arrive;               // grid barrier: arrivals so far
-    unsigned abort;                // a wait expired
+    unsigned pad0[31];
+    unsigned epoch;                // barriers completed, written by the last arrival; polled (a line of its own:
+    unsigned abort;                // the polls do not delay the arrivals); a wait expired
+    unsigned pad1[30];
     double inertia;
-    unsigned long long pad;
+    unsigned long long pad2[15];
 };
 
 // Grid-wide barrier number `epoch` (1, 2, ...) for G CTAs.  Returns false when the wait expired or
@@ -43,12 +50,17 @@ __device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, un
     __shared__ int s_ok;
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(&sc->arrive, 1u);
         int ok = 0;
-        for (unsigned i = 0; i < CF_SPIN_LIMIT; ++i) {
-            if (*reinterpret_cast<volatile unsigned*>(&sc->arrive) >= epoch * G) { ok = 1; break; }
-            if ((i & 255u) == 255u && *reinterpret_cast<volatile unsigned*>(&sc->abort)) break;
-            __nanosleep(32);
+        if (atomicAdd(&sc->arrive, 1u) == epoch * G - 1u) {         // the last arrival opens the barrier
+            __threadfence();
+            *reinterpret_cast<volatile unsigned*>(&sc->epoch) = epoch;
+            ok = 1;
+        } else {
+            for (unsigned i = 0; i < CF_SPIN_LIMIT; ++i) {
+                if (*reinterpret_cast<volatile unsigned*>(&sc->epoch) >= epoch) { ok = 1; break; }
+                if ((i & 255u) == 255u && *reinterpret_cast<volatile unsigned*>(&sc->abort)) break;
+                __nanosleep(64);
+            }
         }
         if (!ok) atomicExch(&sc->abort, 1u);
         __threadfence();
@@ -65,7 +77,7 @@ __global__ void __launch_bounds__(cf_threads(D))
 fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
                 int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, CoopScratch* __restrict__ sc,
-                float* __restrict__ table /* [3][K*D + K] sums then counts (as int) */,
+                float* __restrict__ table /* [3][CF_NC][K*D + K] sums then counts (as int) */,
                 unsigned long long* __restrict__ rep_key /* [K], cleared */, int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
     constexpr int CF_T = cf_threads(D), P = CF_T / SLOTS, CAP = SLOTS * CF_R;
@@ -78,10 +90,8 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
     int* parg = reinterpret_cast<int*>(pbest + P * CAP);            // [P][CAP] and its centroid
     float* rbest = reinterpret_cast<float*>(parg + P * CAP);        // [CAP] best over the parts
     int* rarg = reinterpret_cast<int*>(rbest + CAP);                // [CAP]
-    int* hist = rarg + CAP;                                         // [K] counts, then scatter cursors
-    int* offs = hist + K;                                           // [K+1]
-    unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [CAP] local row ids in label order
-    __shared__ int s_scan[CF_T / 32];
+    int* hist = rarg + CAP;                                         // [K] this CTA's rows per cluster, then the totals
+    float* ssum = reinterpret_cast<float*>(hist + K);               // [K][D] this CTA's column sums per cluster
     __shared__ double s_red[CF_T / 32];
     const int G = gridDim.x, g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows_per = (N + G - 1) / G;
@@ -145,6 +155,10 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
                 parg[part * CAP + slot + u * SLOTS] = arg[u];
             }
         }
+        if (it < iters) {
+            for (int e = tid; e < KD; e += CF_T) ssum[e] = 0.f;
+            for (int j = tid; j < K; j += CF_T) hist[j] = 0;
+        }
         __syncthreads();
         for (int r = tid; r < rows; r += CF_T) {
             float bb = pbest[r];
@@ -159,76 +173,73 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
         }
         if (it == iters) break;                                     // the final assign has no update after it
 
-        float* tab = table + (size_t)(it % 3) * TS;
-        // CTA 0 clears the table of the next iteration (nobody reads or writes it during this one)
-        if (g == 0) {
-            float* nxt = table + (size_t)((it + 1) % 3) * TS;
+        float* tab0 = table + (size_t)(it % 3) * CF_NC * TS;
+        float* tab = tab0 + (size_t)(g % CF_NC) * TS;
+        // the first CTAs clear the table of the next iteration (nobody reads or writes it during this one)
+        if (g < CF_NC) {
+            float* nxt = table + ((size_t)((it + 1) % 3) * CF_NC + g) * TS;
             for (int e = tid; e < TS; e += CF_T) nxt[e] = 0.f;
         }
-        // ---- update: counting sort by label, then (cluster, column) sums of this CTA's rows ----
-        for (int j = tid; j < K; j += CF_T) hist[j] = 0;
+        // ---- update: (cluster, column) sums of this CTA's rows in shared memory, then into the table ----
+        // (ssum and hist were cleared before the combine above)
         __syncthreads();
-        for (int r = tid; r < rows; r += CF_T) atomicAdd(&hist[rarg[r]], 1);
-        __syncthreads();
-        {   // exclusive scan of hist (contiguous slices per thread)
-            const int per = (K + CF_T - 1) / CF_T;
-            const int j0 = min(K, tid * per), j1 = min(K, j0 + per);
-            int local = 0;
-            for (int j = j0; j < j1; ++j) local += hist[j];
-            int incl = local;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            if (lane == 31) s_scan[warp] = incl;
-            __syncthreads();
-            int base = 0;
-            for (int w = 0; w < warp; ++w) base += s_scan[w];
-            int run = base + incl - local;
-            for (int j = j0; j < j1; ++j) { offs[j] = run; run += hist[j]; }
-            if (tid == CF_T - 1) offs[K] = run;
+        for (int e = tid; e < rows * D; e += CF_T) {
+            const int r = e / D, d = e - r * D;                     // a warp covers consecutive columns of one row
+            const int a = rarg[r];
+            atomicAdd(ssum + a * D + d, zs[(size_t)r * ZS + d]);
+            if (d == 0) atomicAdd(hist + a, 1);
         }
         __syncthreads();
-        for (int j = tid; j < K; j += CF_T) hist[j] = offs[j];      // scatter cursors
-        __syncthreads();
-        for (int r = tid; r < rows; r += CF_T) perm[atomicAdd(&hist[rarg[r]], 1)] = (unsigned short)r;
-        __syncthreads();
         for (int e = tid; e < KD; e += CF_T) {
-            const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
-            const int p0 = offs[j], p1 = offs[j + 1];
-            if (p1 > p0) {
-                float s0 = 0.f, s1 = 0.f;
-                int p = p0;
-                for (; p + 1 < p1; p += 2) {
-                    s0 += zs[(size_t)perm[p] * ZS + d];
-                    s1 += zs[(size_t)perm[p + 1] * ZS + d];
-                }
-                if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
-                atomicAdd(tab + e, s0 + s1);
-                if (d == 0) atomicAdd(reinterpret_cast<int*>(tab + KD) + j, p1 - p0);
+            const int j = e / D, n = hist[j];
+            if (n > 0) {
+                atomicAdd(tab + e, ssum[e]);
+                if (e - j * D == 0) atomicAdd(reinterpret_cast<int*>(tab + KD) + j, n);
             }
         }
         // ---- everybody's sums are in the table after the barrier ---------------------------------
         ok = grid_barrier(sc, (unsigned)(it + 1), (unsigned)G);
         if (!ok) break;
-        for (int e0 = 0; e0 < KD; e0 += 4 * CF_T) {                 // written by other CTAs: read through L2
-            int n[4];
-            float v[4];
+        // written by other CTAs: read through L2; the counts once per cluster (every CTA reads these lines)
+        {
+            int n[CF_NC];
+            const int j = min(tid, K - 1);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int e = min(e0 + u * CF_T + tid, KD - 1);
-                n[u] = __ldcg(reinterpret_cast<const int*>(tab + KD) + e / D);
-                v[u] = __ldcg(tab + e);
-            }
+            for (int c = 0; c < CF_NC; ++c) n[c] = __ldcg(reinterpret_cast<const int*>(tab0 + (size_t)c * TS + KD) + j);
+            for (int e0 = 0; e0 < KD; e0 += 4 * CF_T) {
+                float v[4][CF_NC];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int e = e0 + u * CF_T + tid;
-                if (e < KD && n[u] > 0) cs[e] = v[u] / (float)n[u]; // an empty cluster keeps its centroid
+                for (int u = 0; u < 4; ++u) {
+                    const int e = min(e0 + u * CF_T + tid, KD - 1);
+#pragma unroll
+                    for (int c = 0; c < CF_NC; ++c) v[u][c] = __ldcg(tab0 + (size_t)c * TS + e);
+                }
+                if (e0 == 0) {
+                    int tot = 0;
+#pragma unroll
+                    for (int c = 0; c < CF_NC; ++c) tot += n[c];
+                    if (tid < K) hist[tid] = tot;
+                    for (int jj = tid + CF_T; jj < K; jj += CF_T) {     // K beyond the block: the rest of the counts
+                        int t2 = 0;
+#pragma unroll
+                        for (int c = 0; c < CF_NC; ++c) t2 += __ldcg(reinterpret_cast<const int*>(tab0 + (size_t)c * TS + KD) + jj);
+                        hist[jj] = t2;
+                    }
+                    __syncthreads();
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e = e0 + u * CF_T + tid;
+                    float sum = v[u][0];
+#pragma unroll
+                    for (int c = 1; c < CF_NC; ++c) sum += v[u][c];
+                    const int cnt = e < KD ? hist[e / D] : 0;
+                    if (cnt > 0) cs[e] = sum / (float)cnt;          // an empty cluster keeps its centroid
+                }
             }
         }
         if (g == 0 && it == iters - 1 && counts)
-            for (int j = tid; j < K; j += CF_T) counts[j] = __ldcg(reinterpret_cast<const int*>(tab + KD) + j);
+            for (int j = tid; j < K; j += CF_T) counts[j] = hist[j];
         __syncthreads();
     }
     if (!ok) {
@@ -291,8 +302,8 @@ __global__ void coop_zero_kernel(size_t n16, uint4* __restrict__ p) {
 int cf_slots(int rows_per) { return rows_per <= 128 ? 64 : (rows_per <= 256 ? 128 : 256); }
 size_t cf_smem(int rows_per, int D, int K) {
     const size_t cap = (size_t)cf_slots(rows_per) * CF_R, P = cf_threads(D) / cf_slots(rows_per);
-    // centroids | rows (padded) | per-part best and argument | per-row best and argument | hist, offs | perm
-    return (size_t)K * D * 4 + cap * (D + 1) * 4 + P * cap * 8 + cap * 8 + (size_t)(2 * K + 2) * 4 + cap * 2 + 32;
+    // centroids | rows (padded) | per-part best and argument | per-row best and argument | hist | column sums
+    return (size_t)K * D * 4 + cap * (D + 1) * 4 + P * cap * 8 + cap * 8 + (size_t)K * 4 + (size_t)K * D * 4 + 32;
 }
 int cf_ctas(const kb_ctx* ctx, int N) {
     long cap = ((long)N + 63) / 64;                     // at least 64 rows per CTA
@@ -300,7 +311,7 @@ int cf_ctas(const kb_ctx* ctx, int N) {
     return (int)(G < 1 ? 1 : G);
 }
 size_t cf_scratch(int D, int K) {
-    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)3 * (K * D + K) * 4) + kb_align256((size_t)K * 8);
+    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)K * 8) + kb_align256((size_t)3 * CF_NC * (K * D + K) * 4) + 256;
 }
 
 }  // namespace
@@ -324,12 +335,13 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
     const int G = cf_ctas(ctx, N);
     const int rows_per = (N + G - 1) / G;
     const size_t smem = cf_smem(rows_per, D, K);
+    // workspace: barrier words | representative keys | tables.  Cleared here: everything up to the end of
+    // the first table (the kernel clears the table of iteration i + 1 during iteration i).
     char* ws = ctx->ws;
     CoopScratch* sc = reinterpret_cast<CoopScratch*>(ws);
-    float* table = reinterpret_cast<float*>(ws + kb_align256(sizeof(CoopScratch)));
-    unsigned long long* rep_key =
-        reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(table) + kb_align256((size_t)3 * (K * D + K) * 4));
-    const size_t zbytes = cf_scratch(D, K);
+    unsigned long long* rep_key = reinterpret_cast<unsigned long long*>(ws + kb_align256(sizeof(CoopScratch)));
+    float* table = reinterpret_cast<float*>(reinterpret_cast<char*>(rep_key) + kb_align256((size_t)K * 8));
+    const size_t zbytes = (size_t)(reinterpret_cast<char*>(table) - ws) + kb_align256((size_t)CF_NC * (K * D + K) * 4);
     kb_launch(coop_zero_kernel, (unsigned)((zbytes / 16 + 255) / 256), 256, 0, ctx->stream, zbytes / 16,
               reinterpret_cast<uint4*>(ws));
     KB_LAUNCH_CHECK(ctx, "coop_zero_kernel");
