@@ -203,9 +203,16 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
  *             chosen centroid for the tf32 split, the largest of the instance
  *             for the fp16 split) is re-evaluated exactly (direct form, fp32).
  *             <= 0 keeps the default 2^-16.
- * kb_get_assign_path reports what the last kb_cluster_assign ran (1, 2 or 3). */
+ * kb_get_assign_path reports what the last kb_cluster_assign ran (1, 2 or 3).
+ * kb_get_assign_presplit reports (1 or 0) whether that assignment, if it ran
+ * the fp16 tensor-core kernel, multiplied out of a pre-split image of Z:
+ * kb_cluster_fit (and kb_bandit_step through it) converts Z to its fp16 pieces
+ * once, keeps the image in the workspace for the duration of the fit and lets
+ * every assignment of the loop read it; a lone kb_cluster_assign splits the
+ * rows on the fly. */
 kb_status kb_set_assign_options(kb_ctx* ctx, int path, float tc_eps);
 kb_status kb_get_assign_path(kb_ctx* ctx, int* out);
+kb_status kb_get_assign_presplit(kb_ctx* ctx, int* out);
 
 /* Diagnostic for the tensor-core assign kernel: runs it on (z, centroids) and
  * returns, besides the labels, the expanded-form squared distance it ranked

@@ -144,14 +144,22 @@ kb_status kb_set_stream(kb_ctx* ctx, void* cuda_stream) {
     return KB_OK;
 }
 
+// Scratch of the calls a fit makes; the pre-split image of Z that a fit keeps across its iterations
+// lies behind it (the other calls never run inside a fit and may use that space).
+static size_t fit_scratch_bytes(int B, int N, int D, int K) {
+    size_t need = 256;
+    need = max_sz(need, kb_ws_need_assign(B, N, D, K));
+    need = max_sz(need, kb_ws_need_update(B, N, D, K));
+    need = max_sz(need, kb_ws_need_fit_coop(B, N, D, K));
+    return kb_align256(need) + 1024;
+}
+
 kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     if (!out || B < 0 || N < 0 || D < 0 || K < 0 || S < 0) return KB_ERR_INVALID_ARG;
     size_t need = 256;
     need = max_sz(need, kb_ws_need_normalize(B, N, D));
-    need = max_sz(need, kb_ws_need_assign(B, N, D, K));
-    need = max_sz(need, kb_ws_need_update(B, N, D, K));
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
-    need = max_sz(need, kb_ws_need_fit_coop(B, N, D, K));
+    need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_zsplit(B, N, D, K));
     *out = need;
     return KB_OK;
 }
@@ -244,6 +252,12 @@ kb_status kb_get_assign_path(kb_ctx* ctx, int* out) {
     return KB_OK;
 }
 
+kb_status kb_get_assign_presplit(kb_ctx* ctx, int* out) {
+    if (!ctx || !out) return KB_ERR_INVALID_ARG;
+    *out = ctx->last_assign_presplit;
+    return KB_OK;
+}
+
 kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const float* centroids,
                              int32_t* labels, float* approx_dist2, int32_t* flagged) {
     KB_COMMON(ctx, B, N);
@@ -323,13 +337,22 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
         TimeScope ts__(ctx, KB_T_FIT);
         return kb_launch_fit_coop(ctx, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
     }
-    for (int it = 0; it < iters; ++it) {
-        kb_status s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
-        if (s != KB_OK) return s;
-        s = kb_cluster_update(ctx, B, N, D, K, z, labels, centroids, counts);
-        if (s != KB_OK) return s;
+    // Tensor-core assignments of the same matrix, several times over: split Z into its fp16 pieces once and let
+    // every assignment multiply out of that image (kept behind the scratch of the calls below).
+    kb_status s = KB_OK;
+    const size_t zneed = kb_ws_need_zsplit(B, N, D, K), zoff = fit_scratch_bytes(B, N, D, K);
+    if (iters >= 2 && N > 0 && z && zneed > 0 && ctx->ws_bytes >= zoff + zneed && ctx->assign_path != 1 &&
+        (ctx->assign_path >= 2 || kb_assign_tc_eligible(ctx, B, N, D, K))) {
+        TimeScope ts__(ctx, KB_T_ASSIGN);
+        s = kb_zsplit_prepare(ctx, ctx->ws + zoff, B, N, D, K, z);
     }
-    return kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+    for (int it = 0; it < iters && s == KB_OK; ++it) {
+        s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
+        if (s == KB_OK) s = kb_cluster_update(ctx, B, N, D, K, z, labels, centroids, counts);
+    }
+    if (s == KB_OK) s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+    kb_zsplit_forget(ctx);
+    return s;
 }
 
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {

@@ -200,6 +200,7 @@ kb_status kb_launch_assign(kb_ctx* ctx, int B, int N, int D, int K, const float*
         } else {
             s = launch_rowwise(ctx, B, N, D, K, z, c, labels, dist2, ws_inertia, ws_rep);
             ctx->last_assign_path = 1;
+            ctx->last_assign_presplit = 0;
         }
         if (s != KB_OK) return s;
     }

@@ -58,6 +58,8 @@ constexpr int PREP_MAXG = 64;             // blocks per instance of the fp16 pre
 constexpr int INST_STRIDE = 1 + PREP_MAXG; // floats per instance: s_c, then every preparation block's largest ||c||^2
 constexpr int NSTAGE = 4;
 constexpr int TC_THREADS = 448;
+constexpr int TC_THREADS_APRE = 480;     // pre-split A: one more warp, which loads the A panels
+constexpr int AINFO = BM * 8;             // bytes of a tile's row table (||z||^2, s_z per row)
 constexpr int TMEM_COLS = 512;
 constexpr int COL_ACC = 0;         // two accumulators: columns [0,128) and [128,256)
 constexpr int COL_A = 256;         // A buffers from here: hi part | lo part (| constant terms), two buffers when they fit
@@ -170,6 +172,15 @@ __device__ __forceinline__ void tc_mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, 
             ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
             : "memory");
 }
+// D[tmem] += A[smem desc] * B[smem desc], kind::f16 (both operands K-major panels in shared memory)
+__device__ __forceinline__ void tc_mma_ss_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
@@ -245,6 +256,9 @@ struct TcParams {
     int resident;                  // 1: the whole B image of the (single) instance stays in the stage ring
     float eps;                     // near-tie bound, relative to ||z||^2 + ||c||^2
     const float* z;
+    const unsigned char* aimg;     // pre-split A: [tile][nkb][hi panel | lo panel], the layout of a B stage
+    const float* ainfo;            // pre-split A: [tile][BM][2]  ||z||^2 and s_z of every row
+    int nstage_alloc;              // stage slots that exist in shared memory (the whole ring unless B is resident)
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
     const float* cnorm;            // [B][Kpad]
     const unsigned char* bext;     // fp16 split: [B][NT][EXT] constant-term operand of every centroid tile
@@ -408,6 +422,47 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
     }
 }
 
+// The A side of the fp16 split, made ONCE for a matrix Z that many assignments will read (the Lloyd
+// loop of a fit): every 128-row tile becomes the same kind of image as a B stage,
+//   aimg  [tile][nkb][hi panel | lo panel]   128-byte-swizzled K-major panels of s_z z (s_z brings the
+//                                            row's largest magnitude into [0.5, 1))
+//   ainfo [tile][128][2]                     ||z||^2 and s_z of every row
+// so that an assignment fetches a tile with one bulk copy per k-block and multiplies straight out of
+// shared memory; only the row's constant-term operand, which depends on the centroids' scale, is
+// still formed per assignment.  One warp per row, lane q owns the 16-byte chunk q of the fp32 row.
+// Rows past the end of an instance are zeros.
+__global__ void __launch_bounds__(256)
+tc_prep_z_f16_kernel(int N, int D, int nkb, int tiles_per_inst, const float* __restrict__ z,
+                     unsigned char* __restrict__ aimg, float* __restrict__ ainfo) {
+    kb_grid_dependency_wait();
+    const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long slot = (long)blockIdx.x * 8 + warp;                 // row slot inside the instance's tiles
+    if (slot >= (long)tiles_per_inst * BM) return;
+    const int t = (int)(slot / BM), r = (int)(slot - (long)t * BM);
+    const size_t tile = (size_t)b * tiles_per_inst + t;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (slot < N && lane < D / 4) v = __ldg(reinterpret_cast<const float4*>(z + ((size_t)b * N + slot) * D) + lane);
+    float xn = fmaf(v.w, v.w, fmaf(v.z, v.z, fmaf(v.y, v.y, v.x * v.x)));
+    float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xn += __shfl_xor_sync(0xffffffffu, xn, o);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    }
+    const float sz = pow2_scale(m);
+    if (lane < nkb * 16) {
+        const int kb = lane >> 4, within = (lane & 15) * 8;                // byte offset inside the 128-byte row
+        const size_t off = (tile * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
+                           (((within >> 4) ^ (r & 7)) << 4) + (within & 15);
+        uint32_t h0, l0, h1, l1;
+        split_f16x2(v.x * sz, v.y * sz, h0, l0);
+        split_f16x2(v.z * sz, v.w * sz, h1, l1);
+        *reinterpret_cast<uint2*>(aimg + off) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2*>(aimg + off + PANEL) = make_uint2(l0, l1);
+    }
+    if (lane == 0) *reinterpret_cast<float2*>(ainfo + (tile * BM + r) * 2) = make_float2(xn, sz);
+}
+
 // ---- the contraction -------------------------------------------------------------------
 // Running smallest squared distances of one row, kept as integer KEYS: the fp32 bits of
 // d2 = ||z||^2 + ||c||^2 - 2 z.c with the low KEY_BITS replaced by the column's index inside
@@ -471,11 +526,51 @@ struct RowBest {
     __device__ __forceinline__ int column(int key, int tile) const { return tile * BN + (key & ~KEY_MASK); }
 };
 
-template <bool TRACK2, bool F16>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+// fp16 split: what a row's three smallest keys decide.  key = n * KQ_MUL + column (column inside the
+// thread's 64; the tile id carries the half); n * kstep is the squared distance.  A slightly negative
+// distance gives a negative key: it ranks first and reads as zero.  Writes the label (and the
+// diagnostic distance) and queues the row for the exact re-evaluation when its runner-up lies inside
+// the error bound.
+__device__ __forceinline__ void emit_row_f16(const TcParams& p, const RowBest<true>& rb, size_t flat, float xn,
+                                             float cmaxn, float rscale) {
+    const float range_d2 = fmaxf(2.f * (xn + cmaxn), 1e-30f);
+    const float kstep = range_d2 * (1.f / KQ_TOP);
+    auto quant = [](int key) {             // floor division: a negative key keeps its column
+        return key >= 0 ? key / (int)KQ_MUL : -((-key + (int)KQ_MUL - 1) / (int)KQ_MUL);
+    };
+    const int n0 = quant(rb.r0), n1 = quant(rb.r1), n2 = quant(rb.r2);
+    const int l0 = rb.r0 - n0 * (int)KQ_MUL, l1 = rb.r1 - n1 * (int)KQ_MUL;
+    const int a0 = (rb.t0 >> 1) * BN + (rb.t0 & 1) * (BN / 2) + l0;
+    const int a1 = (rb.t1 >> 1) * BN + (rb.t1 & 1) * (BN / 2) + l1;
+    const float b0 = (float)max(n0, 0) * kstep, b1 = (float)max(n1, 0) * kstep, b2 = (float)max(n2, 0) * kstep;
+    // near-tie bound: the split product's error, relative to ||z||^2 plus the largest centroid norm of
+    // the instance (its centroids share one scale), plus two quantisation steps
+    const float delta = p.eps * (xn + cmaxn) + 2.f * kstep;
+    // the third smallest is only known when the two smallest come from different sub-chunks (the 64
+    // columns of an accumulator tile that one thread ranks: each hands over its two smallest keys)
+    const bool third_known = rb.t0 != rb.t1;
+    p.labels[flat] = a0;
+    if (p.approx) p.approx[flat] = b0;
+    if (rscale < 0.f) {                                // row outside the fp16 range: exact scan over all K
+        const int slot = atomicAdd(p.flag_count + 1, 1);
+        p.full_rows[slot] = (int32_t)flat;
+    } else if (fabsf(b1 - b0) <= delta) {
+        if (third_known && fabsf(b2 - b0) > delta) {   // exactly two candidates: compare them exactly
+            const int slot = atomicAdd(p.flag_count, 1);
+            p.pair_rows[slot] = make_int2((int)flat, a1);
+        } else {                                       // three or more (or unknown): exact scan over all K
+            const int slot = atomicAdd(p.flag_count + 1, 1);
+            p.full_rows[slot] = (int32_t)flat;
+        }
+    }
+}
+
+template <bool TRACK2, bool F16, bool APRE>
+__global__ void __launch_bounds__(APRE ? TC_THREADS_APRE : TC_THREADS, 1)
 assign_tc_kernel(const TcParams p) {
-    // fp16 split: the hot loop keeps the two smallest keys of each sub-chunk (the 32 columns one
-    // tracker sees in an accumulator tile); the row's running best keeps three keys.  The third
+    static_assert(!APRE || F16, "the pre-split A image exists for the fp16 split only");
+    // fp16 split: the hot loop keeps the two smallest keys of each sub-chunk (the 64 columns one
+    // thread ranks in an accumulator tile); the row's running best keeps three keys.  The third
     // smallest distance of the row is then known unless the two smallest come from the same
     // sub-chunk, in which case a near-tie goes to the full re-evaluation.
     constexpr bool HOT3 = F16 ? false : TRACK2;           // hot-loop trackers keep a third key
@@ -489,17 +584,22 @@ assign_tc_kernel(const TcParams p) {
     const int nab = 2 * AST <= 256 ? 2 : 1;               // A buffers that fit beside the accumulators in TMEM
     constexpr int SLOT = F16 ? SLOT_F16 : STAGE;          // bytes of one stage slot
     const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
-    unsigned char* st_base = smem;                                        // NSTAGE x SLOT
-    float* xs = reinterpret_cast<float*>(smem + NSTAGE * SLOT);           // nxb x [BM][D+4]
-    float* cn = xs + (size_t)p.nxb * BM * xs_stride;                      // tf32: [B][Kpad] norms; fp16: [B][2] (s_c, max norm)
+    unsigned char* st_base = smem;                                        // nstage_alloc x SLOT
+    float* xs = reinterpret_cast<float*>(smem + (size_t)p.nstage_alloc * SLOT);   // nxb x [BM][D+4]
+    // pre-split A: nxb x [nkb][hi panel | lo panel], then nxb x [BM][2] row tables, instead of xs
+    unsigned char* as_base = smem + (size_t)p.nstage_alloc * SLOT;
+    const int ABUF = nkb * STAGE;                                         // bytes of one tile's A panels
+    float* as_info = reinterpret_cast<float*>(as_base + (size_t)p.nxb * ABUF);
+    float* cn = APRE ? as_info + (size_t)p.nxb * BM * 2                   // tf32: [B][Kpad] norms; fp16: [B][2] (s_c, max norm)
+                     : xs + (size_t)p.nxb * BM * xs_stride;
     float* xnorm = cn + (F16 ? (size_t)2 * p.B : (size_t)p.B * p.Kpad);   // [2][BM]
-    float* xscale = xnorm + 2 * BM;                                       // [2][BM]  fp16: 1 / g_i (negative: row out of range)
-    float* merge_buf = xscale + 2 * BM;                                   // [2][BM][5]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(merge_buf + 2 * BM * 5 + 2);   // (+2 floats: 8-byte alignment)
+    float* xscale = xnorm + 2 * BM;                                       // [2][BM]  fp16: the row's key factor (negative: row out of range)
+    float* merge_buf = xscale + 2 * BM;                                   // [2][2][BM][5]  (tile parity, half, row)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(merge_buf + 4 * BM * 5 + 2);   // (+2 floats: 8-byte alignment)
     // barrier indices
     enum { B_FULL = 0, B_EMPTY = NSTAGE, A_FULL = 2 * NSTAGE, A_EMPTY = A_FULL + 8, ACC_FULL = A_EMPTY + 8,
            ACC_EMPTY = ACC_FULL + 2, XN_FULL = ACC_EMPTY + 2, XN_EMPTY = XN_FULL + 2, X_FULL = XN_EMPTY + 2,
-           NBAR = X_FULL + 2 };
+           AS_EMPTY = X_FULL + 3, MG_FULL = AS_EMPTY + 3, MG_FREE = MG_FULL + 2, NBAR = MG_FREE + 2 };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -513,8 +613,11 @@ assign_tc_kernel(const TcParams p) {
         for (int k = 0; k < 2; ++k) {
             mbar_init(BAR(ACC_FULL + k), 1); mbar_init(BAR(ACC_EMPTY + k), 8);
             mbar_init(BAR(XN_FULL + k), 4); mbar_init(BAR(XN_EMPTY + k), 8);
-            mbar_init(BAR(X_FULL + k), 128);
         }
+        // staged rows: one arrival per producer thread; pre-split A: the loader's expect-tx arrival
+        for (int k = 0; k < 3; ++k) { mbar_init(BAR(X_FULL + k), APRE ? 1 : 128); mbar_init(BAR(AS_EMPTY + k), 1); }
+        // pre-split A: the epilogue hands every row's candidates to the row's thread among warps 0-3
+        for (int k = 0; k < 2; ++k) { mbar_init(BAR(MG_FULL + k), 8); mbar_init(BAR(MG_FREE + k), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -527,7 +630,7 @@ assign_tc_kernel(const TcParams p) {
     // the preceding kernel; from here on its results are read
     kb_grid_dependency_wait();
     if (F16) {
-        for (int j = tid; j < p.B; j += TC_THREADS) {                          // per instance: s_c, largest ||c||^2
+        for (int j = tid; j < p.B; j += (int)blockDim.x) {                     // per instance: s_c, largest ||c||^2
             const float* ib = p.inst + (size_t)j * INST_STRIDE;
             float nm = 0.f;
             for (int g = 0; g < p.gprep; ++g) nm = fmaxf(nm, ib[1 + g]);
@@ -535,7 +638,7 @@ assign_tc_kernel(const TcParams p) {
             cn[2 * j + 1] = nm;
         }
     } else {
-        for (int j = tid; j < p.B * p.Kpad; j += TC_THREADS) cn[j] = p.cnorm[j];   // all instances' centroid norms
+        for (int j = tid; j < p.B * p.Kpad; j += (int)blockDim.x) cn[j] = p.cnorm[j];   // all instances' centroid norms
     }
     tc_fence_before();
     __syncthreads();
@@ -545,7 +648,79 @@ assign_tc_kernel(const TcParams p) {
     const int first = blockIdx.x, stride = gridDim.x;
     bool ok = true;
 
-    if (warp < 4) {
+    if (APRE && warp < 4) {
+        // ============================ A: constant terms only ==========================
+        // The tile's panels arrive pre-split by bulk copy; what is left per row is its constant-term
+        // operand (it depends on the centroids' scale s_c) and the two numbers the epilogue wants.
+        const int row_in_tile = tid;                       // = TMEM lane
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // What the epilogue found for this thread's row of tile number `jt` (of this CTA): merge the two
+        // halves' candidates, write the label, queue a near-tie.
+        auto finish_row = [&](int jt, int tile, float xn, float rscale) -> bool {
+            if (!mbar_wait(BAR(MG_FULL + (jt & 1)), (uint32_t)((jt >> 1) & 1), abort_flag)) return false;
+            const float* m0 = merge_buf + ((size_t)((jt & 1) * 2) * BM + row_in_tile) * 5;
+            const float* m1 = m0 + BM * 5;
+            RowBest<true> rb;
+            rb.r0 = __float_as_int(m0[0]); rb.r1 = __float_as_int(m0[1]); rb.r2 = __float_as_int(m0[2]);
+            rb.t0 = __float_as_int(m0[3]); rb.t1 = __float_as_int(m0[4]);
+            const int u0 = __float_as_int(m1[0]), u1 = __float_as_int(m1[1]), u2 = __float_as_int(m1[2]);
+            const int v0 = __float_as_int(m1[3]), v1 = __float_as_int(m1[4]);
+            mbar_arrive_warp(BAR(MG_FREE + (jt & 1)));
+            rb.insert(u0, v0);
+            rb.insert(u1, v1);
+            rb.r2 = min(rb.r2, u2);
+            const int b = tile / p.tiles_per_inst, row = (tile - b * p.tiles_per_inst) * BM + row_in_tile;
+            if (row < p.N) emit_row_f16(p, rb, (size_t)b * p.N + row, xn, cn[2 * b + 1], rscale);
+            return true;
+        };
+        // rows are finished two tiles behind: the constant terms of tile i + 1 must be in place when the
+        // epilogue hands back the first accumulator of tile i, long before it is through with tile i - 1
+        int it = 0, tile1 = -1, tile2 = -1;                // the previous tile and the one before it
+        float xn1 = 0.f, rs1 = 1.f, xn2 = 0.f, rs2 = 1.f;
+        for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+            const int buf = it % p.nxb, ab = it & 1, use = it >> 1;
+            ok = mbar_wait(BAR(X_FULL + buf), (uint32_t)((it / p.nxb) & 1), abort_flag);
+            if (!ok) break;
+            const float2 info = *reinterpret_cast<const float2*>(as_info + ((size_t)buf * BM + row_in_tile) * 2);
+            const float xn = info.x, sz = info.y;
+            const float s_c = cn[2 * (tile / p.tiles_per_inst)];
+            float rho = sz / s_c;                                  // both powers of two: exact
+            const float g = sz * s_c;
+            float pterm = g * xn;                                  // s_z s_c ||z||^2
+            // a row far outside the centroids' range (s_z / s_c outside fp16's normal range, or a norm
+            // term that would overflow fp16) is handed to the exact re-evaluation
+            const bool out_of_range = !(rho >= 6.103515625e-05f && rho <= 16384.f) || !(pterm < 60000.f);
+            const float rscale = out_of_range ? -1.f : 1.f / g;
+            if (out_of_range) { rho = 0.f; pterm = 0.f; }
+            __half p0, p1, p2;
+            split3_f16(pterm, p0, p1, p2);
+            const __half hr = __float2half_rn(rho);
+            const uint32_t e0 = pack_h2(p0, p1), e1 = pack_h2(p2, hr), e2 = pack_h2(hr, hr), ez = 0u;
+            ok = mbar_wait(BAR(A_EMPTY + ab * 4), (uint32_t)((use & 1) ^ 1), abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                         ::"r"(lane_addr + COL_A + ab * XCOLS), "r"(e0), "r"(e1), "r"(e2), "r"(ez), "r"(ez),
+                           "r"(ez), "r"(ez), "r"(ez)
+                         : "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive_warp(BAR(A_FULL + ab * 4));
+            ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
+            if (!ok) break;
+            xnorm[(it & 1) * BM + row_in_tile] = xn;
+            // the factor that maps an accumulator value onto the key range (the row's largest possible
+            // value, 2 g (||z||^2 + max ||c||^2), lands on the top)
+            xscale[(it & 1) * BM + row_in_tile] =
+                KQ_TOP * fabsf(rscale) / fmaxf(2.f * (xn + cn[2 * (tile / p.tiles_per_inst) + 1]), 1e-30f);
+            mbar_arrive_warp(BAR(XN_FULL + (it & 1)));
+            if (tile2 >= 0) ok = finish_row(it - 2, tile2, xn2, rs2);
+            tile2 = tile1; xn2 = xn1; rs2 = rs1;
+            tile1 = tile; xn1 = xn; rs1 = rscale;
+        }
+        if (ok && tile2 >= 0) ok = finish_row(it - 2, tile2, xn2, rs2);
+        if (ok && tile1 >= 0) ok = finish_row(it - 1, tile1, xn1, rs1);
+    } else if (warp < 4) {
         // ============================ A producers ====================================
         const int row_in_tile = tid;                       // = TMEM lane
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
@@ -659,6 +834,9 @@ assign_tc_kernel(const TcParams p) {
             ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
             if (!ok) break;
             xnorm[(it & 1) * BM + row_in_tile] = xn;
+            // fp16 split: the factor that maps an accumulator value onto the key range (the row's largest
+            // possible value, 2 g (||z||^2 + max ||c||^2), lands on the top), negative for a row out of range
+            if (F16) rscale = copysignf(KQ_TOP * fabsf(rscale) / fmaxf(2.f * (xn + cn[2 * (tile / p.tiles_per_inst) + 1]), 1e-30f), rscale);
             xscale[(it & 1) * BM + row_in_tile] = rscale;
             mbar_arrive_warp(BAR(XN_FULL + (it & 1)));
         }
@@ -695,9 +873,7 @@ assign_tc_kernel(const TcParams p) {
             // fp16 split: quantisation step of the keys in units of d2, and the factor that maps an
             // accumulator value onto the key range
             const float cmaxn = F16 ? cn[2 * b + 1] : 0.f;
-            const float range_d2 = fmaxf(2.f * (xn + cmaxn), 1e-30f);
-            const float kstep = range_d2 * (1.f / KQ_TOP);
-            const float kmul = KQ_TOP * fabsf(rscale) / range_d2;
+            const float kmul = fabsf(rscale);                      // fp16 split: the producer left the key factor here
             for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                 const uint32_t buf = q & 1u;
                 const uint32_t acc = lane_addr + COL_ACC + buf * BN + half * (BN / 2);
@@ -757,12 +933,11 @@ assign_tc_kernel(const TcParams p) {
                 }
                 process(r[1], 1);
                 if (F16) {
-                    // both sub-chunks hand over their two smallest keys; the tile id carries the half
+                    // the two smallest keys of this thread's 64 columns; the tile id carries the half
                     const int tid2 = nt * 2 + half;
+                    ta.merge(tb);
                     rb.insert(ta.b0, tid2);
                     rb.insert(ta.b1, tid2);
-                    rb.insert(tb.b0, tid2);
-                    rb.insert(tb.b1, tid2);
                 } else {
                     ta.merge(tb);
                     const int hbit = half * (BN / 2);              // the upper half's columns start at 64
@@ -772,6 +947,17 @@ assign_tc_kernel(const TcParams p) {
                 }
             }
             if (!ok) break;
+            if (APRE) {
+                // both halves leave the row's candidates in shared memory for the row's thread among warps
+                // 0-3, which has little else to do here, and go straight on to the next tile
+                ok = mbar_wait(BAR(MG_FREE + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                float* mo = merge_buf + ((size_t)((it & 1) * 2 + half) * BM + row_in_tile) * 5;
+                mo[0] = __int_as_float(rb.r0); mo[1] = __int_as_float(rb.r1); mo[2] = __int_as_float(rb.r2);
+                mo[3] = __int_as_float(rb.t0); mo[4] = __int_as_float(rb.t1);
+                mbar_arrive_warp(BAR(MG_FULL + (it & 1)));
+                continue;
+            }
             // fold the upper half's running best into the lower half's through shared memory
             float* mg = merge_buf + ((size_t)(it & 1) * BM + row_in_tile) * 5;
             if (half == 1) {
@@ -786,48 +972,24 @@ assign_tc_kernel(const TcParams p) {
             const int row = r0 + row_in_tile;
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
-                int a0, a1;
-                float b0, b1, b2, delta;
-                bool third_known = ROW3;
-                if (F16) {
-                    // key = n * KQ_MUL + column (column inside the thread's 64; the tile id carries the
-                    // half); n * kstep is the squared distance.  A slightly negative distance gives a
-                    // negative key: it ranks first and reads as zero.
-                    auto quant = [](int key) {             // floor division: a negative key keeps its column
-                        return key >= 0 ? key / (int)KQ_MUL : -((-key + (int)KQ_MUL - 1) / (int)KQ_MUL);
-                    };
-                    const int n0 = quant(rb.r0), n1 = quant(rb.r1), n2 = quant(rb.r2);
-                    const int l0 = rb.r0 - n0 * (int)KQ_MUL, l1 = rb.r1 - n1 * (int)KQ_MUL;
-                    a0 = (rb.t0 >> 1) * BN + (rb.t0 & 1) * (BN / 2) + l0;
-                    a1 = (rb.t1 >> 1) * BN + (rb.t1 & 1) * (BN / 2) + l1;
-                    b0 = (float)max(n0, 0) * kstep; b1 = (float)max(n1, 0) * kstep; b2 = (float)max(n2, 0) * kstep;
-                    // near-tie bound: the split product's error, relative to ||z||^2 plus the largest
-                    // centroid norm of the instance (its centroids share one scale), plus two
-                    // quantisation steps
-                    delta = p.eps * (xn + cmaxn) + 2.f * kstep;
-                    // the third smallest is only known when the two smallest come from different
-                    // sub-chunks (same accumulator tile, same half, same tracker = same sub-chunk)
-                    third_known = !(rb.t0 == rb.t1 && ((l0 ^ l1) & 2) == 0);
+                if constexpr (F16) {
+                    emit_row_f16(p, rb, flat, xn, cmaxn, rscale);
                 } else {
-                    a0 = rb.column(rb.r0, rb.t0);
-                    a1 = rb.column(rb.r1, rb.t1);
-                    b0 = rb.value(rb.r0); b1 = rb.value(rb.r1); b2 = rb.value(rb.r2);
+                    const int a0 = rb.column(rb.r0, rb.t0), a1 = rb.column(rb.r1, rb.t1);
+                    const float b0 = rb.value(rb.r0), b1 = rb.value(rb.r1), b2 = rb.value(rb.r2);
                     // near-tie bound: the split product's error, relative to ||z||^2 plus the chosen
                     // centroid's norm, plus what the dropped key bits can hide
-                    delta = p.eps * (xn + cnb[a0]) + 1.52587890625e-5f * fabsf(b1);
-                }
-                p.labels[flat] = a0;
-                if (p.approx) p.approx[flat] = b0;
-                if (F16 && rscale < 0.f) {                     // row outside the fp16 range: exact scan over all K
-                    const int slot = atomicAdd(p.flag_count + 1, 1);
-                    p.full_rows[slot] = (int32_t)flat;
-                } else if (fabsf(b1 - b0) <= delta) {
-                    if (third_known && fabsf(b2 - b0) > delta) {   // exactly two candidates: compare them exactly
-                        const int slot = atomicAdd(p.flag_count, 1);
-                        p.pair_rows[slot] = make_int2((int)flat, a1);
-                    } else {                                   // three or more (or unknown): exact scan over all K
-                        const int slot = atomicAdd(p.flag_count + 1, 1);
-                        p.full_rows[slot] = (int32_t)flat;
+                    const float delta = p.eps * (xn + cnb[a0]) + 1.52587890625e-5f * fabsf(b1);
+                    p.labels[flat] = a0;
+                    if (p.approx) p.approx[flat] = b0;
+                    if (fabsf(b1 - b0) <= delta) {
+                        if (ROW3 && fabsf(b2 - b0) > delta) {      // exactly two candidates: compare them exactly
+                            const int slot = atomicAdd(p.flag_count, 1);
+                            p.pair_rows[slot] = make_int2((int)flat, a1);
+                        } else {                                   // three or more (or unknown): exact scan over all K
+                            const int slot = atomicAdd(p.flag_count + 1, 1);
+                            p.full_rows[slot] = (int32_t)flat;
+                        }
                     }
                 }
             }
@@ -852,9 +1014,15 @@ assign_tc_kernel(const TcParams p) {
             const uint32_t ext_lo32 = ((smem_u32(st_base + STAGE) & 0x3FFFFu) >> 4) | ((128u >> 4) << 16);
             const uint32_t ext_hi32 = (256u >> 4) | (1u << 14);
             const int ring = p.resident ? nt_count * nkb : NSTAGE;
+            const uint32_t adesc_lo32 = (uint32_t)smem_desc_sw128(smem_u32(as_base));   // pre-split A: buffer 0, hi panel
             for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
-                const int ab = it % nab, use = it / nab;
+                const int ab = APRE ? (it & 1) : it % nab, use = APRE ? (it >> 1) : it / nab;
                 const uint32_t a_base = tmem + COL_A + ab * AST;
+                const int sbuf = APRE ? it % p.nxb : 0;
+                if (APRE) {                                        // this tile's panels have landed
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(X_FULL + sbuf), (uint32_t)((it / p.nxb) & 1), abort_flag));
+                    if (!ok) break;
+                }
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
@@ -862,7 +1030,7 @@ assign_tc_kernel(const TcParams p) {
                     tc_fence_after();
                     const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
                     for (int kb = 0; kb < nkb; ++kb) {
-                        if (nt == 0) {
+                        if (nt == 0 && (!APRE || kb == 0)) {       // pre-split A: only the constant terms come this way
                             ok = __all_sync(0xffffffffu, mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag));
                             if (!ok) break;
                         }
@@ -873,6 +1041,25 @@ assign_tc_kernel(const TcParams p) {
                         tc_fence_after();
                         const uint32_t a_hi = a_base + kb * 32, a_lo = a_hi + DC;
                         const uint32_t blo = desc_lo32 + s * (SLOT >> 4);         // this stage's hi panel
+                        if (APRE) {
+                        if (elect_one()) {
+                            // both operands from shared memory; the constant-term product (A from tensor memory)
+                            // comes first and overwrites the accumulator tile
+                            const uint32_t ahi = adesc_lo32 + (uint32_t)((sbuf * ABUF + kb * STAGE) >> 4);
+                            if (kb == 0)
+                                tc_mma_ts<F16>(d_tmem, tmem + COL_A + ab * XCOLS, mk_desc(ext_lo32 + s * (SLOT >> 4), ext_hi32), IDESC, 0u);
+#pragma unroll
+                            for (int k8 = 0; k8 < KBF / 8; ++k8) {
+                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + (PANEL >> 4) + k8 * 2, desc_hi32), mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + k8 * 2, desc_hi32), mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
+                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + k8 * 2, desc_hi32), mk_desc(blo + k8 * 2, desc_hi32), IDESC);
+                            }
+                            if (!p.resident) tc_commit(BAR(B_EMPTY + s));
+                            if (nt == nt_count - 1 && kb == 0) tc_commit(BAR(A_EMPTY + ab * 4));          // constant terms reusable
+                            if (nt == nt_count - 1 && kb == nkb - 1) tc_commit(BAR(AS_EMPTY + sbuf));     // panels reusable
+                            if (kb == nkb - 1) tc_commit(BAR(ACC_FULL + buf));
+                        }
+                        } else
                         if (elect_one()) {
                         // The very first product of an accumulator tile overwrites it.  fp16 split: that is
                         // the constant-term product (the row's 16 extra features against the centroid
@@ -899,7 +1086,7 @@ assign_tc_kernel(const TcParams p) {
                 }
             }
         }
-    } else {
+    } else if (warp == 13) {
         // ============================ B loader ========================================
         if (lane == 0) {
             uint32_t s = 0, ph = 0;
@@ -928,6 +1115,33 @@ assign_tc_kernel(const TcParams p) {
                     const uint32_t idx = issued - 1 - k;
                     const uint32_t st = idx % NSTAGE, par = (idx / NSTAGE) & 1u;
                     for (uint32_t i = 0; i < WAIT_LIMIT && !mbar_try(BAR(B_FULL + st), par); ++i) {}
+                }
+            }
+        }
+    }
+
+    else if (APRE) {
+        // ============================ A loader (pre-split image) ======================
+        if (lane == 0) {
+            uint32_t issued = 0;
+            int it = 0;
+            for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
+                const int buf = it % p.nxb;
+                ok = mbar_wait(BAR(AS_EMPTY + buf), (uint32_t)(((it / p.nxb) & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(BAR(X_FULL + buf), (uint32_t)(ABUF + AINFO));
+                for (int kb = 0; kb < nkb; ++kb)
+                    bulk_g2s(smem_u32(as_base + (size_t)buf * ABUF + (size_t)kb * STAGE),
+                             p.aimg + ((size_t)tile * nkb + kb) * STAGE, STAGE, BAR(X_FULL + buf));
+                bulk_g2s(smem_u32(as_info + (size_t)buf * BM * 2), p.ainfo + (size_t)tile * BM * 2, AINFO, BAR(X_FULL + buf));
+                ++issued;
+            }
+            if (!ok) {
+                // let copies that are still in flight land before the CTA's shared memory goes away
+                const uint32_t nb = (uint32_t)p.nxb, pending = issued < nb ? issued : nb;
+                for (uint32_t k = 0; k < pending; ++k) {
+                    const uint32_t idx = issued - 1 - k;
+                    for (uint32_t i = 0; i < WAIT_LIMIT && !mbar_try(BAR(X_FULL + idx % nb), (idx / nb) & 1u); ++i) {}
                 }
             }
         }
@@ -1176,12 +1390,13 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
     }
 }
 
-size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool f16) {
+// nstage: stage slots kept in shared memory; apre: nxb buffers of pre-split A panels instead of fp32 rows
+size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool f16, int nstage = NSTAGE, bool apre = false) {
     size_t s = 1024;                                       // alignment slack
-    s += (size_t)NSTAGE * (f16 ? SLOT_F16 : STAGE);
-    s += (size_t)nxb * BM * (D + 4) * 4;
-    s += (f16 ? (size_t)2 * (Kpad / BN) * 4 : (size_t)Kpad * 4) + 4 * BM * 4 + (2 * BM * 5 + 2) * 4;
-    s += 40 * 8 + 16;                                      // barriers, TMEM slot, abort flag
+    s += (size_t)nstage * (f16 ? SLOT_F16 : STAGE);
+    s += apre ? (size_t)nxb * ((size_t)((D + 63) / 64) * STAGE + AINFO) : (size_t)nxb * BM * (D + 4) * 4;
+    s += (f16 ? (size_t)2 * (Kpad / BN) * 4 : (size_t)Kpad * 4) + 4 * BM * 4 + (4 * BM * 5 + 2) * 4;
+    s += 48 * 8 + 16;                                      // barriers, TMEM slot, abort flag
     return s;
 }
 
@@ -1194,6 +1409,47 @@ size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
     return kb_align256(B * Kpad * D * 8) + kb_align256(B * Kpad * 4) + kb_align256(B * Kpad * 32) +
            kb_align256((size_t)B * INST_STRIDE * 4) + 256 + kb_align256((size_t)B * N * 8) + kb_align256((size_t)B * N * 4);
 }
+
+// ---- the pre-split image of Z ------------------------------------------------------------
+// Bytes of the image (panels, then the row tables) for a matrix the fp16 kernel can take; 0 otherwise.
+size_t kb_ws_need_zsplit(int B, int N, int D, int K) {
+    if (B < 1 || N < 1 || D % KBF != 0 || D > 128 || K < 128) return 0;
+    const size_t tiles = (size_t)B * ((N + BM - 1) / BM), nkb = (D + 63) / 64;
+    return kb_align256(tiles * nkb * STAGE) + kb_align256(tiles * AINFO) + 1024;
+}
+
+// Shared-memory plan of the pre-split kernel: the B ring only as long as it has to be, then as many
+// A buffers as fit (two at least, three at most).  Returns 0 buffers when it does not fit.
+static int apre_plan(const kb_ctx* ctx, int B, int D, int Kpad, int* nstage_alloc) {
+    const int nkb = (D + 63) / 64;
+    const bool resident = B == 1 && (Kpad / BN) * nkb <= NSTAGE;
+    *nstage_alloc = resident ? (Kpad / BN) * nkb : NSTAGE;
+    for (int nxb = 3; nxb >= 2; --nxb)
+        if (tc_smem_bytes(D, Kpad * B, nxb, true, *nstage_alloc, true) <= (size_t)ctx->max_smem_optin) return nxb;
+    return 0;
+}
+
+// Builds the image of z at `img` (kb_ws_need_zsplit bytes, 1024-byte aligned) and remembers it in the
+// context: assignments of exactly this matrix then run from the image until kb_zsplit_forget.
+kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z) {
+    ctx->zs_src = nullptr;
+    const int Kpad = (K + BN - 1) / BN * BN;
+    int nstage_alloc = 0;
+    if (ctx->assign_path == 3 || kb_ws_need_zsplit(B, N, D, K) == 0 || !kb_assign_tc_supported(ctx, B, D, K) ||
+        apre_plan(ctx, B, D, Kpad, &nstage_alloc) == 0)
+        return KB_OK;                                      // the kernel that splits rows itself will run
+    const int tiles_per_inst = (N + BM - 1) / BM, nkb = (D + 63) / 64;
+    const size_t tiles = (size_t)B * tiles_per_inst;
+    unsigned char* aimg = reinterpret_cast<unsigned char*>(((uintptr_t)img + 1023) & ~(uintptr_t)1023);
+    float* ainfo = reinterpret_cast<float*>(aimg + kb_align256(tiles * nkb * STAGE));
+    kb_launch(tc_prep_z_f16_kernel, dim3((unsigned)(tiles_per_inst * BM / 8), B), 256, 0, ctx->stream, N, D, nkb,
+              tiles_per_inst, z, aimg, ainfo);
+    KB_LAUNCH_CHECK(ctx, "tc_prep_z_f16_kernel");
+    ctx->zs_src = z; ctx->zs_B = B; ctx->zs_N = N; ctx->zs_D = D;
+    ctx->zs_img = aimg; ctx->zs_info = ainfo;
+    return KB_OK;
+}
+void kb_zsplit_forget(kb_ctx* ctx) { ctx->zs_src = nullptr; }
 
 // what the kernel can run at all
 bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K) {
@@ -1242,25 +1498,37 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     p.tiles_per_inst = (N + BM - 1) / BM;
     p.total_tiles = p.tiles_per_inst * B;
     p.nxb = tc_smem_bytes(D, Kpad * B, 2, f16) <= (size_t)ctx->max_smem_optin ? 2 : 1;
+    p.nstage_alloc = NSTAGE;
     p.eps = eps;
     p.resident = (B == 1 && (Kpad / BN) * nkb <= NSTAGE) ? 1 : 0;
+    // a pre-split image of exactly this matrix (made by the fit that is calling): multiply out of it
+    bool apre = f16 && ctx->zs_src == z && ctx->zs_B == B && ctx->zs_N == N && ctx->zs_D == D;
+    if (apre) {
+        const int nxb = apre_plan(ctx, B, D, Kpad, &p.nstage_alloc);
+        if (nxb == 0) { apre = false; p.nstage_alloc = NSTAGE; }
+        else p.nxb = nxb;
+    }
+    ctx->last_assign_presplit = apre ? 1 : 0;
+    p.aimg = apre ? ctx->zs_img : nullptr;
+    p.ainfo = apre ? ctx->zs_info : nullptr;
     p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.bext = bext; p.inst = inst; p.labels = labels; p.approx = approx;
     p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
-    const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb, f16);
+    const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb, f16, p.nstage_alloc, apre);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
     // with few features per row the epilogue's per-column cost is what limits the kernel:
     // track less there and let the (cheap, K*D is small) full re-evaluation settle near-ties
     const bool track2 = f16 || D >= 96;
-#define KB_TC_LAUNCH(T2, F)                                                                    \
+#define KB_TC_LAUNCH(T2, F, AP)                                                                \
     do {                                                                                       \
-        KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F>), smem);                                   \
-        kb_launch(assign_tc_kernel<T2, F>, grid, TC_THREADS, smem, ctx->stream, p);                   \
+        KB_SMEM_OPTIN(ctx, (assign_tc_kernel<T2, F, AP>), smem);                               \
+        kb_launch(assign_tc_kernel<T2, F, AP>, grid, AP ? TC_THREADS_APRE : TC_THREADS, smem, ctx->stream, p); \
     } while (0)
     const int tslot = kb_time_begin(ctx, KB_T_ASSIGN_KERNEL);
-    if (track2 && f16) KB_TC_LAUNCH(true, true);
-    else if (track2) KB_TC_LAUNCH(true, false);
-    else if (f16) KB_TC_LAUNCH(false, true);
-    else KB_TC_LAUNCH(false, false);
+    if (apre) KB_TC_LAUNCH(true, true, true);
+    else if (track2 && f16) KB_TC_LAUNCH(true, true, false);
+    else if (track2) KB_TC_LAUNCH(true, false, false);
+    else if (f16) KB_TC_LAUNCH(false, true, false);
+    else KB_TC_LAUNCH(false, false, false);
 #undef KB_TC_LAUNCH
     kb_time_end(ctx, tslot);
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");

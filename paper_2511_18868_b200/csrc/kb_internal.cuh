@@ -26,7 +26,13 @@ struct kb_ctx {
     // assign path control: 0 = automatic, 1 = row-wise FFMA, 2 = tensor cores
     int assign_path;
     int last_assign_path;  // path the most recent kb_cluster_assign took (1 or 2; 0 = nothing ran)
+    int last_assign_presplit;   // 1: that assignment multiplied out of the pre-split image of Z
     float tc_eps;          // near-tie bound of the tensor path, relative to ||z||^2 + ||c||^2
+    // pre-split fp16 image of a matrix Z that a running fit keeps in the workspace (zs_src == nullptr: none)
+    const float* zs_src;
+    int zs_B, zs_N, zs_D;
+    const unsigned char* zs_img;
+    const float* zs_info;
     char err[256];
 };
 #define KB_EV_PAIRS 4096
@@ -79,6 +85,9 @@ static inline void kb_time_end(kb_ctx* ctx, int slot) {
 size_t kb_ws_need_normalize(int B, int N, int D);
 size_t kb_ws_need_assign(int B, int N, int D, int K);
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
+size_t kb_ws_need_zsplit(int B, int N, int D, int K);
+kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z);
+void kb_zsplit_forget(kb_ctx* ctx);
 bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K);
 bool kb_assign_tc_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
 kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K, const float* z, const float* c,

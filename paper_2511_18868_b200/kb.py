@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 # every symbol include/kb.h declares
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
-           "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_assign_tc_probe",
+           "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc"]
@@ -90,6 +90,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_score_select.argtypes = [_VP, i, i, i, i, ScoreParams] + [_VP] * 14
     lib.kb_set_assign_options.argtypes = [_VP, i, f]
     lib.kb_get_assign_path.argtypes = [_VP, ctypes.POINTER(i)]
+    lib.kb_get_assign_presplit.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_assign_tc_probe.argtypes = [_VP, i, i, i, i] + [_VP] * 5
     lib.kb_cluster_update_noalloc.argtypes = [_VP, i, i, i, _VP, _VP, _VP, _VP]
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
@@ -251,6 +252,11 @@ class KB:
         out = ctypes.c_int()
         self._check(self.lib.kb_get_assign_path(self.h, ctypes.byref(out)), "kb_get_assign_path")
         return out.value
+
+    def assign_presplit(self) -> bool:
+        out = ctypes.c_int()
+        self._check(self.lib.kb_get_assign_presplit(self.h, ctypes.byref(out)), "kb_get_assign_presplit")
+        return bool(out.value)
 
     def assign_tc_probe(self, z, centroids, labels, approx_dist2=None, flagged=None):
         B, N, D = z.shape

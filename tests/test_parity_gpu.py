@@ -388,6 +388,48 @@ def test_cluster_fit_cooperative(kbx, N, D, K, iters):
     parity.rep_match(got["rep"], chk, chk["dist2"], chk["labels"])
 
 
+@pytest.mark.parametrize("B,N,D,K,iters", [(1, 8229, 64, 256, 4), (3, 5000, 32, 128, 3), (1, 20011, 64, 130, 2),
+                                           (1, 6000, 64, 640, 2)])
+def test_cluster_fit_presplit(kbx, B, N, D, K, iters):
+    """A fit on the tensor path converts Z to its fp16 pieces once and every assignment of the loop multiplies out of
+    that image.  Its result must agree with the same loop made of single calls (which split rows on the fly), and
+    the final labels must be optimal for the returned centroids (checked in double)."""
+    cfg = wl.scaled(wl.CONFIGS["large"], B=B, N=N, D=D, K=K, components=max(4, K // 2), S=2, iters=iters)
+    inp = wl.make_inputs(cfg, seed=N + K)
+    z, _, _ = oracle.normalize(inp["x"])
+    c0 = oracle.init_centroids(z, inp["init_rows"])
+    ws(kbx, B, N, D, K, 2)
+    zd = dev(z)
+
+    def outputs():
+        return dict(labels=empty((B, N), torch.int32), d2=empty((B, N)), inertia=empty((B,)),
+                    rep=empty((B, K), torch.int32), counts=empty((B, K), torch.int32))
+
+    fit, c_fit = outputs(), dev(c0.copy())
+    kbx.cluster_fit(zd, c_fit, fit["labels"], iters, dist2=fit["d2"], inertia=fit["inertia"], rep=fit["rep"],
+                    counts=fit["counts"])
+    assert kbx.assign_path() == 2 and kbx.assign_presplit()
+    one, c_one = outputs(), dev(c0.copy())
+    for _ in range(iters):
+        kbx.cluster_assign(zd, c_one, one["labels"])
+        assert kbx.assign_path() == 2 and not kbx.assign_presplit()
+        kbx.cluster_update(zd, one["labels"], c_one, one["counts"])
+    kbx.cluster_assign(zd, c_one, one["labels"], one["d2"], one["inertia"], one["rep"])
+    assert kbx.device_status() == 0
+    got = {k: host(v) for k, v in fit.items()}
+    ref = {k: host(v) for k, v in one.items()}
+    assert np.mean(got["labels"] == ref["labels"]) > 0.995
+    parity.close(got["inertia"], ref["inertia"], atol=0, rtol=1e-3, what="inertia")
+    assert np.abs(got["counts"] - ref["counts"]).sum() <= 0.02 * B * N
+    cg = host(c_fit)
+    chk = oracle.cluster_assign(z, cg, want_margins=True, want_rep=True)
+    parity.labels_match(z, cg, got["labels"], chk)
+    same = got["labels"] == chk["labels"]
+    parity.close(got["d2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
+    parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia vs own labels")
+    parity.rep_match(got["rep"], chk, chk["dist2"], chk["labels"])
+
+
 def test_argument_errors(kbx):
     from paper_2511_18868_b200.kb import KbError
     z = empty((1, 8, 4))
