@@ -172,15 +172,6 @@ __device__ __forceinline__ void tc_mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, 
             ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
             : "memory");
 }
-// D[tmem] += A[smem desc] * B[smem desc], kind::f16 (both operands K-major panels in shared memory)
-__device__ __forceinline__ void tc_mma_ss_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.eq.b32 p, 0, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
-        : "memory");
-}
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
@@ -256,7 +247,7 @@ struct TcParams {
     int resident;                  // 1: the whole B image of the (single) instance stays in the stage ring
     float eps;                     // near-tie bound, relative to ||z||^2 + ||c||^2
     const float* z;
-    const unsigned char* aimg;     // pre-split A: [tile][nkb][hi panel | lo panel], the layout of a B stage
+    const unsigned char* aimg;     // pre-split A: [tile][BM][row image], see tc_prep_z_f16_kernel
     const float* ainfo;            // pre-split A: [tile][BM][2]  ||z||^2 and s_z of every row
     int nstage_alloc;              // stage slots that exist in shared memory (the whole ring unless B is resident)
     const unsigned char* bimg;     // [B][NT][NKB][STAGE]
@@ -423,14 +414,19 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
 }
 
 // The A side of the fp16 split, made ONCE for a matrix Z that many assignments will read (the Lloyd
-// loop of a fit): every 128-row tile becomes the same kind of image as a B stage,
-//   aimg  [tile][nkb][hi panel | lo panel]   128-byte-swizzled K-major panels of s_z z (s_z brings the
-//                                            row's largest magnitude into [0.5, 1))
-//   ainfo [tile][128][2]                     ||z||^2 and s_z of every row
-// so that an assignment fetches a tile with one bulk copy per k-block and multiplies straight out of
-// shared memory; only the row's constant-term operand, which depends on the centroids' scale, is
-// still formed per assignment.  One warp per row, lane q owns the 16-byte chunk q of the fp32 row.
-// Rows past the end of an instance are zeros.
+// loop of a fit).  Every 128-row tile becomes one contiguous image,
+//   aimg  [tile][128 rows][per k-block: 64 hi halfs | 64 lo halfs]
+//         the fp16 pieces of s_z z (s_z brings the row's largest magnitude into [0.5, 1)), each row
+//         in the order the tensor core reads a 16-bit A operand from tensor memory, except that the
+//         eight 16-byte chunks of a piece are stored at chunk index ^ (row & 7)
+//   ainfo [tile][128][2]   ||z||^2 and s_z of every row
+// so that an assignment fetches a tile with ONE bulk copy and its row threads only move their row
+// from shared to tensor memory (the chunk swizzle keeps their 16-byte reads free of bank conflicts); the
+// row's constant-term operand, which depends on the centroids' scale, is still formed per assignment.
+// One warp per row, lane q owns the 16-byte chunk q of the fp32 row.  Rows past the end of an
+// instance are zeros.
+__host__ __device__ constexpr int a_row_bytes(int nkb) { return nkb * 256; }
+
 __global__ void __launch_bounds__(256)
 tc_prep_z_f16_kernel(int N, int D, int nkb, int tiles_per_inst, const float* __restrict__ z,
                      unsigned char* __restrict__ aimg, float* __restrict__ ainfo) {
@@ -450,15 +446,16 @@ tc_prep_z_f16_kernel(int N, int D, int nkb, int tiles_per_inst, const float* __r
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     }
     const float sz = pow2_scale(m);
+    const int RB = a_row_bytes(nkb);
+    unsigned char* row = aimg + (tile * BM + r) * (size_t)RB;
     if (lane < nkb * 16) {
-        const int kb = lane >> 4, within = (lane & 15) * 8;                // byte offset inside the 128-byte row
-        const size_t off = (tile * nkb + kb) * STAGE + (size_t)(r >> 3) * 1024 + (r & 7) * 128 +
-                           (((within >> 4) ^ (r & 7)) << 4) + (within & 15);
+        const int kb = lane >> 4, within = (lane & 15) * 8;                // byte offset inside the 128 bytes of a piece
+        const int pos = (((within >> 4) ^ (r & 7)) << 4) + (within & 15);  // the same, with the chunk swizzled
         uint32_t h0, l0, h1, l1;
         split_f16x2(v.x * sz, v.y * sz, h0, l0);
         split_f16x2(v.z * sz, v.w * sz, h1, l1);
-        *reinterpret_cast<uint2*>(aimg + off) = make_uint2(h0, h1);
-        *reinterpret_cast<uint2*>(aimg + off + PANEL) = make_uint2(l0, l1);
+        *reinterpret_cast<uint2*>(row + kb * 256 + pos) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2*>(row + kb * 256 + 128 + pos) = make_uint2(l0, l1);
     }
     if (lane == 0) *reinterpret_cast<float2*>(ainfo + (tile * BM + r) * 2) = make_float2(xn, sz);
 }
@@ -586,9 +583,9 @@ assign_tc_kernel(const TcParams p) {
     const int xs_stride = D + 4;                          // floats; keeps float4 row reads conflict-free
     unsigned char* st_base = smem;                                        // nstage_alloc x SLOT
     float* xs = reinterpret_cast<float*>(smem + (size_t)p.nstage_alloc * SLOT);   // nxb x [BM][D+4]
-    // pre-split A: nxb x [nkb][hi panel | lo panel], then nxb x [BM][2] row tables, instead of xs
+    // pre-split A: nxb x [BM][row image], then nxb x [BM][2] row tables, instead of xs
     unsigned char* as_base = smem + (size_t)p.nstage_alloc * SLOT;
-    const int ABUF = nkb * STAGE;                                         // bytes of one tile's A panels
+    const int ARB = a_row_bytes(nkb), ABUF = BM * ARB;                    // bytes of a row image, of a tile's
     float* as_info = reinterpret_cast<float*>(as_base + (size_t)p.nxb * ABUF);
     float* cn = APRE ? as_info + (size_t)p.nxb * BM * 2                   // tf32: [B][Kpad] norms; fp16: [B][2] (s_c, max norm)
                      : xs + (size_t)p.nxb * BM * xs_stride;
@@ -615,7 +612,7 @@ assign_tc_kernel(const TcParams p) {
             mbar_init(BAR(XN_FULL + k), 4); mbar_init(BAR(XN_EMPTY + k), 8);
         }
         // staged rows: one arrival per producer thread; pre-split A: the loader's expect-tx arrival
-        for (int k = 0; k < 3; ++k) { mbar_init(BAR(X_FULL + k), APRE ? 1 : 128); mbar_init(BAR(AS_EMPTY + k), 1); }
+        for (int k = 0; k < 3; ++k) { mbar_init(BAR(X_FULL + k), APRE ? 1 : 128); mbar_init(BAR(AS_EMPTY + k), 4); }
         // pre-split A: the epilogue hands every row's candidates to the row's thread among warps 0-3
         for (int k = 0; k < 2; ++k) { mbar_init(BAR(MG_FULL + k), 8); mbar_init(BAR(MG_FREE + k), 4); }
         *abort_flag = 0;
@@ -649,9 +646,10 @@ assign_tc_kernel(const TcParams p) {
     bool ok = true;
 
     if (APRE && warp < 4) {
-        // ============================ A: constant terms only ==========================
-        // The tile's panels arrive pre-split by bulk copy; what is left per row is its constant-term
-        // operand (it depends on the centroids' scale s_c) and the two numbers the epilogue wants.
+        // ============================ A from the pre-split image ======================
+        // The tile arrives pre-split by one bulk copy; each thread moves its row from shared to tensor
+        // memory and forms the row's constant-term operand (it depends on the centroids' scale s_c) and
+        // the two numbers the epilogue wants.
         const int row_in_tile = tid;                       // = TMEM lane
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
         // What the epilogue found for this thread's row of tile number `jt` (of this CTA): merge the two
@@ -678,7 +676,7 @@ assign_tc_kernel(const TcParams p) {
         int it = 0, tile1 = -1, tile2 = -1;                // the previous tile and the one before it
         float xn1 = 0.f, rs1 = 1.f, xn2 = 0.f, rs2 = 1.f;
         for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
-            const int buf = it % p.nxb, ab = it & 1, use = it >> 1;
+            const int buf = it % p.nxb, ab = it % nab, use = it / nab;
             ok = mbar_wait(BAR(X_FULL + buf), (uint32_t)((it / p.nxb) & 1), abort_flag);
             if (!ok) break;
             const float2 info = *reinterpret_cast<const float2*>(as_info + ((size_t)buf * BM + row_in_tile) * 2);
@@ -692,20 +690,38 @@ assign_tc_kernel(const TcParams p) {
             const bool out_of_range = !(rho >= 6.103515625e-05f && rho <= 16384.f) || !(pterm < 60000.f);
             const float rscale = out_of_range ? -1.f : 1.f / g;
             if (out_of_range) { rho = 0.f; pterm = 0.f; }
-            __half p0, p1, p2;
-            split3_f16(pterm, p0, p1, p2);
-            const __half hr = __float2half_rn(rho);
-            const uint32_t e0 = pack_h2(p0, p1), e1 = pack_h2(p2, hr), e2 = pack_h2(hr, hr), ez = 0u;
-            ok = mbar_wait(BAR(A_EMPTY + ab * 4), (uint32_t)((use & 1) ^ 1), abort_flag);
+            const unsigned char* xr = as_base + (size_t)buf * ABUF + (size_t)row_in_tile * ARB;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                uint32_t hi[32], lo[32];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int pos = (q ^ (row_in_tile & 7)) << 4;      // chunk q of the piece, where the image keeps it
+                    const uint4 h = *reinterpret_cast<const uint4*>(xr + kb * 256 + pos);
+                    const uint4 l = *reinterpret_cast<const uint4*>(xr + kb * 256 + 128 + pos);
+                    hi[4 * q] = h.x; hi[4 * q + 1] = h.y; hi[4 * q + 2] = h.z; hi[4 * q + 3] = h.w;
+                    lo[4 * q] = l.x; lo[4 * q + 1] = l.y; lo[4 * q + 2] = l.z; lo[4 * q + 3] = l.w;
+                }
+                ok = mbar_wait(BAR(A_EMPTY + ab * 4 + kb), (uint32_t)((use & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                TC_ST32(lane_addr + COL_A + ab * AST + kb * 32, hi);
+                TC_ST32(lane_addr + COL_A + ab * AST + DC + kb * 32, lo);
+                if (kb == 0) {     // the row's constant-term operand travels with the first k-block
+                    __half p0, p1, p2;
+                    split3_f16(pterm, p0, p1, p2);
+                    const __half hr = __float2half_rn(rho);
+                    const uint32_t e0 = pack_h2(p0, p1), e1 = pack_h2(p2, hr), e2 = pack_h2(hr, hr), ez = 0u;
+                    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                 ::"r"(lane_addr + COL_A + ab * AST + 2 * DC), "r"(e0), "r"(e1), "r"(e2), "r"(ez), "r"(ez),
+                                   "r"(ez), "r"(ez), "r"(ez)
+                                 : "memory");
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive_warp(BAR(A_FULL + ab * 4 + kb));
+            }
             if (!ok) break;
-            tc_fence_after();
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                         ::"r"(lane_addr + COL_A + ab * XCOLS), "r"(e0), "r"(e1), "r"(e2), "r"(ez), "r"(ez),
-                           "r"(ez), "r"(ez), "r"(ez)
-                         : "memory");
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            tc_fence_before();
-            mbar_arrive_warp(BAR(A_FULL + ab * 4));
+            mbar_arrive_warp(BAR(AS_EMPTY + buf));                 // the row image has been read: the slot may be refilled
             ok = mbar_wait(BAR(XN_EMPTY + (it & 1)), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag);
             if (!ok) break;
             xnorm[(it & 1) * BM + row_in_tile] = xn;
@@ -1014,15 +1030,9 @@ assign_tc_kernel(const TcParams p) {
             const uint32_t ext_lo32 = ((smem_u32(st_base + STAGE) & 0x3FFFFu) >> 4) | ((128u >> 4) << 16);
             const uint32_t ext_hi32 = (256u >> 4) | (1u << 14);
             const int ring = p.resident ? nt_count * nkb : NSTAGE;
-            const uint32_t adesc_lo32 = (uint32_t)smem_desc_sw128(smem_u32(as_base));   // pre-split A: buffer 0, hi panel
             for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
-                const int ab = APRE ? (it & 1) : it % nab, use = APRE ? (it >> 1) : it / nab;
+                const int ab = it % nab, use = it / nab;
                 const uint32_t a_base = tmem + COL_A + ab * AST;
-                const int sbuf = APRE ? it % p.nxb : 0;
-                if (APRE) {                                        // this tile's panels have landed
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(X_FULL + sbuf), (uint32_t)((it / p.nxb) & 1), abort_flag));
-                    if (!ok) break;
-                }
                 for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
                     const uint32_t buf = q & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
@@ -1030,7 +1040,7 @@ assign_tc_kernel(const TcParams p) {
                     tc_fence_after();
                     const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
                     for (int kb = 0; kb < nkb; ++kb) {
-                        if (nt == 0 && (!APRE || kb == 0)) {       // pre-split A: only the constant terms come this way
+                        if (nt == 0) {
                             ok = __all_sync(0xffffffffu, mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag));
                             if (!ok) break;
                         }
@@ -1041,25 +1051,6 @@ assign_tc_kernel(const TcParams p) {
                         tc_fence_after();
                         const uint32_t a_hi = a_base + kb * 32, a_lo = a_hi + DC;
                         const uint32_t blo = desc_lo32 + s * (SLOT >> 4);         // this stage's hi panel
-                        if (APRE) {
-                        if (elect_one()) {
-                            // both operands from shared memory; the constant-term product (A from tensor memory)
-                            // comes first and overwrites the accumulator tile
-                            const uint32_t ahi = adesc_lo32 + (uint32_t)((sbuf * ABUF + kb * STAGE) >> 4);
-                            if (kb == 0)
-                                tc_mma_ts<F16>(d_tmem, tmem + COL_A + ab * XCOLS, mk_desc(ext_lo32 + s * (SLOT >> 4), ext_hi32), IDESC, 0u);
-#pragma unroll
-                            for (int k8 = 0; k8 < KBF / 8; ++k8) {
-                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + (PANEL >> 4) + k8 * 2, desc_hi32), mk_desc(blo + k8 * 2, desc_hi32), IDESC);
-                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + k8 * 2, desc_hi32), mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
-                                tc_mma_ss_acc(d_tmem, mk_desc(ahi + k8 * 2, desc_hi32), mk_desc(blo + k8 * 2, desc_hi32), IDESC);
-                            }
-                            if (!p.resident) tc_commit(BAR(B_EMPTY + s));
-                            if (nt == nt_count - 1 && kb == 0) tc_commit(BAR(A_EMPTY + ab * 4));          // constant terms reusable
-                            if (nt == nt_count - 1 && kb == nkb - 1) tc_commit(BAR(AS_EMPTY + sbuf));     // panels reusable
-                            if (kb == nkb - 1) tc_commit(BAR(ACC_FULL + buf));
-                        }
-                        } else
                         if (elect_one()) {
                         // The very first product of an accumulator tile overwrites it.  fp16 split: that is
                         // the constant-term product (the row's 16 extra features against the centroid
@@ -1130,9 +1121,7 @@ assign_tc_kernel(const TcParams p) {
                 ok = mbar_wait(BAR(AS_EMPTY + buf), (uint32_t)(((it / p.nxb) & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(BAR(X_FULL + buf), (uint32_t)(ABUF + AINFO));
-                for (int kb = 0; kb < nkb; ++kb)
-                    bulk_g2s(smem_u32(as_base + (size_t)buf * ABUF + (size_t)kb * STAGE),
-                             p.aimg + ((size_t)tile * nkb + kb) * STAGE, STAGE, BAR(X_FULL + buf));
+                bulk_g2s(smem_u32(as_base + (size_t)buf * ABUF), p.aimg + (size_t)tile * ABUF, (uint32_t)ABUF, BAR(X_FULL + buf));
                 bulk_g2s(smem_u32(as_info + (size_t)buf * BM * 2), p.ainfo + (size_t)tile * BM * 2, AINFO, BAR(X_FULL + buf));
                 ++issued;
             }
@@ -1394,7 +1383,7 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
 size_t tc_smem_bytes(int D, int Kpad /* summed over instances */, int nxb, bool f16, int nstage = NSTAGE, bool apre = false) {
     size_t s = 1024;                                       // alignment slack
     s += (size_t)nstage * (f16 ? SLOT_F16 : STAGE);
-    s += apre ? (size_t)nxb * ((size_t)((D + 63) / 64) * STAGE + AINFO) : (size_t)nxb * BM * (D + 4) * 4;
+    s += apre ? (size_t)nxb * ((size_t)BM * a_row_bytes((D + 63) / 64) + AINFO) : (size_t)nxb * BM * (D + 4) * 4;
     s += (f16 ? (size_t)2 * (Kpad / BN) * 4 : (size_t)Kpad * 4) + 4 * BM * 4 + (4 * BM * 5 + 2) * 4;
     s += 48 * 8 + 16;                                      // barriers, TMEM slot, abort flag
     return s;
@@ -1415,7 +1404,7 @@ size_t kb_ws_need_assign_tc(int B, int N, int D, int K) {
 size_t kb_ws_need_zsplit(int B, int N, int D, int K) {
     if (B < 1 || N < 1 || D % KBF != 0 || D > 128 || K < 128) return 0;
     const size_t tiles = (size_t)B * ((N + BM - 1) / BM), nkb = (D + 63) / 64;
-    return kb_align256(tiles * nkb * STAGE) + kb_align256(tiles * AINFO) + 1024;
+    return kb_align256(tiles * BM * a_row_bytes((int)nkb)) + kb_align256(tiles * AINFO) + 1024;
 }
 
 // Shared-memory plan of the pre-split kernel: the B ring only as long as it has to be, then as many
@@ -1441,7 +1430,7 @@ kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, 
     const int tiles_per_inst = (N + BM - 1) / BM, nkb = (D + 63) / 64;
     const size_t tiles = (size_t)B * tiles_per_inst;
     unsigned char* aimg = reinterpret_cast<unsigned char*>(((uintptr_t)img + 1023) & ~(uintptr_t)1023);
-    float* ainfo = reinterpret_cast<float*>(aimg + kb_align256(tiles * nkb * STAGE));
+    float* ainfo = reinterpret_cast<float*>(aimg + kb_align256(tiles * BM * a_row_bytes(nkb)));
     kb_launch(tc_prep_z_f16_kernel, dim3((unsigned)(tiles_per_inst * BM / 8), B), 256, 0, ctx->stream, N, D, nkb,
               tiles_per_inst, z, aimg, ainfo);
     KB_LAUNCH_CHECK(ctx, "tc_prep_z_f16_kernel");
