@@ -130,6 +130,16 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  : "memory");
 }
 
+// The same copy for data that is read once per kernel and is large (the pre-split image of Z): its lines
+// are marked evict-first in L2, so that streaming them does not push out what later kernels re-read.
+__device__ __forceinline__ void bulk_g2s_stream(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -1121,7 +1131,7 @@ assign_tc_kernel(const TcParams p) {
                 ok = mbar_wait(BAR(AS_EMPTY + buf), (uint32_t)(((it / p.nxb) & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(BAR(X_FULL + buf), (uint32_t)(ABUF + AINFO));
-                bulk_g2s(smem_u32(as_base + (size_t)buf * ABUF), p.aimg + (size_t)tile * ABUF, (uint32_t)ABUF, BAR(X_FULL + buf));
+                bulk_g2s_stream(smem_u32(as_base + (size_t)buf * ABUF), p.aimg + (size_t)tile * ABUF, (uint32_t)ABUF, BAR(X_FULL + buf));
                 bulk_g2s(smem_u32(as_info + (size_t)buf * BM * 2), p.ainfo + (size_t)tile * BM * 2, AINFO, BAR(X_FULL + buf));
                 ++issued;
             }
