@@ -119,8 +119,11 @@ assign_rowwise_kernel(int N, int D, int K, int TM, int CT, const float* __restri
         labels[i] = arg;
         if (dist2) dist2[i] = best;
         if (ws_rep) {
-            unsigned long long key = ((unsigned long long)__float_as_uint(best) << 32) | (unsigned)(r0 + tid);
-            atomicMin(&ws_rep[(size_t)b * K + arg], key);
+            // all rows of a cluster meet in one word: only a key that beats the value seen so far (a cached,
+            // possibly stale, hence larger one) goes to the atomic unit
+            const unsigned long long key = ((unsigned long long)__float_as_uint(best) << 32) | (unsigned)(r0 + tid);
+            unsigned long long* slot = &ws_rep[(size_t)b * K + arg];
+            if (key < __ldca(slot)) atomicMin(slot, key);
         }
     }
     if (ws_inertia) {

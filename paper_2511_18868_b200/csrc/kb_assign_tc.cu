@@ -433,33 +433,35 @@ tc_prep_f16_kernel(int K, int D, int Kpad, int nkb, const float* __restrict__ ce
 // so that an assignment fetches a tile with ONE bulk copy and its row threads only move their row
 // from shared to tensor memory (the chunk swizzle keeps their 16-byte reads free of bank conflicts); the
 // row's constant-term operand, which depends on the centroids' scale, is still formed per assignment.
-// One warp per row, lane q owns the 16-byte chunk q of the fp32 row.  Rows past the end of an
-// instance are zeros.
+// Rows past the end of an instance are zeros.
 __host__ __device__ constexpr int a_row_bytes(int nkb) { return nkb * 256; }
 
 __global__ void __launch_bounds__(256)
 tc_prep_z_f16_kernel(int N, int D, int nkb, int tiles_per_inst, const float* __restrict__ z,
                      unsigned char* __restrict__ aimg, float* __restrict__ ainfo) {
     kb_grid_dependency_wait();
+    // a group of LPR lanes owns a row (lane q of the group: the 16-byte chunk q of the fp32 row, or zeros
+    // behind the row's end up to the k-block's 64 features), RPW rows per warp
+    const int LPR = nkb * 16, RPW = 32 / LPR;
     const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long slot = (long)blockIdx.x * 8 + warp;                 // row slot inside the instance's tiles
-    if (slot >= (long)tiles_per_inst * BM) return;
+    const int q = lane % LPR;
+    const long slot = ((long)blockIdx.x * 8 + warp) * RPW + lane / LPR;    // row slot inside the instance's tiles
+    const bool live = slot < (long)tiles_per_inst * BM;
     const int t = (int)(slot / BM), r = (int)(slot - (long)t * BM);
     const size_t tile = (size_t)b * tiles_per_inst + t;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (slot < N && lane < D / 4) v = __ldg(reinterpret_cast<const float4*>(z + ((size_t)b * N + slot) * D) + lane);
+    if (live && slot < N && q < D / 4) v = __ldg(reinterpret_cast<const float4*>(z + ((size_t)b * N + slot) * D) + q);
     float xn = fmaf(v.w, v.w, fmaf(v.z, v.z, fmaf(v.y, v.y, v.x * v.x)));
     float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = LPR >> 1; o > 0; o >>= 1) {
         xn += __shfl_xor_sync(0xffffffffu, xn, o);
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     }
+    if (!live) return;
     const float sz = pow2_scale(m);
-    const int RB = a_row_bytes(nkb);
-    unsigned char* row = aimg + (tile * BM + r) * (size_t)RB;
-    if (lane < nkb * 16) {
-        const int kb = lane >> 4, within = (lane & 15) * 8;                // byte offset inside the 128 bytes of a piece
+    unsigned char* row = aimg + (tile * BM + r) * (size_t)a_row_bytes(nkb);
+    {
+        const int kb = q >> 4, within = (q & 15) * 8;                      // byte offset inside the 128 bytes of a piece
         const int pos = (((within >> 4) ^ (r & 7)) << 4) + (within & 15);  // the same, with the chunk swizzled
         uint32_t h0, l0, h1, l1;
         split_f16x2(v.x * sz, v.y * sz, h0, l0);
@@ -467,7 +469,7 @@ tc_prep_z_f16_kernel(int N, int D, int nkb, int tiles_per_inst, const float* __r
         *reinterpret_cast<uint2*>(row + kb * 256 + pos) = make_uint2(h0, h1);
         *reinterpret_cast<uint2*>(row + kb * 256 + 128 + pos) = make_uint2(l0, l1);
     }
-    if (lane == 0) *reinterpret_cast<float2*>(ainfo + (tile * BM + r) * 2) = make_float2(xn, sz);
+    if (q == 0) *reinterpret_cast<float2*>(ainfo + (tile * BM + r) * 2) = make_float2(xn, sz);
 }
 
 // ---- the contraction -------------------------------------------------------------------
@@ -1377,8 +1379,11 @@ assign_finish_kernel(int N, int D, int K, const float* __restrict__ z, const flo
                 if (dist2) dist2[flat] = a;
                 local += (double)a;
                 if (ws_rep) {
-                    unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned)r;
-                    atomicMin(&ws_rep[(size_t)b * K + lab[u]], key);
+                    // all rows of a cluster meet in one word: only a key that beats the value seen so far (a
+                    // cached, possibly stale, hence larger one) goes to the atomic unit
+                    const unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned)r;
+                    unsigned long long* slot = &ws_rep[(size_t)b * K + lab[u]];
+                    if (key < __ldca(slot)) atomicMin(slot, key);
                 }
             }
         }
@@ -1441,7 +1446,8 @@ kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, 
     const size_t tiles = (size_t)B * tiles_per_inst;
     unsigned char* aimg = reinterpret_cast<unsigned char*>(((uintptr_t)img + 1023) & ~(uintptr_t)1023);
     float* ainfo = reinterpret_cast<float*>(aimg + kb_align256(tiles * BM * a_row_bytes(nkb)));
-    kb_launch(tc_prep_z_f16_kernel, dim3((unsigned)(tiles_per_inst * BM / 8), B), 256, 0, ctx->stream, N, D, nkb,
+    const int rows_per_block = 8 * (32 / (nkb * 16));      // 8 warps, one or two rows each
+    kb_launch(tc_prep_z_f16_kernel, dim3((unsigned)(tiles_per_inst * BM / rows_per_block), B), 256, 0, ctx->stream, N, D, nkb,
               tiles_per_inst, z, aimg, ainfo);
     KB_LAUNCH_CHECK(ctx, "tc_prep_z_f16_kernel");
     ctx->zs_src = z; ctx->zs_B = B; ctx->zs_N = N; ctx->zs_D = D;

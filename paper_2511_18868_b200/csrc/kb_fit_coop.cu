@@ -258,7 +258,10 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
         mine += (double)bb;
         // the representative is the member with the smallest (dist2, row): keys are stored inverted so
         // that the cleared word means "no member" and atomicMax keeps the smallest key
-        if (rep) atomicMax(&rep_key[a], ~(((unsigned long long)__float_as_uint(bb) << 32) | (unsigned)r));
+        if (rep) {                                          // (a key that cannot win is dropped after a cached read)
+            const unsigned long long inv = ~(((unsigned long long)__float_as_uint(bb) << 32) | (unsigned)r);
+            if (inv > __ldca(rep_key + a)) atomicMax(&rep_key[a], inv);
+        }
     }
     if (g == 0) {
         for (int e = tid; e < KD / 4; e += CF_T)
