@@ -1299,22 +1299,17 @@ fixup_full(int N, int D, int K, int total, const float* __restrict__ z, const fl
     }
 }
 
-// The two queues are settled by two kernels: the two-candidate rows by warps that need no shared
-// memory (full occupancy), the rows that need all K centroids by blocks that stage centroid tiles
-// in shared memory, in groups sized to the queue's length.
-__global__ void __launch_bounds__(FX_T)
-assign_fixup_pairs_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                          const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
-                          int32_t* __restrict__ labels) {
-    kb_grid_dependency_wait();
-    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
-}
-
+// Both queues are settled by one launch (each is short: a second launch would cost more than it
+// runs): first the two-candidate rows, a warp each, then the rows that need all K centroids, by
+// blocks that stage centroid tiles in shared memory, in groups sized to the queue's length.
+// (Giving each queue its own share of the blocks was slower: fewer blocks then carry more rows
+// through the full re-evaluation, whose time grows with the rows per block.)
 __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
-                    const int* __restrict__ flag_count, const int32_t* __restrict__ full_rows,
-                    int32_t* __restrict__ labels) {
+                    const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
     kb_grid_dependency_wait();
+    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
     extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_MAXROWS][FX_T / 32];
     __shared__ int red_i[FX_MAXROWS][FX_T / 32];
@@ -1538,13 +1533,11 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     kb_time_end(ctx, tslot);
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
-    kb_launch(assign_fixup_pairs_kernel, 8 * ctx->sm_count, FX_T, 0, ctx->stream, N, D, K, z, c, flag_count, pair_rows, labels);
-    KB_LAUNCH_CHECK(ctx, "assign_fixup_pairs_kernel");
     const size_t fsmem = (size_t)FX_MAXROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
     const int fblocks = (int)(((size_t)ctx->max_smem_optin / (fsmem + 2048)) < 1 ? 1 : ((size_t)ctx->max_smem_optin / (fsmem + 2048)));
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
     kb_launch(assign_fixup_kernel, (fblocks > 4 ? 4 : fblocks) * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count,
-              full_rows, labels);
+              pair_rows, full_rows, labels);
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
         KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
