@@ -540,6 +540,9 @@ struct RowBest {
 // distance gives a negative key: it ranks first and reads as zero.  Writes the label (and the
 // diagnostic distance) and queues the row for the exact re-evaluation when its runner-up lies inside
 // the error bound.
+// FINE: each of a thread's two trackers (alternate column pairs, 32 columns of the tile) handed over its
+// own two smallest keys; otherwise the thread's trackers were merged first (64 columns per sub-chunk).
+template <bool FINE>
 __device__ __forceinline__ void emit_row_f16(const TcParams& p, const RowBest<true>& rb, size_t flat, float xn,
                                              float cmaxn, float rscale) {
     const float range_d2 = fmaxf(2.f * (xn + cmaxn), 1e-30f);
@@ -555,9 +558,9 @@ __device__ __forceinline__ void emit_row_f16(const TcParams& p, const RowBest<tr
     // near-tie bound: the split product's error, relative to ||z||^2 plus the largest centroid norm of
     // the instance (its centroids share one scale), plus two quantisation steps
     const float delta = p.eps * (xn + cmaxn) + 2.f * kstep;
-    // the third smallest is only known when the two smallest come from different sub-chunks (the 64
-    // columns of an accumulator tile that one thread ranks: each hands over its two smallest keys)
-    const bool third_known = rb.t0 != rb.t1;
+    // the third smallest is only known when the two smallest come from different sub-chunks (each
+    // sub-chunk hands over its two smallest keys only)
+    const bool third_known = FINE ? !(rb.t0 == rb.t1 && ((l0 ^ l1) & 2) == 0) : rb.t0 != rb.t1;
     p.labels[flat] = a0;
     if (p.approx) p.approx[flat] = b0;
     if (rscale < 0.f) {                                // row outside the fp16 range: exact scan over all K
@@ -578,8 +581,9 @@ template <bool TRACK2, bool F16, bool APRE>
 __global__ void __launch_bounds__(APRE ? TC_THREADS_APRE : TC_THREADS, 1)
 assign_tc_kernel(const TcParams p) {
     static_assert(!APRE || F16, "the pre-split A image exists for the fp16 split only");
-    // fp16 split: the hot loop keeps the two smallest keys of each sub-chunk (the 64 columns one
-    // thread ranks in an accumulator tile); the row's running best keeps three keys.  The third
+    // fp16 split: the hot loop keeps the two smallest keys of each sub-chunk (the 32 columns one
+    // tracker sees in an accumulator tile; the pre-split kernel merges a thread's two trackers: 64
+    // columns); the row's running best keeps three keys.  The third
     // smallest distance of the row is then known unless the two smallest come from the same
     // sub-chunk, in which case a near-tie goes to the full re-evaluation.
     constexpr bool HOT3 = F16 ? false : TRACK2;           // hot-loop trackers keep a third key
@@ -680,7 +684,7 @@ assign_tc_kernel(const TcParams p) {
             rb.insert(u1, v1);
             rb.r2 = min(rb.r2, u2);
             const int b = tile / p.tiles_per_inst, row = (tile - b * p.tiles_per_inst) * BM + row_in_tile;
-            if (row < p.N) emit_row_f16(p, rb, (size_t)b * p.N + row, xn, cn[2 * b + 1], rscale);
+            if (row < p.N) emit_row_f16<false>(p, rb, (size_t)b * p.N + row, xn, cn[2 * b + 1], rscale);
             return true;
         };
         // rows are finished two tiles behind: the constant terms of tile i + 1 must be in place when the
@@ -961,11 +965,18 @@ assign_tc_kernel(const TcParams p) {
                 }
                 process(r[1], 1);
                 if (F16) {
-                    // the two smallest keys of this thread's 64 columns; the tile id carries the half
+                    // the tile id carries the half
                     const int tid2 = nt * 2 + half;
-                    ta.merge(tb);
-                    rb.insert(ta.b0, tid2);
-                    rb.insert(ta.b1, tid2);
+                    if (APRE) {            // the two smallest keys of this thread's 64 columns: fewer inserts on the
+                        ta.merge(tb);      // epilogue's chain, a few more rows in the full re-evaluation
+                        rb.insert(ta.b0, tid2);
+                        rb.insert(ta.b1, tid2);
+                    } else {               // both trackers hand over their two smallest keys
+                        rb.insert(ta.b0, tid2);
+                        rb.insert(ta.b1, tid2);
+                        rb.insert(tb.b0, tid2);
+                        rb.insert(tb.b1, tid2);
+                    }
                 } else {
                     ta.merge(tb);
                     const int hbit = half * (BN / 2);              // the upper half's columns start at 64
@@ -1001,7 +1012,7 @@ assign_tc_kernel(const TcParams p) {
             if (row < p.N) {
                 const size_t flat = (size_t)b * p.N + row;
                 if constexpr (F16) {
-                    emit_row_f16(p, rb, flat, xn, cmaxn, rscale);
+                    emit_row_f16<true>(p, rb, flat, xn, cmaxn, rscale);
                 } else {
                     const int a0 = rb.column(rb.r0, rb.t0), a1 = rb.column(rb.r1, rb.t1);
                     const float b0 = rb.value(rb.r0), b1 = rb.value(rb.r1), b2 = rb.value(rb.r2);
@@ -1299,17 +1310,26 @@ fixup_full(int N, int D, int K, int total, const float* __restrict__ z, const fl
     }
 }
 
-// Both queues are settled by one launch (each is short: a second launch would cost more than it
-// runs): first the two-candidate rows, a warp each, then the rows that need all K centroids, by
-// blocks that stage centroid tiles in shared memory, in groups sized to the queue's length.
-// (Giving each queue its own share of the blocks was slower: fewer blocks then carry more rows
-// through the full re-evaluation, whose time grows with the rows per block.)
+// The two-candidate rows are settled by warps that need no shared memory, the rows that need all K
+// centroids by blocks that stage centroid tiles in shared memory, in groups sized to the queue's
+// length.  With few rows in all (both queues are short: a second launch would cost more than it runs)
+// one launch does both, one after the other (`pair_rows` non-null); with many rows the pairs get a
+// launch of their own at full occupancy.  (Giving each queue its own share of the blocks of one
+// launch was slower: fewer blocks then carry more rows through the full re-evaluation.)
+__global__ void __launch_bounds__(FX_T)
+assign_fixup_pairs_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
+                          const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
+                          int32_t* __restrict__ labels) {
+    kb_grid_dependency_wait();
+    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
+}
+
 __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                     const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
                     const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
     kb_grid_dependency_wait();
-    fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
+    if (pair_rows) fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
     extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_MAXROWS][FX_T / 32];
     __shared__ int red_i[FX_MAXROWS][FX_T / 32];
@@ -1533,11 +1553,16 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     kb_time_end(ctx, tslot);
     KB_LAUNCH_CHECK(ctx, "assign_tc_kernel");
 
+    const bool one_launch = (long long)B * N <= 524288;     // about five thousand queued rows at most
+    if (!one_launch) {
+        kb_launch(assign_fixup_pairs_kernel, 8 * ctx->sm_count, FX_T, 0, ctx->stream, N, D, K, z, c, flag_count, pair_rows, labels);
+        KB_LAUNCH_CHECK(ctx, "assign_fixup_pairs_kernel");
+    }
     const size_t fsmem = (size_t)FX_MAXROWS * D * 4 + (size_t)FX_T * (D + 4) * 4;
     const int fblocks = (int)(((size_t)ctx->max_smem_optin / (fsmem + 2048)) < 1 ? 1 : ((size_t)ctx->max_smem_optin / (fsmem + 2048)));
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
     kb_launch(assign_fixup_kernel, (fblocks > 4 ? 4 : fblocks) * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count,
-              pair_rows, full_rows, labels);
+              one_launch ? pair_rows : static_cast<int2*>(nullptr), full_rows, labels);
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
         KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
