@@ -40,14 +40,22 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
     const int q = tid % vps;
     const int rstep = PV_T / vps;
     const bool sat = labels != nullptr;
+    // per-strategy constants: the block forms the reciprocals once (a thread handles only a few rows, so eight
+    // divisions of its own would cost as much as its share of the work)
+    __shared__ float s_rP[32], s_rW[32];
+    if (tid < S) {
+        s_rP[tid] = 1.f / peak_flops[tid];
+        s_rW[tid] = 1.f / peak_bw[tid];
+    }
+    __syncthreads();
     float P[4], W[4], rP[4], rW[4];
     int tg[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         P[i] = peak_flops[4 * q + i];
         W[i] = peak_bw[4 * q + i];
-        rP[i] = 1.f / P[i];
-        rW[i] = 1.f / W[i];
+        rP[i] = s_rP[4 * q + i];
+        rW[i] = s_rW[4 * q + i];
         int t = sat ? target[4 * q + i] : 0;
         if (t < 0 || t >= R) { if (sat) atomicOr(dev_status, 2); t = 0; }
         tg[i] = t;
@@ -193,7 +201,16 @@ kb_status kb_launch_prune(kb_ctx* ctx, int B, int N, int S, int K, int R, const 
     if (N == 0) return KB_OK;
     const bool vec = (S == 4 || S == 8 || S == 16 || S == 32) && (((uintptr_t)bound & 15) == 0);
     if (vec) {
-        long want = (8L * ctx->sm_count + B - 1) / B;
+        // one full wave: as many blocks as the device holds at once (the kernel's registers decide), split
+        // over the instances; a grid of a wave and a fraction would run as long as two waves
+        static int per_sm = 0;
+        if (per_sm == 0) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_vec_kernel, PV_T, 0) != cudaSuccess || n < 1) n = 2;
+            per_sm = n;
+        }
+        long want = ((long)per_sm * ctx->sm_count) / B;
+        if (want < 1) want = 1;
         long cap = ((long)N * (S / 4) + PV_T - 1) / PV_T;
         int G = (int)(want > cap ? cap : want);
         if (G < 1) G = 1;
