@@ -388,6 +388,42 @@ def test_cluster_fit_cooperative(kbx, N, D, K, iters):
     parity.rep_match(got["rep"], chk, chk["dist2"], chk["labels"])
 
 
+@pytest.mark.parametrize("D,K", [(32, 64), (16, 9), (64, 40)])
+def test_cluster_fit_cooperative_ties_and_empty_clusters(kbx, D, K):
+    """The cooperative fit splits a row's centroid scan over several threads: duplicate centroids that fall into
+    different parts must still resolve to the lowest id, and a centroid that attracts no row keeps its
+    coordinates, reports count 0 and representative -1."""
+    N = 3000
+    rng = np.random.default_rng(D * 100 + K)
+    z = rng.standard_normal((1, N, D)).astype(np.float32)
+    c0 = z[:, rng.choice(N, K, replace=False)].copy()
+    c0[0, K - 1] = c0[0, 0]                       # duplicate of centroid 0 in the last part: must never win
+    c0[0, K // 2] = c0[0, 1]                      # duplicate of centroid 1 in a middle part
+    far = K // 3
+    c0[0, far] = 1e3                              # attracts no row
+    ws(kbx, 1, N, D, K, 2)
+    for iters in (0, 3):
+        c = dev(c0.copy())
+        labels, d2 = empty((1, N), torch.int32), empty((1, N))
+        inertia, rep, counts = empty((1,)), empty((1, K), torch.int32), empty((1, K), torch.int32)
+        kbx.cluster_fit(dev(z), c, labels, iters, dist2=d2, inertia=inertia, rep=rep, counts=counts)
+        assert kbx.device_status() == 0
+        lab, cg = host(labels), host(c)
+        assert not np.any(lab == far)
+        np.testing.assert_array_equal(cg[0, far], c0[0, far])
+        assert host(rep)[0, far] == -1
+        if iters == 0:
+            # (after an update the originals move and their untouched duplicates become centroids of their own)
+            assert not np.any(lab == K - 1) and not np.any(lab == K // 2)
+            assert host(rep)[0, K - 1] == -1 and host(rep)[0, K // 2] == -1
+        else:
+            cnt = host(counts)
+            assert cnt[0, far] == 0 and cnt.sum() == N
+        chk = oracle.cluster_assign(z, cg, want_margins=True, want_rep=True)
+        parity.labels_match(z, cg, lab, chk)
+        parity.close(host(inertia), chk["inertia"], atol=1e-6, what="inertia")
+
+
 @pytest.mark.parametrize("B,N,D,K,iters", [(1, 8229, 64, 256, 4), (3, 5000, 32, 128, 3), (1, 20011, 64, 130, 2),
                                            (1, 6000, 64, 640, 2)])
 def test_cluster_fit_presplit(kbx, B, N, D, K, iters):
