@@ -319,8 +319,12 @@ typedef struct {
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
 
 /* The same step for a caller whose data lives in HOST memory: copies the
- * inputs to the device, runs kb_bandit_step, copies the requested outputs
- * back and synchronises the stream before returning.  The device staging
+ * inputs to the device, runs the calls of kb_bandit_step, copies the requested
+ * outputs back and synchronises the stream before returning.  The inputs that
+ * only pruning and scoring read (work, traffic, runtimes, signatures, pulls,
+ * rewards) travel on a second stream owned by the context while the clustering
+ * runs on the caller's stream; the caller's stream waits for them before
+ * kb_prune.  The device staging
  * area is carved from the registered workspace, which must hold
  * kb_step_workspace_bytes(...) bytes.  Pinned host memory makes the copies
  * asynchronous; pageable memory works too. */

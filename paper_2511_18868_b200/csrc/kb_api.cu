@@ -87,10 +87,17 @@ kb_status kb_create(kb_ctx** out, int device, void* cuda_stream) {
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->coop_launch, cudaDevAttrCooperativeLaunch, device);
+    // the host-buffer step copies the inputs its last calls need on a stream of its own, beside the clustering
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_step_begin, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_late_inputs, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
     if (e != cudaSuccess) {
         if (ctx->dev_status) cudaFree(ctx->dev_status);
+        if (ctx->ev_late_inputs) cudaEventDestroy(ctx->ev_late_inputs);
+        if (ctx->ev_step_begin) cudaEventDestroy(ctx->ev_step_begin);
+        if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
         delete ctx;
         return KB_ERR_CUDA;
     }
@@ -134,6 +141,9 @@ kb_status kb_destroy(kb_ctx* ctx) {
         delete[] ctx->ev_class;
     }
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->ev_late_inputs) cudaEventDestroy(ctx->ev_late_inputs);
+    if (ctx->ev_step_begin) cudaEventDestroy(ctx->ev_step_begin);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     delete ctx;
     return KB_OK;
 }
@@ -456,37 +466,59 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
         return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_bandit_step_host needs %zu bytes of workspace", scratch + stage);
     carve_step(ctx->ws + scratch, *h, &d);
     const size_t B = h->B, N = h->N, D = h->D, K = h->K, S = h->S, R = h->R;
-    cudaStream_t st = ctx->stream;
-#define KB_H2D(field, count, type)                                                                     \
+    cudaStream_t st = ctx->stream, cs = ctx->copy_stream;
+#define KB_H2D(field, count, type, stream)                                                             \
     do {                                                                                               \
         if ((count) > 0) {                                                                             \
             KB_REQUIRE(ctx, h->field, "kb_bandit_step_host: input " #field " is required");            \
             KB_CUDA(ctx, cudaMemcpyAsync(const_cast<type*>(d.field), h->field, (count) * sizeof(type), \
-                                         cudaMemcpyHostToDevice, st));                                 \
+                                         cudaMemcpyHostToDevice, stream));                             \
         }                                                                                              \
     } while (0)
-    KB_H2D(x, B * N * D, float);
-    KB_H2D(init_rows, B * K, int32_t);
-    KB_H2D(flops, B * N, float);
-    KB_H2D(bytes, B * N, float);
-    KB_H2D(peak_flops, S, float);
-    KB_H2D(peak_bw, S, float);
-    KB_H2D(t_incumbent, B, float);
-    KB_H2D(t_cur, B * N, float);
-    KB_H2D(hsig, B * K * R, float);
-    KB_H2D(target, S, int32_t);
-    KB_H2D(pulls, B * N * S, int32_t);
-    KB_H2D(reward_sum, B * N * S, float);
-    KB_H2D(t, B, int32_t);
+    // What normalise and the clustering read goes first, on the caller's stream.  Everything that only the
+    // pruning and the scoring read (two thirds of the input bytes when S is large) is copied on a second
+    // stream while the clustering runs; that stream starts behind whatever the caller's stream held before
+    // this call (the staging area may still be in use by it).
+    KB_CUDA(ctx, cudaEventRecord(ctx->ev_step_begin, st));
+    KB_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->ev_step_begin, 0));
+    KB_H2D(x, B * N * D, float, st);
+    KB_H2D(init_rows, B * K, int32_t, st);
+    KB_H2D(flops, B * N, float, cs);
+    KB_H2D(bytes, B * N, float, cs);
+    KB_H2D(peak_flops, S, float, cs);
+    KB_H2D(peak_bw, S, float, cs);
+    KB_H2D(t_incumbent, B, float, cs);
+    KB_H2D(t_cur, B * N, float, cs);
+    KB_H2D(hsig, B * K * R, float, cs);
+    KB_H2D(target, S, int32_t, cs);
+    KB_H2D(pulls, B * N * S, int32_t, cs);
+    KB_H2D(reward_sum, B * N * S, float, cs);
+    KB_H2D(t, B, int32_t, cs);
 #undef KB_H2D
+    KB_CUDA(ctx, cudaEventRecord(ctx->ev_late_inputs, cs));
     // run on the workspace's scratch part only
     char* ws_saved = ctx->ws;
     size_t bytes_saved = ctx->ws_bytes;
     ctx->ws_bytes = scratch;
-    kb_status s = kb_bandit_step(ctx, &d);
+    kb_status s = kb_normalize(ctx, d.B, d.N, d.D, d.x, d.z, nullptr, nullptr);
+    if (s == KB_OK) s = kb_init_centroids(ctx, d.B, d.N, d.D, d.K, d.z, d.init_rows, d.centroids);
+    if (s == KB_OK)
+        s = kb_cluster_fit(ctx, d.B, d.N, d.D, d.K, d.iters, d.z, d.centroids, d.labels, d.dist2, d.inertia, d.rep, d.counts);
+    if (s == KB_OK && cudaStreamWaitEvent(st, ctx->ev_late_inputs, 0) != cudaSuccess)
+        s = kb_fail(ctx, KB_ERR_CUDA, "kb_bandit_step_host: cudaStreamWaitEvent failed");
+    if (s == KB_OK)
+        s = kb_prune(ctx, d.B, d.N, d.S, d.K, d.R, d.flops, d.bytes, d.peak_flops, d.peak_bw, d.t_incumbent, d.t_cur,
+                     d.labels, d.hsig, d.target, d.theta_sat, d.keep, d.kept_count, d.bound);
+    if (s == KB_OK)
+        s = kb_score_select(ctx, d.B, d.N, d.K, d.S, d.score, d.labels, d.dist2, d.pulls, d.reward_sum, d.keep, d.bound,
+                            d.t, d.cl_pulls, d.cl_mean, d.cl_index, d.arm_index, d.best_arm, d.best_val,
+                            d.best_cluster_arm);
     ctx->ws = ws_saved;
     ctx->ws_bytes = bytes_saved;
-    if (s != KB_OK) return s;
+    if (s != KB_OK) {
+        cudaStreamSynchronize(cs);             // nothing of this call may still be writing the staging area
+        return s;
+    }
 #define KB_D2H(field, count, type)                                                                          \
     do {                                                                                                    \
         if (h->field && (count) > 0)                                                                        \

@@ -16,6 +16,8 @@ struct kb_ctx {
     char* ws;             // caller's workspace (device)
     size_t ws_bytes;
     int* dev_status;      // device status word (owned)
+    cudaStream_t copy_stream;       // host-buffer step: copies of the late inputs (owned)
+    cudaEvent_t ev_step_begin, ev_late_inputs;
     uint64_t launches;    // kernels queued so far
     uint64_t memsets;     // memset nodes queued so far
     // optional per-call event timing

@@ -32,6 +32,8 @@ def test_fullsize_step(name):
         torch.cuda.synchronize()
         assert ctx.device_status() == 0
         assert ctx.assign_path() == 2                      # the tensor-core kernel is what the benchmark times
+        # large: the fit keeps a pre-split image of Z; contraction (D = 128): rows are split inside the kernel
+        assert ctx.assign_presplit() == (name == "large")
         got = {k: v.cpu().numpy() for k, v in t.items()}
     finally:
         ctx.close()
