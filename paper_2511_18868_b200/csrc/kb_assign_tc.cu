@@ -279,10 +279,11 @@ struct TcParams {
 // and every centroid is scaled by its own exact factor and the product is unscaled afterwards.
 __device__ __forceinline__ float pow2_scale(float m) {
     if (!(m > 0.f) || !(m < INFINITY)) return 1.f;
-    int e;
-    frexpf(m, &e);
+    // m = f 2^e with f in [0.5, 1): e is the biased exponent field minus 126 (a subnormal m has e < -126)
+    const int field = (int)((__float_as_uint(m) >> 23) & 0xffu);
+    int e = field == 0 ? -127 : field - 126;
     e = e < -100 ? -100 : (e > 100 ? 100 : e);
-    return ldexpf(1.f, -e);
+    return __uint_as_float((uint32_t)(127 - e) << 23);     // 2^-e
 }
 // (hi, lo) fp16 split of two scaled values, packed the way the tensor core reads 16-bit
 // operands: the lower k index in the low half of the 32-bit word
