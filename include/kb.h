@@ -315,7 +315,11 @@ typedef struct {
 /* The whole step on device-resident data: normalise, seed centroids, fit,
  * prune (both masks, after the final assign because the saturation mask is
  * indexed by the candidate's cluster), score and select.  Needs the workspace
- * of kb_workspace_bytes. */
+ * of kb_workspace_bytes.  Instances of at most 512 rows with D in {16, 32, 64}
+ * (and 16-byte aligned x, z, centroids) go from raw features to labels in one
+ * launch: normalisation and the gather of the initial centroids then happen
+ * inside the clustering kernel, with the results kb_normalize and
+ * kb_init_centroids would give. */
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
 
 /* The same step for a caller whose data lives in HOST memory: copies the

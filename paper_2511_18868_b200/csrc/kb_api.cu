@@ -339,7 +339,8 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
         // small instances: the whole loop in one launch, one CTA per instance
         KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_fit: D and K must be >= 1");
         TimeScope ts__(ctx, KB_T_FIT);
-        return kb_launch_fit_fused(ctx, B, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
+        return kb_launch_fit_fused(ctx, B, N, D, K, iters, z, nullptr, nullptr, nullptr, centroids, labels, dist2, inertia,
+                                   rep, counts);
     }
     if (ctx->assign_path == 0 && !kb_assign_tc_eligible(ctx, B, N, D, K) && kb_fit_coop_eligible(ctx, B, N, D, K) && z &&
         centroids && labels && (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
@@ -365,15 +366,28 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
     return s;
 }
 
-kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
-    if (!ctx || !a) return KB_ERR_INVALID_ARG;
-    KB_COMMON(ctx, a->B, a->N);
+// normalise, initial centroids, Lloyd loop: three calls, or one launch for small instances
+static kb_status step_cluster(kb_ctx* ctx, const kb_step_args* a) {
+    if (ctx->assign_path == 0 && a->iters >= 0 && kb_fit_fused_eligible(ctx, a->B, a->N, a->D, a->K) && a->x && a->z &&
+        a->init_rows && a->centroids && a->labels &&
+        (((uintptr_t)a->x | (uintptr_t)a->z | (uintptr_t)a->centroids) & 15) == 0) {
+        // at most 512 rows per instance: one CTA takes its instance from raw features to labels
+        TimeScope ts__(ctx, KB_T_FIT);
+        return kb_launch_fit_fused(ctx, a->B, a->N, a->D, a->K, a->iters, nullptr, a->x, a->z, a->init_rows, a->centroids,
+                                   a->labels, a->dist2, a->inertia, a->rep, a->counts);
+    }
     kb_status s = kb_normalize(ctx, a->B, a->N, a->D, a->x, a->z, nullptr, nullptr);
     if (s != KB_OK) return s;
     s = kb_init_centroids(ctx, a->B, a->N, a->D, a->K, a->z, a->init_rows, a->centroids);
     if (s != KB_OK) return s;
-    s = kb_cluster_fit(ctx, a->B, a->N, a->D, a->K, a->iters, a->z, a->centroids, a->labels, a->dist2, a->inertia,
-                       a->rep, a->counts);
+    return kb_cluster_fit(ctx, a->B, a->N, a->D, a->K, a->iters, a->z, a->centroids, a->labels, a->dist2, a->inertia,
+                          a->rep, a->counts);
+}
+
+kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
+    if (!ctx || !a) return KB_ERR_INVALID_ARG;
+    KB_COMMON(ctx, a->B, a->N);
+    kb_status s = step_cluster(ctx, a);
     if (s != KB_OK) return s;
     s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
                  a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count, a->bound);
@@ -500,10 +514,7 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     char* ws_saved = ctx->ws;
     size_t bytes_saved = ctx->ws_bytes;
     ctx->ws_bytes = scratch;
-    kb_status s = kb_normalize(ctx, d.B, d.N, d.D, d.x, d.z, nullptr, nullptr);
-    if (s == KB_OK) s = kb_init_centroids(ctx, d.B, d.N, d.D, d.K, d.z, d.init_rows, d.centroids);
-    if (s == KB_OK)
-        s = kb_cluster_fit(ctx, d.B, d.N, d.D, d.K, d.iters, d.z, d.centroids, d.labels, d.dist2, d.inertia, d.rep, d.counts);
+    kb_status s = step_cluster(ctx, &d);
     if (s == KB_OK && cudaStreamWaitEvent(st, ctx->ev_late_inputs, 0) != cudaSuccess)
         s = kb_fail(ctx, KB_ERR_CUDA, "kb_bandit_step_host: cudaStreamWaitEvent failed");
     if (s == KB_OK)

@@ -16,6 +16,13 @@
 //   * the final assign also produces dist2, inertia (double, fixed-order block reduction)
 //     and the representative member per cluster (64-bit shared atomicMin on (dist2, row)).
 // X is read from HBM exactly once per fit.
+//
+// The whole-step drivers hand this kernel the RAW features instead (`xraw`): the CTA then also does
+// what kb_normalize and kb_init_centroids would have done for its instance -- column statistics of
+// the staged rows (shifted by the first row, accumulated in double, threads of a column added in a
+// fixed order), z = ((x - mean_hi) - mean_lo) / sd applied in shared memory and written out once,
+// initial centroids gathered from the normalised rows -- so a small instance goes from raw
+// features to labels in one launch and its features cross HBM once in each direction.
 #include "kb_internal.cuh"
 
 namespace {
@@ -26,9 +33,10 @@ __host__ __device__ constexpr int ff_rows(int D) { return D <= 32 ? 4 : 2; }
 
 template <int D>
 __global__ void __launch_bounds__(FF_MAXROWS / ff_rows(D))
-fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
+fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, const float* xraw, float* zout,
+                 const int32_t* __restrict__ init_rows, float* __restrict__ cent,
                  int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
-                 int32_t* __restrict__ rep, int32_t* __restrict__ counts) {
+                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
     constexpr int FF_R = ff_rows(D), FF_T = FF_MAXROWS / FF_R;
     extern __shared__ __align__(16) unsigned char ff_raw[];
@@ -42,18 +50,76 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
     __shared__ double s_red[FF_MAXROWS / 64];
     __shared__ int s_scan[FF_MAXROWS / 64];
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* zb = z + (size_t)b * N * D;
+    const float* zb = (xraw ? xraw : z) + (size_t)b * N * D;
     float* cb = cent + (size_t)b * K * D;
 
-    // stage the instance (coalesced float4 reads) and the initial centroids
+    // stage the instance (coalesced float4 reads; plain loads: raw features may be normalised in place)
     for (int e = tid; e < N * (D / 4); e += FF_T) {
         const int r = e / (D / 4), q = e - r * (D / 4);
-        const float4 v = __ldg(reinterpret_cast<const float4*>(zb) + e);
+        const float4 v = *(reinterpret_cast<const float4*>(zb) + e);
         float* d = zs + (size_t)r * ZS + 4 * q;
         d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
     }
-    for (int e = tid; e < K * D / 4; e += FF_T)
-        reinterpret_cast<float4*>(cs)[e] = __ldg(reinterpret_cast<const float4*>(cb) + e);
+    __syncthreads();
+    if (xraw) {
+        // ---- column z-score of the staged rows (population standard deviation) ----------------
+        double* red = reinterpret_cast<double*>((reinterpret_cast<uintptr_t>(perm + N) + 7) & ~(uintptr_t)7);   // [FF_T][2]
+        float* st_mh = reinterpret_cast<float*>(red + 2 * FF_T);    // [D] mean, high part
+        float* st_ml = st_mh + D;                                   // [D] mean, low part
+        float* st_inv = st_ml + D;                                  // [D] 1 / standard deviation
+        constexpr int SL = FF_T / D;                                // threads per column
+        const int c = tid % D, sl = tid / D;
+        const float pivot = zs[c];                                  // first row: the same shift for every thread
+        double s1 = 0.0, s2 = 0.0;
+        for (int r = sl; r < N; r += SL) {
+            const float e = zs[(size_t)r * ZS + c] - pivot;
+            s1 += (double)e;
+            s2 += (double)e * (double)e;
+        }
+        red[2 * tid] = s1; red[2 * tid + 1] = s2;
+        __syncthreads();
+        if (tid < D) {
+            for (int q = 1; q < SL; ++q) { s1 += red[2 * (q * D + c)]; s2 += red[2 * (q * D + c) + 1]; }
+            const double ms = s1 / (double)N;
+            double var = s2 / (double)N - ms * ms;
+            if (var < 0.0) var = 0.0;
+            const double mean = (double)pivot + ms;
+            const double sd = sqrt(var);
+            const double sc = sd < 1e-12 ? 1.0 : sd;                // a constant column is only centred
+            const float mh = (float)mean;
+            st_mh[c] = mh;
+            st_ml[c] = (float)(mean - (double)mh);
+            st_inv[c] = (float)(1.0 / sc);
+        }
+        __syncthreads();
+        float* zo = zout + (size_t)b * N * D;
+        for (int e = tid; e < N * (D / 4); e += FF_T) {
+            const int r = e / (D / 4), q = e - r * (D / 4);
+            float* d = zs + (size_t)r * ZS + 4 * q;
+            float4 v;
+            v.x = ((d[0] - st_mh[4 * q]) - st_ml[4 * q]) * st_inv[4 * q];
+            v.y = ((d[1] - st_mh[4 * q + 1]) - st_ml[4 * q + 1]) * st_inv[4 * q + 1];
+            v.z = ((d[2] - st_mh[4 * q + 2]) - st_ml[4 * q + 2]) * st_inv[4 * q + 2];
+            v.w = ((d[3] - st_mh[4 * q + 3]) - st_ml[4 * q + 3]) * st_inv[4 * q + 3];
+            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+            reinterpret_cast<float4*>(zo)[e] = v;
+        }
+        __syncthreads();
+    }
+    // initial centroids: the caller's, or the normalised rows the caller names
+    for (int e = tid; e < K * D / 4; e += FF_T) {
+        float4 v;
+        const int j = e / (D / 4), q = e - j * (D / 4);
+        const int r = init_rows ? init_rows[(size_t)b * K + j] : -1;
+        if (init_rows && r >= 0 && r < N) {
+            const float* d = zs + (size_t)r * ZS + 4 * q;
+            v = make_float4(d[0], d[1], d[2], d[3]);
+        } else {
+            if (init_rows && q == 0) atomicOr(dev_status, 4);        // a row id out of range: the centroid stays as it was
+            v = *(reinterpret_cast<const float4*>(cb) + e);
+        }
+        reinterpret_cast<float4*>(cs)[e] = v;
+    }
     __syncthreads();
     bool active[FF_R];
     float x[FF_R][D];
@@ -185,7 +251,9 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, float* __
 
 size_t ff_smem(int N, int D, int K) {
     // centroids | instance (padded) | hist [K] + offs [K+1] (reused as K 64-bit keys: needs 2K ints) | perm
-    return (size_t)K * D * 4 + (size_t)N * (D + 1) * 4 + 8 + (size_t)(2 * K + 2) * 4 + (size_t)N * 2 + 16;
+    // ... | column statistics of the in-kernel normalisation: [threads][2] doubles and three floats per column
+    return (size_t)K * D * 4 + (size_t)N * (D + 1) * 4 + 8 + (size_t)(2 * K + 2) * 4 + (size_t)N * 2 + 16 +
+           8 + (size_t)(FF_MAXROWS / 2) * 16 + 3 * 64 * 4;
 }
 
 }  // namespace
@@ -196,18 +264,21 @@ bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
     return ff_smem(N, D, K) + 256 <= (size_t)ctx->max_smem_optin;
 }
 
-kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* cent,
-                              int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+// z: normalised features (input), or null with xraw (raw features, input), zout (normalised, output; may be
+// xraw itself) and init_rows (row ids of the initial centroids; null: `cent` holds them)
+kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
+                              float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
+                              float* inertia, int32_t* rep, int32_t* counts) {
     const size_t smem = ff_smem(N, D, K);
     if (D == 16) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
     } else if (D == 32) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
     } else {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, cent, labels, dist2, inertia, rep, counts);
+        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;

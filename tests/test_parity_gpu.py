@@ -346,6 +346,38 @@ def test_step_free_running(kbx, name, host_buffers):
     print(f"[{name}] label agreement with the free-running oracle: {agree:.6f}")
 
 
+@pytest.mark.parametrize("B,N,D,K", [(3, 300, 16, 5), (2, 512, 32, 16), (5, 77, 64, 9)])
+@pytest.mark.parametrize("host_buffers", [False, True])
+def test_step_small_instances_one_launch(kbx, B, N, D, K, host_buffers):
+    """Instances of at most 512 rows go from raw features to labels in ONE launch inside the whole-step drivers
+    (normalisation and the gather of the initial centroids happen in the clustering kernel).  Columns that are
+    constant, far from zero or of tiny spread must normalise as kb_normalize does; with no Lloyd iteration the
+    centroids are exactly the named rows of z."""
+    for iters in (0, 4):
+        cfg = wl.scaled(wl.CONFIGS["tiny"], B=B, N=N, D=D, K=K, S=8, iters=iters)
+        inp = wl.make_inputs(cfg, seed=B * 1000 + N)
+        x = inp["x"]
+        x[:, :, 0] = 3.25                                  # constant column: only centred
+        x[:, :, 1] = x[:, :, 1] * 0.5 + 1.0e4              # far from zero
+        x[:, :, 2] = x[:, :, 2] * 1.0e-3                   # tiny spread
+        launches0 = kbx.launch_count()[0]
+        got = run_step(kbx, cfg, inp, host_buffers)
+        launches = kbx.launch_count()[0] - launches0
+        assert kbx.device_status() == 0
+        assert launches <= 6, f"{launches} kernels: the clustering part did not run as one launch"
+        zr, _, _ = oracle.normalize(x)
+        parity.close(got["z"], zr, atol=2e-5, what="z")
+        assert np.all(got["z"][:, :, 0] == 0.0)
+        if iters == 0:
+            c0 = np.stack([got["z"][b, inp["init_rows"][b]] for b in range(B)])
+            np.testing.assert_array_equal(got["centroids"], c0)
+        chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
+        parity.labels_match(got["z"], got["centroids"], got["labels"], chk)
+        same = got["labels"] == chk["labels"]
+        parity.close(got["dist2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
+        parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia")
+
+
 @pytest.mark.parametrize("N,D,K,iters", [(16384, 32, 64, 20), (5000, 16, 8, 7), (1025, 64, 100, 3), (40000, 32, 17, 4),
                                          (2048, 32, 64, 0)])
 def test_cluster_fit_cooperative(kbx, N, D, K, iters):
