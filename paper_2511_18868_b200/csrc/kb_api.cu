@@ -384,12 +384,24 @@ static kb_status step_cluster(kb_ctx* ctx, const kb_step_args* a) {
                           a->rep, a->counts);
 }
 
+// prune, score and select: two calls, or one launch for small instances
+static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a);
+
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
     if (!ctx || !a) return KB_ERR_INVALID_ARG;
     KB_COMMON(ctx, a->B, a->N);
     kb_status s = step_cluster(ctx, a);
     if (s != KB_OK) return s;
-    s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
+    return step_tail(ctx, a);
+}
+
+static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a) {
+    if (kb_step_tail_small_eligible(ctx, a)) {
+        // at most 1024 candidates per instance: one CTA prunes, scores and selects for its instance
+        TimeScope ts__(ctx, KB_T_SCORE);
+        return kb_launch_step_tail_small(ctx, a);
+    }
+    kb_status s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
                  a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count, a->bound);
     if (s != KB_OK) return s;
     return kb_score_select(ctx, a->B, a->N, a->K, a->S, a->score, a->labels, a->dist2, a->pulls, a->reward_sum,
@@ -517,13 +529,7 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     kb_status s = step_cluster(ctx, &d);
     if (s == KB_OK && cudaStreamWaitEvent(st, ctx->ev_late_inputs, 0) != cudaSuccess)
         s = kb_fail(ctx, KB_ERR_CUDA, "kb_bandit_step_host: cudaStreamWaitEvent failed");
-    if (s == KB_OK)
-        s = kb_prune(ctx, d.B, d.N, d.S, d.K, d.R, d.flops, d.bytes, d.peak_flops, d.peak_bw, d.t_incumbent, d.t_cur,
-                     d.labels, d.hsig, d.target, d.theta_sat, d.keep, d.kept_count, d.bound);
-    if (s == KB_OK)
-        s = kb_score_select(ctx, d.B, d.N, d.K, d.S, d.score, d.labels, d.dist2, d.pulls, d.reward_sum, d.keep, d.bound,
-                            d.t, d.cl_pulls, d.cl_mean, d.cl_index, d.arm_index, d.best_arm, d.best_val,
-                            d.best_cluster_arm);
+    if (s == KB_OK) s = step_tail(ctx, &d);
     ctx->ws = ws_saved;
     ctx->ws_bytes = bytes_saved;
     if (s != KB_OK) {

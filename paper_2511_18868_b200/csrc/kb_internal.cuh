@@ -88,6 +88,8 @@ size_t kb_ws_need_normalize(int B, int N, int D);
 size_t kb_ws_need_assign(int B, int N, int D, int K);
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
 size_t kb_ws_need_zsplit(int B, int N, int D, int K);
+bool kb_step_tail_small_eligible(const kb_ctx* ctx, const kb_step_args* a);
+kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* a);
 kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z);
 void kb_zsplit_forget(kb_ctx* ctx);
 bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K);
@@ -173,6 +175,12 @@ __device__ __forceinline__ double kb_warp_sum(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+// a / d with r = 1/d (correctly rounded): one residual step on the first estimate
+__device__ __forceinline__ float kb_div_by(float a, float d, float r) {
+    const float q0 = a * r;
+    const float e = fmaf(-q0, d, a);
+    return fmaf(e, r, q0);     // d = 0 or a non-finite operand gives NaN here, which the callers map like 0/0
 }
 // monotone map float -> uint32 (larger float <=> larger uint)
 __device__ __forceinline__ uint32_t kb_orderable(float f) {

@@ -19,12 +19,6 @@ namespace {
 constexpr int PR_T = 128;
 constexpr int PV_T = 256;
 
-// a / d with r = 1/d (correctly rounded): one residual step on the first estimate
-__device__ __forceinline__ float div_by(float a, float d, float r) {
-    const float q0 = a * r;
-    const float e = fmaf(-q0, d, a);
-    return fmaf(e, r, q0);     // d = 0 or a non-finite operand gives NaN here, which the callers map like 0/0
-}
 
 __global__ void __launch_bounds__(PV_T)
 prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ flops, const float* __restrict__ bytes,
@@ -93,11 +87,11 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
             const float rT = 1.f / Tk[u];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float tlb = fmaxf(div_by(F[u], P[k], rP[k]), div_by(Q[u], W[k], rW[k]));
+                const float tlb = fmaxf(kb_div_by(F[u], P[k], rP[k]), kb_div_by(Q[u], W[k], rW[k]));
                 bool ok = tlb < tinc;
                 if (sat) ok = ok && (__ldg(h + tg[k]) < theta);
                 if (ok) bits |= 1u << (4 * q + k);
-                float v = div_by(Tk[u] - tlb, Tk[u], rT);
+                float v = kb_div_by(Tk[u] - tlb, Tk[u], rT);
                 v = v > 0.f ? v : 0.f;       // also maps NaN (0/0) to 0, as the definition does
                 g[k] = v < 1.f ? v : 1.f;
             }

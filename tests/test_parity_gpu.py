@@ -346,15 +346,16 @@ def test_step_free_running(kbx, name, host_buffers):
     print(f"[{name}] label agreement with the free-running oracle: {agree:.6f}")
 
 
-@pytest.mark.parametrize("B,N,D,K", [(3, 300, 16, 5), (2, 512, 32, 16), (5, 77, 64, 9)])
+@pytest.mark.parametrize("B,N,D,K,S", [(3, 300, 16, 5, 8), (2, 512, 32, 16, 32), (5, 77, 64, 9, 4), (4, 200, 32, 7, 16)])
 @pytest.mark.parametrize("host_buffers", [False, True])
-def test_step_small_instances_one_launch(kbx, B, N, D, K, host_buffers):
+def test_step_small_instances_one_launch(kbx, B, N, D, K, S, host_buffers):
     """Instances of at most 512 rows go from raw features to labels in ONE launch inside the whole-step drivers
-    (normalisation and the gather of the initial centroids happen in the clustering kernel).  Columns that are
-    constant, far from zero or of tiny spread must normalise as kb_normalize does; with no Lloyd iteration the
-    centroids are exactly the named rows of z."""
+    (normalisation and the gather of the initial centroids happen in the clustering kernel), and a second launch
+    prunes, scores and selects.  Columns that are constant, far from zero or of tiny spread must normalise as
+    kb_normalize does; with no Lloyd iteration the centroids are exactly the named rows of z; keep bits, cluster
+    tables, per-arm indices and both selections must be what the oracle derives from the GPU's own labels."""
     for iters in (0, 4):
-        cfg = wl.scaled(wl.CONFIGS["tiny"], B=B, N=N, D=D, K=K, S=8, iters=iters)
+        cfg = wl.scaled(wl.CONFIGS["tiny"], B=B, N=N, D=D, K=K, S=S, iters=iters)
         inp = wl.make_inputs(cfg, seed=B * 1000 + N)
         x = inp["x"]
         x[:, :, 0] = 3.25                                  # constant column: only centred
@@ -364,7 +365,7 @@ def test_step_small_instances_one_launch(kbx, B, N, D, K, host_buffers):
         got = run_step(kbx, cfg, inp, host_buffers)
         launches = kbx.launch_count()[0] - launches0
         assert kbx.device_status() == 0
-        assert launches <= 6, f"{launches} kernels: the clustering part did not run as one launch"
+        assert launches == 2, f"{launches} kernels: the step did not run as two launches"
         zr, _, _ = oracle.normalize(x)
         parity.close(got["z"], zr, atol=2e-5, what="z")
         assert np.all(got["z"][:, :, 0] == 0.0)
@@ -376,6 +377,21 @@ def test_step_small_instances_one_launch(kbx, B, N, D, K, host_buffers):
         same = got["labels"] == chk["labels"]
         parity.close(got["dist2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
         parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia")
+        p_chk = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+                             got["labels"], inp["hsig"], inp["target"], 75.0, want_bound=True, want_margin=True)
+        keep = got["keep"].view(np.uint32)
+        ties = parity.keep_match(keep, p_chk, S)
+        pop = sum(int(v).bit_count() for v in keep.reshape(-1))
+        assert int(got["kept_count"].view(np.uint32).sum()) == pop and abs(pop - int(p_chk["kept_count"].sum())) <= ties
+        parity.close(got["bound"], p_chk["bound"], atol=1e-6, what="bound")
+        s_chk = oracle.score_select(got["labels"], got["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], K,
+                                    keep=keep, c=2.0, lipschitz_L=float(inp["lipschitz_L"]))
+        parity.close(got["cl_pulls"], s_chk["cl_pulls"], atol=1e-6, what="cl_pulls")
+        parity.close(got["cl_mean"], s_chk["cl_mean"], atol=1e-6, what="cl_mean")
+        parity.close(got["cl_index"], s_chk["cl_index"], atol=1e-6, what="cl_index")
+        parity.close(got["arm_index"], s_chk["arm_index"], atol=1e-6, what="arm_index")
+        parity.select_match(got["best_arm"], got["best_val"], s_chk, s_chk["arm_index"])
+        parity.cluster_select_match(got["best_cluster_arm"], s_chk, s_chk["cl_index"])
 
 
 @pytest.mark.parametrize("N,D,K,iters", [(16384, 32, 64, 20), (5000, 16, 8, 7), (1025, 64, 100, 3), (40000, 32, 17, 4),
