@@ -91,12 +91,13 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
     float* rbest = reinterpret_cast<float*>(parg + P * CAP);        // [CAP] best over the parts
     int* rarg = reinterpret_cast<int*>(rbest + CAP);                // [CAP]
     int* hist = rarg + CAP;                                         // [K] this CTA's rows per cluster, then the totals
-    float* ssum = reinterpret_cast<float*>(hist + K);               // [K][D] this CTA's column sums per cluster
+    // [K][D] this CTA's column sums per cluster (16-byte aligned: read as float4)
+    float* ssum = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(hist + K) + 15) & ~(uintptr_t)15);
     __shared__ double s_red[CF_T / 32];
     const int G = gridDim.x, g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows_per = (N + G - 1) / G;
     const int r0 = g * rows_per, rows = max(0, min(N, r0 + rows_per) - r0);      // rows <= CAP (host)
-    const int KD = K * D, TS = KD + K;                              // floats per table
+    const int KD = K * D, TS = KD + ((K + 3) & ~3);                 // floats per table (a multiple of four: every copy 16-byte aligned)
     const int slot = tid % SLOTS, part = tid / SLOTS;
     const int kper = (K + P - 1) / P;
     const int jlo = min(K, part * kper), jhi = min(K, jlo + kper);
@@ -190,10 +191,12 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
             if (d == 0) atomicAdd(hist + a, 1);
         }
         __syncthreads();
-        for (int e = tid; e < KD; e += CF_T) {
-            const int j = e / D, n = hist[j];
+        for (int e4 = tid; e4 < KD / 4; e4 += CF_T) {               // four columns per reduction: a quarter of the operations
+            const int e = 4 * e4, j = e / D, n = hist[j];
             if (n > 0) {
-                atomicAdd(tab + e, ssum[e]);
+                const float4 v = *reinterpret_cast<const float4*>(ssum + e);
+                asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                             ::"l"(tab + e), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
                 if (e - j * D == 0) atomicAdd(reinterpret_cast<int*>(tab + KD) + j, n);
             }
         }
@@ -306,7 +309,7 @@ int cf_slots(int rows_per) { return rows_per <= 128 ? 64 : (rows_per <= 256 ? 12
 size_t cf_smem(int rows_per, int D, int K) {
     const size_t cap = (size_t)cf_slots(rows_per) * CF_R, P = cf_threads(D) / cf_slots(rows_per);
     // centroids | rows (padded) | per-part best and argument | per-row best and argument | hist | column sums
-    return (size_t)K * D * 4 + cap * (D + 1) * 4 + P * cap * 8 + cap * 8 + (size_t)K * 4 + (size_t)K * D * 4 + 32;
+    return (size_t)K * D * 4 + cap * (D + 1) * 4 + P * cap * 8 + cap * 8 + (size_t)K * 4 + (size_t)K * D * 4 + 64;
 }
 int cf_ctas(const kb_ctx* ctx, int N) {
     long cap = ((long)N + 63) / 64;                     // at least 64 rows per CTA
@@ -314,7 +317,7 @@ int cf_ctas(const kb_ctx* ctx, int N) {
     return (int)(G < 1 ? 1 : G);
 }
 size_t cf_scratch(int D, int K) {
-    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)K * 8) + kb_align256((size_t)3 * CF_NC * (K * D + K) * 4) + 256;
+    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)K * 8) + kb_align256((size_t)3 * CF_NC * (K * D + ((K + 3) & ~3)) * 4) + 256;
 }
 
 }  // namespace
@@ -344,7 +347,7 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
     CoopScratch* sc = reinterpret_cast<CoopScratch*>(ws);
     unsigned long long* rep_key = reinterpret_cast<unsigned long long*>(ws + kb_align256(sizeof(CoopScratch)));
     float* table = reinterpret_cast<float*>(reinterpret_cast<char*>(rep_key) + kb_align256((size_t)K * 8));
-    const size_t zbytes = (size_t)(reinterpret_cast<char*>(table) - ws) + kb_align256((size_t)CF_NC * (K * D + K) * 4);
+    const size_t zbytes = (size_t)(reinterpret_cast<char*>(table) - ws) + kb_align256((size_t)CF_NC * (K * D + ((K + 3) & ~3)) * 4);
     kb_launch(coop_zero_kernel, (unsigned)((zbytes / 16 + 255) / 256), 256, 0, ctx->stream, zbytes / 16,
               reinterpret_cast<uint4*>(ws));
     KB_LAUNCH_CHECK(ctx, "coop_zero_kernel");
