@@ -169,7 +169,7 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     size_t need = 256;
     need = max_sz(need, kb_ws_need_normalize(B, N, D));
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
-    need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_zsplit(B, N, D, K));
+    need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K));
     *out = need;
     return KB_OK;
 }
@@ -350,18 +350,28 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
     }
     // Tensor-core assignments of the same matrix, several times over: split Z into its fp16 pieces once and let
     // every assignment multiply out of that image (kept behind the scratch of the calls below).
+    // Behind the scratch of the calls below: the accumulators of the loop's updates, then the image.
     kb_status s = KB_OK;
-    const size_t zneed = kb_ws_need_zsplit(B, N, D, K), zoff = fit_scratch_bytes(B, N, D, K);
-    if (iters >= 2 && N > 0 && z && zneed > 0 && ctx->ws_bytes >= zoff + zneed && ctx->assign_path != 1 &&
-        (ctx->assign_path >= 2 || kb_assign_tc_eligible(ctx, B, N, D, K))) {
+    const size_t aoff = fit_scratch_bytes(B, N, D, K), aneed = kb_ws_need_fit_acc(B, D, K);
+    const size_t zneed = kb_ws_need_zsplit(B, N, D, K), zoff = aoff + aneed;
+    const bool tensor = N > 0 && z && ctx->assign_path != 1 &&
+                        (ctx->assign_path >= 2 ? kb_assign_tc_supported(ctx, B, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
+    if (tensor && iters >= 2 && zneed > 0 && ctx->ws_bytes >= zoff + zneed) {
         TimeScope ts__(ctx, KB_T_ASSIGN);
         s = kb_zsplit_prepare(ctx, ctx->ws + zoff, B, N, D, K, z);
+    }
+    if (tensor && iters >= 1 && ctx->ws_bytes >= aoff + aneed) {
+        // every assignment of the loop clears these in its fix-up kernel, the update that follows adds into them
+        ctx->fit_acc = ctx->ws + aoff;
+        ctx->fit_acc_bytes = aneed;
+        ctx->fit_acc_clean = 0;
     }
     for (int it = 0; it < iters && s == KB_OK; ++it) {
         s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
         if (s == KB_OK) s = kb_cluster_update(ctx, B, N, D, K, z, labels, centroids, counts);
     }
     if (s == KB_OK) s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+    ctx->fit_acc = nullptr;
     kb_zsplit_forget(ctx);
     return s;
 }

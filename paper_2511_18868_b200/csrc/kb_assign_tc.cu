@@ -1328,8 +1328,12 @@ assign_fixup_pairs_kernel(int N, int D, int K, const float* __restrict__ z, cons
 __global__ void __launch_bounds__(FX_T)
 assign_fixup_kernel(int N, int D, int K, const float* __restrict__ z, const float* __restrict__ cent,
                     const int* __restrict__ flag_count, const int2* __restrict__ pair_rows,
-                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels) {
+                    const int32_t* __restrict__ full_rows, int32_t* __restrict__ labels, uint4* __restrict__ zero,
+                    size_t zero_n16) {
     kb_grid_dependency_wait();
+    // inside a fit: the accumulators of the centroid update that follows are cleared here (one launch fewer)
+    for (size_t i = (size_t)blockIdx.x * FX_T + threadIdx.x; i < zero_n16; i += (size_t)gridDim.x * FX_T)
+        zero[i] = make_uint4(0u, 0u, 0u, 0u);
     if (pair_rows) fixup_pairs(gridDim.x, N, D, K, z, cent, flag_count, pair_rows, labels);
     extern __shared__ __align__(16) float fx[];            // [FX_MAXROWS][D] rows | [FX_T][D+4] centroid tile
     __shared__ float red_v[FX_MAXROWS][FX_T / 32];
@@ -1563,7 +1567,9 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     const int fblocks = (int)(((size_t)ctx->max_smem_optin / (fsmem + 2048)) < 1 ? 1 : ((size_t)ctx->max_smem_optin / (fsmem + 2048)));
     KB_SMEM_OPTIN(ctx, assign_fixup_kernel, fsmem);
     kb_launch(assign_fixup_kernel, (fblocks > 4 ? 4 : fblocks) * ctx->sm_count, FX_T, fsmem, ctx->stream, N, D, K, z, c, flag_count,
-              one_launch ? pair_rows : static_cast<int2*>(nullptr), full_rows, labels);
+              one_launch ? pair_rows : static_cast<int2*>(nullptr), full_rows, labels,
+              reinterpret_cast<uint4*>(ctx->fit_acc), ctx->fit_acc ? ctx->fit_acc_bytes / 16 : (size_t)0);
+    if (ctx->fit_acc) ctx->fit_acc_clean = 1;
     KB_LAUNCH_CHECK(ctx, "assign_fixup_kernel");
     if (flagged) {   // two counters: rows checked against the runner-up, rows re-evaluated against all centroids
         KB_CUDA(ctx, cudaMemcpyAsync(flagged, flag_count, 2 * sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));

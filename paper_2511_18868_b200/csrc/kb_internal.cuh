@@ -35,6 +35,11 @@ struct kb_ctx {
     int zs_B, zs_N, zs_D;
     const unsigned char* zs_img;
     const float* zs_info;
+    // accumulators (sums, then counts) that a running tensor-path fit sets aside for its updates, behind the
+    // scratch of the calls: the assignment's fix-up kernel clears them, so the update needs no clearing launch
+    char* fit_acc;               // null outside such a fit
+    size_t fit_acc_bytes;
+    int fit_acc_clean;           // 1: cleared since the last update used them
     char err[256];
 };
 #define KB_EV_PAIRS 4096
@@ -108,6 +113,7 @@ kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
                               float* inertia, int32_t* rep, int32_t* counts);
 size_t kb_ws_need_update(int B, int N, int D, int K);
+size_t kb_ws_need_fit_acc(int B, int D, int K);
 size_t kb_ws_need_score(int B, int N, int K, int S);
 #define KB_NORM_MAXG 1024
 int kb_norm_blocks_per_instance(int B, int N);

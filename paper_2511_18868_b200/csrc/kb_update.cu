@@ -306,6 +306,11 @@ size_t kb_ws_need_update(int B, int N, int D, int K) {
     return need;
 }
 
+// A fit's own accumulators: sums [B][K][D], then counts [B][K].
+size_t kb_ws_need_fit_acc(int B, int D, int K) {
+    return kb_align256((size_t)B * K * D * sizeof(float)) + kb_align256((size_t)B * K * sizeof(int));
+}
+
 kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* labels,
                            float* c, int32_t* counts) {
     if (B == 0) return KB_OK;
@@ -339,11 +344,18 @@ kb_status kb_launch_update(kb_ctx* ctx, int B, int N, int D, int K, const float*
         KB_LAUNCH_CHECK(ctx, "update_table_finalize_kernel");
         return KB_OK;
     }
-    float* g_sums = reinterpret_cast<float*>(ctx->ws);
-    int* g_counts = reinterpret_cast<int*>(ctx->ws + kb_align256((size_t)B * K * D * sizeof(float)));
-    kb_launch(update_zero_kernel, (unsigned)((need / 16 + 255) / 256), 256, 0, ctx->stream, need / 16,
-              reinterpret_cast<uint4*>(ctx->ws));
-    KB_LAUNCH_CHECK(ctx, "update_zero_kernel");
+    // inside a tensor-path fit the accumulators are the fit's own, already cleared by the assignment before
+    const bool own = ctx->fit_acc && ctx->fit_acc_clean && ctx->fit_acc_bytes == kb_ws_need_fit_acc(B, D, K);
+    char* acc = own ? ctx->fit_acc : ctx->ws;
+    float* g_sums = reinterpret_cast<float*>(acc);
+    int* g_counts = reinterpret_cast<int*>(acc + kb_align256((size_t)B * K * D * sizeof(float)));
+    if (own) {
+        ctx->fit_acc_clean = 0;
+    } else {
+        kb_launch(update_zero_kernel, (unsigned)((need / 16 + 255) / 256), 256, 0, ctx->stream, need / 16,
+                  reinterpret_cast<uint4*>(ctx->ws));
+        KB_LAUNCH_CHECK(ctx, "update_zero_kernel");
+    }
 
     // CTAs per instance: about two per SM in total, each with at most UP_MAXROWS rows and
     // enough rows to be worth a sort
