@@ -618,6 +618,40 @@ def test_assign_tensor_path_value_ranges(kbx, path, scale):
     print(f"[tc ranges path={path} scale={scale:g}] near-ties={ties}")
 
 
+@pytest.mark.parametrize("scale", [1e-6, 1.0, 3e4], ids=["tiny", "unit", "huge"])
+def test_cluster_fit_presplit_value_ranges(kbx, scale):
+    """The same value ranges through a fit, whose assignments multiply out of the pre-split image of Z (rows scaled
+    once, before the centroids' scale of an iteration is known): outlier rows, zero rows, tiny rows and a zero
+    centroid must still end with labels that are optimal for the returned centroids."""
+    B, N, D, K = 1, 6000, 64, 256
+    cfg = wl.scaled(wl.CONFIGS["large"], B=B, N=N, D=D, K=K, components=96, S=2)
+    z, _, _ = oracle.normalize(wl.make_inputs(cfg, seed=17)["x"])
+    rng = np.random.default_rng(5)
+    c0 = z[:, rng.choice(N, K, replace=False)].copy()
+    z = z.copy()
+    z[0, 10:20] *= 1e5
+    z[0, 20:24] *= 1e9
+    z[0, 30:34] = 0.0
+    z[0, 40:44] *= 1e-7
+    c0[0, 7] = 0.0
+    z, c0 = (z * np.float32(scale)).astype(np.float32), (c0 * np.float32(scale)).astype(np.float32)
+    ws(kbx, B, N, D, K, 1)
+    for iters in (2, 3):
+        c = dev(c0.copy())
+        labels, d2, inertia = empty((B, N), torch.int32), empty((B, N)), empty((B,))
+        counts = empty((B, K), torch.int32)
+        kbx.cluster_fit(dev(z), c, labels, iters, dist2=d2, inertia=inertia, counts=counts)
+        assert kbx.assign_path() == 2 and kbx.assign_presplit()
+        assert kbx.device_status() == 0
+        cg, got = host(c), host(labels)
+        assert np.all(np.isfinite(cg)) and host(counts).sum() == N
+        chk = oracle.cluster_assign(z, cg, want_margins=True)
+        ties = parity.labels_match(z, cg, got, chk)
+        same = got == chk["labels"]
+        parity.close(host(d2)[same], chk["dist2"][same], atol=1e-7 * scale * scale, what="dist2")
+        print(f"[presplit ranges scale={scale:g} iters={iters}] near-ties={ties}")
+
+
 def test_step_uses_tensor_path_when_eligible(kbx):
     cfg = wl.scaled(wl.CONFIGS["large"], N=8192 + 37, iters=2)
     inp = wl.make_inputs(cfg)
