@@ -26,18 +26,29 @@
 //     by every CTA (no multicast of any kind).  The whole image stays resident when it fits.
 //   * accumulators: two 128 x 128 fp32 buffers in TMEM; the epilogue warps read one with
 //     tcgen05.ld while the MMA fills the other.
-//   * epilogue: every value becomes an integer key (fp32 bits, low 7 bits replaced by the column
-//     index), so integer min/max rank value and index together; per row the three smallest keys
+//   * epilogue: every value becomes an integer key that carries its column (tf32 split: the fp32 bits
+//     with the low 7 bits replaced; fp16 split: a 22-bit fixed-point distance times KQ_MUL plus the
+//     column), so integer min/max rank value and index together; per row the three smallest keys
 //     are kept across all centroid tiles.  A row whose runner-up lies inside the error bound of
 //     the split product is queued and decided in the exact direct form by a fix-up kernel (two
 //     candidates: a warp compares them; three or more: all K are re-evaluated), so labels follow
 //     the fp32 direct-form distances wherever it matters.
 //
-// Roles in a 448-thread persistent CTA (one per SM):
-//   warps 0-3   A producers  (bulk copy of the next Z tile -> split -> TMEM)
+//   * pre-split image (template parameter APRE; inside kb_cluster_fit, fp16 split, D <= 64).  A fit assigns
+//     the same Z many times, so it converts Z to its fp16 pieces ONCE (tc_prep_z_f16_kernel: per 128-row
+//     tile a contiguous image of swizzled rows plus ||z||^2 and s_z per row) and its assignments run this
+//     kernel with APRE: a fifth role brings a whole tile with one bulk copy (evict-first in L2) into a ring
+//     of three, the producers only move their row from shared to tensor memory and form its constant-term
+//     operand, and -- two tiles later -- take the row's candidates over from the epilogue through shared
+//     memory, merge them, write the label and queue near-ties, so the epilogue goes straight on.
+//
+// Roles in a 448-thread persistent CTA (480 with APRE; one CTA per SM):
+//   warps 0-3   A producers  (bulk copy of the next Z tile -> split -> TMEM; APRE: row image -> TMEM,
+//                             constant terms, the rows' results two tiles behind)
 //   warps 4-11  epilogue     (TMEM -> registers -> keys -> argmin; two warps per lane quarter)
 //   warp  12    MMA issuer   (one elected lane), owns the TMEM allocation
 //   warp  13    B loader     (one elected lane)
+//   warp  14    A loader     (APRE only; one elected lane)
 // The roles meet only at mbarriers (one arrival per warp).  Every wait is bounded and suspends
 // the waiting thread between polls; on expiry the CTA raises an abort flag, all roles drain,
 // copies in flight are awaited, TMEM is released and the device status word reports a timeout.
