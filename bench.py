@@ -172,35 +172,85 @@ def job_value(world: int, arms: int, ms_per_step: float) -> float:
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML (read-only) every 10 ms in a thread."""
+    """Samples SM clock and throttle reasons (read-only) during the timed region: NVML every 10 ms in a thread,
+    addressed by the CUDA device's UUID (the NVML index of a GPU need not be its CUDA index); when NVML cannot be
+    used, `nvidia-smi --query-gpu` in a loop instead.  Whatever went wrong is reported, never swallowed."""
     REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+    SMI_FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+    def __init__(self, index: int, uuid: str | None = None):
+        self.index, self.uuid = index, uuid
+        self.samples, self.reasons, self.max_mhz, self.source, self.error = [], set(), None, None, None
         self._stop, self._thread = None, None
 
-    def _run(self):
+    def _nvml_open(self):
+        """NVML start-up (slow the first time on a fresh machine): done before the timed region, not inside it."""
         import pynvml
-        try:
-            pynvml.nvmlInit()
-            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
-            while not self._stop.is_set():
-                self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+        pynvml.nvmlInit()
+        h = None
+        if self.uuid:
+            for name in (self.uuid, self.uuid.encode()):
                 try:
-                    mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                    h = pynvml.nvmlDeviceGetHandleByUUID(name)
+                    break
                 except Exception:
-                    mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-                for name, bit in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-                self._stop.wait(0.01)
-        except Exception:
-            pass
+                    h = None
+        if h is None:
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        self.source = "nvml"
+        self._h = h
+
+    def _nvml_loop(self):
+        import pynvml
+        h = self._h
+        while not self._stop.is_set():
+            self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+            try:
+                mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+            except Exception:
+                mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+            for name, bit in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+            self._stop.wait(0.01)
+
+    def _smi_once(self):
+        import subprocess
+        sel = ["-i", self.uuid] if self.uuid else ["-i", str(self.index)]
+        out = subprocess.run(["nvidia-smi"] + sel + ["--query-gpu=" + self.SMI_FIELDS, "--format=csv,noheader,nounits"],
+                             capture_output=True, text=True, timeout=10).stdout.strip().splitlines()
+        f = [x.strip() for x in out[0].split(",")]
+        self.samples.append(float(f[0]))
+        self.max_mhz = float(f[1])
+        for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], f[2:6]):
+            if val.lower().startswith("active"):
+                self.reasons.add(name)
+
+    def _run(self):
+        if self._h is not None:
+            try:
+                self._nvml_loop()
+                return
+            except Exception as e:                   # NVML stopped answering: say so and fall back
+                self.error = f"nvml: {type(e).__name__}: {e}"
+        try:
+            self.source = "nvidia-smi"
+            while not self._stop.is_set():
+                self._smi_once()
+                self._stop.wait(0.05)
+        except Exception as e:
+            self.error = (self.error or "") + f"; nvidia-smi: {type(e).__name__}: {e}"
 
     def start(self):
         import threading
         self._stop = threading.Event()
+        self._h = None
+        try:
+            self._nvml_open()
+        except Exception as e:                       # NVML unusable here: say so, nvidia-smi takes over
+            self.error = f"nvml: {type(e).__name__}: {e}"
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
         time.sleep(0.05)
@@ -210,11 +260,14 @@ class ClockSampler:
         if self._thread is None:
             return out
         self._stop.set()
-        self._thread.join(timeout=2)
+        self._thread.join(timeout=15)
         if self.samples:
             out.update(sm_mhz=float(np.median(self.samples)), sm_min_mhz=float(min(self.samples)),
                        sm_max_mhz=self.max_mhz, samples=len(self.samples))
         out["reasons"] = sorted(self.reasons)
+        out["source"] = self.source
+        if self.error:
+            out["error"] = self.error
         return out
 
 
@@ -258,7 +311,11 @@ def run_ours(args, cfg):
     for _ in range(args.warmup):
         flush.zero_()
         ctx.bandit_step(dims, params, dev_t)
-    sampler = ClockSampler(local)
+    try:                                            # NVML addresses GPUs by UUID, whatever CUDA_VISIBLE_DEVICES says
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        gpu_uuid = None
+    sampler = ClockSampler(local, gpu_uuid)
     barrier()
     sampler.start()
     k0, m0 = ctx.launch_count()
