@@ -319,7 +319,9 @@ typedef struct {
  * (and 16-byte aligned x, z, centroids) go from raw features to labels in one
  * launch: normalisation and the gather of the initial centroids then happen
  * inside the clustering kernel, with the results kb_normalize and
- * kb_init_centroids would give.  Instances of at most 1024 candidates with S in
+ * kb_init_centroids would give; a single instance that kb_cluster_fit would
+ * run as one cooperative launch does the same there (column statistics across
+ * all its CTAs, one more grid barrier).  Instances of at most 1024 candidates with S in
  * {4, 8, 16, 32}, K*S <= 8192 and 16-byte aligned per-arm arrays are pruned,
  * scored and selected by one more launch (one CTA per instance, the arithmetic
  * of kb_prune and kb_score_select). */

@@ -346,7 +346,8 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
         centroids && labels && (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
         // one mid-sized instance: the whole loop in one cooperative launch, the rows resident on chip
         TimeScope ts__(ctx, KB_T_FIT);
-        return kb_launch_fit_coop(ctx, N, D, K, iters, z, centroids, labels, dist2, inertia, rep, counts);
+        return kb_launch_fit_coop(ctx, N, D, K, iters, z, nullptr, nullptr, nullptr, centroids, labels, dist2, inertia, rep,
+                                  counts);
     }
     // Tensor-core assignments of the same matrix, several times over: split Z into its fp16 pieces once and let
     // every assignment multiply out of that image (kept behind the scratch of the calls below).
@@ -385,6 +386,14 @@ static kb_status step_cluster(kb_ctx* ctx, const kb_step_args* a) {
         TimeScope ts__(ctx, KB_T_FIT);
         return kb_launch_fit_fused(ctx, a->B, a->N, a->D, a->K, a->iters, nullptr, a->x, a->z, a->init_rows, a->centroids,
                                    a->labels, a->dist2, a->inertia, a->rep, a->counts);
+    }
+    if (ctx->assign_path == 0 && a->iters >= 0 && !kb_assign_tc_eligible(ctx, a->B, a->N, a->D, a->K) &&
+        kb_fit_coop_eligible(ctx, a->B, a->N, a->D, a->K) && a->x && a->z && a->init_rows && a->centroids && a->labels &&
+        (((uintptr_t)a->x | (uintptr_t)a->z | (uintptr_t)a->centroids) & 15) == 0) {
+        // one mid-sized instance: one cooperative launch takes it from raw features to labels
+        TimeScope ts__(ctx, KB_T_FIT);
+        return kb_launch_fit_coop(ctx, a->N, a->D, a->K, a->iters, nullptr, a->x, a->z, a->init_rows, a->centroids, a->labels,
+                                  a->dist2, a->inertia, a->rep, a->counts);
     }
     kb_status s = kb_normalize(ctx, a->B, a->N, a->D, a->x, a->z, nullptr, nullptr);
     if (s != KB_OK) return s;

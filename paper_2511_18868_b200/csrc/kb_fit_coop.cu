@@ -21,6 +21,14 @@
 // is kept in CF_NC copies (CTA g adds into copy g % CF_NC and the readers add the copies up): all
 // CTAs reduce into the same few lines, and the reductions on one line are serviced one at a time.
 // Z is read from HBM exactly once per fit.
+//
+// The whole-step drivers hand this kernel the RAW features instead (`xraw`): it then also does what
+// kb_normalize and kb_init_centroids would have done.  Every CTA adds up its rows per column (shifted
+// by the instance's first row, in double) and stores the partial sums; after one more grid barrier
+// every CTA adds all partials in CTA order (so all of them, and every run, get the same statistics),
+// normalises its rows in shared memory with kb_normalize's expression and writes z once.  The rows
+// that seed the centroids are fetched raw BEFORE that barrier (z may overwrite x in place) and
+// normalised with the same expression afterwards.
 #include "kb_internal.cuh"
 
 namespace {
@@ -74,7 +82,9 @@ __device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, un
 // threads of a slot each scan a contiguous P-th of the centroids, so a CTA with few rows still fills its SM.
 template <int D, int SLOTS>
 __global__ void __launch_bounds__(cf_threads(D))
-fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __restrict__ cent,
+fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, const float* xraw, float* zout,
+                const int32_t* __restrict__ init_rows, double* __restrict__ npart /* [G][D][2] column sums per CTA */,
+                float* __restrict__ cent,
                 int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, CoopScratch* __restrict__ sc,
                 float* __restrict__ table /* [3][CF_NC][K*D + K] sums then counts (as int) */,
@@ -102,17 +112,91 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
     const int kper = (K + P - 1) / P;
     const int jlo = min(K, part * kper), jhi = min(K, jlo + kper);
 
-    // stage this CTA's rows (coalesced float4 reads) and the initial centroids
-    const float* zb = z + (size_t)r0 * D;
+    // stage this CTA's rows (coalesced float4 reads; plain loads: raw features may be normalised in place)
+    // and the initial centroids: the caller's, or the (still raw) rows the caller names
+    const unsigned epoch0 = xraw ? 1u : 0u;                         // barriers taken before the Lloyd loop
+    const float* zb = (xraw ? xraw : z) + (size_t)r0 * D;
     for (int e = tid; e < rows * (D / 4); e += CF_T) {
         const int r = e / (D / 4), q = e - r * (D / 4);
-        const float4 v = __ldg(reinterpret_cast<const float4*>(zb) + e);
+        const float4 v = *(reinterpret_cast<const float4*>(zb) + e);
         float* d = zs + (size_t)r * ZS + 4 * q;
         d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
     }
-    for (int e = tid; e < KD / 4; e += CF_T)
-        reinterpret_cast<float4*>(cs)[e] = __ldg(reinterpret_cast<const float4*>(cent) + e);
+    for (int e = tid; e < KD / 4; e += CF_T) {
+        const int j = e / (D / 4), q = e - j * (D / 4);
+        const int r = (xraw && init_rows) ? init_rows[j] : -1;
+        if (xraw && init_rows && (r < 0 || r >= N)) {
+            if (q == 0 && g == 0) atomicOr(dev_status, 4);           // a row id out of range: the centroid stays as it was
+        }
+        reinterpret_cast<float4*>(cs)[e] = (r >= 0 && r < N) ? *(reinterpret_cast<const float4*>(xraw + (size_t)r * D) + q)
+                                                             : __ldg(reinterpret_cast<const float4*>(cent) + e);
+    }
     __syncthreads();
+    if (xraw) {
+        // ---- column z-score over the whole instance (population standard deviation) -------------------
+        double* red = reinterpret_cast<double*>(pbest);             // [CF_T][2] (the assign's scratch: free here)
+        constexpr int SL = CF_T / D;                                // threads per column
+        const int c = tid % D, sl = tid / D;
+        const float pivot = xraw[c];                                // first row of the instance: the same shift everywhere
+        double s1 = 0.0, s2 = 0.0;
+        for (int r = sl; r < rows; r += SL) {
+            const float e = zs[(size_t)r * ZS + c] - pivot;
+            s1 += (double)e;
+            s2 += (double)e * (double)e;
+        }
+        red[2 * tid] = s1; red[2 * tid + 1] = s2;
+        __syncthreads();
+        if (tid < D) {
+            for (int q = 1; q < SL; ++q) { s1 += red[2 * (q * D + c)]; s2 += red[2 * (q * D + c) + 1]; }
+            npart[((size_t)g * D + c) * 2] = s1;
+            npart[((size_t)g * D + c) * 2 + 1] = s2;
+        }
+        if (!grid_barrier(sc, 1u, (unsigned)G)) {
+            if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
+            return;
+        }
+        // every CTA adds all partials, slices of the CTA index per thread, then the slices in order
+        s1 = 0.0; s2 = 0.0;
+        for (int k = sl; k < G; k += SL) {
+            s1 += __ldcg(npart + ((size_t)k * D + c) * 2);
+            s2 += __ldcg(npart + ((size_t)k * D + c) * 2 + 1);
+        }
+        red[2 * tid] = s1; red[2 * tid + 1] = s2;
+        __syncthreads();
+        float* st_mh = reinterpret_cast<float*>(red + 2 * CF_T);    // [D] mean high | [D] mean low | [D] 1 / sd
+        if (tid < D) {
+            for (int q = 1; q < SL; ++q) { s1 += red[2 * (q * D + c)]; s2 += red[2 * (q * D + c) + 1]; }
+            const double ms = s1 / (double)N;
+            double var = s2 / (double)N - ms * ms;
+            if (var < 0.0) var = 0.0;
+            const double mean = (double)pivot + ms;
+            const double sd = sqrt(var);
+            const double scd = sd < 1e-12 ? 1.0 : sd;               // a constant column is only centred
+            const float mh = (float)mean;
+            st_mh[c] = mh;
+            st_mh[D + c] = (float)(mean - (double)mh);
+            st_mh[2 * D + c] = (float)(1.0 / scd);
+        }
+        __syncthreads();
+        float* zo = zout + (size_t)r0 * D;
+        for (int e = tid; e < rows * (D / 4); e += CF_T) {
+            const int r = e / (D / 4), q = e - r * (D / 4);
+            float* d = zs + (size_t)r * ZS + 4 * q;
+            float4 v;
+            v.x = ((d[0] - st_mh[4 * q]) - st_mh[D + 4 * q]) * st_mh[2 * D + 4 * q];
+            v.y = ((d[1] - st_mh[4 * q + 1]) - st_mh[D + 4 * q + 1]) * st_mh[2 * D + 4 * q + 1];
+            v.z = ((d[2] - st_mh[4 * q + 2]) - st_mh[D + 4 * q + 2]) * st_mh[2 * D + 4 * q + 2];
+            v.w = ((d[3] - st_mh[4 * q + 3]) - st_mh[D + 4 * q + 3]) * st_mh[2 * D + 4 * q + 3];
+            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+            reinterpret_cast<float4*>(zo)[e] = v;
+        }
+        if (init_rows)
+            for (int e = tid; e < KD; e += CF_T) {
+                const int j = e / D, d = e - j * D, r = init_rows[j];
+                if (r >= 0 && r < N) cs[e] = ((cs[e] - st_mh[d]) - st_mh[D + d]) * st_mh[2 * D + d];
+            }
+        __syncthreads();
+    }
     float x[CF_R][D];
 #pragma unroll
     for (int u = 0; u < CF_R; ++u) {
@@ -201,7 +285,7 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
             }
         }
         // ---- everybody's sums are in the table after the barrier ---------------------------------
-        ok = grid_barrier(sc, (unsigned)(it + 1), (unsigned)G);
+        ok = grid_barrier(sc, epoch0 + (unsigned)(it + 1), (unsigned)G);
         if (!ok) break;
         // written by other CTAs: read through L2; the counts once per cluster (every CTA reads these lines)
         {
@@ -284,7 +368,7 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, float* __r
     }
     if (inertia || rep) {
         // one more barrier, then CTA 0 publishes what needed every CTA's contribution
-        if (!grid_barrier(sc, (unsigned)(iters + 1), (unsigned)G)) {
+        if (!grid_barrier(sc, epoch0 + (unsigned)(iters + 1), (unsigned)G)) {
             if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
             return;
         }
@@ -316,8 +400,10 @@ int cf_ctas(const kb_ctx* ctx, int N) {
     long G = ctx->sm_count < cap ? ctx->sm_count : cap;
     return (int)(G < 1 ? 1 : G);
 }
+constexpr size_t CF_NPART_BYTES = (size_t)256 * 64 * 2 * 8;   // column sums of up to 256 CTAs x 64 columns (in-kernel normalisation)
+size_t cf_tables(int D, int K) { return kb_align256((size_t)3 * CF_NC * (K * D + ((K + 3) & ~3)) * 4); }
 size_t cf_scratch(int D, int K) {
-    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)K * 8) + kb_align256((size_t)3 * CF_NC * (K * D + ((K + 3) & ~3)) * 4) + 256;
+    return kb_align256(sizeof(CoopScratch)) + kb_align256((size_t)K * 8) + cf_tables(D, K) + CF_NPART_BYTES + 256;
 }
 
 }  // namespace
@@ -336,9 +422,13 @@ bool kb_fit_coop_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
     return cf_smem(rows_per, D, K) + 1024 <= (size_t)ctx->max_smem_optin && ctx->ws_bytes >= cf_scratch(D, K);
 }
 
-kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, float* cent, int32_t* labels,
-                             float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+// z: normalised features (input), or null with xraw (raw features, input), zout (normalised, output; may be xraw
+// itself) and init_rows (row ids of the initial centroids; null: `cent` holds them)
+kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, const float* xraw, float* zout,
+                             const int32_t* init_rows, float* cent, int32_t* labels, float* dist2, float* inertia,
+                             int32_t* rep, int32_t* counts) {
     const int G = cf_ctas(ctx, N);
+    if (G > 256) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_cluster_fit: more than 256 SMs");
     const int rows_per = (N + G - 1) / G;
     const size_t smem = cf_smem(rows_per, D, K);
     // workspace: barrier words | representative keys | tables.  Cleared here: everything up to the end of
@@ -347,6 +437,7 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
     CoopScratch* sc = reinterpret_cast<CoopScratch*>(ws);
     unsigned long long* rep_key = reinterpret_cast<unsigned long long*>(ws + kb_align256(sizeof(CoopScratch)));
     float* table = reinterpret_cast<float*>(reinterpret_cast<char*>(rep_key) + kb_align256((size_t)K * 8));
+    double* npart = reinterpret_cast<double*>(reinterpret_cast<char*>(table) + cf_tables(D, K));   // plain stores: never cleared
     const size_t zbytes = (size_t)(reinterpret_cast<char*>(table) - ws) + kb_align256((size_t)CF_NC * (K * D + ((K + 3) & ~3)) * 4);
     kb_launch(coop_zero_kernel, (unsigned)((zbytes / 16 + 255) / 256), 256, 0, ctx->stream, zbytes / 16,
               reinterpret_cast<uint4*>(ws));
@@ -366,8 +457,8 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
 #define KB_CF_LAUNCH(DD, SS)                                                                                      \
     do {                                                                                                          \
         KB_SMEM_OPTIN(ctx, (fit_coop_kernel<DD, SS>), smem);                                                      \
-        e = cudaLaunchKernelEx(&cfg, fit_coop_kernel<DD, SS>, N, K, iters, z, cent, labels, dist2, inertia, rep,  \
-                               counts, sc, table, rep_key, ctx->dev_status);                                      \
+        e = cudaLaunchKernelEx(&cfg, fit_coop_kernel<DD, SS>, N, K, iters, z, xraw, zout, init_rows, npart, cent, \
+                               labels, dist2, inertia, rep, counts, sc, table, rep_key, ctx->dev_status);        \
     } while (0)
 #define KB_CF_LAUNCH_D(DD)                            \
     do {                                              \

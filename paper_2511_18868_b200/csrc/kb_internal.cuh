@@ -107,8 +107,9 @@ kb_status kb_launch_assign_finish(kb_ctx* ctx, int B, int N, int D, int K, const
 bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
 bool kb_fit_coop_eligible(const kb_ctx* ctx, int B, int N, int D, int K);
 size_t kb_ws_need_fit_coop(int B, int N, int D, int K);
-kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, float* cent, int32_t* labels,
-                             float* dist2, float* inertia, int32_t* rep, int32_t* counts);
+kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const float* z, const float* xraw, float* zout,
+                             const int32_t* init_rows, float* cent, int32_t* labels, float* dist2, float* inertia,
+                             int32_t* rep, int32_t* counts);
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
                               float* inertia, int32_t* rep, int32_t* counts);

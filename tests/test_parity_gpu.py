@@ -394,6 +394,37 @@ def test_step_small_instances_one_launch(kbx, B, N, D, K, S, host_buffers):
         parity.cluster_select_match(got["best_cluster_arm"], s_chk, s_chk["cl_index"])
 
 
+@pytest.mark.parametrize("N,D,K", [(5000, 16, 8), (20011, 32, 64), (40000, 64, 40)])
+@pytest.mark.parametrize("host_buffers", [False, True])
+def test_step_mid_sized_instance_one_launch(kbx, N, D, K, host_buffers):
+    """One mid-sized instance goes from raw features to labels in one cooperative launch inside the whole-step
+    drivers (column statistics across all CTAs, z written once, the seeding rows fetched before z may overwrite
+    x in place).  z must be what kb_normalize gives, also for constant, offset and tiny-spread columns; with no
+    Lloyd iteration the centroids are exactly the named rows of z."""
+    for iters in (0, 3):
+        cfg = wl.scaled(wl.CONFIGS["medium"], N=N, D=D, K=K, components=max(4, K // 2), S=8, iters=iters)
+        inp = wl.make_inputs(cfg, seed=N + D)
+        x = inp["x"]
+        x[:, :, 0] = -7.5
+        x[:, :, 1] = x[:, :, 1] * 0.5 + 1.0e4
+        x[:, :, 2] = x[:, :, 2] * 1.0e-3
+        launches0 = kbx.launch_count()[0]
+        got = run_step(kbx, cfg, inp, host_buffers)
+        launches = kbx.launch_count()[0] - launches0
+        assert kbx.device_status() == 0
+        assert launches <= 7, f"{launches} kernels: the clustering part did not run as one cooperative launch"
+        zr, _, _ = oracle.normalize(x)
+        parity.close(got["z"], zr, atol=2e-5, what="z")
+        assert np.all(got["z"][:, :, 0] == 0.0)
+        if iters == 0:
+            np.testing.assert_array_equal(got["centroids"][0], got["z"][0, inp["init_rows"][0]])
+        chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
+        parity.labels_match(got["z"], got["centroids"], got["labels"], chk)
+        same = got["labels"] == chk["labels"]
+        parity.close(got["dist2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
+        parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia")
+
+
 @pytest.mark.parametrize("N,D,K,iters", [(16384, 32, 64, 20), (5000, 16, 8, 7), (1025, 64, 100, 3), (40000, 32, 17, 4),
                                          (2048, 32, 64, 0)])
 def test_cluster_fit_cooperative(kbx, N, D, K, iters):
