@@ -333,8 +333,11 @@ kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
  * only pruning and scoring read (work, traffic, runtimes, signatures, pulls,
  * rewards) travel on a second stream owned by the context while the clustering
  * runs on the caller's stream; the caller's stream waits for them before
- * kb_prune.  The device staging
- * area is carved from the registered workspace, which must hold
+ * kb_prune.  When bound is requested and holds a megabyte or more, the gain
+ * bound, which depends on none of the clustering, is computed on a third stream
+ * as soon as its six inputs are up and travels back while the clustering runs;
+ * the values are the ones kb_prune gives.  The device
+ * staging area is carved from the registered workspace, which must hold
  * kb_step_workspace_bytes(...) bytes.  Pinned host memory makes the copies
  * asynchronous; pageable memory works too. */
 kb_status kb_step_workspace_bytes(int B, int N, int D, int K, int S, int R, size_t* out);

@@ -91,10 +91,16 @@ kb_status kb_create(kb_ctx** out, int device, void* cuda_stream) {
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_step_begin, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_late_inputs, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->early_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_prune_inputs, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_bound_done, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
     if (e != cudaSuccess) {
         if (ctx->dev_status) cudaFree(ctx->dev_status);
+        if (ctx->ev_bound_done) cudaEventDestroy(ctx->ev_bound_done);
+        if (ctx->ev_prune_inputs) cudaEventDestroy(ctx->ev_prune_inputs);
+        if (ctx->early_stream) cudaStreamDestroy(ctx->early_stream);
         if (ctx->ev_late_inputs) cudaEventDestroy(ctx->ev_late_inputs);
         if (ctx->ev_step_begin) cudaEventDestroy(ctx->ev_step_begin);
         if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -141,6 +147,9 @@ kb_status kb_destroy(kb_ctx* ctx) {
         delete[] ctx->ev_class;
     }
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->ev_bound_done) cudaEventDestroy(ctx->ev_bound_done);
+    if (ctx->ev_prune_inputs) cudaEventDestroy(ctx->ev_prune_inputs);
+    if (ctx->early_stream) cudaStreamDestroy(ctx->early_stream);
     if (ctx->ev_late_inputs) cudaEventDestroy(ctx->ev_late_inputs);
     if (ctx->ev_step_begin) cudaEventDestroy(ctx->ev_step_begin);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -404,7 +413,7 @@ static kb_status step_cluster(kb_ctx* ctx, const kb_step_args* a) {
 }
 
 // prune, score and select: two calls, or one launch for small instances
-static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a);
+static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a, bool bound_done = false);
 
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
     if (!ctx || !a) return KB_ERR_INVALID_ARG;
@@ -414,14 +423,16 @@ kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
     return step_tail(ctx, a);
 }
 
-static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a) {
+// bound_done: a->bound already holds the gain bound (it does not depend on the clustering): only the keep bits are due
+static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a, bool bound_done) {
     if (kb_step_tail_small_eligible(ctx, a)) {
         // at most 1024 candidates per instance: one CTA prunes, scores and selects for its instance
         TimeScope ts__(ctx, KB_T_SCORE);
-        return kb_launch_step_tail_small(ctx, a);
+        return kb_launch_step_tail_small(ctx, a, bound_done);
     }
     kb_status s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
-                 a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count, a->bound);
+                 a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count,
+                 bound_done ? nullptr : a->bound);
     if (s != KB_OK) return s;
     return kb_score_select(ctx, a->B, a->N, a->K, a->S, a->score, a->labels, a->dist2, a->pulls, a->reward_sum,
                            a->keep, a->bound, a->t, a->cl_pulls, a->cl_mean, a->cl_index, a->arm_index, a->best_arm,
@@ -534,6 +545,23 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     KB_H2D(peak_bw, S, float, cs);
     KB_H2D(t_incumbent, B, float, cs);
     KB_H2D(t_cur, B * N, float, cs);
+    // The gain bound B(k,s) depends on none of the clustering: once the six arrays above are up it is computed on a
+    // third stream and sent back while the clustering runs (large S: a quarter of the bytes that travel).  Below a
+    // megabyte the copy is shorter than what the extra launch and the two events cost the host.
+    const bool early_bound = d.bound && h->bound && B * N * S * sizeof(float) >= ((size_t)1 << 20);
+    if (early_bound) {
+        cudaStream_t es = ctx->early_stream;
+        KB_CUDA(ctx, cudaEventRecord(ctx->ev_prune_inputs, cs));
+        KB_CUDA(ctx, cudaStreamWaitEvent(es, ctx->ev_prune_inputs, 0));
+        ctx->stream = es;
+        const kb_status sp = kb_launch_prune(ctx, d.B, d.N, d.S, d.K, d.R, d.flops, d.bytes, d.peak_flops, d.peak_bw,
+                                             d.t_incumbent, d.t_cur, nullptr, nullptr, nullptr, d.theta_sat, d.keep, nullptr,
+                                             d.bound);
+        ctx->stream = st;
+        if (sp != KB_OK) { cudaStreamSynchronize(cs); cudaStreamSynchronize(es); return sp; }
+        KB_CUDA(ctx, cudaMemcpyAsync(h->bound, d.bound, B * N * S * sizeof(float), cudaMemcpyDeviceToHost, es));
+        KB_CUDA(ctx, cudaEventRecord(ctx->ev_bound_done, es));
+    }
     KB_H2D(hsig, B * K * R, float, cs);
     KB_H2D(target, S, int32_t, cs);
     KB_H2D(pulls, B * N * S, int32_t, cs);
@@ -548,11 +576,15 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     kb_status s = step_cluster(ctx, &d);
     if (s == KB_OK && cudaStreamWaitEvent(st, ctx->ev_late_inputs, 0) != cudaSuccess)
         s = kb_fail(ctx, KB_ERR_CUDA, "kb_bandit_step_host: cudaStreamWaitEvent failed");
-    if (s == KB_OK) s = step_tail(ctx, &d);
+    // (the early pass also wrote roofline-only keep bits: the real ones must come after it)
+    if (s == KB_OK && early_bound && cudaStreamWaitEvent(st, ctx->ev_bound_done, 0) != cudaSuccess)
+        s = kb_fail(ctx, KB_ERR_CUDA, "kb_bandit_step_host: cudaStreamWaitEvent failed");
+    if (s == KB_OK) s = step_tail(ctx, &d, early_bound);
     ctx->ws = ws_saved;
     ctx->ws_bytes = bytes_saved;
     if (s != KB_OK) {
         cudaStreamSynchronize(cs);             // nothing of this call may still be writing the staging area
+        cudaStreamSynchronize(ctx->early_stream);
         return s;
     }
 #define KB_D2H(field, count, type)                                                                          \
@@ -569,7 +601,7 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     KB_D2H(rep, B * K, int32_t);
     KB_D2H(keep, B * N, uint32_t);
     KB_D2H(kept_count, B, uint32_t);
-    KB_D2H(bound, B * N * S, float);
+    if (!early_bound) KB_D2H(bound, B * N * S, float);
     KB_D2H(cl_pulls, B * K * S, float);
     KB_D2H(cl_mean, B * K * S, float);
     KB_D2H(cl_index, B * K * S, float);

@@ -17,7 +17,8 @@ struct kb_ctx {
     size_t ws_bytes;
     int* dev_status;      // device status word (owned)
     cudaStream_t copy_stream;       // host-buffer step: copies of the late inputs (owned)
-    cudaEvent_t ev_step_begin, ev_late_inputs;
+    cudaStream_t early_stream;      // host-buffer step: the gain bound, computed and sent back while the clustering runs (owned)
+    cudaEvent_t ev_step_begin, ev_late_inputs, ev_prune_inputs, ev_bound_done;
     uint64_t launches;    // kernels queued so far
     uint64_t memsets;     // memset nodes queued so far
     // optional per-call event timing
@@ -94,7 +95,7 @@ size_t kb_ws_need_assign(int B, int N, int D, int K);
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
 size_t kb_ws_need_zsplit(int B, int N, int D, int K);
 bool kb_step_tail_small_eligible(const kb_ctx* ctx, const kb_step_args* a);
-kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* a);
+kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* a, bool bound_done = false);
 kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z);
 void kb_zsplit_forget(kb_ctx* ctx);
 bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K);

@@ -21,6 +21,7 @@ constexpr int ST_T = 256;
 
 struct TailArgs {
     int N, S, K, R;
+    int write_bound;        // 0: bound is there already (it does not depend on the clustering) and is only read
     float theta;
     kb_score_params prm;
     const float *flops, *bytes, *peak_flops, *peak_bw, *t_inc, *t_cur, *hsig, *dist2, *reward_sum;
@@ -115,7 +116,8 @@ step_tail_small_kernel(const TailArgs a) {
         for (int o = 1; o < vps; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
         if (live) {
             if (q == 0) { a.keep[i] = bits; skeep[r] = bits; count += __popc(bits); }
-            if (a.bound) *reinterpret_cast<float4*>(a.bound + i * S + 4 * q) = make_float4(g[0], g[1], g[2], g[3]);
+            if (a.bound && a.write_bound)
+                *reinterpret_cast<float4*>(a.bound + i * S + 4 * q) = make_float4(g[0], g[1], g[2], g[3]);
             if (lab_ok) {
                 int* dp = sp + lab * S + 4 * q;
                 float* dr = sr + lab * S + 4 * q;
@@ -178,7 +180,7 @@ step_tail_small_kernel(const TailArgs a) {
         const float4 tv = *reinterpret_cast<const float4*>(tab + lb_ * S + 4 * q);
         float uu[4] = {tv.x + smooth, tv.y + smooth, tv.z + smooth, tv.w + smooth};
         if (cap) {
-            const float4 bv = *reinterpret_cast<const float4*>(a.bound + i * S + 4 * q);   // written above by this thread
+            const float4 bv = *reinterpret_cast<const float4*>(a.bound + i * S + 4 * q);   // written above by this thread, or before this launch
             uu[0] = fminf(uu[0], bv.x); uu[1] = fminf(uu[1], bv.y); uu[2] = fminf(uu[2], bv.z); uu[3] = fminf(uu[3], bv.w);
         }
         const unsigned flat0 = (unsigned)(r * S + 4 * q);
@@ -227,8 +229,9 @@ bool kb_step_tail_small_eligible(const kb_ctx* ctx, const kb_step_args* a) {
     return (al & 15) == 0;
 }
 
-kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* s) {
+kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* s, bool bound_done) {
     TailArgs a;
+    a.write_bound = bound_done ? 0 : 1;
     a.N = s->N; a.S = s->S; a.K = s->K; a.R = s->R;
     a.theta = s->theta_sat;
     a.prm = s->score;

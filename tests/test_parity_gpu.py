@@ -346,7 +346,8 @@ def test_step_free_running(kbx, name, host_buffers):
     print(f"[{name}] label agreement with the free-running oracle: {agree:.6f}")
 
 
-@pytest.mark.parametrize("B,N,D,K,S", [(3, 300, 16, 5, 8), (2, 512, 32, 16, 32), (5, 77, 64, 9, 4), (4, 200, 32, 7, 16)])
+@pytest.mark.parametrize("B,N,D,K,S", [(3, 300, 16, 5, 8), (2, 512, 32, 16, 32), (5, 77, 64, 9, 4), (4, 200, 32, 7, 16),
+                                       (36, 512, 16, 6, 16)])
 @pytest.mark.parametrize("host_buffers", [False, True])
 def test_step_small_instances_one_launch(kbx, B, N, D, K, S, host_buffers):
     """Instances of at most 512 rows go from raw features to labels in ONE launch inside the whole-step drivers
@@ -365,7 +366,9 @@ def test_step_small_instances_one_launch(kbx, B, N, D, K, S, host_buffers):
         got = run_step(kbx, cfg, inp, host_buffers)
         launches = kbx.launch_count()[0] - launches0
         assert kbx.device_status() == 0
-        assert launches == 2, f"{launches} kernels: the step did not run as two launches"
+        # (from host buffers a gain bound of a megabyte or more is computed early, beside the clustering: one more)
+        early = int(host_buffers and B * N * S * 4 >= 1 << 20)
+        assert launches == 2 + early, f"{launches} kernels: the step did not run as two launches"
         zr, _, _ = oracle.normalize(x)
         parity.close(got["z"], zr, atol=2e-5, what="z")
         assert np.all(got["z"][:, :, 0] == 0.0)
@@ -412,7 +415,10 @@ def test_step_mid_sized_instance_one_launch(kbx, N, D, K, host_buffers):
         got = run_step(kbx, cfg, inp, host_buffers)
         launches = kbx.launch_count()[0] - launches0
         assert kbx.device_status() == 0
-        assert launches <= 7, f"{launches} kernels: the clustering part did not run as one cooperative launch"
+        # (the host-buffer form adds one when the gain bound is a megabyte or more: it is computed early, beside
+        # the clustering)
+        assert launches <= 7 + int(host_buffers), \
+            f"{launches} kernels: the clustering part did not run as one cooperative launch"
         zr, _, _ = oracle.normalize(x)
         parity.close(got["z"], zr, atol=2e-5, what="z")
         assert np.all(got["z"][:, :, 0] == 0.0)
