@@ -156,6 +156,31 @@ def init_centroids(z, rows):
     return c
 
 
+def philox4x32_10(counter, key):
+    """One block of the counter-based generator: counter = 4 words, key = 2 words -> 4 words (uint32)."""
+    c = np.ascontiguousarray(counter, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.empty((4,), np.uint32)
+    _load().kbo_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def sample_member(labels, cluster_arm, h_cand, target, theta_sat, seed, t, K, want_pert=True, want_prob=False):
+    """Within-cluster draw of k_t (Algorithm 1, "Sample k_t"): see kbo_sample_member."""
+    labels, cluster_arm, h_cand, target, t = _i32(labels), _i32(cluster_arm), _f32(h_cand), _i32(target), _i32(t)
+    B, N, R = h_cand.shape
+    S = target.shape[0]
+    member = np.empty((B,), np.int32)
+    val = np.empty((B,), np.float64)
+    pert = np.empty((B, N), np.float64) if want_pert else None
+    prob = np.empty((B, N), np.float64) if want_prob else None
+    _check(_load().kbo_sample_member(B, N, K, S, R, _p(labels), _p(cluster_arm), _p(h_cand), _p(target),
+                                     ctypes.c_float(theta_sat), ctypes.c_uint64(int(seed) & (2**64 - 1)), _p(t),
+                                     _p(member), _p(val), _p(pert), _p(prob)), "sample_member")
+    return {"member": member, "member_val": val, "pert": pert, "prob": prob}
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

@@ -310,4 +310,101 @@ int kbo_init_centroids(int B, int N, int D, int K, const float* z, const int32_t
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Counter-based random numbers: Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, "Parallel random
+// numbers: as easy as 1, 2, 3", SC'11), written out from the published round function: two 32x32 -> 64 bit
+// products by the constants below, a word permutation with the key mixed in, and a Weyl bump of the key
+// between rounds.  Pinned by the known-answer vectors of the generator's reference distribution.
+// ---------------------------------------------------------------------------
+void kbo_philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4]) {
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---------------------------------------------------------------------------
+// Within-cluster sampling of the kernel k_t (Sec. 3.4, "Action selection"; Algorithm 1, the line
+// "Sample k_t in C_{I_t}"): once the pair (I_t, S_t) is chosen, k_t is drawn from the members of
+// cluster I_t with P(k) proportional to exp(V_hw(k, S_t)), V_hw(k, s) = theta_sat - h(k)[Target(s)].
+//
+// The draw uses the Gumbel-max rule, which samples exactly that distribution: every member gets
+// V_hw + G, G = -ln(-ln u) with u uniform in (0, 1), and the largest perturbed value wins (lowest
+// index on ties).  u comes from the counter-based generator above so that a parallel
+// implementation draws the same numbers in any order:
+//     counter = (candidate index, instance index, t[b], 0),  key = (low, high word of seed),
+//     u = ((first output word >> 9) + 0.5) * 2^-23          (23 bits: exact in fp32 and in double).
+// Readings: h(k) is given per candidate (h_cand[B][N][R]); the paper profiles only
+// the cluster representatives, so a caller without per-candidate profiles passes its estimate.  The
+// paper states no temperature: none is applied.  A member whose signature entry is NaN is never drawn.
+//
+// cluster_arm[b] = I_t * S + S_t as kbo_score_select returns it, or negative: no draw.
+// member[b]: the drawn candidate, or -1 (no pair chosen, or the cluster has no drawable member).
+// pert (optional, double [B][N]): the perturbed value of every drawable member of the chosen
+// cluster, -inf elsewhere (lets a test rank the members itself).
+// prob (optional, double [B][N]): the softmax probabilities by their plain definition
+// exp(V - max V) / sum, 0 for non-members (what the draw must follow in distribution).
+// ---------------------------------------------------------------------------
+int kbo_sample_member(int B, int N, int K, int S, int R, const int32_t* labels, const int32_t* cluster_arm,
+                      const float* h_cand, const int32_t* target, float theta_sat, uint64_t seed,
+                      const int32_t* t, int32_t* member, double* member_val, double* pert, double* prob) {
+    const uint32_t key[2] = {(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32)};
+    for (int b = 0; b < B; ++b) {
+        member[b] = -1;
+        if (member_val) member_val[b] = -kInf;
+        if (pert) for (int k = 0; k < N; ++k) pert[ix2(b, k, N)] = -kInf;
+        if (prob) for (int k = 0; k < N; ++k) prob[ix2(b, k, N)] = 0.0;
+        const int ca = cluster_arm[b];
+        if (ca < 0) continue;
+        if (ca >= K * S) return 2;
+        const int I = ca / S, s = ca % S;
+        const int col = target[s];
+        if (col < 0 || col >= R) return 2;
+        double best = -kInf, vmax = -kInf;
+        int arg = -1;
+        for (int k = 0; k < N; ++k) {
+            if (labels[ix2(b, k, N)] != I) continue;
+            const double h = (double)h_cand[ix3(b, k, col, N, R)];
+            if (std::isnan(h)) continue;
+            const double V = (double)theta_sat - h;
+            if (V > vmax) vmax = V;
+            const uint32_t ctr[4] = {(uint32_t)k, (uint32_t)b, (uint32_t)t[b], 0u};
+            uint32_t rnd[4];
+            kbo_philox4x32_10(ctr, key, rnd);
+            const double u = ((double)(rnd[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+            const double G = -std::log(-std::log(u));
+            const double v = V + G;
+            if (pert) pert[ix2(b, k, N)] = v;
+            if (v > best) { best = v; arg = k; }
+        }
+        member[b] = arg;
+        if (member_val && arg >= 0) member_val[b] = best;
+        if (prob && arg >= 0) {
+            double sum = 0.0;
+            for (int k = 0; k < N; ++k) {
+                if (labels[ix2(b, k, N)] != I) continue;
+                const double h = (double)h_cand[ix3(b, k, col, N, R)];
+                if (std::isnan(h)) continue;
+                sum += std::exp(((double)theta_sat - h) - vmax);
+            }
+            for (int k = 0; k < N; ++k) {
+                if (labels[ix2(b, k, N)] != I) continue;
+                const double h = (double)h_cand[ix3(b, k, col, N, R)];
+                if (std::isnan(h)) continue;
+                prob[ix2(b, k, N)] = std::exp(((double)theta_sat - h) - vmax) / sum;
+            }
+        }
+    }
+    return 0;
+}
+
 }  // extern "C"

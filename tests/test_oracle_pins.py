@@ -384,3 +384,104 @@ def test_workload_shapes_and_determinism():
     assert wl.CONFIGS["contraction"].arms == 33554432 and wl.CONFIGS["batched"].arms == 8388608
     m = wl.make_inputs(wl.scaled(wl.CONFIGS["medium"], N=4096))
     assert 0.08 < np.mean(m["pulls"] == 0) < 0.16       # 10 % forced zeros + Poisson(4) zeros (1.8 %)
+
+
+# ------------------------------------------------- within-cluster draw of k_t
+def test_philox_known_answers():
+    for row in read_golden("philox4x32_10.txt"):
+        w = [int(v) for v in row]
+        out = oracle.philox4x32_10(w[0:4], w[4:6])
+        assert [int(v) for v in out] == w[6:10]
+
+
+def _sample_case(M, h_members, theta=75.0, seed=0x1234_5678_9ABC_DEF0):
+    """M independent instances with the same candidates: rows 0, 2, 4, ... are the members of cluster 1."""
+    n_mem = len(h_members)
+    N, K, S, R = 2 * n_mem + 1, 3, 4, 5
+    labels = np.zeros((M, N), np.int32)
+    labels[:, 1::2] = 2
+    labels[:, 0:2 * n_mem:2] = 1
+    h = np.full((M, N, R), 1.0e3, np.float32)              # any other column or row would dominate if it were read
+    target = np.array([4, 0, 3, 1], np.int32)
+    s = 2                                                  # strategy 2 looks at resource 3
+    h[:, 0:2 * n_mem:2, 3] = np.asarray(h_members, np.float32)
+    h[:, 1::2, 3] = -1.0e3                                 # non-members with a huge potential: never drawn
+    cluster_arm = np.full((M,), 1 * S + s, np.int32)
+    t = np.arange(1, M + 1, dtype=np.int32)
+    return dict(labels=labels, cluster_arm=cluster_arm, h_cand=h, target=target, theta_sat=theta, seed=seed, t=t, K=K)
+
+
+def test_sample_member_follows_the_softmax():
+    """Frequencies over many independent draws match exp(V) / sum exp(V), V = theta_sat - h[Target(s)], computed
+    here from the definition: a flipped sign of V or of the perturbation, a wrong column or a biased uniform fails."""
+    hm = np.array([70.0, 70.5, 71.0, 72.0, 69.2, 73.5])
+    M = 120000
+    a = _sample_case(M, hm)
+    out = oracle.sample_member(**a, want_prob=True)
+    V = 75.0 - hm.astype(np.float32).astype(np.float64)    # the signatures are stored in fp32
+    p = np.exp(V - V.max())
+    p /= p.sum()
+    assert np.all(out["member"] % 2 == 0) and np.all(out["member"] < 2 * len(hm))
+    freq = np.bincount(out["member"] // 2, minlength=len(hm)) / M
+    sigma = np.sqrt(p * (1 - p) / M)
+    assert np.all(np.abs(freq - p) < 4.5 * sigma), (freq, p)
+    np.testing.assert_allclose(out["prob"][0, 0:2 * len(hm):2], p, rtol=1e-12)
+    assert np.all(out["prob"][:, 1::2] == 0.0)
+    # equal potentials: uniform over the members
+    out_u = oracle.sample_member(**_sample_case(M, np.full(5, 60.0)))
+    fu = np.bincount(out_u["member"] // 2, minlength=5) / M
+    assert np.all(np.abs(fu - 0.2) < 4.5 * np.sqrt(0.16 / M))
+
+
+def test_sample_member_rule_and_counter_layout():
+    """The drawn member is the largest of V + G over the cluster's members, G = -ln(-ln u), with u taken from the
+    generator at counter (candidate, instance, t, 0) and key = the two halves of the seed."""
+    hm = np.array([40.0, 41.5, 39.0, 44.0])
+    a = _sample_case(50, hm, seed=(0xCAFEBABE << 32) | 0x0BADF00D)
+    out = oracle.sample_member(**a)
+    for b in range(50):
+        vals = {}
+        for j, h in enumerate(hm):
+            k = 2 * j
+            w = oracle.philox4x32_10([k, b, int(a["t"][b]), 0], [0x0BADF00D, 0xCAFEBABE])
+            u = ((int(w[0]) >> 9) + 0.5) / 2.0 ** 23
+            vals[k] = (75.0 - h) - math.log(-math.log(u))
+        best = max(vals, key=lambda k: (vals[k], -k))
+        assert out["member"][b] == best
+        assert out["member_val"][b] == pytest.approx(vals[best], rel=1e-12)
+        for k, v in vals.items():
+            assert out["pert"][b, k] == pytest.approx(v, rel=1e-12)
+        assert np.all(np.isneginf(np.delete(out["pert"][b], list(vals))))
+
+
+def test_sample_member_special_cases():
+    hm = np.array([10.0, 20.0, 30.0])
+    a = _sample_case(8, hm)
+    # theta_sat shifts every potential alike: the draw does not move
+    m0 = oracle.sample_member(**a)["member"]
+    a2 = dict(a, theta_sat=12.5)
+    np.testing.assert_array_equal(oracle.sample_member(**a2)["member"], m0)
+    # a potential far above the others always wins; a single member is always drawn
+    far = _sample_case(64, np.array([90.0, 5.0, 90.0]))
+    assert np.all(oracle.sample_member(**far)["member"] == 2)
+    one = _sample_case(64, np.array([33.0]))
+    assert np.all(oracle.sample_member(**one)["member"] == 0)
+    # no pair chosen, or a cluster without members: no draw
+    a["cluster_arm"][0] = -1
+    a["cluster_arm"][1] = 0 * 4 + 1                         # cluster 0 holds only the last row
+    a["cluster_arm"][2] = 2 * 4 + 2                         # cluster 2: the odd rows, potential 75 + 1000 each
+    a["labels"][3, :] = 0                                   # instance 3: cluster 1 is empty
+    out = oracle.sample_member(**a)
+    assert out["member"][0] == -1 and out["member"][3] == -1
+    assert out["member"][1] == a["labels"].shape[1] - 1
+    assert out["member"][2] % 2 == 1
+    # a NaN signature entry is never drawn
+    a["h_cand"][4, 0, 3] = np.nan
+    a["h_cand"][4, 2, 3] = np.nan
+    assert oracle.sample_member(**a)["member"][4] == 4
+    # another seed gives other draws, the same seed the same ones
+    b1 = oracle.sample_member(**_sample_case(200, np.array([50.0, 50.3, 50.6, 50.9])))["member"]
+    b2 = oracle.sample_member(**_sample_case(200, np.array([50.0, 50.3, 50.6, 50.9])))["member"]
+    b3 = oracle.sample_member(**_sample_case(200, np.array([50.0, 50.3, 50.6, 50.9]), seed=7))["member"]
+    np.testing.assert_array_equal(b1, b2)
+    assert np.any(b1 != b3)
