@@ -94,7 +94,8 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_INIT 5
 #define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
 #define KB_T_ASSIGN_KERNEL 7 /* the tensor-core contraction kernel alone (nested inside KB_T_ASSIGN or KB_T_FIT) */
-#define KB_T_COUNT 8
+#define KB_T_SAMPLE 8 /* kb_sample_member */
+#define KB_T_COUNT 9
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
 
@@ -185,6 +186,37 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
                           const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
                           float* arm_index, int32_t* best_arm, float* best_val,
                           int32_t* best_cluster_arm);
+
+/* Within-cluster draw of the kernel k_t (Sec. 3.4, "Action selection";
+ * Algorithm 1, "Sample k_t in C_{I_t}"): once the pair (I_t, S_t) is chosen,
+ * k_t is drawn from the members of cluster I_t with
+ *   P(k) proportional to exp(V_hw(k, S_t)),  V_hw(k, s) = theta_sat - h(k)[Target(s)].
+ * The draw is a Gumbel-max: every member gets V_hw + G, G = -ln(-ln u), and the
+ * largest perturbed value wins (lowest index on ties), which samples exactly
+ * that softmax.  u comes from the counter-based generator Philox4x32 (10
+ * rounds): counter = (candidate index, instance index, t[b], 0), key = (low,
+ * high 32 bits of seed), u = ((first output word >> 9) + 0.5) * 2^-23.  The
+ * same seed and t repeat the draw; the result does not depend on the launch
+ * shape.  fp32 arithmetic (logf); no temperature (the paper states none).
+ *   labels [B][N] in: the candidates' clusters
+ *   cluster_arm [B] in: I_t*S + S_t as kb_score_select writes best_cluster_arm;
+ *                       negative = no pair chosen, member = -1
+ *   h_cand [B][N][R] in: the signature h(k) of every candidate (the paper
+ *                       profiles only representatives: a caller without
+ *                       per-candidate profiles passes its estimate); a NaN
+ *                       entry (or a potential of -inf) is never drawn
+ *   target [S] in, values in [0, R);  t [B] in: the step counter (draw index)
+ *   member [B] out: the drawn candidate in [0, N), or -1 (no pair, or no
+ *                       drawable member in the cluster)
+ *   member_val [B] out, nullable: its perturbed value (-inf if none)
+ * All arrays in DEVICE memory; seed by value.  cluster_arm >= K*S sets bit 4,
+ * a target outside [0, R) bit 2 of the device status word (member = -1).
+ * Needs the workspace of kb_workspace_bytes when an instance spans several
+ * CTAs (more than 8192 candidates). */
+kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const int32_t* labels,
+                           const int32_t* cluster_arm, const float* h_cand, const int32_t* target,
+                           float theta_sat, uint64_t seed, const int32_t* t, int32_t* member,
+                           float* member_val);
 
 /* Which kernel kb_cluster_assign uses.
  *   path: 0 = automatic (tensor cores when K >= 128, D a multiple of 32 and

@@ -178,6 +178,7 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     size_t need = 256;
     need = max_sz(need, kb_ws_need_normalize(B, N, D));
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
+    need = max_sz(need, kb_ws_need_sample(B));
     need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K));
     *out = need;
     return KB_OK;
@@ -325,6 +326,22 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
     TimeScope ts__(ctx, KB_T_SCORE);
     return kb_launch_score(ctx, B, N, K, S, p, labels, dist2, pulls, reward_sum, keep, bound, t, cl_pulls, cl_mean,
                            cl_index, arm_index, best_arm, best_val, best_cluster_arm);
+}
+
+kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const int32_t* labels,
+                           const int32_t* cluster_arm, const float* h_cand, const int32_t* target, float theta_sat,
+                           uint64_t seed, const int32_t* t, int32_t* member, float* member_val) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, K >= 1 && S >= 1 && R >= 1, "kb_sample_member: K, S and R must be >= 1");
+    if ((long long)K * S > 0x7fffffffLL)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_sample_member: K*S exceeds the 31-bit pair index");
+    if (B > 0)
+        KB_REQUIRE(ctx, cluster_arm && target && t && member,
+                   "kb_sample_member: cluster_arm, target, t and member are required");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, labels && h_cand, "kb_sample_member: labels and h_cand are required");
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_sample_member(ctx, B, N, K, S, R, labels, cluster_arm, h_cand, target, theta_sat, seed, t, member,
+                                   member_val);
 }
 
 kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,

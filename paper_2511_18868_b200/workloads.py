@@ -158,3 +158,19 @@ def make_inputs(cfg: Workload, seed: int | None = None) -> Dict[str, np.ndarray]
     out["prior_pulls"] = np.float32(1.0)
     out["prior_mean"] = np.float32(0.5)
     return out
+
+
+def make_candidate_signatures(hsig: np.ndarray, labels: np.ndarray, seed: int, spread: float = 3.0) -> np.ndarray:
+    """Per-candidate hardware signatures h(k) [B,N,R] f32 for the within-cluster draw of k_t.
+
+    The paper profiles only each cluster's representative (Sec. 3.4); the candidates of a cluster are behaviourally
+    similar by construction (Sec. 3.3), so a candidate's signature is drawn here as its cluster's signature plus
+    normal noise of `spread` percentage points, clipped to [0, 100].  Input data only: nothing of the draw itself.
+    """
+    rng = np.random.default_rng(seed)
+    B, N = labels.shape
+    R = hsig.shape[2]
+    base = np.take_along_axis(hsig, np.clip(labels, 0, hsig.shape[1] - 1)[:, :, None].astype(np.int64), axis=1) \
+        if N > 0 else np.zeros((B, 0, R), np.float32)
+    h = base + spread * rng.standard_normal((B, N, R))
+    return np.clip(h, 0.0, 100.0).astype(np.float32)

@@ -106,3 +106,27 @@ def rep_match(got, ref, dist2_ref, labels_ref, what="rep"):
                 assert dg - dw <= NEAR_TIE * max(dg, 1e-30) + 1e-12, f"{what}: member {g} is not nearest"
                 n += 1
     return n
+
+
+def member_match(got, got_val, ref, tol, what="member"):
+    """The drawn member is the largest perturbed value of the chosen cluster.  The library forms that value in fp32
+    (two logf), the oracle in double: where the oracle's two largest values are closer than `tol` either candidate
+    is a valid draw, everywhere else the index must agree; the returned value must be the chosen candidate's."""
+    pert = ref["pert"]
+    loose = 0
+    for b in range(got.shape[0]):
+        want = int(ref["member"][b])
+        g = int(got[b])
+        if want < 0:
+            assert g == -1, f"{what}[{b}]: drew {g} where no member can be drawn"
+            assert got_val is None or np.isneginf(got_val[b])
+            continue
+        assert 0 <= g < pert.shape[1] and np.isfinite(pert[b, g]) or pert[b, g] == np.inf, \
+            f"{what}[{b}]: {g} is not a drawable member of the chosen cluster"
+        if g != want:
+            assert pert[b, g] >= pert[b, want] - tol, \
+                f"{what}[{b}]: drew {g} ({pert[b, g]}) but {want} ({pert[b, want]}) is larger by more than {tol}"
+            loose += 1
+        if got_val is not None:
+            assert abs(float(got_val[b]) - pert[b, g]) <= tol, f"{what}_val[{b}]: {got_val[b]} vs {pert[b, g]}"
+    return loose

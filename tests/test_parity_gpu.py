@@ -696,3 +696,117 @@ def test_step_uses_tensor_path_when_eligible(kbx):
     assert kbx.assign_path() == 2
     a_chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
     parity.labels_match(got["z"], got["centroids"], got["labels"], a_chk)
+
+
+# -------------------------------------------------- within-cluster draw of k_t
+# fp32 against double: theta - h is one rounding of a value below 128 (8e-6), the inner logf one ulp of a value
+# whose logarithm is then taken (1.2e-7 absolute), the outer logf and the sum one ulp each of values below 128.
+SAMPLE_TOL = 5e-5
+
+
+def _sample_inputs(B, N, K, S, seed):
+    rng = np.random.default_rng(seed)
+    R = wl.R_RESOURCES
+    labels = rng.integers(0, K, size=(B, N)).astype(np.int32)
+    hsig = rng.uniform(0.0, 100.0, size=(B, K, R)).astype(np.float32)
+    h_cand = wl.make_candidate_signatures(hsig, labels, seed + 1)
+    target = (np.arange(S) % R).astype(np.int32)
+    cluster_arm = rng.integers(0, K * S, size=(B,)).astype(np.int32)
+    t = rng.integers(1, 100000, size=(B,)).astype(np.int32)
+    return labels, h_cand, target, cluster_arm, t
+
+
+def _run_sample(kbx, labels, h_cand, target, cluster_arm, t, K, theta, seed):
+    B = labels.shape[0]
+    member, val = empty((B,), torch.int32), empty((B,))
+    kbx.sample_member(dev(labels), dev(cluster_arm), dev(h_cand), dev(target), dev(t), member, K, theta, seed, val)
+    return host(member), host(val)
+
+
+@pytest.mark.parametrize("B,N,K,S", [(1, 256, 8, 8), (3, 1000, 5, 4), (2, 20011, 64, 16), (1, 262144, 256, 32),
+                                     (64, 512, 16, 16), (5, 1, 1, 1), (2, 8193, 3, 32), (1, 70001, 2, 2)])
+def test_sample_member(kbx, B, N, K, S):
+    labels, h_cand, target, cluster_arm, t = _sample_inputs(B, N, K, S, seed=B * 7 + N)
+    ws(kbx, B, N, 16, K, S)
+    seed = 0x9E3779B97F4A7C15 ^ N
+    got, val = _run_sample(kbx, labels, h_cand, target, cluster_arm, t, K, 75.0, seed)
+    ref = oracle.sample_member(labels, cluster_arm, h_cand, target, 75.0, seed, t, K)
+    loose = parity.member_match(got, val, ref, SAMPLE_TOL)
+    assert loose <= max(1, B // 50)
+    assert kbx.device_status() == 0
+    # the same seed and step repeat the draw; another step counter is another draw
+    again, _ = _run_sample(kbx, labels, h_cand, target, cluster_arm, t, K, 75.0, seed)
+    np.testing.assert_array_equal(again, got)
+    if N >= 256:
+        other, _ = _run_sample(kbx, labels, h_cand, target, cluster_arm, t + 1, K, 75.0, seed)
+        ref2 = oracle.sample_member(labels, cluster_arm, h_cand, target, 75.0, seed, t + 1, K)
+        parity.member_match(other, None, ref2, SAMPLE_TOL)
+
+
+def test_sample_member_edge_cases(kbx):
+    B, N, K, S = 8, 3000, 6, 4
+    labels, h_cand, target, cluster_arm, t = _sample_inputs(B, N, K, S, seed=11)
+    cluster_arm[0] = -1                                  # no pair chosen
+    labels[1][labels[1] == cluster_arm[1] // S] = (cluster_arm[1] // S + 1) % K     # the chosen cluster is empty
+    i2 = cluster_arm[2] // S
+    labels[2][labels[2] == i2] = (i2 + 1) % K
+    labels[2][1234] = i2                                 # exactly one member
+    i3, c3 = cluster_arm[3] // S, target[cluster_arm[3] % S]
+    m3 = np.flatnonzero(labels[3] == i3)
+    h_cand[3, m3[: len(m3) // 2], c3] = np.nan           # half of the members cannot be drawn
+    i4, c4 = cluster_arm[4] // S, target[cluster_arm[4] % S]
+    m4 = np.flatnonzero(labels[4] == i4)
+    h_cand[4, m4, c4] = np.nan                           # none can
+    i5, c5 = cluster_arm[5] // S, target[cluster_arm[5] % S]
+    h_cand[5, np.flatnonzero(labels[5] == i5), c5] = 42.0   # equal potentials: the perturbation alone decides
+    i6, c6 = cluster_arm[6] // S, target[cluster_arm[6] % S]
+    m6 = np.flatnonzero(labels[6] == i6)
+    h_cand[6, m6[-1], c6] = -np.inf                      # an infinite potential wins outright
+    h_cand[6, m6[0], c6] = np.inf                        # a potential of -inf is never drawn
+    ws(kbx, B, N, 16, K, S)
+    got, val = _run_sample(kbx, labels, h_cand, target, cluster_arm, t, K, 75.0, 5)
+    ref = oracle.sample_member(labels, cluster_arm, h_cand, target, 75.0, 5, t, K)
+    assert ref["member"][0] == -1 and ref["member"][1] == -1 and ref["member"][2] == 1234 and ref["member"][4] == -1
+    assert ref["member"][6] == m6[-1]
+    np.testing.assert_array_equal(got[[0, 1, 2, 4, 6]], ref["member"][[0, 1, 2, 4, 6]])
+    assert np.isneginf(val[[0, 1, 4]]).all() and val[6] == np.inf
+    for b in (3, 5, 7):
+        parity.member_match(got[b:b + 1], val[b:b + 1],
+                            {"member": ref["member"][b:b + 1], "pert": ref["pert"][b:b + 1]}, SAMPLE_TOL)
+    assert got[3] not in set(m3[: len(m3) // 2].tolist())
+    # zero instances, zero candidates
+    kbx.sample_member(empty((0, 5), torch.int32), empty((0,), torch.int32), empty((0, 5, 3)), dev(target),
+                      empty((0,), torch.int32), empty((0,), torch.int32), K, 75.0, 1)
+    m = empty((2,), torch.int32)
+    kbx.sample_member(empty((2, 0), torch.int32), dev(np.zeros(2, np.int32)), empty((2, 0, 3)), dev(target),
+                      dev(np.ones(2, np.int32)), m, K, 75.0, 1)
+    assert (host(m) == -1).all()
+    assert kbx.device_status() == 0
+
+
+def test_sample_member_frequencies(kbx):
+    """A property that holds at any size: over many instances with the same candidates the drawn members follow
+    exp(V) / sum exp(V), computed here from the definition."""
+    M, n_mem, rounds = 50000, 6, 4              # 200 000 draws: four calls, each with its own step counters
+    hm = np.array([70.0, 70.5, 71.0, 72.0, 69.25, 73.5], np.float32)
+    N, K, S = 2 * n_mem + 1, 3, 4
+    labels = np.zeros((M, N), np.int32)
+    labels[:, 1::2] = 2
+    labels[:, 0:2 * n_mem:2] = 1
+    h = np.full((M, N, wl.R_RESOURCES), 1.0e3, np.float32)
+    h[:, 0:2 * n_mem:2, 2] = hm
+    h[:, 1::2, 2] = -1.0e3
+    target = np.array([1, 0, 2, 1], np.int32)
+    cluster_arm = np.full((M,), 1 * S + 2, np.int32)
+    ws(kbx, M, N, 16, K, S)
+    counts = np.zeros(n_mem, np.int64)
+    for r in range(rounds):
+        t = np.arange(1 + r * M, 1 + (r + 1) * M, dtype=np.int32)
+        got, _ = _run_sample(kbx, labels, h, target, cluster_arm, t, K, 75.0, 2024)
+        assert np.all(got % 2 == 0) and np.all(got < 2 * n_mem) and np.all(got >= 0)
+        counts += np.bincount(got // 2, minlength=n_mem)
+    V = 75.0 - hm.astype(np.float64)
+    p = np.exp(V - V.max())
+    p /= p.sum()
+    freq = counts / (M * rounds)
+    assert np.all(np.abs(freq - p) < 4.5 * np.sqrt(p * (1 - p) / (M * rounds))), (freq, p)
