@@ -365,6 +365,38 @@ def run_ours(args, cfg):
     barrier()
     e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
 
+    # ---- the within-cluster draw of k_t (Algorithm 1's line after the selection; outside the timed step) ----
+    lab_host = dev_t["labels"].cpu().numpy()
+    h_cand = torch.from_numpy(wl.make_candidate_signatures(inp["hsig"], lab_host, seed=77)).to(device)
+    member = torch.empty((cfg.B,), dtype=torch.int32, device=device)
+
+    def draw(step):
+        ctx.sample_member(dev_t["labels"], dev_t["best_cluster_arm"], h_cand, dev_t["target"], dev_t["t"], member,
+                          cfg.K, float(inp["theta_sat"]), 0xC0FFEE + step)
+
+    for i in range(3):
+        draw(i)
+    barrier()
+    # timed by the library's own event pair around the call's work on the stream: the L2 flush before each call
+    # also gives the host time to queue the call, so the pair sees the device's time, not the host's
+    ks0, _ = ctx.launch_count()
+    ctx.timing_enable(True)
+    for i in range(args.steps):
+        flush.zero_()
+        draw(10 + i)
+    barrier()
+    smp_ms, smp_calls = ctx.timing_read()["sample"]
+    ctx.timing_enable(False)
+    ks1, _ = ctx.launch_count()
+    smp_us = smp_ms / max(smp_calls, 1) * 1e3
+    chosen = dev_t["best_cluster_arm"].cpu().numpy() // cfg.S
+    members = int(sum((lab_host[b] == chosen[b]).sum() for b in range(cfg.B) if chosen[b] >= 0))
+    smp_bytes = 4 * cfg.B * cfg.N + 4 * members + 16 * cfg.B      # labels, one signature entry per member, per-instance words
+    sample_line = {"avg_us": smp_us, "algorithmic_bytes": smp_bytes, "GBps": smp_bytes / (smp_us * 1e-6) / 1e9,
+                   "kernels_per_call": (ks1 - ks0) / args.steps, "members_of_chosen_clusters": members,
+                   "what": "kb_sample_member on the step's labels and chosen pairs (not part of the timed step)"}
+    del h_cand
+
     # ---- max over ranks -----------------------------------------------------------
     total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], dist, device)
     if rank != 0:
@@ -449,6 +481,7 @@ def run_ours(args, cfg):
         "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
         "device_status": int(status), "peaks": peaks,
         "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
+        "sample_member": sample_line,
     }
     print(json.dumps(line))
     ctx.close()

@@ -212,7 +212,7 @@ kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
  * All arrays in DEVICE memory; seed by value.  cluster_arm >= K*S sets bit 4,
  * a target outside [0, R) bit 2 of the device status word (member = -1).
  * Needs the workspace of kb_workspace_bytes when an instance spans several
- * CTAs (more than 8192 candidates). */
+ * CTAs (more than 4096 candidates). */
 kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const int32_t* labels,
                            const int32_t* cluster_arm, const float* h_cand, const int32_t* target,
                            float theta_sat, uint64_t seed, const int32_t* t, int32_t* member,

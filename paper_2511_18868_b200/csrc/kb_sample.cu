@@ -20,7 +20,7 @@ namespace {
 
 constexpr int SM_T = 256;      // threads per CTA
 constexpr int SM_U = 4;        // label loads in flight per thread
-constexpr int SM_ROWS = SM_T * SM_U * 8;   // rows per CTA at least (when the instance is split)
+constexpr int SM_ROWS = SM_T * SM_U * 4;   // rows per CTA at least (when the instance is split): one vector trip
 
 // Philox4x32 with 10 rounds (Salmon et al., SC'11): first output word only.
 __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
@@ -55,8 +55,9 @@ __device__ __forceinline__ void sample_store(unsigned long long key, int32_t* me
     }
 }
 
+template <bool VEC>
 __global__ void __launch_bounds__(SM_T)
-sample_member_kernel(int N, int K, int S, int R, int G, const int32_t* __restrict__ labels,
+sample_member_kernel(int N, int K, int S, int R, int rows_per, int G, const int32_t* __restrict__ labels,
                      const int32_t* __restrict__ cluster_arm, const float* __restrict__ h_cand,
                      const int32_t* __restrict__ target, float theta, uint32_t seed_lo, uint32_t seed_hi,
                      const int32_t* __restrict__ t, SampleWs w, int32_t* __restrict__ member,
@@ -82,33 +83,50 @@ sample_member_kernel(int N, int K, int S, int R, int G, const int32_t* __restric
         }
     }
     if (draw) {
-        const int rows_per = (N + G - 1) / G;
         const int r0 = blockIdx.x * rows_per, r1 = min(N, r0 + rows_per);
         const int32_t* lb = labels + (size_t)b * N;
         const float* hb = h_cand + (size_t)b * N * R + col;
         const uint32_t tb = (uint32_t)t[b];
-        for (int base = r0 + tid; base < r1; base += SM_T * SM_U) {
-            int lab[SM_U];
+        // one candidate of the chosen cluster: signature entry, uniform, perturbed value, packed key
+        auto take = [&](int r) {
+            const float h = __ldg(hb + (size_t)r * R);
+            const uint32_t w0 = philox4x32_10_word0((uint32_t)r, (uint32_t)b, tb, 0u, seed_lo, seed_hi);
+            const float uni = ((float)(w0 >> 9) + 0.5f) * (1.0f / 8388608.0f);   // 23 bits: exact
+            const float v = (theta - h) - logf(-logf(uni));
+            if (!(v > -INFINITY)) return;                                        // NaN or -inf: never drawn
+            const unsigned long long key =
+                ((unsigned long long)kb_orderable(v) << 32) | (unsigned long long)(0xffffffffu - (unsigned)r);
+            best = key > best ? key : best;
+        };
+        if (VEC) {
+            // r0 is a multiple of 4 (the host rounds rows_per up): 16 labels per thread and trip, four loads in flight
+            const int4* lb4 = reinterpret_cast<const int4*>(lb);
+            const int q1 = (r1 + 3) >> 2;                      // N % 4 == 0 on this path, so whole quads only
+            for (int q = (r0 >> 2) + tid; q < q1; q += SM_T * SM_U) {
+                int4 lab[SM_U];
 #pragma unroll
-            for (int u = 0; u < SM_U; ++u) {
-                const int r = base + u * SM_T;
-                lab[u] = r < r1 ? __ldg(lb + r) : -1;
+                for (int u = 0; u < SM_U; ++u)
+                    lab[u] = q + u * SM_T < q1 ? __ldg(lb4 + q + u * SM_T) : make_int4(-1, -1, -1, -1);
+#pragma unroll
+                for (int u = 0; u < SM_U; ++u) {
+                    const int r = (q + u * SM_T) << 2;
+                    if (lab[u].x == I) take(r);
+                    if (lab[u].y == I) take(r + 1);
+                    if (lab[u].z == I) take(r + 2);
+                    if (lab[u].w == I) take(r + 3);
+                }
             }
-            float h[SM_U];
+        } else {
+            for (int base = r0 + tid; base < r1; base += SM_T * SM_U) {
+                int lab[SM_U];
 #pragma unroll
-            for (int u = 0; u < SM_U; ++u)
-                h[u] = lab[u] == I ? __ldg(hb + (size_t)(base + u * SM_T) * R) : 0.f;
+                for (int u = 0; u < SM_U; ++u) {
+                    const int r = base + u * SM_T;
+                    lab[u] = r < r1 ? __ldg(lb + r) : -1;
+                }
 #pragma unroll
-            for (int u = 0; u < SM_U; ++u) {
-                if (lab[u] != I) continue;
-                const int r = base + u * SM_T;
-                const uint32_t w0 = philox4x32_10_word0((uint32_t)r, (uint32_t)b, tb, 0u, seed_lo, seed_hi);
-                const float uni = ((float)(w0 >> 9) + 0.5f) * (1.0f / 8388608.0f);   // 23 bits: exact
-                const float v = (theta - h[u]) - logf(-logf(uni));
-                if (!(v > -INFINITY)) continue;                                     // NaN or -inf: never drawn
-                const unsigned long long key =
-                    ((unsigned long long)kb_orderable(v) << 32) | (unsigned long long)(0xffffffffu - (unsigned)r);
-                best = key > best ? key : best;
+                for (int u = 0; u < SM_U; ++u)
+                    if (lab[u] == I) take(base + u * SM_T);
             }
         }
     }
@@ -137,7 +155,7 @@ sample_member_kernel(int N, int K, int S, int R, int G, const int32_t* __restric
 }
 
 int sample_ctas(const kb_ctx* ctx, int B, int N) {
-    long want = (2L * ctx->sm_count + B - 1) / B;
+    long want = (8L * ctx->sm_count + B - 1) / B;      // eight CTAs of 256 threads fit an SM
     long cap = ((long)N + SM_ROWS - 1) / SM_ROWS;
     long g = want < cap ? want : cap;
     return (int)(g < 1 ? 1 : g);
@@ -162,9 +180,16 @@ kb_status kb_launch_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R
         w.done = reinterpret_cast<unsigned*>(ctx->ws + kb_align256((size_t)B * 8));
         KB_MEMSET(ctx, ctx->ws, 0, need);
     }
-    kb_launch(sample_member_kernel, dim3(G, B), SM_T, 0, ctx->stream, N, K, S, R, G, labels, cluster_arm, h_cand, target,
-              theta_sat, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), t, w, member, member_val,
-              ctx->dev_status);
+    const bool vec = (N % 4 == 0) && (((uintptr_t)labels & 15) == 0);
+    int rows_per = (N + G - 1) / G;
+    rows_per = (rows_per + 3) & ~3;                    // every CTA starts on a quad of labels
+    const uint32_t s_lo = (uint32_t)(seed & 0xffffffffu), s_hi = (uint32_t)(seed >> 32);
+    if (vec)
+        kb_launch(sample_member_kernel<true>, dim3(G, B), SM_T, 0, ctx->stream, N, K, S, R, rows_per, G, labels, cluster_arm,
+                  h_cand, target, theta_sat, s_lo, s_hi, t, w, member, member_val, ctx->dev_status);
+    else
+        kb_launch(sample_member_kernel<false>, dim3(G, B), SM_T, 0, ctx->stream, N, K, S, R, rows_per, G, labels, cluster_arm,
+                  h_cand, target, theta_sat, s_lo, s_hi, t, w, member, member_val, ctx->dev_status);
     KB_LAUNCH_CHECK(ctx, "sample_member_kernel");
     return KB_OK;
 }

@@ -35,6 +35,15 @@ def test_fullsize_step(name):
         # large: the fit keeps a pre-split image of Z; contraction (D = 128): rows are split inside the kernel
         assert ctx.assign_presplit() == (name == "large")
         got = {k: v.cpu().numpy() for k, v in t.items()}
+        # the within-cluster draw of k_t, chained on the step's device results (labels, chosen pair)
+        h_cand = wl.make_candidate_signatures(inp["hsig"], got["labels"], seed=77)
+        member = torch.empty((B,), dtype=torch.int32, device=ctx.device)
+        member_val = torch.empty((B,), dtype=torch.float32, device=ctx.device)
+        ctx.sample_member(t["labels"], t["best_cluster_arm"], torch.from_numpy(h_cand).to(ctx.device), t["target"],
+                          t["t"], member, K, float(inp["theta_sat"]), 0xC0FFEE, member_val)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        got["member"], got["member_val"] = member.cpu().numpy(), member_val.cpu().numpy()
     finally:
         ctx.close()
     del t
@@ -85,5 +94,10 @@ def test_fullsize_step(name):
     parity.close(got["arm_index"], s["arm_index"], atol=1e-6, what="arm_index")
     sel_ties = parity.select_match(got["best_arm"], got["best_val"], s, s["arm_index"])
     parity.cluster_select_match(got["best_cluster_arm"], s, s["cl_index"])
+    # the draw: every instance in full, from the GPU's own labels and chosen pair
+    d = oracle.sample_member(labels, got["best_cluster_arm"], h_cand, inp["target"], float(inp["theta_sat"]), 0xC0FFEE,
+                             inp["t"], K)
+    assert d["member"][0] >= 0 and labels[0, got["member"][0]] == got["best_cluster_arm"][0] // S
+    parity.member_match(got["member"], got["member_val"], d, 5e-5)
     print(f"[{name} full size] near-ties: labels (sample of {len(rows)}) {ties}, keep bits {prune_ties}, "
           f"selection {sel_ties}")
