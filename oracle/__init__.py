@@ -181,6 +181,20 @@ def sample_member(labels, cluster_arm, h_cand, target, theta_sat, seed, t, K, wa
     return {"member": member, "member_val": val, "pert": pert, "prob": prob}
 
 
+def record_outcome(member, cluster_arm, t_cur, t_new, pulls, reward_sum, t, verified=None, failures_count=False):
+    """Reward clip and statistics update of one iteration (see kbo_record_outcome).  Returns new copies."""
+    member, cluster_arm, t_cur, t_new = _i32(member), _i32(cluster_arm), _f32(t_cur), _f32(t_new)
+    pulls, reward_sum, t = _i32(pulls).copy(), _f32(reward_sum).copy(), _i32(t).copy()
+    if verified is not None:
+        verified = _i32(verified)
+    B, N, S = pulls.shape
+    reward = np.empty((B,), np.float32)
+    _check(_load().kbo_record_outcome(B, N, S, int(bool(failures_count)), _p(member), _p(cluster_arm), _p(t_cur),
+                                      _p(t_new), _p(verified), _p(pulls), _p(reward_sum), _p(t), _p(reward)),
+           "record_outcome")
+    return {"pulls": pulls, "reward_sum": reward_sum, "t": t, "reward": reward}
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

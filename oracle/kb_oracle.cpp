@@ -407,4 +407,49 @@ int kbo_sample_member(int B, int N, int K, int S, int R, const int32_t* labels, 
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Outcome of one iteration (Sec. 2.2 "Formal Model": r_t = Clip((L(k_t) - L(k'_t)) / L(k_t), 0, 1);
+// Algorithm 1, "Generation & update": if Verify(k'_t): N_{I,S} <- N_{I,S} + 1,
+// mu_{I,S} <- mu_{I,S} + (r_t - mu_{I,S}) / N_{I,S}).
+//
+// The statistics are kept per arm as (pulls, reward_sum), from which kbo_score_select forms
+// N_{i,s} and mu_{i,s} per cluster in closed form (so that a re-clustering re-aggregates them);
+// the update of the pair (I_t, S_t) through its drawn member k_t is therefore
+//     pulls[k_t][S_t] += 1,  reward_sum[k_t][S_t] += r_t,
+// which gives exactly the running mean above for the cluster that holds k_t.
+// Readings: Algorithm 1 skips the update when verification fails, the formal model assigns
+// zero reward to failures; `failures_count` = 0 takes Algorithm 1's line (no update), non-zero
+// the other (one pull with reward 0).  A runtime L(k_t) <= 0 or a NaN ratio gives reward 0.
+// The iteration counter t[b] advances in every case (it is the loop index of Algorithm 1).
+//
+// member [B]: k_t (negative: nothing was drawn, only t advances); cluster_arm [B]: I_t*S + S_t;
+// t_cur [B][N]: L(k) of every candidate; t_new [B]: L(k'_t); verified [B] (nullable = all pass).
+// reward [B] (optional out): r_t as used (0 where nothing was updated).
+// ---------------------------------------------------------------------------
+int kbo_record_outcome(int B, int N, int S, int failures_count, const int32_t* member, const int32_t* cluster_arm,
+                       const float* t_cur, const float* t_new, const int32_t* verified, int32_t* pulls,
+                       float* reward_sum, int32_t* t, float* reward) {
+    for (int b = 0; b < B; ++b) {
+        if (reward) reward[b] = 0.0f;
+        t[b] += 1;
+        const int k = member[b];
+        if (k < 0) continue;
+        if (k >= N || cluster_arm[b] < 0) return 2;
+        const int s = cluster_arm[b] % S;
+        const bool ok = verified ? verified[b] != 0 : true;
+        if (!ok && !failures_count) continue;
+        double r = 0.0;
+        if (ok) {
+            const double L = (double)t_cur[ix2(b, k, N)], Ln = (double)t_new[b];
+            r = L > 0.0 ? (L - Ln) / L : 0.0;
+            if (!(r > 0.0)) r = 0.0;          // regressions and NaN
+            if (r > 1.0) r = 1.0;
+        }
+        pulls[ix3(b, k, s, N, S)] += 1;
+        reward_sum[ix3(b, k, s, N, S)] = (float)((double)reward_sum[ix3(b, k, s, N, S)] + r);
+        if (reward) reward[b] = (float)r;
+    }
+    return 0;
+}
+
 }  // extern "C"

@@ -485,3 +485,58 @@ def test_sample_member_special_cases():
     b3 = oracle.sample_member(**_sample_case(200, np.array([50.0, 50.3, 50.6, 50.9]), seed=7))["member"]
     np.testing.assert_array_equal(b1, b2)
     assert np.any(b1 != b3)
+
+
+# ------------------------------------------------------ outcome of an iteration
+def test_record_outcome_reproduces_algorithm1_statistics():
+    """Feeding the golden reward sequences through the update, one iteration at a time and through different member
+    kernels of one cluster, leaves statistics whose cluster aggregate is Algorithm 1's (N, mu)."""
+    for r1, r2, r3, r4, n_fin, mu_fin in read_golden("running_mean.txt"):
+        N, S = 3, 2
+        pulls = np.zeros((1, N, S), np.int32)
+        rsum = np.zeros((1, N, S), np.float32)
+        t = np.array([1], np.int32)
+        t_cur = np.array([[2.0, 4.0, 8.0]], np.float32)
+        for j, r in enumerate([r1, r2, r3, r4]):
+            k = j % 2                                             # members 0 and 1 of cluster 0 take turns
+            t_new = np.array([t_cur[0, k] * (1.0 - r)], np.float32)   # a kernel faster by the fraction r
+            out = oracle.record_outcome([k], [0 * S + 1], t_cur, t_new, pulls, rsum, t)
+            assert out["reward"][0] == pytest.approx(r, abs=1e-7)
+            pulls, rsum, t = out["pulls"], out["reward_sum"], out["t"]
+        assert t[0] == 5 and pulls[0, :, 1].tolist() == [2, 2, 0] and not pulls[0, :, 0].any()
+        sc = oracle.score_select(np.array([[0, 0, 1]], np.int32), np.zeros((1, N), np.float32), pulls, rsum, t, K=2)
+        assert sc["cl_pulls"][0, 0, 1] == n_fin
+        assert sc["cl_mean"][0, 0, 1] == pytest.approx(mu_fin, abs=1e-6)
+        assert sc["cl_pulls"][0, 0, 0] == 1 and sc["cl_mean"][0, 0, 0] == 0.5        # untouched pair: the prior
+
+
+def test_record_outcome_clip_and_failures():
+    N, S = 4, 3
+    t_cur = np.array([[10.0, 5.0, 0.0, 2.0]] * 6, np.float32)
+    member = np.array([0, 0, 1, 2, -1, 3], np.int32)
+    arm = np.array([2, 2, 4, 0, 1, 5], np.int32)                   # strategies 2, 2, 1, 0, 1, 2
+    t_new = np.array([12.0, 0.0, np.nan, 1.0, 1.0, 1.5], np.float32)
+    pulls = np.ones((6, N, S), np.int32)
+    rsum = np.full((6, N, S), 0.25, np.float32)
+    t = np.arange(6, dtype=np.int32) + 7
+    out = oracle.record_outcome(member, arm, t_cur, t_new, pulls, rsum, t)
+    # a regression, a kernel of zero runtime, a NaN measurement, a zero incumbent runtime, nothing drawn, a gain
+    np.testing.assert_allclose(out["reward"], [0.0, 1.0, 0.0, 0.0, 0.0, 0.25], atol=1e-7)
+    np.testing.assert_array_equal(out["t"], t + 1)
+    want_p, want_r = pulls.copy(), rsum.copy()
+    for b, upd in enumerate([(0, 2, 0.0), (0, 2, 1.0), (1, 1, 0.0), (2, 0, 0.0), None, (3, 2, 0.25)]):
+        if upd is not None:
+            k, s, r = upd
+            want_p[b, k, s] += 1
+            want_r[b, k, s] += r
+    np.testing.assert_array_equal(out["pulls"], want_p)
+    np.testing.assert_allclose(out["reward_sum"], want_r, atol=1e-7)
+    # failed verification: Algorithm 1 leaves the statistics alone; the formal model's reading counts a zero
+    ver = np.array([1, 0, 1, 1, 1, 0], np.int32)
+    a1 = oracle.record_outcome(member, arm, t_cur, t_new, pulls, rsum, t, verified=ver)
+    assert a1["pulls"][1].tolist() == pulls[1].tolist() and a1["pulls"][5].tolist() == pulls[5].tolist()
+    assert a1["reward"][1] == 0.0 and a1["reward"][5] == 0.0 and a1["t"][1] == t[1] + 1
+    np.testing.assert_array_equal(a1["pulls"][[0, 2, 3]], want_p[[0, 2, 3]])
+    fm = oracle.record_outcome(member, arm, t_cur, t_new, pulls, rsum, t, verified=ver, failures_count=True)
+    assert fm["pulls"][1, 0, 2] == 2 and fm["reward_sum"][1, 0, 2] == pytest.approx(0.25)
+    assert fm["pulls"][5, 3, 2] == 2 and fm["reward_sum"][5, 3, 2] == pytest.approx(0.25) and fm["reward"][5] == 0.0
