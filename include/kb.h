@@ -94,7 +94,7 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_INIT 5
 #define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
 #define KB_T_ASSIGN_KERNEL 7 /* the tensor-core contraction kernel alone (nested inside KB_T_ASSIGN or KB_T_FIT) */
-#define KB_T_SAMPLE 8 /* kb_sample_member */
+#define KB_T_SAMPLE 8 /* kb_sample_member, kb_record_outcome */
 #define KB_T_COUNT 9
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
@@ -217,6 +217,33 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
                            const int32_t* cluster_arm, const float* h_cand, const int32_t* target,
                            float theta_sat, uint64_t seed, const int32_t* t, int32_t* member,
                            float* member_val);
+
+/* Outcome of one iteration (Sec. 2.2 "Formal Model": r_t = Clip((L(k_t) -
+ * L(k'_t)) / L(k_t), 0, 1); Algorithm 1, "Generation & update": N <- N + 1,
+ * mu <- mu + (r_t - mu) / N for the chosen pair).  The statistics are kept per
+ * arm as (pulls, reward_sum), from which kb_score_select forms N_{i,s} and
+ * mu_{i,s} per cluster in closed form; the update of the pair (I_t, S_t)
+ * through its drawn member k_t is
+ *   pulls[k_t][S_t] += 1,  reward_sum[k_t][S_t] += r_t,  t += 1.
+ * A regression, a NaN ratio or L(k_t) <= 0 gives r_t = 0.  When verification
+ * failed (verified[b] == 0): failures_count == 0 leaves the statistics alone
+ * (Algorithm 1), non-zero records one pull with reward 0 (the formal model's
+ * "zero reward ... to compilation failures").  t advances in every case (it
+ * is the loop index); member[b] < 0 (nothing drawn) changes nothing else.
+ *   member [B] in: k_t as kb_sample_member writes it
+ *   cluster_arm [B] in: I_t*S + S_t as kb_score_select writes best_cluster_arm
+ *   t_cur [B][N] in: L(k) of every candidate;  t_new [B] in: L(k'_t)
+ *   verified [B] in, nullable = every k'_t passed
+ *   pulls, reward_sum [B][N][S] in/out;  t [B] in/out
+ *   reward [B] out, nullable: r_t as recorded (0 where nothing was updated)
+ * All arrays in DEVICE memory.  member >= N, or a negative cluster_arm beside
+ * a drawn member, sets bit 4 of the device status word and updates nothing.
+ * One launch, no workspace; meant to be chained after kb_score_select and
+ * kb_sample_member on one stream (or inside one CUDA graph). */
+kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,
+                            const int32_t* cluster_arm, const float* t_cur, const float* t_new,
+                            const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
+                            float* reward);
 
 /* Which kernel kb_cluster_assign uses.
  *   path: 0 = automatic (tensor cores when K >= 128, D a multiple of 32 and

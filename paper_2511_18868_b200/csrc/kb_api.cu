@@ -344,6 +344,20 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
                                    member_val);
 }
 
+kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,
+                            const int32_t* cluster_arm, const float* t_cur, const float* t_new,
+                            const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t, float* reward) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, S >= 1, "kb_record_outcome: S must be >= 1");
+    if (B > 0) {
+        KB_REQUIRE(ctx, member && cluster_arm && t_new && t, "kb_record_outcome: member, cluster_arm, t_new and t are required");
+        if (N > 0) KB_REQUIRE(ctx, t_cur && pulls && reward_sum, "kb_record_outcome: t_cur, pulls and reward_sum are required");
+    }
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_record_outcome(ctx, B, N, S, failures_count, member, cluster_arm, t_cur, t_new, verified, pulls,
+                                    reward_sum, t, reward);
+}
+
 kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
                             float* centroids) {
     KB_COMMON(ctx, B, N);

@@ -135,6 +135,10 @@ kb_status kb_launch_score(kb_ctx*, int B, int N, int K, int S, kb_score_params p
                           const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
                           const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
                           float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm);
+kb_status kb_launch_record_outcome(kb_ctx*, int B, int N, int S, int failures_count, const int32_t* member,
+                                   const int32_t* cluster_arm, const float* t_cur, const float* t_new,
+                                   const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
+                                   float* reward);
 size_t kb_ws_need_sample(int B);
 kb_status kb_launch_sample_member(kb_ctx*, int B, int N, int K, int S, int R, const int32_t* labels,
                                   const int32_t* cluster_arm, const float* h_cand, const int32_t* target,

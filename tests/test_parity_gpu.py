@@ -810,3 +810,112 @@ def test_sample_member_frequencies(kbx):
     p /= p.sum()
     freq = counts / (M * rounds)
     assert np.all(np.abs(freq - p) < 4.5 * np.sqrt(p * (1 - p) / (M * rounds))), (freq, p)
+
+
+# -------------------------------------------------- outcome of an iteration
+@pytest.mark.parametrize("B,N,S", [(1, 256, 8), (37, 1000, 3), (1024, 64, 16), (5, 1, 1)])
+@pytest.mark.parametrize("failures_count", [False, True])
+def test_record_outcome(kbx, B, N, S, failures_count):
+    rng = np.random.default_rng(B + N + S)
+    member = rng.integers(0, N, size=(B,)).astype(np.int32)
+    member[rng.uniform(size=B) < 0.1] = -1
+    arm = rng.integers(0, 4 * S, size=(B,)).astype(np.int32)
+    t_cur = rng.uniform(0.5, 20.0, size=(B, N)).astype(np.float32)
+    t_cur[rng.uniform(size=(B, N)) < 0.02] = 0.0
+    base = t_cur[np.arange(B), np.maximum(member, 0)]
+    t_new = (base * rng.uniform(0.0, 1.6, size=B)).astype(np.float32)   # gains and regressions
+    t_new[rng.uniform(size=B) < 0.05] = np.nan
+    verified = (rng.uniform(size=B) < 0.8).astype(np.int32)
+    pulls = rng.poisson(2.0, size=(B, N, S)).astype(np.int32)
+    rsum = (pulls * rng.uniform(0, 1, size=(B, N, S))).astype(np.float32)
+    t = rng.integers(1, 1000, size=B).astype(np.int32)
+    for ver in (None, verified):
+        ref = oracle.record_outcome(member, arm, t_cur, t_new, pulls, rsum, t, verified=ver,
+                                    failures_count=failures_count)
+        p_d, r_d, t_d, rew = dev(pulls), dev(rsum), dev(t), empty((B,))
+        kbx.record_outcome(dev(member), dev(arm), dev(t_cur), dev(t_new), p_d, r_d, t_d,
+                           verified=None if ver is None else dev(ver), reward=rew, failures_count=failures_count)
+        np.testing.assert_array_equal(host(p_d), ref["pulls"])
+        np.testing.assert_array_equal(host(t_d), ref["t"])
+        # the ratio is one fp32 division here, a double one rounded once in the oracle
+        parity.close(host(rew), ref["reward"], atol=1e-7, what="reward")
+        parity.close(host(r_d), ref["reward_sum"], atol=1e-6, what="reward_sum")
+    assert kbx.device_status() == 0
+
+
+@pytest.mark.parametrize("use_graph", [False, True])
+def test_lockstep_loop_stays_on_device(kbx, use_graph):
+    """B searches in lock-step: select the pair, draw k_t, observe a synthetic outcome, record it -- T iterations
+    queued on one stream, no host read in between; with use_graph the iteration is captured once into a CUDA graph
+    and replayed (the draw still changes from replay to replay: its counter holds t, which the graph itself
+    advances).  Afterwards every iteration is checked against the oracle, fed the state the GPU had at that point
+    (the copies below are queued on the same stream, outside the iteration)."""
+    B, N, K, S, T = 6, 700, 5, 4, 25
+    cfg = wl.scaled(wl.CONFIGS["medium"], B=B, N=N, D=16, K=K, components=5, S=S, iters=3)
+    inp = wl.make_inputs(cfg, seed=5)
+    rng = np.random.default_rng(9)
+    labels = rng.integers(0, K, size=(B, N)).astype(np.int32)
+    dist2 = rng.uniform(0, 4, size=(B, N)).astype(np.float32)
+    h_cand = wl.make_candidate_signatures(inp["hsig"], labels, seed=3)
+    gain = rng.uniform(-0.3, 0.6, size=(B, N, S)).astype(np.float32)     # the synthetic environment: L' = L (1 - gain)
+    ws(kbx, B, N, 16, K, S)
+    d = {k: dev(v) for k, v in dict(labels=labels, dist2=dist2, pulls=inp["pulls"], reward_sum=inp["reward_sum"],
+                                    t=inp["t"], h_cand=h_cand, target=inp["target"], t_cur=inp["t_cur"],
+                                    gain=gain).items()}
+    cl = [empty((B, K, S)) for _ in range(3)]
+    best_arm, best_val, pair = empty((B,), torch.int32), empty((B,)), empty((B,), torch.int32)
+    member, reward = empty((B,), torch.int32), empty((B,))
+    t_new = empty((B,))
+    ar = torch.arange(B, device="cuda")
+
+    def iteration():
+        kbx.score_select(d["labels"], d["dist2"], d["pulls"], d["reward_sum"], d["t"], cl[0], cl[1], cl[2], best_arm,
+                         best_val, pair, lipschitz_L=0.1)
+        kbx.sample_member(d["labels"], pair, d["h_cand"], d["target"], d["t"], member, K, 75.0, 4242)
+        # environment (test scaffolding, device-side): the runtime of the generated kernel
+        k = member.clamp(min=0).long()
+        s = (pair.clamp(min=0) % S).long()
+        t_new.copy_(d["t_cur"][ar, k] * (1.0 - d["gain"][ar, k, s]))
+        kbx.record_outcome(member, pair, d["t_cur"], t_new, d["pulls"], d["reward_sum"], d["t"], reward=reward)
+
+    graph = None
+    if use_graph:
+        main = torch.cuda.current_stream()
+        side = torch.cuda.Stream()
+        side.wait_stream(main)
+        kbx.set_stream(side)
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                iteration()
+        finally:
+            kbx.set_stream(main)
+        main.wait_stream(side)
+    trace = []
+    for it in range(T):
+        before = (d["pulls"].clone(), d["reward_sum"].clone(), d["t"].clone())
+        if graph is not None:
+            graph.replay()
+        else:
+            iteration()
+        trace.append((before, pair.clone(), member.clone(), t_new.clone(), reward.clone(),
+                      (d["pulls"].clone(), d["reward_sum"].clone(), d["t"].clone())))
+    torch.cuda.synchronize()
+    assert kbx.device_status() == 0
+    drawn = 0
+    for before, pair_g, member_g, t_new_g, reward_g, after in trace:
+        p0, r0, t0 = (host(x) for x in before)
+        sc = oracle.score_select(labels, dist2, p0, r0, t0, K, c=2.0, lipschitz_L=0.1)
+        parity.cluster_select_match(host(pair_g), sc, sc["cl_index"])
+        dr = oracle.sample_member(labels, host(pair_g), h_cand, inp["target"], 75.0, 4242, t0, K)
+        parity.member_match(host(member_g), None, dr, SAMPLE_TOL)
+        ro = oracle.record_outcome(host(member_g), host(pair_g), inp["t_cur"], host(t_new_g), p0, r0, t0)
+        np.testing.assert_array_equal(host(after[0]), ro["pulls"])
+        np.testing.assert_array_equal(host(after[2]), ro["t"])
+        parity.close(host(after[1]), ro["reward_sum"], atol=1e-6, what="reward_sum")
+        parity.close(host(reward_g), ro["reward"], atol=1e-7, what="reward")
+        drawn += int((host(member_g) >= 0).sum())
+    assert drawn == B * T
+    # the loop moved: T pulls were added per instance, and the iteration counters advanced by T
+    assert int(host(d["pulls"]).sum() - inp["pulls"].sum()) == B * T
+    np.testing.assert_array_equal(host(d["t"]), inp["t"] + T)
