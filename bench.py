@@ -395,7 +395,55 @@ def run_ours(args, cfg):
     sample_line = {"avg_us": smp_us, "algorithmic_bytes": smp_bytes, "GBps": smp_bytes / (smp_us * 1e-6) / 1e9,
                    "kernels_per_call": (ks1 - ks0) / args.steps, "members_of_chosen_clusters": members,
                    "what": "kb_sample_member on the step's labels and chosen pairs (not part of the timed step)"}
-    del h_cand
+    # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
+    # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
+    # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
+    loop_t = {k: dev_t[k].clone() for k in ("pulls", "reward_sum", "t")}
+    t_new = (dev_t["t_cur"][:, 0] * 0.9).contiguous()
+    outs = {k: dev_t[k] for k in ("cl_pulls", "cl_mean", "cl_index", "best_arm", "best_val", "best_cluster_arm")}
+
+    def iteration():
+        ctx.score_select(dev_t["labels"], dev_t["dist2"], loop_t["pulls"], loop_t["reward_sum"], loop_t["t"],
+                         outs["cl_pulls"], outs["cl_mean"], outs["cl_index"], outs["best_arm"], outs["best_val"],
+                         outs["best_cluster_arm"], keep=dev_t["keep"], lipschitz_L=float(inp["lipschitz_L"]))
+        ctx.sample_member(dev_t["labels"], outs["best_cluster_arm"], h_cand, dev_t["target"], loop_t["t"], member,
+                          cfg.K, float(inp["theta_sat"]), 0xC0FFEE)
+        ctx.record_outcome(member, outs["best_cluster_arm"], dev_t["t_cur"], t_new, loop_t["pulls"],
+                           loop_t["reward_sum"], loop_t["t"])
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        barrier()
+        return a.elapsed_time(b) / n * 1e3
+
+    kl0, _ = ctx.launch_count()
+    iteration()
+    kl1, _ = ctx.launch_count()
+    n_loop = max(args.steps, 20)
+    eager_us = timed(iteration, n_loop)
+    main_stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(main_stream)
+    ctx.set_stream(side)
+    try:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            iteration()
+    finally:
+        ctx.set_stream(main_stream)
+    main_stream.wait_stream(side)
+    graph_us = timed(graph.replay, n_loop)
+    loop_line = {"eager_us": eager_us, "graph_us": graph_us, "kernels": int(kl1 - kl0), "iterations_timed": n_loop,
+                 "what": "kb_score_select + kb_sample_member + kb_record_outcome on the step's labels, consecutive "
+                         "iterations (L2 not flushed), per rank"}
+    del h_cand, graph
 
     # ---- max over ranks -----------------------------------------------------------
     total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], dist, device)
@@ -481,7 +529,7 @@ def run_ours(args, cfg):
         "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
         "device_status": int(status), "peaks": peaks,
         "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
-        "sample_member": sample_line,
+        "sample_member": sample_line, "online_iteration": loop_line,
     }
     print(json.dumps(line))
     ctx.close()
