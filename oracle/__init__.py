@@ -195,6 +195,30 @@ def record_outcome(member, cluster_arm, t_cur, t_new, pulls, reward_sum, t, veri
     return {"pulls": pulls, "reward_sum": reward_sum, "t": t, "reward": reward}
 
 
+def kmeanspp_round(z, chosen, seed, want_pert=True, want_weights=False):
+    """One round of k-means++ seeding given the rows chosen so far (chosen [B][round]); see kbo_kmeanspp_round."""
+    z = _f32(z)
+    chosen = _i32(chosen)
+    B, N, D = z.shape
+    rnd = chosen.shape[1]
+    row = np.empty((B,), np.int32)
+    pert = np.empty((B, N), np.float64) if want_pert else None
+    w = np.empty((B, N), np.float64) if want_weights else None
+    _check(_load().kbo_kmeanspp_round(B, N, D, rnd, _p(z), _p(chosen), max(rnd, 1),
+                                      ctypes.c_uint64(int(seed) & (2**64 - 1)), _p(row), _p(pert), _p(w)),
+           "kmeanspp_round")
+    return {"row": row, "pert": pert, "weights": w}
+
+
+def kmeanspp(z, K, seed):
+    """k-means++ seeding: rows [B][K] (see kbo_kmeanspp)."""
+    z = _f32(z)
+    B, N, D = z.shape
+    rows = np.zeros((B, K), np.int32)
+    _check(_load().kbo_kmeanspp(B, N, D, K, _p(z), ctypes.c_uint64(int(seed) & (2**64 - 1)), _p(rows)), "kmeanspp")
+    return rows
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

@@ -452,4 +452,75 @@ int kbo_record_outcome(int B, int N, int S, int failures_count, const int32_t* m
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// k-means++ seeding (Arthur & Vassilvitskii, "k-means++: the advantages of careful seeding", SODA'07;
+// what "scikit-learn's KMeans" of Sec. 3.5 starts from by default, here without its extra greedy
+// trials): the first centre is a row drawn uniformly; every further centre is a row drawn with
+// probability D(x)^2 / sum D^2, D(x) = distance of x to the nearest centre chosen so far.
+//
+// Each draw is a Gumbel-max over the weights w (1 in round 0, D^2 afterwards): the row with the
+// largest ln(w) + G wins, G = -ln(-ln u), u from the counter-based generator at
+//     counter = (row, instance, round, 1),  key = (low, high word of seed),
+//     u = ((first output word >> 9) + 0.5) * 2^-23;
+// rows of weight 0 (chosen rows and their duplicates) are never drawn.  If every weight is 0 (fewer
+// distinct rows than K) the round draws uniformly among all rows instead (weights 1, same G).
+//
+// One round, given the centres chosen so far (so that a test can follow another implementation's
+// choices round by round): chosen[B][round] in; row[B] out; pert (optional, double [B][N]) the
+// perturbed value of every drawable row (-inf elsewhere); mind2 (optional, double [B][N]) the
+// weights D^2 of the round (1 in round 0).
+// ---------------------------------------------------------------------------
+int kbo_kmeanspp_round(int B, int N, int D, int round, const float* z, const int32_t* chosen, int chosen_stride,
+                       uint64_t seed, int32_t* row, double* pert, double* mind2) {
+    if (N < 1) return 1;
+    const uint32_t key[2] = {(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32)};
+    std::vector<double> w(N);
+    for (int b = 0; b < B; ++b) {
+        bool any = false;
+        for (int k = 0; k < N; ++k) {
+            double m = round == 0 ? 1.0 : kInf;
+            for (int j = 0; j < round; ++j) {
+                const int c = chosen[(size_t)b * chosen_stride + j];
+                if (c < 0 || c >= N) return 2;
+                double d2 = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    const double e = (double)z[ix3(b, k, d, N, D)] - (double)z[ix3(b, c, d, N, D)];
+                    d2 += e * e;
+                }
+                if (d2 < m) m = d2;
+            }
+            w[k] = m;
+            if (m > 0.0) any = true;
+        }
+        double best = -kInf;
+        int arg = -1;
+        for (int k = 0; k < N; ++k) {
+            const double wk = any ? w[k] : 1.0;
+            if (mind2) mind2[ix2(b, k, N)] = wk;
+            if (pert) pert[ix2(b, k, N)] = -kInf;
+            if (!(wk > 0.0)) continue;
+            const uint32_t ctr[4] = {(uint32_t)k, (uint32_t)b, (uint32_t)round, 1u};
+            uint32_t rnd[4];
+            kbo_philox4x32_10(ctr, key, rnd);
+            const double u = ((double)(rnd[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+            const double v = std::log(wk) - std::log(-std::log(u));
+            if (pert) pert[ix2(b, k, N)] = v;
+            if (v > best) { best = v; arg = k; }
+        }
+        row[b] = arg;
+    }
+    return 0;
+}
+
+// All K rounds, each fed the rows this function chose before: rows[B][K].
+int kbo_kmeanspp(int B, int N, int D, int K, const float* z, uint64_t seed, int32_t* rows) {
+    std::vector<int32_t> r(B > 0 ? B : 1);
+    for (int j = 0; j < K; ++j) {
+        const int rc = kbo_kmeanspp_round(B, N, D, j, z, rows, K, seed, r.data(), nullptr, nullptr);
+        if (rc) return rc;
+        for (int b = 0; b < B; ++b) rows[(size_t)b * K + j] = r[b];
+    }
+    return 0;
+}
+
 }  // extern "C"

@@ -540,3 +540,51 @@ def test_record_outcome_clip_and_failures():
     fm = oracle.record_outcome(member, arm, t_cur, t_new, pulls, rsum, t, verified=ver, failures_count=True)
     assert fm["pulls"][1, 0, 2] == 2 and fm["reward_sum"][1, 0, 2] == pytest.approx(0.25)
     assert fm["pulls"][5, 3, 2] == 2 and fm["reward_sum"][5, 3, 2] == pytest.approx(0.25) and fm["reward"][5] == 0.0
+
+
+# --------------------------------------------------------- k-means++ seeding
+def test_kmeanspp_rounds_follow_the_d2_weights():
+    """Round 0 is uniform; a later round draws row x with probability D(x)^2 / sum D^2, D the distance to the NEAREST
+    chosen centre (weights computed here from the definition with scipy's cdist)."""
+    pts = np.array([[0, 0], [1, 0], [0, 2], [3, 3], [-2, 1], [0.5, 0.5], [4, 0], [1, 0]], np.float32)   # rows 1, 7 equal
+    M, N = 100000, len(pts)
+    z = np.broadcast_to(pts, (M, N, 2)).copy()
+    r0 = oracle.kmeanspp_round(z, np.zeros((M, 0), np.int32), seed=11)["row"]
+    f0 = np.bincount(r0, minlength=N) / M
+    assert np.all(np.abs(f0 - 1 / N) < 4.5 * np.sqrt((1 / N) * (1 - 1 / N) / M))
+    for chosen in ([1], [3, 0], [6, 4, 1]):
+        out = oracle.kmeanspp_round(z, np.tile(np.array(chosen, np.int32), (M, 1)), seed=12, want_weights=True)
+        d2 = scipy.spatial.distance.cdist(pts.astype(np.float64), pts[chosen].astype(np.float64), "sqeuclidean").min(axis=1)
+        p = d2 / d2.sum()
+        np.testing.assert_allclose(out["weights"][0], d2, rtol=1e-12)
+        f = np.bincount(out["row"], minlength=N) / M
+        assert np.all(np.abs(f - p) < 4.5 * np.sqrt(p * (1 - p) / M) + 1e-12), (chosen, f, p)
+        assert f[chosen].max() == 0.0                        # a chosen row (and its duplicate) is never drawn again
+        if 1 in chosen:
+            assert f[7] == 0.0
+
+
+def test_kmeanspp_full_seeding():
+    rng = np.random.default_rng(3)
+    # well separated blobs: D^2 seeding puts one seed in every blob nearly always; uniform seeding would manage
+    # that for K = 6 equal blobs only 6!/6^6 = 1.5 % of the time
+    K, per, B = 6, 40, 300
+    centres = 100.0 * np.stack([np.cos(2 * np.pi * np.arange(K) / K), np.sin(2 * np.pi * np.arange(K) / K)], 1)
+    z = (centres[None, :, None, :] + rng.standard_normal((B, K, per, 2))).reshape(B, K * per, 2).astype(np.float32)
+    rows = oracle.kmeanspp(z, K, seed=99)
+    assert rows.min() >= 0 and rows.max() < K * per
+    blobs = rows // per
+    hit = np.mean([len(set(b)) == K for b in blobs])
+    assert hit > 0.97, hit
+    # the whole seeding is its rounds, each fed the rows chosen before
+    for j in range(K):
+        np.testing.assert_array_equal(oracle.kmeanspp_round(z, rows[:, :j], seed=99)["row"], rows[:, j])
+    # fewer distinct rows than K: still K valid rows (the surplus rounds draw uniformly)
+    dup = np.zeros((50, 7, 3), np.float32)
+    dup[:, 3:, :] = 1.0
+    r = oracle.kmeanspp(dup, 4, seed=5)
+    assert r.min() >= 0 and r.max() < 7
+    assert np.all((r[:, 0] < 3) != (r[:, 1] < 3))            # the second seed is always the other point
+    # another seed, other seeds; the same seed, the same ones
+    np.testing.assert_array_equal(oracle.kmeanspp(z[:20], K, seed=99), rows[:20])
+    assert np.any(oracle.kmeanspp(z[:20], K, seed=100) != rows[:20])
