@@ -218,6 +218,24 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
                            float theta_sat, uint64_t seed, const int32_t* t, int32_t* member,
                            float* member_val);
 
+/* k-means++ seeding (Arthur & Vassilvitskii, SODA'07; the initialisation of
+ * the "scikit-learn's KMeans" of Sec. 3.5, without its extra greedy trials):
+ * rows[b][0] is a row of instance b drawn uniformly, rows[b][j] a row drawn
+ * with probability D(x)^2 / sum D^2, D(x) = distance of x to the nearest of
+ * the j centres chosen before.  Each draw is a Gumbel-max over the weights w
+ * (1 in round 0, D^2 after): the row with the largest ln(w) + G, G = -ln(-ln u),
+ * u from Philox4x32-10 at counter (row, instance, round, 1), key = the halves
+ * of seed, u = ((first word >> 9) + 0.5) * 2^-23.  Rows of weight 0 (chosen
+ * rows, their duplicates) are never drawn; when every weight is 0 (fewer
+ * distinct rows than K) the round draws uniformly among all rows.  The result
+ * feeds kb_init_centroids or the init_rows of kb_bandit_step.
+ *   z [B][N][D] in (N >= 1);  rows [B][K] out, values in [0, N)
+ * DEVICE memory; seed by value.  K launches (one per round, each reading z
+ * once); needs the workspace of kb_workspace_bytes (4 bytes per row plus 20
+ * per centre).  fp32 distances in the direct form. */
+kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
+                           int32_t* rows);
+
 /* Outcome of one iteration (Sec. 2.2 "Formal Model": r_t = Clip((L(k_t) -
  * L(k'_t)) / L(k_t), 0, 1); Algorithm 1, "Generation & update": N <- N + 1,
  * mu <- mu + (r_t - mu) / N for the chosen pair).  The statistics are kept per

@@ -179,6 +179,7 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     need = max_sz(need, kb_ws_need_normalize(B, N, D));
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
     need = max_sz(need, kb_ws_need_sample(B));
+    need = max_sz(need, kb_ws_need_seed(B, N, K));
     need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K));
     *out = need;
     return KB_OK;
@@ -342,6 +343,17 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
     TimeScope ts__(ctx, KB_T_SAMPLE);
     return kb_launch_sample_member(ctx, B, N, K, S, R, labels, cluster_arm, h_cand, target, theta_sat, seed, t, member,
                                    member_val);
+}
+
+kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed, int32_t* rows) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_seed_kmeanspp: D and K must be >= 1");
+    if (B > 0) {
+        KB_REQUIRE(ctx, N >= 1, "kb_seed_kmeanspp: needs at least one row to draw from");
+        KB_REQUIRE(ctx, z && rows, "kb_seed_kmeanspp: z and rows are required");
+    }
+    TimeScope ts__(ctx, KB_T_INIT);
+    return kb_launch_seed_kmeanspp(ctx, B, N, D, K, z, seed, rows);
 }
 
 kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,

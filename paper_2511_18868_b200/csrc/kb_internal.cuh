@@ -139,6 +139,8 @@ kb_status kb_launch_record_outcome(kb_ctx*, int B, int N, int S, int failures_co
                                    const int32_t* cluster_arm, const float* t_cur, const float* t_new,
                                    const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
                                    float* reward);
+size_t kb_ws_need_seed(int B, int N, int K);
+kb_status kb_launch_seed_kmeanspp(kb_ctx*, int B, int N, int D, int K, const float* z, uint64_t seed, int32_t* rows);
 size_t kb_ws_need_sample(int B);
 kb_status kb_launch_sample_member(kb_ctx*, int B, int N, int K, int S, int R, const int32_t* labels,
                                   const int32_t* cluster_arm, const float* h_cand, const int32_t* target,
@@ -199,6 +201,25 @@ __device__ __forceinline__ float kb_div_by(float a, float d, float r) {
     const float e = fmaf(-q0, d, a);
     return fmaf(e, r, q0);     // d = 0 or a non-finite operand gives NaN here, which the callers map like 0/0
 }
+// Philox4x32 with 10 rounds (Salmon et al., SC'11): first output word only.
+__device__ __forceinline__ uint32_t kb_philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                       uint32_t k0, uint32_t k1) {
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += W0;
+        k1 += W1;
+    }
+    return c0;
+}
+// the uniform in (0, 1) the draws use: 23 bits of the word, centred, exact in fp32
+__device__ __forceinline__ float kb_uniform23(uint32_t w) { return ((float)(w >> 9) + 0.5f) * (1.0f / 8388608.0f); }
 // monotone map float -> uint32 (larger float <=> larger uint)
 __device__ __forceinline__ uint32_t kb_orderable(float f) {
     uint32_t u = __float_as_uint(f);

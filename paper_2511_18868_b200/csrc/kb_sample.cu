@@ -22,24 +22,6 @@ constexpr int SM_T = 256;      // threads per CTA
 constexpr int SM_U = 4;        // label loads in flight per thread
 constexpr int SM_ROWS = SM_T * SM_U * 4;   // rows per CTA at least (when the instance is split): one vector trip
 
-// Philox4x32 with 10 rounds (Salmon et al., SC'11): first output word only.
-__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                       uint32_t k0, uint32_t k1) {
-    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
-        k0 += W0;
-        k1 += W1;
-    }
-    return c0;
-}
-
 struct SampleWs {
     unsigned long long* key;   // [B] packed (perturbed value, inverted row)
     unsigned* done;            // [B] CTAs of the instance that have finished
@@ -90,7 +72,7 @@ sample_member_kernel(int N, int K, int S, int R, int rows_per, int G, const int3
         // one candidate of the chosen cluster: signature entry, uniform, perturbed value, packed key
         auto take = [&](int r) {
             const float h = __ldg(hb + (size_t)r * R);
-            const uint32_t w0 = philox4x32_10_word0((uint32_t)r, (uint32_t)b, tb, 0u, seed_lo, seed_hi);
+            const uint32_t w0 = kb_philox4x32_10_word0((uint32_t)r, (uint32_t)b, tb, 0u, seed_lo, seed_hi);
             const float uni = ((float)(w0 >> 9) + 0.5f) * (1.0f / 8388608.0f);   // 23 bits: exact
             const float v = (theta - h) - logf(-logf(uni));
             if (!(v > -INFINITY)) return;                                        // NaN or -inf: never drawn

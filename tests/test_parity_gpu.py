@@ -919,3 +919,82 @@ def test_lockstep_loop_stays_on_device(kbx, use_graph):
     # the loop moved: T pulls were added per instance, and the iteration counters advanced by T
     assert int(host(d["pulls"]).sum() - inp["pulls"].sum()) == B * T
     np.testing.assert_array_equal(host(d["t"]), inp["t"] + T)
+
+
+# --------------------------------------------------------- k-means++ seeding
+def _follow_seeding(z, rows, seed, tol=SAMPLE_TOL):
+    """Every round's row must be the largest perturbed value ln(D^2) + G given the rows the GPU chose before (the
+    oracle's double values; where its two largest are closer than the fp32 tolerance either is a valid draw)."""
+    B, K = rows.shape
+    loose = 0
+    for j in range(K):
+        o = oracle.kmeanspp_round(z, rows[:, :j], seed)
+        for b in range(B):
+            g = int(rows[b, j])
+            assert 0 <= g < z.shape[1]
+            if g != o["row"][b]:
+                assert o["pert"][b, g] >= o["pert"][b, o["row"][b]] - tol, \
+                    f"round {j}, instance {b}: drew {g} ({o['pert'][b, g]}), oracle {o['row'][b]} ({o['pert'][b, o['row'][b]]})"
+                loose += 1
+    return loose
+
+
+@pytest.mark.parametrize("B,N,D,K", [(1, 256, 16, 8), (3, 1000, 20, 5), (2, 5003, 5, 7), (1, 40000, 64, 24),
+                                     (40, 512, 32, 16), (2, 1, 8, 1), (1, 3000, 128, 3)])
+def test_seed_kmeanspp(kbx, B, N, D, K):
+    cfg = wl.scaled(wl.CONFIGS["medium"], B=B, N=N, D=D, K=max(K, 2), components=max(2, K), S=4, iters=1)
+    x = wl.make_inputs(cfg, seed=N + K)["x"]
+    z, _, _ = oracle.normalize(x)
+    ws(kbx, B, N, D, K, 4)
+    rows = empty((B, K), torch.int32)
+    kbx.seed_kmeanspp(dev(z), rows, seed=2025 + N)
+    got = host(rows)
+    loose = _follow_seeding(z, got, 2025 + N)
+    assert loose <= max(1, B * K // 50)
+    if N >= K:
+        assert all(len(set(r.tolist())) == K for r in got)          # distinct data: distinct seeds
+    again = empty((B, K), torch.int32)
+    kbx.seed_kmeanspp(dev(z), again, seed=2025 + N)
+    np.testing.assert_array_equal(host(again), got)
+    assert kbx.device_status() == 0
+
+
+def test_seed_kmeanspp_properties(kbx):
+    rng = np.random.default_rng(3)
+    K, per, B = 6, 40, 300
+    centres = 100.0 * np.stack([np.cos(2 * np.pi * np.arange(K) / K), np.sin(2 * np.pi * np.arange(K) / K)], 1)
+    z = (centres[None, :, None, :] + rng.standard_normal((B, K, per, 2))).reshape(B, K * per, 2).astype(np.float32)
+    ws(kbx, B, K * per, 2, K, 4)
+    rows = empty((B, K), torch.int32)
+    kbx.seed_kmeanspp(dev(z), rows, seed=99)
+    got = host(rows)
+    hit = np.mean([len(set(b)) == K for b in got // per])
+    assert hit > 0.97, hit                                           # one seed per blob (uniform seeding: 1.5 %)
+    _follow_seeding(z, got, 99)
+    # fewer distinct rows than K: the surplus rounds draw uniformly, every row stays valid
+    dup = np.zeros((50, 7, 4), np.float32)
+    dup[:, 3:, :] = 1.0
+    rows = empty((50, 4), torch.int32)
+    ws(kbx, 50, 7, 4, 4, 4)
+    kbx.seed_kmeanspp(dev(dup), rows, seed=5)
+    r = host(rows)
+    assert r.min() >= 0 and r.max() < 7
+    assert np.all((r[:, 0] < 3) != (r[:, 1] < 3))
+    _follow_seeding(dup, r, 5)
+    # the rows feed the clustering: seeding, gather, fit on the device without a host read in between
+    cfg = wl.scaled(wl.CONFIGS["medium"], B=2, N=6000, D=32, K=12, components=12, S=4, iters=5)
+    zz, _, _ = oracle.normalize(wl.make_inputs(cfg, seed=8)["x"])
+    ws(kbx, 2, 6000, 32, 12, 4)
+    zd, rows, c = dev(zz), empty((2, 12), torch.int32), empty((2, 12, 32))
+    labels, inertia = empty((2, 6000), torch.int32), empty((2,))
+    kbx.seed_kmeanspp(zd, rows, seed=1)
+    kbx.init_centroids(zd, rows, c)
+    kbx.cluster_fit(zd, c, labels, 5, inertia=inertia)
+    c0 = oracle.init_centroids(zz, host(rows))
+    ref_c = c0
+    for _ in range(5):
+        a = oracle.cluster_assign(zz, ref_c, want_rep=False)
+        ref_c, _ = oracle.cluster_update(zz, a["labels"], ref_c)
+    a = oracle.cluster_assign(zz, ref_c, want_rep=False)
+    parity.close(host(inertia), a["inertia"], atol=0, rtol=1e-3, what="inertia after seeded fit")
+    assert kbx.device_status() == 0
