@@ -395,6 +395,26 @@ def run_ours(args, cfg):
     sample_line = {"avg_us": smp_us, "algorithmic_bytes": smp_bytes, "GBps": smp_bytes / (smp_us * 1e-6) / 1e9,
                    "kernels_per_call": (ks1 - ks0) / args.steps, "members_of_chosen_clusters": members,
                    "what": "kb_sample_member on the step's labels and chosen pairs (not part of the timed step)"}
+    # ---- k-means++ seeding of the step's z (an alternative to caller-supplied initial rows; outside the timed step)
+    seed_rows = torch.empty((cfg.B, cfg.K), dtype=torch.int32, device=device)
+    ctx.seed_kmeanspp(dev_t["z"], seed_rows, 1)
+    barrier()
+    kq0, _ = ctx.launch_count()
+    sa, sb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush.zero_()
+    sa.record()
+    ctx.seed_kmeanspp(dev_t["z"], seed_rows, 2)
+    sb.record()
+    barrier()
+    kq1, _ = ctx.launch_count()
+    seed_ms = sa.elapsed_time(sb)
+    round_bytes = cfg.B * cfg.N * (cfg.D * 4 + 8)          # z once, min D^2 read and written
+    seed_line = {"ms": seed_ms, "rounds": cfg.K, "us_per_round": seed_ms * 1e3 / cfg.K, "kernels": int(kq1 - kq0),
+                 "algorithmic_bytes_per_round": round_bytes,
+                 "GBps": round_bytes / (seed_ms * 1e-3 / cfg.K) / 1e9,
+                 "hbm_frac": round_bytes / (seed_ms * 1e-3 / cfg.K) / 1e9 / peaks["hbm_gbs"],
+                 "what": "kb_seed_kmeanspp on the step's z: K rounds, one launch each (not part of the timed step)"}
+
     # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
     # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
     # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
@@ -529,7 +549,7 @@ def run_ours(args, cfg):
         "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
         "device_status": int(status), "peaks": peaks,
         "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
-        "sample_member": sample_line, "online_iteration": loop_line,
+        "sample_member": sample_line, "online_iteration": loop_line, "seed_kmeanspp": seed_line,
     }
     print(json.dumps(line))
     ctx.close()

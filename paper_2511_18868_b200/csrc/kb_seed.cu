@@ -56,41 +56,50 @@ seed_round_kernel(int N, int D, int K, int round, int G, int rows_per, const flo
     const float* zc = zb + (size_t)c * D;
     unsigned long long bestW = 0ull, bestU = 0ull;
     constexpr int U = 4;
-    const int step = (SD_T / 32) * rpw;                         // rows per block step
-    // the trip count is the same for every thread of the block, so the shuffles below always run with full
-    // warps; rows past the end are computed on the last row and dropped
-    const int trips = (max(r1 - r0, 0) + U * step - 1) / (U * step);
+    __shared__ float s_d2[SD_T / 32][32];
+    // A warp takes 32 consecutive rows per trip.  Phase 1: lane groups (lpr lanes = the columns of a row) form the
+    // squared distance to the newest centre, U row loads in flight per lane, and leave it in shared memory.
+    // Phase 2: one row per lane -- min with the stored weight (coalesced), the generator, the logarithms, the keys.
+    // The trip count is the same for every thread of the block; rows past the end are computed on the last row
+    // and dropped in phase 2.
+    const int trips = (max(r1 - r0, 0) + SD_T - 1) / SD_T;
     for (int it = 0; it < trips; ++it) {
-        const int rb = r0 + it * U * step + warp * rpw + lane_r;
-        float acc[U];
+        const int base = r0 + (it * (SD_T / 32) + warp) * 32;
+        if (round > 0) {
+            for (int v0 = 0; v0 < 32 / rpw; v0 += U) {
+                float acc[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int r = min(rb + u * step, r1 - 1);
-            float a = 0.f;
-            if (round > 0) {
-                const float* x = zb + (size_t)r * D;
-                for (int q = lane_c; q < vpr; q += lpr) {
-                    if (V == 4) {
-                        const float4 xv = __ldg(reinterpret_cast<const float4*>(x) + q);
-                        const float4 cv = __ldg(reinterpret_cast<const float4*>(zc) + q);
-                        const float e0 = xv.x - cv.x, e1 = xv.y - cv.y, e2 = xv.z - cv.z, e3 = xv.w - cv.w;
-                        a = fmaf(e0, e0, a); a = fmaf(e1, e1, a); a = fmaf(e2, e2, a); a = fmaf(e3, e3, a);
-                    } else {
-                        const float e = __ldg(x + q) - __ldg(zc + q);
-                        a = fmaf(e, e, a);
+                for (int u = 0; u < U; ++u) {
+                    const int r = min(base + (v0 + u) * rpw + lane_r, r1 - 1);
+                    const float* x = zb + (size_t)r * D;
+                    float a = 0.f;
+                    for (int q = lane_c; q < vpr; q += lpr) {
+                        if (V == 4) {
+                            const float4 xv = __ldg(reinterpret_cast<const float4*>(x) + q);
+                            const float4 cv = __ldg(reinterpret_cast<const float4*>(zc) + q);
+                            const float e0 = xv.x - cv.x, e1 = xv.y - cv.y, e2 = xv.z - cv.z, e3 = xv.w - cv.w;
+                            a = fmaf(e0, e0, a); a = fmaf(e1, e1, a); a = fmaf(e2, e2, a); a = fmaf(e3, e3, a);
+                        } else {
+                            const float e = __ldg(x + q) - __ldg(zc + q);
+                            a = fmaf(e, e, a);
+                        }
                     }
+                    acc[u] = a;
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    float a = acc[u];
+                    for (int o = 1; o < lpr; o <<= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                    if (lane_c == 0 && v0 + u < 32 / rpw) s_d2[warp][(v0 + u) * rpw + lane_r] = a;   // (narrow rows: fewer than U steps)
                 }
             }
-            acc[u] = a;
+            __syncwarp();
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float a = acc[u];
-            for (int o = 1; o < lpr; o <<= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            const int r = rb + u * step;
-            if (lane_c != 0 || r >= r1) continue;
+        const int r = base + lane;
+        if (r < r1) {
             float wgt = 1.f;
             if (round > 0) {
+                const float a = s_d2[warp][lane];
                 wgt = round == 1 ? a : fminf(md[r], a);
                 if (round + 1 < K) md[r] = wgt;
             }
@@ -103,6 +112,7 @@ seed_round_kernel(int N, int D, int K, int round, int G, int rows_per, const flo
                 bestW = kw > bestW ? kw : bestW;
             }
         }
+        __syncwarp();                                           // s_d2 is rewritten by the next trip
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -135,7 +145,7 @@ seed_round_kernel(int N, int D, int K, int round, int G, int rows_per, const flo
 
 int seed_ctas(const kb_ctx* ctx, int B, int N) {
     long want = (4L * ctx->sm_count + B - 1) / B;
-    long cap = ((long)N + 511) / 512;                            // at least 512 rows per CTA
+    long cap = ((long)N + SD_T - 1) / SD_T;                      // at least one trip of rows per CTA
     long g = want < cap ? want : cap;
     return (int)(g < 1 ? 1 : g);
 }
