@@ -219,6 +219,15 @@ def kmeanspp(z, K, seed):
     return rows
 
 
+def cluster_radius(labels, dist2, K):
+    """radius [B][K]: the largest member distance to the centroid per cluster (see kbo_cluster_radius)."""
+    labels, dist2 = _i32(labels), _f32(dist2)
+    B, N = labels.shape
+    radius = np.empty((B, K), np.float32)
+    _check(_load().kbo_cluster_radius(B, N, K, _p(labels), _p(dist2), _p(radius)), "cluster_radius")
+    return radius
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

@@ -523,4 +523,25 @@ int kbo_kmeanspp(int B, int N, int D, int K, const float* z, uint64_t seed, int3
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Cluster radius: radius[b][i] = max over the members k of cluster i of ||z_k - c_i|| = sqrt(dist2[k])
+// (0 for an empty cluster).  Theorem 1's bound carries the term L * max_i diam(C_i); by the triangle
+// inequality through the centroid diam(C_i) <= 2 radius_i, so 2 L max_i radius_i bounds that term with one
+// pass over the candidates instead of all pairs.
+// ---------------------------------------------------------------------------
+int kbo_cluster_radius(int B, int N, int K, const int32_t* labels, const float* dist2, float* radius) {
+    for (int b = 0; b < B; ++b) {
+        for (int i = 0; i < K; ++i) radius[ix2(b, i, K)] = 0.0f;
+        for (int k = 0; k < N; ++k) {
+            const int lab = labels[ix2(b, k, N)];
+            if (lab < 0 || lab >= K) return 2;
+            const double d2 = (double)dist2[ix2(b, k, N)];
+            if (!(d2 > 0.0)) continue;
+            const float r = (float)std::sqrt(d2);
+            if (r > radius[ix2(b, lab, K)]) radius[ix2(b, lab, K)] = r;
+        }
+    }
+    return 0;
+}
+
 }  // extern "C"

@@ -588,3 +588,34 @@ def test_kmeanspp_full_seeding():
     # another seed, other seeds; the same seed, the same ones
     np.testing.assert_array_equal(oracle.kmeanspp(z[:20], K, seed=99), rows[:20])
     assert np.any(oracle.kmeanspp(z[:20], K, seed=100) != rows[:20])
+
+
+# ------------------------------------------------------------ cluster radius
+def test_cluster_radius_bounds_the_diameter():
+    rng = np.random.default_rng(21)
+    B, N, D, K = 2, 400, 5, 6
+    z = rng.standard_normal((B, N, D)).astype(np.float32)
+    c = rng.standard_normal((B, K, D)).astype(np.float32)
+    a = oracle.cluster_assign(z, c, want_rep=False)
+    c2, _ = oracle.cluster_update(z, a["labels"], c)
+    d2 = oracle.dist2_at(z, c2, a["labels"]).astype(np.float32)
+    rad = oracle.cluster_radius(a["labels"], d2, K)
+    for b in range(B):
+        for i in range(K):
+            m = z[b][a["labels"][b] == i].astype(np.float64)
+            if len(m) == 0:
+                assert rad[b, i] == 0.0
+                continue
+            # brute force from the definition, with the distances recomputed by scipy
+            want = scipy.spatial.distance.cdist(m, c2[b, i][None].astype(np.float64)).max()
+            assert rad[b, i] == pytest.approx(want, rel=1e-5)
+            if len(m) > 1:
+                diam = scipy.spatial.distance.pdist(m).max()
+                assert diam <= 2.0 * rad[b, i] * (1 + 1e-6)          # the term of Theorem 1 is bounded from above
+                assert diam >= rad[b, i] * (1 - 1e-6)                # and not by more than a factor 2 (centroid = member mean)
+    # members on a circle of radius 3 around their centroid; an empty cluster
+    ang = np.linspace(0, 2 * np.pi, 12, endpoint=False)
+    pts = 3.0 * np.stack([np.cos(ang), np.sin(ang)], 1)
+    d2c = (pts ** 2).sum(1).astype(np.float32)[None]
+    r = oracle.cluster_radius(np.zeros((1, 12), np.int32), d2c, 2)
+    assert r[0, 0] == pytest.approx(3.0, rel=1e-6) and r[0, 1] == 0.0
