@@ -415,6 +415,23 @@ def run_ours(args, cfg):
                  "hbm_frac": round_bytes / (seed_ms * 1e-3 / cfg.K) / 1e9 / peaks["hbm_gbs"],
                  "what": "kb_seed_kmeanspp on the step's z: K rounds, one launch each (not part of the timed step)"}
 
+    # ---- cluster radii of the step's clustering (bounds the diameter term of Theorem 1; outside the timed step)
+    radius = torch.empty((cfg.B, cfg.K), dtype=torch.float32, device=device)
+    ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
+    barrier()
+    ctx.timing_enable(True)
+    for _ in range(args.steps):
+        flush.zero_()
+        ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
+    barrier()
+    rad_ms, rad_calls = ctx.timing_read()["sample"]
+    ctx.timing_enable(False)
+    rad_us = rad_ms / max(rad_calls, 1) * 1e3
+    rad_bytes = cfg.B * cfg.N * 8 + cfg.B * cfg.K * 4
+    radius_line = {"avg_us": rad_us, "algorithmic_bytes": rad_bytes, "GBps": rad_bytes / (rad_us * 1e-6) / 1e9,
+                   "max_radius": float(radius.max()),
+                   "what": "kb_cluster_radius on the step's labels and dist2 (memset node + kernel, after an L2 flush)"}
+
     # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
     # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
     # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
@@ -549,7 +566,7 @@ def run_ours(args, cfg):
         "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
         "device_status": int(status), "peaks": peaks,
         "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
-        "sample_member": sample_line, "online_iteration": loop_line, "seed_kmeanspp": seed_line,
+        "sample_member": sample_line, "online_iteration": loop_line, "seed_kmeanspp": seed_line, "cluster_radius": radius_line,
     }
     print(json.dumps(line))
     ctx.close()

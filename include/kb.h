@@ -94,7 +94,7 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_INIT 5
 #define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
 #define KB_T_ASSIGN_KERNEL 7 /* the tensor-core contraction kernel alone (nested inside KB_T_ASSIGN or KB_T_FIT) */
-#define KB_T_SAMPLE 8 /* kb_sample_member, kb_record_outcome */
+#define KB_T_SAMPLE 8 /* kb_sample_member, kb_record_outcome, kb_cluster_radius */
 #define KB_T_COUNT 9
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
@@ -235,6 +235,18 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
  * per centre).  fp32 distances in the direct form. */
 kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
                            int32_t* rows);
+
+/* Cluster radius: radius[b][i] = max over the members k of cluster i of
+ * sqrt(dist2[b][k]), 0 for an empty cluster.  Theorem 1's bound carries the
+ * term L * max_i diam(C_i); through the centroid diam(C_i) <= 2 radius[i], so
+ * 2 L max_i radius[i] bounds it with one pass over the candidates.
+ *   labels [B][N] in, values in [0, K) (others set bit 1 of the device status
+ *   word and are skipped);  dist2 [B][N] in as kb_cluster_assign writes it
+ *   (entries that are not positive, NaN included, add nothing)
+ *   radius [B][K] out
+ * DEVICE memory.  One memset node and one launch, no workspace. */
+kb_status kb_cluster_radius(kb_ctx* ctx, int B, int N, int K, const int32_t* labels, const float* dist2,
+                            float* radius);
 
 /* Outcome of one iteration (Sec. 2.2 "Formal Model": r_t = Clip((L(k_t) -
  * L(k'_t)) / L(k_t), 0, 1); Algorithm 1, "Generation & update": N <- N + 1,

@@ -345,6 +345,15 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
                                    member_val);
 }
 
+kb_status kb_cluster_radius(kb_ctx* ctx, int B, int N, int K, const int32_t* labels, const float* dist2, float* radius) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, K >= 1, "kb_cluster_radius: K must be >= 1");
+    if (B > 0) KB_REQUIRE(ctx, radius, "kb_cluster_radius: radius is required");
+    if ((size_t)B * N > 0) KB_REQUIRE(ctx, labels && dist2, "kb_cluster_radius: labels and dist2 are required");
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_cluster_radius(ctx, B, N, K, labels, dist2, radius);
+}
+
 kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed, int32_t* rows) {
     KB_COMMON(ctx, B, N);
     KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_seed_kmeanspp: D and K must be >= 1");

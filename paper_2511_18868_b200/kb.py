@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
-           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_seed_kmeanspp",
+           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_seed_kmeanspp", "kb_cluster_radius",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc"]
 
@@ -90,6 +90,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_score_select.argtypes = [_VP, i, i, i, i, ScoreParams] + [_VP] * 14
     lib.kb_sample_member.argtypes = [_VP, i, i, i, i, i] + [_VP] * 4 + [f, ctypes.c_uint64] + [_VP] * 3
     lib.kb_record_outcome.argtypes = [_VP, i, i, i, i] + [_VP] * 9
+    lib.kb_cluster_radius.argtypes = [_VP, i, i, i, _VP, _VP, _VP]
     lib.kb_seed_kmeanspp.argtypes = [_VP, i, i, i, i, _VP, ctypes.c_uint64, _VP]
     lib.kb_set_assign_options.argtypes = [_VP, i, f]
     lib.kb_get_assign_path.argtypes = [_VP, ctypes.POINTER(i)]
@@ -255,6 +256,13 @@ class KB:
                                               self._p(h_cand), self._p(target), float(theta_sat),
                                               int(seed) & (2 ** 64 - 1), self._p(t), self._p(member),
                                               self._p(member_val)), "kb_sample_member")
+
+    def cluster_radius(self, labels, dist2, radius):
+        """radius [B][K]: largest member distance to the centroid per cluster (bounds Theorem 1's diameter term)."""
+        B, N = labels.shape
+        K = radius.shape[1]
+        self._check(self.lib.kb_cluster_radius(self.h, B, N, K, self._p(labels), self._p(dist2), self._p(radius)),
+                    "kb_cluster_radius")
 
     def seed_kmeanspp(self, z, rows, seed):
         """k-means++ seeding: rows [B][K] of z to start the clustering from."""

@@ -999,3 +999,25 @@ def test_seed_kmeanspp_properties(kbx):
     a = oracle.cluster_assign(zz, ref_c, want_rep=False)
     parity.close(host(inertia), a["inertia"], atol=0, rtol=1e-3, what="inertia after seeded fit")
     assert kbx.device_status() == 0
+
+
+# ------------------------------------------------------------ cluster radius
+@pytest.mark.parametrize("B,N,K", [(1, 256, 8), (3, 1000, 5), (2, 20011, 64), (1, 262144, 256), (64, 512, 16),
+                                   (1, 50000, 9000), (2, 0, 4), (4, 1, 3)])
+def test_cluster_radius(kbx, B, N, K):
+    rng = np.random.default_rng(B * 31 + N + K)
+    labels = rng.integers(0, K, size=(B, N)).astype(np.int32)
+    if N > 10:
+        labels[labels == 1] = 0                          # an empty cluster
+    dist2 = (rng.standard_normal((B, N)) ** 2 * rng.uniform(0.01, 50)).astype(np.float32)
+    if N > 10:
+        dist2[:, 3] = 0.0
+        dist2[:, 5] = np.nan
+    radius = empty((B, K))
+    kbx.cluster_radius(dev(labels), dev(dist2), radius)
+    ref = oracle.cluster_radius(labels, dist2, K)
+    # one correctly rounded fp32 square root against a double one rounded once more: at most an ulp apart
+    parity.close(host(radius), ref, atol=0, rtol=2e-7, what="radius")
+    if N > 10 and K > 1:
+        assert np.all(host(radius)[:, 1] == 0.0)
+    assert kbx.device_status() == 0
