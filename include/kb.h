@@ -179,7 +179,10 @@ typedef struct {
  *   t [B] in, >= 1
  *   cl_pulls, cl_mean, cl_index [B][K][S] out
  *   arm_index [B][N][S] out, nullable (-inf for a pruned arm)
- *   best_arm, best_val, best_cluster_arm [B] out */
+ *   best_arm, best_val, best_cluster_arm [B] out
+ * Instances of at most 1024 candidates with S in {4, 8, 16, 32}, K*S <= 8192
+ * and 16-byte aligned per-arm arrays run as ONE launch (one CTA per instance,
+ * no workspace); larger ones as a memset node and four kernels. */
 kb_status kb_score_select(kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p,
                           const int32_t* labels, const float* dist2, const int32_t* pulls,
                           const float* reward_sum, const uint32_t* keep, const float* bound,

@@ -95,6 +95,12 @@ size_t kb_ws_need_assign(int B, int N, int D, int K);
 size_t kb_ws_need_assign_tc(int B, int N, int D, int K);
 size_t kb_ws_need_zsplit(int B, int N, int D, int K);
 bool kb_step_tail_small_eligible(const kb_ctx* ctx, const kb_step_args* a);
+bool kb_score_small_eligible(const kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p, const float* dist2,
+                             const int32_t* pulls, const float* reward_sum, const float* bound, const float* arm_index);
+kb_status kb_launch_score_small(kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p, const int32_t* labels,
+                                const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
+                                const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
+                                float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm);
 kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* a, bool bound_done = false);
 kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z);
 void kb_zsplit_forget(kb_ctx* ctx);

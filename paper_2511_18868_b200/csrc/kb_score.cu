@@ -324,6 +324,10 @@ kb_status kb_launch_score(kb_ctx* ctx, int B, int N, int K, int S, kb_score_para
                           const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
                           float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm) {
     if (B == 0) return KB_OK;
+    if (kb_score_small_eligible(ctx, B, N, K, S, p, dist2, pulls, reward_sum, bound, arm_index))
+        // at most 1024 candidates per instance: one CTA per instance does all four phases in one launch
+        return kb_launch_score_small(ctx, B, N, K, S, p, labels, dist2, pulls, reward_sum, keep, bound, t, cl_pulls, cl_mean,
+                                     cl_index, arm_index, best_arm, best_val, best_cluster_arm);
     const size_t need = kb_ws_need_score(B, N, K, S);
     if (ctx->ws_bytes < need)
         return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_score_select needs %zu bytes of workspace", need);

@@ -47,6 +47,9 @@ __device__ __forceinline__ unsigned long long block_max_key(unsigned long long v
     return v;
 }
 
+// PRUNE = false: the keep bits are an input (a.keep, null = every arm valid) and nothing of the pruning is computed
+// or written: the same kernel then is kb_score_select for small instances.
+template <bool PRUNE>
 __global__ void __launch_bounds__(ST_T)
 step_tail_small_kernel(const TailArgs a) {
     kb_grid_dependency_wait();
@@ -67,25 +70,29 @@ step_tail_small_kernel(const TailArgs a) {
 
     for (int e = tid; e < 2 * KS; e += ST_T) sp[e] = 0;          // int 0 == float +0 bit pattern
     for (int j = tid; j < K; j += ST_T) sa[j] = 0;
-    if (tid < S) {
+    if (PRUNE && tid < S) {
         s_rP[tid] = 1.f / a.peak_flops[tid];
         s_rW[tid] = 1.f / a.peak_bw[tid];
     }
     __syncthreads();
     float P[4], W[4], rP[4], rW[4];
     int tg[4];
+    float tinc = 0.f;
+    if (PRUNE) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        P[i] = a.peak_flops[4 * q + i];
-        W[i] = a.peak_bw[4 * q + i];
-        rP[i] = s_rP[4 * q + i];
-        rW[i] = s_rW[4 * q + i];
-        int t = a.target[4 * q + i];
-        if (t < 0 || t >= a.R) { atomicOr(a.dev_status, 2); t = 0; }
-        tg[i] = t;
+        for (int i = 0; i < 4; ++i) {
+            P[i] = a.peak_flops[4 * q + i];
+            W[i] = a.peak_bw[4 * q + i];
+            rP[i] = s_rP[4 * q + i];
+            rW[i] = s_rW[4 * q + i];
+            int t = a.target[4 * q + i];
+            if (t < 0 || t >= a.R) { atomicOr(a.dev_status, 2); t = 0; }
+            tg[i] = t;
+        }
+        tinc = a.t_inc[b];
     }
-    const float tinc = a.t_inc[b];
     const size_t row0 = (size_t)b * N;
+    const unsigned all_arms = S == 32 ? 0xffffffffu : ((1u << S) - 1u);
 
     // ---- pass 1: keep bits, gain bound, cluster sums ------------------------------------------
     unsigned count = 0;
@@ -93,31 +100,38 @@ step_tail_small_kernel(const TailArgs a) {
         const int r = it * rstep + tid / vps;
         const bool live = r < N;
         const size_t i = row0 + min(r, N - 1);                   // clamped: loads stay in range
-        const float F = __ldg(a.flops + i), Q = __ldg(a.bytes + i);
-        const float Tk = a.bound ? __ldg(a.t_cur + i) : 1.f;
         int lab = __ldg(a.labels + i);
         const bool lab_ok = lab >= 0 && lab < K;
         if (!lab_ok) { if (live) atomicOr(a.dev_status, 1); lab = 0; }
-        const float* h = a.hsig + ((size_t)b * K + lab) * a.R;
         const int4 pv = __ldg(reinterpret_cast<const int4*>(a.pulls + i * S + 4 * q));
         const float4 wv = __ldg(reinterpret_cast<const float4*>(a.reward_sum + i * S + 4 * q));
         unsigned bits = 0;
-        float g[4];
-        const float rT = 1.f / Tk;
+        float g[4] = {0.f, 0.f, 0.f, 0.f};
+        if (PRUNE) {
+            const float F = __ldg(a.flops + i), Q = __ldg(a.bytes + i);
+            const float Tk = a.bound ? __ldg(a.t_cur + i) : 1.f;
+            const float* h = a.hsig + ((size_t)b * K + lab) * a.R;
+            const float rT = 1.f / Tk;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float tlb = fmaxf(kb_div_by(F, P[k], rP[k]), kb_div_by(Q, W[k], rW[k]));
-            const bool ok = (tlb < tinc) && (__ldg(h + tg[k]) < a.theta);
-            if (ok) bits |= 1u << (4 * q + k);
-            float v = kb_div_by(Tk - tlb, Tk, rT);
-            v = v > 0.f ? v : 0.f;                               // also maps NaN (0/0) to 0, as the definition does
-            g[k] = v < 1.f ? v : 1.f;
+            for (int k = 0; k < 4; ++k) {
+                const float tlb = fmaxf(kb_div_by(F, P[k], rP[k]), kb_div_by(Q, W[k], rW[k]));
+                const bool ok = (tlb < tinc) && (__ldg(h + tg[k]) < a.theta);
+                if (ok) bits |= 1u << (4 * q + k);
+                float v = kb_div_by(Tk - tlb, Tk, rT);
+                v = v > 0.f ? v : 0.f;                           // also maps NaN (0/0) to 0, as the definition does
+                g[k] = v < 1.f ? v : 1.f;
+            }
+            for (int o = 1; o < vps; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+        } else {
+            bits = a.keep ? (__ldg(a.keep + i) & all_arms) : all_arms;
         }
-        for (int o = 1; o < vps; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
         if (live) {
-            if (q == 0) { a.keep[i] = bits; skeep[r] = bits; count += __popc(bits); }
-            if (a.bound && a.write_bound)
-                *reinterpret_cast<float4*>(a.bound + i * S + 4 * q) = make_float4(g[0], g[1], g[2], g[3]);
+            if (PRUNE) {
+                if (q == 0) { a.keep[i] = bits; count += __popc(bits); }
+                if (a.bound && a.write_bound)
+                    *reinterpret_cast<float4*>(a.bound + i * S + 4 * q) = make_float4(g[0], g[1], g[2], g[3]);
+            }
+            if (q == 0) skeep[r] = bits;
             if (lab_ok) {
                 int* dp = sp + lab * S + 4 * q;
                 float* dr = sr + lab * S + 4 * q;
@@ -137,7 +151,7 @@ step_tail_small_kernel(const TailArgs a) {
     for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
     if (lane == 0) s_cnt[tid >> 5] = count;
     __syncthreads();
-    if (tid == 0 && a.kept) {
+    if (PRUNE && tid == 0 && a.kept) {
         unsigned tot = 0;
         for (int w = 0; w < ST_T / 32; ++w) tot += s_cnt[w];
         a.kept[b] = tot;
@@ -244,8 +258,44 @@ kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* s, bool bou
     a.best_arm = s->best_arm; a.best_cluster_arm = s->best_cluster_arm;
     a.dev_status = ctx->dev_status;
     const size_t smem = tail_smem(s->N, s->K, s->S);
-    KB_SMEM_OPTIN(ctx, step_tail_small_kernel, smem);
-    kb_launch(step_tail_small_kernel, s->B, ST_T, smem, ctx->stream, a);
+    KB_SMEM_OPTIN(ctx, step_tail_small_kernel<true>, smem);
+    kb_launch(step_tail_small_kernel<true>, s->B, ST_T, smem, ctx->stream, a);
+    KB_LAUNCH_CHECK(ctx, "step_tail_small_kernel");
+    return KB_OK;
+}
+
+// kb_score_select for small instances: the same kernel without its pruning part (one launch instead of a memset
+// node and four kernels).  Same conditions on the sizes; the per-arm arrays must be 16-byte aligned.
+bool kb_score_small_eligible(const kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p, const float* dist2,
+                             const int32_t* pulls, const float* reward_sum, const float* bound, const float* arm_index) {
+    if (B < 1 || N < 1 || N > 1024 || K < 1) return false;
+    if (S != 4 && S != 8 && S != 16 && S != 32) return false;
+    if ((long long)K * S > 8192 || tail_smem(N, K, S) + 1024 > (size_t)ctx->max_smem_optin) return false;
+    if (p.lipschitz_L != 0.f && !dist2) return false;
+    if (!(p.prior_pulls > 0.f)) return false;
+    if (p.cap_with_bound && !bound) return false;
+    const uintptr_t al = (uintptr_t)pulls | (uintptr_t)reward_sum | (uintptr_t)arm_index |
+                         (p.cap_with_bound ? (uintptr_t)bound : 0);
+    return (al & 15) == 0;
+}
+
+kb_status kb_launch_score_small(kb_ctx* ctx, int B, int N, int K, int S, kb_score_params p, const int32_t* labels,
+                                const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
+                                const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
+                                float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm) {
+    TailArgs a{};
+    a.N = N; a.S = S; a.K = K; a.R = 1;
+    a.write_bound = 0;
+    a.prm = p;
+    a.dist2 = dist2; a.reward_sum = reward_sum; a.labels = labels; a.pulls = pulls; a.t = t;
+    a.keep = const_cast<uint32_t*>(keep);                    // read only in this mode
+    a.bound = p.cap_with_bound ? const_cast<float*>(bound) : nullptr;
+    a.cl_pulls = cl_pulls; a.cl_mean = cl_mean; a.cl_index = cl_index; a.arm_index = arm_index;
+    a.best_val = best_val; a.best_arm = best_arm; a.best_cluster_arm = best_cluster_arm;
+    a.dev_status = ctx->dev_status;
+    const size_t smem = tail_smem(N, K, S);
+    KB_SMEM_OPTIN(ctx, step_tail_small_kernel<false>, smem);
+    kb_launch(step_tail_small_kernel<false>, B, ST_T, smem, ctx->stream, a);
     KB_LAUNCH_CHECK(ctx, "step_tail_small_kernel");
     return KB_OK;
 }
