@@ -235,7 +235,9 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
  *   z [B][N][D] in (N >= 1);  rows [B][K] out, values in [0, N)
  * DEVICE memory; seed by value.  K launches (one per round, each reading z
  * once); needs the workspace of kb_workspace_bytes (4 bytes per row plus 20
- * per centre).  fp32 distances in the direct form. */
+ * per centre).  Many small instances (N <= 1024, B at least half the number
+ * of SMs) run all rounds in one launch, one CTA per instance, no workspace.
+ * fp32 distances in the direct form. */
 kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
                            int32_t* rows);
 

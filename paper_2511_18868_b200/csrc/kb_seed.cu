@@ -143,6 +143,93 @@ seed_round_kernel(int N, int D, int K, int round, int G, int rows_per, const flo
     rows[slot] = (int32_t)(0xffffffffu - (unsigned)(k & 0xffffffffull));
 }
 
+// Small instances (at most SD_T * SD_R rows): all K rounds in one launch, one CTA per instance.  A thread owns up
+// to SD_R rows and keeps their weights in registers; the rows are re-read every round (the instance stays in L1/L2),
+// each round ends in two block maxima (weighted and uniform draw) instead of atomics and a ticket.
+// STAGE: the instance is first copied into shared memory (rows padded by four floats, so that a warp's float4 reads
+// of 32 different rows meet no bank twice) and every round reads it from there; without it the K re-reads of all
+// instances in flight go to L2, which then bounds the kernel.
+constexpr int SD_R = 4;
+
+__device__ __forceinline__ unsigned long long seed_block_max(unsigned long long v, unsigned long long* s_red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+        v = other > v ? other : v;
+    }
+    __syncthreads();                                             // s_red may still be read from the reduction before
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    v = s_red[0];
+#pragma unroll
+    for (int w = 1; w < SD_T / 32; ++w) v = s_red[w] > v ? s_red[w] : v;
+    return v;
+}
+
+template <int V, bool STAGE>
+__global__ void __launch_bounds__(SD_T)
+seed_small_kernel(int N, int D, int K, const float* __restrict__ z, int32_t* __restrict__ rows, uint32_t seed_lo,
+                  uint32_t seed_hi) {
+    kb_grid_dependency_wait();
+    extern __shared__ __align__(16) float s_z[];                 // STAGE: [N][D + 4]
+    __shared__ unsigned long long s_red[SD_T / 32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const float* zg = z + (size_t)b * N * D;
+    const int ld = STAGE ? D + 4 : D;                            // floats between two rows
+    if (STAGE) {
+        const int vpr = D / 4;
+        for (int e = tid; e < N * vpr; e += SD_T) {
+            const int r = e / vpr, q = e - r * vpr;
+            *reinterpret_cast<float4*>(s_z + (size_t)r * ld + 4 * q) = __ldg(reinterpret_cast<const float4*>(zg) + e);
+        }
+        __syncthreads();
+    }
+    const float* zb = STAGE ? s_z : zg;
+    float wgt[SD_R];
+#pragma unroll
+    for (int j = 0; j < SD_R; ++j) wgt[j] = 1.f;
+    int c = 0;
+    for (int round = 0; round < K; ++round) {
+        unsigned long long bestW = 0ull, bestU = 0ull;
+        const float* zc = zb + (size_t)c * ld;
+#pragma unroll
+        for (int j = 0; j < SD_R; ++j) {
+            const int r = tid + j * SD_T;
+            if (r >= N) continue;
+            if (round > 0) {
+                const float* x = zb + (size_t)r * ld;
+                float a = 0.f;
+                if (V == 4) {
+                    for (int q = 0; q < D / 4; ++q) {
+                        const float4 xv = STAGE ? reinterpret_cast<const float4*>(x)[q] : __ldg(reinterpret_cast<const float4*>(x) + q);
+                        const float4 cv = STAGE ? reinterpret_cast<const float4*>(zc)[q] : __ldg(reinterpret_cast<const float4*>(zc) + q);
+                        const float e0 = xv.x - cv.x, e1 = xv.y - cv.y, e2 = xv.z - cv.z, e3 = xv.w - cv.w;
+                        a = fmaf(e0, e0, a); a = fmaf(e1, e1, a); a = fmaf(e2, e2, a); a = fmaf(e3, e3, a);
+                    }
+                } else {
+                    for (int q = 0; q < D; ++q) {
+                        const float e = __ldg(x + q) - __ldg(zc + q);
+                        a = fmaf(e, e, a);
+                    }
+                }
+                wgt[j] = round == 1 ? a : fminf(wgt[j], a);
+            }
+            const uint32_t w0 = kb_philox4x32_10_word0((uint32_t)r, (uint32_t)b, (uint32_t)round, 1u, seed_lo, seed_hi);
+            const float g = -logf(-logf(kb_uniform23(w0)));
+            const unsigned long long ku = seed_pack(g, r);
+            bestU = ku > bestU ? ku : bestU;
+            if (wgt[j] > 0.f) {
+                const unsigned long long kw = seed_pack(logf(wgt[j]) + g, r);
+                bestW = kw > bestW ? kw : bestW;
+            }
+        }
+        bestW = seed_block_max(bestW, s_red);
+        if (bestW == 0ull) bestW = seed_block_max(bestU, s_red);   // every weight zero (uniform over the block): the uniform draw
+        c = (int)(0xffffffffu - (unsigned)(bestW & 0xffffffffull));
+        if (tid == 0) rows[(size_t)b * K + round] = c;
+    }
+}
+
 int seed_ctas(const kb_ctx* ctx, int B, int N) {
     long want = (4L * ctx->sm_count + B - 1) / B;
     long cap = ((long)N + SD_T - 1) / SD_T;                      // at least one trip of rows per CTA
@@ -160,6 +247,22 @@ size_t kb_ws_need_seed(int B, int N, int K) {
 kb_status kb_launch_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
                                   int32_t* rows) {
     if (B == 0) return KB_OK;
+    const bool vec = (D % 4 == 0) && (((uintptr_t)z & 15) == 0);
+    const uint32_t s_lo = (uint32_t)(seed & 0xffffffffu), s_hi = (uint32_t)(seed >> 32);
+    if (N <= SD_T * SD_R && (long)B * 2 >= ctx->sm_count) {
+        // many small instances: every round of an instance in one CTA, one launch in all
+        const size_t stage = (size_t)N * (D + 4) * sizeof(float);
+        if (vec && stage + 1024 <= (size_t)ctx->max_smem_optin) {
+            KB_SMEM_OPTIN(ctx, (seed_small_kernel<4, true>), stage);
+            kb_launch((seed_small_kernel<4, true>), B, SD_T, stage, ctx->stream, N, D, K, z, rows, s_lo, s_hi);
+        } else if (vec) {
+            kb_launch((seed_small_kernel<4, false>), B, SD_T, 0, ctx->stream, N, D, K, z, rows, s_lo, s_hi);
+        } else {
+            kb_launch((seed_small_kernel<1, false>), B, SD_T, 0, ctx->stream, N, D, K, z, rows, s_lo, s_hi);
+        }
+        KB_LAUNCH_CHECK(ctx, "seed_small_kernel");
+        return KB_OK;
+    }
     const size_t need = kb_ws_need_seed(B, N, K);
     if (ctx->ws_bytes < need)
         return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_seed_kmeanspp needs %zu bytes of workspace", need);
@@ -169,8 +272,6 @@ kb_status kb_launch_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const
     const int G = seed_ctas(ctx, B, N);
     if (G > 1) KB_MEMSET(ctx, ctx->ws, 0, zero_bytes);
     const int rows_per = (N + G - 1) / G;
-    const bool vec = (D % 4 == 0) && (((uintptr_t)z & 15) == 0);
-    const uint32_t s_lo = (uint32_t)(seed & 0xffffffffu), s_hi = (uint32_t)(seed >> 32);
     for (int round = 0; round < K; ++round) {
         if (vec)
             kb_launch(seed_round_kernel<4>, dim3(G, B), SD_T, 0, ctx->stream, N, D, K, round, G, rows_per, z, rows, s_lo, s_hi,

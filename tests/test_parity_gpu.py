@@ -941,7 +941,8 @@ def _follow_seeding(z, rows, seed, tol=SAMPLE_TOL):
 
 @pytest.mark.parametrize("B,N,D,K", [(1, 256, 16, 8), (3, 1000, 20, 5), (2, 5003, 5, 7), (1, 40000, 64, 24),
                                      (40, 512, 32, 16), (2, 1, 8, 1), (1, 3000, 128, 3), (2, 700, 4, 4), (2, 333, 1, 3),
-                                     (1, 900, 8, 5)])
+                                     (1, 900, 8, 5), (200, 300, 16, 6), (160, 1000, 5, 4), (150, 1024, 32, 8),
+                                     (300, 7, 4, 7)])
 def test_seed_kmeanspp(kbx, B, N, D, K):
     cfg = wl.scaled(wl.CONFIGS["medium"], B=B, N=N, D=D, K=max(K, 2), components=max(2, K), S=4, iters=1)
     x = wl.make_inputs(cfg, seed=N + K)["x"]
