@@ -365,131 +365,145 @@ def run_ours(args, cfg):
     barrier()
     e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
 
-    # ---- the within-cluster draw of k_t (Algorithm 1's line after the selection; outside the timed step) ----
-    lab_host = dev_t["labels"].cpu().numpy()
-    h_cand = torch.from_numpy(wl.make_candidate_signatures(inp["hsig"], lab_host, seed=77)).to(device)
-    member = torch.empty((cfg.B,), dtype=torch.int32, device=device)
-
-    def draw(step):
-        ctx.sample_member(dev_t["labels"], dev_t["best_cluster_arm"], h_cand, dev_t["target"], dev_t["t"], member,
-                          cfg.K, float(inp["theta_sat"]), 0xC0FFEE + step)
-
-    for i in range(3):
-        draw(i)
-    barrier()
-    # timed by the library's own event pair around the call's work on the stream: the L2 flush before each call
-    # also gives the host time to queue the call, so the pair sees the device's time, not the host's
-    ks0, _ = ctx.launch_count()
-    ctx.timing_enable(True)
-    for i in range(args.steps):
-        flush.zero_()
-        draw(10 + i)
-    barrier()
-    smp_ms, smp_calls = ctx.timing_read()["sample"]
-    ctx.timing_enable(False)
-    ks1, _ = ctx.launch_count()
-    smp_us = smp_ms / max(smp_calls, 1) * 1e3
-    chosen = dev_t["best_cluster_arm"].cpu().numpy() // cfg.S
-    members = int(sum((lab_host[b] == chosen[b]).sum() for b in range(cfg.B) if chosen[b] >= 0))
-    smp_bytes = 4 * cfg.B * cfg.N + 4 * members + 16 * cfg.B      # labels, one signature entry per member, per-instance words
-    sample_line = {"avg_us": smp_us, "algorithmic_bytes": smp_bytes, "GBps": smp_bytes / (smp_us * 1e-6) / 1e9,
-                   "kernels_per_call": (ks1 - ks0) / args.steps, "members_of_chosen_clusters": members,
-                   "what": "kb_sample_member on the step's labels and chosen pairs (not part of the timed step)"}
-    # ---- k-means++ seeding of the step's z (an alternative to caller-supplied initial rows; outside the timed step)
-    seed_rows = torch.empty((cfg.B, cfg.K), dtype=torch.int32, device=device)
-    ctx.seed_kmeanspp(dev_t["z"], seed_rows, 1)
-    barrier()
-    kq0, _ = ctx.launch_count()
-    sa, sb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    flush.zero_()
-    sa.record()
-    ctx.seed_kmeanspp(dev_t["z"], seed_rows, 2)
-    sb.record()
-    barrier()
-    kq1, _ = ctx.launch_count()
-    seed_ms = sa.elapsed_time(sb)
-    one_launch = (kq1 - kq0) == 1                           # many small instances: all rounds on chip, z read once
-    seed_bytes = cfg.B * cfg.N * cfg.D * 4 if one_launch else cfg.K * cfg.B * cfg.N * (cfg.D * 4 + 8)
-    seed_line = {"ms": seed_ms, "rounds": cfg.K, "us_per_round": seed_ms * 1e3 / cfg.K, "kernels": int(kq1 - kq0),
-                 "algorithmic_bytes": seed_bytes, "GBps": seed_bytes / (seed_ms * 1e-3) / 1e9,
-                 "hbm_frac": seed_bytes / (seed_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                 "what": "kb_seed_kmeanspp on the step's z (not part of the timed step): " +
-                         ("one launch, every instance staged in shared memory, z read once" if one_launch else
-                          "one launch per round, each reading z once plus 8 bytes of weight per row")}
-
-    # ---- cluster radii of the step's clustering (bounds the diameter term of Theorem 1; outside the timed step)
-    radius = torch.empty((cfg.B, cfg.K), dtype=torch.float32, device=device)
-    ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
-    barrier()
-    ctx.timing_enable(True)
-    for _ in range(args.steps):
-        flush.zero_()
-        ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
-    barrier()
-    rad_ms, rad_calls = ctx.timing_read()["sample"]
-    ctx.timing_enable(False)
-    rad_us = rad_ms / max(rad_calls, 1) * 1e3
-    rad_bytes = cfg.B * cfg.N * 8 + cfg.B * cfg.K * 4
-    radius_line = {"avg_us": rad_us, "algorithmic_bytes": rad_bytes, "GBps": rad_bytes / (rad_us * 1e-6) / 1e9,
-                   "max_radius": float(radius.max()),
-                   "what": "kb_cluster_radius on the step's labels and dist2 (memset node + kernel, after an L2 flush)"}
-
-    # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
-    # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
-    # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
-    loop_t = {k: dev_t[k].clone() for k in ("pulls", "reward_sum", "t")}
-    t_new = (dev_t["t_cur"][:, 0] * 0.9).contiguous()
-    outs = {k: dev_t[k] for k in ("cl_pulls", "cl_mean", "cl_index", "best_arm", "best_val", "best_cluster_arm")}
-
-    def iteration():
-        ctx.score_select(dev_t["labels"], dev_t["dist2"], loop_t["pulls"], loop_t["reward_sum"], loop_t["t"],
-                         outs["cl_pulls"], outs["cl_mean"], outs["cl_index"], outs["best_arm"], outs["best_val"],
-                         outs["best_cluster_arm"], keep=dev_t["keep"], lipschitz_L=float(inp["lipschitz_L"]))
-        ctx.sample_member(dev_t["labels"], outs["best_cluster_arm"], h_cand, dev_t["target"], loop_t["t"], member,
-                          cfg.K, float(inp["theta_sat"]), 0xC0FFEE)
-        ctx.record_outcome(member, outs["best_cluster_arm"], dev_t["t_cur"], t_new, loop_t["pulls"],
-                           loop_t["reward_sum"], loop_t["t"])
-
-    def timed(fn, n):
-        for _ in range(3):
-            fn()
-        barrier()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(n):
-            fn()
-        b.record()
-        barrier()
-        return a.elapsed_time(b) / n * 1e3
-
-    kl0, _ = ctx.launch_count()
-    iteration()
-    kl1, _ = ctx.launch_count()
-    n_loop = max(args.steps, 20)
-    eager_us = timed(iteration, n_loop)
-    main_stream = torch.cuda.current_stream()
-    side = torch.cuda.Stream()
-    side.wait_stream(main_stream)
-    ctx.set_stream(side)
-    try:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            iteration()
-    finally:
-        ctx.set_stream(main_stream)
-    main_stream.wait_stream(side)
-    graph_us = timed(graph.replay, n_loop)
-    loop_line = {"eager_us": eager_us, "graph_us": graph_us, "kernels": int(kl1 - kl0), "iterations_timed": n_loop,
-                 "what": "kb_score_select + kb_sample_member + kb_record_outcome on the step's labels, consecutive "
-                         "iterations (L2 not flushed), per rank"}
-    del h_cand, graph
-
     # ---- max over ranks -----------------------------------------------------------
     total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], dist, device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
+
+    # ---- beyond the timed step, rank 0 only and without collectives: the calls that follow the step in Algorithm 1.
+    # A failure here must not cost the line: it is reported in place of the figures.
+    def extras():
+        # ---- the within-cluster draw of k_t (Algorithm 1's line after the selection; outside the timed step) ----
+        lab_host = dev_t["labels"].cpu().numpy()
+        h_cand = torch.from_numpy(wl.make_candidate_signatures(inp["hsig"], lab_host, seed=77)).to(device)
+        member = torch.empty((cfg.B,), dtype=torch.int32, device=device)
+
+        def draw(step):
+            ctx.sample_member(dev_t["labels"], dev_t["best_cluster_arm"], h_cand, dev_t["target"], dev_t["t"], member,
+                              cfg.K, float(inp["theta_sat"]), 0xC0FFEE + step)
+
+        for i in range(3):
+            draw(i)
+        torch.cuda.synchronize()
+        # timed by the library's own event pair around the call's work on the stream: the L2 flush before each call
+        # also gives the host time to queue the call, so the pair sees the device's time, not the host's
+        ks0, _ = ctx.launch_count()
+        ctx.timing_enable(True)
+        for i in range(args.steps):
+            flush.zero_()
+            draw(10 + i)
+        torch.cuda.synchronize()
+        smp_ms, smp_calls = ctx.timing_read()["sample"]
+        ctx.timing_enable(False)
+        ks1, _ = ctx.launch_count()
+        smp_us = smp_ms / max(smp_calls, 1) * 1e3
+        chosen = dev_t["best_cluster_arm"].cpu().numpy() // cfg.S
+        members = int(sum((lab_host[b] == chosen[b]).sum() for b in range(cfg.B) if chosen[b] >= 0))
+        smp_bytes = 4 * cfg.B * cfg.N + 4 * members + 16 * cfg.B      # labels, one signature entry per member, per-instance words
+        sample_line = {"avg_us": smp_us, "algorithmic_bytes": smp_bytes, "GBps": smp_bytes / (smp_us * 1e-6) / 1e9,
+                       "kernels_per_call": (ks1 - ks0) / args.steps, "members_of_chosen_clusters": members,
+                       "what": "kb_sample_member on the step's labels and chosen pairs (not part of the timed step)"}
+        # ---- k-means++ seeding of the step's z (an alternative to caller-supplied initial rows; outside the timed step)
+        seed_rows = torch.empty((cfg.B, cfg.K), dtype=torch.int32, device=device)
+        ctx.seed_kmeanspp(dev_t["z"], seed_rows, 1)
+        torch.cuda.synchronize()
+        kq0, _ = ctx.launch_count()
+        sa, sb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush.zero_()
+        sa.record()
+        ctx.seed_kmeanspp(dev_t["z"], seed_rows, 2)
+        sb.record()
+        torch.cuda.synchronize()
+        kq1, _ = ctx.launch_count()
+        seed_ms = sa.elapsed_time(sb)
+        one_launch = (kq1 - kq0) == 1                           # many small instances: all rounds on chip, z read once
+        seed_bytes = cfg.B * cfg.N * cfg.D * 4 if one_launch else cfg.K * cfg.B * cfg.N * (cfg.D * 4 + 8)
+        seed_line = {"ms": seed_ms, "rounds": cfg.K, "us_per_round": seed_ms * 1e3 / cfg.K, "kernels": int(kq1 - kq0),
+                     "algorithmic_bytes": seed_bytes, "GBps": seed_bytes / (seed_ms * 1e-3) / 1e9,
+                     "hbm_frac": seed_bytes / (seed_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "what": "kb_seed_kmeanspp on the step's z (not part of the timed step): " +
+                             ("one launch, every instance staged in shared memory, z read once" if one_launch else
+                              "one launch per round, each reading z once plus 8 bytes of weight per row")}
+
+        # ---- cluster radii of the step's clustering (bounds the diameter term of Theorem 1; outside the timed step)
+        radius = torch.empty((cfg.B, cfg.K), dtype=torch.float32, device=device)
+        ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
+        torch.cuda.synchronize()
+        ctx.timing_enable(True)
+        for _ in range(args.steps):
+            flush.zero_()
+            ctx.cluster_radius(dev_t["labels"], dev_t["dist2"], radius)
+        torch.cuda.synchronize()
+        rad_ms, rad_calls = ctx.timing_read()["sample"]
+        ctx.timing_enable(False)
+        rad_us = rad_ms / max(rad_calls, 1) * 1e3
+        rad_bytes = cfg.B * cfg.N * 8 + cfg.B * cfg.K * 4
+        radius_line = {"avg_us": rad_us, "algorithmic_bytes": rad_bytes, "GBps": rad_bytes / (rad_us * 1e-6) / 1e9,
+                       "max_radius": float(radius.max()),
+                       "what": "kb_cluster_radius on the step's labels and dist2 (memset node + kernel, after an L2 flush)"}
+
+        # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
+        # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
+        # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
+        loop_t = {k: dev_t[k].clone() for k in ("pulls", "reward_sum", "t")}
+        t_new = (dev_t["t_cur"][:, 0] * 0.9).contiguous()
+        outs = {k: dev_t[k] for k in ("cl_pulls", "cl_mean", "cl_index", "best_arm", "best_val", "best_cluster_arm")}
+
+        def iteration():
+            ctx.score_select(dev_t["labels"], dev_t["dist2"], loop_t["pulls"], loop_t["reward_sum"], loop_t["t"],
+                             outs["cl_pulls"], outs["cl_mean"], outs["cl_index"], outs["best_arm"], outs["best_val"],
+                             outs["best_cluster_arm"], keep=dev_t["keep"], lipschitz_L=float(inp["lipschitz_L"]))
+            ctx.sample_member(dev_t["labels"], outs["best_cluster_arm"], h_cand, dev_t["target"], loop_t["t"], member,
+                              cfg.K, float(inp["theta_sat"]), 0xC0FFEE)
+            ctx.record_outcome(member, outs["best_cluster_arm"], dev_t["t_cur"], t_new, loop_t["pulls"],
+                               loop_t["reward_sum"], loop_t["t"])
+
+        def timed(fn, n):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n * 1e3
+
+        kl0, _ = ctx.launch_count()
+        iteration()
+        kl1, _ = ctx.launch_count()
+        n_loop = max(args.steps, 20)
+        eager_us = timed(iteration, n_loop)
+        main_stream = torch.cuda.current_stream()
+        side = torch.cuda.Stream()
+        side.wait_stream(main_stream)
+        ctx.set_stream(side)
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+                iteration()
+        finally:
+            ctx.set_stream(main_stream)
+        main_stream.wait_stream(side)
+        graph_us = timed(graph.replay, n_loop)
+        loop_line = {"eager_us": eager_us, "graph_us": graph_us, "kernels": int(kl1 - kl0), "iterations_timed": n_loop,
+                     "what": "kb_score_select + kb_sample_member + kb_record_outcome on the step's labels, consecutive "
+                             "iterations (L2 not flushed), per rank"}
+
+        return {"sample_member": sample_line, "seed_kmeanspp": seed_line, "cluster_radius": radius_line,
+                "online_iteration": loop_line}
+
+    try:
+        extra = extras()
+    except Exception as exc:                                  # noqa: BLE001
+        extra = {"extras_error": f"{type(exc).__name__}: {exc}"}
+        try:
+            ctx.set_stream(torch.cuda.current_stream())
+        except Exception:                                     # noqa: BLE001
+            pass
 
     ms_per_step = total_ms / args.steps
     value = job_value(world, cfg.arms, ms_per_step)
@@ -568,8 +582,8 @@ def run_ours(args, cfg):
         "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
         "device_status": int(status), "peaks": peaks,
         "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
-        "sample_member": sample_line, "online_iteration": loop_line, "seed_kmeanspp": seed_line, "cluster_radius": radius_line,
     }
+    line.update(extra)
     print(json.dumps(line))
     ctx.close()
     if dist is not None:
