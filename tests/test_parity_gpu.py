@@ -187,7 +187,11 @@ def run_score(kbx, labels, dist2, pulls, rsum, t, K, keep=None, bound=None, **pr
 
 @pytest.mark.parametrize("B,N,K,S,L,masked,cap", [(1, 256, 8, 8, 0.1, True, False), (3, 1000, 7, 13, 0.0, True, False),
                                                   (2, 500, 1, 6, 0.0, False, False), (1, 4000, 64, 32, 0.1, True, True),
-                                                  (4, 129, 16, 16, 0.3, False, False), (1, 3000, 1024, 8, 0.1, True, False)])
+                                                  (4, 129, 16, 16, 0.3, False, False), (1, 3000, 1024, 8, 0.1, True, False),
+                                                  # instances of at most 1024 candidates, S in {4, 8, 16, 32}: one launch
+                                                  (2, 1024, 256, 32, 0.1, True, True), (3, 100, 4, 4, 0.0, False, True),
+                                                  (5, 777, 12, 8, 0.2, False, False), (70, 64, 3, 16, 0.0, True, False),
+                                                  (2, 1025, 8, 8, 0.1, True, False)])
 def test_score_select(kbx, B, N, K, S, L, masked, cap):
     rng = np.random.default_rng(N + K + S)
     labels = rng.integers(0, max(1, K - 1), (B, N)).astype(np.int32)
@@ -210,6 +214,30 @@ def test_score_select(kbx, B, N, K, S, L, masked, cap):
     if L == 0.0 and not cap:
         # exact ties inside the winning cluster: the lowest flat index must win
         assert np.array_equal(got["best_arm"], ref["best_arm"])
+
+
+def test_score_select_small_is_one_launch_and_optional_outputs(kbx):
+    """Small instances: kb_score_select is one launch; without arm_index the selections are unchanged."""
+    rng = np.random.default_rng(4)
+    B, N, K, S = 6, 300, 5, 8
+    labels = rng.integers(0, K, (B, N)).astype(np.int32)
+    dist2 = rng.uniform(0, 4, (B, N)).astype(np.float32)
+    pulls = rng.poisson(3.0, (B, N, S)).astype(np.int32)
+    rsum = (pulls * rng.uniform(0, 2, pulls.shape)).astype(np.float32)
+    t = (1 + pulls.reshape(B, -1).sum(1)).astype(np.int32)
+    k0 = kbx.launch_count()
+    full = run_score(kbx, labels, dist2, pulls, rsum, t, K, lipschitz_L=0.1)
+    k1 = kbx.launch_count()
+    assert k1[0] - k0[0] == 1 and k1[1] - k0[1] == 0
+    o = dict(cl_pulls=empty((B, K, S)), cl_mean=empty((B, K, S)), cl_index=empty((B, K, S)),
+             best_arm=empty((B,), torch.int32), best_val=empty((B,)), best_cluster_arm=empty((B,), torch.int32))
+    kbx.score_select(dev(labels), dev(dist2), dev(pulls), dev(rsum), dev(t), **o, lipschitz_L=0.1)
+    # (reward sums are added in shared memory in no fixed order: last-bit differences between two runs are expected)
+    ref = oracle.score_select(labels, dist2, pulls, rsum, t, K, c=2.0, lipschitz_L=0.1)
+    parity.close(host(o["cl_index"]), ref["cl_index"], atol=1e-6, what="cl_index")
+    parity.select_match(host(o["best_arm"]), host(o["best_val"]), ref, ref["arm_index"])
+    parity.cluster_select_match(host(o["best_cluster_arm"]), ref, ref["cl_index"])
+    parity.select_match(full["best_arm"], full["best_val"], ref, ref["arm_index"])
 
 
 def test_score_all_masked_and_unplayed(kbx):
