@@ -228,6 +228,17 @@ def cluster_radius(labels, dist2, K):
     return radius
 
 
+def top_m(arm_index, M):
+    """The M best arms per instance by arm_index [B][N][S] (see kbo_top_m): (top_arm [B][M], top_val [B][M])."""
+    a = _f32(arm_index)
+    B = a.shape[0]
+    NS = int(np.prod(a.shape[1:])) if a.ndim > 1 else 0
+    top_arm = np.empty((B, M), np.int32)
+    top_val = np.empty((B, M), np.float32)
+    _check(_load().kbo_top_m(B, NS, M, _p(a), _p(top_arm), _p(top_val)), "top_m")
+    return top_arm, top_val
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

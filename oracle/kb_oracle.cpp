@@ -544,4 +544,37 @@ int kbo_cluster_radius(int B, int N, int K, const int32_t* labels, const float* 
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Top-M arms of an instance by the per-arm index U(k, s) (the masked argmax of Sec. 3.4 generalised from
+// one arm to M, for generating M candidates per iteration; Sec. 5 mentions batched generation): the M arms
+// with the largest arm_index, larger value first, lower flat index k*S + s first among equal values.  Pruned
+// arms (-inf) and NaN entries never appear; when fewer than M arms are valid the tail is -1 / -inf.
+// Written as its definition: order all valid arms, take the first M.
+// ---------------------------------------------------------------------------
+int kbo_top_m(int B, int NS, int M, const float* arm_index, int32_t* top_arm, float* top_val) {
+    std::vector<int32_t> order;
+    for (int b = 0; b < B; ++b) {
+        const float* v = arm_index + (size_t)b * NS;
+        order.clear();
+        for (int i = 0; i < NS; ++i)
+            if (v[i] > -std::numeric_limits<float>::infinity()) order.push_back(i);     // false for NaN too
+        // insertion of one arm at a time into the first M places (plain selection, no library sort)
+        std::vector<int32_t> top;
+        for (int32_t i : order) {
+            size_t pos = top.size();
+            while (pos > 0 && (v[top[pos - 1]] < v[i])) --pos;      // equal values keep the earlier (lower) index first
+            if (pos < (size_t)M) {
+                top.insert(top.begin() + pos, i);
+                if (top.size() > (size_t)M) top.pop_back();
+            }
+        }
+        for (int j = 0; j < M; ++j) {
+            const bool have = (size_t)j < top.size();
+            top_arm[(size_t)b * M + j] = have ? top[j] : -1;
+            top_val[(size_t)b * M + j] = have ? v[top[j]] : -std::numeric_limits<float>::infinity();
+        }
+    }
+    return 0;
+}
+
 }  // extern "C"

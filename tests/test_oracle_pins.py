@@ -619,3 +619,40 @@ def test_cluster_radius_bounds_the_diameter():
     d2c = (pts ** 2).sum(1).astype(np.float32)[None]
     r = oracle.cluster_radius(np.zeros((1, 12), np.int32), d2c, 2)
     assert r[0, 0] == pytest.approx(3.0, rel=1e-6) and r[0, 1] == 0.0
+
+
+# ------------------------------------------------------------------ top-M arms
+def test_top_m_is_the_sorted_prefix():
+    rng = np.random.default_rng(31)
+    B, N, S = 4, 300, 8
+    a = rng.integers(0, 40, size=(B, N, S)).astype(np.float32) / 8.0      # many exact ties
+    a[rng.uniform(size=a.shape) < 0.3] = -np.inf                         # pruned arms
+    a[0, 5, 3] = np.nan
+    a[3] = -np.inf                                                       # an instance with nothing valid
+    a[3, 7, 1], a[3, 2, 6] = 1.5, 1.5                                    # ... but two equal arms
+    for M in (1, 5, 64):
+        arm, val = oracle.top_m(a, M)
+        for b in range(B):
+            flat = a[b].reshape(-1)
+            ok = np.flatnonzero(flat > -np.inf)                          # drops NaN as well
+            # brute force with numpy: value descending, then index ascending
+            order = ok[np.lexsort((ok, -flat[ok]))][:M]
+            want = np.full(M, -1)
+            want[: len(order)] = order
+            np.testing.assert_array_equal(arm[b], want)
+            np.testing.assert_array_equal(val[b][: len(order)], flat[order])
+            assert np.all(np.isneginf(val[b][len(order):]))
+    assert oracle.top_m(a, 3)[0][3].tolist() == [2 * S + 6, 7 * S + 1, -1]
+    # M = 1 is the masked argmax of score_select; top-M is a prefix of top-(M+1)
+    labels = rng.integers(0, 5, (2, 200)).astype(np.int32)
+    pulls = rng.poisson(3.0, (2, 200, 4)).astype(np.int32)
+    rs = (pulls * rng.uniform(0, 1, pulls.shape)).astype(np.float32)
+    keep = rng.integers(0, 16, (2, 200)).astype(np.uint32)
+    sc = oracle.score_select(labels, rng.uniform(0, 2, (2, 200)).astype(np.float32), pulls, rs, [50, 60], K=5, keep=keep,
+                             lipschitz_L=0.2)
+    a1, v1 = oracle.top_m(sc["arm_index"], 1)
+    np.testing.assert_array_equal(a1[:, 0], sc["best_arm"])
+    np.testing.assert_array_equal(v1[:, 0], sc["best_val"])
+    a7, _ = oracle.top_m(sc["arm_index"], 7)
+    a8, _ = oracle.top_m(sc["arm_index"], 8)
+    np.testing.assert_array_equal(a8[:, :7], a7)
