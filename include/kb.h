@@ -241,6 +241,21 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
 kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
                            int32_t* rows);
 
+/* The M best arms of every instance by the per-arm index (the masked argmax
+ * of Sec. 3.4 taken M times, for generating M candidates per iteration):
+ * top_arm[b][j] = flat index k*S + s of the arm with the j-th largest
+ * arm_index[b], larger value first, lower flat index first among equal
+ * values; pruned arms (-inf) and NaN entries never appear; when fewer than M
+ * arms are valid the tail is -1 (top_val -inf).  top_arm[b][0] is
+ * kb_score_select's best_arm.  Exact: comparisons only.
+ *   arm_index [B][N][S] in, as kb_score_select writes it
+ *   top_arm [B][M] out;  top_val [B][M] out, nullable;  0 <= M <= KB_TOP_M_MAX
+ * DEVICE memory.  M launches, each one pass over arm_index (meant for small
+ * M); needs the workspace of kb_workspace_bytes. */
+#define KB_TOP_M_MAX 128
+kb_status kb_select_top_m(kb_ctx* ctx, int B, int N, int S, int M, const float* arm_index, int32_t* top_arm,
+                          float* top_val);
+
 /* Cluster radius: radius[b][i] = max over the members k of cluster i of
  * sqrt(dist2[b][k]), 0 for an empty cluster.  Theorem 1's bound carries the
  * term L * max_i diam(C_i); through the centroid diam(C_i) <= 2 radius[i], so

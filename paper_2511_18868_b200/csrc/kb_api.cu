@@ -180,6 +180,7 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     need = max_sz(need, kb_ws_need_score(B, N, K, S));
     need = max_sz(need, kb_ws_need_sample(B));
     need = max_sz(need, kb_ws_need_seed(B, N, K));
+    need = max_sz(need, kb_ws_need_topm(B, KB_TOP_M_MAX));
     need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K));
     *out = need;
     return KB_OK;
@@ -343,6 +344,19 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
     TimeScope ts__(ctx, KB_T_SAMPLE);
     return kb_launch_sample_member(ctx, B, N, K, S, R, labels, cluster_arm, h_cand, target, theta_sat, seed, t, member,
                                    member_val);
+}
+
+kb_status kb_select_top_m(kb_ctx* ctx, int B, int N, int S, int M, const float* arm_index, int32_t* top_arm,
+                          float* top_val) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, S >= 1 && M >= 0, "kb_select_top_m: S must be >= 1 and M >= 0");
+    if (M > KB_TOP_M_MAX) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_select_top_m: M = %d exceeds %d", M, KB_TOP_M_MAX);
+    if ((long long)N * S > 0x7fffffffLL)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_select_top_m: N*S exceeds the 31-bit arm index");
+    if (B > 0 && M > 0) KB_REQUIRE(ctx, top_arm, "kb_select_top_m: top_arm is required");
+    if ((size_t)B * N > 0 && M > 0) KB_REQUIRE(ctx, arm_index, "kb_select_top_m: arm_index is required");
+    TimeScope ts__(ctx, KB_T_SCORE);
+    return kb_launch_top_m(ctx, B, N * S, M, arm_index, top_arm, top_val);
 }
 
 kb_status kb_cluster_radius(kb_ctx* ctx, int B, int N, int K, const int32_t* labels, const float* dist2, float* radius) {

@@ -1103,3 +1103,39 @@ def test_online_loop_regret_against_theorem1(kbx):
     assert int(host(d["pulls"]).sum()) == B * T
     print(f"[regret] first quarter {first:.4f}, last quarter {last:.4f}, average {reg.mean():.4f}, bound {bound:.4f}, "
           f"max radius {float(host(radius).max()):.3f}")
+
+
+# ------------------------------------------------------------------ top-M arms
+@pytest.mark.parametrize("B,N,S,M", [(1, 256, 8, 4), (3, 1000, 13, 7), (2, 20011, 16, 16), (1, 262144, 32, 8),
+                                     (64, 512, 16, 5), (2, 3, 4, 20), (1, 5000, 3, 128), (4, 0, 8, 3)])
+def test_select_top_m(kbx, B, N, S, M):
+    rng = np.random.default_rng(B + N + S + M)
+    a = (rng.integers(0, 4000, size=(B, N, S)) / 64.0).astype(np.float32)        # many exact ties
+    a[rng.uniform(size=a.shape) < 0.3] = -np.inf
+    if N > 10:
+        a[0, 5, 1] = np.nan
+        a[-1, N // 2:, :] = -np.inf
+    ws(kbx, B, N, 1, 1, S)
+    arm, val = empty((B, M), torch.int32), empty((B, M))
+    kbx.select_top_m(dev(a), arm, val)
+    ra, rv = oracle.top_m(a, M)
+    np.testing.assert_array_equal(host(arm), ra)                                 # comparisons only: bit-exact
+    np.testing.assert_array_equal(host(val), rv)
+    assert kbx.device_status() == 0
+
+
+def test_select_top_m_follows_score_select(kbx):
+    cfg = wl.scaled(wl.CONFIGS["medium"], B=2, N=3000, K=16, S=8)
+    inp = wl.make_inputs(cfg, seed=2)
+    rng = np.random.default_rng(1)
+    labels = rng.integers(0, 16, (2, 3000)).astype(np.int32)
+    dist2 = rng.uniform(0, 3, (2, 3000)).astype(np.float32)
+    keep = rng.integers(0, 256, (2, 3000)).astype(np.uint32)
+    got = run_score(kbx, labels, dist2, inp["pulls"], inp["reward_sum"], inp["t"], 16, keep, lipschitz_L=0.1)
+    arm, val = empty((2, 6), torch.int32), empty((2, 6))
+    kbx.select_top_m(dev(got["arm_index"]), arm, val)
+    np.testing.assert_array_equal(host(arm)[:, 0], got["best_arm"])
+    np.testing.assert_array_equal(host(val)[:, 0], got["best_val"])
+    ra, rv = oracle.top_m(got["arm_index"], 6)
+    np.testing.assert_array_equal(host(arm), ra)
+    np.testing.assert_array_equal(host(val), rv)
