@@ -444,6 +444,24 @@ def run_ours(args, cfg):
                        "max_radius": float(radius.max()),
                        "what": "kb_cluster_radius on the step's labels and dist2 (memset node + kernel, after an L2 flush)"}
 
+        # ---- the 8 best arms of the step's per-arm index (M candidates per iteration; outside the timed step)
+        top_m = 8
+        top_arm = torch.empty((cfg.B, top_m), dtype=torch.int32, device=device)
+        ctx.select_top_m(dev_t["arm_index"], top_arm)
+        torch.cuda.synchronize()
+        ta, tb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush.zero_()
+        ta.record()
+        ctx.select_top_m(dev_t["arm_index"], top_arm)
+        tb.record()
+        torch.cuda.synchronize()
+        top_ms = ta.elapsed_time(tb)
+        top_bytes = top_m * cfg.arms * 4
+        top_line = {"M": top_m, "us": top_ms * 1e3, "us_per_rank": top_ms * 1e3 / top_m, "algorithmic_bytes": top_bytes,
+                    "GBps": top_bytes / (top_ms * 1e-3) / 1e9, "hbm_frac": top_bytes / (top_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "what": "kb_select_top_m on the step's arm_index: M launches, each one pass (after an L2 flush; the "
+                            "later passes may find the array in L2)"}
+
         # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
         # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
         # replayed as one CUDA graph; consecutive iterations, so L2 keeps what it can (no flush: that is the loop's state).
@@ -494,7 +512,7 @@ def run_ours(args, cfg):
                              "iterations (L2 not flushed), per rank"}
 
         return {"sample_member": sample_line, "seed_kmeanspp": seed_line, "cluster_radius": radius_line,
-                "online_iteration": loop_line}
+                "online_iteration": loop_line, "select_top_m": top_line}
 
     try:
         extra = extras()
