@@ -239,6 +239,30 @@ def top_m(arm_index, M):
     return top_arm, top_val
 
 
+def select_pair(cl_pulls, cl_mean, t, c=2.0, hsig=None, target=None, theta_sat=75.0):
+    """Masked-UCB choice of (I_t, S_t) from the cluster tables (see kbo_select_pair)."""
+    cl_pulls, cl_mean, t = _f32(cl_pulls), _f32(cl_mean), _i32(t)
+    B, K, S = cl_pulls.shape
+    R = 1
+    if hsig is not None:
+        hsig, target = _f32(hsig), _i32(target)
+        R = hsig.shape[2]
+    cl_index = np.empty((B, K, S), np.float32)
+    pair = np.empty((B,), np.int32)
+    _check(_load().kbo_select_pair(B, K, S, R, ctypes.c_float(c), _p(cl_pulls), _p(cl_mean), _p(t), _p(hsig),
+                                   _p(target), ctypes.c_float(theta_sat), _p(cl_index), _p(pair)), "select_pair")
+    return {"pair": pair, "cl_index": cl_index}
+
+
+def update_pair(pair, reward, cl_pulls, cl_mean):
+    """Algorithm 1's N <- N + 1, mu <- mu + (r - mu) / N for the chosen pair.  Returns new copies."""
+    pair, reward = _i32(pair), _f32(reward)
+    cl_pulls, cl_mean = _f32(cl_pulls).copy(), _f32(cl_mean).copy()
+    B, K, S = cl_pulls.shape
+    _check(_load().kbo_update_pair(B, K, S, _p(pair), _p(reward), _p(cl_pulls), _p(cl_mean)), "update_pair")
+    return cl_pulls, cl_mean
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

@@ -577,4 +577,52 @@ int kbo_top_m(int B, int NS, int M, const float* arm_index, int32_t* top_arm, fl
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Algorithm 1's loop kept on the cluster tables themselves (no pass over the candidates):
+//
+// kbo_select_pair: the masked-UCB choice (Sec. 3.4, masked-UCB equation; Algorithm 1 "Select (I_t, S_t)")
+//     (I_t, S_t) = argmax over pairs with M_{i,s} = 1 of  mu_{i,s} + c sqrt(ln t / N_{i,s}),
+//     M_{i,s} = [ h_c^(i)[Target(s)] < theta_sat ]  (Algorithm 1, "Hardware-constrained selection";
+//     hsig null: no pair is masked).  Lowest i*S + s on ties; -1 when every pair is masked.
+// kbo_update_pair: Algorithm 1's two statistics lines for the chosen pair, literally:
+//     N <- N + 1,  mu <- mu + (r - mu) / N.
+// ---------------------------------------------------------------------------
+int kbo_select_pair(int B, int K, int S, int R, float c, const float* cl_pulls, const float* cl_mean, const int32_t* t,
+                    const float* hsig, const int32_t* target, float theta_sat, float* cl_index, int32_t* pair) {
+    for (int b = 0; b < B; ++b) {
+        const double lnt = std::log((double)t[b]);
+        double best = -kInf;
+        int arg = -1;
+        for (int i = 0; i < K; ++i)
+            for (int s = 0; s < S; ++s) {
+                const double n = (double)cl_pulls[ix3(b, i, s, K, S)];
+                const double u = (double)cl_mean[ix3(b, i, s, K, S)] + (double)c * std::sqrt(lnt / n);
+                if (cl_index) cl_index[ix3(b, i, s, K, S)] = (float)u;
+                bool valid = true;
+                if (hsig) {
+                    const int col = target[s];
+                    if (col < 0 || col >= R) return 2;
+                    valid = (double)hsig[ix3(b, i, col, K, R)] < (double)theta_sat;
+                }
+                if (valid && u > best) { best = u; arg = i * S + s; }
+            }
+        pair[b] = arg;
+    }
+    return 0;
+}
+
+int kbo_update_pair(int B, int K, int S, const int32_t* pair, const float* reward, float* cl_pulls, float* cl_mean) {
+    for (int b = 0; b < B; ++b) {
+        const int p = pair[b];
+        if (p < 0) continue;
+        if (p >= K * S) return 2;
+        const size_t i = (size_t)b * K * S + p;
+        const double n = (double)cl_pulls[i] + 1.0;
+        const double mu = (double)cl_mean[i] + ((double)reward[b] - (double)cl_mean[i]) / n;
+        cl_pulls[i] = (float)n;
+        cl_mean[i] = (float)mu;
+    }
+    return 0;
+}
+
 }  // extern "C"

@@ -656,3 +656,64 @@ def test_top_m_is_the_sorted_prefix():
     a7, _ = oracle.top_m(sc["arm_index"], 7)
     a8, _ = oracle.top_m(sc["arm_index"], 8)
     np.testing.assert_array_equal(a8[:, :7], a7)
+
+
+# -------------------------------------------- the loop on the cluster tables
+def test_select_pair_worked_values_and_mask():
+    # the golden index values, one pair at a time
+    for t, n, mu, c, u in read_golden("masked_ucb_index.txt"):
+        out = oracle.select_pair(np.full((1, 1, 1), n, np.float32), np.full((1, 1, 1), mu, np.float32), [int(t)], c=c)
+        assert out["cl_index"][0, 0, 0] == pytest.approx(u, abs=2e-6) and out["pair"][0] == 0
+    # against the whole-array statistics: same tables in, same cluster-level choice out (no arm masked)
+    rng = np.random.default_rng(8)
+    B, N, K, S = 5, 300, 6, 4
+    labels = rng.integers(0, K, (B, N)).astype(np.int32)
+    pulls = rng.poisson(2.0, (B, N, S)).astype(np.int32)
+    rs = (pulls * rng.uniform(0, 1, pulls.shape)).astype(np.float32)
+    t = (1 + pulls.reshape(B, -1).sum(1)).astype(np.int32)
+    sc = oracle.score_select(labels, np.zeros((B, N), np.float32), pulls, rs, t, K=K)
+    sp = oracle.select_pair(sc["cl_pulls"], sc["cl_mean"], t)
+    np.testing.assert_array_equal(sp["pair"], sc["best_cluster_arm"])
+    np.testing.assert_allclose(sp["cl_index"], sc["cl_index"], atol=2e-6)
+    # the saturation mask of Algorithm 1: M_{i,s} = [h_c^(i)[Target(s)] < theta]; brute force over the unmasked pairs
+    hsig = rng.uniform(0, 100, (B, K, 3)).astype(np.float32)
+    target = np.array([2, 0, 1, 0], np.int32)
+    spm = oracle.select_pair(sc["cl_pulls"], sc["cl_mean"], t, hsig=hsig, target=target, theta_sat=60.0)
+    for b in range(B):
+        valid = hsig[b][:, target] < 60.0                                   # [K][S]
+        u = np.where(valid, sc["cl_index"][b].astype(np.float64), -np.inf)
+        assert spm["pair"][b] == (int(np.argmax(u.reshape(-1))) if valid.any() else -1)
+    none = oracle.select_pair(sc["cl_pulls"], sc["cl_mean"], t, hsig=hsig, target=target, theta_sat=-1.0)
+    assert np.all(none["pair"] == -1)
+
+
+def test_update_pair_is_algorithm1_and_matches_the_aggregate():
+    for r1, r2, r3, r4, n_fin, mu_fin in read_golden("running_mean.txt"):
+        n = np.ones((1, 2, 3), np.float32)
+        mu = np.full((1, 2, 3), 0.5, np.float32)
+        for r in (r1, r2, r3, r4):
+            n, mu = oracle.update_pair([1 * 3 + 2], [r], n, mu)
+        assert n[0, 1, 2] == n_fin and mu[0, 1, 2] == pytest.approx(mu_fin, abs=1e-6)
+        assert n.sum() == 5 + n_fin and mu[0, 0, 0] == 0.5                   # the other pairs untouched
+    n2, mu2 = oracle.update_pair([-1], [0.7], n, mu)                         # nothing chosen: nothing changes
+    assert np.array_equal(n2, n) and np.array_equal(mu2, mu)
+    # incremental tables track the per-arm bookkeeping of record_outcome + score_select
+    rng = np.random.default_rng(2)
+    B, N, K, S = 3, 50, 4, 3
+    labels = rng.integers(0, K, (B, N)).astype(np.int32)
+    pulls = np.zeros((B, N, S), np.int32)
+    rs = np.zeros((B, N, S), np.float32)
+    t = np.ones(B, np.int32)
+    n = np.ones((B, K, S), np.float32)
+    mu = np.full((B, K, S), 0.5, np.float32)
+    for it in range(40):
+        k = rng.integers(0, N, B).astype(np.int32)
+        s = rng.integers(0, S, B)
+        pair = (labels[np.arange(B), k] * S + s).astype(np.int32)
+        t_new = rng.uniform(0.2, 1.4, B).astype(np.float32)
+        out = oracle.record_outcome(k, pair, np.ones((B, N), np.float32), t_new, pulls, rs, t)
+        pulls, rs, t = out["pulls"], out["reward_sum"], out["t"]
+        n, mu = oracle.update_pair(pair, out["reward"], n, mu)
+    sc = oracle.score_select(labels, np.zeros((B, N), np.float32), pulls, rs, t, K=K)
+    np.testing.assert_array_equal(n, sc["cl_pulls"])
+    np.testing.assert_allclose(mu, sc["cl_mean"], atol=2e-6)
