@@ -286,14 +286,38 @@ kb_status kb_cluster_radius(kb_ctx* ctx, int B, int N, int K, const int32_t* lab
  *   verified [B] in, nullable = every k'_t passed
  *   pulls, reward_sum [B][N][S] in/out;  t [B] in/out
  *   reward [B] out, nullable: r_t as recorded (0 where nothing was updated)
- * All arrays in DEVICE memory.  member >= N, or a negative cluster_arm beside
- * a drawn member, sets bit 4 of the device status word and updates nothing.
- * One launch, no workspace; meant to be chained after kb_score_select and
- * kb_sample_member on one stream (or inside one CUDA graph). */
-kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,
+ *   cl_pulls, cl_mean [B][K][S] in/out, nullable (both or neither): the
+ *     cluster tables kept alongside, updated for the chosen pair by
+ *     Algorithm 1's two lines literally (N <- N + 1, mu <- mu + (r_t - mu)/N)
+ *     whenever a pull is recorded, so that kb_select_pair can choose the next
+ *     pair without a pass over the candidates
+ * All arrays in DEVICE memory.  member >= N, a negative cluster_arm beside a
+ * drawn member, or (with tables) cluster_arm >= K*S sets bit 4 of the device
+ * status word and updates nothing.  One launch, no workspace; meant to be
+ * chained after the selection and kb_sample_member on one stream (or inside
+ * one CUDA graph). */
+kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int K, int S, int failures_count, const int32_t* member,
                             const int32_t* cluster_arm, const float* t_cur, const float* t_new,
                             const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
-                            float* reward);
+                            float* reward, float* cl_pulls, float* cl_mean);
+
+/* The masked-UCB choice of the pair from the cluster tables alone (Sec. 3.4,
+ * masked-UCB equation; Algorithm 1, "Select (I_t, S_t)"):
+ *   pair[b] = lowest i*S + s maximising mu_{i,s} + c*sqrt(ln t / N_{i,s})
+ *             over the pairs with M_{i,s} = 1 (-1 if none),
+ *   M_{i,s} = [ hsig[b][i][target[s]] < theta_sat ]   (Algorithm 1,
+ *             "Hardware-constrained selection"); hsig null: no pair is masked.
+ * With tables that kb_score_select produced once after a (re-)clustering and
+ * kb_record_outcome keeps current, an iteration costs K*S entries instead of
+ * a pass over all arms.
+ *   cl_pulls, cl_mean [B][K][S] in;  t [B] in, >= 1
+ *   hsig [B][K][R] in, nullable;  target [S] in (required with hsig)
+ *   cl_index [B][K][S] out, nullable;  pair [B] out
+ * DEVICE memory.  One launch (one CTA per instance), no workspace.  A target
+ * outside [0, R) sets bit 2 of the device status word (pair masked). */
+kb_status kb_select_pair(kb_ctx* ctx, int B, int K, int S, int R, float c, const float* cl_pulls,
+                         const float* cl_mean, const int32_t* t, const float* hsig, const int32_t* target,
+                         float theta_sat, float* cl_index, int32_t* pair);
 
 /* Which kernel kb_cluster_assign uses.
  *   path: 0 = automatic (tensor cores when K >= 128, D a multiple of 32 and

@@ -379,18 +379,34 @@ kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float*
     return kb_launch_seed_kmeanspp(ctx, B, N, D, K, z, seed, rows);
 }
 
-kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,
+kb_status kb_select_pair(kb_ctx* ctx, int B, int K, int S, int R, float c, const float* cl_pulls, const float* cl_mean,
+                         const int32_t* t, const float* hsig, const int32_t* target, float theta_sat, float* cl_index,
+                         int32_t* pair) {
+    KB_COMMON(ctx, B, 0);
+    KB_REQUIRE(ctx, K >= 1 && S >= 1 && R >= 1, "kb_select_pair: K, S and R must be >= 1");
+    if ((long long)K * S > 0x7fffffffLL) return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_select_pair: K*S exceeds 31 bits");
+    if (B > 0) {
+        KB_REQUIRE(ctx, cl_pulls && cl_mean && t && pair, "kb_select_pair: cl_pulls, cl_mean, t and pair are required");
+        KB_REQUIRE(ctx, !hsig || target, "kb_select_pair: the saturation mask needs target");
+    }
+    TimeScope ts__(ctx, KB_T_SCORE);
+    return kb_launch_select_pair(ctx, B, K, S, R, c, cl_pulls, cl_mean, t, hsig, target, theta_sat, cl_index, pair);
+}
+
+kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int K, int S, int failures_count, const int32_t* member,
                             const int32_t* cluster_arm, const float* t_cur, const float* t_new,
-                            const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t, float* reward) {
+                            const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t, float* reward,
+                            float* cl_pulls, float* cl_mean) {
     KB_COMMON(ctx, B, N);
-    KB_REQUIRE(ctx, S >= 1, "kb_record_outcome: S must be >= 1");
+    KB_REQUIRE(ctx, S >= 1 && K >= 1, "kb_record_outcome: K and S must be >= 1");
+    KB_REQUIRE(ctx, (cl_pulls != nullptr) == (cl_mean != nullptr), "kb_record_outcome: cl_pulls and cl_mean go together");
     if (B > 0) {
         KB_REQUIRE(ctx, member && cluster_arm && t_new && t, "kb_record_outcome: member, cluster_arm, t_new and t are required");
         if (N > 0) KB_REQUIRE(ctx, t_cur && pulls && reward_sum, "kb_record_outcome: t_cur, pulls and reward_sum are required");
     }
     TimeScope ts__(ctx, KB_T_SAMPLE);
-    return kb_launch_record_outcome(ctx, B, N, S, failures_count, member, cluster_arm, t_cur, t_new, verified, pulls,
-                                    reward_sum, t, reward);
+    return kb_launch_record_outcome(ctx, B, N, K, S, failures_count, member, cluster_arm, t_cur, t_new, verified, pulls,
+                                    reward_sum, t, reward, cl_pulls, cl_mean);
 }
 
 kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,

@@ -141,10 +141,13 @@ kb_status kb_launch_score(kb_ctx*, int B, int N, int K, int S, kb_score_params p
                           const float* dist2, const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
                           const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
                           float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm);
-kb_status kb_launch_record_outcome(kb_ctx*, int B, int N, int S, int failures_count, const int32_t* member,
+kb_status kb_launch_record_outcome(kb_ctx*, int B, int N, int K, int S, int failures_count, const int32_t* member,
                                    const int32_t* cluster_arm, const float* t_cur, const float* t_new,
                                    const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
-                                   float* reward);
+                                   float* reward, float* cl_pulls, float* cl_mean);
+kb_status kb_launch_select_pair(kb_ctx*, int B, int K, int S, int R, float c, const float* cl_pulls, const float* cl_mean,
+                                const int32_t* t, const float* hsig, const int32_t* target, float theta_sat,
+                                float* cl_index, int32_t* pair);
 kb_status kb_launch_cluster_radius(kb_ctx*, int B, int N, int K, const int32_t* labels, const float* dist2, float* radius);
 size_t kb_ws_need_topm(int B, int M);
 kb_status kb_launch_top_m(kb_ctx*, int B, int NS, int M, const float* arm_index, int32_t* top_arm, float* top_val);

@@ -12,11 +12,12 @@
 
 namespace {
 
-__global__ void record_outcome_kernel(int B, int N, int S, int failures_count, const int32_t* __restrict__ member,
+__global__ void record_outcome_kernel(int B, int N, int K, int S, int failures_count, const int32_t* __restrict__ member,
                                       const int32_t* __restrict__ cluster_arm, const float* __restrict__ t_cur,
                                       const float* __restrict__ t_new, const int32_t* __restrict__ verified,
                                       int32_t* __restrict__ pulls, float* __restrict__ reward_sum,
                                       int32_t* __restrict__ t, float* __restrict__ reward,
+                                      float* __restrict__ cl_pulls, float* __restrict__ cl_mean,
                                       int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -26,7 +27,7 @@ __global__ void record_outcome_kernel(int B, int N, int S, int failures_count, c
     const int k = member[b];
     const int ca = cluster_arm[b];
     if (k >= 0) {
-        if (k >= N || ca < 0) {
+        if (k >= N || ca < 0 || (cl_pulls && ca >= K * S)) {
             atomicOr(dev_status, 4);
         } else {
             const bool ok = verified ? verified[b] != 0 : true;
@@ -40,6 +41,14 @@ __global__ void record_outcome_kernel(int B, int N, int S, int failures_count, c
                 const size_t i = ((size_t)b * N + k) * S + (ca % S);
                 pulls[i] += 1;
                 reward_sum[i] += r;
+                if (cl_pulls) {
+                    // the cluster tables kept alongside: Algorithm 1's two lines, literally
+                    const size_t p = (size_t)b * K * S + ca;
+                    const float n = cl_pulls[p] + 1.f;
+                    const float mu = cl_mean[p];
+                    cl_pulls[p] = n;
+                    cl_mean[p] = mu + (r - mu) / n;
+                }
             }
         }
     }
@@ -48,13 +57,65 @@ __global__ void record_outcome_kernel(int B, int N, int S, int failures_count, c
 
 }  // namespace
 
-kb_status kb_launch_record_outcome(kb_ctx* ctx, int B, int N, int S, int failures_count, const int32_t* member,
+kb_status kb_launch_record_outcome(kb_ctx* ctx, int B, int N, int K, int S, int failures_count, const int32_t* member,
                                    const int32_t* cluster_arm, const float* t_cur, const float* t_new,
                                    const int32_t* verified, int32_t* pulls, float* reward_sum, int32_t* t,
-                                   float* reward) {
+                                   float* reward, float* cl_pulls, float* cl_mean) {
     if (B == 0) return KB_OK;
-    kb_launch(record_outcome_kernel, (B + 127) / 128, 128, 0, ctx->stream, B, N, S, failures_count, member, cluster_arm,
-              t_cur, t_new, verified, pulls, reward_sum, t, reward, ctx->dev_status);
+    kb_launch(record_outcome_kernel, (B + 127) / 128, 128, 0, ctx->stream, B, N, K, S, failures_count, member, cluster_arm,
+              t_cur, t_new, verified, pulls, reward_sum, t, reward, cl_pulls, cl_mean, ctx->dev_status);
     KB_LAUNCH_CHECK(ctx, "record_outcome_kernel");
+    return KB_OK;
+}
+
+// ---- the masked-UCB choice of the pair from the cluster tables (Sec. 3.4; Algorithm 1, "Select (I_t, S_t)") ----
+namespace {
+constexpr int SP_T = 128;
+__global__ void __launch_bounds__(SP_T)
+select_pair_kernel(int K, int S, int R, float c, const float* __restrict__ cl_pulls, const float* __restrict__ cl_mean,
+                   const int32_t* __restrict__ t, const float* __restrict__ hsig, const int32_t* __restrict__ target,
+                   float theta, float* __restrict__ cl_index, int32_t* __restrict__ pair, int* __restrict__ dev_status) {
+    kb_grid_dependency_wait();
+    __shared__ unsigned long long s_red[SP_T / 32];
+    const int b = blockIdx.x, tid = threadIdx.x, KS = K * S;
+    const float lnt = logf((float)t[b]);
+    unsigned long long best = 0ull;
+    for (int e = tid; e < KS; e += SP_T) {
+        const size_t o = (size_t)b * KS + e;
+        const float u = cl_mean[o] + c * sqrtf(lnt / cl_pulls[o]);
+        if (cl_index) cl_index[o] = u;
+        bool valid = true;
+        if (hsig) {
+            const int i = e / S, col = target[e - i * S];
+            if (col < 0 || col >= R) { atomicOr(dev_status, 2); valid = false; }
+            else valid = hsig[((size_t)b * K + i) * R + col] < theta;
+        }
+        if (valid) {
+            const unsigned long long key = ((unsigned long long)kb_orderable(u) << 32) | (0xffffffffu - (unsigned)e);
+            best = key > best ? key : best;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+        best = other > best ? other : best;
+    }
+    if ((tid & 31) == 0) s_red[tid >> 5] = best;
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+        for (int w = 1; w < SP_T / 32; ++w) best = s_red[w] > best ? s_red[w] : best;
+        pair[b] = best ? (int32_t)(0xffffffffu - (unsigned)(best & 0xffffffffull)) : -1;
+    }
+}
+}  // namespace
+
+kb_status kb_launch_select_pair(kb_ctx* ctx, int B, int K, int S, int R, float c, const float* cl_pulls,
+                                const float* cl_mean, const int32_t* t, const float* hsig, const int32_t* target,
+                                float theta_sat, float* cl_index, int32_t* pair) {
+    if (B == 0) return KB_OK;
+    kb_launch(select_pair_kernel, B, SP_T, 0, ctx->stream, K, S, R, c, cl_pulls, cl_mean, t, hsig, target, theta_sat, cl_index,
+              pair, ctx->dev_status);
+    KB_LAUNCH_CHECK(ctx, "select_pair_kernel");
     return KB_OK;
 }

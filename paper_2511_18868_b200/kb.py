@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
-           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m",
+           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc"]
 
@@ -89,7 +89,8 @@ def load_library() -> ctypes.CDLL:
     lib.kb_cluster_update.argtypes = [_VP, i, i, i, i] + [_VP] * 4
     lib.kb_score_select.argtypes = [_VP, i, i, i, i, ScoreParams] + [_VP] * 14
     lib.kb_sample_member.argtypes = [_VP, i, i, i, i, i] + [_VP] * 4 + [f, ctypes.c_uint64] + [_VP] * 3
-    lib.kb_record_outcome.argtypes = [_VP, i, i, i, i] + [_VP] * 9
+    lib.kb_record_outcome.argtypes = [_VP, i, i, i, i, i] + [_VP] * 11
+    lib.kb_select_pair.argtypes = [_VP, i, i, i, i, f] + [_VP] * 5 + [f, _VP, _VP]
     lib.kb_cluster_radius.argtypes = [_VP, i, i, i, _VP, _VP, _VP]
     lib.kb_select_top_m.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_seed_kmeanspp.argtypes = [_VP, i, i, i, i, _VP, ctypes.c_uint64, _VP]
@@ -280,13 +281,24 @@ class KB:
                                               self._p(rows)), "kb_seed_kmeanspp")
 
     def record_outcome(self, member, cluster_arm, t_cur, t_new, pulls, reward_sum, t, verified=None, reward=None,
-                       failures_count=False):
-        """Reward clip and statistics update of one iteration (Algorithm 1, "Generation & update"), in place."""
+                       failures_count=False, cl_pulls=None, cl_mean=None):
+        """Reward clip and statistics update of one iteration (Algorithm 1, "Generation & update"), in place;
+        with cl_pulls / cl_mean [B][K][S] the cluster tables are updated alongside."""
         B, N, S = pulls.shape
-        self._check(self.lib.kb_record_outcome(self.h, B, N, S, int(bool(failures_count)), self._p(member),
+        K = cl_pulls.shape[1] if cl_pulls is not None else 1
+        self._check(self.lib.kb_record_outcome(self.h, B, N, K, S, int(bool(failures_count)), self._p(member),
                                                self._p(cluster_arm), self._p(t_cur), self._p(t_new),
                                                self._p(verified), self._p(pulls), self._p(reward_sum), self._p(t),
-                                               self._p(reward)), "kb_record_outcome")
+                                               self._p(reward), self._p(cl_pulls), self._p(cl_mean)),
+                    "kb_record_outcome")
+
+    def select_pair(self, cl_pulls, cl_mean, t, pair, c=2.0, hsig=None, target=None, theta_sat=75.0, cl_index=None):
+        """Masked-UCB choice of (I_t, S_t) from the cluster tables alone (Algorithm 1, "Select (I_t, S_t)")."""
+        B, K, S = cl_pulls.shape
+        R = hsig.shape[2] if hsig is not None else 1
+        self._check(self.lib.kb_select_pair(self.h, B, K, S, R, float(c), self._p(cl_pulls), self._p(cl_mean),
+                                            self._p(t), self._p(hsig), self._p(target), float(theta_sat),
+                                            self._p(cl_index), self._p(pair)), "kb_select_pair")
 
     def set_assign_options(self, path: int = 0, tc_eps: float = 0.0):
         """path: 0 automatic, 1 fp32 row-wise kernel, 2 tensor-core kernel."""

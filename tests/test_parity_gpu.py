@@ -1139,3 +1139,89 @@ def test_select_top_m_follows_score_select(kbx):
     ra, rv = oracle.top_m(got["arm_index"], 6)
     np.testing.assert_array_equal(host(arm), ra)
     np.testing.assert_array_equal(host(val), rv)
+
+
+# -------------------------------------------- the loop on the cluster tables
+@pytest.mark.parametrize("B,K,S,masked", [(1, 8, 8, True), (5, 3, 4, False), (64, 16, 16, True), (2, 1024, 8, True),
+                                          (3, 1, 1, False), (2, 300, 32, True)])
+def test_select_pair(kbx, B, K, S, masked):
+    rng = np.random.default_rng(B + K + S)
+    n = (1 + rng.poisson(5.0, (B, K, S))).astype(np.float32)
+    mu = rng.uniform(0, 1, (B, K, S)).astype(np.float32)
+    t = rng.integers(1, 5000, B).astype(np.int32)
+    hsig = rng.uniform(0, 100, (B, K, wl.R_RESOURCES)).astype(np.float32) if masked else None
+    target = (np.arange(S) % wl.R_RESOURCES).astype(np.int32)
+    if masked and B > 1:
+        hsig[1] = 99.0                                   # instance 1: every pair saturated
+    pair, cl_index = empty((B,), torch.int32), empty((B, K, S))
+    kbx.select_pair(dev(n), dev(mu), dev(t), pair, c=2.0, hsig=None if hsig is None else dev(hsig), target=dev(target),
+                    theta_sat=75.0, cl_index=cl_index)
+    ref = oracle.select_pair(n, mu, t, c=2.0, hsig=hsig, target=target, theta_sat=75.0)
+    parity.close(host(cl_index), ref["cl_index"], atol=1e-6, what="cl_index")
+    got = host(pair)
+    u = ref["cl_index"].astype(np.float64).reshape(B, -1)
+    for b in range(B):
+        if ref["pair"][b] < 0:
+            assert got[b] == -1
+        elif got[b] != ref["pair"][b]:                   # a near-tie of two pairs: either is a valid choice
+            assert got[b] >= 0 and abs(u[b, got[b]] - u[b, ref["pair"][b]]) <= 1e-5 * max(1.0, abs(u[b, ref["pair"][b]]))
+            if hsig is not None:
+                assert hsig[b, got[b] // S, target[got[b] % S]] < 75.0
+    if masked and B > 1:
+        assert got[1] == -1
+    assert kbx.device_status() == 0
+
+
+def test_table_loop_matches_the_per_arm_bookkeeping(kbx):
+    """Algorithm 1's loop on the cluster tables: kb_score_select once, then T iterations of kb_select_pair ->
+    kb_sample_member -> kb_record_outcome (which keeps per-arm statistics and tables current), with no pass over the
+    arms.  Every iteration is checked against the oracle from the GPU's state; at the end the tables must equal what
+    kb_score_select makes of the per-arm statistics (counts exactly, means within rounding)."""
+    B, N, K, S, T = 8, 900, 6, 4, 60
+    cfg = wl.scaled(wl.CONFIGS["medium"], B=B, N=N, D=16, K=K, components=6, S=S, iters=2)
+    inp = wl.make_inputs(cfg, seed=12)
+    rng = np.random.default_rng(5)
+    labels = rng.integers(0, K, (B, N)).astype(np.int32)
+    h_cand = wl.make_candidate_signatures(inp["hsig"], labels, seed=4)
+    gain = rng.uniform(-0.3, 0.7, (B, N, S)).astype(np.float32)
+    ws(kbx, B, N, 16, K, S)
+    d = {k: dev(v) for k, v in dict(labels=labels, dist2=np.zeros((B, N), np.float32), pulls=inp["pulls"],
+                                    reward_sum=inp["reward_sum"], t=inp["t"], h_cand=h_cand, target=inp["target"],
+                                    t_cur=inp["t_cur"], gain=gain, hsig=inp["hsig"]).items()}
+    cl_pulls, cl_mean, cl_index = empty((B, K, S)), empty((B, K, S)), empty((B, K, S))
+    best_arm, best_val, pair0 = empty((B,), torch.int32), empty((B,)), empty((B,), torch.int32)
+    kbx.score_select(d["labels"], d["dist2"], d["pulls"], d["reward_sum"], d["t"], cl_pulls, cl_mean, cl_index, best_arm,
+                     best_val, pair0)
+    pair, member, t_new, reward = empty((B,), torch.int32), empty((B,), torch.int32), empty((B,)), empty((B,))
+    ar = torch.arange(B, device="cuda")
+    trace = []
+    for it in range(T):
+        before = (cl_pulls.clone(), cl_mean.clone(), d["t"].clone())
+        kbx.select_pair(cl_pulls, cl_mean, d["t"], pair, c=2.0, hsig=d["hsig"], target=d["target"], theta_sat=75.0)
+        kbx.sample_member(d["labels"], pair, d["h_cand"], d["target"], d["t"], member, K, 75.0, 777)
+        k, s = member.clamp(min=0).long(), (pair.clamp(min=0) % S).long()
+        t_new.copy_(d["t_cur"][ar, k] * (1.0 - d["gain"][ar, k, s]))
+        kbx.record_outcome(member, pair, d["t_cur"], t_new, d["pulls"], d["reward_sum"], d["t"], reward=reward,
+                           cl_pulls=cl_pulls, cl_mean=cl_mean)
+        trace.append((before, pair.clone(), member.clone(), reward.clone(), (cl_pulls.clone(), cl_mean.clone())))
+    # what the full pass makes of the per-arm statistics now
+    f_pulls, f_mean = empty((B, K, S)), empty((B, K, S))
+    kbx.score_select(d["labels"], d["dist2"], d["pulls"], d["reward_sum"], d["t"], f_pulls, f_mean, cl_index, best_arm,
+                     best_val, pair0)
+    torch.cuda.synchronize()
+    assert kbx.device_status() == 0
+    for before, pair_g, member_g, reward_g, after in trace:
+        n0, m0, t0 = (host(x) for x in before)
+        sp = oracle.select_pair(n0, m0, t0, c=2.0, hsig=inp["hsig"], target=inp["target"], theta_sat=75.0)
+        pg = host(pair_g)
+        u = sp["cl_index"].astype(np.float64).reshape(B, -1)
+        for b in range(B):
+            assert pg[b] == sp["pair"][b] or (pg[b] >= 0 and abs(u[b, pg[b]] - u[b, sp["pair"][b]]) <= 1e-5 * max(1.0, abs(u[b, sp["pair"][b]])))
+        dr = oracle.sample_member(labels, pg, h_cand, inp["target"], 75.0, 777, t0, K)
+        parity.member_match(host(member_g), None, dr, SAMPLE_TOL)
+        n1, m1 = oracle.update_pair(np.where(host(member_g) >= 0, pg, -1), host(reward_g), n0, m0)
+        np.testing.assert_array_equal(host(after[0]), n1)
+        parity.close(host(after[1]), m1, atol=1e-6, what="cl_mean after the update")
+    np.testing.assert_array_equal(host(cl_pulls), host(f_pulls))
+    parity.close(host(cl_mean), host(f_mean), atol=2e-6, what="tables against the full pass")
+    assert int(host(d["pulls"]).sum() - inp["pulls"].sum()) == int((np.stack([host(x[2]) for x in trace]) >= 0).sum())
