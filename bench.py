@@ -507,7 +507,38 @@ def run_ours(args, cfg):
             ctx.set_stream(main_stream)
         main_stream.wait_stream(side)
         graph_us = timed(graph.replay, n_loop)
+        # the same iteration on the cluster tables: kb_select_pair instead of the pass over the arms, the tables kept
+        # current by kb_record_outcome (Algorithm 1's own bookkeeping)
+        tab_pulls, tab_mean = outs["cl_pulls"].clone(), outs["cl_mean"].clone()
+        pair_t = torch.empty((cfg.B,), dtype=torch.int32, device=device)
+
+        def table_iteration():
+            ctx.select_pair(tab_pulls, tab_mean, loop_t["t"], pair_t, c=float(inp["c"]), hsig=dev_t["hsig"],
+                            target=dev_t["target"], theta_sat=float(inp["theta_sat"]))
+            ctx.sample_member(dev_t["labels"], pair_t, h_cand, dev_t["target"], loop_t["t"], member, cfg.K,
+                              float(inp["theta_sat"]), 0xC0FFEE)
+            ctx.record_outcome(member, pair_t, dev_t["t_cur"], t_new, loop_t["pulls"], loop_t["reward_sum"], loop_t["t"],
+                               cl_pulls=tab_pulls, cl_mean=tab_mean)
+
+        kt0, _ = ctx.launch_count()
+        table_iteration()
+        kt1, _ = ctx.launch_count()
+        table_eager_us = timed(table_iteration, n_loop)
+        side2 = torch.cuda.Stream()
+        side2.wait_stream(main_stream)
+        ctx.set_stream(side2)
+        try:
+            graph2 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph2, stream=side2, capture_error_mode="thread_local"):
+                table_iteration()
+        finally:
+            ctx.set_stream(main_stream)
+        main_stream.wait_stream(side2)
+        table_graph_us = timed(graph2.replay, n_loop)
         loop_line = {"eager_us": eager_us, "graph_us": graph_us, "kernels": int(kl1 - kl0), "iterations_timed": n_loop,
+                     "on_tables": {"eager_us": table_eager_us, "graph_us": table_graph_us, "kernels": int(kt1 - kt0),
+                                   "what": "kb_select_pair + kb_sample_member + kb_record_outcome (cluster tables kept "
+                                           "current; no pass over the arms)"},
                      "what": "kb_score_select + kb_sample_member + kb_record_outcome on the step's labels, consecutive "
                              "iterations (L2 not flushed), per rank"}
 

@@ -70,17 +70,18 @@ kb_status kb_launch_record_outcome(kb_ctx* ctx, int B, int N, int K, int S, int 
 
 // ---- the masked-UCB choice of the pair from the cluster tables (Sec. 3.4; Algorithm 1, "Select (I_t, S_t)") ----
 namespace {
-constexpr int SP_T = 128;
-__global__ void __launch_bounds__(SP_T)
+constexpr int SP_MAX_T = 1024;   // one CTA per instance; its width follows K*S (a thread should see few entries:
+                                 // each costs a dependent round trip to L2 for its table entries and its mask)
+__global__ void __launch_bounds__(SP_MAX_T)
 select_pair_kernel(int K, int S, int R, float c, const float* __restrict__ cl_pulls, const float* __restrict__ cl_mean,
                    const int32_t* __restrict__ t, const float* __restrict__ hsig, const int32_t* __restrict__ target,
                    float theta, float* __restrict__ cl_index, int32_t* __restrict__ pair, int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
-    __shared__ unsigned long long s_red[SP_T / 32];
-    const int b = blockIdx.x, tid = threadIdx.x, KS = K * S;
+    __shared__ unsigned long long s_red[SP_MAX_T / 32];
+    const int b = blockIdx.x, tid = threadIdx.x, KS = K * S, T = blockDim.x;
     const float lnt = logf((float)t[b]);
     unsigned long long best = 0ull;
-    for (int e = tid; e < KS; e += SP_T) {
+    for (int e = tid; e < KS; e += T) {
         const size_t o = (size_t)b * KS + e;
         const float u = cl_mean[o] + c * sqrtf(lnt / cl_pulls[o]);
         if (cl_index) cl_index[o] = u;
@@ -103,8 +104,7 @@ select_pair_kernel(int K, int S, int R, float c, const float* __restrict__ cl_pu
     if ((tid & 31) == 0) s_red[tid >> 5] = best;
     __syncthreads();
     if (tid == 0) {
-#pragma unroll
-        for (int w = 1; w < SP_T / 32; ++w) best = s_red[w] > best ? s_red[w] : best;
+        for (int w = 1; w < T / 32; ++w) best = s_red[w] > best ? s_red[w] : best;
         pair[b] = best ? (int32_t)(0xffffffffu - (unsigned)(best & 0xffffffffull)) : -1;
     }
 }
@@ -114,7 +114,10 @@ kb_status kb_launch_select_pair(kb_ctx* ctx, int B, int K, int S, int R, float c
                                 const float* cl_mean, const int32_t* t, const float* hsig, const int32_t* target,
                                 float theta_sat, float* cl_index, int32_t* pair) {
     if (B == 0) return KB_OK;
-    kb_launch(select_pair_kernel, B, SP_T, 0, ctx->stream, K, S, R, c, cl_pulls, cl_mean, t, hsig, target, theta_sat, cl_index,
+    long ks = (long)K * S;
+    int threads = (int)(ks >= SP_MAX_T ? SP_MAX_T : ((ks + 31) / 32) * 32);
+    if (threads < 32) threads = 32;
+    kb_launch(select_pair_kernel, B, threads, 0, ctx->stream, K, S, R, c, cl_pulls, cl_mean, t, hsig, target, theta_sat, cl_index,
               pair, ctx->dev_status);
     KB_LAUNCH_CHECK(ctx, "select_pair_kernel");
     return KB_OK;
