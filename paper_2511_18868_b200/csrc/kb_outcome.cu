@@ -8,6 +8,10 @@
 // reward_sum[k_t][S_t] += r_t: one thread per instance, three words touched.  The kernel exists so
 // that selection, draw and update of B lock-step searches stay on the device, in one stream or one
 // CUDA graph, with no host round trip between them.
+//
+// Given the K x S cluster tables (cl_pulls, cl_mean) the same thread also applies Algorithm 1's own two lines
+// to the chosen pair, so the tables stay current and the next pair can be chosen by kb_select_pair (below) from
+// K*S entries, without a pass over the arms.
 #include "kb_internal.cuh"
 
 namespace {
