@@ -1052,7 +1052,8 @@ def test_cluster_radius(kbx, B, N, K):
     assert kbx.device_status() == 0
 
 
-def test_online_loop_regret_against_theorem1(kbx):
+@pytest.mark.parametrize("on_tables", [False, True])
+def test_online_loop_regret_against_theorem1(kbx, on_tables):
     """An empirical look at Theorem 1 with everything on the device: B lock-step searches over a fixed frontier
     whose mean reward is Lipschitz in the (2-D) features, T iterations of select -> draw -> record.  The average
     regret must fall over the run and end below C sqrt(K |S| ln T / T) + L max_i diam(C_i), with the diameter
@@ -1082,13 +1083,23 @@ def test_online_loop_regret_against_theorem1(kbx):
     ar = torch.arange(B, device="cuda")
     regret = torch.zeros((T, B), device="cuda")
     mu_star = d["mu"].amax(dim=(1, 2))
-    for it in range(T):
+    if on_tables:                                                             # the K x S tables once, then kept current
         kbx.score_select(d["labels"], d["dist2"], d["pulls"], d["reward_sum"], d["t"], cl[0], cl[1], cl[2], best_arm,
                          best_val, pair, c=2.0, lipschitz_L=0.0)
+    for it in range(T):
+        if on_tables:
+            kbx.select_pair(cl[0], cl[1], d["t"], pair, c=2.0)
+        else:
+            kbx.score_select(d["labels"], d["dist2"], d["pulls"], d["reward_sum"], d["t"], cl[0], cl[1], cl[2], best_arm,
+                             best_val, pair, c=2.0, lipschitz_L=0.0)
         kbx.sample_member(d["labels"], pair, d["h_cand"], d["target"], d["t"], member, K, 75.0, 31337)
         got_mu = d["mu"][ar, member.long(), (pair % S).long()]                # environment: deterministic reward
         t_new.copy_(1.0 - got_mu)                                             # L(k) = 1, L(k') = 1 - mu
-        kbx.record_outcome(member, pair, d["t_cur"], t_new, d["pulls"], d["reward_sum"], d["t"])
+        if on_tables:
+            kbx.record_outcome(member, pair, d["t_cur"], t_new, d["pulls"], d["reward_sum"], d["t"], cl_pulls=cl[0],
+                               cl_mean=cl[1])
+        else:
+            kbx.record_outcome(member, pair, d["t_cur"], t_new, d["pulls"], d["reward_sum"], d["t"])
         regret[it] = mu_star - got_mu
     radius = empty((B, K))
     kbx.cluster_radius(d["labels"], d["dist2"], radius)
