@@ -717,3 +717,22 @@ def test_update_pair_is_algorithm1_and_matches_the_aggregate():
     sc = oracle.score_select(labels, np.zeros((B, N), np.float32), pulls, rs, t, K=K)
     np.testing.assert_array_equal(n, sc["cl_pulls"])
     np.testing.assert_allclose(mu, sc["cl_mean"], atol=2e-6)
+
+
+# ------------------------------------------------------------- input recipe
+def test_candidate_signatures_recipe():
+    """Seeded, clipped to the percent range, centred on the cluster's signature (input data only)."""
+    rng = np.random.default_rng(0)
+    hsig = rng.uniform(0, 100, (2, 5, wl.R_RESOURCES)).astype(np.float32)
+    labels = rng.integers(0, 5, (2, 4000)).astype(np.int32)
+    h1 = wl.make_candidate_signatures(hsig, labels, seed=3)
+    h2 = wl.make_candidate_signatures(hsig, labels, seed=3)
+    h3 = wl.make_candidate_signatures(hsig, labels, seed=4)
+    assert h1.dtype == np.float32 and h1.shape == (2, 4000, wl.R_RESOURCES)
+    np.testing.assert_array_equal(h1, h2)
+    assert np.any(h1 != h3)
+    assert h1.min() >= 0.0 and h1.max() <= 100.0
+    base = hsig[np.arange(2)[:, None], labels]
+    inner = (base > 15) & (base < 85)                       # away from the clip
+    assert abs(float((h1 - base)[inner].mean())) < 0.1 and 2.7 < float((h1 - base)[inner].std()) < 3.3
+    assert wl.make_candidate_signatures(hsig, np.zeros((2, 0), np.int32), seed=1).shape == (2, 0, wl.R_RESOURCES)
