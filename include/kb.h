@@ -13,6 +13,15 @@
  *   kb_score_select     cluster statistics, masked-UCB index with a
  *                       Lipschitz term, arm selection    (Sec. 3.4, Assumption 2)
  *
+ * and, around the step, the other lines of Algorithm 1 that run on the device:
+ *
+ *   kb_seed_kmeanspp    k-means++ rows to start the clustering from (Sec. 3.5)
+ *   kb_select_pair      masked-UCB choice of (I_t, S_t) from the K x S tables
+ *   kb_sample_member    softmax draw of k_t inside the chosen cluster (Sec. 3.4)
+ *   kb_record_outcome   reward clip, N <- N + 1, running mean      (Sec. 2.2, Algorithm 1)
+ *   kb_cluster_radius   per-cluster radius, bounds diam(C_i)       (Theorem 1)
+ *   kb_select_top_m     the M best arms instead of one
+ *
  * Conventions (all entry points unless stated otherwise)
  *  - Arrays are dense, row-major, batch-major: X[B][N][D], C[B][K][D],
  *    labels[B][N], pulls[B][N][S], hsig[B][K][R].  B instances, N candidates,
