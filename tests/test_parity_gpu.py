@@ -1236,3 +1236,47 @@ def test_table_loop_matches_the_per_arm_bookkeeping(kbx):
     np.testing.assert_array_equal(host(cl_pulls), host(f_pulls))
     parity.close(host(cl_mean), host(f_mean), atol=2e-6, what="tables against the full pass")
     assert int(host(d["pulls"]).sum() - inp["pulls"].sum()) == int((np.stack([host(x[2]) for x in trace]) >= 0).sum())
+
+
+# ------------------------------------------------- the whole step as a CUDA graph
+@pytest.mark.parametrize("name", ["tiny", "medium", "large/32", "batched/64"])
+def test_step_replays_as_a_cuda_graph(kbx, name):
+    """kb_bandit_step allocates nothing and never synchronises with the host, so a caller can capture it once and
+    replay it (the fused one-CTA path, the cooperative launch, the tensor path with its memset nodes alike).  The
+    replay must leave what an eager call leaves: the oracle's checks hold on its outputs, and they equal the eager
+    outputs wherever the path is deterministic (integer outputs outside near-ties)."""
+    from paper_2511_18868_b200 import kb
+    cfg = STEP_CASES[name]
+    inp = wl.make_inputs(cfg)
+    dims = dict(B=cfg.B, N=cfg.N, D=cfg.D, K=cfg.K, S=cfg.S, R=wl.R_RESOURCES, iters=cfg.iters)
+    params = dict(theta_sat=float(inp["theta_sat"]), c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
+                  prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]))
+    eager = run_step(kbx, cfg, inp)
+    t = kb.step_tensors(inp, kbx.device)
+    x0 = t["x"].clone()
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(main)
+    kbx.set_stream(side)
+    try:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+            kbx.bandit_step(dims, params, t)
+    finally:
+        kbx.set_stream(main)
+    main.wait_stream(side)
+    for k in ("labels", "best_arm", "z", "arm_index"):
+        t[k].zero_()                                   # whatever the capture may have left: the replay must write it
+    t["x"].copy_(x0)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert kbx.device_status() == 0
+    got = {k: host(v) for k, v in t.items()}
+    parity.close(got["z"], eager["z"], atol=0, rtol=0, what="z (replay against eager)")
+    chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
+    parity.labels_match(got["z"], got["centroids"], got["labels"], chk)
+    assert float(np.mean(got["labels"] == eager["labels"])) > 0.999
+    s_chk = oracle.score_select(got["labels"], got["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], cfg.K,
+                                keep=got["keep"].view(np.uint32), c=2.0, lipschitz_L=float(inp["lipschitz_L"]))
+    parity.close(got["arm_index"], s_chk["arm_index"], atol=1e-6, what="arm_index")
+    parity.select_match(got["best_arm"], got["best_val"], s_chk, s_chk["arm_index"])
