@@ -71,8 +71,10 @@ kb_status kb_destroy(kb_ctx* ctx);
 /* Rebinds the context to another stream (borrowed). */
 kb_status kb_set_stream(kb_ctx* ctx, void* cuda_stream);
 
-/* Bytes of scratch the five calls and kb_cluster_fit need for these sizes
- * (host pointer `out`).  kb_bandit_step* need kb_step_workspace_bytes. */
+/* Bytes of scratch the five calls, kb_cluster_fit, kb_bandit_step and the
+ * calls around the step (kb_seed_kmeanspp, kb_sample_member, kb_select_top_m
+ * up to KB_TOP_M_MAX) need for these sizes (host pointer `out`).
+ * kb_bandit_step_host needs kb_step_workspace_bytes. */
 kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out);
 /* Registers a device buffer (borrowed, 256-byte aligned) as scratch.  Its
  * contents need not be initialised and are not preserved between calls. */
