@@ -263,6 +263,15 @@ def update_pair(pair, reward, cl_pulls, cl_mean):
     return cl_pulls, cl_mean
 
 
+def best_restart(inertia):
+    """inertia [G][n_init] -> best [G]: the restart with the smallest inertia (see kbo_best_restart)."""
+    x = _f32(inertia)
+    G, n_init = x.shape
+    best = np.empty((G,), np.int32)
+    _check(_load().kbo_best_restart(G, n_init, _p(x), _p(best)), "best_restart")
+    return best
+
+
 def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = True) -> Dict[str, np.ndarray]:
     """One whole bandit step in the order the library runs it: normalise, seed
     the centroids from data rows, `iters` x (assign, update), a final assign,

@@ -625,4 +625,24 @@ int kbo_update_pair(int B, int K, int S, const int32_t* pair, const float* rewar
     return 0;
 }
 
+// ---------------------------------------------------------------------------
+// Restarts (the n_init of the "scikit-learn's KMeans" of Sec. 3.5): a search instance is clustered n_init
+// times from different seeds, as n_init consecutive instances of the batch; the run with the smallest
+// inertia is kept.  best[g] = the index in [0, n_init) of the smallest inertia[g][.], lowest index on ties;
+// NaN inertias are never chosen (-1 if all are NaN).
+// ---------------------------------------------------------------------------
+int kbo_best_restart(int G, int n_init, const float* inertia, int32_t* best) {
+    for (int g = 0; g < G; ++g) {
+        int arg = -1;
+        double v = kInf;
+        for (int r = 0; r < n_init; ++r) {
+            const double x = (double)inertia[(size_t)g * n_init + r];
+            if (std::isnan(x)) continue;
+            if (arg < 0 || x < v) { v = x; arg = r; }
+        }
+        best[g] = arg;
+    }
+    return 0;
+}
+
 }  // extern "C"

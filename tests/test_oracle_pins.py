@@ -736,3 +736,30 @@ def test_candidate_signatures_recipe():
     inner = (base > 15) & (base < 85)                       # away from the clip
     assert abs(float((h1 - base)[inner].mean())) < 0.1 and 2.7 < float((h1 - base)[inner].std()) < 3.3
     assert wl.make_candidate_signatures(hsig, np.zeros((2, 0), np.int32), seed=1).shape == (2, 0, wl.R_RESOURCES)
+
+
+# ------------------------------------------------------------------ restarts
+def test_best_restart_is_numpy_argmin():
+    rng = np.random.default_rng(6)
+    x = rng.integers(0, 6, (50, 7)).astype(np.float32)            # many ties: numpy's argmin also takes the first
+    np.testing.assert_array_equal(oracle.best_restart(x), np.argmin(x, axis=1))
+    x[0, :] = np.nan
+    x[1, 0] = np.nan
+    x[2, 3] = np.inf
+    b = oracle.best_restart(x)
+    assert b[0] == -1 and b[1] == 1 + int(np.argmin(x[1, 1:])) and b[2] == int(np.nanargmin(x[2]))
+    assert oracle.best_restart(np.array([[3.0]], np.float32))[0] == 0
+    # restarts help: the best of several seedings is never worse than the first
+    K, per, B, n_init = 5, 30, 6, 4
+    cen = rng.standard_normal((K, 3)) * 4
+    z = (cen[None, :, None, :] + rng.standard_normal((B, K, per, 3))).reshape(B, K * per, 3).astype(np.float32)
+    zz = np.repeat(z, n_init, axis=0)                             # n_init consecutive copies of every instance
+    rows = oracle.kmeanspp(zz, K, seed=1)                         # the instance index is in the counter: seeds differ
+    c = oracle.init_centroids(zz, rows)
+    for _ in range(5):
+        a = oracle.cluster_assign(zz, c, want_rep=False)
+        c, _ = oracle.cluster_update(zz, a["labels"], c)
+    inertia = oracle.cluster_assign(zz, c, want_rep=False)["inertia"].reshape(B, n_init)
+    best = oracle.best_restart(inertia)
+    assert np.all(inertia[np.arange(B), best] <= inertia[:, 0])
+    assert len({tuple(r) for r in rows.reshape(B, n_init, K)[0].tolist()}) > 1
