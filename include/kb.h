@@ -16,6 +16,7 @@
  * and, around the step, the other lines of Algorithm 1 that run on the device:
  *
  *   kb_seed_kmeanspp    k-means++ rows to start the clustering from (Sec. 3.5)
+ *   kb_best_restart     the run with the smallest inertia among n_init
  *   kb_select_pair      masked-UCB choice of (I_t, S_t) from the K x S tables
  *   kb_sample_member    softmax draw of k_t inside the chosen cluster (Sec. 3.4)
  *   kb_record_outcome   reward clip, N <- N + 1, running mean      (Sec. 2.2, Algorithm 1)
@@ -251,6 +252,17 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
  * fp32 distances in the direct form. */
 kb_status kb_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const float* z, uint64_t seed,
                            int32_t* rows);
+
+/* Restarts (the n_init of the "scikit-learn's KMeans" of Sec. 3.5): a search
+ * instance is clustered n_init times from different seeds as n_init
+ * CONSECUTIVE instances of the batch (kb_seed_kmeanspp draws differently for
+ * each: the instance index is part of its counter), and the run with the
+ * smallest inertia is kept:
+ *   best[g] = index in [0, n_init) of the smallest inertia[g*n_init + .],
+ *             lowest index on ties; NaN is never chosen (-1 if all are NaN).
+ *   inertia [G*n_init] in, as kb_cluster_fit writes it;  best [G] out
+ * DEVICE memory.  One launch, no workspace. */
+kb_status kb_best_restart(kb_ctx* ctx, int G, int n_init, const float* inertia, int32_t* best);
 
 /* The M best arms of every instance by the per-arm index (the masked argmax
  * of Sec. 3.4 taken M times, for generating M candidates per iteration):

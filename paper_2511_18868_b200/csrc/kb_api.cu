@@ -346,6 +346,14 @@ kb_status kb_sample_member(kb_ctx* ctx, int B, int N, int K, int S, int R, const
                                    member_val);
 }
 
+kb_status kb_best_restart(kb_ctx* ctx, int G, int n_init, const float* inertia, int32_t* best) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    KB_REQUIRE(ctx, G >= 0 && n_init >= 1, "kb_best_restart: G must be >= 0 and n_init >= 1");
+    if (G > 0) KB_REQUIRE(ctx, inertia && best, "kb_best_restart: inertia and best are required");
+    TimeScope ts__(ctx, KB_T_INIT);
+    return kb_launch_best_restart(ctx, G, n_init, inertia, best);
+}
+
 kb_status kb_select_top_m(kb_ctx* ctx, int B, int N, int S, int M, const float* arm_index, int32_t* top_arm,
                           float* top_val) {
     KB_COMMON(ctx, B, N);

@@ -151,6 +151,7 @@ kb_status kb_launch_select_pair(kb_ctx*, int B, int K, int S, int R, float c, co
 kb_status kb_launch_cluster_radius(kb_ctx*, int B, int N, int K, const int32_t* labels, const float* dist2, float* radius);
 size_t kb_ws_need_topm(int B, int M);
 kb_status kb_launch_top_m(kb_ctx*, int B, int NS, int M, const float* arm_index, int32_t* top_arm, float* top_val);
+kb_status kb_launch_best_restart(kb_ctx*, int G, int n_init, const float* inertia, int32_t* best);
 size_t kb_ws_need_seed(int B, int N, int K);
 kb_status kb_launch_seed_kmeanspp(kb_ctx*, int B, int N, int D, int K, const float* z, uint64_t seed, int32_t* rows);
 size_t kb_ws_need_sample(int B);

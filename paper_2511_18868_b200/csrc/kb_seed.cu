@@ -283,3 +283,27 @@ kb_status kb_launch_seed_kmeanspp(kb_ctx* ctx, int B, int N, int D, int K, const
     }
     return KB_OK;
 }
+
+// ---- restarts: the run with the smallest inertia among n_init consecutive instances --------------------
+namespace {
+__global__ void best_restart_kernel(int G, int n_init, const float* __restrict__ inertia, int32_t* __restrict__ best) {
+    kb_grid_dependency_wait();
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= G) return;
+    int arg = -1;
+    float v = INFINITY;
+    for (int r = 0; r < n_init; ++r) {
+        const float x = inertia[(size_t)g * n_init + r];
+        if (x != x) continue;                                    // NaN: never chosen
+        if (arg < 0 || x < v) { v = x; arg = r; }
+    }
+    best[g] = arg;
+}
+}  // namespace
+
+kb_status kb_launch_best_restart(kb_ctx* ctx, int G, int n_init, const float* inertia, int32_t* best) {
+    if (G == 0) return KB_OK;
+    kb_launch(best_restart_kernel, (G + 127) / 128, 128, 0, ctx->stream, G, n_init, inertia, best);
+    KB_LAUNCH_CHECK(ctx, "best_restart_kernel");
+    return KB_OK;
+}

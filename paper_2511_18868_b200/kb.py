@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
-           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m",
+           "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc"]
 
@@ -93,6 +93,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_select_pair.argtypes = [_VP, i, i, i, i, f] + [_VP] * 5 + [f, _VP, _VP]
     lib.kb_cluster_radius.argtypes = [_VP, i, i, i, _VP, _VP, _VP]
     lib.kb_select_top_m.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
+    lib.kb_best_restart.argtypes = [_VP, i, i, _VP, _VP]
     lib.kb_seed_kmeanspp.argtypes = [_VP, i, i, i, i, _VP, ctypes.c_uint64, _VP]
     lib.kb_set_assign_options.argtypes = [_VP, i, f]
     lib.kb_get_assign_path.argtypes = [_VP, ctypes.POINTER(i)]
@@ -258,6 +259,12 @@ class KB:
                                               self._p(h_cand), self._p(target), float(theta_sat),
                                               int(seed) & (2 ** 64 - 1), self._p(t), self._p(member),
                                               self._p(member_val)), "kb_sample_member")
+
+    def best_restart(self, inertia, best):
+        """inertia [G*n_init] (n_init consecutive instances per search) -> best [G]: the run with the smallest inertia."""
+        G = best.shape[0]
+        n_init = inertia.numel() // max(G, 1)
+        self._check(self.lib.kb_best_restart(self.h, G, n_init, self._p(inertia), self._p(best)), "kb_best_restart")
 
     def select_top_m(self, arm_index, top_arm, top_val=None):
         """The M best arms per instance by arm_index [B][N][S]: top_arm [B][M] (flat k*S+s), sorted."""

@@ -1280,3 +1280,35 @@ def test_step_replays_as_a_cuda_graph(kbx, name):
                                 keep=got["keep"].view(np.uint32), c=2.0, lipschitz_L=float(inp["lipschitz_L"]))
     parity.close(got["arm_index"], s_chk["arm_index"], atol=1e-6, what="arm_index")
     parity.select_match(got["best_arm"], got["best_val"], s_chk, s_chk["arm_index"])
+
+
+# ------------------------------------------------------------------ restarts
+def test_best_restart_and_the_restart_flow(kbx):
+    rng = np.random.default_rng(6)
+    x = rng.integers(0, 6, (300, 7)).astype(np.float32)
+    x[0, :] = np.nan
+    x[1, 0] = np.nan
+    x[2, 3] = np.inf
+    best = empty((300,), torch.int32)
+    kbx.best_restart(dev(x.reshape(-1)), best)
+    np.testing.assert_array_equal(host(best), oracle.best_restart(x))
+    # n_init consecutive copies of every instance: seed, gather, fit, pick -- all on the device
+    K, per, B, n_init = 5, 60, 40, 4
+    cen = rng.standard_normal((K, 16)) * 3
+    z = (cen[None, :, None, :] + rng.standard_normal((B, K, per, 16))).reshape(B, K * per, 16).astype(np.float32)
+    zz = np.repeat(z, n_init, axis=0)
+    BB, N = zz.shape[0], zz.shape[1]
+    ws(kbx, BB, N, 16, K, 4)
+    zd, rows, c = dev(zz), empty((BB, K), torch.int32), empty((BB, K, 16))
+    labels, inertia, pick = empty((BB, N), torch.int32), empty((BB,)), empty((B,), torch.int32)
+    kbx.seed_kmeanspp(zd, rows, seed=3)
+    kbx.init_centroids(zd, rows, c)
+    kbx.cluster_fit(zd, c, labels, 6, inertia=inertia)
+    kbx.best_restart(inertia, pick)
+    torch.cuda.synchronize()
+    got_i = host(inertia).reshape(B, n_init)
+    np.testing.assert_array_equal(host(pick), oracle.best_restart(got_i))
+    assert np.all(got_i[np.arange(B), host(pick)] <= got_i[:, 0])
+    r = host(rows).reshape(B, n_init, K)
+    assert np.mean([len({tuple(v) for v in r[b].tolist()}) > 1 for b in range(B)]) > 0.9   # the copies are seeded differently
+    assert kbx.device_status() == 0
