@@ -136,15 +136,14 @@ def score_select(labels, dist2, pulls, reward_sum, t, K, keep=None, bound=None, 
     best_arm = np.empty((B,), np.int32)
     best_val = np.empty((B,), np.float32)
     best_cl = np.empty((B,), np.int32)
-    margin = np.empty((B, 2), np.float64)
     _check(_load().kbo_score_select(B, N, K, S, ctypes.c_float(c), ctypes.c_float(lipschitz_L),
                                     ctypes.c_float(prior_pulls), ctypes.c_float(prior_mean),
                                     int(bool(cap_with_bound)), _p(labels), _p(dist2), _p(pulls), _p(reward_sum),
                                     _p(keep), _p(bound), _p(t), _p(cl_pulls), _p(cl_mean), _p(cl_index),
-                                    _p(arm_index), _p(best_arm), _p(best_val), _p(best_cl), _p(margin)),
+                                    _p(arm_index), _p(best_arm), _p(best_val), _p(best_cl)),
            "score_select")
     return {"cl_pulls": cl_pulls, "cl_mean": cl_mean, "cl_index": cl_index, "arm_index": arm_index,
-            "best_arm": best_arm, "best_val": best_val, "best_cluster_arm": best_cl, "margin": margin}
+            "best_arm": best_arm, "best_val": best_val, "best_cluster_arm": best_cl}
 
 
 def init_centroids(z, rows):
@@ -296,5 +295,5 @@ def bandit_step(inp: Dict[str, np.ndarray], iters: int, want_arm_index: bool = T
     out = {"z": z, "mean": mean, "scale": scale, "centroids": c, "counts": counts, "labels": a["labels"],
            "dist2": a["dist2"], "inertia": a["inertia"], "rep": a["rep"], "inertia_trace": np.array(inertia_trace),
            "keep": p["keep"], "kept_count": p["kept_count"], "bound": p["bound"]}
-    out.update({k: v for k, v in s.items() if k != "margin"})
+    out.update(s)
     return out

@@ -74,8 +74,13 @@ int kbo_normalize(int B, int N, int D, const float* x, float* z, float* mean, fl
 //      the gap between current performance and the limit, in reward units of
 //      the reward definition in Sec. 2.2)
 // keep[b][k] bit s = roofline keep AND saturation keep.
-// margin (optional, [B][N][S]): smallest relative distance of a deciding
-// comparison from its threshold, for near-tie accounting in the tests.
+// margin (optional, [B][N][S]): the relative distance from its threshold of the
+// comparison(s) that DECIDE the bit, for near-tie accounting in the tests:
+//   |T_lb - T_inc| / T_inc  and  |h - theta_sat| / theta_sat  per comparison;
+//   a kept arm passes both, and either one flipping prunes it: the smaller;
+//   an arm pruned by one comparison only: that comparison's;
+//   an arm pruned by both: both must flip to keep it: the larger.
+// (Without the saturation inputs only the roofline comparison exists.)
 // ---------------------------------------------------------------------------
 int kbo_prune(int B, int N, int S, int K, int R, const float* flops, const float* bytes,
               const float* peak_flops, const float* peak_bw, const float* t_incumbent,
@@ -92,17 +97,22 @@ int kbo_prune(int B, int N, int S, int K, int R, const float* flops, const float
                 double tf = (double)flops[ix2(b, k, N)] / (double)peak_flops[s];
                 double tq = (double)bytes[ix2(b, k, N)] / (double)peak_bw[s];
                 double tlb = tf > tq ? tf : tq;
-                bool ok = tlb < tinc;
-                double mg = std::fabs(tlb - tinc) / std::fabs(tinc);
+                const bool roof_ok = tlb < tinc;
+                const double m_roof = std::fabs(tlb - tinc) / std::fabs(tinc);
+                bool ok = roof_ok;
+                double mg = m_roof;
                 if (sat) {
                     int lab = labels[ix2(b, k, N)];
                     if (lab < 0 || lab >= K) return 2;
                     int r = target[s];
                     if (r < 0 || r >= R) return 3;
                     double h = (double)hsig[ix3(b, lab, r, K, R)];
-                    ok = ok && (h < (double)theta_sat);
-                    double mh = std::fabs(h - (double)theta_sat) / std::fabs((double)theta_sat);
-                    if (mh < mg) mg = mh;
+                    const bool sat_ok = h < (double)theta_sat;
+                    const double m_sat = std::fabs(h - (double)theta_sat) / std::fabs((double)theta_sat);
+                    ok = roof_ok && sat_ok;
+                    if (roof_ok && sat_ok) mg = m_sat < m_roof ? m_sat : m_roof;        // the first to flip prunes
+                    else if (!roof_ok && !sat_ok) mg = m_sat > m_roof ? m_sat : m_roof; // the last to flip keeps
+                    else mg = roof_ok ? m_sat : m_roof;                                 // the one failing comparison
                 }
                 if (ok) { bits |= (1u << s); ++kept; }
                 if (margin) margin[ix3(b, k, s, N, S)] = mg;
@@ -223,15 +233,13 @@ int kbo_cluster_update(int B, int N, int D, int K, const float* z, const int32_t
 //  pairs with at least one kept member arm (the paper's M_{i,s} when the mask
 //  is constant within a cluster), -1 if none.
 //  arm_index holds -inf for a pruned arm.
-//  sel_margin (optional, double [B][2]): (best - runner-up with a different
-//  value) / |best| at arm level and at cluster level; +inf if no runner-up.
 // ---------------------------------------------------------------------------
 int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, float prior_pulls,
                      float prior_mean, int cap_with_bound, const int32_t* labels, const float* dist2,
                      const int32_t* pulls, const float* reward_sum, const uint32_t* keep,
                      const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean,
                      float* cl_index, float* arm_index, int32_t* best_arm, float* best_val,
-                     int32_t* best_cluster_arm, double* sel_margin) {
+                     int32_t* best_cluster_arm) {
     if (S > 32) return 1;
     const size_t KS = (size_t)K * (size_t)S;
     std::vector<int64_t> np_(KS ? KS : 1);
@@ -250,7 +258,7 @@ int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, flo
             }
         }
         const double lnt = std::log((double)t[b]);
-        double cbest = -kInf, csecond = -kInf;
+        double cbest = -kInf;
         int carg = -1;
         for (int i = 0; i < K; ++i)
             for (int s = 0; s < S; ++s) {
@@ -262,13 +270,12 @@ int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, flo
                 cl_mean[ix3(b, i, s, K, S)] = (float)mu;
                 cl_index[ix3(b, i, s, K, S)] = (float)u;
                 if (anyk[ix2(i, s, S)]) {
-                    if (u > cbest) { csecond = cbest; cbest = u; carg = i * S + s; }
-                    else if (u < cbest && u > csecond) { csecond = u; }
+                    if (u > cbest) { cbest = u; carg = i * S + s; }
                 }
             }
         best_cluster_arm[b] = carg;
 
-        double abest = -kInf, asecond = -kInf;
+        double abest = -kInf;
         int64_t aarg = -1;
         for (int k = 0; k < N; ++k) {
             int lab = labels[ix2(b, k, N)];
@@ -284,16 +291,11 @@ int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, flo
                 bool ok = (bits >> s) & 1u;
                 if (arm_index) arm_index[ix3(b, k, s, N, S)] = ok ? (float)u : -std::numeric_limits<float>::infinity();
                 if (!ok) continue;
-                if (u > abest) { asecond = abest; abest = u; aarg = (int64_t)k * S + s; }
-                else if (u < abest && u > asecond) { asecond = u; }
+                if (u > abest) { abest = u; aarg = (int64_t)k * S + s; }
             }
         }
         best_arm[b] = (int32_t)aarg;
         best_val[b] = aarg >= 0 ? (float)abest : -std::numeric_limits<float>::infinity();
-        if (sel_margin) {
-            sel_margin[2 * b + 0] = (aarg >= 0 && asecond > -kInf) ? (abest - asecond) / std::fabs(abest) : kInf;
-            sel_margin[2 * b + 1] = (carg >= 0 && csecond > -kInf) ? (cbest - csecond) / std::fabs(cbest) : kInf;
-        }
     }
     return 0;
 }

@@ -95,6 +95,77 @@ def test_prune_invariants_and_saturation_mask():
     assert r["keep"][0, 0] == 0b010
 
 
+def test_prune_margin_worked_values():
+    """The near-tie margin that arbitrates every keep-bit disagreement in the GPU parity tests, by hand.
+    Roofline comparison alone, exactly representable inputs: T_lb = max(3/2, 1/4) = 1.5 against
+    T_inc = 1.5 (1 + 2^-18): margin = 2^-18 / (1 + 2^-18)."""
+    e = 2.0 ** -18
+    r = oracle.prune([[3.0]], [[1.0]], [2.0], [4.0], [1.5 * (1 + e)], want_margin=True)
+    assert r["keep"][0, 0] == 1 and r["margin"][0, 0, 0] == pytest.approx(e / (1 + e), rel=1e-12)
+    r = oracle.prune([[3.0]], [[1.0]], [2.0], [4.0], [1.5 * (1 - e)], want_margin=True)          # pruned side
+    assert r["keep"][0, 0] == 0 and r["margin"][0, 0, 0] == pytest.approx(e / (1 - e), rel=1e-12)
+    # the golden floor 5e-5 s against an incumbent 3e-6 above it (fp32 rounding of both: 1.2e-7)
+    F, Q, P, W, tlb = read_golden("roofline_floor.txt")[0]
+    r = oracle.prune([[F]], [[Q]], [P], [W], [tlb * (1 + 3e-6)], want_margin=True)
+    assert r["keep"][0, 0] == 1 and r["margin"][0, 0, 0] == pytest.approx(3e-6, abs=2e-7)
+    # saturation comparison: 74.9997 % against theta = 75 %: 0.0003 / 75 = 4e-6 (fp32 rounding of h: 5e-8)
+    hs = np.array([[[74.9997, 90.0, 60.0]]], np.float32)
+    wide = dict(flops=[[1.0]], bytes_=[[1.0]], peak_flops=[1.0] * 3, peak_bw=[1.0] * 3)
+    # roofline decisively kept (floor 1 against incumbent 2: margin 0.5): the saturation comparison decides alone
+    r = oracle.prune(t_inc=[2.0], labels=[[0]], hsig=hs, target=[0, 1, 2], theta_sat=75.0, want_margin=True, **wide)
+    assert r["keep"][0, 0] == 0b101
+    np.testing.assert_allclose(r["margin"][0, 0], [4e-6, 0.2, 0.2], atol=1e-7)     # kept: min(0.5, .); pruned by h: 0.2
+    # both comparisons pass, the roofline one nearer its threshold: the smaller margin decides
+    r = oracle.prune(t_inc=[1.0 + 2.0 ** -19], labels=[[0]], hsig=hs, target=[2, 2, 2], want_margin=True, **wide)
+    assert r["keep"][0, 0] == 0b111 and r["margin"][0, 0, 0] == pytest.approx(2.0 ** -19, rel=1e-5)
+    # pruned by the roofline comparison alone, by a hair, while h is far below theta: the hair decides
+    r = oracle.prune(t_inc=[1.0 - 2.0 ** -19], labels=[[0]], hsig=hs, target=[2, 2, 2], want_margin=True, **wide)
+    assert r["keep"][0, 0] == 0 and r["margin"][0, 0, 0] == pytest.approx(2.0 ** -19, rel=1e-5)
+    # pruned by BOTH, one by a hair and one decisively (h = 90): no small change keeps it: the larger margin
+    r = oracle.prune(t_inc=[1.0 - 2.0 ** -19], labels=[[0]], hsig=hs, target=[1, 1, 1], want_margin=True, **wide)
+    assert r["keep"][0, 0] == 0 and r["margin"][0, 0, 0] == pytest.approx(0.2, rel=1e-6)
+
+
+def test_prune_margin_says_exactly_which_bits_a_small_change_can_flip():
+    """What the margin is for: a bit whose margin exceeds delta must survive every change of the two
+    thresholds by less than delta (relative); a bit whose margin is below delta must flip under one.  Inputs are
+    built so that thousands of comparisons sit within 1e-7 .. 1e-3 of their thresholds, on both sides."""
+    rng = np.random.default_rng(11)
+    B, N, S, K = 2, 3000, 6, 4
+    delta = 1e-5
+    t_inc = np.array([3e-4, 7e-3], np.float32)
+    eps = np.exp(rng.uniform(np.log(1e-7), np.log(1e-3), (B, N))) * rng.choice([-1.0, 1.0], (B, N))
+    pf, pb = np.full(S, 1e12, np.float32), np.full(S, 1e11, np.float32)
+    pf[1::2] *= 4.0                                              # odd strategies: a floor 4x lower (decisively kept)
+    flops = (t_inc[:, None].astype(np.float64) * (1 + eps) * 1e12).astype(np.float32)
+    byts = np.ones((B, N), np.float32)
+    far = rng.uniform(size=(B, N)) < 0.3                         # a third of the candidates far above the incumbent
+    flops[far] *= 50.0
+    labels = rng.integers(0, K, (B, N)).astype(np.int32)
+    theta = 75.0
+    hs = (theta * (1 + np.exp(rng.uniform(np.log(1e-7), np.log(1e-1), (B, K, 3))) * rng.choice([-1.0, 1.0], (B, K, 3))))
+    hs = hs.astype(np.float32)
+    target = (np.arange(S) % 3).astype(np.int32)
+
+    def run(ti, th):
+        return oracle.prune(flops, byts, pf, pb, ti, None, labels, hs, target, th, want_margin=True)
+
+    nom = run(t_inc, theta)
+    bits = lambda r: ((r["keep"][..., None] >> np.arange(S, dtype=np.uint32)) & 1).astype(bool)
+    lo = bits(run((t_inc.astype(np.float64) * (1 - delta)).astype(np.float32), theta * (1 - delta)))
+    hi = bits(run((t_inc.astype(np.float64) * (1 + delta)).astype(np.float32), theta * (1 + delta)))
+    b0, m = bits(nom), nom["margin"]
+    flipped = (lo != b0) | (hi != b0)
+    safe, frail = m > 1.05 * delta, m < 0.95 * delta
+    assert safe.sum() > 10000 and frail.sum() > 500
+    assert not np.any(flipped & safe)
+    assert np.all(flipped[frail])
+    # without the saturation inputs the margin is the roofline comparison's alone
+    r = oracle.prune(flops, byts, pf, pb, t_inc, want_margin=True)
+    floor = np.maximum(flops.astype(np.float64)[..., None] / pf, byts.astype(np.float64)[..., None] / pb)
+    np.testing.assert_allclose(r["margin"], np.abs(floor / t_inc.astype(np.float64)[:, None, None] - 1), rtol=1e-9, atol=1e-15)
+
+
 # -------------------------------------------------------------------- assign
 def test_assign_against_cdist_and_optimality():
     rng = np.random.default_rng(4)
@@ -369,6 +440,36 @@ def test_select_brute_force_on_tiny_inputs():
                     best, arg = u, k * S + s
         assert out["best_arm"][0] == arg
         assert out["best_val"][0] == pytest.approx(best, rel=1e-6)
+
+
+# ------------------------------------------------------- initial centroids
+def test_init_centroids_is_a_row_gather():
+    """C[b][i] = Z[b][rows[b][i]], written out with numpy indexing: several instances (so that the batch
+    strides count), rows unsorted and repeated, first and last row, K > N."""
+    rng = np.random.default_rng(21)
+    B, N, D, K = 3, 37, 5, 41
+    z = rng.standard_normal((B, N, D)).astype(np.float32)
+    rows = rng.integers(0, N, (B, K)).astype(np.int32)          # unsorted, with repeats (K > N forces them)
+    rows[0, :4] = [N - 1, 0, N - 1, 17]
+    rows[2, -1] = 0
+    c = oracle.init_centroids(z, rows)
+    assert c.shape == (B, K, D)
+    for b in range(B):
+        for i in range(K):
+            assert np.array_equal(c[b, i], z[b, rows[b, i]]), (b, i)
+    # every value is distinct, so a wrong stride or a swapped (b, i) cannot pass by accident
+    z2 = np.arange(B * N * D, dtype=np.float32).reshape(B, N, D)
+    c2 = oracle.init_centroids(z2, rows)
+    want = (np.arange(B)[:, None, None] * N + rows[:, :, None]) * D + np.arange(D)[None, None, :]
+    assert np.array_equal(c2, want.astype(np.float32))
+    # a row id outside [0, N) is rejected
+    bad = rows.copy()
+    bad[1, 3] = N
+    with pytest.raises(ValueError):
+        oracle.init_centroids(z, bad)
+    bad[1, 3] = -1
+    with pytest.raises(ValueError):
+        oracle.init_centroids(z, bad)
 
 
 # ------------------------------------------------------------ input recipes
