@@ -1,8 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the batched bandit step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--only] [--impl reference]
 
+The line's workload is `contraction`, the largest single-GPU configuration, unless --workload names
+another; the other four workloads are timed after it on the same GPU and reported, with their per-call
+roofline fractions, under `workloads` (skipped with --only).
 A step is one pass of the whole hot path (normalise, seed centroids, iters x
 (assign, update), final assign, prune, score/select) over one synthetic batch.
 `value` is arms scored per second with all inputs resident in HBM; `e2e` is the
@@ -34,16 +37,17 @@ from paper_2511_18868_b200 import workloads as wl  # noqa: E402
 
 METRIC = "arms scored/sec per bandit step"
 UNIT = "arms/s"
-DEFAULT_WORKLOAD = "large"
+DEFAULT_WORKLOAD = "contraction"      # the largest single-GPU configuration
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant call's main kernel, per launch, from the
-# ncu captures summarised under profiles/ (bytes; None where no capture exists for that workload)
-TRAFFIC_FROM_NCU = {
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant call's main kernel, per launch, as CAPTURED by ncu on
+# an earlier build of that kernel (bytes; the summary under profiles/ names the command).  Printed as
+# roofline.traffic with its source; not measured in the run.
+TRAFFIC_FROM_CAPTURE = {
     # assign_tc_kernel (pre-split image of Z), one launch: 69.35 MB read + 1.11 MB written
-    # (profiles/assign_tc_and_update_kernels.txt)
-    ("large", "assign"): 70.46e6,
+    ("large", "assign"): {"bytes": 70.46e6, "source": "profiles/assign_tc_and_update_kernels.txt"},
     # assign_tc_kernel at N = 262144: 134.85 + 4.03 MB; traffic grows with N, scaled x16 to N = 4194304
-    ("contraction", "assign"): 16 * 138.88e6,
+    ("contraction", "assign"): {"bytes": 16 * 138.88e6,
+                                "source": "profiles/assign_tc_and_update_kernels.txt (N = 262144 capture, scaled x16 by rows)"},
 }
 
 # rows of the workload the CPU oracle is timed on (per instance), and instances
@@ -272,6 +276,185 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ GPU arm
+DTYPE = ("f32 (the assign contraction of large/contraction: fp16 hi/lo split x3 products on tcgen05 kind::f16 with "
+         "fp32 accumulation, near-ties settled exactly in the fp32 direct form)")
+
+
+def median_stats(ms_list):
+    a = np.asarray(ms_list, dtype=np.float64)
+    return {"median": float(np.median(a)), "min": float(a.min()), "max": float(a.max()), "mean": float(a.mean()),
+            "steps": int(a.size), "seconds": float(a.sum() * 1e-3)}
+
+
+def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms):
+    """Per-call table of one workload from the library's event pairs: average duration, achieved GB/s and
+    TFLOP/s on the call's ALGORITHMIC bytes / flops, and its fraction of the roofline that binds it."""
+    alg = algorithmic(cfg)
+    hbm = peaks["hbm_gbs"]
+    ffma_peak = probe["ffma_tflops"]
+    # three tensor-core products per fp32-equivalent product; kind::f16 runs at the measured 16-bit GEMM rate,
+    # kind::tf32 at half of it (nominal ratio)
+    tensor_peak = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5) / 3.0
+    mma_issue_peak = (probe["mma_f16_tflops"] if assign_path == 2 else probe["mma_tf32_tflops"]) / 3.0
+    out = {}
+    for name in ["normalize", "prep", "assign", "update", "fit", "prune", "score"]:
+        ms, calls = per_class.get(name, (0.0, 0))
+        if calls == 0:
+            continue
+        avg_s = ms / calls * 1e-3
+        row = {"calls": int(calls), "avg_us": avg_s * 1e6, "share": ms / max(breakdown_ms, 1e-9)}
+        if name in alg:
+            gbs = alg[name]["bytes"] / avg_s / 1e9
+            tfl = alg[name]["flops"] / avg_s / 1e12
+            row.update(GBps=gbs, hbm_frac=gbs / hbm, TFLOPs=tfl)
+            hbm_time = alg[name]["bytes"] / (hbm * 1e9)
+            if name == "assign" and assign_path in (2, 3):
+                row.update(bound="tensor", frac=tfl / tensor_peak, frac_of_mma_issue_peak=tfl / mma_issue_peak)
+            elif name in ("assign", "fit") and alg[name]["flops"] / (ffma_peak * 1e12) > hbm_time:
+                row.update(bound="alu", frac=tfl / ffma_peak)
+            else:
+                row.update(bound="hbm", frac=gbs / hbm)
+        out[name] = row
+    kms, kcalls = per_class.get("assign_kernel", (0.0, 0))
+    if kcalls and assign_path in (2, 3):
+        k_s = kms / kcalls * 1e-3
+        tfl = alg["assign"]["flops"] / k_s / 1e12
+        out["assign_kernel"] = {"calls": int(kcalls), "avg_us": k_s * 1e6, "share": kms / max(breakdown_ms, 1e-9),
+                                "TFLOPs": tfl, "bound": "tensor", "frac": tfl / tensor_peak,
+                                "frac_of_mma_issue_peak": tfl / mma_issue_peak}
+    return out, {"tensor_fp32_equiv_tflops": tensor_peak, "mma_issue_fp32_equiv_tflops": mma_issue_peak,
+                 "ffma_tflops": ffma_peak, "hbm_gbs": hbm}
+
+
+def measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, steps, warmup, min_seconds, flush, barrier,
+                     reduce_first=lambda v: v):
+    """Device-resident timing of one workload: `warmup` untimed steps, then loops of exactly `steps` steps, each
+    step between its own pair of CUDA events with an L2 flush before it, repeated until `min_seconds` of timed
+    steps have run (the warm-up-then-at-least-a-second, report-the-median protocol); then one more pass of
+    `steps` steps with the library's per-call event pairs ON for the breakdown (those events sit in the stream
+    between the kernels, so that pass is not the one `ms_per_step` comes from)."""
+    R = wl.R_RESOURCES
+    dims = dict(B=cfg.B, N=cfg.N, D=cfg.D, K=cfg.K, S=cfg.S, R=R, iters=cfg.iters)
+    params = dict(theta_sat=float(inp["theta_sat"]), c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
+                  prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]))
+    ctx.ensure_workspace(max(ctx.workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S),
+                             ctx.step_workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S, R)))
+    dev_t = kb.step_tensors(inp, device)
+    for _ in range(warmup):
+        flush.zero_()
+        ctx.bandit_step(dims, params, dev_t)
+    barrier()
+    k0, m0 = ctx.launch_count()
+    per_step = []
+
+    def timed_loop():
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.zero_()
+            a.record()
+            ctx.bandit_step(dims, params, dev_t)
+            b.record()
+        barrier()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    per_step += timed_loop()
+    # how many more loops make up `min_seconds`: decided once, from the slowest rank's first loop, so that every
+    # rank runs the same number of loops (and of barriers)
+    first = reduce_first([sum(per_step) * 1e-3])[0]
+    more = int(min(200, max(0, np.ceil(min_seconds / max(first, 1e-9)) - 1)))
+    for _ in range(more):
+        per_step += timed_loop()
+    k1, m1 = ctx.launch_count()
+    ctx.timing_enable(True)
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev2:
+        flush.zero_()
+        a.record()
+        ctx.bandit_step(dims, params, dev_t)
+        b.record()
+    barrier()
+    breakdown_ms = sum(a.elapsed_time(b) for a, b in ev2)
+    per_class = ctx.timing_read()
+    ctx.timing_enable(False)
+    status = ctx.device_status()
+    assign_path, presplit = ctx.assign_path(), ctx.assign_presplit()
+    calls, denominators = call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms)
+    # the library's own count of near-ties of the final assignment on the tensor path: rows whose runner-up lay within
+    # the re-evaluation bound and were settled exactly (two-candidate compare, full re-evaluation)
+    near = None
+    if assign_path in (2, 3):
+        flagged = torch.zeros((2,), dtype=torch.int32, device=device)
+        scratch_labels = torch.empty_like(dev_t["labels"])
+        ctx.assign_tc_probe(dev_t["z"], dev_t["centroids"], scratch_labels, None, flagged)
+        f = flagged.cpu().numpy()
+        near = {"rows": int(cfg.B * cfg.N), "settled_against_runner_up": int(f[0]), "settled_against_all_K": int(f[1]),
+                "labels_equal_to_the_step's": bool(torch.equal(scratch_labels, dev_t["labels"]))}
+    st = median_stats(per_step)
+    return {"dims": dims, "params": params, "dev_t": dev_t, "stats": st, "launches": int(k1 - k0), "memsets": int(m1 - m0),
+            "calls": calls, "denominators": denominators, "status": int(status), "assign_path": int(assign_path),
+            "presplit": int(presplit), "breakdown_ms_per_step": breakdown_ms / steps, "near": near}
+
+
+def workload_summary(cfg, m, world):
+    """What the line carries for a workload beside the headline one."""
+    st = m["stats"]
+    keep = ("avg_us", "calls", "share", "bound", "frac", "frac_of_mma_issue_peak", "GBps", "TFLOPs")
+    return {"config": {k: v for k, v in workload_config(cfg).items() if k in ("B", "N", "D", "K", "S", "iters", "arms")},
+            "ms_per_step": st["median"], "ms_min": st["min"], "ms_max": st["max"], "timed_steps": st["steps"],
+            "timed_seconds": st["seconds"], "arms_per_s": job_value(world, cfg.arms, st["median"]),
+            "gpu_launches_per_step": m["launches"] / st["steps"], "assign_path": m["assign_path"],
+            "calls": {n: {k: v for k, v in row.items() if k in keep} for n, row in m["calls"].items()},
+            "near_ties_tensor_assign": m["near"], "device_status": m["status"]}
+
+
+def dominant_roofline(cfg, m, peaks):
+    """The `roofline` object of the line: the dominant KERNEL of the workload's step, with the per-call fractions
+    of assign, update and score (the three the target names) beside it."""
+    calls = m["calls"]
+    alg = algorithmic(cfg)
+    den = m["denominators"]
+    timed = {n: r for n, r in calls.items() if n != "assign_kernel"}
+    dominant = max(timed, key=lambda n: timed[n]["share"])
+    dk = calls[dominant]
+    if dominant == "assign" and "assign_kernel" in calls:
+        ak = calls["assign_kernel"]
+        split = "fp16 hi/lo split, kind::f16" if m["assign_path"] == 2 else "3xTF32, kind::tf32"
+        roof = {"bound": "tensor", "achieved": ak["TFLOPs"], "peak": den["tensor_fp32_equiv_tflops"], "unit": "TFLOP/s",
+                "frac": ak["frac"], "traffic": None,
+                "kernel": f"assign_tc_kernel (tcgen05 {split}), the contraction kernel of kb_cluster_assign",
+                "kernel_avg_us": ak["avg_us"], "kernel_launches": ak["calls"],
+                "frac_of_mma_issue_peak": ak["frac_of_mma_issue_peak"],
+                "whole_call": {"avg_us": dk["avg_us"], "TFLOPs": dk["TFLOPs"], "frac": dk["frac"],
+                               "what": "preparation + contraction + fix-up kernels of one kb_cluster_assign; the "
+                                       "once-per-fit conversion of Z to its fp16 image is its own class (prep)"},
+                "peak_source": f"{peaks['source']} bf16 GEMM peak" + (" x 0.5 (tf32)" if m["assign_path"] == 3 else "") +
+                               " / 3 (split products), fp32-equivalent; frac_of_mma_issue_peak divides by the "
+                               "tcgen05.mma issue rate measured in this run / 3",
+                "algorithmic_flops_per_launch": alg["assign"]["flops"],
+                "executed_tensor_TFLOPs": 3.0 * ak["TFLOPs"],
+                "a_operand": ("pre-split fp16 image of Z, made once per fit (class prep)") if m["presplit"]
+                             else "rows split to fp16 pieces inside the kernel"}
+    elif dk.get("bound") == "alu":
+        roof = {"bound": "alu", "achieved": dk["TFLOPs"], "peak": den["ffma_tflops"], "unit": "TFLOP/s",
+                "frac": dk["frac"], "traffic": None,
+                "kernel": "kb_cluster_assign (fp32 FFMA path)" if dominant == "assign"
+                          else "kb_cluster_fit (fp32 FFMA kernel, all iterations in one launch)",
+                "peak_source": "fp32 FMA rate measured in this run (kb_probe_peaks); derived figure 148 SM x 128 lanes "
+                               "x 2 flop x max SM clock = %.1f" % (148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12),
+                "algorithmic_flops_per_launch": alg[dominant]["flops"]}
+    else:
+        roof = {"bound": "hbm", "achieved": dk["GBps"], "peak": den["hbm_gbs"], "unit": "GB/s", "frac": dk["frac"],
+                "traffic": None, "kernel": f"kb_{dominant}", "peak_source": f"{peaks['source']} copy bandwidth",
+                "algorithmic_bytes_per_launch": alg[dominant]["bytes"]}
+    cap = TRAFFIC_FROM_CAPTURE.get((cfg.name, dominant))
+    if cap is not None:
+        roof["traffic"] = cap["bytes"]
+        roof["traffic_source"] = cap["source"]
+    roof["calls"] = {n: {k: calls[n][k] for k in ("bound", "frac", "avg_us", "calls") if k in calls[n]}
+                     for n in ("assign", "update", "score", "prune", "normalize", "fit") if n in calls}
+    return roof
+
+
 def run_ours(args, cfg):
     import torch
     from paper_2511_18868_b200 import kb
@@ -287,15 +470,7 @@ def run_ours(args, cfg):
     device = torch.device("cuda", local)
     peaks = load_peaks()
 
-    inp = wl.make_inputs(cfg, seed=replica_seed(cfg, rank))
     ctx = kb.KB(local)
-    R = wl.R_RESOURCES
-    dims = dict(B=cfg.B, N=cfg.N, D=cfg.D, K=cfg.K, S=cfg.S, R=R, iters=cfg.iters)
-    params = dict(theta_sat=float(inp["theta_sat"]), c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
-                  prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]))
-    ctx.ensure_workspace(max(ctx.workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S),
-                             ctx.step_workspace_bytes(cfg.B, cfg.N, cfg.D, cfg.K, cfg.S, R)))
-    dev_t = kb.step_tensors(inp, device)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
 
     def barrier():
@@ -304,45 +479,22 @@ def run_ours(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing -------------------------------------------------
-    # The timed region (value, ms_per_step) runs with the library's per-call event pairs OFF: the
-    # events themselves sit in the stream between the kernels.  The per-call breakdown and the
-    # roofline's kernel time come from a second pass of the same K steps with the event pairs ON.
-    for _ in range(args.warmup):
-        flush.zero_()
-        ctx.bandit_step(dims, params, dev_t)
+    # arithmetic ceilings of this GPU, measured now (fp32 FMA; tcgen05.mma issue rate for both kinds)
+    probe = ctx.probe_peaks()
     try:                                            # NVML addresses GPUs by UUID, whatever CUDA_VISIBLE_DEVICES says
         gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
     except Exception:
         gpu_uuid = None
+
+    # ---- the headline workload: device-resident timing ------------------------------------
+    inp = wl.make_inputs(cfg, seed=replica_seed(cfg, rank))
     sampler = ClockSampler(local, gpu_uuid)
-    barrier()
     sampler.start()
-    k0, m0 = ctx.launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in ev:
-        flush.zero_()
-        a.record()
-        ctx.bandit_step(dims, params, dev_t)
-        b.record()
-    barrier()
-    k1, m1 = ctx.launch_count()
-    total_ms = sum(a.elapsed_time(b) for a, b in ev)
-    ctx.timing_enable(True)
-    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in ev2:
-        flush.zero_()
-        a.record()
-        ctx.bandit_step(dims, params, dev_t)
-        b.record()
-    barrier()
+    m = measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, args.steps, args.warmup, args.min_seconds,
+                         flush, barrier, lambda v: reduce_max(v, dist, device))
     clocks = sampler.stop()
-    breakdown_ms = sum(a.elapsed_time(b) for a, b in ev2)
-    per_class = ctx.timing_read()
-    ctx.timing_enable(False)
-    status = ctx.device_status()
-    assign_path = ctx.assign_path()
-    presplit = ctx.assign_presplit()
+    dims, params, dev_t = m["dims"], m["params"], m["dev_t"]
+    R = wl.R_RESOURCES
 
     # ---- end to end through the host-buffer entry point ----------------------------
     host_t = kb.step_tensors(inp, None, pinned_host=True)
@@ -363,10 +515,13 @@ def run_ours(args, cfg):
         ctx.bandit_step_host(dims, params, e2e_t)
         b.record()
     barrier()
-    e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
+    e2e_ms = float(np.median([a.elapsed_time(b) for a, b in e2e_ev]))
+    del host_t, e2e_t
 
-    # ---- max over ranks -----------------------------------------------------------
-    total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], dist, device)
+    # ---- max over ranks (the slowest replica defines the job's time) -------------------------
+    st = m["stats"]
+    ms_per_step, ms_min, ms_max, ms_mean, e2e_ms = reduce_max([st["median"], st["min"], st["max"], st["mean"], e2e_ms],
+                                                               dist, device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -554,64 +709,9 @@ def run_ours(args, cfg):
         except Exception:                                     # noqa: BLE001
             pass
 
-    ms_per_step = total_ms / args.steps
     value = job_value(world, cfg.arms, ms_per_step)
-    e2e_value = job_value(world, cfg.arms, e2e_ms / e2e_steps)
-
-    # ---- per-call rooflines ---------------------------------------------------------
-    alg = algorithmic(cfg)
-    hbm = peaks["hbm_gbs"]
-    ffma_tflops = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # 148 SMs x 128 fp32 lanes x 2 flop x clock
-    kernels = {}
-    for name in ["normalize", "assign", "update", "fit", "prune", "score"]:
-        ms, calls = per_class[name]
-        if calls == 0:
-            continue
-        avg_s = ms / calls * 1e-3
-        gbs = alg[name]["bytes"] / avg_s / 1e9
-        kernels[name] = {"calls": int(calls), "avg_us": avg_s * 1e6, "share": ms / max(breakdown_ms, 1e-9),
-                         "GBps": gbs, "hbm_frac": gbs / hbm, "TFLOPs": alg[name]["flops"] / avg_s / 1e12}
-    dominant = max(kernels, key=lambda n: kernels[n]["share"])
-    dk = kernels[dominant]
-    hbm_time = alg[dominant]["bytes"] / (hbm * 1e9)
-    alu_time = alg[dominant]["flops"] / (ffma_tflops * 1e12)
-    if dominant == "assign" and assign_path in (2, 3):
-        # the dominant KERNEL is the contraction kernel: its own event pairs give its launch duration; the
-        # whole call (preparation + contraction + fix-up kernels) is reported beside it
-        kms, kcalls = per_class.get("assign_kernel", (0.0, 0))
-        k_s = (kms / kcalls * 1e-3) if kcalls else dk["avg_us"] * 1e-6
-        k_tflops = alg["assign"]["flops"] / k_s / 1e12
-        # three tensor-core products per fp32-equivalent product.  fp16 split (path 2): the measured bf16
-        # GEMM peak is the 16-bit tensor rate itself; tf32 split (path 3): half of it (nominal ratio).
-        kind_peak = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5)
-        split = "fp16 hi/lo split, kind::f16" if assign_path == 2 else "3xTF32, kind::tf32"
-        roof = {"bound": "tensor", "achieved": k_tflops, "peak": kind_peak / 3.0, "unit": "TFLOP/s",
-                "frac": k_tflops / (kind_peak / 3.0), "traffic": None,
-                "kernel": f"assign_tc_kernel (tcgen05 {split}), the contraction kernel of kb_cluster_assign",
-                "kernel_avg_us": k_s * 1e6, "kernel_launches": int(kcalls),
-                "whole_call": {"avg_us": dk["avg_us"], "TFLOPs": dk["TFLOPs"], "frac": dk["TFLOPs"] / (kind_peak / 3.0),
-                               "what": "preparation + contraction + fix-up kernels of one kb_cluster_assign"},
-                "peak_source": f"{peaks['source']} bf16 GEMM peak" + (" x 0.5 (tf32)" if assign_path == 3 else "") +
-                               " / 3 (split products), fp32-equivalent",
-                "algorithmic_flops_per_launch": alg["assign"]["flops"],
-                "executed_tensor_TFLOPs": 3.0 * k_tflops,
-                "a_operand": ("pre-split fp16 image of Z, made once per fit (its conversion is timed inside the "
-                              "step and counted with the assign calls)") if presplit
-                             else "rows split to fp16 pieces inside the kernel"}
-    elif dominant in ("assign", "fit") and alu_time > hbm_time:
-        roof = {"bound": "alu", "achieved": dk["TFLOPs"], "peak": ffma_tflops, "unit": "TFLOP/s",
-                "frac": dk["TFLOPs"] / ffma_tflops, "traffic": None,
-                "kernel": "kb_cluster_assign (fp32 FFMA path)" if dominant == "assign"
-                          else "kb_cluster_fit (fused fp32 FFMA kernel, all iterations in one launch)",
-                "peak_source": "148 SM x 128 lanes x 2 flop x max SM clock",
-                "algorithmic_flops_per_launch": alg["assign"]["flops"]}
-    else:
-        roof = {"bound": "hbm", "achieved": dk["GBps"], "peak": hbm, "unit": "GB/s", "frac": dk["hbm_frac"],
-                "traffic": None, "kernel": f"kb_{dominant}", "peak_source": f"{peaks['source']} copy bandwidth",
-                "algorithmic_bytes_per_launch": alg[dominant]["bytes"]}
-    traffic = TRAFFIC_FROM_NCU.get((cfg.name, dominant))
-    if traffic is not None:
-        roof["traffic"] = traffic
+    e2e_value = job_value(world, cfg.arms, e2e_ms)
+    roof = dominant_roofline(cfg, m, peaks)
 
     # ---- CPU oracle beside it (bounded sample) ----------------------------------------
     cpu = None
@@ -621,16 +721,52 @@ def run_ours(args, cfg):
         cpu = {"value": cfg.arms / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
                "seconds_spent": spent, "host_cores": os.cpu_count()}
 
+    # ---- the other workloads, one after the other on the same context (rank 0; device-resident only) ----------
+    headline = workload_summary(cfg, m, world)
+    del dev_t, m["dev_t"]
+    torch.cuda.empty_cache()
+    others = {}
+    if not args.only and args.rows == 0:
+        for name, ocfg in wl.CONFIGS.items():
+            if name == cfg.name:
+                continue
+            try:
+                oinp = wl.make_inputs(ocfg)
+                om = measure_workload(ctx, kb, torch, ocfg, oinp, device, peaks, probe, args.steps, args.warmup,
+                                      min(args.min_seconds, 0.25), flush, torch.cuda.synchronize)
+                others[name] = workload_summary(ocfg, om, 1)
+                del om, oinp
+                torch.cuda.empty_cache()
+            except Exception as exc:                          # noqa: BLE001
+                others[name] = {"error": f"{type(exc).__name__}: {exc}"}
+    workloads = {cfg.name: headline}
+    workloads.update(others)
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": workload_config(cfg),
+        "ms_per_step": ms_per_step, "ms_per_step_min": ms_min, "ms_per_step_max": ms_max, "ms_per_step_mean": ms_mean,
+        "timed_steps": st["steps"], "timed_seconds": st["seconds"],
+        "timing": "median over the timed steps; loops of exactly `steps` steps repeated until >= %g s of timed steps; "
+                  "each step between its own CUDA events, L2 flushed before it" % args.min_seconds,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": DTYPE, "data": "synthetic", "config": workload_config(cfg),
         "roofline": roof, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
-        "gpu_launches": int(k1 - k0), "memset_nodes": int(m1 - m0), "clocks": clocks, "kernels": kernels,
-        "device_status": int(status), "peaks": peaks,
-        "breakdown_pass_ms_per_step": breakdown_ms / args.steps,
+                "ms_per_step": e2e_ms, "steps": e2e_steps},
+        "gpu_launches": m["launches"], "gpu_launches_per_step": m["launches"] / st["steps"], "memset_nodes": m["memsets"],
+        "clocks": clocks, "kernels": m["calls"],
+        "device_status": m["status"],
+        "peaks": dict(peaks, measured_in_run=probe,
+                      note="hbm_gbs and bf16_tflops: the pool's measured copy and GEMM peaks; measured_in_run: "
+                           "kb_probe_peaks on this GPU (fp32 FMA chains; tcgen05.mma M128 N128 issue rate, "
+                           "kind::f16 K16 and kind::tf32 K8, fp32-equivalent = / 3)"),
+        "breakdown_pass_ms_per_step": m["breakdown_ms_per_step"],
+        "near_ties": {"tensor_assign_final": m["near"],
+                      "note": "rows of the final assignment whose runner-up lay within the tensor path's re-evaluation "
+                              "bound and were settled in the exact fp32 direct form (the library's own counters); the "
+                              "oracle-arbitrated near-tie counts of labels, keep bits and selections are printed by "
+                              "the full-size parity tests"},
+        "workloads": workloads,
     }
     line.update(extra)
     print(json.dumps(line))
@@ -647,6 +783,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", action="store_true", help="time the named workload alone (no table of the other four)")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="repeat the loop of `steps` timed steps until this many seconds of timed steps have run")
     ap.add_argument("--rows", type=int, default=0,
                     help="override N (rows per instance): a smaller case of the same kernels for ncu captures; "
                          "numbers from such a run are not bench values")

@@ -84,9 +84,35 @@ kb_status kb_set_workspace(kb_ctx* ctx, void* dev_ptr, size_t bytes);
 const char* kb_status_string(kb_status s);
 /* Text of the last failure on this context (host string owned by the context). */
 const char* kb_last_error(kb_ctx* ctx);
-/* Reads the device status word (0 = fine).  Synchronises the stream; not for
- * the hot path.  `out` is a host pointer. */
+/* Conditions that only the device can see are OR-ed into the context's device
+ * status word; the call that queued the work has long returned KB_OK by then.
+ *
+ *   bit     set by                                   meaning
+ *   0x001   update, score, prune, radius kernels     a label outside [0, K): the row / candidate was skipped
+ *                                                    (prune: treated as cluster 0)
+ *   0x002   prune, sample, select_pair kernels       a target[s] outside [0, R): the arm / pair was masked
+ *   0x004   init_centroids, sample, record kernels   a row, member or pair index out of range: nothing written for it
+ *   0x100   tensor-core assign kernel                a bounded wait between its roles expired; the CTA drained and
+ *                                                    left; labels of that launch are unspecified
+ *   0x200   cooperative fit kernel                   its bounded grid-wide barrier expired; results unspecified
+ *
+ * kb_get_device_status synchronises the stream (not for the hot path), stores
+ * the word in *out (host pointer) and returns KB_ERR_TIMEOUT if 0x100 or 0x200
+ * is set, else KB_OK (the contract bits 0x001..0x004 are the caller's to read).
+ * The word keeps its bits until kb_clear_device_status queues its clearing on
+ * the stream.  After a timeout the context stays usable: clear and call again. */
+#define KB_STATUS_BAD_LABEL 0x001
+#define KB_STATUS_BAD_TARGET 0x002
+#define KB_STATUS_BAD_INDEX 0x004
+#define KB_STATUS_TIMEOUT_ASSIGN 0x100
+#define KB_STATUS_TIMEOUT_FIT 0x200
 kb_status kb_get_device_status(kb_ctx* ctx, int* out);
+kb_status kb_clear_device_status(kb_ctx* ctx);
+/* The mapping itself, as a pure host function (no context, no device): the
+ * kb_status that a status word stands for -- KB_ERR_TIMEOUT for a timeout bit;
+ * with contract_bits_too != 0 also KB_ERR_INVALID_ARG for 0x001..0x004, which
+ * is what kb_bandit_step_host returns; else KB_OK. */
+kb_status kb_status_of_device_word(int word, int contract_bits_too);
 /* Number of kernels of this library the context has queued since creation
  * (`kernels`) and of memset nodes (`memsets`, nullable).  Host pointers. */
 kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets);
@@ -107,9 +133,25 @@ kb_status kb_get_launch_count(kb_ctx* ctx, uint64_t* kernels, uint64_t* memsets)
 #define KB_T_FIT 6 /* kb_cluster_fit when it runs as one fused launch (small instances) */
 #define KB_T_ASSIGN_KERNEL 7 /* the tensor-core contraction kernel alone (nested inside KB_T_ASSIGN or KB_T_FIT) */
 #define KB_T_SAMPLE 8 /* kb_sample_member, kb_record_outcome, kb_cluster_radius */
-#define KB_T_COUNT 9
+#define KB_T_PREP 9   /* once per tensor-path kb_cluster_fit: the conversion of Z to its pre-split fp16 image */
+#define KB_T_COUNT 10
 kb_status kb_timing_enable(kb_ctx* ctx, int on);
 kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
+
+/* Arithmetic ceilings of the device the context is bound to, measured in the
+ * instruction shapes this library's kernels use (a benchmark's denominators;
+ * the paper has no counterpart).  fp32: independent register-resident FMA
+ * chains on every SM.  Tensor cores: back-to-back tcgen05.mma M = 128, N = 128,
+ * A from tensor memory, B from shared memory, fp32 accumulation, one CTA per SM,
+ * for kind::f16 (K = 16) and kind::tf32 (K = 8).  Three launches of about a
+ * millisecond each (after a warm-up launch each) on the context's stream;
+ * synchronises; no workspace.  `out` is a host pointer.  Every wait in the
+ * probe kernels is bounded; KB_ERR_TIMEOUT if the products did not retire. */
+typedef struct {
+    double ffma_tflops, mma_f16_tflops, mma_tf32_tflops; /* 2 flop per multiply-add */
+    float ffma_ms, mma_f16_ms, mma_tf32_ms;              /* duration of the timed launch */
+} kb_peak_probe;
+kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out);
 
 /* ---- the five calls ----------------------------------------------------- */
 
@@ -401,11 +443,20 @@ kb_status kb_assign_tc_probe(kb_ctx* ctx, int B, int N, int D, int K, const floa
  *   device attributes; make that first call before any stream capture begins.
  *   Every call on a device shares the one array (the call clears what it needs first), so
  *   two calls that overlap on the GPU -- different streams, no ordering -- race: order them.
- *   Label errors are recorded in the array's own status word, not in a context. */
+ *   (The per-device look-up itself is idempotent: two host threads making the first call at
+ *   once store the same values.)
+ *   A label outside [0, K) is skipped (it adds to no sum and no count) and sets bit 1 of the
+ *   array's own status word -- there is no context to carry it.  The call still returns KB_OK:
+ *   read the word with kb_cluster_update_noalloc_status. */
 #define KB_NOALLOC_MAX_KD 65536
 #define KB_NOALLOC_MAX_K 4096
 kb_status kb_cluster_update_noalloc(void* cuda_stream, int N, int D, int K, const float* z,
                                     const int32_t* labels, float* centroids, int32_t* counts);
+/* Reads the status word of the allocation-free update on the CURRENT device into *out (host
+ * pointer; 0 = fine, bit 1 = a label outside [0, K) was skipped since the last read) and clears
+ * it.  Synchronises `cuda_stream` (so it sees every call queued there before it); allocates
+ * nothing.  Not for the hot path. */
+kb_status kb_cluster_update_noalloc_status(void* cuda_stream, int* out);
 
 /* ---- conveniences built from the five calls ----------------------------- */
 
@@ -495,7 +546,10 @@ kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
  * the values are the ones kb_prune gives.  The device
  * staging area is carved from the registered workspace, which must hold
  * kb_step_workspace_bytes(...) bytes.  Pinned host memory makes the copies
- * asynchronous; pageable memory works too. */
+ * asynchronous; pageable memory works too.  Since this call synchronises
+ * anyway, it also reads the device status word before returning: a timeout bit
+ * gives KB_ERR_TIMEOUT, a contract bit (label, target or index out of range)
+ * KB_ERR_INVALID_ARG; the outputs are then unspecified. */
 kb_status kb_step_workspace_bytes(int B, int N, int D, int K, int S, int R, size_t* out);
 kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* host_args);
 

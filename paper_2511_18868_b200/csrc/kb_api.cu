@@ -50,6 +50,16 @@ struct TimeScope {
 
 }  // namespace
 
+// What a device status word means for the caller of a synchronising entry point.
+kb_status kb_status_from_device_word(kb_ctx* ctx, int word, bool contract_bits_too) {
+    if (word & (KB_STATUS_TIMEOUT_ASSIGN | KB_STATUS_TIMEOUT_FIT))
+        return kb_fail(ctx, KB_ERR_TIMEOUT, "a bounded device-side wait expired (device status 0x%x)", word);
+    if (contract_bits_too && (word & (KB_STATUS_BAD_LABEL | KB_STATUS_BAD_TARGET | KB_STATUS_BAD_INDEX)))
+        return kb_fail(ctx, KB_ERR_INVALID_ARG, "a label, target or index on the device was out of range (device status 0x%x)",
+                       word);
+    return KB_OK;
+}
+
 kb_status kb_launch_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
                                    float* c) {
     if (B == 0 || K == 0) return KB_OK;
@@ -201,6 +211,16 @@ kb_status kb_get_device_status(kb_ctx* ctx, int* out) {
     if (!ctx || !out) return KB_ERR_INVALID_ARG;
     KB_CUDA(ctx, cudaMemcpyAsync(out, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     KB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return kb_status_from_device_word(ctx, *out, false);
+}
+
+kb_status kb_status_of_device_word(int word, int contract_bits_too) {
+    return kb_status_from_device_word(nullptr, word, contract_bits_too != 0);
+}
+
+kb_status kb_clear_device_status(kb_ctx* ctx) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    KB_MEMSET(ctx, ctx->dev_status, 0, sizeof(int));
     return KB_OK;
 }
 
@@ -457,7 +477,7 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
     const bool tensor = N > 0 && z && ctx->assign_path != 1 &&
                         (ctx->assign_path >= 2 ? kb_assign_tc_supported(ctx, B, D, K) : kb_assign_tc_eligible(ctx, B, N, D, K));
     if (tensor && iters >= 2 && zneed > 0 && ctx->ws_bytes >= zoff + zneed) {
-        TimeScope ts__(ctx, KB_T_ASSIGN);
+        TimeScope ts__(ctx, KB_T_PREP);
         s = kb_zsplit_prepare(ctx, ctx->ws + zoff, B, N, D, K, z);
     }
     if (tensor && iters >= 1 && ctx->ws_bytes >= aoff + aneed) {
@@ -700,8 +720,11 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     KB_D2H(best_val, B, float);
     KB_D2H(best_cluster_arm, B, int32_t);
 #undef KB_D2H
+    // this call synchronises anyway: the status word comes back with the results
+    int word = 0;
+    KB_CUDA(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st));
     KB_CUDA(ctx, cudaStreamSynchronize(st));
-    return KB_OK;
+    return kb_status_from_device_word(ctx, word, true);
 }
 
 }  // extern "C"

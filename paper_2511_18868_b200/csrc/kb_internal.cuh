@@ -47,6 +47,7 @@ struct kb_ctx {
 
 // ---- error plumbing ---------------------------------------------------------
 kb_status kb_fail(kb_ctx* ctx, kb_status s, const char* fmt, ...);
+kb_status kb_status_from_device_word(kb_ctx* ctx, int word, bool contract_bits_too);
 
 #define KB_CUDA(ctx, expr)                                                                     \
     do {                                                                                       \

@@ -412,6 +412,37 @@ int g_noalloc_sms[NOALLOC_MAX_DEVICES];
 int g_noalloc_smem[NOALLOC_MAX_DEVICES];
 }  // namespace
 
+// Set-up of the current device, once: the scratch array's device address and two attributes.
+// Two threads that race here write the same values (the look-up is idempotent).
+static kb_status noalloc_setup(int* dev_out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return KB_ERR_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, kb_noalloc_scratch) != cudaSuccess || !p) return KB_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&g_noalloc_smem[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return KB_ERR_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    *dev_out = dev;
+    return KB_OK;
+}
+
+extern "C" kb_status kb_cluster_update_noalloc_status(void* cuda_stream, int* out) {
+    if (!out) return KB_ERR_INVALID_ARG;
+    int dev = -1;
+    const kb_status s = noalloc_setup(&dev);
+    if (s != KB_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, g_noalloc_ptr[dev], sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KB_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KB_ERR_CUDA;
+    if (word != 0 && cudaMemsetAsync(g_noalloc_ptr[dev], 0, sizeof(int), st) != cudaSuccess) return KB_ERR_CUDA;
+    *out = word;
+    return KB_OK;
+}
+
 extern "C" kb_status kb_cluster_update_noalloc(void* cuda_stream, int N, int D, int K, const float* z,
                                                const int32_t* labels, float* centroids, int32_t* counts) {
     if (N < 0 || D < 1 || K < 1) return KB_ERR_INVALID_ARG;
@@ -420,16 +451,8 @@ extern "C" kb_status kb_cluster_update_noalloc(void* cuda_stream, int N, int D, 
     // sizes beyond the built-in scratch are refused, never truncated
     if ((long long)K * D > KB_NOALLOC_MAX_KD || K > KB_NOALLOC_MAX_K) return KB_ERR_UNSUPPORTED;
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return KB_ERR_CUDA;
-    if (!g_noalloc_ptr[dev]) {
-        // first call on this device (it is the current one): look the symbol up, read two attributes
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, kb_noalloc_scratch) != cudaSuccess || !p) return KB_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&g_noalloc_smem[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-            return KB_ERR_CUDA;
-        g_noalloc_ptr[dev] = p;
-    }
+    const kb_status su = noalloc_setup(&dev);      // first call on this device (it is the current one)
+    if (su != KB_OK) return su;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
     int* status = reinterpret_cast<int*>(base);

@@ -22,14 +22,19 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 
 # every symbol include/kb.h declares
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
-           "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_get_launch_count",
-           "kb_timing_enable", "kb_timing_read", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
+           "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_clear_device_status", "kb_status_of_device_word", "kb_get_launch_count",
+           "kb_timing_enable", "kb_timing_read", "kb_probe_peaks", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
-           "kb_bandit_step_host", "kb_cluster_update_noalloc"]
+           "kb_bandit_step_host", "kb_cluster_update_noalloc", "kb_cluster_update_noalloc_status"]
 
 
-TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fit", "assign_kernel", "sample"]
+TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fit", "assign_kernel", "sample", "prep"]
+
+
+class PeakProbe(ctypes.Structure):
+    _fields_ = [("ffma_tflops", ctypes.c_double), ("mma_f16_tflops", ctypes.c_double), ("mma_tf32_tflops", ctypes.c_double),
+                ("ffma_ms", ctypes.c_float), ("mma_f16_ms", ctypes.c_float), ("mma_tf32_ms", ctypes.c_float)]
 
 
 class KbError(RuntimeError):
@@ -80,9 +85,12 @@ def load_library() -> ctypes.CDLL:
     lib.kb_last_error.argtypes = [_VP]
     lib.kb_last_error.restype = ctypes.c_char_p
     lib.kb_get_device_status.argtypes = [_VP, ctypes.POINTER(i)]
+    lib.kb_clear_device_status.argtypes = [_VP]
+    lib.kb_status_of_device_word.argtypes = [i, i]
     lib.kb_get_launch_count.argtypes = [_VP, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
     lib.kb_timing_enable.argtypes = [_VP, i]
     lib.kb_timing_read.argtypes = [_VP, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    lib.kb_probe_peaks.argtypes = [_VP, ctypes.POINTER(PeakProbe)]
     lib.kb_normalize.argtypes = [_VP, i, i, i, _VP, _VP, _VP, _VP]
     lib.kb_prune.argtypes = [_VP, i, i, i, i, i] + [_VP] * 9 + [f] + [_VP] * 3
     lib.kb_cluster_assign.argtypes = [_VP, i, i, i, i] + [_VP] * 6
@@ -100,6 +108,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_get_assign_presplit.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_assign_tc_probe.argtypes = [_VP, i, i, i, i] + [_VP] * 5
     lib.kb_cluster_update_noalloc.argtypes = [_VP, i, i, i, _VP, _VP, _VP, _VP]
+    lib.kb_cluster_update_noalloc_status.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
     lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
@@ -185,10 +194,16 @@ class KB:
         if have < nbytes:
             self.set_workspace(torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device))
 
-    def device_status(self) -> int:
+    def device_status(self, raise_on_timeout: bool = True) -> int:
+        """The device status word (synchronises).  A timeout bit raises KbError(KB_ERR_TIMEOUT) unless told not to."""
         out = ctypes.c_int()
-        self._check(self.lib.kb_get_device_status(self.h, ctypes.byref(out)), "kb_get_device_status")
+        rc = self.lib.kb_get_device_status(self.h, ctypes.byref(out))
+        if rc != KB_OK and (raise_on_timeout or rc != 5):
+            self._check(rc, "kb_get_device_status")
         return out.value
+
+    def clear_device_status(self):
+        self._check(self.lib.kb_clear_device_status(self.h), "kb_clear_device_status")
 
     def launch_count(self):
         """(kernels, memset nodes) queued by this context so far."""
@@ -205,6 +220,12 @@ class KB:
         n = (ctypes.c_int64 * len(TIMING_CLASSES))()
         self._check(self.lib.kb_timing_read(self.h, ms, n), "kb_timing_read")
         return {name: (ms[i], n[i]) for i, name in enumerate(TIMING_CLASSES)}
+
+    def probe_peaks(self) -> Dict[str, float]:
+        """kb_probe_peaks: measured fp32 FMA and tcgen05 (kind::f16, kind::tf32) ceilings of this device, TFLOP/s."""
+        p = PeakProbe()
+        self._check(self.lib.kb_probe_peaks(self.h, ctypes.byref(p)), "kb_probe_peaks")
+        return {name: float(getattr(p, name)) for name, _ in PeakProbe._fields_}
 
     def _p(self, t):
         return _ptr(t, self.device)
@@ -369,14 +390,39 @@ def cluster_update_noalloc(z, labels, centroids, counts=None, stream=None):
     """kb_cluster_update_noalloc: one instance, scratch built into the library, nothing allocated.
     z [N][D], labels [N], centroids [K][D] (updated in place), counts [K] or None; device tensors."""
     lib = load_library()
+    # the C entry point takes bare pointers: a wrong shape or dtype here would be an out-of-bounds device access
+    if z.dim() != 2 or centroids.dim() != 2 or labels.dim() != 1:
+        raise ValueError("cluster_update_noalloc: z [N][D], labels [N], centroids [K][D]")
     N, D = z.shape
     K = centroids.shape[0]
+    if centroids.shape[1] != D or labels.numel() != N or (counts is not None and counts.numel() != K):
+        raise ValueError("cluster_update_noalloc: shapes disagree")
+    if z.dtype != torch.float32 or centroids.dtype != torch.float32 or labels.dtype != torch.int32 or \
+            (counts is not None and counts.dtype != torch.int32):
+        raise ValueError("cluster_update_noalloc: z, centroids float32; labels, counts int32")
+    for a in (z, labels, centroids, counts):
+        if a is not None and (not a.is_cuda or not a.is_contiguous() or a.device != z.device):
+            raise ValueError("cluster_update_noalloc: contiguous tensors on one CUDA device")
     st = stream if stream is not None else torch.cuda.current_stream(z.device)
     with torch.cuda.device(z.device):
         rc = lib.kb_cluster_update_noalloc(_VP(st.cuda_stream), N, D, K, _ptr(z), _ptr(labels), _ptr(centroids),
                                            _ptr(counts))
     if rc != KB_OK:
         raise KbError(rc, "kb_cluster_update_noalloc")
+
+
+def cluster_update_noalloc_status(device=None, stream=None) -> int:
+    """kb_cluster_update_noalloc_status: reads and clears the status word of the allocation-free update on
+    `device` (bit 1: a label outside [0, K) was skipped).  Synchronises the stream."""
+    lib = load_library()
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    st = stream if stream is not None else torch.cuda.current_stream(device)
+    out = ctypes.c_int()
+    with torch.cuda.device(device):
+        rc = lib.kb_cluster_update_noalloc_status(_VP(st.cuda_stream), ctypes.byref(out))
+    if rc != KB_OK:
+        raise KbError(rc, "kb_cluster_update_noalloc_status")
+    return out.value
 
 
 def step_tensors(inp: Dict, device, want_arm_index=True, want_bound=True, pinned_host=False) -> Dict[str, torch.Tensor]:

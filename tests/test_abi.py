@@ -62,3 +62,18 @@ def test_struct_layout_matches_header():
     assert ctypes.sizeof(kb.ScoreParams) == 20
     assert ctypes.sizeof(kb.StepArgs) == 56 + 8 * 30
     assert len(kb._STEP_IN) == 13 and len(kb._STEP_OUT) == 17
+
+
+def test_device_status_word_maps_to_a_status(lib):
+    """What a synchronising entry point returns for a device status word (no device needed: the mapping
+    is a pure host function).  Timeout bits win over contract bits; contract bits count only where asked."""
+    f = lib.kb_status_of_device_word
+    assert f(0, 0) == 0 and f(0, 1) == 0
+    assert f(0x100, 0) == 5 and f(0x200, 0) == 5 and f(0x300, 1) == 5
+    assert lib.kb_status_string(f(0x100, 0)) == b"KB_ERR_TIMEOUT"
+    for bit in (1, 2, 4, 7):
+        assert f(bit, 0) == 0                       # kb_get_device_status leaves these to the caller
+        assert f(bit, 1) == 1                       # kb_bandit_step_host reports them
+        assert f(bit | 0x200, 1) == 5
+    assert lib.kb_clear_device_status(None) == 1
+    assert lib.kb_cluster_update_noalloc_status(None, None) == 1

@@ -1,7 +1,11 @@
-"""Full-size parity: the workloads the benchmark times (`large`, `contraction`), in the launch
-configuration it uses (kb_bandit_step on device buffers), checked against the oracle on what the
-oracle can afford: every streaming call in full, the assignment on a seeded row sample, and
-properties that hold at any size (counts, centroid = member mean, objective not increasing)."""
+"""Full-size parity: the workloads the benchmark times, in the launch configuration it uses
+(kb_bandit_step on device buffers; `batched` also through kb_bandit_step_host), checked against the
+oracle: every streaming call in full, the assignment on a seeded row sample element by element AND
+on every row for optimality (the oracle's row loop spread over the host's cores), the centroid
+update recomputed by the oracle from the verified labels, and properties that hold at any size."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -13,6 +17,33 @@ from paper_2511_18868_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 SAMPLE = {"large": 32768, "contraction": 65536}
+
+
+def full_argmin_check(z, c, labels, chunk=4096):
+    """For EVERY row: d2(row, centroid named by `labels`) <= min_j d2(row, c_j) * (1 + 1e-5), in double.
+    The single-threaded oracle functions run on row ranges from a thread pool (they release the
+    interpreter lock while they run), one range per task; nothing is computed here but the comparison.
+    Returns (rows whose label differs from the oracle's argmin, worst relative excess)."""
+    B, N, _ = z.shape
+    assert B == 1
+    workers = len(os.sched_getaffinity(0))
+
+    def part(lo):
+        hi = min(N, lo + chunk)
+        zs = z[:, lo:hi]                                         # a contiguous view: no copy
+        a = oracle.cluster_assign(zs, c, want_rep=False, want_margins=True)
+        d_at = oracle.dist2_at(zs, c, labels[:, lo:hi])
+        excess = (d_at - a["best"]) / np.maximum(d_at, 1e-300)
+        differ = int((a["labels"] != labels[:, lo:hi]).sum())
+        return differ, float(excess.max()), int((excess > parity.NEAR_TIE).sum())
+
+    with ThreadPoolExecutor(workers) as pool:
+        out = list(pool.map(part, range(0, N, chunk)))
+    differ = sum(o[0] for o in out)
+    worst = max(o[1] for o in out)
+    bad = sum(o[2] for o in out)
+    assert bad == 0, f"{bad} of {N} rows sit with a centroid worse than the optimum by more than 1e-5 (worst {worst:.3e})"
+    return differ, worst, workers
 
 
 @pytest.mark.parametrize("name", ["large", "contraction"])
@@ -44,6 +75,14 @@ def test_fullsize_step(name):
         torch.cuda.synchronize()
         assert ctx.device_status() == 0
         got["member"], got["member_val"] = member.cpu().numpy(), member_val.cpu().numpy()
+        # one more centroid update on the device from the step's own final labels (checked below against
+        # the oracle's update from the same labels, once every label has been verified)
+        c_upd, n_upd = t["centroids"].clone(), torch.empty((B, K), dtype=torch.int32, device=ctx.device)
+        ctx.cluster_update(t["z"], t["labels"], c_upd, n_upd)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        got["c_upd"], got["n_upd"] = c_upd.cpu().numpy(), n_upd.cpu().numpy()
+        del c_upd, n_upd
     finally:
         ctx.close()
     del t
@@ -63,8 +102,11 @@ def test_fullsize_step(name):
     same = labels[:, rows] == a["labels"]
     parity.close(got["dist2"][:, rows][same], a["dist2"][same], atol=1e-7, what="dist2 (sample)")
 
-    # properties at full size: every label in range, counts add up, inertia is the sum of dist2
+    # assign, every row: the label's centroid is optimal within the near-tie margin (double, all K centroids)
     assert labels.min() >= 0 and labels.max() < K
+    differ, worst, workers = full_argmin_check(z, c, labels)
+
+    # properties at full size: counts add up, inertia is the sum of dist2
     assert got["counts"].sum() == N
     parity.close(got["inertia"], np.array([got["dist2"].astype(np.float64).sum()]), atol=0, rtol=1e-5, what="inertia")
     # one more oracle update from the GPU's labels must not move the objective up (Lloyd's invariant),
@@ -72,6 +114,9 @@ def test_fullsize_step(name):
     c_next, n_next = oracle.cluster_update(z, labels, c)
     member = np.bincount(labels[0], minlength=K)
     assert np.array_equal(n_next[0], member)
+    # the device's update from the same (now verified) labels: counts exact, centroids within 1e-4
+    assert np.array_equal(got["n_upd"], n_next)
+    parity.close(got["c_upd"], c_next, atol=1e-5, what="centroids recomputed from the verified labels")
     d_next = oracle.dist2_at(z, c_next, labels).sum()
     assert d_next <= got["dist2"].astype(np.float64).sum() * (1 + 1e-6)
     rep = got["rep"][0]
@@ -99,5 +144,68 @@ def test_fullsize_step(name):
                              inp["t"], K)
     assert d["member"][0] >= 0 and labels[0, got["member"][0]] == got["best_cluster_arm"][0] // S
     parity.member_match(got["member"], got["member_val"], d, 5e-5)
-    print(f"[{name} full size] near-ties: labels (sample of {len(rows)}) {ties}, keep bits {prune_ties}, "
-          f"selection {sel_ties}")
+    print(f"[{name} full size] near-ties: labels (sample of {len(rows)}) {ties}, labels (all {N} rows, {workers} "
+          f"threads) {differ} with worst excess {worst:.2e}, keep bits {prune_ties}, selection {sel_ties}")
+
+
+@pytest.mark.parametrize("host_buffers", [False, True], ids=["device", "host"])
+def test_fullsize_batched(host_buffers):
+    """`batched` at its full size, 1024 instances (more one-CTA instances than the GPU keeps resident at
+    once), through kb_bandit_step and kb_bandit_step_host: every instance against the oracle -- the
+    free-running whole step (objective, label agreement) and each call's result from the GPU's own
+    inputs to that call."""
+    from paper_2511_18868_b200 import kb
+    cfg = wl.CONFIGS["batched"]
+    inp = wl.make_inputs(cfg)
+    B, N, D, K, S = cfg.B, cfg.N, cfg.D, cfg.K, cfg.S
+    dims = dict(B=B, N=N, D=D, K=K, S=S, R=wl.R_RESOURCES, iters=cfg.iters)
+    params = dict(theta_sat=float(inp["theta_sat"]), c=float(inp["c"]), lipschitz_L=float(inp["lipschitz_L"]),
+                  prior_pulls=float(inp["prior_pulls"]), prior_mean=float(inp["prior_mean"]))
+    ctx = kb.KB(0)
+    try:
+        if host_buffers:
+            ctx.ensure_workspace(ctx.step_workspace_bytes(B, N, D, K, S, wl.R_RESOURCES))
+            t = kb.step_tensors(inp, None, pinned_host=True)
+            ctx.bandit_step_host(dims, params, t)
+            got = {k: v.numpy() for k, v in t.items()}
+        else:
+            ctx.ensure_workspace(ctx.workspace_bytes(B, N, D, K, S))
+            t = kb.step_tensors(inp, ctx.device)
+            ctx.bandit_step(dims, params, t)
+            torch.cuda.synchronize()
+            got = {k: v.cpu().numpy() for k, v in t.items()}
+        assert ctx.device_status() == 0
+    finally:
+        ctx.close()
+    ref = oracle.bandit_step(inp, cfg.iters)
+    parity.close(got["z"], ref["z"], atol=2e-5, what="z")
+    parity.close(got["inertia"], ref["inertia"], atol=0, rtol=1e-3, what="inertia")
+    agree = (got["labels"] == ref["labels"]).mean(axis=1)
+    # a near-tie flip in an early iteration moves a centroid and cascades inside that one instance
+    assert np.median(agree) == 1.0 and (agree > 0.9).mean() > 0.99, f"label agreement per instance: min {agree.min()}"
+    # every instance: labels optimal for the returned centroids, dist2 / inertia / counts consistent
+    chk = oracle.cluster_assign(got["z"], got["centroids"], want_margins=True)
+    ties = parity.labels_match(got["z"], got["centroids"], got["labels"], chk)
+    same = got["labels"] == chk["labels"]
+    parity.close(got["dist2"][same], chk["dist2"][same], atol=1e-7, what="dist2")
+    parity.close(got["inertia"], chk["inertia"], atol=1e-6, what="inertia")
+    assert np.array_equal(got["counts"].sum(1), np.full(B, N))
+    parity.rep_match(got["rep"], chk, got["dist2"], got["labels"]) if ties == 0 else None
+    # prune, statistics, index and both selections of every instance from the GPU's own labels / dist2
+    p = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+                     got["labels"], inp["hsig"], inp["target"], 75.0, want_bound=True, want_margin=True)
+    keep = got["keep"].view(np.uint32)
+    prune_ties = parity.keep_match(keep, p, S)
+    assert int(got["kept_count"].view(np.uint32).astype(np.int64).sum()) == int(np.bitwise_count(keep).sum())
+    parity.close(got["bound"], p["bound"], atol=1e-6, what="bound")
+    s = oracle.score_select(got["labels"], got["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], K, keep=keep,
+                            c=2.0, lipschitz_L=float(inp["lipschitz_L"]))
+    assert np.array_equal(got["cl_pulls"], s["cl_pulls"])
+    parity.close(got["cl_mean"], s["cl_mean"], atol=1e-6, what="cl_mean")
+    parity.close(got["cl_index"], s["cl_index"], atol=1e-6, what="cl_index")
+    parity.close(got["arm_index"], s["arm_index"], atol=1e-6, what="arm_index")
+    sel_ties = parity.select_match(got["best_arm"], got["best_val"], s, s["arm_index"])
+    pair_ties = parity.cluster_select_match(got["best_cluster_arm"], s, s["cl_index"])
+    print(f"[batched full size, {'host' if host_buffers else 'device'} buffers] label agreement with the free-running "
+          f"oracle: mean {agree.mean():.6f}, min {agree.min():.4f}; near-ties: labels {ties}, keep bits {prune_ties}, "
+          f"arm selection {sel_ties}, pair selection {pair_ties}")
