@@ -83,6 +83,10 @@ def algorithmic(cfg: wl.Workload):
         "update": {"bytes": 4 * R * D + 4 * R + 4 * B * K * (D + 1), "flops": R * D},
         "prune": {"bytes": 16 * R + 4 * R + 4 * R * S, "flops": 4 * R * S},
         "score": {"bytes": 8 * R * S + 16 * R + 4 * R * S, "flops": 3 * R * S},
+        # prune and score fused into one call (the tail of a whole step): every array once --
+        # flops, bytes, t_cur, labels, dist2 in (20 R), pulls and reward_sum in (8 R S), keep out (4 R),
+        # bound and arm_index out (8 R S)
+        "tail": {"bytes": 24 * R + 16 * R * S, "flops": 7 * R * S},
         # fused fit (small instances): the instance is read once for all iterations
         "fit": {"bytes": 4 * R * D + 8 * B * K * D + 8 * R, "flops": 2 * R * K * D * (cfg.iters + 1)},
     }
@@ -286,7 +290,7 @@ def median_stats(ms_list):
             "steps": int(a.size), "seconds": float(a.sum() * 1e-3)}
 
 
-def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms):
+def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms, sustained=False):
     """Per-call table of one workload from the library's event pairs: average duration, achieved GB/s and
     TFLOP/s on the call's ALGORITHMIC bytes / flops, and its fraction of the roofline that binds it."""
     alg = algorithmic(cfg)
@@ -294,7 +298,11 @@ def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms):
     ffma_peak = probe["ffma_tflops"]
     # three tensor-core products per fp32-equivalent product; kind::f16 runs at the measured 16-bit GEMM rate,
     # kind::tf32 at half of it (nominal ratio)
-    tensor_peak = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5) / 3.0
+    # (the GEMM peak is the burst figure for kernels timed in short runs at full clock, the sustained one when the
+    # kernel ran inside a loop of a second or more with the power cap active: the clock record decides)
+    gemm_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    tensor_peak = gemm_peak * (1.0 if assign_path == 2 else 0.5) / 3.0
+    tensor_peak_burst = peaks["bf16_tflops"] * (1.0 if assign_path == 2 else 0.5) / 3.0
     mma_issue_peak = (probe["mma_f16_tflops"] if assign_path == 2 else probe["mma_tf32_tflops"]) / 3.0
     out = {}
     for name in ["normalize", "prep", "assign", "update", "fit", "prune", "score"]:
@@ -303,13 +311,18 @@ def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms):
             continue
         avg_s = ms / calls * 1e-3
         row = {"calls": int(calls), "avg_us": avg_s * 1e6, "share": ms / max(breakdown_ms, 1e-9)}
-        if name in alg:
-            gbs = alg[name]["bytes"] / avg_s / 1e9
-            tfl = alg[name]["flops"] / avg_s / 1e12
+        # inside a whole step the pruning rides on the scoring's pass (no call of its own): the bytes are the tail's
+        key = "tail" if name == "score" and per_class.get("prune", (0.0, 0))[1] == 0 else name
+        if key == "tail":
+            row["what"] = "kb_prune + kb_score_select fused (the tail of the step): algorithmic bytes 24 R + 16 R S"
+        if key in alg:
+            gbs = alg[key]["bytes"] / avg_s / 1e9
+            tfl = alg[key]["flops"] / avg_s / 1e12
             row.update(GBps=gbs, hbm_frac=gbs / hbm, TFLOPs=tfl)
-            hbm_time = alg[name]["bytes"] / (hbm * 1e9)
+            hbm_time = alg[key]["bytes"] / (hbm * 1e9)
             if name == "assign" and assign_path in (2, 3):
-                row.update(bound="tensor", frac=tfl / tensor_peak, frac_of_mma_issue_peak=tfl / mma_issue_peak)
+                row.update(bound="tensor", frac=tfl / tensor_peak, frac_of_burst_peak=tfl / tensor_peak_burst,
+                           frac_of_mma_issue_peak=tfl / mma_issue_peak)
             elif name in ("assign", "fit") and alg[name]["flops"] / (ffma_peak * 1e12) > hbm_time:
                 row.update(bound="alu", frac=tfl / ffma_peak)
             else:
@@ -321,13 +334,15 @@ def call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms):
         tfl = alg["assign"]["flops"] / k_s / 1e12
         out["assign_kernel"] = {"calls": int(kcalls), "avg_us": k_s * 1e6, "share": kms / max(breakdown_ms, 1e-9),
                                 "TFLOPs": tfl, "bound": "tensor", "frac": tfl / tensor_peak,
+                                "frac_of_burst_peak": tfl / tensor_peak_burst,
                                 "frac_of_mma_issue_peak": tfl / mma_issue_peak}
-    return out, {"tensor_fp32_equiv_tflops": tensor_peak, "mma_issue_fp32_equiv_tflops": mma_issue_peak,
+    return out, {"tensor_fp32_equiv_tflops": tensor_peak, "tensor_peak_is": "sustained" if sustained else "burst",
+                 "mma_issue_fp32_equiv_tflops": mma_issue_peak,
                  "ffma_tflops": ffma_peak, "hbm_gbs": hbm}
 
 
 def measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, steps, warmup, min_seconds, flush, barrier,
-                     reduce_first=lambda v: v):
+                     reduce_first=lambda v: v, sampler=None):
     """Device-resident timing of one workload: `warmup` untimed steps, then loops of exactly `steps` steps, each
     step between its own pair of CUDA events with an L2 flush before it, repeated until `min_seconds` of timed
     steps have run (the warm-up-then-at-least-a-second, report-the-median protocol); then one more pass of
@@ -344,6 +359,8 @@ def measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, steps, warm
         flush.zero_()
         ctx.bandit_step(dims, params, dev_t)
     barrier()
+    if sampler is not None:
+        sampler.start()
     k0, m0 = ctx.launch_count()
     per_step = []
 
@@ -376,9 +393,15 @@ def measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, steps, warm
     breakdown_ms = sum(a.elapsed_time(b) for a, b in ev2)
     per_class = ctx.timing_read()
     ctx.timing_enable(False)
+    clocks = sampler.stop() if sampler is not None else None
+    sustained = bool(clocks and "sw_power_cap" in clocks.get("reasons", []) and sum(per_step) * 1e-3 >= 1.0)
     status = ctx.device_status()
-    assign_path, presplit = ctx.assign_path(), ctx.assign_presplit()
-    calls, denominators = call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms)
+    # which assign kernel this workload ran: the tensor-core kernel has its own event pairs; without them the
+    # context's "last path" is left over from an earlier workload (the fused and cooperative fits never set it)
+    tensor_ran = per_class.get("assign_kernel", (0.0, 0))[1] > 0
+    assign_path = ctx.assign_path() if tensor_ran else 1
+    presplit = ctx.assign_presplit() if tensor_ran else 0
+    calls, denominators = call_fractions(cfg, per_class, peaks, probe, assign_path, breakdown_ms, sustained)
     # the library's own count of near-ties of the final assignment on the tensor path: rows whose runner-up lay within
     # the re-evaluation bound and were settled exactly (two-candidate compare, full re-evaluation)
     near = None
@@ -392,13 +415,13 @@ def measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, steps, warm
     st = median_stats(per_step)
     return {"dims": dims, "params": params, "dev_t": dev_t, "stats": st, "launches": int(k1 - k0), "memsets": int(m1 - m0),
             "calls": calls, "denominators": denominators, "status": int(status), "assign_path": int(assign_path),
-            "presplit": int(presplit), "breakdown_ms_per_step": breakdown_ms / steps, "near": near}
+            "presplit": int(presplit), "breakdown_ms_per_step": breakdown_ms / steps, "near": near, "clocks": clocks}
 
 
 def workload_summary(cfg, m, world):
     """What the line carries for a workload beside the headline one."""
     st = m["stats"]
-    keep = ("avg_us", "calls", "share", "bound", "frac", "frac_of_mma_issue_peak", "GBps", "TFLOPs")
+    keep = ("avg_us", "calls", "share", "bound", "frac", "frac_of_burst_peak", "frac_of_mma_issue_peak", "GBps", "TFLOPs", "what")
     return {"config": {k: v for k, v in workload_config(cfg).items() if k in ("B", "N", "D", "K", "S", "iters", "arms")},
             "ms_per_step": st["median"], "ms_min": st["min"], "ms_max": st["max"], "timed_steps": st["steps"],
             "timed_seconds": st["seconds"], "arms_per_s": job_value(world, cfg.arms, st["median"]),
@@ -423,13 +446,15 @@ def dominant_roofline(cfg, m, peaks):
                 "frac": ak["frac"], "traffic": None,
                 "kernel": f"assign_tc_kernel (tcgen05 {split}), the contraction kernel of kb_cluster_assign",
                 "kernel_avg_us": ak["avg_us"], "kernel_launches": ak["calls"],
-                "frac_of_mma_issue_peak": ak["frac_of_mma_issue_peak"],
+                "frac_of_burst_peak": ak["frac_of_burst_peak"], "frac_of_mma_issue_peak": ak["frac_of_mma_issue_peak"],
                 "whole_call": {"avg_us": dk["avg_us"], "TFLOPs": dk["TFLOPs"], "frac": dk["frac"],
                                "what": "preparation + contraction + fix-up kernels of one kb_cluster_assign; the "
                                        "once-per-fit conversion of Z to its fp16 image is its own class (prep)"},
-                "peak_source": f"{peaks['source']} bf16 GEMM peak" + (" x 0.5 (tf32)" if m["assign_path"] == 3 else "") +
-                               " / 3 (split products), fp32-equivalent; frac_of_mma_issue_peak divides by the "
-                               "tcgen05.mma issue rate measured in this run / 3",
+                "peak_source": f"{peaks['source']} bf16 GEMM peak, the {den['tensor_peak_is']} figure (sustained when the "
+                               "timed loop ran a second or more with sw_power_cap active, else burst)" +
+                               (" x 0.5 (tf32)" if m["assign_path"] == 3 else "") +
+                               " / 3 (split products), fp32-equivalent; frac_of_burst_peak divides by the burst figure / 3, "
+                               "frac_of_mma_issue_peak by the tcgen05.mma issue rate measured in this run / 3",
                 "algorithmic_flops_per_launch": alg["assign"]["flops"],
                 "executed_tensor_TFLOPs": 3.0 * ak["TFLOPs"],
                 "a_operand": ("pre-split fp16 image of Z, made once per fit (class prep)") if m["presplit"]
@@ -450,7 +475,7 @@ def dominant_roofline(cfg, m, peaks):
     if cap is not None:
         roof["traffic"] = cap["bytes"]
         roof["traffic_source"] = cap["source"]
-    roof["calls"] = {n: {k: calls[n][k] for k in ("bound", "frac", "avg_us", "calls") if k in calls[n]}
+    roof["calls"] = {n: {k: calls[n][k] for k in ("bound", "frac", "avg_us", "calls", "what") if k in calls[n]}
                      for n in ("assign", "update", "score", "prune", "normalize", "fit") if n in calls}
     return roof
 
@@ -488,11 +513,9 @@ def run_ours(args, cfg):
 
     # ---- the headline workload: device-resident timing ------------------------------------
     inp = wl.make_inputs(cfg, seed=replica_seed(cfg, rank))
-    sampler = ClockSampler(local, gpu_uuid)
-    sampler.start()
     m = measure_workload(ctx, kb, torch, cfg, inp, device, peaks, probe, args.steps, args.warmup, args.min_seconds,
-                         flush, barrier, lambda v: reduce_max(v, dist, device))
-    clocks = sampler.stop()
+                         flush, barrier, lambda v: reduce_max(v, dist, device), ClockSampler(local, gpu_uuid))
+    clocks = m["clocks"]
     dims, params, dev_t = m["dims"], m["params"], m["dev_t"]
     R = wl.R_RESOURCES
 

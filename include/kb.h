@@ -534,6 +534,21 @@ typedef struct {
  * of kb_prune and kb_score_select). */
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
 
+/* The tail of the step alone: kb_prune (both masks and, when `bound` is given,
+ * the gain bound) followed by kb_score_select, from labels and dist2 that the
+ * CALLER provides (here `labels` and `dist2` of kb_step_args are INPUTS), with
+ * the results those two calls give.  Reads B, N, K, S, R, theta_sat, score, the
+ * pruning and scoring inputs, and writes keep, kept_count, bound (nullable),
+ * the three cluster tables, arm_index (nullable) and the two selections; x,
+ * init_rows, z, centroids, counts, inertia, rep, D and iters are ignored.
+ * S in {4, 8, 16, 32} with 16-byte aligned per-arm arrays runs fused: the
+ * pruning rides on the pass that gathers the cluster statistics, so a
+ * candidate's label and keep word are touched once (Sec. 5's batched setting
+ * scores millions of arms per step); three launches, or one for instances of
+ * at most 1024 candidates.  Other shapes run the two calls one after the other.
+ * Device pointers; needs the workspace of kb_workspace_bytes. */
+kb_status kb_bandit_step_tail(kb_ctx* ctx, const kb_step_args* args);
+
 /* The same step for a caller whose data lives in HOST memory: copies the
  * inputs to the device, runs the calls of kb_bandit_step, copies the requested
  * outputs back and synchronises the stream before returning.  The inputs that

@@ -533,12 +533,23 @@ kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* a) {
     return step_tail(ctx, a);
 }
 
+kb_status kb_bandit_step_tail(kb_ctx* ctx, const kb_step_args* a) {
+    if (!ctx || !a) return KB_ERR_INVALID_ARG;
+    KB_COMMON(ctx, a->B, a->N);
+    return step_tail(ctx, a);
+}
+
 // bound_done: a->bound already holds the gain bound (it does not depend on the clustering): only the keep bits are due
 static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a, bool bound_done) {
     if (kb_step_tail_small_eligible(ctx, a)) {
         // at most 1024 candidates per instance: one CTA prunes, scores and selects for its instance
         TimeScope ts__(ctx, KB_T_SCORE);
         return kb_launch_step_tail_small(ctx, a, bound_done);
+    }
+    if (kb_step_tail_fused_eligible(ctx, a)) {
+        // larger instances: the pruning rides on the statistics pass (three launches, labels and keep touched once)
+        TimeScope ts__(ctx, KB_T_SCORE);
+        return kb_launch_step_tail_fused(ctx, a, bound_done);
     }
     kb_status s = kb_prune(ctx, a->B, a->N, a->S, a->K, a->R, a->flops, a->bytes, a->peak_flops, a->peak_bw, a->t_incumbent,
                  a->t_cur, a->labels, a->hsig, a->target, a->theta_sat, a->keep, a->kept_count,

@@ -103,6 +103,8 @@ kb_status kb_launch_score_small(kb_ctx* ctx, int B, int N, int K, int S, kb_scor
                                 const float* bound, const int32_t* t, float* cl_pulls, float* cl_mean, float* cl_index,
                                 float* arm_index, int32_t* best_arm, float* best_val, int32_t* best_cluster_arm);
 kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* a, bool bound_done = false);
+bool kb_step_tail_fused_eligible(const kb_ctx* ctx, const kb_step_args* a);
+kb_status kb_launch_step_tail_fused(kb_ctx* ctx, const kb_step_args* a, bool bound_done = false);
 kb_status kb_zsplit_prepare(kb_ctx* ctx, char* img, int B, int N, int D, int K, const float* z);
 void kb_zsplit_forget(kb_ctx* ctx);
 bool kb_assign_tc_supported(const kb_ctx* ctx, int B, int D, int K);

@@ -60,7 +60,8 @@ constexpr uint32_t PM_IDESC_TF32 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32
 constexpr uint32_t PM_WAIT_LIMIT = 1u << 24;                // polls of the one bounded wait (well under a second)
 constexpr int PM_SMEM = 16 * 1024 + 1024;                   // one B tile (128 rows x 128 bytes) + alignment slack
 
-// tf32 != 0: kind::tf32, else kind::f16.  Two accumulators are used alternately, as the assign kernel does.
+// tf32 != 0: kind::tf32, else kind::f16.  Two accumulators take turns, 32 products each (the first of a run
+// overwrites), as the assign kernel's tiles do.
 __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, int* __restrict__ fail) {
     extern __shared__ unsigned char pm_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)pm_raw + 1023) & ~(uintptr_t)1023);
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, 
         const uint64_t bdesc = pr_desc_sw128(pr_smem_u32(smem));
         for (int i = 0; i < iters; ++i) {
             const uint32_t koff = (uint32_t)(i & 3) * 2u;              // 32-byte k-step inside the swizzled row
-            const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
+            const uint32_t d = tmem + (uint32_t)((i >> 5) & 1) * 128u;     // 32 products per accumulator, then the other
             const uint32_t a_t = tmem + 256u + (uint32_t)(i & 15) * 8u;
             uint32_t elected;
             asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(elected));
@@ -98,13 +99,13 @@ __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, 
                     asm volatile(
                         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                         "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a_t),
-                        "l"(bdesc + koff), "r"(PM_IDESC_TF32), "r"(i >> 1)
+                        "l"(bdesc + koff), "r"(PM_IDESC_TF32), "r"(i & 31)
                         : "memory");
                 } else {
                     asm volatile(
                         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a_t),
-                        "l"(bdesc + koff), "r"(PM_IDESC_F16), "r"(i >> 1)
+                        "l"(bdesc + koff), "r"(PM_IDESC_F16), "r"(i & 31)
                         : "memory");
                 }
             }

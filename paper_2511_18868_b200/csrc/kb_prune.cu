@@ -5,11 +5,12 @@
 //
 // Vector path (S in {4, 8, 16, 32}): a thread owns four strategies of a row, so the
 // bound leaves as float4 stores and the keep bits of a row are OR-ed across its
-// S/4 lanes with shuffles.  The kernel is bound by its divisions (three per arm), not by memory:
-// a quotient whose divisor is fixed per thread is formed from the divisor's reciprocal and one
-// fused residual correction, which gives the correctly rounded fp32 quotient for ordinary operands
-// in three operations, so an arm whose floor equals the incumbent exactly is still pruned
-// (strict <), as the definition says.
+// S/4 lanes with shuffles.  Divisions would bind the kernel (three per arm), so a quotient whose
+// divisor is fixed per thread is the product with the divisor's reciprocal; only where that leaves
+// the floor within a few roundings of the incumbent is it redone with one fused residual correction,
+// which gives the correctly rounded fp32 quotient for ordinary operands, so an arm whose floor
+// equals the incumbent exactly is still pruned (strict <), as the definition says.  The bound is
+// 1 - T_lb / T_k by one saturating multiply-add (absolute error below 3e-7).
 // Generic path (any S <= 32): one thread per candidate, bound rows staged through
 // shared memory so that they still leave the SM as full lines.
 #include "kb_internal.cuh"
@@ -87,13 +88,15 @@ prune_vec_kernel(int N, int S, int K, int R, int G, const float* __restrict__ fl
             const float rT = 1.f / Tk[u];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float tlb = fmaxf(kb_div_by(F[u], P[k], rP[k]), kb_div_by(Q[u], W[k], rW[k]));
+                // quotients by the reciprocal; where that leaves the floor within a few roundings of the incumbent
+                // the decision is taken on the correctly rounded quotients (strict <: equality prunes)
+                float tlb = fmaxf(F[u] * rP[k], Q[u] * rW[k]);
+                if (fabsf(tlb - tinc) <= 2e-6f * tinc)
+                    tlb = fmaxf(kb_div_by(F[u], P[k], rP[k]), kb_div_by(Q[u], W[k], rW[k]));
                 bool ok = tlb < tinc;
                 if (sat) ok = ok && (__ldg(h + tg[k]) < theta);
                 if (ok) bits |= 1u << (4 * q + k);
-                float v = kb_div_by(Tk[u] - tlb, Tk[u], rT);
-                v = v > 0.f ? v : 0.f;       // also maps NaN (0/0) to 0, as the definition does
-                g[k] = v < 1.f ? v : 1.f;
+                g[k] = __saturatef(fmaf(-tlb, rT, 1.f));     // clip(1 - T_lb / T_k, 0, 1); NaN (0/0) -> 0, as the definition does
             }
             for (int o = 1; o < vps; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
             if (live && q == 0) { keep[i] = bits; count += __popc(bits); }

@@ -25,7 +25,7 @@ EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_clear_device_status", "kb_status_of_device_word", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_probe_peaks", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
-           "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_step_workspace_bytes",
+           "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_bandit_step_tail", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc", "kb_cluster_update_noalloc_status"]
 
 
@@ -112,6 +112,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
     lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
+    lib.kb_bandit_step_tail.argtypes = [_VP, ctypes.POINTER(StepArgs)]
     lib.kb_step_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(sz)]
     lib.kb_bandit_step_host.argtypes = [_VP, ctypes.POINTER(StepArgs)]
     for name in EXPORTS:
@@ -379,6 +380,11 @@ class KB:
         """Whole step on device tensors (dict keyed by the field names of kb_step_args)."""
         a = self._step_args(dims, params, tensors, host=False)
         self._check(self.lib.kb_bandit_step(self.h, ctypes.byref(a)), "kb_bandit_step")
+
+    def bandit_step_tail(self, dims, params, tensors):
+        """kb_bandit_step_tail: prune + score + select from the caller's labels and dist2 (device tensors)."""
+        a = self._step_args(dims, params, tensors, host=False)
+        self._check(self.lib.kb_bandit_step_tail(self.h, ctypes.byref(a)), "kb_bandit_step_tail")
 
     def bandit_step_host(self, dims, params, tensors):
         """Whole step on HOST tensors (ideally pinned); returns after the results are in host memory."""

@@ -254,6 +254,113 @@ def test_score_all_masked_and_unplayed(kbx):
     assert np.all(np.isneginf(got["arm_index"]))
 
 
+# ------------------------------------------------- prune + score in one pass
+def run_tail(kbx, inp, labels, dist2, K, want_bound=True, want_arm_index=True, **prm):
+    """kb_bandit_step_tail on the caller's labels / dist2: returns the host copies of everything it writes."""
+    B, N, S = inp["pulls"].shape
+    ws(kbx, B, N, 1, K, S)
+    t = {"flops": dev(inp["flops"]), "bytes": dev(inp["bytes"]), "peak_flops": dev(inp["peak_flops"]),
+         "peak_bw": dev(inp["peak_bw"]), "t_incumbent": dev(inp["t_inc"]), "t_cur": dev(inp["t_cur"]),
+         "hsig": dev(inp["hsig"]), "target": dev(inp["target"]), "pulls": dev(inp["pulls"]),
+         "reward_sum": dev(inp["reward_sum"]), "t": dev(inp["t"]), "labels": dev(labels), "dist2": dev(dist2),
+         "keep": empty((B, N), torch.int32), "kept_count": empty((B,), torch.int32),
+         "cl_pulls": empty((B, K, S)), "cl_mean": empty((B, K, S)), "cl_index": empty((B, K, S)),
+         "best_arm": empty((B,), torch.int32), "best_val": empty((B,)), "best_cluster_arm": empty((B,), torch.int32)}
+    if want_bound:
+        t["bound"] = empty((B, N, S))
+    if want_arm_index:
+        t["arm_index"] = empty((B, N, S))
+    dims = dict(B=B, N=N, D=1, K=K, S=S, R=inp["hsig"].shape[2], iters=0)
+    params = dict(theta_sat=75.0, c=2.0, prior_pulls=1.0, prior_mean=0.5)
+    params.update(prm)
+    kbx.bandit_step_tail(dims, params, t)
+    outs = ["keep", "kept_count", "bound", "cl_pulls", "cl_mean", "cl_index", "arm_index", "best_arm", "best_val",
+            "best_cluster_arm"]
+    return {k: host(t[k]) for k in outs if k in t}
+
+
+@pytest.mark.parametrize("B,N,K,S,L,cap", [(1, 5000, 64, 32, 0.1, False), (2, 3001, 7, 8, 0.0, False),
+                                           (1, 20011, 1024, 8, 0.1, True), (3, 1500, 256, 16, 0.3, False),
+                                           (1, 1025, 3, 4, 0.0, True), (2, 40000, 130, 32, 0.1, False),
+                                           (1, 300, 5, 8, 0.1, False), (2, 2000, 9, 13, 0.1, False)])
+def test_step_tail_matches_prune_then_score(kbx, B, N, K, S, L, cap):
+    """The fused tail (pruning on the statistics' pass) against the oracle's kb_prune followed by its
+    kb_score_select, teacher-forced on the same labels and distances: keep bits exact outside the near-tie
+    margin, kept_count = their population count, bound, the three cluster tables and the per-arm index
+    element by element, both selections.  (S = 13 and N <= 1024 take the unfused / one-CTA forms: same rule.)"""
+    cfg = wl.scaled(wl.CONFIGS["tiny"], B=B, N=N, S=S, K=K)
+    inp = wl.make_inputs(cfg, seed=N + K)
+    rng = np.random.default_rng(N * 7 + S)
+    labels = rng.integers(0, max(1, K - 1), (B, N)).astype(np.int32)        # the last cluster stays empty
+    dist2 = rng.uniform(0, 4, (B, N)).astype(np.float32)
+    # some floors within a few ulp of the incumbent, on both sides, and a few exactly on it
+    f = inp["flops"]
+    tl = inp["t_inc"][:, None].astype(np.float64) * inp["peak_flops"][0].astype(np.float64)
+    idx = rng.choice(N, min(N, 200), replace=False)
+    f[:, idx] = (tl * (1 + rng.integers(-3, 4, (B, idx.size)) * 6e-8)).astype(np.float32)
+    inp["bytes"][:, idx] = 1.0
+    prm = dict(lipschitz_L=L, cap_with_bound=cap)
+    got = run_tail(kbx, inp, labels, dist2, K, **prm)
+    assert kbx.device_status() == 0
+    p = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
+                     labels, inp["hsig"], inp["target"], 75.0, want_bound=True, want_margin=True)
+    keep = got["keep"].view(np.uint32)
+    ties = parity.keep_match(keep, p, S)
+    assert int(got["kept_count"].view(np.uint32).astype(np.int64).sum()) == int(np.bitwise_count(keep).sum())
+    assert np.array_equal(got["kept_count"].view(np.uint32), np.bitwise_count(keep).sum(axis=1).astype(np.uint32))
+    parity.close(got["bound"], p["bound"], atol=1e-6, what="bound")
+    s = oracle.score_select(labels, dist2, inp["pulls"], inp["reward_sum"], inp["t"], K, keep=keep,
+                            bound=p["bound"] if cap else None, c=2.0, lipschitz_L=L, cap_with_bound=cap)
+    assert np.array_equal(got["cl_pulls"], s["cl_pulls"])
+    parity.close(got["cl_mean"], s["cl_mean"], atol=1e-6, what="cl_mean")
+    parity.close(got["cl_index"], s["cl_index"], atol=1e-6, what="cl_index")
+    if cap:
+        # the cap is the GPU's own bound (within 1e-6 of the oracle's): compare against the oracle run on it
+        s = oracle.score_select(labels, dist2, inp["pulls"], inp["reward_sum"], inp["t"], K, keep=keep,
+                                bound=got["bound"], c=2.0, lipschitz_L=L, cap_with_bound=True)
+    parity.close(got["arm_index"], s["arm_index"], atol=1e-6, what="arm_index")
+    parity.select_match(got["best_arm"], got["best_val"], s, s["arm_index"])
+    parity.cluster_select_match(got["best_cluster_arm"], s, s["cl_index"])
+    # the optional outputs left out: same selections
+    slim = run_tail(kbx, inp, labels, dist2, K, want_bound=cap, want_arm_index=False, **prm)
+    assert np.array_equal(slim["keep"], got["keep"]) and np.array_equal(slim["best_cluster_arm"], got["best_cluster_arm"])
+    parity.select_match(slim["best_arm"], slim["best_val"], s, s["arm_index"])
+    print(f"[tail B={B} N={N} K={K} S={S}] keep-bit near-ties {ties}")
+
+
+def test_step_tail_threshold_edges_and_bad_labels(kbx):
+    """Strictness survives the fused arithmetic: a floor EQUAL to the incumbent is pruned, h == theta is pruned;
+    a label outside [0, K) raises status bit 1, adds to no statistic and is pruned as cluster 0 would be."""
+    N, K, S = 2048, 4, 4
+    flops = np.full((1, N), 1e9, np.float32)
+    flops[0, 1::2] = 2e9
+    byts = np.ones((1, N), np.float32)
+    pf, pb = np.full(S, 1e12, np.float32), np.full(S, 1e12, np.float32)
+    tinc = np.array([np.float32(2e9) / np.float32(1e12)], np.float32)       # exactly the floor of the odd candidates
+    hs = np.zeros((1, K, 3), np.float32)
+    hs[0, 1, 0] = 75.0                                                      # cluster 1, resource 0: exactly theta
+    hs[0, 2, 0] = np.nextafter(np.float32(75.0), np.float32(0))             # cluster 2: one ulp below
+    labels = (np.arange(N) % 3).astype(np.int32)[None].copy()
+    inp = dict(flops=flops, bytes=byts, peak_flops=pf, peak_bw=pb, t_inc=tinc, t_cur=np.full((1, N), 1.0, np.float32),
+               hsig=hs, target=np.zeros(S, np.int32), pulls=np.ones((1, N, S), np.int32),
+               reward_sum=np.full((1, N, S), 0.5, np.float32), t=np.array([1 + N * S], np.int32))
+    got = run_tail(kbx, inp, labels, np.zeros((1, N), np.float32), K)
+    keep = got["keep"].view(np.uint32)[0]
+    want = np.where((np.arange(N) % 2 == 0) & (labels[0] != 1), 0xF, 0).astype(np.uint32)
+    assert np.array_equal(keep, want)
+    assert kbx.device_status() == 0
+    bad = labels.copy()
+    bad[0, 10], bad[0, 11] = K, -1
+    got = run_tail(kbx, inp, bad, np.zeros((1, N), np.float32), K)
+    assert kbx.device_status(raise_on_timeout=False) & 1
+    kbx.clear_device_status()
+    ok = np.ones(N, bool)
+    ok[[10, 11]] = False
+    ref = oracle.score_select(bad[:, ok], None, inp["pulls"][:, ok], inp["reward_sum"][:, ok], inp["t"], K)
+    assert np.array_equal(got["cl_pulls"], ref["cl_pulls"])
+    assert kbx.device_status() == 0
+
+
 # ------------------------------------------------------------- whole step
 STEP_CASES = {
     "tiny": wl.CONFIGS["tiny"],
@@ -365,8 +472,13 @@ def test_step_free_running(kbx, name, host_buffers):
     p_chk = oracle.prune(inp["flops"], inp["bytes"], inp["peak_flops"], inp["peak_bw"], inp["t_inc"], inp["t_cur"],
                          got["labels"], inp["hsig"], inp["target"], 75.0, want_bound=True, want_margin=True)
     parity.keep_match(got["keep"].view(np.uint32), p_chk, cfg.S)
+    parity.close(got["bound"], p_chk["bound"], atol=1e-6, what="bound")
+    assert np.array_equal(got["kept_count"].view(np.uint32),
+                          np.bitwise_count(got["keep"].view(np.uint32)).sum(axis=1).astype(np.uint32))
     s_chk = oracle.score_select(got["labels"], got["dist2"], inp["pulls"], inp["reward_sum"], inp["t"], cfg.K,
                                 keep=got["keep"].view(np.uint32), c=2.0, lipschitz_L=float(inp["lipschitz_L"]))
+    assert np.array_equal(got["cl_pulls"], s_chk["cl_pulls"])
+    parity.close(got["cl_mean"], s_chk["cl_mean"], atol=1e-6, what="cl_mean")
     parity.close(got["cl_index"], s_chk["cl_index"], atol=1e-6, what="cl_index")
     parity.close(got["arm_index"], s_chk["arm_index"], atol=1e-6, what="arm_index")
     parity.select_match(got["best_arm"], got["best_val"], s_chk, s_chk["arm_index"])
