@@ -150,6 +150,9 @@ kb_status kb_timing_read(kb_ctx* ctx, double* ms, int64_t* calls);
 typedef struct {
     double ffma_tflops, mma_f16_tflops, mma_tf32_tflops; /* 2 flop per multiply-add */
     float ffma_ms, mma_f16_ms, mma_tf32_ms;              /* duration of the timed launch */
+    /* one SM's view of its own stream of products: SM cycles per instruction, and the SM clock it ran at
+     * (cycles / nanoseconds of the global timer) -- the power cap lowers the clock under tensor load */
+    float mma_f16_cycles_per_instr, mma_tf32_cycles_per_instr, mma_f16_sm_mhz, mma_tf32_sm_mhz;
 } kb_peak_probe;
 kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out);
 

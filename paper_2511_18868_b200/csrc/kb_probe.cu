@@ -62,7 +62,8 @@ constexpr int PM_SMEM = 16 * 1024 + 1024;                   // one B tile (128 r
 
 // tf32 != 0: kind::tf32, else kind::f16.  Two accumulators take turns, 32 products each (the first of a run
 // overwrites), as the assign kernel's tiles do.
-__global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, int* __restrict__ fail) {
+__global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, int* __restrict__ fail,
+                                                           long long* __restrict__ stamps) {
     extern __shared__ unsigned char pm_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)pm_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar;
@@ -88,6 +89,9 @@ __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, 
         // one elected lane of a converged warp issues, as in the assign kernel (a lone thread inside a divergent
         // branch issues measurably slower)
         const uint64_t bdesc = pr_desc_sw128(pr_smem_u32(smem));
+        const long long c0 = clock64();
+        unsigned long long n0;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(n0));
         for (int i = 0; i < iters; ++i) {
             const uint32_t koff = (uint32_t)(i & 3) * 2u;              // 32-byte k-step inside the swizzled row
             const uint32_t d = tmem + (uint32_t)((i >> 5) & 1) * 128u;     // 32 products per accumulator, then the other
@@ -117,6 +121,12 @@ __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, 
             bool ok = false;
             for (uint32_t i = 0; i < PM_WAIT_LIMIT && !ok; ++i) ok = pr_mbar_try(pr_smem_u32(&bar), 0u);
             if (!ok) atomicAdd(fail, 1);                              // the products did not retire in time: no figure
+            if (blockIdx.x == 0) {                                    // SM cycles and nanoseconds of the whole stream
+                unsigned long long n1;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(n1));
+                stamps[0] = clock64() - c0;
+                stamps[1] = (long long)(n1 - n0);
+            }
         }
         __syncwarp();
     }
@@ -137,13 +147,15 @@ extern "C" kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out) {
     KB_CUDA(ctx, cudaEventCreate(&e0));
     KB_CUDA(ctx, cudaEventCreate(&e1));
     int* sink = ctx->dev_status + 16;                    // spare words behind the status word (256 bytes are owned)
+    long long* stamps = reinterpret_cast<long long*>(ctx->dev_status + 32);   // [kind][cycles, ns], 8-byte aligned
     cudaStream_t st = ctx->stream;
     kb_status s = KB_OK;
     auto elapsed = [&](float* ms) -> bool {
         return cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(ms, e0, e1) == cudaSuccess;
     };
     do {
-        if (cudaMemsetAsync(sink, 0, 2 * sizeof(int), st) != cudaSuccess) { s = KB_ERR_CUDA; break; }
+        if (cudaMemsetAsync(sink, 0, 2 * sizeof(int), st) != cudaSuccess ||
+            cudaMemsetAsync(stamps, 0, 4 * sizeof(long long), st) != cudaSuccess) { s = KB_ERR_CUDA; break; }
         // ---- fp32 FMA: warm-up launch, then the timed one
         const int ff_iters = 4096, ff_grid = ctx->sm_count * FF_CTAS_PER_SM;
         float ms = 0.f;
@@ -165,7 +177,7 @@ extern "C" kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out) {
         for (int tf32 = 0; tf32 < 2 && s == KB_OK; ++tf32) {
             for (int rep = 0; rep < 2; ++rep) {
                 cudaEventRecord(e0, st);
-                probe_mma_kernel<<<ctx->sm_count, 128, PM_SMEM, st>>>(tf32, mm_iters, sink + 1);
+                probe_mma_kernel<<<ctx->sm_count, 128, PM_SMEM, st>>>(tf32, mm_iters, sink + 1, stamps + 2 * tf32);
                 cudaEventRecord(e1, st);
                 if (cudaGetLastError() != cudaSuccess || !elapsed(&ms)) { s = KB_ERR_CUDA; break; }
             }
@@ -176,8 +188,14 @@ extern "C" kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out) {
         }
         if (s != KB_OK) break;
         int host[2] = {0, 0};
+        long long hst[4] = {0, 0, 0, 0};
         if (cudaMemcpyAsync(host, sink, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaMemcpyAsync(hst, stamps, sizeof(hst), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
             cudaStreamSynchronize(st) != cudaSuccess) { s = KB_ERR_CUDA; break; }
+        out->mma_f16_cycles_per_instr = (float)((double)hst[0] / mm_iters);
+        out->mma_tf32_cycles_per_instr = (float)((double)hst[2] / mm_iters);
+        out->mma_f16_sm_mhz = hst[1] > 0 ? (float)((double)hst[0] / (double)hst[1] * 1e3) : 0.f;
+        out->mma_tf32_sm_mhz = hst[3] > 0 ? (float)((double)hst[2] / (double)hst[3] * 1e3) : 0.f;
         if (host[1] != 0) s = kb_fail(ctx, KB_ERR_TIMEOUT, "kb_probe_peaks: %d CTAs did not see their products retire", host[1]);
     } while (0);
     if (s == KB_ERR_CUDA) kb_fail(ctx, KB_ERR_CUDA, "kb_probe_peaks: %s", cudaGetErrorString(cudaGetLastError()));

@@ -34,7 +34,9 @@ TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fi
 
 class PeakProbe(ctypes.Structure):
     _fields_ = [("ffma_tflops", ctypes.c_double), ("mma_f16_tflops", ctypes.c_double), ("mma_tf32_tflops", ctypes.c_double),
-                ("ffma_ms", ctypes.c_float), ("mma_f16_ms", ctypes.c_float), ("mma_tf32_ms", ctypes.c_float)]
+                ("ffma_ms", ctypes.c_float), ("mma_f16_ms", ctypes.c_float), ("mma_tf32_ms", ctypes.c_float),
+                ("mma_f16_cycles_per_instr", ctypes.c_float), ("mma_tf32_cycles_per_instr", ctypes.c_float),
+                ("mma_f16_sm_mhz", ctypes.c_float), ("mma_tf32_sm_mhz", ctypes.c_float)]
 
 
 class KbError(RuntimeError):
