@@ -262,6 +262,51 @@ def update_pair(pair, reward, cl_pulls, cl_mean):
     return cl_pulls, cl_mean
 
 
+def append_candidate(state, parent, x_new, t_new, verified=None, flops_new=None, bytes_new=None, h_new=None):
+    """Frontier growth (see kbo_append_candidate).  `state`: dict of the capacity-padded arrays n_active [B], x [B,Ncap,D],
+    t_cur [B,Ncap], labels [B,Ncap], pulls / reward_sum [B,Ncap,S] and optionally flops, bytes [B,Ncap], h_cand [B,Ncap,R],
+    dist2 [B,Ncap], t_inc [B].  Returns (new state, appended [B], full [B]); the input is not modified."""
+    st = {k: np.array(v, copy=True, order="C") for k, v in state.items()}
+    B, Ncap, D = st["x"].shape
+    S = st["pulls"].shape[2]
+    R = st["h_cand"].shape[2] if "h_cand" in st else 1
+    f32 = lambda a: None if a is None else _f32(a)
+    parent, x_new, t_new = _i32(parent), _f32(x_new), _f32(t_new)
+    verified = None if verified is None else _i32(verified)
+    flops_new, bytes_new, h_new = f32(flops_new), f32(bytes_new), f32(h_new)
+    appended = np.empty((B,), np.int32)
+    full = np.empty((B,), np.int32)
+    assert st["n_active"].dtype == np.int32 and st["labels"].dtype == np.int32 and st["pulls"].dtype == np.int32
+    for k in ("x", "t_cur", "reward_sum", "flops", "bytes", "h_cand", "dist2", "t_inc"):
+        assert k not in st or st[k].dtype == np.float32, k
+    _check(_load().kbo_append_candidate(B, Ncap, D, S, R, _p(verified), _p(parent), _p(x_new), _p(t_new), _p(flops_new),
+                                        _p(bytes_new), _p(h_new), _p(st["n_active"]), _p(st["x"]), _p(st["t_cur"]),
+                                        _p(st.get("flops")), _p(st.get("bytes")), _p(st.get("h_cand")), _p(st["labels"]),
+                                        _p(st.get("dist2")), _p(st["pulls"]), _p(st["reward_sum"]), _p(st.get("t_inc")),
+                                        _p(appended), _p(full)), "append_candidate")
+    return st, appended, full
+
+
+def recluster_due(t, n_active, tau, K):
+    """Algorithm 1's test `t mod tau = 0 and |P| >= 2K` per search: due [B] (see kbo_recluster_due)."""
+    t, n_active = _i32(t), _i32(n_active)
+    due = np.empty(t.shape, np.int32)
+    _check(_load().kbo_recluster_due(t.shape[0], int(tau), int(K), _p(t), _p(n_active), _p(due)), "recluster_due")
+    return due
+
+
+def signatures_from_reps(rep, h_cand, hsig_prev=None, run=None):
+    """hsig [B,K,R]: the signature of every cluster's representative, +inf for an empty cluster
+    (see kbo_signatures_from_reps); instances with run[b] == 0 keep hsig_prev."""
+    rep, h_cand = _i32(rep), _f32(h_cand)
+    B, K = rep.shape
+    N, R = h_cand.shape[1], h_cand.shape[2]
+    hsig = np.zeros((B, K, R), np.float32) if hsig_prev is None else np.array(hsig_prev, np.float32, copy=True, order="C")
+    run = None if run is None else _i32(run)
+    _check(_load().kbo_signatures_from_reps(B, N, K, R, _p(rep), _p(h_cand), _p(run), _p(hsig)), "signatures_from_reps")
+    return hsig
+
+
 def best_restart(inertia):
     """inertia [G][n_init] -> best [G]: the restart with the smallest inertia (see kbo_best_restart)."""
     x = _f32(inertia)

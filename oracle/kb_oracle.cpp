@@ -628,6 +628,83 @@ int kbo_update_pair(int B, int K, int S, const int32_t* pair, const float* rewar
 }
 
 // ---------------------------------------------------------------------------
+// The expanding frontier (Sec. 2.2: the action space A_t = P_t x S grows with the frontier; Algorithm 1:
+// "P <- {k_0}, C <- {P}" (one initial cluster), and inside "if Verify(k'_t)": "P <- P ∪ {k'_t}").
+//
+// The frontier of every search lives in arrays of a fixed capacity N_cap per instance, of which the first
+// n_active[b] rows are candidates; the rest is padding whose label is -1.
+//
+// kbo_append_candidate: where the new kernel k'_t passed verification (verified[b] != 0; null = all passed) it
+// becomes row j = n_active[b] of its instance:
+//     x[b][j] = x_new[b] (its raw features),  t_cur[b][j] = t_new[b] (its runtime T(k'_t)),
+//     flops / bytes / h_cand rows likewise (each array pair nullable together),
+//     pulls[b][j][.] = 0, reward_sum[b][j][.] = 0   (an arm nobody has played),
+//     labels[b][j] = labels[b][parent[b]], dist2[b][j] = dist2[b][parent[b]]
+//         (Reading: until the next re-clustering the new kernel sits in the cluster of the kernel k_t it was
+//          generated from -- Algorithm 1 re-partitions only every tau iterations, and a candidate outside
+//          every cluster could never be drawn),
+//     t_inc[b] = min(t_inc[b], t_new[b])   (the incumbent of Algorithm 1's return line, argmin T(k)),
+//     n_active[b] += 1;   appended[b] = j.
+// Nothing happens (appended[b] = -1) where verification failed, where nothing was drawn (parent[b] < 0), or
+// where the frontier is full (n_active[b] == N_cap; full[b] = 1 reports it).  parent[b] >= n_active[b] is an error.
+//
+// kbo_recluster_due: Algorithm 1's test "t mod tau = 0 and |P| >= 2K" per search.
+// ---------------------------------------------------------------------------
+int kbo_append_candidate(int B, int N_cap, int D, int S, int R, const int32_t* verified, const int32_t* parent,
+                         const float* x_new, const float* t_new, const float* flops_new, const float* bytes_new,
+                         const float* h_new, int32_t* n_active, float* x, float* t_cur, float* flops, float* bytes,
+                         float* h_cand, int32_t* labels, float* dist2, int32_t* pulls, float* reward_sum, float* t_inc,
+                         int32_t* appended, int32_t* full) {
+    for (int b = 0; b < B; ++b) {
+        if (appended) appended[b] = -1;
+        if (full) full[b] = 0;
+        const int p = parent[b];
+        if (p < 0) continue;
+        const int n = n_active[b];
+        if (n < 0 || n > N_cap || p >= n) return 2;
+        if (verified && verified[b] == 0) continue;
+        if (n == N_cap) { if (full) full[b] = 1; continue; }
+        for (int d = 0; d < D; ++d) x[ix3(b, n, d, N_cap, D)] = x_new[ix2(b, d, D)];
+        t_cur[ix2(b, n, N_cap)] = t_new[b];
+        if (flops && flops_new) flops[ix2(b, n, N_cap)] = flops_new[b];
+        if (bytes && bytes_new) bytes[ix2(b, n, N_cap)] = bytes_new[b];
+        if (h_cand && h_new)
+            for (int r = 0; r < R; ++r) h_cand[ix3(b, n, r, N_cap, R)] = h_new[ix2(b, r, R)];
+        for (int s = 0; s < S; ++s) { pulls[ix3(b, n, s, N_cap, S)] = 0; reward_sum[ix3(b, n, s, N_cap, S)] = 0.0f; }
+        labels[ix2(b, n, N_cap)] = labels[ix2(b, p, N_cap)];
+        if (dist2) dist2[ix2(b, n, N_cap)] = dist2[ix2(b, p, N_cap)];
+        if (t_inc && t_new[b] < t_inc[b]) t_inc[b] = t_new[b];
+        n_active[b] = n + 1;
+        if (appended) appended[b] = n;
+    }
+    return 0;
+}
+
+int kbo_recluster_due(int B, int tau, int K, const int32_t* t, const int32_t* n_active, int32_t* due) {
+    if (tau < 1) return 1;
+    for (int b = 0; b < B; ++b) due[b] = (t[b] % tau == 0 && n_active[b] >= 2 * K) ? 1 : 0;
+    return 0;
+}
+
+// The profile of every cluster's representative (Algorithm 1: "profile h_c^(i) <- NCU(k_c^(i))", with the
+// per-candidate signatures standing in for the profiler): hsig[b][i][:] = h_cand[b][rep[b][i]][:], and +inf for an
+// empty cluster (rep = -1), whose mask entry M_{i,s} = [h < theta_sat] is then 0: an empty cluster is never
+// selected.  run (nullable): instances with run[b] == 0 are left as they are.
+int kbo_signatures_from_reps(int B, int N, int K, int R, const int32_t* rep, const float* h_cand, const int32_t* run,
+                             float* hsig) {
+    for (int b = 0; b < B; ++b) {
+        if (run && run[b] == 0) continue;
+        for (int i = 0; i < K; ++i) {
+            const int k = rep[ix2(b, i, K)];
+            if (k >= N) return 2;
+            for (int r = 0; r < R; ++r)
+                hsig[ix3(b, i, r, K, R)] = k < 0 ? std::numeric_limits<float>::infinity() : h_cand[ix3(b, k, r, N, R)];
+        }
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
 // Restarts (the n_init of the "scikit-learn's KMeans" of Sec. 3.5): a search instance is clustered n_init
 // times from different seeds, as n_init consecutive instances of the batch; the run with the smallest
 // inertia is kept.  best[g] = the index in [0, n_init) of the smallest inertia[g][.], lowest index on ties;

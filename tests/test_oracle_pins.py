@@ -864,3 +864,124 @@ def test_best_restart_is_numpy_argmin():
     best = oracle.best_restart(inertia)
     assert np.all(inertia[np.arange(B), best] <= inertia[:, 0])
     assert len({tuple(r) for r in rows.reshape(B, n_init, K)[0].tolist()}) > 1
+
+
+# ------------------------------------------------------- the expanding frontier
+def _frontier_state(B, cap, D, S, R, rng):
+    """One initial kernel k_0 per search (Algorithm 1: P <- {k_0}, one initial cluster); padding rows carry label -1."""
+    st = {"n_active": np.ones(B, np.int32), "x": np.zeros((B, cap, D), np.float32),
+          "t_cur": np.zeros((B, cap), np.float32), "labels": np.full((B, cap), -1, np.int32),
+          "dist2": np.zeros((B, cap), np.float32), "pulls": np.zeros((B, cap, S), np.int32),
+          "reward_sum": np.zeros((B, cap, S), np.float32), "h_cand": np.zeros((B, cap, R), np.float32),
+          "flops": np.zeros((B, cap), np.float32), "bytes": np.zeros((B, cap), np.float32),
+          "t_inc": np.zeros(B, np.float32)}
+    st["x"][:, 0] = rng.standard_normal((B, D)).astype(np.float32)
+    st["t_cur"][:, 0] = rng.uniform(1.0, 2.0, B).astype(np.float32)
+    st["h_cand"][:, 0] = rng.uniform(0, 100, (B, R)).astype(np.float32)
+    st["flops"][:, 0], st["bytes"][:, 0] = 1e9, 1e8
+    st["labels"][:, 0] = 0
+    st["t_inc"][:] = st["t_cur"][:, 0]
+    return st
+
+
+def test_frontier_growth_and_trigger_against_algorithm1_with_python_lists():
+    """Algorithm 1's frontier as plain Python lists (P.append(k') inside `if Verify`, the test
+    `t % tau == 0 and len(P) >= 2 * K`), run beside the array form for the paper's own sizes
+    (T = 40, tau = 10, K = 3, |S| = 6, phi in R^5, one initial kernel) on three searches."""
+    T, tau, K, S, D, R, cap, B = 40, 10, 3, 6, 5, 3, 24, 3
+    rng = np.random.default_rng(7)
+    st = _frontier_state(B, cap, D, S, R, rng)
+    st["pulls"][:, 0] = rng.integers(0, 4, (B, S))                   # history of k_0 must survive every append
+    st["reward_sum"][:, 0] = rng.uniform(0, 1, (B, S)).astype(np.float32)
+    P = [[dict(phi=st["x"][b, 0].copy(), T=float(st["t_cur"][b, 0]), h=st["h_cand"][b, 0].copy(), cluster=0,
+               F=float(st["flops"][b, 0]), Q=float(st["bytes"][b, 0]), pulls=st["pulls"][b, 0].copy(),
+               rsum=st["reward_sum"][b, 0].copy(), d2=0.0)] for b in range(B)]
+    best = [P[b][0]["T"] for b in range(B)]
+    n_due = 0
+    for t in range(1, T + 1):
+        tt = np.full(B, t, np.int32)
+        # ---- the trigger
+        lit_due = [int(t % tau == 0 and len(P[b]) >= 2 * K) for b in range(B)]
+        assert list(oracle.recluster_due(tt, st["n_active"], tau, K)) == lit_due
+        for b in range(B):
+            if lit_due[b]:                                           # some re-partition: the growth rule only needs labels to change
+                n_due += 1
+                for j, k in enumerate(P[b]):
+                    k["cluster"] = (j * 7 + t) % K
+                    k["d2"] = float(np.float32(0.01 * j))
+                    st["labels"][b, j] = k["cluster"]
+                    st["dist2"][b, j] = k["d2"]
+        # ---- one generation per search: a parent among the active kernels, sometimes nothing drawn, sometimes rejected
+        parent = np.array([rng.integers(0, len(P[b])) if rng.uniform() > 0.1 else -1 for b in range(B)], np.int32)
+        verified = (rng.uniform(size=B) < 0.8).astype(np.int32)
+        x_new = rng.standard_normal((B, D)).astype(np.float32)
+        t_new = rng.uniform(0.3, 2.5, B).astype(np.float32)
+        f_new, q_new = rng.uniform(1e6, 1e9, B).astype(np.float32), rng.uniform(1e6, 1e9, B).astype(np.float32)
+        h_new = rng.uniform(0, 100, (B, R)).astype(np.float32)
+        want_row, want_full = [], []
+        for b in range(B):
+            ok = parent[b] >= 0 and verified[b] != 0
+            if ok and len(P[b]) < cap:
+                want_row.append(len(P[b]))
+                P[b].append(dict(phi=x_new[b].copy(), T=float(t_new[b]), h=h_new[b].copy(), cluster=P[b][parent[b]]["cluster"],
+                                 F=float(f_new[b]), Q=float(q_new[b]), pulls=np.zeros(S, np.int32),
+                                 rsum=np.zeros(S, np.float32), d2=P[b][parent[b]]["d2"]))
+                best[b] = min(best[b], float(t_new[b]))
+                want_full.append(0)
+            else:
+                want_row.append(-1)
+                want_full.append(int(ok))
+        st, row, full = oracle.append_candidate(st, parent, x_new, t_new, verified, f_new, q_new, h_new)
+        assert list(row) == want_row and list(full) == want_full
+        # ---- the arrays are the lists, row for row; padding untouched
+        for b in range(B):
+            n = len(P[b])
+            assert st["n_active"][b] == n
+            assert np.array_equal(st["x"][b, :n], np.stack([k["phi"] for k in P[b]]))
+            assert np.array_equal(st["t_cur"][b, :n], np.array([k["T"] for k in P[b]], np.float32))
+            assert np.array_equal(st["h_cand"][b, :n], np.stack([k["h"] for k in P[b]]))
+            assert np.array_equal(st["flops"][b, :n], np.array([k["F"] for k in P[b]], np.float32))
+            assert np.array_equal(st["bytes"][b, :n], np.array([k["Q"] for k in P[b]], np.float32))
+            assert list(st["labels"][b, :n]) == [k["cluster"] for k in P[b]]
+            assert np.array_equal(st["dist2"][b, :n], np.array([k["d2"] for k in P[b]], np.float32))
+            assert np.array_equal(st["pulls"][b, :n], np.stack([k["pulls"] for k in P[b]]))
+            assert np.array_equal(st["reward_sum"][b, :n], np.stack([k["rsum"] for k in P[b]]))
+            assert np.all(st["labels"][b, n:] == -1) and np.all(st["x"][b, n:] == 0) and np.all(st["pulls"][b, n:] == 0)
+            assert st["t_inc"][b] == np.float32(best[b])             # argmin of T over the frontier (the return line)
+    assert n_due >= 4 and max(len(p) for p in P) == cap             # the trigger fired and one frontier filled up
+    # an index beyond the frontier is an error, not a silent append
+    with pytest.raises(ValueError):
+        oracle.append_candidate(st, np.array([cap, 0, 0], np.int32), x_new, t_new)
+
+
+def test_recluster_trigger_values():
+    # t mod tau == 0 and |P| >= 2K, each factor alone is not enough
+    t = np.array([10, 10, 20, 15, 0, 30], np.int32)
+    n = np.array([6, 5, 100, 100, 6, 6], np.int32)
+    assert list(oracle.recluster_due(t, n, 10, 3)) == [1, 0, 1, 0, 1, 1]
+    assert list(oracle.recluster_due(t, n, 5, 3)) == [1, 0, 1, 1, 1, 1]
+    assert list(oracle.recluster_due(t, n, 10, 4)) == [0, 0, 1, 0, 0, 0]
+
+
+def test_signatures_from_reps_masks_empty_clusters():
+    rng = np.random.default_rng(3)
+    B, N, K, R = 2, 9, 4, 3
+    h = rng.uniform(0, 100, (B, N, R)).astype(np.float32)
+    rep = np.array([[3, -1, 8, 0], [-1, -1, 2, 2]], np.int32)
+    hs = oracle.signatures_from_reps(rep, h)
+    for b in range(B):
+        for i in range(K):
+            if rep[b, i] < 0:
+                assert np.all(np.isposinf(hs[b, i]))
+            else:
+                assert np.array_equal(hs[b, i], h[b, rep[b, i]])
+    # an empty cluster is never the masked-UCB choice, whatever its statistics say
+    cl_pulls, cl_mean = np.ones((B, K, 2), np.float32), np.full((B, K, 2), 0.5, np.float32)
+    cl_mean[:, 1] = 10.0                                             # cluster 1 (empty in both) would win otherwise
+    pair = oracle.select_pair(cl_pulls, cl_mean, np.array([5, 5], np.int32), hsig=hs, target=np.array([0, 1], np.int32),
+                              theta_sat=200.0)["pair"]
+    assert pair[0] // 2 in (0, 2, 3) and pair[1] // 2 in (2, 3)
+    # instances that are not due keep their signatures
+    prev = np.full((B, K, R), 7.0, np.float32)
+    hs2 = oracle.signatures_from_reps(rep, h, hsig_prev=prev, run=np.array([0, 1], np.int32))
+    assert np.all(hs2[0] == 7.0) and np.array_equal(hs2[1], hs[1])
