@@ -92,6 +92,7 @@ const char* kb_last_error(kb_ctx* ctx);
  *                                                    (prune: treated as cluster 0)
  *   0x002   prune, sample, select_pair kernels       a target[s] outside [0, R): the arm / pair was masked
  *   0x004   init_centroids, sample, record kernels   a row, member or pair index out of range: nothing written for it
+ *   0x008   append_candidate kernel                  a frontier was full: the verified kernel was dropped (no error)
  *   0x100   tensor-core assign kernel                a bounded wait between its roles expired; the CTA drained and
  *                                                    left; labels of that launch are unspecified
  *   0x200   cooperative fit kernel                   its bounded grid-wide barrier expired; results unspecified
@@ -104,6 +105,7 @@ const char* kb_last_error(kb_ctx* ctx);
 #define KB_STATUS_BAD_LABEL 0x001
 #define KB_STATUS_BAD_TARGET 0x002
 #define KB_STATUS_BAD_INDEX 0x004
+#define KB_STATUS_FRONTIER_FULL 0x008
 #define KB_STATUS_TIMEOUT_ASSIGN 0x100
 #define KB_STATUS_TIMEOUT_FIT 0x200
 kb_status kb_get_device_status(kb_ctx* ctx, int* out);
@@ -520,6 +522,10 @@ typedef struct {
     int32_t* best_arm;          /* [B] */
     float* best_val;            /* [B] */
     int32_t* best_cluster_arm;  /* [B] */
+    /* expanding frontier (both nullable; see kb_append_candidate): */
+    const int32_t* n_active;    /* [B] candidates per instance: the arrays keep N rows per instance (the
+                                 * capacity), the step sees the first n_active[b] of them */
+    const int32_t* run_mask;    /* [B] instances with 0 are skipped: none of their outputs is touched */
 } kb_step_args;
 
 /* The whole step on device-resident data: normalise, seed centroids, fit,
@@ -536,6 +542,68 @@ typedef struct {
  * scored and selected by one more launch (one CTA per instance, the arithmetic
  * of kb_prune and kb_score_select). */
 kb_status kb_bandit_step(kb_ctx* ctx, const kb_step_args* args);
+
+/* ---- the expanding frontier ------------------------------------------------
+ * Sec. 2.2: the action space A_t = P_t x S grows with the frontier P_t, which
+ * is what sets the problem apart from a fixed-arm bandit; Algorithm 1: "P <-
+ * {k_0}, C <- {P}" (one initial cluster) and, inside "if Verify(k'_t)", "P <- P
+ * U {k'_t}"; re-partition "if t mod tau = 0 and |P| >= 2K".
+ *
+ * The frontier of every search lives in arrays of a fixed capacity N_cap rows
+ * per instance; n_active[b] of them are candidates, the rest is padding whose
+ * label the caller initialises to -1 (so that no padding row is ever drawn).
+ * kb_bandit_step and kb_bandit_step_tail take n_active (and run_mask) in
+ * kb_step_args for instances that run as one CTA each (at most 512 rows with D
+ * in {16, 32, 64} for the clustering, at most 1024 with S in {4, 8, 16, 32} for
+ * the tail; KB_ERR_UNSUPPORTED otherwise): features are z-scored over the
+ * active rows only, initial rows must be active, outputs of padding rows are
+ * not written.  kb_sample_member needs no change (a padding row's label -1 is
+ * no cluster), kb_record_outcome and kb_select_pair neither. */
+
+/* Appends the verified kernel k'_t of every search to its frontier.  Where
+ * verified[b] != 0 (null: all), parent[b] >= 0 (the drawn k_t, as
+ * kb_sample_member wrote it) and n_active[b] < N_cap, row j = n_active[b]
+ * becomes the new candidate:
+ *   x[b][j] = x_new[b], t_cur[b][j] = t_new[b]; flops, bytes, h_cand rows from
+ *   flops_new, bytes_new, h_new (each pair nullable together);
+ *   pulls[b][j][.] = 0, reward_sum[b][j][.] = 0 (nobody has played it);
+ *   labels[b][j] = labels[b][parent[b]], dist2[b][j] = dist2[b][parent[b]]
+ *   (until the next re-clustering it sits in the cluster of the kernel it was
+ *   generated from); t_incumbent[b] = min(t_incumbent[b], t_new[b]) (the best
+ *   runtime so far, Algorithm 1's return line); n_active[b] += 1.
+ * appended [B] out, nullable: the row written, or -1.  A full frontier drops
+ * the candidate and sets bit 0x008 of the device status word; parent[b] >=
+ * n_active[b] sets 0x004 and appends nothing.
+ *   verified [B], parent [B] in; x_new [B][D], t_new [B], flops_new [B],
+ *   bytes_new [B], h_new [B][R] in; n_active [B] in/out;
+ *   x [B][N_cap][D], t_cur, flops, bytes, dist2 [B][N_cap], h_cand
+ *   [B][N_cap][R], labels [B][N_cap], pulls, reward_sum [B][N_cap][S] in/out;
+ *   t_incumbent [B] in/out, nullable; dist2 nullable.
+ * DEVICE memory.  One launch (one warp per instance), no workspace. */
+kb_status kb_append_candidate(kb_ctx* ctx, int B, int N_cap, int D, int S, int R, const int32_t* verified,
+                              const int32_t* parent, const float* x_new, const float* t_new,
+                              const float* flops_new, const float* bytes_new, const float* h_new,
+                              int32_t* n_active, float* x, float* t_cur, float* flops, float* bytes,
+                              float* h_cand, int32_t* labels, float* dist2, int32_t* pulls, float* reward_sum,
+                              float* t_incumbent, int32_t* appended);
+
+/* Algorithm 1's test per search: due[b] = (t[b] mod tau == 0 and n_active[b]
+ * >= 2K); any_due [1] out, nullable: 1 if any search is due, else 0 -- the one
+ * word a host reads to decide whether to queue the re-clustering (which it may
+ * also queue unconditionally with run_mask = due).  DEVICE memory; one launch. */
+kb_status kb_recluster_due(kb_ctx* ctx, int B, int tau, int K, const int32_t* t, const int32_t* n_active,
+                           int32_t* due, int32_t* any_due);
+
+/* The signature of every cluster after a re-clustering (Algorithm 1: "profile
+ * h_c^(i) <- NCU(k_c^(i))", the per-candidate signatures standing in for the
+ * profiler): hsig[b][i][:] = h_cand[b][rep[b][i]][:], and +inf for an empty
+ * cluster (rep -1), whose mask entry M_{i,s} = [h < theta_sat] is then 0, so
+ * kb_select_pair never picks an empty cluster.  Instances with run_mask[b] ==
+ * 0 (nullable: all run) keep their hsig.
+ *   rep [B][K], h_cand [B][N][R], run_mask [B] in;  hsig [B][K][R] out.
+ * DEVICE memory; one launch. */
+kb_status kb_signatures_from_reps(kb_ctx* ctx, int B, int N, int K, int R, const int32_t* rep, const float* h_cand,
+                                  const int32_t* run_mask, float* hsig);
 
 /* The tail of the step alone: kb_prune (both masks and, when `bound` is given,
  * the gain bound) followed by kb_score_select, from labels and dist2 that the

@@ -437,6 +437,45 @@ kb_status kb_record_outcome(kb_ctx* ctx, int B, int N, int K, int S, int failure
                                     reward_sum, t, reward, cl_pulls, cl_mean);
 }
 
+kb_status kb_append_candidate(kb_ctx* ctx, int B, int N_cap, int D, int S, int R, const int32_t* verified,
+                              const int32_t* parent, const float* x_new, const float* t_new, const float* flops_new,
+                              const float* bytes_new, const float* h_new, int32_t* n_active, float* x, float* t_cur,
+                              float* flops, float* bytes, float* h_cand, int32_t* labels, float* dist2, int32_t* pulls,
+                              float* reward_sum, float* t_incumbent, int32_t* appended) {
+    KB_COMMON(ctx, B, N_cap);
+    KB_REQUIRE(ctx, D >= 1 && S >= 1 && R >= 1, "kb_append_candidate: D, S and R must be >= 1");
+    if (B > 0) {
+        KB_REQUIRE(ctx, parent && x_new && t_new && n_active, "kb_append_candidate: parent, x_new, t_new and n_active are required");
+        KB_REQUIRE(ctx, N_cap == 0 || (x && t_cur && labels && pulls && reward_sum),
+                   "kb_append_candidate: x, t_cur, labels, pulls and reward_sum are required");
+        KB_REQUIRE(ctx, (flops != nullptr) == (flops_new != nullptr) && (bytes != nullptr) == (bytes_new != nullptr) &&
+                            (h_cand != nullptr) == (h_new != nullptr),
+                   "kb_append_candidate: flops, bytes and h_cand each go with their new row");
+    }
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_append_candidate(ctx, B, N_cap, D, S, R, verified, parent, x_new, t_new, flops_new, bytes_new, h_new,
+                                      n_active, x, t_cur, flops, bytes, h_cand, labels, dist2, pulls, reward_sum, t_incumbent,
+                                      appended);
+}
+
+kb_status kb_recluster_due(kb_ctx* ctx, int B, int tau, int K, const int32_t* t, const int32_t* n_active, int32_t* due,
+                           int32_t* any_due) {
+    KB_COMMON(ctx, B, 0);
+    KB_REQUIRE(ctx, tau >= 1 && K >= 1, "kb_recluster_due: tau and K must be >= 1");
+    if (B > 0) KB_REQUIRE(ctx, t && n_active && due, "kb_recluster_due: t, n_active and due are required");
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_recluster_due(ctx, B, tau, K, t, n_active, due, any_due);
+}
+
+kb_status kb_signatures_from_reps(kb_ctx* ctx, int B, int N, int K, int R, const int32_t* rep, const float* h_cand,
+                                  const int32_t* run_mask, float* hsig) {
+    KB_COMMON(ctx, B, N);
+    KB_REQUIRE(ctx, K >= 1 && R >= 1, "kb_signatures_from_reps: K and R must be >= 1");
+    if (B > 0) KB_REQUIRE(ctx, rep && hsig && (N == 0 || h_cand), "kb_signatures_from_reps: rep, h_cand and hsig are required");
+    TimeScope ts__(ctx, KB_T_SAMPLE);
+    return kb_launch_signatures_from_reps(ctx, B, N, K, R, rep, h_cand, run_mask, hsig);
+}
+
 kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z, const int32_t* rows,
                             float* centroids) {
     KB_COMMON(ctx, B, N);
@@ -504,8 +543,11 @@ static kb_status step_cluster(kb_ctx* ctx, const kb_step_args* a) {
         // at most 512 rows per instance: one CTA takes its instance from raw features to labels
         TimeScope ts__(ctx, KB_T_FIT);
         return kb_launch_fit_fused(ctx, a->B, a->N, a->D, a->K, a->iters, nullptr, a->x, a->z, a->init_rows, a->centroids,
-                                   a->labels, a->dist2, a->inertia, a->rep, a->counts);
+                                   a->labels, a->dist2, a->inertia, a->rep, a->counts, a->n_active, a->run_mask);
     }
+    if (a->n_active || a->run_mask)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "n_active / run_mask need instances that cluster as one CTA each: at most "
+                                                 "512 rows, D in {16, 32, 64}, 16-byte aligned x, z, centroids");
     if (ctx->assign_path == 0 && a->iters >= 0 && !kb_assign_tc_eligible(ctx, a->B, a->N, a->D, a->K) &&
         kb_fit_coop_eligible(ctx, a->B, a->N, a->D, a->K) && a->x && a->z && a->init_rows && a->centroids && a->labels &&
         (((uintptr_t)a->x | (uintptr_t)a->z | (uintptr_t)a->centroids) & 15) == 0) {
@@ -546,6 +588,9 @@ static kb_status step_tail(kb_ctx* ctx, const kb_step_args* a, bool bound_done) 
         TimeScope ts__(ctx, KB_T_SCORE);
         return kb_launch_step_tail_small(ctx, a, bound_done);
     }
+    if (a->n_active || a->run_mask)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "n_active / run_mask need a tail that runs as one CTA per instance: at most "
+                                                 "1024 rows, S in {4, 8, 16, 32}, K*S <= 8192, aligned per-arm arrays");
     if (kb_step_tail_fused_eligible(ctx, a)) {
         // larger instances: the pruning rides on the statistics pass (three launches, labels and keep touched once)
         TimeScope ts__(ctx, KB_T_SCORE);
@@ -634,6 +679,9 @@ kb_status kb_bandit_step_host(kb_ctx* ctx, const kb_step_args* h) {
     if (!ctx || !h) return KB_ERR_INVALID_ARG;
     KB_COMMON(ctx, h->B, h->N);
     KB_REQUIRE(ctx, h->D >= 1 && h->K >= 1 && h->S >= 1 && h->R >= 1, "kb_bandit_step_host: sizes must be >= 1");
+    if (h->n_active || h->run_mask)
+        return kb_fail(ctx, KB_ERR_UNSUPPORTED, "kb_bandit_step_host: an expanding frontier lives on the device (n_active, "
+                                                 "run_mask are for kb_bandit_step)");
     size_t scratch = 0;
     kb_workspace_bytes(h->B, h->N, h->D, h->K, h->S, &scratch);
     scratch = kb_align256(scratch);

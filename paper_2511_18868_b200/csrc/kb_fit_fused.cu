@@ -33,25 +33,38 @@ __host__ __device__ constexpr int ff_rows(int D) { return D <= 32 ? 4 : 2; }
 
 template <int D>
 __global__ void __launch_bounds__(FF_MAXROWS / ff_rows(D))
-fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, const float* xraw, float* zout,
+fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const float* xraw, float* zout,
                  const int32_t* __restrict__ init_rows, float* __restrict__ cent,
                  int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
-                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, int* __restrict__ dev_status) {
+                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, const int32_t* __restrict__ n_active,
+                 const int32_t* __restrict__ run_mask, int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
+    // An expanding frontier: the instance's arrays have NCAP rows of which the first n_active[b] are candidates
+    // (N below); without n_active every row is.  An instance whose run_mask entry is 0 is left exactly as it is.
+    if (run_mask && run_mask[blockIdx.x] == 0) return;
+    const int N = n_active ? min(max(n_active[blockIdx.x], 0), NCAP) : NCAP;
     constexpr int FF_R = ff_rows(D), FF_T = FF_MAXROWS / FF_R;
     extern __shared__ __align__(16) unsigned char ff_raw[];
     constexpr int ZS = D + 1;                                       // padded row stride: conflict-free column walks
     float* cs = reinterpret_cast<float*>(ff_raw);                   // [K][D] centroids (16-byte aligned rows)
     float* zs = cs + (size_t)K * D;                                 // [N][D+1] the instance
     // [K] counts, then scatter cursors; 8-byte aligned because the space is reused for 64-bit keys
-    int* hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(zs + (size_t)N * ZS) + 7) & ~(uintptr_t)7);
+    int* hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(zs + (size_t)NCAP * ZS) + 7) & ~(uintptr_t)7);
     int* offs = hist + K;                                           // [K+1]
-    unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [N] row ids in label order
+    unsigned short* perm = reinterpret_cast<unsigned short*>(offs + K + 1);   // [NCAP] row ids in label order
     __shared__ double s_red[FF_MAXROWS / 64];
     __shared__ int s_scan[FF_MAXROWS / 64];
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* zb = (xraw ? xraw : z) + (size_t)b * N * D;
+    const float* zb = (xraw ? xraw : z) + (size_t)b * NCAP * D;
     float* cb = cent + (size_t)b * K * D;
+    if (N == 0) {                                                   // nothing to cluster: centroids stay, every cluster is empty
+        for (int j = tid; j < K; j += FF_T) {
+            if (counts) counts[(size_t)b * K + j] = 0;
+            if (rep) rep[(size_t)b * K + j] = -1;
+        }
+        if (inertia && tid == 0) inertia[b] = 0.f;
+        return;
+    }
 
     // stage the instance (coalesced float4 reads; plain loads: raw features may be normalised in place)
     for (int e = tid; e < N * (D / 4); e += FF_T) {
@@ -63,7 +76,7 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, const flo
     __syncthreads();
     if (xraw) {
         // ---- column z-score of the staged rows (population standard deviation) ----------------
-        double* red = reinterpret_cast<double*>((reinterpret_cast<uintptr_t>(perm + N) + 7) & ~(uintptr_t)7);   // [FF_T][2]
+        double* red = reinterpret_cast<double*>((reinterpret_cast<uintptr_t>(perm + NCAP) + 7) & ~(uintptr_t)7);   // [FF_T][2]
         float* st_mh = reinterpret_cast<float*>(red + 2 * FF_T);    // [D] mean, high part
         float* st_ml = st_mh + D;                                   // [D] mean, low part
         float* st_inv = st_ml + D;                                  // [D] 1 / standard deviation
@@ -92,7 +105,7 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, const flo
             st_inv[c] = (float)(1.0 / sc);
         }
         __syncthreads();
-        float* zo = zout + (size_t)b * N * D;
+        float* zo = zout + (size_t)b * NCAP * D;
         for (int e = tid; e < N * (D / 4); e += FF_T) {
             const int r = e / (D / 4), q = e - r * (D / 4);
             float* d = zs + (size_t)r * ZS + 4 * q;
@@ -220,7 +233,7 @@ fit_fused_kernel(int N, int K, int iters, const float* __restrict__ z, const flo
     for (int u = 0; u < FF_R; ++u)
         if (active[u]) {
             const int r = tid + u * FF_T;
-            const size_t flat = (size_t)b * N + r;
+            const size_t flat = (size_t)b * NCAP + r;
             labels[flat] = arg[u];
             if (dist2) dist2[flat] = best[u];
             if (rep) atomicMin(&rep_key[arg[u]], ((unsigned long long)__float_as_uint(best[u]) << 32) | (unsigned)r);
@@ -268,17 +281,18 @@ bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
 // xraw itself) and init_rows (row ids of the initial centroids; null: `cent` holds them)
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
-                              float* inertia, int32_t* rep, int32_t* counts) {
+                              float* inertia, int32_t* rep, int32_t* counts, const int32_t* n_active,
+                              const int32_t* run_mask) {
     const size_t smem = ff_smem(N, D, K);
     if (D == 16) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
+        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
     } else if (D == 32) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
+        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
     } else {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, ctx->dev_status);
+        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;

@@ -122,7 +122,8 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
                              int32_t* rep, int32_t* counts);
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
-                              float* inertia, int32_t* rep, int32_t* counts);
+                              float* inertia, int32_t* rep, int32_t* counts, const int32_t* n_active = nullptr,
+                              const int32_t* run_mask = nullptr);
 size_t kb_ws_need_update(int B, int N, int D, int K);
 size_t kb_ws_need_fit_acc(int B, int D, int K);
 size_t kb_ws_need_score(int B, int N, int K, int S);
@@ -164,6 +165,15 @@ kb_status kb_launch_sample_member(kb_ctx*, int B, int N, int K, int S, int R, co
                                   float* member_val);
 kb_status kb_launch_init_centroids(kb_ctx*, int B, int N, int D, int K, const float* z, const int32_t* rows,
                                    float* c);
+kb_status kb_launch_append_candidate(kb_ctx* ctx, int B, int N_cap, int D, int S, int R, const int32_t* verified,
+                                     const int32_t* parent, const float* x_new, const float* t_new, const float* flops_new,
+                                     const float* bytes_new, const float* h_new, int32_t* n_active, float* x, float* t_cur,
+                                     float* flops, float* bytes, float* h_cand, int32_t* labels, float* dist2,
+                                     int32_t* pulls, float* reward_sum, float* t_inc, int32_t* appended);
+kb_status kb_launch_recluster_due(kb_ctx* ctx, int B, int tau, int K, const int32_t* t, const int32_t* n_active,
+                                  int32_t* due, int32_t* any_due);
+kb_status kb_launch_signatures_from_reps(kb_ctx* ctx, int B, int N, int K, int R, const int32_t* rep, const float* h_cand,
+                                         const int32_t* run_mask, float* hsig);
 
 // Opts a kernel into more than 48 KB of dynamic shared memory when it needs it.
 #define KB_SMEM_OPTIN(ctx, kernel, bytes)                                                        \

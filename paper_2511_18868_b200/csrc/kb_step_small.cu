@@ -29,6 +29,7 @@ struct TailArgs {
     uint32_t *keep, *kept;
     float *bound, *cl_pulls, *cl_mean, *cl_index, *arm_index, *best_val;
     int32_t *best_arm, *best_cluster_arm;
+    const int32_t *n_active, *run_mask;   // expanding frontier: candidates per instance (of N rows), instances to run
     int* dev_status;
 };
 
@@ -54,7 +55,11 @@ __global__ void __launch_bounds__(ST_T)
 step_tail_small_kernel(const TailArgs a) {
     kb_grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char sraw[];
-    const int N = a.N, S = a.S, K = a.K, KS = K * S;
+    // An expanding frontier: the arrays have a.N rows per instance of which the first n_active[b] are candidates
+    // (N below; NP is the pitch); an instance whose run_mask entry is 0 is left exactly as it is.
+    if (a.run_mask && a.run_mask[blockIdx.x] == 0) return;
+    const int NP = a.N, S = a.S, K = a.K, KS = K * S;
+    const int N = a.n_active ? min(max(a.n_active[blockIdx.x], 0), NP) : NP;
     int* sp = reinterpret_cast<int*>(sraw);                      // [K][S] pull sums
     float* sr = reinterpret_cast<float*>(sraw) + KS;             // [K][S] reward sums
     float* tab = sr + KS;                                        // [K][S] U_cl
@@ -91,7 +96,7 @@ step_tail_small_kernel(const TailArgs a) {
         }
         tinc = a.t_inc[b];
     }
-    const size_t row0 = (size_t)b * N;
+    const size_t row0 = (size_t)b * NP;
     const unsigned all_arms = S == 32 ? 0xffffffffu : ((1u << S) - 1u);
 
     // ---- pass 1: keep bits, gain bound, cluster sums ------------------------------------------
@@ -99,7 +104,7 @@ step_tail_small_kernel(const TailArgs a) {
     for (int it = 0; it < trips; ++it) {
         const int r = it * rstep + tid / vps;
         const bool live = r < N;
-        const size_t i = row0 + min(r, N - 1);                   // clamped: loads stay in range
+        const size_t i = row0 + min(r, N - 1);                   // clamped: loads stay in range (no trip when N == 0)
         int lab = __ldg(a.labels + i);
         const bool lab_ok = lab >= 0 && lab < K;
         if (!lab_ok) { if (live) atomicOr(a.dev_status, 1); lab = 0; }
@@ -256,6 +261,7 @@ kb_status kb_launch_step_tail_small(kb_ctx* ctx, const kb_step_args* s, bool bou
     a.bound = s->bound; a.cl_pulls = s->cl_pulls; a.cl_mean = s->cl_mean; a.cl_index = s->cl_index;
     a.arm_index = s->arm_index; a.best_val = s->best_val;
     a.best_arm = s->best_arm; a.best_cluster_arm = s->best_cluster_arm;
+    a.n_active = s->n_active; a.run_mask = s->run_mask;
     a.dev_status = ctx->dev_status;
     const size_t smem = tail_smem(s->N, s->K, s->S);
     KB_SMEM_OPTIN(ctx, step_tail_small_kernel<true>, smem);

@@ -26,7 +26,8 @@ EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb
            "kb_timing_enable", "kb_timing_read", "kb_probe_peaks", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
            "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_bandit_step_tail", "kb_step_workspace_bytes",
-           "kb_bandit_step_host", "kb_cluster_update_noalloc", "kb_cluster_update_noalloc_status"]
+           "kb_bandit_step_host", "kb_cluster_update_noalloc", "kb_cluster_update_noalloc_status",
+           "kb_append_candidate", "kb_recluster_due", "kb_signatures_from_reps"]
 
 
 TIMING_CLASSES = ["normalize", "assign", "update", "prune", "score", "init", "fit", "assign_kernel", "sample", "prep"]
@@ -55,12 +56,13 @@ _STEP_IN = ["x", "init_rows", "flops", "bytes", "peak_flops", "peak_bw", "t_incu
             "pulls", "reward_sum", "t"]
 _STEP_OUT = ["z", "centroids", "counts", "labels", "dist2", "inertia", "rep", "keep", "kept_count", "bound",
              "cl_pulls", "cl_mean", "cl_index", "arm_index", "best_arm", "best_val", "best_cluster_arm"]
+_STEP_OPT = ["n_active", "run_mask"]          # expanding frontier: candidates per instance, instances to run
 
 
 class StepArgs(ctypes.Structure):
     _fields_ = ([(n, ctypes.c_int) for n in ["B", "N", "D", "K", "S", "R", "iters"]] +
                 [("theta_sat", ctypes.c_float), ("score", ScoreParams)] +
-                [(n, _VP) for n in _STEP_IN + _STEP_OUT])
+                [(n, _VP) for n in _STEP_IN + _STEP_OUT + _STEP_OPT])
 
 
 _lib = None
@@ -113,6 +115,9 @@ def load_library() -> ctypes.CDLL:
     lib.kb_cluster_update_noalloc_status.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
+    lib.kb_append_candidate.argtypes = [_VP, i, i, i, i, i] + [_VP] * 19
+    lib.kb_recluster_due.argtypes = [_VP, i, i, i] + [_VP] * 4
+    lib.kb_signatures_from_reps.argtypes = [_VP, i, i, i, i] + [_VP] * 4
     lib.kb_bandit_step.argtypes = [_VP, ctypes.POINTER(StepArgs)]
     lib.kb_bandit_step_tail.argtypes = [_VP, ctypes.POINTER(StepArgs)]
     lib.kb_step_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(sz)]
@@ -373,7 +378,7 @@ class KB:
         a.score = ScoreParams(float(params.get("c", 2.0)), float(params.get("lipschitz_L", 0.0)),
                               float(params.get("prior_pulls", 1.0)), float(params.get("prior_mean", 0.5)),
                               int(bool(params.get("cap_with_bound", False))))
-        for name in _STEP_IN + _STEP_OUT:
+        for name in _STEP_IN + _STEP_OUT + _STEP_OPT:
             t = tensors.get(name)
             setattr(a, name, None if t is None else _ptr(t, None if host else self.device))
         return a
@@ -382,6 +387,30 @@ class KB:
         """Whole step on device tensors (dict keyed by the field names of kb_step_args)."""
         a = self._step_args(dims, params, tensors, host=False)
         self._check(self.lib.kb_bandit_step(self.h, ctypes.byref(a)), "kb_bandit_step")
+
+    def append_candidate(self, st, parent, x_new, t_new, verified=None, flops_new=None, bytes_new=None, h_new=None,
+                         appended=None):
+        """kb_append_candidate on a frontier `st`: dict of device tensors n_active [B], x [B,Ncap,D], t_cur, labels
+        [B,Ncap], pulls, reward_sum [B,Ncap,S] and optionally flops, bytes, dist2 [B,Ncap], h_cand [B,Ncap,R], t_inc [B]."""
+        B, Ncap, D = st["x"].shape
+        S = st["pulls"].shape[2]
+        R = st["h_cand"].shape[2] if st.get("h_cand") is not None else 1
+        p = self._p
+        self._check(self.lib.kb_append_candidate(
+            self.h, B, Ncap, D, S, R, p(verified), p(parent), p(x_new), p(t_new), p(flops_new), p(bytes_new), p(h_new),
+            p(st["n_active"]), p(st["x"]), p(st["t_cur"]), p(st.get("flops")), p(st.get("bytes")), p(st.get("h_cand")),
+            p(st["labels"]), p(st.get("dist2")), p(st["pulls"]), p(st["reward_sum"]), p(st.get("t_inc")), p(appended)),
+            "kb_append_candidate")
+
+    def recluster_due(self, t, n_active, tau, K, due, any_due=None):
+        self._check(self.lib.kb_recluster_due(self.h, t.shape[0], int(tau), int(K), self._p(t), self._p(n_active),
+                                              self._p(due), self._p(any_due)), "kb_recluster_due")
+
+    def signatures_from_reps(self, rep, h_cand, hsig, run_mask=None):
+        B, K = rep.shape
+        N, R = h_cand.shape[1], h_cand.shape[2]
+        self._check(self.lib.kb_signatures_from_reps(self.h, B, N, K, R, self._p(rep), self._p(h_cand), self._p(run_mask),
+                                                     self._p(hsig)), "kb_signatures_from_reps")
 
     def bandit_step_tail(self, dims, params, tensors):
         """kb_bandit_step_tail: prune + score + select from the caller's labels and dist2 (device tensors)."""

@@ -58,9 +58,9 @@ def test_null_context_is_rejected(lib):
 
 
 def test_struct_layout_matches_header():
-    # 7 ints + float + 5-word params + 30 pointers, pointer-aligned
+    # 7 ints + float + 5-word params + 32 pointers (13 inputs, 17 outputs, 2 for the expanding frontier), pointer-aligned
     assert ctypes.sizeof(kb.ScoreParams) == 20
-    assert ctypes.sizeof(kb.StepArgs) == 56 + 8 * 30
+    assert ctypes.sizeof(kb.StepArgs) == 56 + 8 * 32
     assert len(kb._STEP_IN) == 13 and len(kb._STEP_OUT) == 17
 
 
