@@ -155,6 +155,26 @@ def init_centroids(z, rows):
     return c
 
 
+def lloyd_tol(z, centroids, max_iter, tol):
+    """Lloyd's iteration with a tolerance stop per instance (see kbo_lloyd_tol).  Returns a dict with centroids, labels,
+    dist2, inertia, rep, counts, n_iter [B] and last_shift [B]; `centroids` (initial) is not modified."""
+    z = _f32(z)
+    c = np.array(centroids, dtype=np.float32, order="C", copy=True)
+    B, N, D = z.shape
+    K = c.shape[1]
+    labels = np.empty((B, N), np.int32)
+    dist2 = np.empty((B, N), np.float32)
+    inertia = np.empty((B,), np.float32)
+    rep = np.empty((B, K), np.int32)
+    counts = np.empty((B, K), np.int32)
+    n_iter = np.empty((B,), np.int32)
+    shift = np.empty((B,), np.float64)
+    _check(_load().kbo_lloyd_tol(B, N, D, K, int(max_iter), ctypes.c_float(tol), _p(z), _p(c), _p(labels), _p(dist2),
+                                 _p(inertia), _p(rep), _p(counts), _p(n_iter), _p(shift)), "lloyd_tol")
+    return {"centroids": c, "labels": labels, "dist2": dist2, "inertia": inertia, "rep": rep, "counts": counts,
+            "n_iter": n_iter, "last_shift": shift}
+
+
 def philox4x32_10(counter, key):
     """One block of the counter-based generator: counter = 4 words, key = 2 words -> 4 words (uint32)."""
     c = np.ascontiguousarray(counter, dtype=np.uint32)

@@ -302,13 +302,60 @@ int kbo_score_select(int B, int N, int K, int S, float c, float lipschitz_L, flo
 
 // Gather of initial centroids: C[b][i][:] = Z[b][rows[b][i]][:] (plain Lloyd
 // started from K data rows supplied by the caller).
+// rows[b][i] == -1 names no row: cluster i of that instance is UNUSED -- its centroid is put at 1e18 in every
+// coordinate, farther from any data than any other centroid, so no row is ever assigned to it, it stays empty and
+// keeps that centroid through every update.  This is how instances with fewer than K clusters share a batch (the
+// K in {1, 2, 3, 5} sensitivity study of Sec. 4 as four instances of one call with K = 5).
 int kbo_init_centroids(int B, int N, int D, int K, const float* z, const int32_t* rows, float* centroids) {
     for (int b = 0; b < B; ++b)
         for (int i = 0; i < K; ++i) {
             int r = rows[ix2(b, i, K)];
-            if (r < 0 || r >= N) return 2;
-            for (int d = 0; d < D; ++d) centroids[ix3(b, i, d, K, D)] = z[ix3(b, r, d, N, D)];
+            if (r < -1 || r >= N) return 2;
+            for (int d = 0; d < D; ++d) centroids[ix3(b, i, d, K, D)] = r < 0 ? 1e18f : z[ix3(b, r, d, N, D)];
         }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Lloyd's iteration with a tolerance stop (the `tol` of the "scikit-learn's KMeans" of Sec. 3.5): per instance,
+//   repeat: assign, update, shift = sum_j ||c_j(new) - c_j(old)||^2;  stop after this update if shift <= tol
+//   or max_iter updates are done;  then one more assign, so that labels and dist2 belong to the returned centroids.
+// (Unchanged labels give unchanged centroids, shift = 0 <= tol: the rule also covers "labels did not change".)
+// n_iter[b] = updates done for instance b;  last_shift[b] (optional) = the shift of its last update.
+// Instances stop independently of one another.
+// ---------------------------------------------------------------------------
+int kbo_lloyd_tol(int B, int N, int D, int K, int max_iter, float tol, const float* z, float* centroids,
+                  int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts, int32_t* n_iter,
+                  double* last_shift) {
+    std::vector<float> old((size_t)K * (size_t)D);
+    for (int b = 0; b < B; ++b) {
+        const float* zb = z + (size_t)b * N * D;
+        float* cb = centroids + (size_t)b * K * D;
+        int32_t* lb = labels + (size_t)b * N;
+        int32_t* nb = counts ? counts + (size_t)b * K : nullptr;
+        int it = 0;
+        double shift = 0.0;
+        if (nb) for (int i = 0; i < K; ++i) nb[i] = 0;
+        while (it < max_iter) {
+            int rc = kbo_cluster_assign(1, N, D, K, zb, cb, lb, nullptr, nullptr, nullptr, nullptr, nullptr);
+            if (rc) return rc;
+            for (size_t e = 0; e < old.size(); ++e) old[e] = cb[e];
+            rc = kbo_cluster_update(1, N, D, K, zb, lb, cb, nb);
+            if (rc) return rc;
+            ++it;
+            shift = 0.0;
+            for (size_t e = 0; e < old.size(); ++e) {
+                const double dlt = (double)cb[e] - (double)old[e];
+                shift += dlt * dlt;
+            }
+            if (shift <= (double)tol) break;
+        }
+        int rc = kbo_cluster_assign(1, N, D, K, zb, cb, lb, dist2 ? dist2 + (size_t)b * N : nullptr,
+                                    inertia ? inertia + b : nullptr, rep ? rep + (size_t)b * K : nullptr, nullptr, nullptr);
+        if (rc) return rc;
+        n_iter[b] = it;
+        if (last_shift) last_shift[b] = shift;
+    }
     return 0;
 }
 

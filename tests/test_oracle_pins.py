@@ -467,7 +467,7 @@ def test_init_centroids_is_a_row_gather():
     bad[1, 3] = N
     with pytest.raises(ValueError):
         oracle.init_centroids(z, bad)
-    bad[1, 3] = -1
+    bad[1, 3] = -2                                                   # (-1 alone names an unused cluster)
     with pytest.raises(ValueError):
         oracle.init_centroids(z, bad)
 
@@ -985,3 +985,80 @@ def test_signatures_from_reps_masks_empty_clusters():
     prev = np.full((B, K, R), 7.0, np.float32)
     hs2 = oracle.signatures_from_reps(rep, h, hsig_prev=prev, run=np.array([0, 1], np.int32))
     assert np.all(hs2[0] == 7.0) and np.array_equal(hs2[1], hs[1])
+
+
+# ----------------------------------------------------- tolerance stop, unused clusters
+def test_lloyd_tol_matches_sklearn_iteration_counts():
+    """The tolerance stop against scikit-learn's KMeans (Sec. 3.5) from the same initial centres: the number of
+    iterations it reports, its centres and its labels.  scikit-learn scales `tol` by the mean column variance
+    (1 for z-scored features without constant columns) and also stops when the labels repeat, which the shift
+    rule covers (unchanged labels -> unchanged centres -> shift 0)."""
+    sklearn_cluster = pytest.importorskip("sklearn.cluster")
+    rng = np.random.default_rng(12)
+    for N, D, K, tol in [(400, 5, 3, 1e-4), (900, 8, 6, 1e-2), (600, 4, 5, 0.0), (300, 16, 4, 1e-3), (500, 6, 3, 0.3)]:
+        centres = 2.0 * rng.standard_normal((K, D))
+        x = (centres[rng.integers(0, K, N)] + rng.standard_normal((N, D))).astype(np.float32)
+        z, _, _ = oracle.normalize(x[None])
+        init = z[0, rng.choice(N, K, replace=False)]
+        scaled_tol = tol * float(np.mean(np.var(z[0].astype(np.float64), axis=0)))
+        km = sklearn_cluster.KMeans(n_clusters=K, init=init.astype(np.float64), n_init=1, max_iter=50, tol=tol,
+                                    algorithm="lloyd").fit(z[0].astype(np.float64))
+        got = oracle.lloyd_tol(z, init[None], 50, scaled_tol)
+        assert got["n_iter"][0] == km.n_iter_, (N, D, K, tol, got["n_iter"][0], km.n_iter_)
+        np.testing.assert_allclose(got["centroids"][0], km.cluster_centers_, atol=2e-5)
+        assert np.array_equal(got["labels"][0], km.labels_)
+        assert got["inertia"][0] == pytest.approx(km.inertia_, rel=1e-5)
+        assert got["last_shift"][0] <= scaled_tol or got["n_iter"][0] == 50
+        assert got["counts"][0].sum() == N                             # (the members of the last update, not of the final labels)
+
+
+def test_lloyd_tol_is_the_plain_loop_cut_short():
+    """tol < 0 never stops early: exactly max_iter plain iterations; with a tolerance the result is the plain loop's
+    after n_iter iterations; instances of one batch stop independently."""
+    rng = np.random.default_rng(13)
+    B, N, D, K = 4, 300, 6, 5
+    z = rng.standard_normal((B, N, D)).astype(np.float32)
+    z[0] *= 0.01                                                       # instance 0 converges at once on any scale
+    init = np.stack([z[b, rng.choice(N, K, replace=False)] for b in range(B)])
+    full = oracle.lloyd_tol(z, init, 7, -1.0)
+    assert np.all(full["n_iter"] == 7)
+    c = init.copy()
+    for _ in range(7):
+        a = oracle.cluster_assign(z, c, want_rep=False)
+        c, n = oracle.cluster_update(z, a["labels"], c)
+    assert np.array_equal(full["centroids"], c) and np.array_equal(full["counts"], n)
+    tol = oracle.lloyd_tol(z, init, 50, 1e-3)
+    assert len(set(tol["n_iter"].tolist())) > 1 and tol["n_iter"].max() < 50
+    for b in range(B):
+        c = init[b:b + 1].copy()
+        for _ in range(int(tol["n_iter"][b])):
+            a = oracle.cluster_assign(z[b:b + 1], c, want_rep=False)
+            c, _ = oracle.cluster_update(z[b:b + 1], a["labels"], c)
+        assert np.array_equal(tol["centroids"][b:b + 1], c)
+        a = oracle.cluster_assign(z[b:b + 1], c)
+        assert np.array_equal(tol["labels"][b:b + 1], a["labels"]) and np.array_equal(tol["rep"][b:b + 1], a["rep"])
+    assert np.all(oracle.lloyd_tol(z, init, 0, 1.0)["n_iter"] == 0)     # no iteration: the labels of the initial centres
+
+
+def test_unused_clusters_share_a_batch_with_fewer_clusters():
+    """rows = -1 marks a cluster as unused (centroid far away): an instance with K_b < K clusters then clusters exactly
+    as it would alone with K_b -- the K in {1, 2, 3, 5} sensitivity study as four instances of one call with K = 5."""
+    rng = np.random.default_rng(14)
+    N, D, K = 200, 5, 5
+    x = (3.0 * rng.standard_normal((4, 1, D)) * (rng.integers(0, 3, (4, N, 1)) - 1) + rng.standard_normal((4, N, D))).astype(np.float32)
+    z, _, _ = oracle.normalize(x)
+    rows = np.full((4, K), -1, np.int32)
+    for b, kb in enumerate([1, 2, 3, 5]):
+        rows[b, :kb] = rng.choice(N, kb, replace=False)
+    c0 = oracle.init_centroids(z, rows)
+    assert np.all(c0[0, 1:] == np.float32(1e18)) and np.array_equal(c0[1, :2], z[1, rows[1, :2]])
+    got = oracle.lloyd_tol(z, c0, 10, -1.0)
+    for b, kb in enumerate([1, 2, 3, 5]):
+        alone = oracle.lloyd_tol(z[b:b + 1], oracle.init_centroids(z[b:b + 1], rows[b:b + 1, :kb]), 10, -1.0)
+        assert np.array_equal(got["labels"][b], alone["labels"][0]) and got["labels"][b].max() < kb
+        assert np.array_equal(got["centroids"][b, :kb], alone["centroids"][0])
+        assert np.all(got["centroids"][b, kb:] == np.float32(1e18))       # never moved, never chosen
+        assert np.all(got["counts"][b, kb:] == 0) and np.all(got["rep"][b, kb:] == -1)
+        assert got["inertia"][b] == alone["inertia"][0]
+    with pytest.raises(ValueError):
+        oracle.init_centroids(z, np.full((4, K), -2, np.int32))
