@@ -470,6 +470,15 @@ kb_status kb_cluster_update_noalloc_status(void* cuda_stream, int* out);
  * rows [B][K] in, values in [0,N). */
 kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float* z,
                             const int32_t* rows, float* centroids);
+/* rows[b][i] == -1 (here and in init_rows of kb_bandit_step for instances of at
+ * most 512 rows) marks cluster i of instance b as UNUSED: its centroid is put
+ * at 1e18 in every coordinate, out of every row's reach, so it stays empty
+ * (count 0, rep -1, never selected) and keeps that centroid through every
+ * update.  Instances with fewer than K clusters can so share one batch -- the
+ * K in {1, 2, 3, 5} sensitivity study of Sec. 4 as four instances of one call
+ * with K = 5.  Meant for the fp32 kernels (K < 128 or small instances); the
+ * tensor-core kernel stays exact but sends every row through its fp32
+ * re-evaluation, because the far centroid spoils the instance's fp16 scale. */
 
 /* iters x (assign, update) followed by a final assign, so that labels/dist2
  * are consistent with the returned centroids (Sec. 3.3).  Same arguments as
@@ -482,6 +491,26 @@ kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float
 kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z,
                          float* centroids, int32_t* labels, float* dist2, float* inertia,
                          int32_t* rep, int32_t* counts);
+
+/* kb_cluster_fit with the tolerance stop of the "scikit-learn's KMeans" of
+ * Sec. 3.5: per instance, after every update shift = sum_j ||c_j(new) -
+ * c_j(old)||^2; the instance stops after the first update with shift <= tol
+ * (that update stays) or after max_iter updates; one more assignment then makes
+ * labels / dist2 / inertia / rep belong to the returned centroids.  Unchanged
+ * labels give shift 0, so "labels repeat" is covered.  (scikit-learn's own
+ * `tol` is relative: multiply it by the mean column variance of z, which is 1
+ * for z-scored features without constant columns.)  Instances stop
+ * independently; everything stays on the device.
+ *   tol >= 0;  n_iter [B] out: updates done per instance;  counts: the members
+ *   at the instance's last update;  other arguments as kb_cluster_fit.
+ * Instances of at most 512 rows with D in {16, 32, 64} stop inside their
+ * one-CTA launch.  Otherwise the loop of calls runs all max_iter iterations and
+ * a small kernel after every update undoes the updates of instances that have
+ * stopped (the result of stopping, not its saving); needs the workspace of
+ * kb_workspace_bytes. */
+kb_status kb_cluster_fit_tol(kb_ctx* ctx, int B, int N, int D, int K, int max_iter, float tol, const float* z,
+                             float* centroids, int32_t* labels, float* dist2, float* inertia, int32_t* rep,
+                             int32_t* counts, int32_t* n_iter);
 
 /* Sizes and inputs/outputs of one whole bandit step.  Every pointer is a
  * device pointer for kb_bandit_step and a HOST pointer for kb_bandit_step_host. */

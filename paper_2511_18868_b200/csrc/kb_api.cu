@@ -24,13 +24,73 @@ __global__ void gather_rows_kernel(int N, int D, int K, const float* __restrict_
     kb_grid_dependency_wait();
     const int b = blockIdx.y, i = blockIdx.x;
     int r = rows[(size_t)b * K + i];
+    float* dst = c + ((size_t)b * K + i) * D;
+    if (r == -1) {                                                  // an unused cluster: out of every row's reach
+        for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = KB_UNUSED_CENTROID;
+        return;
+    }
     if (r < 0 || r >= N) { if (threadIdx.x == 0) atomicOr(dev_status, 4); return; }
     const float* src = z + ((size_t)b * N + r) * D;
-    float* dst = c + ((size_t)b * K + i) * D;
     for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = src[d];
 }
 
 size_t max_sz(size_t a, size_t b) { return a > b ? a : b; }
+
+// Tolerance stop for a fit that runs as a loop of calls (no host read, no change to the kernels of the loop): after
+// every update this kernel (one CTA per instance) measures the instance's total squared centroid shift against the
+// copy it keeps of the previous centroids.  An instance whose shift has dropped to `tol` is DONE from then on: the
+// update that got it there stays, every later update (and its counts) is undone by restoring the copy, so the
+// remaining iterations recompute the same labels and the final assignment sees the centroids the instance stopped
+// at -- the result of stopping, at the cost of the idle iterations.
+// mode 0: before the loop (copy <- centroids, done <- 0); mode 1: after update number `it`; mode 2: n_iter out.
+__global__ void __launch_bounds__(256) tol_gate_kernel(int mode, int it, int KD, int K, float tol, float* __restrict__ cent,
+                                                       int32_t* __restrict__ counts, float* __restrict__ prev,
+                                                       int32_t* __restrict__ prev_counts, int32_t* __restrict__ done,
+                                                       int32_t* __restrict__ n_iter) {
+    kb_grid_dependency_wait();
+    __shared__ double s_red[8];
+    __shared__ int s_frozen;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    float* c = cent + (size_t)b * KD;
+    float* p = prev + (size_t)b * KD;
+    if (mode == 0) {
+        for (int e = tid; e < KD; e += 256) p[e] = c[e];
+        if (tid == 0) done[b] = 0;
+        return;
+    }
+    if (mode == 2) {
+        if (tid == 0 && n_iter) n_iter[b] = done[b] ? done[b] : it;
+        return;
+    }
+    if (tid == 0) s_frozen = done[b];
+    __syncthreads();
+    const bool frozen = s_frozen != 0;
+    if (frozen) {
+        for (int e = tid; e < KD; e += 256) c[e] = p[e];
+        if (counts) for (int j = tid; j < K; j += 256) counts[(size_t)b * K + j] = prev_counts[(size_t)b * K + j];
+        return;
+    }
+    double moved = 0.0;
+    for (int e = tid; e < KD; e += 256) {
+        const float dlt = c[e] - p[e];
+        moved += (double)dlt * (double)dlt;
+        p[e] = c[e];
+    }
+    if (counts) for (int j = tid; j < K; j += 256) prev_counts[(size_t)b * K + j] = counts[(size_t)b * K + j];
+    const double w = kb_warp_sum(moved);
+    if ((tid & 31) == 0) s_red[tid >> 5] = w;
+    __syncthreads();
+    if (tid == 0) {
+        double shift = 0.0;
+        for (int q = 0; q < 8; ++q) shift += s_red[q];
+        if (shift <= (double)tol) done[b] = it;
+    }
+}
+
+size_t ws_need_tol(int B, int D, int K) {
+    return kb_align256((size_t)B * K * D * sizeof(float)) + kb_align256((size_t)B * K * sizeof(int32_t)) +
+           kb_align256((size_t)B * sizeof(int32_t));
+}
 
 // brackets the work one public call queues with a pair of events (when timing is on)
 struct TimeScope {
@@ -191,7 +251,8 @@ kb_status kb_workspace_bytes(int B, int N, int D, int K, int S, size_t* out) {
     need = max_sz(need, kb_ws_need_sample(B));
     need = max_sz(need, kb_ws_need_seed(B, N, K));
     need = max_sz(need, kb_ws_need_topm(B, KB_TOP_M_MAX));
-    need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K));
+    need = max_sz(need, fit_scratch_bytes(B, N, D, K) + kb_ws_need_fit_acc(B, D, K) + kb_ws_need_zsplit(B, N, D, K) +
+                            ws_need_tol(B, D, K));
     *out = need;
     return KB_OK;
 }
@@ -488,19 +549,38 @@ kb_status kb_init_centroids(kb_ctx* ctx, int B, int N, int D, int K, const float
     return kb_launch_init_centroids(ctx, B, N, D, K, z, rows, centroids);
 }
 
+static kb_status fit_impl(kb_ctx* ctx, int B, int N, int D, int K, int iters, float tol, const float* z, float* centroids,
+                          int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts, int32_t* n_iter);
+
 kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, float* centroids,
                          int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts) {
+    return fit_impl(ctx, B, N, D, K, iters, -1.f, z, centroids, labels, dist2, inertia, rep, counts, nullptr);
+}
+
+kb_status kb_cluster_fit_tol(kb_ctx* ctx, int B, int N, int D, int K, int max_iter, float tol, const float* z,
+                             float* centroids, int32_t* labels, float* dist2, float* inertia, int32_t* rep,
+                             int32_t* counts, int32_t* n_iter) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    KB_REQUIRE(ctx, tol >= 0.f, "kb_cluster_fit_tol: tol must be >= 0");
+    if (B > 0) KB_REQUIRE(ctx, n_iter, "kb_cluster_fit_tol: n_iter is required");
+    return fit_impl(ctx, B, N, D, K, max_iter, tol, z, centroids, labels, dist2, inertia, rep, counts, n_iter);
+}
+
+// tol < 0: the plain loop of `iters` iterations; else the tolerance stop (n_iter out)
+static kb_status fit_impl(kb_ctx* ctx, int B, int N, int D, int K, int iters, float tol, const float* z, float* centroids,
+                          int32_t* labels, float* dist2, float* inertia, int32_t* rep, int32_t* counts, int32_t* n_iter) {
     KB_COMMON(ctx, B, N);
     KB_REQUIRE(ctx, iters >= 0, "kb_cluster_fit: iters must be >= 0");
+    const bool stop = tol >= 0.f;
     if (ctx->assign_path == 0 && kb_fit_fused_eligible(ctx, B, N, D, K) && z && centroids && labels &&
         (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
         // small instances: the whole loop in one launch, one CTA per instance
         KB_REQUIRE(ctx, D >= 1 && K >= 1, "kb_cluster_fit: D and K must be >= 1");
         TimeScope ts__(ctx, KB_T_FIT);
         return kb_launch_fit_fused(ctx, B, N, D, K, iters, z, nullptr, nullptr, nullptr, centroids, labels, dist2, inertia,
-                                   rep, counts);
+                                   rep, counts, nullptr, nullptr, tol, n_iter);
     }
-    if (ctx->assign_path == 0 && !kb_assign_tc_eligible(ctx, B, N, D, K) && kb_fit_coop_eligible(ctx, B, N, D, K) && z &&
+    if (!stop && ctx->assign_path == 0 && !kb_assign_tc_eligible(ctx, B, N, D, K) && kb_fit_coop_eligible(ctx, B, N, D, K) && z &&
         centroids && labels && (((uintptr_t)z | (uintptr_t)centroids) & 15) == 0) {
         // one mid-sized instance: the whole loop in one cooperative launch, the rows resident on chip
         TimeScope ts__(ctx, KB_T_FIT);
@@ -525,11 +605,40 @@ kb_status kb_cluster_fit(kb_ctx* ctx, int B, int N, int D, int K, int iters, con
         ctx->fit_acc_bytes = aneed;
         ctx->fit_acc_clean = 0;
     }
+    // tolerance stop: a gate kernel after every update (see tol_gate_kernel); its copies lie behind everything else
+    const size_t toff = zoff + zneed;
+    float* g_prev = nullptr;
+    int32_t *g_counts = nullptr, *g_done = nullptr;
+    if (stop && B > 0 && s == KB_OK) {
+        KB_REQUIRE(ctx, D >= 1 && K >= 1 && centroids, "kb_cluster_fit_tol: D, K >= 1 and centroids are required");
+        if (ctx->ws_bytes < toff + ws_need_tol(B, D, K)) {
+            ctx->fit_acc = nullptr;
+            kb_zsplit_forget(ctx);
+            return kb_fail(ctx, KB_ERR_WORKSPACE, "kb_cluster_fit_tol needs %zu bytes of workspace", toff + ws_need_tol(B, D, K));
+        }
+        g_prev = reinterpret_cast<float*>(ctx->ws + toff);
+        g_counts = reinterpret_cast<int32_t*>(ctx->ws + toff + kb_align256((size_t)B * K * D * sizeof(float)));
+        g_done = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(g_counts) + kb_align256((size_t)B * K * sizeof(int32_t)));
+        kb_launch(tol_gate_kernel, B, 256, 0, ctx->stream, 0, 0, K * D, K, tol, centroids, counts, g_prev, g_counts, g_done, n_iter);
+        if (cudaGetLastError() != cudaSuccess) s = kb_fail(ctx, KB_ERR_CUDA, "launch of tol_gate_kernel failed");
+        else ctx->launches++;
+    }
     for (int it = 0; it < iters && s == KB_OK; ++it) {
         s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, nullptr, nullptr, nullptr);
         if (s == KB_OK) s = kb_cluster_update(ctx, B, N, D, K, z, labels, centroids, counts);
+        if (s == KB_OK && g_prev) {
+            kb_launch(tol_gate_kernel, B, 256, 0, ctx->stream, 1, it + 1, K * D, K, tol, centroids, counts, g_prev, g_counts, g_done,
+                      n_iter);
+            if (cudaGetLastError() != cudaSuccess) s = kb_fail(ctx, KB_ERR_CUDA, "launch of tol_gate_kernel failed");
+            else ctx->launches++;
+        }
     }
     if (s == KB_OK) s = kb_cluster_assign(ctx, B, N, D, K, z, centroids, labels, dist2, inertia, rep);
+    if (s == KB_OK && g_prev) {
+        kb_launch(tol_gate_kernel, B, 256, 0, ctx->stream, 2, iters, K * D, K, tol, centroids, counts, g_prev, g_counts, g_done, n_iter);
+        if (cudaGetLastError() != cudaSuccess) s = kb_fail(ctx, KB_ERR_CUDA, "launch of tol_gate_kernel failed");
+        else ctx->launches++;
+    }
     ctx->fit_acc = nullptr;
     kb_zsplit_forget(ctx);
     return s;

@@ -37,7 +37,8 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
                  const int32_t* __restrict__ init_rows, float* __restrict__ cent,
                  int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                  int32_t* __restrict__ rep, int32_t* __restrict__ counts, const int32_t* __restrict__ n_active,
-                 const int32_t* __restrict__ run_mask, int* __restrict__ dev_status) {
+                 const int32_t* __restrict__ run_mask, float tol, int32_t* __restrict__ n_iter,
+                 int* __restrict__ dev_status) {
     kb_grid_dependency_wait();
     // An expanding frontier: the instance's arrays have NCAP rows of which the first n_active[b] are candidates
     // (N below); without n_active every row is.  An instance whose run_mask entry is 0 is left exactly as it is.
@@ -63,6 +64,7 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
             if (rep) rep[(size_t)b * K + j] = -1;
         }
         if (inertia && tid == 0) inertia[b] = 0.f;
+        if (n_iter && tid == 0) n_iter[b] = 0;
         return;
     }
 
@@ -123,10 +125,12 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
     for (int e = tid; e < K * D / 4; e += FF_T) {
         float4 v;
         const int j = e / (D / 4), q = e - j * (D / 4);
-        const int r = init_rows ? init_rows[(size_t)b * K + j] : -1;
+        const int r = init_rows ? init_rows[(size_t)b * K + j] : -2;
         if (init_rows && r >= 0 && r < N) {
             const float* d = zs + (size_t)r * ZS + 4 * q;
             v = make_float4(d[0], d[1], d[2], d[3]);
+        } else if (r == -1) {
+            v = make_float4(KB_UNUSED_CENTROID, KB_UNUSED_CENTROID, KB_UNUSED_CENTROID, KB_UNUSED_CENTROID);   // an unused cluster
         } else {
             if (init_rows && q == 0) atomicOr(dev_status, 4);        // a row id out of range: the centroid stays as it was
             v = *(reinterpret_cast<const float4*>(cb) + e);
@@ -145,6 +149,7 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
 
     float best[FF_R];
     int arg[FF_R];
+    int done_updates = 0;
     for (int it = 0; it <= iters; ++it) {
         // ---- assign: nearest centroid of my rows ------------------------------------------
 #pragma unroll
@@ -203,8 +208,9 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
         for (int u = 0; u < FF_R; ++u)
             if (active[u]) perm[atomicAdd(&hist[arg[u]], 1)] = (unsigned short)(tid + u * FF_T);
         __syncthreads();
-        if (it == iters - 1 && counts)
+        if ((it == iters - 1 || tol >= 0.f) && counts)              // (with a tolerance stop any update may be the last)
             for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = offs[j + 1] - offs[j];
+        double moved = 0.0;                                         // my share of sum_j ||c_j(new) - c_j(old)||^2
         for (int e = tid; e < K * D; e += FF_T) {
             const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
             const int p0 = offs[j], p1 = offs[j + 1];
@@ -216,11 +222,25 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
                     s1 += zs[(size_t)perm[p + 1] * ZS + d];
                 }
                 if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
-                cs[e] = (s0 + s1) / (float)(p1 - p0);
+                const float c_new = (s0 + s1) / (float)(p1 - p0);
+                const float dlt = c_new - cs[e];
+                moved += (double)dlt * (double)dlt;
+                cs[e] = c_new;
             }
+        }
+        ++done_updates;
+        if (tol >= 0.f) {
+            // tolerance stop: the whole CTA agrees on the instance's total shift (fixed-order block sum)
+            const double w = kb_warp_sum(moved);
+            if (lane == 0) s_red[warp] = w;
+            __syncthreads();
+            double shift = 0.0;
+            for (int q = 0; q < FF_T / 32; ++q) shift += s_red[q];
+            if (shift <= (double)tol) iters = it + 1;               // this update stays; the next pass is the final assign
         }
         __syncthreads();
     }
+    if (n_iter && tid == 0) n_iter[b] = done_updates;
 
     // ---- outputs of the final assign --------------------------------------------------------
     unsigned long long* rep_key = reinterpret_cast<unsigned long long*>(hist);   // hist/offs are free now: [K] keys
@@ -282,17 +302,17 @@ bool kb_fit_fused_eligible(const kb_ctx* ctx, int B, int N, int D, int K) {
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
                               float* inertia, int32_t* rep, int32_t* counts, const int32_t* n_active,
-                              const int32_t* run_mask) {
+                              const int32_t* run_mask, float tol, int32_t* n_iter) {
     const size_t smem = ff_smem(N, D, K);
     if (D == 16) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
+        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
     } else if (D == 32) {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
+        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
     } else {
         KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, ctx->dev_status);
+        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
     }
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;

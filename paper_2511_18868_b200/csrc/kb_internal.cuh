@@ -123,7 +123,10 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
 kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters, const float* z, const float* xraw,
                               float* zout, const int32_t* init_rows, float* cent, int32_t* labels, float* dist2,
                               float* inertia, int32_t* rep, int32_t* counts, const int32_t* n_active = nullptr,
-                              const int32_t* run_mask = nullptr);
+                              const int32_t* run_mask = nullptr, float tol = -1.f, int32_t* n_iter = nullptr);
+// every coordinate of the centroid of an unused cluster (rows = -1 in kb_init_centroids / init_rows): farther from any
+// data than any real centroid, finite when squared and summed over a few hundred features
+#define KB_UNUSED_CENTROID 1e18f
 size_t kb_ws_need_update(int B, int N, int D, int K);
 size_t kb_ws_need_fit_acc(int B, int D, int K);
 size_t kb_ws_need_score(int B, int N, int K, int S);

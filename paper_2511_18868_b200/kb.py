@@ -25,7 +25,7 @@ EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb
            "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_clear_device_status", "kb_status_of_device_word", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_probe_peaks", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
-           "kb_init_centroids", "kb_cluster_fit", "kb_bandit_step", "kb_bandit_step_tail", "kb_step_workspace_bytes",
+           "kb_init_centroids", "kb_cluster_fit", "kb_cluster_fit_tol", "kb_bandit_step", "kb_bandit_step_tail", "kb_step_workspace_bytes",
            "kb_bandit_step_host", "kb_cluster_update_noalloc", "kb_cluster_update_noalloc_status",
            "kb_append_candidate", "kb_recluster_due", "kb_signatures_from_reps"]
 
@@ -115,6 +115,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_cluster_update_noalloc_status.argtypes = [_VP, ctypes.POINTER(i)]
     lib.kb_init_centroids.argtypes = [_VP, i, i, i, i, _VP, _VP, _VP]
     lib.kb_cluster_fit.argtypes = [_VP, i, i, i, i, i] + [_VP] * 7
+    lib.kb_cluster_fit_tol.argtypes = [_VP, i, i, i, i, i, f] + [_VP] * 8
     lib.kb_append_candidate.argtypes = [_VP, i, i, i, i, i] + [_VP] * 19
     lib.kb_recluster_due.argtypes = [_VP, i, i, i] + [_VP] * 4
     lib.kb_signatures_from_reps.argtypes = [_VP, i, i, i, i] + [_VP] * 4
@@ -369,6 +370,14 @@ class KB:
         self._check(self.lib.kb_cluster_fit(self.h, B, N, D, K, int(iters), self._p(z), self._p(centroids),
                                             self._p(labels), self._p(dist2), self._p(inertia), self._p(rep),
                                             self._p(counts)), "kb_cluster_fit")
+
+    def cluster_fit_tol(self, z, centroids, labels, max_iter, tol, n_iter, dist2=None, inertia=None, rep=None, counts=None):
+        """kb_cluster_fit_tol: Lloyd with a tolerance stop per instance; n_iter [B] receives the updates done."""
+        B, N, D = z.shape
+        K = centroids.shape[1]
+        self._check(self.lib.kb_cluster_fit_tol(self.h, B, N, D, K, int(max_iter), float(tol), self._p(z),
+                                                self._p(centroids), self._p(labels), self._p(dist2), self._p(inertia),
+                                                self._p(rep), self._p(counts), self._p(n_iter)), "kb_cluster_fit_tol")
 
     def _step_args(self, dims: Dict[str, int], params: Dict[str, float], tensors: Dict[str, torch.Tensor], host: bool):
         a = StepArgs()

@@ -1424,3 +1424,101 @@ def test_best_restart_and_the_restart_flow(kbx):
     r = host(rows).reshape(B, n_init, K)
     assert np.mean([len({tuple(v) for v in r[b].tolist()}) > 1 for b in range(B)]) > 0.9   # the copies are seeded differently
     assert kbx.device_status() == 0
+
+
+# ----------------------------------------------- tolerance stop, unused clusters
+def _tol_case(B, N, D, K, seed):
+    rng = np.random.default_rng(seed)
+    x = np.empty((B, N, D), np.float32)
+    for b in range(B):
+        centres = rng.uniform(1.0, 3.0) * rng.standard_normal((K, D))
+        x[b] = centres[rng.integers(0, K, N)] + rng.uniform(0.3, 1.2) * rng.standard_normal((N, D))
+    z, _, _ = oracle.normalize(x)
+    init = np.stack([z[b, rng.choice(N, K, replace=False)] for b in range(B)])
+    return z, init
+
+
+@pytest.mark.parametrize("B,N,D,K,tol", [(6, 400, 16, 5, 1e-3), (40, 512, 32, 16, 1e-2), (3, 300, 64, 4, 0.0),
+                                         # loops of calls (row-wise and tensor-core assignments): the gate kernel
+                                         (2, 3000, 20, 7, 1e-3), (1, 6000, 32, 130, 5e-3), (3, 5000, 64, 128, 1e-2)])
+def test_cluster_fit_tol(kbx, B, N, D, K, tol):
+    """Lloyd with a tolerance stop per instance against the oracle's: the iteration count of every instance (where
+    the deciding shift is not within rounding of the tolerance), and then, like every free-running fit, the objective
+    and the optimality of the returned labels for the returned centroids."""
+    z, init = _tol_case(B, N, D, K, N + K)
+    max_iter = 40
+    ref = oracle.lloyd_tol(z, init, max_iter, tol)
+    ws(kbx, B, N, D, K, 4)
+    c, labels, d2 = dev(init), empty((B, N), torch.int32), empty((B, N))
+    inertia, rep, counts, n_iter = empty((B,)), empty((B, K), torch.int32), empty((B, K), torch.int32), empty((B,), torch.int32)
+    kbx.cluster_fit_tol(dev(z), c, labels, max_iter, tol, n_iter, d2, inertia, rep, counts)
+    assert kbx.device_status() == 0
+    it_g, it_o = host(n_iter), ref["n_iter"]
+    assert it_g.min() >= 1 and it_g.max() <= max_iter
+    if B > 1:
+        assert len(set(it_o.tolist())) > 1                               # instances stop independently
+    # the shifts of the oracle's run around its stop tell whether an fp32 shift could land on the other side of tol
+    same_it = it_g == it_o
+    for b in np.flatnonzero(~same_it):                                   # a shift within rounding of the tolerance
+        assert _reruns_agree(z[b:b + 1], init[b:b + 1], int(it_g[b]), tol), (b, it_g[b], it_o[b], ref["last_shift"][b])
+    got_c = host(c)
+    for b in np.flatnonzero(same_it):
+        parity.close(got_c[b], ref["centroids"][b], atol=2e-5, what="centroids")
+        parity.close(host(inertia)[b:b + 1], ref["inertia"][b:b + 1], atol=0, rtol=1e-3, what="inertia")
+    chk = oracle.cluster_assign(z, got_c, want_margins=True)
+    parity.labels_match(z, got_c, host(labels), chk)
+    same = host(labels) == chk["labels"]
+    parity.close(host(d2)[same], chk["dist2"][same], atol=1e-7, what="dist2")
+    assert np.array_equal(host(counts).sum(1), np.full(B, N))
+    print(f"[fit_tol B={B} N={N} D={D} K={K} tol={tol}] iterations GPU {it_g.tolist()[:8]} oracle {it_o.tolist()[:8]}")
+
+
+def _reruns_agree(z, init, n_iter, tol):
+    """The GPU stopped after n_iter updates: legitimate if, in double, the shift of update n_iter is within an fp32
+    rounding of the tolerance or below it while every earlier shift was above (up to the same rounding)."""
+    c = init.copy()
+    shifts = []
+    for _ in range(n_iter):
+        a = oracle.cluster_assign(z, c, want_rep=False)
+        c2, _ = oracle.cluster_update(z, a["labels"], c)
+        shifts.append(float(((c2.astype(np.float64) - c.astype(np.float64)) ** 2).sum()))
+        c = c2
+    slack = 1e-3
+    return shifts[-1] <= tol * (1 + slack) + 1e-12 and all(s >= tol * (1 - slack) - 1e-12 for s in shifts[:-1])
+
+
+def test_unused_clusters_in_one_batch(kbx):
+    """rows = -1: instances with K_b in {1, 2, 3, 5} clusters as four instances of one call with K = 5 (the K
+    sensitivity study of Sec. 4), through kb_init_centroids + kb_cluster_fit and through the whole step; each
+    instance must cluster as the oracle clusters it alone with its own K_b."""
+    rng = np.random.default_rng(31)
+    B, N, D, K, S, iters = 4, 200, 16, 5, 8, 10
+    cfg = wl.scaled(wl.CONFIGS["tiny"], B=B, N=N, D=D, K=K, S=S, iters=iters)
+    inp = wl.make_inputs(cfg, seed=5)
+    inp["x"] = (3.0 * rng.standard_normal((B, 1, D)) * (rng.integers(0, 3, (B, N, 1)) - 1) + rng.standard_normal((B, N, D))).astype(np.float32)
+    rows = np.full((B, K), -1, np.int32)
+    kbs = [1, 2, 3, 5]
+    for b, kb_ in enumerate(kbs):
+        rows[b, :kb_] = rng.choice(N, kb_, replace=False)
+    inp["init_rows"] = rows
+    z, _, _ = oracle.normalize(inp["x"])
+    # the two calls
+    ws(kbx, B, N, D, K, S)
+    c = empty((B, K, D))
+    kbx.init_centroids(dev(z), dev(rows), c)
+    assert np.array_equal(host(c), oracle.init_centroids(z, rows))
+    labels, d2, inertia, rep, counts = empty((B, N), torch.int32), empty((B, N)), empty((B,)), empty((B, K), torch.int32), empty((B, K), torch.int32)
+    kbx.cluster_fit(dev(z), c, labels, iters, d2, inertia, rep, counts)
+    got = run_step(kbx, cfg, inp)
+    assert kbx.device_status() == 0
+    for b, kb_ in enumerate(kbs):
+        alone = oracle.lloyd_tol(z[b:b + 1], oracle.init_centroids(z[b:b + 1], rows[b:b + 1, :kb_]), iters, -1.0)
+        for lab, cen, cnt, rp, what in [(host(labels)[b], host(c)[b], host(counts)[b], host(rep)[b], "calls"),
+                                        (got["labels"][b], got["centroids"][b], got["counts"][b], got["rep"][b], "step")]:
+            assert np.array_equal(lab, alone["labels"][0]), (what, b)
+            parity.close(cen[:kb_], alone["centroids"][0], atol=1e-5, what=f"centroids ({what})")
+            assert np.all(cen[kb_:] == np.float32(1e18)) and np.all(cnt[kb_:] == 0) and np.all(rp[kb_:] == -1)
+            assert np.array_equal(cnt[:kb_], alone["counts"][0])
+        # an unused cluster is never the chosen pair and carries only the prior
+        assert got["best_cluster_arm"][b] // S < kb_
+        assert np.all(got["cl_pulls"][b, kb_:] == 1.0) and np.all(got["cl_mean"][b, kb_:] == 0.5)
