@@ -1455,7 +1455,7 @@ def test_cluster_fit_tol(kbx, B, N, D, K, tol):
     assert kbx.device_status() == 0
     it_g, it_o = host(n_iter), ref["n_iter"]
     assert it_g.min() >= 1 and it_g.max() <= max_iter
-    if B > 1:
+    if B >= 6:
         assert len(set(it_o.tolist())) > 1                               # instances stop independently
     # the shifts of the oracle's run around its stop tell whether an fp32 shift could land on the other side of tol
     same_it = it_g == it_o
