@@ -320,8 +320,11 @@ kb_status kb_best_restart(kb_ctx* ctx, int G, int n_init, const float* inertia, 
  * kb_score_select's best_arm.  Exact: comparisons only.
  *   arm_index [B][N][S] in, as kb_score_select writes it
  *   top_arm [B][M] out;  top_val [B][M] out, nullable;  0 <= M <= KB_TOP_M_MAX
- * DEVICE memory.  M launches, each one pass over arm_index (meant for small
- * M); needs the workspace of kb_workspace_bytes. */
+ * DEVICE memory.  arm_index is read ONCE, whatever M: every CTA keeps the M
+ * largest keys of its slice (a shared-memory buffer cut back to M by a sort
+ * whenever it fills; after the first cut only about M keys in a few thousand
+ * still pass its threshold), a second launch merges the slices (skipped when
+ * an instance is one slice).  Needs the workspace of kb_workspace_bytes. */
 #define KB_TOP_M_MAX 128
 kb_status kb_select_top_m(kb_ctx* ctx, int B, int N, int S, int M, const float* arm_index, int32_t* top_arm,
                           float* top_val);
