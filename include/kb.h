@@ -110,6 +110,19 @@ const char* kb_last_error(kb_ctx* ctx);
 #define KB_STATUS_TIMEOUT_FIT 0x200
 kb_status kb_get_device_status(kb_ctx* ctx, int* out);
 kb_status kb_clear_device_status(kb_ctx* ctx);
+/* Test hook for the bounded device-side waits (no counterpart in the paper).
+ * Kernels whose roles or CTAs wait on one another -- the tensor-core assign
+ * kernel (mbarrier waits between its roles) and the cooperative fit (its
+ * grid-wide barrier) -- give every wait a limit; when it runs out the CTA
+ * raises its abort flag, every role drains, copies in flight are awaited,
+ * tensor memory is freed, the kernel returns and the status word carries 0x100
+ * or 0x200.  polls != 0 replaces the limit (a wait of a few hundred polls takes
+ * well under a millisecond); leave_one_out != 0 makes one participant stay
+ * away -- the B-operand loader of CTA 0 of the assign kernel, the last CTA of
+ * the cooperative fit -- so that the others' waits do run out.  That is how a
+ * test sees the expiry path run: nothing spins without a limit, nothing
+ * faults.  polls = 0, leave_one_out = 0 restores normal operation. */
+kb_status kb_debug_wait_limit(kb_ctx* ctx, unsigned polls, int leave_one_out);
 /* The mapping itself, as a pure host function (no context, no device): the
  * kb_status that a status word stands for -- KB_ERR_TIMEOUT for a timeout bit;
  * with contract_bits_too != 0 also KB_ERR_INVALID_ARG for 0x001..0x004, which

@@ -279,6 +279,13 @@ kb_status kb_status_of_device_word(int word, int contract_bits_too) {
     return kb_status_from_device_word(nullptr, word, contract_bits_too != 0);
 }
 
+kb_status kb_debug_wait_limit(kb_ctx* ctx, unsigned polls, int leave_one_out) {
+    if (!ctx) return KB_ERR_INVALID_ARG;
+    ctx->dbg_wait_limit = polls;
+    ctx->dbg_skip_arrival = leave_one_out != 0;
+    return KB_OK;
+}
+
 kb_status kb_clear_device_status(kb_ctx* ctx) {
     if (!ctx) return KB_ERR_INVALID_ARG;
     KB_MEMSET(ctx, ctx->dev_status, 0, sizeof(int));

@@ -126,9 +126,11 @@ __device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, 
 }
 // Bounded wait (about a second at most).  Returns false (and raises the CTA's abort flag) when
 // the limit is hit or another role has already aborted.
+// (abort_flag[1] holds the limit in polls: WAIT_LIMIT unless a test shortened it.)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try(bar, parity)) return true;
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_suspend(bar, parity, WAIT_SUSPEND_NS)) return true;
         if ((i & 7u) == 7u && *abort_flag) return false;
     }
@@ -282,6 +284,8 @@ struct TcParams {
     int2* pair_rows;               // (flat row id b * N + k, runner-up centroid)
     int32_t* full_rows;            // flat row ids
     int* dev_status;
+    uint32_t wait_limit;           // polls of a bounded wait (WAIT_LIMIT; a test may shorten it)
+    int absent_b_loader;           // test only: the B loader of CTA 0 never loads, so that CTA's waits run out
 };
 
 // ---- preparation: split centroids into swizzled hi/lo panels, squared norms ----------
@@ -643,7 +647,8 @@ assign_tc_kernel(const TcParams p) {
         for (int k = 0; k < 3; ++k) { mbar_init(BAR(X_FULL + k), APRE ? 1 : 128); mbar_init(BAR(AS_EMPTY + k), 4); }
         // pre-split A: the epilogue hands every row's candidates to the row's thread among warps 0-3
         for (int k = 0; k < 2; ++k) { mbar_init(BAR(MG_FULL + k), 8); mbar_init(BAR(MG_FREE + k), 4); }
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 12) {  // TMEM allocation (whole warp), address lands in shared memory
@@ -1114,7 +1119,7 @@ assign_tc_kernel(const TcParams p) {
         }
     } else if (warp == 13) {
         // ============================ B loader ========================================
-        if (lane == 0) {
+        if (lane == 0 && !(p.absent_b_loader && blockIdx.x == 0)) {
             uint32_t s = 0, ph = 0;
             uint32_t issued = 0;
             for (int tile = first; tile < p.total_tiles && ok; tile += stride) {
@@ -1549,6 +1554,8 @@ kb_status kb_launch_assign_tc(kb_ctx* ctx, char* ws, int B, int N, int D, int K,
     p.ainfo = apre ? ctx->zs_info : nullptr;
     p.z = z; p.bimg = bimg; p.cnorm = cnorm; p.bext = bext; p.inst = inst; p.labels = labels; p.approx = approx;
     p.flag_count = flag_count; p.pair_rows = pair_rows; p.full_rows = full_rows; p.dev_status = ctx->dev_status;
+    p.wait_limit = ctx->dbg_wait_limit ? ctx->dbg_wait_limit : WAIT_LIMIT;
+    p.absent_b_loader = ctx->dbg_skip_arrival;
     const size_t smem = tc_smem_bytes(D, Kpad * B, p.nxb, f16, p.nstage_alloc, apre);
     const int grid = p.total_tiles < ctx->sm_count ? p.total_tiles : ctx->sm_count;
     // with few features per row the epilogue's per-column cost is what limits the kernel:

@@ -53,7 +53,7 @@ struct CoopScratch {               // device scratch, cleared before the launch
 
 // Grid-wide barrier number `epoch` (1, 2, ...) for G CTAs.  Returns false when the wait expired or
 // another CTA gave up.
-__device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, unsigned G) {
+__device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, unsigned G, unsigned spin_limit) {
     __syncthreads();
     __shared__ int s_ok;
     if (threadIdx.x == 0) {
@@ -64,7 +64,7 @@ __device__ __forceinline__ bool grid_barrier(CoopScratch* sc, unsigned epoch, un
             *reinterpret_cast<volatile unsigned*>(&sc->epoch) = epoch;
             ok = 1;
         } else {
-            for (unsigned i = 0; i < CF_SPIN_LIMIT; ++i) {
+            for (unsigned i = 0; i < spin_limit; ++i) {
                 if (*reinterpret_cast<volatile unsigned*>(&sc->epoch) >= epoch) { ok = 1; break; }
                 if ((i & 255u) == 255u && *reinterpret_cast<volatile unsigned*>(&sc->abort)) break;
                 __nanosleep(64);
@@ -88,8 +88,10 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, const floa
                 int32_t* __restrict__ labels, float* __restrict__ dist2, float* __restrict__ inertia,
                 int32_t* __restrict__ rep, int32_t* __restrict__ counts, CoopScratch* __restrict__ sc,
                 float* __restrict__ table /* [3][CF_NC][K*D + K] sums then counts (as int) */,
-                unsigned long long* __restrict__ rep_key /* [K], cleared */, int* __restrict__ dev_status) {
+                unsigned long long* __restrict__ rep_key /* [K], cleared */, int* __restrict__ dev_status,
+                unsigned spin_limit /* polls of a barrier wait */, int absent_cta /* -1; test only: this CTA never arrives */) {
     kb_grid_dependency_wait();
+    if ((int)blockIdx.x == absent_cta) return;                      // (the others give up at their first barrier)
     constexpr int CF_T = cf_threads(D), P = CF_T / SLOTS, CAP = SLOTS * CF_R;
     static_assert(SLOTS % 32 == 0 && P >= 1, "a warp scans one part of the centroids");
     extern __shared__ __align__(16) unsigned char cf_raw[];
@@ -151,7 +153,7 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, const floa
             npart[((size_t)g * D + c) * 2] = s1;
             npart[((size_t)g * D + c) * 2 + 1] = s2;
         }
-        if (!grid_barrier(sc, 1u, (unsigned)G)) {
+        if (!grid_barrier(sc, 1u, (unsigned)G, spin_limit)) {
             if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
             return;
         }
@@ -285,7 +287,7 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, const floa
             }
         }
         // ---- everybody's sums are in the table after the barrier ---------------------------------
-        ok = grid_barrier(sc, epoch0 + (unsigned)(it + 1), (unsigned)G);
+        ok = grid_barrier(sc, epoch0 + (unsigned)(it + 1), (unsigned)G, spin_limit);
         if (!ok) break;
         // written by other CTAs: read through L2; the counts once per cluster (every CTA reads these lines)
         {
@@ -368,7 +370,7 @@ fit_coop_kernel(int N, int K, int iters, const float* __restrict__ z, const floa
     }
     if (inertia || rep) {
         // one more barrier, then CTA 0 publishes what needed every CTA's contribution
-        if (!grid_barrier(sc, epoch0 + (unsigned)(iters + 1), (unsigned)G)) {
+        if (!grid_barrier(sc, epoch0 + (unsigned)(iters + 1), (unsigned)G, spin_limit)) {
             if (tid == 0) atomicOr(dev_status, CF_STATUS_TIMEOUT);
             return;
         }
@@ -458,7 +460,9 @@ kb_status kb_launch_fit_coop(kb_ctx* ctx, int N, int D, int K, int iters, const 
     do {                                                                                                          \
         KB_SMEM_OPTIN(ctx, (fit_coop_kernel<DD, SS>), smem);                                                      \
         e = cudaLaunchKernelEx(&cfg, fit_coop_kernel<DD, SS>, N, K, iters, z, xraw, zout, init_rows, npart, cent, \
-                               labels, dist2, inertia, rep, counts, sc, table, rep_key, ctx->dev_status);        \
+                               labels, dist2, inertia, rep, counts, sc, table, rep_key, ctx->dev_status,         \
+                               ctx->dbg_wait_limit ? ctx->dbg_wait_limit : CF_SPIN_LIMIT,                         \
+                               ctx->dbg_skip_arrival ? G - 1 : -1);                                               \
     } while (0)
 #define KB_CF_LAUNCH_D(DD)                            \
     do {                                              \

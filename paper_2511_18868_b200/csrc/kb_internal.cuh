@@ -41,6 +41,9 @@ struct kb_ctx {
     char* fit_acc;               // null outside such a fit
     size_t fit_acc_bytes;
     int fit_acc_clean;           // 1: cleared since the last update used them
+    // test hooks of the bounded device-side waits (kb_debug_wait_limit): 0 / 0 in normal operation
+    unsigned dbg_wait_limit;     // polls after which a wait gives up (0: the kernels' own limits)
+    int dbg_skip_arrival;        // 1: one participant never arrives, so the others' waits run out
     char err[256];
 };
 #define KB_EV_PAIRS 4096
