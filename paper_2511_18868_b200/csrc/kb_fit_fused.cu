@@ -210,7 +210,7 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
         __syncthreads();
         if ((it == iters - 1 || tol >= 0.f) && counts)              // (with a tolerance stop any update may be the last)
             for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = offs[j + 1] - offs[j];
-        double moved = 0.0;                                         // my share of sum_j ||c_j(new) - c_j(old)||^2
+        float moved = 0.f;                                          // my share of sum_j ||c_j(new) - c_j(old)||^2 (tol >= 0 only)
         for (int e = tid; e < K * D; e += FF_T) {
             const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
             const int p0 = offs[j], p1 = offs[j + 1];
@@ -223,15 +223,14 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
                 }
                 if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
                 const float c_new = (s0 + s1) / (float)(p1 - p0);
-                const float dlt = c_new - cs[e];
-                moved += (double)dlt * (double)dlt;
+                if (tol >= 0.f) { const float dlt = c_new - cs[e]; moved = fmaf(dlt, dlt, moved); }
                 cs[e] = c_new;
             }
         }
         ++done_updates;
         if (tol >= 0.f) {
             // tolerance stop: the whole CTA agrees on the instance's total shift (fixed-order block sum)
-            const double w = kb_warp_sum(moved);
+            const double w = kb_warp_sum((double)moved);
             if (lane == 0) s_red[warp] = w;
             __syncthreads();
             double shift = 0.0;

@@ -58,12 +58,32 @@ constexpr int PM_N = 128;                                   // accumulator tile:
 constexpr uint32_t PM_IDESC_F16 = (1u << 4) | ((uint32_t)(PM_N >> 3) << 17) | (8u << 24);
 constexpr uint32_t PM_IDESC_TF32 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(PM_N >> 3) << 17) | (8u << 24);
 constexpr uint32_t PM_WAIT_LIMIT = 1u << 24;                // polls of the one bounded wait (well under a second)
-constexpr int PM_SMEM = 16 * 1024 + 1024;                   // one B tile (128 rows x 128 bytes) + alignment slack
+constexpr int PM_SMEM = 128 * 1024;                         // one B tile (16 KB) is used; the size keeps one CTA per SM
 
-// tf32 != 0: kind::tf32, else kind::f16.  Two accumulators take turns, 32 products each (the first of a run
-// overwrites), as the assign kernel's tiles do.
-__global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, int* __restrict__ fail,
-                                                           long long* __restrict__ stamps) {
+// One product D[tmem] (+)= A[tmem] * B[smem descriptor]; `acc` == 0 overwrites the accumulator.
+template <bool TF32>
+__device__ __forceinline__ void pr_mma(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t acc) {
+    if (TF32) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a), "l"(bdesc),
+            "r"(PM_IDESC_TF32), "r"(acc)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a), "l"(bdesc),
+            "r"(PM_IDESC_F16), "r"(acc)
+            : "memory");
+    }
+}
+
+// Two accumulators take turns, 16 products each (the first of a run overwrites), as the assign kernel's tiles do.
+// The issuing loop is unrolled by 16 with every operand address a constant offset, so that what is timed is the
+// tensor pipe and not the issuing thread's own address arithmetic (a lone warp runs its dependent integer
+// instructions at a few cycles each: twenty of them per product would cost more than the product).
+template <bool TF32>
+__global__ void __launch_bounds__(128, 1) probe_mma_kernel(int iters, int* __restrict__ fail, long long* __restrict__ stamps) {
     extern __shared__ unsigned char pm_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)pm_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar;
@@ -86,35 +106,22 @@ __global__ void __launch_bounds__(128, 1) probe_mma_kernel(int tf32, int iters, 
     // tensor memory: columns [0, 256) two accumulators, [256, 512) the A operand (its contents are whatever the
     // allocation held: any bit pattern multiplies at the same rate, and the products are never read)
     if (warp == 1) {
-        // one elected lane of a converged warp issues, as in the assign kernel (a lone thread inside a divergent
-        // branch issues measurably slower)
+        // one elected lane of a converged warp issues, as in the assign kernel
         const uint64_t bdesc = pr_desc_sw128(pr_smem_u32(smem));
+        uint32_t elected;
+        asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(elected));
         const long long c0 = clock64();
         unsigned long long n0;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(n0));
-        for (int i = 0; i < iters; ++i) {
-            const uint32_t koff = (uint32_t)(i & 3) * 2u;              // 32-byte k-step inside the swizzled row
-            const uint32_t d = tmem + (uint32_t)((i >> 5) & 1) * 128u;     // 32 products per accumulator, then the other
-            const uint32_t a_t = tmem + 256u + (uint32_t)(i & 15) * 8u;
-            uint32_t elected;
-            asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(elected));
-            if (elected) {
-                if (tf32) {
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a_t),
-                        "l"(bdesc + koff), "r"(PM_IDESC_TF32), "r"(i & 31)
-                        : "memory");
-                } else {
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d), "r"(a_t),
-                        "l"(bdesc + koff), "r"(PM_IDESC_F16), "r"(i & 31)
-                        : "memory");
-                }
+        if (elected) {
+            for (int i = 0; i < iters; i += 16) {
+                const uint32_t d = tmem + (uint32_t)((i >> 4) & 1) * 128u;
+#pragma unroll
+                for (int u = 0; u < 16; ++u)                           // 32-byte k-steps inside the swizzled row
+                    pr_mma<TF32>(d, tmem + 256u + (uint32_t)u * 8u, bdesc + (uint64_t)((u & 3) * 2), u == 0 ? 0u : 1u);
             }
-            __syncwarp();
         }
+        __syncwarp();
         if ((tid & 31) == 0) {
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(pr_smem_u32(&bar))
                          : "memory");
@@ -169,7 +176,8 @@ extern "C" kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out) {
         out->ffma_ms = ms;
         out->ffma_tflops = 2.0 * (double)ff_grid * FF_THREADS * FF_CHAINS * ff_iters / (ms * 1e-3) / 1e12;
         // ---- tensor cores, both kinds
-        if (cudaFuncSetAttribute(probe_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PM_SMEM) != cudaSuccess) {
+        if (cudaFuncSetAttribute(probe_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PM_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(probe_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PM_SMEM) != cudaSuccess) {
             s = KB_ERR_CUDA;
             break;
         }
@@ -177,7 +185,8 @@ extern "C" kb_status kb_probe_peaks(kb_ctx* ctx, kb_peak_probe* out) {
         for (int tf32 = 0; tf32 < 2 && s == KB_OK; ++tf32) {
             for (int rep = 0; rep < 2; ++rep) {
                 cudaEventRecord(e0, st);
-                probe_mma_kernel<<<ctx->sm_count, 128, PM_SMEM, st>>>(tf32, mm_iters, sink + 1, stamps + 2 * tf32);
+                if (tf32) probe_mma_kernel<true><<<ctx->sm_count, 128, PM_SMEM, st>>>(mm_iters, sink + 1, stamps + 2);
+                else probe_mma_kernel<false><<<ctx->sm_count, 128, PM_SMEM, st>>>(mm_iters, sink + 1, stamps);
                 cudaEventRecord(e1, st);
                 if (cudaGetLastError() != cudaSuccess || !elapsed(&ms)) { s = KB_ERR_CUDA; break; }
             }
