@@ -31,7 +31,8 @@ constexpr int FF_MAXROWS = 512;   // rows per instance at most
 // rows per thread (row = tid + u * threads): as many as the register file holds
 __host__ __device__ constexpr int ff_rows(int D) { return D <= 32 ? 4 : 2; }
 
-template <int D>
+// TOL: the tolerance stop is compiled in (its bookkeeping in the update loop costs the plain loop 13 % otherwise)
+template <int D, bool TOL>
 __global__ void __launch_bounds__(FF_MAXROWS / ff_rows(D))
 fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const float* xraw, float* zout,
                  const int32_t* __restrict__ init_rows, float* __restrict__ cent,
@@ -208,9 +209,9 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
         for (int u = 0; u < FF_R; ++u)
             if (active[u]) perm[atomicAdd(&hist[arg[u]], 1)] = (unsigned short)(tid + u * FF_T);
         __syncthreads();
-        if ((it == iters - 1 || tol >= 0.f) && counts)              // (with a tolerance stop any update may be the last)
+        if ((it == iters - 1 || TOL) && counts)                     // (with a tolerance stop any update may be the last)
             for (int j = tid; j < K; j += FF_T) counts[(size_t)b * K + j] = offs[j + 1] - offs[j];
-        float moved = 0.f;                                          // my share of sum_j ||c_j(new) - c_j(old)||^2 (tol >= 0 only)
+        float moved = 0.f;                                          // my share of sum_j ||c_j(new) - c_j(old)||^2 (TOL only)
         for (int e = tid; e < K * D; e += FF_T) {
             const int j = e / D, d = e - j * D;                     // a warp covers consecutive columns of one cluster
             const int p0 = offs[j], p1 = offs[j + 1];
@@ -223,12 +224,12 @@ fit_fused_kernel(int NCAP, int K, int iters, const float* __restrict__ z, const 
                 }
                 if (p < p1) s0 += zs[(size_t)perm[p] * ZS + d];
                 const float c_new = (s0 + s1) / (float)(p1 - p0);
-                if (tol >= 0.f) { const float dlt = c_new - cs[e]; moved = fmaf(dlt, dlt, moved); }
+                if (TOL) { const float dlt = c_new - cs[e]; moved = fmaf(dlt, dlt, moved); }
                 cs[e] = c_new;
             }
         }
         ++done_updates;
-        if (tol >= 0.f) {
+        if (TOL) {
             // tolerance stop: the whole CTA agrees on the instance's total shift (fixed-order block sum)
             const double w = kb_warp_sum((double)moved);
             if (lane == 0) s_red[warp] = w;
@@ -303,16 +304,17 @@ kb_status kb_launch_fit_fused(kb_ctx* ctx, int B, int N, int D, int K, int iters
                               float* inertia, int32_t* rep, int32_t* counts, const int32_t* n_active,
                               const int32_t* run_mask, float tol, int32_t* n_iter) {
     const size_t smem = ff_smem(N, D, K);
-    if (D == 16) {
-        KB_SMEM_OPTIN(ctx, fit_fused_kernel<16>, smem);
-        kb_launch(fit_fused_kernel<16>, B, FF_MAXROWS / ff_rows(16), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
-    } else if (D == 32) {
-        KB_SMEM_OPTIN(ctx, fit_fused_kernel<32>, smem);
-        kb_launch(fit_fused_kernel<32>, B, FF_MAXROWS / ff_rows(32), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
-    } else {
-        KB_SMEM_OPTIN(ctx, fit_fused_kernel<64>, smem);
-        kb_launch(fit_fused_kernel<64>, B, FF_MAXROWS / ff_rows(64), smem, ctx->stream, N, K, iters, z, xraw, zout, init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status);
-    }
+#define KB_FF_LAUNCH(DD, TT)                                                                                             \
+    do {                                                                                                                 \
+        KB_SMEM_OPTIN(ctx, (fit_fused_kernel<DD, TT>), smem);                                                            \
+        kb_launch(fit_fused_kernel<DD, TT>, B, FF_MAXROWS / ff_rows(DD), smem, ctx->stream, N, K, iters, z, xraw, zout,  \
+                  init_rows, cent, labels, dist2, inertia, rep, counts, n_active, run_mask, tol, n_iter, ctx->dev_status); \
+    } while (0)
+    const bool stop = tol >= 0.f;
+    if (D == 16) { if (stop) KB_FF_LAUNCH(16, true); else KB_FF_LAUNCH(16, false); }
+    else if (D == 32) { if (stop) KB_FF_LAUNCH(32, true); else KB_FF_LAUNCH(32, false); }
+    else { if (stop) KB_FF_LAUNCH(64, true); else KB_FF_LAUNCH(64, false); }
+#undef KB_FF_LAUNCH
     KB_LAUNCH_CHECK(ctx, "fit_fused_kernel");
     return KB_OK;
 }
