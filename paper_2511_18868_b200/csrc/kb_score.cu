@@ -20,6 +20,14 @@
 // candidate, read by phases A and C), arm_index written once when requested; fused with the pruning:
 // + 12 bytes per candidate in, the bound (4 bytes per arm) out.
 //
+// Measured and not kept for the statistics pass (same results, no faster): a lane per strategy (every access a
+// contiguous line and the atomics of a row on consecutive words, but four times the load instructions and half
+// the bytes in flight: large 77 against 59 us for the tail, contraction 282 against 189); rows staged through a
+// three-stage shared-memory ring by bulk copies, with and without a dedicated copying warp (200 against 192 us on
+// contraction before the arms kernel below was reshaped): the pass is bound by its shared-memory atomics, not by
+// how its rows arrive -- an fp32 shared-memory atomic add is a compare-and-swap loop (13 cycles per warp
+// instruction on random addresses against 3.7 for an integer add, measured alone).
+//
 // The shared tables are laid out [strategy][label] with an odd row pitch: the lanes of a warp (a few rows x
 // the strategy quads of a row) then fall on different banks unless two rows' labels agree modulo 4, where the
 // [label][strategy] layout put every lane that handled the same strategy offset on the same bank.
@@ -345,8 +353,10 @@ __device__ __forceinline__ void decode_keys(unsigned long long key, unsigned lon
     best_cluster_arm[b] = ckey ? (int32_t)(0xffffffffu - (unsigned)(ckey & 0xffffffffull)) : -1;
 }
 
+constexpr int SA_T = 512;   // threads of the arms kernel
+
 template <int V>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(SA_T)
 score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, const int32_t* __restrict__ labels,
                   const float* __restrict__ dist2, const uint32_t* __restrict__ keep,
                   const float* __restrict__ bound, const float* __restrict__ table, float* __restrict__ arm_index,
@@ -354,10 +364,8 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
                   int32_t* __restrict__ best_arm, float* __restrict__ best_val, int32_t* __restrict__ best_cluster_arm) {
     kb_grid_dependency_wait();
     extern __shared__ __align__(16) float stab[];  // [K][S]
-    __shared__ unsigned long long s_best[8];
+    __shared__ unsigned long long s_best[SA_T / 32];
     const int b = blockIdx.y, tid = threadIdx.x, KS = K * S;
-    for (int e = tid; e < KS; e += blockDim.x) stab[e] = table[(size_t)b * KS + e];
-    __syncthreads();
     const int rows_per = (N + G - 1) / G;
     const int r0 = blockIdx.x * rows_per, r1 = min(N, r0 + rows_per);
     const bool cap = prm.cap_with_bound && bound;
@@ -367,28 +375,37 @@ score_arms_kernel(int N, int K, int S, int G, RowWalk wk, kb_score_params prm, c
     // index among equal values; the 64-bit key is built once per thread
     float bestv = -INFINITY;
     unsigned besti = 0xffffffffu;
-    if (tid < wk.active) {
-        const int q = tid % wk.vps;
-        constexpr int U = 4;                                       // rows in flight per thread
-        for (int rb = r0 + tid / wk.vps; rb < r1; rb += U * wk.rstep) {
-            int lab[U];
-            float d2[U];
-            unsigned bits[U];
-            float4 bv[U];
+    const int q = tid % wk.vps;
+    constexpr int U = 4;                                           // rows in flight per thread
+    int lab[U];
+    float d2[U];
+    unsigned bits[U];
+    float4 bv[U];
+    auto request = [&](int rb) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int r = min(rb + u * wk.rstep, r1 - 1);      // clamped: loads stay in range
-                const size_t row = (size_t)b * N + r;
-                lab[u] = __ldg(labels + row);
-                d2[u] = L != 0.f ? __ldg(dist2 + row) : 0.f;
-                bits[u] = keep ? __ldg(keep + row) : 0xffffffffu;
-                bv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (cap) {
-                    const size_t off = row * S + (size_t)q * V;
-                    if (V == 4) bv[u] = __ldg(reinterpret_cast<const float4*>(bound + off));
-                    else bv[u].x = __ldg(bound + off);
-                }
+        for (int u = 0; u < U; ++u) {
+            const int r = min(rb + u * wk.rstep, r1 - 1);          // clamped: loads stay in range
+            const size_t row = (size_t)b * N + r;
+            lab[u] = __ldg(labels + row);
+            d2[u] = L != 0.f ? __ldg(dist2 + row) : 0.f;
+            bits[u] = keep ? __ldg(keep + row) : 0xffffffffu;
+            bv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (cap) {
+                const size_t off = row * S + (size_t)q * V;
+                if (V == 4) bv[u] = __ldg(reinterpret_cast<const float4*>(bound + off));
+                else bv[u].x = __ldg(bound + off);
             }
+        }
+    };
+    const bool walker = tid < wk.active;
+    const int rb0 = r0 + tid / wk.vps;
+    // the first rows are requested before the table is staged: their latency runs under the staging
+    if (walker && rb0 < r1) request(rb0);
+    for (int e = tid; e < KS; e += SA_T) stab[e] = table[(size_t)b * KS + e];
+    __syncthreads();
+    if (walker) {
+        for (int rb = rb0; rb < r1; rb += U * wk.rstep) {
+            if (rb != rb0) request(rb);
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int r = rb + u * wk.rstep;
@@ -515,19 +532,19 @@ static kb_status launch_score_phases(kb_ctx* ctx, int B, int N, int K, int S, kb
               pr ? kept_count : (uint32_t*)nullptr);
     KB_LAUNCH_CHECK(ctx, "score_table_kernel");
     if (N > 0) {
-        long want = (4L * ctx->sm_count + B - 1) / B;
-        long capg = ((long)N * S + 2047) / 2048;
+        long want = (2L * ctx->sm_count + B - 1) / B;               // two CTAs per SM in all
+        long capg = ((long)N * S + 4095) / 4096;
         int GA = (int)(want < 1 ? 1 : (want > capg ? capg : want));
         if (GA < 1) GA = 1;
-        const RowWalk wa = make_walk(256, S, vec ? 4 : 1);
+        const RowWalk wa = make_walk(SA_T, S, vec ? 4 : 1);
         const uint32_t* keep_c = pr ? pr->keep : keep;
         if (vec) {
             KB_SMEM_OPTIN(ctx, score_arms_kernel<4>, smem_arms);
-            kb_launch(score_arms_kernel<4>, dim3(GA, B), 256, smem_arms, ctx->stream, N, K, S, GA, wa, p, labels, dist2,
+            kb_launch(score_arms_kernel<4>, dim3(GA, B), SA_T, smem_arms, ctx->stream, N, K, S, GA, wa, p, labels, dist2,
                       keep_c, bound, w.table, arm_index, w.key, w.ticket, best_arm, best_val, best_cluster_arm);
         } else {
             KB_SMEM_OPTIN(ctx, score_arms_kernel<1>, smem_arms);
-            kb_launch(score_arms_kernel<1>, dim3(GA, B), 256, smem_arms, ctx->stream, N, K, S, GA, wa, p, labels, dist2,
+            kb_launch(score_arms_kernel<1>, dim3(GA, B), SA_T, smem_arms, ctx->stream, N, K, S, GA, wa, p, labels, dist2,
                       keep_c, bound, w.table, arm_index, w.key, w.ticket, best_arm, best_val, best_cluster_arm);
         }
         KB_LAUNCH_CHECK(ctx, "score_arms_kernel");
