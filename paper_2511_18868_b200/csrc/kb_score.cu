@@ -26,7 +26,10 @@
 // three-stage shared-memory ring by bulk copies, with and without a dedicated copying warp (200 against 192 us on
 // contraction before the arms kernel below was reshaped): the pass is bound by its shared-memory atomics, not by
 // how its rows arrive -- an fp32 shared-memory atomic add is a compare-and-swap loop (13 cycles per warp
-// instruction on random addresses against 3.7 for an integer add, measured alone).
+// instruction on random addresses against 3.7 for an integer add, measured alone). Moving the reward sums out
+// of shared memory, one four-wide fp32 vector reduction per (row, strategy quad) into a global [K][S] table,
+// was slower still (tail 243 against 189 us on contraction, 69 against 59 on large): the table is small, so
+// every SM's reductions meet on the same few hundred L2 lines.
 //
 // The shared tables are laid out [strategy][label] with an odd row pitch: the lanes of a warp (a few rows x
 // the strategy quads of a row) then fall on different banks unless two rows' labels agree modulo 4, where the
