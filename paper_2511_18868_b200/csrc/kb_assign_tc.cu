@@ -109,6 +109,20 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// mbarrier.try_wait may keep the thread suspended for a system-dependent time while the phase is incomplete;
+// where a role only wants to know whether it could go on, and has other work if it cannot, it asks with
+// test_wait, which answers at once.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // The same test, but the hardware may keep the thread suspended for up to `ns` nanoseconds while
 // the phase is incomplete (it resumes at once when the phase completes).  A waiting role then
 // executes one instruction per `ns` instead of spinning, which matters here: the waiting roles
@@ -974,7 +988,7 @@ assign_tc_kernel(const TcParams p) {
                 const bool more = nt + 1 < nt_count || tile + stride < p.total_tiles;
                 if (more) {
                     const uint32_t qn = q + 1u, bufn = qn & 1u;
-                    if (__all_sync(0xffffffffu, mbar_try(BAR(ACC_FULL + bufn), (qn >> 1) & 1u))) {
+                    if (__all_sync(0xffffffffu, mbar_test(BAR(ACC_FULL + bufn), (qn >> 1) & 1u))) {
                         tc_fence_after();
                         TC_LD32(lane_addr + COL_ACC + bufn * BN + half * (BN / 2), r[0]);
                         pref = true;
@@ -1053,14 +1067,26 @@ assign_tc_kernel(const TcParams p) {
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");   // no load may outlive the role (abort path)
     } else if (warp == 12) {
         // ============================ MMA issuer ======================================
-        // One elected lane issues every MMA, so this instruction stream is the critical path of
-        // the whole CTA.  The WHOLE warp runs the loops and the waits, and only the tcgen05
-        // instructions sit under the elected-lane predicate: in warp-uniform control flow the
-        // descriptor arithmetic stays on the uniform datapath (measured: 64 cycles per 128x128x8
-        // MMA, the tensor pipe's own rate, against 83-100 when a single lane runs the loop alone).
+        // One elected lane issues every MMA; the WHOLE warp runs the loop, and only the tcgen05
+        // instructions sit under the elected-lane predicate (in warp-uniform control flow the
+        // descriptor arithmetic stays on the uniform datapath; a loop run by one lane alone issued at
+        // less than half the rate).
+        // The products are queued: the warp issues a tile's 25 in a few hundred cycles, the tensor pipe
+        // needs 1600 for them.  Everything else this warp sends to shared memory (a look at an mbarrier)
+        // is served only after the products queued before it, so a tile has ONE such point, inside the
+        // elected block, in the middle of its last k-block: a non-blocking look (test_wait) at all the
+        // NEXT tile needs.  When it succeeds, the next tile's products follow this tile's last six with
+        // nothing but a vote between them; the blocking wait at the top of a tile runs only when there
+        // really is something to wait for (the first tile of a row tile, whose A panels the producers
+        // can only write once the previous row tile's last products have retired).
+        // What the stream reaches (cycle counters in the issuing warp, this kernel, D = 128, K = 1024):
+        // 64 cycles per product when nothing else runs in the CTA (the pipe's own rate), 80 with every
+        // role present but idle, 67 of those 80 if the waits on the B ring are left out (the ring holds
+        // two accumulator tiles, and a stage comes back one refill later than the stream would like), 83
+        // with the B copies and the row producers working, 96 with the epilogue's loads and ranking.
+        // A second issuing warp taking every other tile, or splitting a tile into more elected blocks,
+        // changed none of these figures; at this rate the B ring already draws 7 TB/s from L2.
         {
-            uint32_t s = 0, ph = 0, q = 0;
-            int it = 0;
             constexpr uint32_t IDESC = F16 ? IDESC_F16 : IDESC_TF32;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
             const uint32_t desc_hi32 = (uint32_t)(desc0 >> 32);
@@ -1069,52 +1095,92 @@ assign_tc_kernel(const TcParams p) {
             // (leading byte offset), 8-row groups 256 bytes apart (stride byte offset)
             const uint32_t ext_lo32 = ((smem_u32(st_base + STAGE) & 0x3FFFFu) >> 4) | ((128u >> 4) << 16);
             const uint32_t ext_hi32 = (256u >> 4) | (1u << 14);
-            const int ring = p.resident ? nt_count * nkb : NSTAGE;
-            for (int tile = first; tile < p.total_tiles && ok; tile += stride, ++it) {
-                const int ab = it % nab, use = it / nab;
-                const uint32_t a_base = tmem + COL_A + ab * AST;
-                for (int nt = 0; nt < nt_count && ok; ++nt, ++q) {
-                    const uint32_t buf = q & 1u;
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(ACC_EMPTY + buf), ((q >> 1) & 1u) ^ 1u, abort_flag));
+            const uint32_t ring = (uint32_t)(p.resident ? nt_count * nkb : NSTAGE);
+            struct AccTile {
+                int tile, nt;               // row tile, accumulator tile inside it
+                uint32_t q;                 // accumulator tiles so far
+                uint32_t s, ph;             // B stage of the tile's first k-block and that stage's phase
+                uint32_t ab, use, first;    // A buffer, how often it was used before, 1 on the CTA's first row tile
+            };
+            auto next_stage = [&](uint32_t& st, uint32_t& phase) { if (++st == ring) { st = 0; phase ^= 1u; } };
+            auto advance = [&](AccTile& x) {
+                for (int kb = 0; kb < nkb; ++kb) next_stage(x.s, x.ph);
+                ++x.q;
+                if (++x.nt == nt_count) {
+                    x.nt = 0; x.tile += stride; x.first = 0u;
+                    if (++x.ab == (uint32_t)nab) { x.ab = 0u; ++x.use; }
+                }
+            };
+            // what a tile needs before its first product: its accumulator buffer handed back, (first tile of a
+            // row tile) the A panels written, its B stages landed
+            auto look = [&](const AccTile& x) -> bool {               // non-blocking, this lane's view
+                bool r = mbar_test(BAR(ACC_EMPTY + (x.q & 1u)), ((x.q >> 1) & 1u) ^ 1u);
+                uint32_t st = x.s, phase = x.ph;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (x.nt == 0) r = mbar_test(BAR(A_FULL + x.ab * 4 + kb), x.use & 1u) & r;
+                    if (!p.resident || x.first) r = mbar_test(BAR(B_FULL + st), phase) & r;
+                    next_stage(st, phase);
+                }
+                return r;
+            };
+            auto await = [&](const AccTile& x) -> bool {              // bounded waits
+                bool r = mbar_wait(BAR(ACC_EMPTY + (x.q & 1u)), ((x.q >> 1) & 1u) ^ 1u, abort_flag);
+                uint32_t st = x.s, phase = x.ph;
+                for (int kb = 0; kb < nkb && r; ++kb) {
+                    if (x.nt == 0) r = mbar_wait(BAR(A_FULL + x.ab * 4 + kb), x.use & 1u, abort_flag);
+                    if (r && (!p.resident || x.first)) r = mbar_wait(BAR(B_FULL + st), phase, abort_flag);
+                    next_stage(st, phase);
+                }
+                return __all_sync(0xffffffffu, r);
+            };
+            AccTile cur = {first, 0, 0u, 0u, 0u, 0u, 0u, 1u};
+            bool ready = false;
+            while (cur.tile < p.total_tiles && ok) {
+                if (!ready) {
+                    ok = await(cur);
                     if (!ok) break;
+                }
+                AccTile nxt = cur;
+                advance(nxt);
+                const bool has_next = nxt.tile < p.total_tiles;
+                const uint32_t a_base = tmem + COL_A + cur.ab * AST;
+                const uint32_t d_tmem = tmem + COL_ACC + (cur.q & 1u) * BN;
+                bool seen = false;                                   // the elected lane's look at the next tile
+                if (elect_one()) {
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem + COL_ACC + buf * BN;
+                    uint32_t st = cur.s, phase = cur.ph;
                     for (int kb = 0; kb < nkb; ++kb) {
-                        if (nt == 0) {
-                            ok = __all_sync(0xffffffffu, mbar_wait(BAR(A_FULL + ab * 4 + kb), (uint32_t)(use & 1), abort_flag));
-                            if (!ok) break;
-                        }
-                        if (!p.resident || it == 0) {              // resident panels are loaded exactly once
-                            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + s), ph, abort_flag));
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
                         const uint32_t a_hi = a_base + kb * 32, a_lo = a_hi + DC;
-                        const uint32_t blo = desc_lo32 + s * (SLOT >> 4);         // this stage's hi panel
-                        if (elect_one()) {
+                        const uint32_t blo = desc_lo32 + st * (SLOT >> 4);            // this stage's hi panel
                         // The very first product of an accumulator tile overwrites it.  fp16 split: that is
                         // the constant-term product (the row's 16 extra features against the centroid
                         // tile's, which sit behind the first k-block's panels without swizzle).
                         if (F16 && kb == 0)
-                            tc_mma_ts<F16>(d_tmem, a_base + 2 * DC, mk_desc(ext_lo32 + s * (SLOT >> 4), ext_hi32), IDESC, 0u);
+                            tc_mma_ts<F16>(d_tmem, a_base + 2 * DC, mk_desc(ext_lo32 + st * (SLOT >> 4), ext_hi32), IDESC, 0u);
                         tc_mma_ts<F16>(d_tmem, a_lo, mk_desc(blo, desc_hi32), IDESC, (F16 || kb != 0) ? 1u : 0u);
                         tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo + (PANEL >> 4), desc_hi32), IDESC);
                         tc_mma_ts_acc<F16>(d_tmem, a_hi, mk_desc(blo, desc_hi32), IDESC);
+                        tc_mma_ts_acc<F16>(d_tmem, a_lo + 8, mk_desc(blo + 2, desc_hi32), IDESC);
+                        tc_mma_ts_acc<F16>(d_tmem, a_hi + 8, mk_desc(blo + (PANEL >> 4) + 2, desc_hi32), IDESC);
+                        tc_mma_ts_acc<F16>(d_tmem, a_hi + 8, mk_desc(blo + 2, desc_hi32), IDESC);
+                        if (kb == nkb - 1 && has_next) {
+                            seen = look(nxt);
+                            tc_fence_after();
+                        }
 #pragma unroll
-                        for (int k8 = 1; k8 < KBF / 8; ++k8) {
+                        for (int k8 = 2; k8 < KBF / 8; ++k8) {
                             tc_mma_ts_acc<F16>(d_tmem, a_lo + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
                             tc_mma_ts_acc<F16>(d_tmem, a_hi + k8 * 8, mk_desc(blo + (PANEL >> 4) + k8 * 2, desc_hi32), IDESC);
                             tc_mma_ts_acc<F16>(d_tmem, a_hi + k8 * 8, mk_desc(blo + k8 * 2, desc_hi32), IDESC);
                         }
-                        if (!p.resident) tc_commit(BAR(B_EMPTY + s));      // stage reusable once these MMAs retire
-                        if (nt == nt_count - 1) tc_commit(BAR(A_EMPTY + ab * 4 + kb));  // A panel reusable
-                        if (kb == nkb - 1) tc_commit(BAR(ACC_FULL + buf));             // accumulator tile complete
-                        }
-                        __syncwarp();
-                        if (++s == (uint32_t)ring) { s = 0; ph ^= 1u; }
+                        if (!p.resident) tc_commit(BAR(B_EMPTY + st));                 // stage reusable once these MMAs retire
+                        if (cur.nt == nt_count - 1) tc_commit(BAR(A_EMPTY + cur.ab * 4 + kb));   // A panel reusable
+                        if (kb == nkb - 1) tc_commit(BAR(ACC_FULL + (cur.q & 1u)));    // accumulator tile complete
+                        next_stage(st, phase);
                     }
-                    if (!ok) break;
                 }
+                ready = __any_sync(0xffffffffu, seen);
+                cur = nxt;
             }
         }
     } else if (warp == 13) {
