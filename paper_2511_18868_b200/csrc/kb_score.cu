@@ -29,7 +29,10 @@
 // instruction on random addresses against 3.7 for an integer add, measured alone). Moving the reward sums out
 // of shared memory, one four-wide fp32 vector reduction per (row, strategy quad) into a global [K][S] table,
 // was slower still (tail 243 against 189 us on contraction, 69 against 59 on large): the table is small, so
-// every SM's reductions meet on the same few hundred L2 lines.
+// every SM's reductions meet on the same few hundred L2 lines.  Taking a CTA's rows in label order (the counting
+// sort of the centroid update, sums of a label's run in registers, the tables touched once per run) lost too:
+// the rows of the history are 32 to 128 bytes, the sort and the second look at the labels cost more than the
+// atomics they replace (tail 312 against 194 us on contraction, 67 against 59 on large, 30 against 22 on medium).
 //
 // The shared tables are laid out [strategy][label] with an odd row pitch: the lanes of a warp (a few rows x
 // the strategy quads of a row) then fall on different banks unless two rows' labels agree modulo 4, where the
