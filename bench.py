@@ -634,11 +634,11 @@ def run_ours(args, cfg):
         tb.record()
         torch.cuda.synchronize()
         top_ms = ta.elapsed_time(tb)
-        top_bytes = top_m * cfg.arms * 4
-        top_line = {"M": top_m, "us": top_ms * 1e3, "us_per_rank": top_ms * 1e3 / top_m, "algorithmic_bytes": top_bytes,
+        top_bytes = cfg.arms * 4
+        top_line = {"M": top_m, "us": top_ms * 1e3, "algorithmic_bytes": top_bytes,
                     "GBps": top_bytes / (top_ms * 1e-3) / 1e9, "hbm_frac": top_bytes / (top_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                    "what": "kb_select_top_m on the step's arm_index: M launches, each one pass (after an L2 flush; the "
-                            "later passes may find the array in L2)"}
+                    "what": "kb_select_top_m on the step's arm_index: one pass over the array (slice kernel + merge "
+                            "kernel), after an L2 flush"}
 
         # ---- one iteration of the online loop between two re-clusterings: select the pair, draw k_t, record the outcome
         # (Algorithm 1 without its LLM call; the outcome is a fixed synthetic runtime per instance).  Queued eagerly and
