@@ -45,8 +45,8 @@ DEFAULT_WORKLOAD = "contraction"      # the largest single-GPU configuration
 TRAFFIC_FROM_CAPTURE = {
     # assign_tc_kernel (pre-split image of Z), one launch: 69.35 MB read + 1.11 MB written
     ("large", "assign"): {"bytes": 70.46e6, "source": "profiles/assign_tc_and_update_kernels.txt"},
-    # assign_tc_kernel at N = 262144: 134.85 + 4.03 MB; traffic grows with N, scaled x16 to N = 4194304
-    ("contraction", "assign"): {"bytes": 16 * 138.88e6,
+    # assign_tc_kernel at N = 262144: 134.83 + 5.09 MB; traffic grows with N, scaled x16 to N = 4194304
+    ("contraction", "assign"): {"bytes": 16 * 139.92e6,
                                 "source": "profiles/assign_tc_and_update_kernels.txt (N = 262144 capture, scaled x16 by rows)"},
 }
 
