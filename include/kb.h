@@ -123,6 +123,12 @@ kb_status kb_clear_device_status(kb_ctx* ctx);
  * test sees the expiry path run: nothing spins without a limit, nothing
  * faults.  polls = 0, leave_one_out = 0 restores normal operation. */
 kb_status kb_debug_wait_limit(kb_ctx* ctx, unsigned polls, int leave_one_out);
+/* Input check for debugging (no counterpart in the paper).  The calls take
+ * finite inputs on trust; this one counts the entries of a device array of n
+ * floats that are NaN or +-inf and hands the count to the host (*out; it
+ * synchronises the stream, so it does not belong on the hot path).  Uses the
+ * spare words behind the status word, no workspace.  n = 0 gives 0. */
+kb_status kb_debug_count_nonfinite(kb_ctx* ctx, const float* x /* device */, size_t n, uint64_t* out /* host */);
 /* The mapping itself, as a pure host function (no context, no device): the
  * kb_status that a status word stands for -- KB_ERR_TIMEOUT for a timeout bit;
  * with contract_bits_too != 0 also KB_ERR_INVALID_ARG for 0x001..0x004, which

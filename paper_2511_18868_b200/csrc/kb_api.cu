@@ -286,6 +286,39 @@ kb_status kb_debug_wait_limit(kb_ctx* ctx, unsigned polls, int leave_one_out) {
     return KB_OK;
 }
 
+namespace {
+__global__ void __launch_bounds__(256) count_nonfinite_kernel(const float* __restrict__ x, size_t n,
+                                                              unsigned long long* __restrict__ out) {
+    unsigned long long c = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const unsigned u = __float_as_uint(__ldg(x + i));
+        c += (u & 0x7f800000u) == 0x7f800000u;               // exponent all ones: NaN or infinity
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(out, c);
+}
+}  // namespace
+
+kb_status kb_debug_count_nonfinite(kb_ctx* ctx, const float* x, size_t n, uint64_t* out) {
+    if (!ctx || !out || (n > 0 && !x)) return KB_ERR_INVALID_ARG;
+    *out = 0;
+    if (n == 0) return KB_OK;
+    // a 64-bit counter in the spare words behind the status word (the context owns 256 bytes there)
+    unsigned long long* cnt = reinterpret_cast<unsigned long long*>(ctx->dev_status + 48);
+    KB_MEMSET(ctx, cnt, 0, sizeof(unsigned long long));
+    size_t blocks = (n + 255) / 256;
+    const size_t cap = (size_t)ctx->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    kb_launch(count_nonfinite_kernel, (unsigned)blocks, 256, 0, ctx->stream, x, n, cnt);
+    KB_LAUNCH_CHECK(ctx, "count_nonfinite_kernel");
+    unsigned long long host = 0;
+    KB_CUDA(ctx, cudaMemcpyAsync(&host, cnt, sizeof(host), cudaMemcpyDeviceToHost, ctx->stream));
+    KB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    *out = host;
+    return KB_OK;
+}
+
 kb_status kb_clear_device_status(kb_ctx* ctx) {
     if (!ctx) return KB_ERR_INVALID_ARG;
     KB_MEMSET(ctx, ctx->dev_status, 0, sizeof(int));

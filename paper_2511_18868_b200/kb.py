@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_UNSUPPORTED", 3:
 
 # every symbol include/kb.h declares
 EXPORTS = ["kb_create", "kb_destroy", "kb_set_stream", "kb_workspace_bytes", "kb_set_workspace",
-           "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_clear_device_status", "kb_debug_wait_limit", "kb_status_of_device_word", "kb_get_launch_count",
+           "kb_status_string", "kb_last_error", "kb_get_device_status", "kb_clear_device_status", "kb_debug_wait_limit", "kb_debug_count_nonfinite", "kb_status_of_device_word", "kb_get_launch_count",
            "kb_timing_enable", "kb_timing_read", "kb_probe_peaks", "kb_set_assign_options", "kb_get_assign_path", "kb_get_assign_presplit", "kb_assign_tc_probe",
            "kb_normalize", "kb_prune", "kb_cluster_assign", "kb_cluster_update", "kb_score_select", "kb_sample_member", "kb_record_outcome", "kb_select_pair", "kb_seed_kmeanspp", "kb_cluster_radius", "kb_select_top_m", "kb_best_restart",
            "kb_init_centroids", "kb_cluster_fit", "kb_cluster_fit_tol", "kb_bandit_step", "kb_bandit_step_tail", "kb_step_workspace_bytes",
@@ -92,6 +92,7 @@ def load_library() -> ctypes.CDLL:
     lib.kb_clear_device_status.argtypes = [_VP]
     lib.kb_status_of_device_word.argtypes = [i, i]
     lib.kb_debug_wait_limit.argtypes = [_VP, ctypes.c_uint, i]
+    lib.kb_debug_count_nonfinite.argtypes = [_VP, _VP, ctypes.c_size_t, ctypes.POINTER(ctypes.c_uint64)]
     lib.kb_get_launch_count.argtypes = [_VP, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
     lib.kb_timing_enable.argtypes = [_VP, i]
     lib.kb_timing_read.argtypes = [_VP, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
@@ -215,6 +216,14 @@ class KB:
     def debug_wait_limit(self, polls: int = 0, leave_one_out: bool = False):
         """kb_debug_wait_limit: shorten the bounded device-side waits / keep one participant away (tests only)."""
         self._check(self.lib.kb_debug_wait_limit(self.h, int(polls), int(bool(leave_one_out))), "kb_debug_wait_limit")
+
+    def count_nonfinite(self, x) -> int:
+        """kb_debug_count_nonfinite: how many entries of a float32 device tensor are NaN or infinite (synchronises)."""
+        out = ctypes.c_uint64()
+        n = int(x.numel())
+        self._check(self.lib.kb_debug_count_nonfinite(self.h, self._p(x) if n else None, n, ctypes.byref(out)),
+                    "kb_debug_count_nonfinite")
+        return int(out.value)
 
     def clear_device_status(self):
         self._check(self.lib.kb_clear_device_status(self.h), "kb_clear_device_status")

@@ -126,3 +126,25 @@ def test_host_step_returns_the_timeout():
         assert ctx.device_status() == 0
     finally:
         ctx.close()
+
+
+def test_nonfinite_count_matches_numpy():
+    """kb_debug_count_nonfinite against its plain definition, on sizes around the grid's stride and with the
+    entries that matter: both infinities, quiet and signalling NaN patterns, the largest finite value, denormals."""
+    from paper_2511_18868_b200 import kb
+    ctx = kb.KB(0)
+    rng = np.random.default_rng(11)
+    for n in (0, 1, 31, 257, 65536 + 3, 3_000_001):
+        x = rng.standard_normal(n).astype(np.float32)
+        if n:
+            bad = rng.choice(n, size=min(n, 1 + n // 7), replace=False)
+            kinds = np.array([np.inf, -np.inf, np.nan], dtype=np.float32)
+            x[bad] = kinds[rng.integers(0, 3, size=bad.size)]
+            x[rng.integers(0, n)] = np.finfo(np.float32).max          # finite: must not count
+            x[rng.integers(0, n)] = np.float32(1e-42)                  # denormal: finite
+        if n > 4:
+            x.view(np.uint32)[3] = 0x7fa00001                          # a signalling NaN pattern
+        want = int((~np.isfinite(x)).sum())
+        got = ctx.count_nonfinite(dev(x) if n else torch.empty(0, device="cuda"))
+        assert got == want, (n, got, want)
+    assert ctx.device_status() == 0
