@@ -711,7 +711,10 @@ def test_argument_errors(kbx):
 
 # ------------------------------------------------- tensor-core assign path
 TC_CASES = [(1, 4096, 32, 128), (1, 5000, 64, 256), (2, 3000, 128, 200), (1, 4097, 96, 1024), (3, 1111, 64, 130),
-            (1, 20000, 128, 1024)]
+            (1, 20000, 128, 1024),
+            # several row tiles per CTA: one accumulator tile per row tile with the B image resident; three per row
+            # tile (their parity alternates from row tile to row tile) through the ring, two and three k-blocks
+            (1, 60000, 64, 128), (1, 50000, 128, 384), (1, 40000, 96, 384)]
 
 
 @pytest.mark.parametrize("path", [2, 3], ids=["f16x3", "tf32x3"])
