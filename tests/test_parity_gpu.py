@@ -650,7 +650,7 @@ def test_cluster_fit_cooperative_ties_and_empty_clusters(kbx, D, K):
 
 
 @pytest.mark.parametrize("B,N,D,K,iters", [(1, 8229, 64, 256, 4), (3, 5000, 32, 128, 3), (1, 20011, 64, 130, 2),
-                                           (1, 6000, 64, 640, 2)])
+                                           (1, 6000, 64, 640, 2), (1, 45000, 64, 384, 2)])
 def test_cluster_fit_presplit(kbx, B, N, D, K, iters):
     """A fit on the tensor path converts Z to its fp16 pieces once and every assignment of the loop multiplies out of
     that image.  Its result must agree with the same loop made of single calls (which split rows on the fly), and
