@@ -1081,11 +1081,11 @@ assign_tc_kernel(const TcParams p) {
         // can only write once the previous row tile's last products have retired).
         // What the stream reaches (cycle counters in the issuing warp, this kernel, D = 128, K = 1024):
         // 64 cycles per product when nothing else runs in the CTA (the pipe's own rate), 80 with every
-        // role present but idle, 67 of those 80 if the waits on the B ring are left out (the ring holds
-        // two accumulator tiles, and a stage comes back one refill later than the stream would like), 83
-        // with the B copies and the row producers working, 96 with the epilogue's loads and ranking.
-        // A second issuing warp taking every other tile, or splitting a tile into more elected blocks,
-        // changed none of these figures; at this rate the B ring already draws 7 TB/s from L2.
+        // role present but idle, 67 of those 80 if the waits on the B ring are left out, 83 with the B
+        // copies and the row producers working, 96 with the epilogue's loads and ranking.  A second
+        // issuing warp taking every other tile, splitting a tile into more elected blocks, or a fifth
+        // ring stage changed none of these figures (three stages cost 17 %); at this rate the B ring
+        // draws 7 TB/s from L2.
         {
             constexpr uint32_t IDESC = F16 ? IDESC_F16 : IDESC_TF32;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(st_base));         // stage 0, hi panel, k-step 0
